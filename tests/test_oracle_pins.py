@@ -1,0 +1,288 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself.
+
+The oracle is the plain definition of decode attention over a head-mixed KV cache
+(Section 3.3 last paragraph; Section 4.3; Appendix B of the paper).  The paper prints
+no numeric attention values, so the pins are: a library routine (all-full == causal
+attention's last row), reductions, brute force with an explicit mask written here in
+numpy, ring-buffer invariants, closed forms, planted needles, and the paper's printed
+"theoretical speedup" column for the retained-token count.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle.rlkv_oracle import Oracle
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def f32(x):
+    """bf16 torch tensor -> float32 numpy."""
+    return x.to(torch.float32).numpy()
+
+
+def rand_bf16(shape, seed):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(shape, generator=g, dtype=torch.float32).to(torch.bfloat16)
+
+
+def fill(oracle, layer, K, V):
+    """K, V: bf16 [n][B][Hkv][D] appended token by token."""
+    for t in range(K.shape[0]):
+        assert oracle.append(layer, K[t], V[t]) == 0
+
+
+def brute_force(q, K, V, keep):
+    """Masked softmax attention written from the definition, float64 numpy.
+
+    q [D], K [n][D], V [n][D] float arrays, keep bool[n]."""
+    q, K, V = q.astype(np.float64), K.astype(np.float64), V.astype(np.float64)
+    s = K @ q / np.sqrt(q.shape[0])
+    s = np.where(keep, s, -np.inf)
+    p = np.exp(s - s[keep].max())
+    p = np.where(keep, p, 0.0)
+    return (p / p.sum()) @ V
+
+
+# ---------------------------------------------------------------------------- I1
+@pytest.mark.parametrize("acc", ["f32", "f64"])
+@pytest.mark.parametrize("Hq,Hkv,D,B,n", [(8, 2, 64, 2, 97), (6, 6, 32, 1, 33), (28, 4, 128, 1, 70)])
+def test_all_full_equals_library_causal_attention(acc, Hq, Hkv, D, B, n):
+    """With every head full the method is ordinary causal attention; the decode step is its
+    last row.  Compared against torch's scaled_dot_product_attention (is_causal=True)."""
+    K = rand_bf16((n, B, Hkv, D), 1)
+    V = rand_bf16((n, B, Hkv, D), 2)
+    Q = rand_bf16((n, B, Hq, D), 3)          # queries for every position; the last one is the decode
+    o = Oracle(1, Hkv, Hq, D, B, n, np.ones(Hkv, np.uint8), 4, 8, acc=acc)
+    fill(o, 0, K, V)
+    out = o.decode(0, Q[-1])
+    G = Hq // Hkv
+    q4 = Q.permute(1, 2, 0, 3).to(torch.float64)                                  # [B][Hq][n][D]
+    k4 = K.permute(1, 2, 0, 3).to(torch.float64).repeat_interleave(G, dim=1)      # head j reads j//G
+    v4 = V.permute(1, 2, 0, 3).to(torch.float64).repeat_interleave(G, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(q4, k4, v4, is_causal=True)[:, :, -1, :]
+    tol = 2e-5 if acc == "f32" else 2e-7      # the output array itself is float32
+    np.testing.assert_allclose(out, ref.numpy(), atol=tol, rtol=0)
+
+
+# ---------------------------------------------------------------------------- I2
+@pytest.mark.parametrize("S,W,n", [(4, 60, 64), (4, 60, 10), (0, 50, 50), (16, 112, 100), (3, 5, 8)])
+def test_compressed_with_budget_at_least_n_equals_full(S, W, n):
+    Hq, Hkv, D, B = 4, 2, 32, 2
+    K, V, q = rand_bf16((n, B, Hkv, D), 4), rand_bf16((n, B, Hkv, D), 5), rand_bf16((B, Hq, D), 6)
+    a = Oracle(1, Hkv, Hq, D, B, n, [1, 1], S, W)
+    b = Oracle(1, Hkv, Hq, D, B, n, [0, 0], S, W)
+    fill(a, 0, K, V)
+    fill(b, 0, K, V)
+    np.testing.assert_array_equal(a.decode(0, q), b.decode(0, q))
+
+
+# ---------------------------------------------------------------------------- I3
+def test_compressed_head_equals_bruteforce_mask_exhaustive():
+    """keep[t] = (t < S) or (t >= n - W), for every small (S, W, n)."""
+    D, Hq, Hkv = 8, 4, 2
+    nmax = 24
+    K, V = rand_bf16((nmax, 1, Hkv, D), 7), rand_bf16((nmax, 1, Hkv, D), 8)
+    checked = 0
+    for S, W in itertools.product([0, 1, 2, 5], [1, 2, 3, 7]):
+        o = Oracle(1, Hkv, Hq, D, 1, nmax, [1, 0], S, W, acc="f64")
+        for n in range(1, nmax + 1):
+            o.append(0, K[n - 1], V[n - 1])
+            q = rand_bf16((1, Hq, D), 100 + n)
+            out = o.decode(0, q)
+            t = np.arange(n)
+            for j in range(Hq):
+                h = j // (Hq // Hkv)
+                keep = np.ones(n, bool) if h == 0 else ((t < S) | (t >= n - W))
+                ref = brute_force(f32(q[0, j]), f32(K[:n, 0, h]), f32(V[:n, 0, h]), keep)
+                np.testing.assert_allclose(out[0, j], ref, atol=1e-6, rtol=0)
+                checked += 1
+    assert checked == 16 * nmax * Hq
+
+
+def test_current_token_is_inside_the_window():
+    """W = 1, S = 0: the head sees only the token appended in this very step."""
+    D = 8
+    K, V = rand_bf16((9, 1, 1, D), 9), rand_bf16((9, 1, 1, D), 10)
+    o = Oracle(1, 1, 1, D, 1, 9, [0], 0, 1)
+    for t in range(9):
+        o.append(0, K[t], V[t])
+        out = o.decode(0, rand_bf16((1, 1, D), t))
+        np.testing.assert_allclose(out[0, 0], f32(V[t, 0, 0]), atol=1e-6)
+
+
+# ---------------------------------------------------------------------------- I4
+@pytest.mark.parametrize("S,W", [(4, 60), (0, 7), (16, 240), (3, 1)])
+def test_ring_holds_sinks_and_last_window_tokens(S, W):
+    D, B, Hkv = 16, 2, 2
+    steps = max(5 * W + S + 3, 40)
+    K, V = rand_bf16((steps, B, Hkv, D), 11), rand_bf16((steps, B, Hkv, D), 12)
+    o = Oracle(1, Hkv, Hkv, D, B, steps, [0, 1], S, W)
+    kb, vb = K.view(torch.int16).numpy().view(np.uint16), V.view(torch.int16).numpy().view(np.uint16)
+    for t in range(steps):
+        assert o.append(0, K[t], V[t]) == 0
+        n = t + 1
+        if n in (1, S, S + 1, S + W, S + W + 1) or n % 17 == 0 or n == steps:
+            for b in range(B):
+                k, v, tok = o.export_head(0, b, 0)
+                want = set(range(min(S, n))) | set(range(max(S, n - W), n))
+                assert set(tok[tok >= 0].tolist()) == want
+                assert len(tok) == S + W
+                for s, tt in enumerate(tok):
+                    if tt >= 0:
+                        assert s == (tt if tt < S else S + (tt - S) % W)
+                        np.testing.assert_array_equal(k[s], kb[tt, b, 0])
+                        np.testing.assert_array_equal(v[s], vb[tt, b, 0])
+                    else:
+                        assert not k[s].any() and not v[s].any()
+                kf, vf, tokf = o.export_head(0, b, 1)
+                np.testing.assert_array_equal(kf[:n], kb[:n, b, 1])
+                np.testing.assert_array_equal(vf[:n], vb[:n, b, 1])
+                assert tokf[:n].tolist() == list(range(n)) and (tokf[n:] == -1).all()
+    assert o.append(0, K[0], V[0]) == -1 and o.length(0) == steps   # full: state unchanged
+
+
+# ---------------------------------------------------------------------------- I5
+@pytest.mark.parametrize("mask", [[1, 1], [0, 0], [1, 0]])
+def test_closed_forms(mask):
+    D, B, Hq, Hkv, n, S, W = 16, 2, 4, 2, 50, 3, 9
+    K, V, q = rand_bf16((n, B, Hkv, D), 13), rand_bf16((n, B, Hkv, D), 14), rand_bf16((B, Hq, D), 15)
+    t = np.arange(n)
+    keep_c = (t < S) | (t >= n - W)
+    # (a) all V rows equal -> out equals that row, whatever the scores
+    vrow = rand_bf16((D,), 16)
+    o = Oracle(1, Hkv, Hq, D, B, n, mask, S, W)
+    fill(o, 0, K, vrow.expand(n, B, Hkv, D).contiguous())
+    np.testing.assert_allclose(o.decode(0, q), np.broadcast_to(f32(vrow), (B, Hq, D)), atol=2e-6)
+    # (b) K = 0 -> arithmetic mean of the retained V rows; (c) q = 0 -> the same mean
+    for kk, qq in ((torch.zeros_like(K), q), (K, torch.zeros_like(q))):
+        o = Oracle(1, Hkv, Hq, D, B, n, mask, S, W)
+        fill(o, 0, kk, V)
+        out = o.decode(0, qq)
+        for j in range(Hq):
+            h = j // 2
+            keep = np.ones(n, bool) if mask[h] else keep_c
+            want = f32(V[:, :, h]).astype(np.float64)[keep].mean(axis=0)          # [B][D]
+            np.testing.assert_allclose(out[:, j], want, atol=2e-6)
+
+
+# ---------------------------------------------------------------------------- I6
+def test_planted_needle_visibility():
+    """A token whose key is strongly aligned with q dominates iff the head retains it."""
+    D, n, S, W = 32, 200, 4, 20
+    base_K, base_V = rand_bf16((n, 1, 2, D), 17), rand_bf16((n, 1, 2, D), 18)
+    q = rand_bf16((1, 2, D), 19)
+    marker = torch.full((D,), 7.0, dtype=torch.bfloat16)
+    for t_star in [0, S - 1, S, n - W - 1, n - W, n - 1, 63, 64, 65, 127, 128]:
+        K, V = base_K.clone(), base_V.clone()
+        for h in range(2):
+            qq = q[0, h].to(torch.float32)
+            K[t_star, 0, h] = (qq / qq.norm() * 60.0).to(torch.bfloat16)   # score ~ 60*|q|/sqrt(D) >> others
+            V[t_star, 0, h] = marker
+        o = Oracle(1, 2, 2, D, 1, n, [1, 0], S, W)
+        fill(o, 0, K, V)
+        out = o.decode(0, q)
+        assert np.abs(out[0, 0] - 7.0).max() < 1e-3                       # full head always sees it
+        visible = t_star < S or t_star >= n - W
+        if visible:
+            assert np.abs(out[0, 1] - 7.0).max() < 1e-3
+        else:
+            assert np.abs(out[0, 1]).max() < 4.0                           # needle evicted: nowhere near 7
+
+
+# ---------------------------------------------------------------------------- I7
+def test_group_and_batch_symmetries():
+    D, B, Hq, Hkv, n = 16, 3, 6, 2, 40
+    K, V = rand_bf16((n, B, Hkv, D), 20), rand_bf16((n, B, Hkv, D), 21)
+    qh = rand_bf16((B, Hkv, 1, D), 22)
+    q = qh.expand(B, Hkv, Hq // Hkv, D).reshape(B, Hq, D).contiguous()     # same q within a group
+    o = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 2, 6)
+    fill(o, 0, K, V)
+    out = o.decode(0, q)
+    for h in range(Hkv):
+        for g in range(1, Hq // Hkv):
+            np.testing.assert_array_equal(out[:, h * 3], out[:, h * 3 + g])
+    # distinct q per head must give distinct outputs (catches a collapsed head index)
+    q2 = rand_bf16((B, Hq, D), 23)
+    out2 = o.decode(0, q2)
+    assert np.abs(out2[:, 0] - out2[:, 1]).max() > 1e-3
+    perm = [2, 0, 1]
+    o2 = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 2, 6)
+    fill(o2, 0, K[:, perm].contiguous(), V[:, perm].contiguous())
+    np.testing.assert_array_equal(o2.decode(0, q2[perm].contiguous()), out2[perm])
+
+
+# ---------------------------------------------------------------------------- I8
+def test_evicted_tokens_do_not_matter():
+    D, n, S, W = 16, 90, 3, 10
+    K, V = rand_bf16((n, 1, 1, D), 24), rand_bf16((n, 1, 1, D), 25)
+    K2, V2 = K.clone(), V.clone()
+    K2[S:n - W] = rand_bf16((n - W - S, 1, 1, D), 26)
+    V2[S:n - W] = rand_bf16((n - W - S, 1, 1, D), 27)
+    q = rand_bf16((1, 1, D), 28)
+    a, b = Oracle(1, 1, 1, D, 1, n, [0], S, W), Oracle(1, 1, 1, D, 1, n, [0], S, W)
+    fill(a, 0, K, V)
+    fill(b, 0, K2, V2)
+    np.testing.assert_array_equal(a.decode(0, q), b.decode(0, q))
+    for x, y in zip(a.export_head(0, 0, 0), b.export_head(0, 0, 0)):
+        np.testing.assert_array_equal(x, y)
+
+
+# ---------------------------------------------------------------------------- cost model
+def test_retained_tokens_reproduce_printed_theoretical_speedups():
+    """Table 3 prints 1/((1-s) + s*W/L); with W = 16 + 64 and L = 3019 (the Math500 mean length
+    the paper quotes) the oracle's retained-token counts reproduce the printed column."""
+    rows = [tuple(map(float, ln.split())) for ln in open(os.path.join(GOLDEN, "table3_theoretical.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 4
+    L, S, W, heads = 3019, 16, 64, 10
+    z = torch.zeros((1, heads, 1), dtype=torch.bfloat16)
+    for s, printed in rows:
+        n_comp = int(round(s * heads))
+        mask = [1] * (heads - n_comp) + [0] * n_comp
+        o = Oracle(1, heads, heads, 1, 1, L, mask, S, W)
+        for _ in range(L):
+            o.append(0, z, z)
+        kept = sum(o.retained(0, h) for h in range(heads))
+        assert o.retained(0, heads - 1) == (S + W if n_comp else L)
+        speedup = heads * L / kept
+        assert abs(round(speedup, 2) - printed) < 1e-9, (s, speedup, printed)
+
+
+# ---------------------------------------------------------------------------- self-check
+def test_f32_build_close_to_f64_build():
+    D, B, Hq, Hkv, n = 128, 1, 8, 2, 3000
+    K, V, q = rand_bf16((n, B, Hkv, D), 29), rand_bf16((n, B, Hkv, D), 30), rand_bf16((B, Hq, D), 31)
+    a = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 16, 112, acc="f32")
+    b = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 16, 112, acc="f64")
+    fill(a, 0, K, V)
+    fill(b, 0, K, V)
+    assert np.abs(a.decode(0, q) - b.decode(0, q)).max() < 2e-6
+
+
+def test_threads_do_not_change_results():
+    D, B, Hq, Hkv, n = 32, 3, 4, 2, 77
+    K, V, q = rand_bf16((n, B, Hkv, D), 32), rand_bf16((n, B, Hkv, D), 33), rand_bf16((B, Hq, D), 34)
+    o = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 4, 9)
+    fill(o, 0, K, V)
+    one = o.decode(0, q)
+    o.set_threads(4)
+    np.testing.assert_array_equal(one, o.decode(0, q))
+
+
+def test_layers_keep_separate_lengths_and_masks():
+    D = 8
+    o = Oracle(2, 2, 2, D, 1, 10, [1, 0, 0, 1], 1, 2)
+    K, V = rand_bf16((6, 1, 2, D), 35), rand_bf16((6, 1, 2, D), 36)
+    for t in range(6):
+        o.append(0, K[t], V[t])
+    for t in range(3):
+        o.append(1, K[t], V[t])
+    assert (o.length(0), o.length(1)) == (6, 3)
+    assert [o.retained(0, 0), o.retained(0, 1), o.retained(1, 0), o.retained(1, 1)] == [6, 3, 3, 3]
+    with pytest.raises(RuntimeError):
+        Oracle(1, 1, 1, D, 1, 4, [1], 0, 1).decode(0, rand_bf16((1, 1, D), 1))   # empty layer
