@@ -1,0 +1,129 @@
+/*
+ * rlkv.h -- C ABI of librlkv: decode attention over a head-mixed KV cache on one B200 (sm_100a).
+ *
+ * The operation (paper: Section 3.3, last paragraph; Section 4.3 "Inference Efficiency";
+ * Appendix B "Local Attention Implementation"):
+ *   every KV head of every layer is either FULL -- it keeps the keys/values of all tokens -- or
+ *   COMPRESSED -- it keeps only the first `sink` tokens and the most recent `window` tokens in a
+ *   constant-size circular buffer.  A decode step appends one token per layer and then runs
+ *   ordinary scaled-dot-product attention, softmax(q.K^T / sqrt(head_dim)).V, of each query head
+ *   over whatever its KV head retains.  Query head j reads KV head j / (q_heads / kv_heads).
+ *
+ * Conventions
+ *   - Every function returns 0 (RLKV_OK) or a negative RLKV_E* code; nothing throws, exits or
+ *     prints.  A call that returns an error leaves the cache state untouched.
+ *   - "device" pointers are CUDA device memory on the GPU that was current at rlkv_cache_create;
+ *     "host" pointers are ordinary host memory.  The caller owns every buffer it passes in.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All GPU work is
+ *     enqueued on it asynchronously; the library never synchronises on the hot path.  Calls on one
+ *     cache must be ordered (one stream, or ordered by events): they share scratch memory.
+ *   - bf16 = IEEE bfloat16 bit patterns, 2 bytes; all tensors are contiguous, row-major, and must
+ *     be 16-byte aligned.
+ *   - Lock-step batch: all `batch` sequences have the same length.  Each layer has its own length
+ *     counter (append then attend, layer by layer).  The token appended in a step is visible to
+ *     that step's attention (it is the newest token of the window).
+ *   - Physical slot of token t in a compressed head: t if t < sink, else
+ *     sink + ((t - sink) mod window).  While length <= sink + window nothing has been evicted.
+ *   - Limits: head_dim in {64, 128}; 1 <= q_heads / kv_heads <= 8; sink >= 0; window >= 1.
+ */
+#ifndef RLKV_H
+#define RLKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rlkv_cache rlkv_cache; /* opaque, library-owned host object */
+
+enum {
+    RLKV_OK = 0,
+    RLKV_EINVAL = -1, /* null/misaligned pointer, index out of range, unsupported shape */
+    RLKV_EFULL = -2,  /* append/prefill would exceed max_len (any layer, uniform rule) */
+    RLKV_EEMPTY = -3, /* decode on a layer that holds no token */
+    RLKV_ENOMEM = -4, /* host or device allocation failed, or device_buf too small */
+    RLKV_ECUDA = -5,  /* a CUDA call failed; rlkv_strerror(RLKV_ECUDA) carries the CUDA text */
+    RLKV_EKERNEL = -6 /* a kernel gave up on a bounded wait (see rlkv_kernel_status) */
+};
+
+/* Bytes of device memory a cache of this shape needs (pools, index tables, split scratch and the
+ * staging area of rlkv_step_host).  head_is_full: host, [layers*kv_heads], 1 = full, 0 =
+ * compressed.  A compressed head costs (sink+window) rows (rounded up to the 64-row tile) however
+ * long the sequence grows -- the constant-size pool of Section 4.3. */
+int rlkv_cache_size(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                    const uint8_t* head_is_full, int sink, int window, size_t* bytes_out);
+
+/* Two-class cache layout (Section 4.3: "dual KV pool").  device_buf == NULL: the library
+ * cudaMallocs the memory and frees it in rlkv_cache_destroy.  Otherwise the caller provides
+ * device_buf (1024-byte aligned, >= rlkv_cache_size bytes) and keeps it alive until destroy.
+ * The pools are zero-filled, head_is_full is copied, all lengths start at 0.  Synchronous. */
+int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, int head_dim,
+                      int batch, int max_len, const uint8_t* head_is_full, int sink, int window,
+                      void* device_buf, size_t device_buf_bytes);
+int rlkv_cache_destroy(rlkv_cache* cache);
+
+/* All lengths back to 0 and the pools re-zeroed (asynchronous on `stream`). */
+int rlkv_cache_reset(rlkv_cache* cache, void* stream);
+
+/* Fused append (Section 4.3 circular buffer; Appendix B "first ... sink tokens and the recent ...
+ * local tokens").  k, v: device bf16 [batch][kv_heads][head_dim] -- all KV heads; the caller does
+ * not need to know their classes.  Token t = length(layer) goes to row t of a full head and to
+ * slot(t) of a compressed head; then length(layer) = t + 1.  Copies are bit-exact.
+ * RLKV_EFULL if length(layer) == max_len. */
+int rlkv_append(rlkv_cache* cache, int layer, const void* k, const void* v, void* stream);
+
+/* Bulk append of n_tokens >= 1 tokens, defined as exactly n_tokens successive rlkv_append calls
+ * (the resulting cache bytes are identical).  k, v: device bf16 [n_tokens][batch][kv_heads][head_dim].
+ * RLKV_EFULL if length(layer) + n_tokens > max_len. */
+int rlkv_prefill(rlkv_cache* cache, int layer, const void* k, const void* v, int n_tokens,
+                 void* stream);
+
+/* Split-KV decode attention over the heterogeneous heads of one layer, one launch for both head
+ * classes (Section 3.3: compressed heads "still use full attention but with compressed KV cache";
+ * Section 4.3 asks for exactly this fused heterogeneous-head kernel).
+ * q: device bf16 [batch][q_heads][head_dim]; out: device fp32 [batch][q_heads][head_dim].
+ * Scores, softmax and accumulation are fp32.  RLKV_EEMPTY if length(layer) == 0. */
+int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out, void* stream);
+
+/* One whole decode step: for every layer, append then attend.  Device buffers:
+ * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];
+ * out fp32 [layers][batch][q_heads][head_dim].  Equivalent to the per-layer calls in order.
+ * RLKV_EFULL (nothing done) if any layer is at max_len. */
+int rlkv_step(rlkv_cache* cache, const void* k, const void* v, const void* q, void* out,
+              void* stream);
+
+/* The same step with HOST buffers of the same shapes: inputs are copied host->device and the
+ * result device->host on `stream` inside the call (pinned host memory makes the copies
+ * asynchronous).  The call returns once the work is enqueued; synchronise `stream` before reading
+ * out_host. */
+int rlkv_step_host(rlkv_cache* cache, const void* k_host, const void* v_host, const void* q_host,
+                   void* out_host, void* stream);
+
+/* ---- introspection (host-side bookkeeping; no GPU work unless stated) ---- */
+int rlkv_length(const rlkv_cache* cache, int layer, int* len_out);
+/* Bytes of K and V rows the next rlkv_decode_attention on `layer` must read:
+ * batch * sum over KV heads of min(length, rows the head retains) * 2 * head_dim * 2
+ * (the cost model of Section 4.3: (1-s) + s*W/L of the full-cache bytes). */
+int rlkv_step_bytes(const rlkv_cache* cache, int layer, uint64_t* kv_bytes_out);
+/* Copies one head's physical rows to the host (synchronises the device).  k_host, v_host: bf16
+ * [rows][head_dim] where rows = max_len for a full head, sink+window for a compressed head;
+ * token_of_slot_host: int32[rows], the token held by each row or -1 if the row is empty. */
+int rlkv_debug_export_head(rlkv_cache* cache, int layer, int batch_row, int kv_head, void* k_host,
+                           void* v_host, int* rows_out, int32_t* token_of_slot_host);
+/* Synchronises the device and reads the kernels' status word: 0 = no kernel ever gave up on a
+ * bounded wait; otherwise a code identifying the wait that ran out (results are then invalid). */
+int rlkv_kernel_status(rlkv_cache* cache, int* status_out);
+/* Number of kernels this cache has launched so far. */
+int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
+/* Tuning knob for the decode kernel's grid: CTAs per SM (1 or 2) and pipeline stages (2..8);
+ * 0 keeps the current value. */
+int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages);
+
+const char* rlkv_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RLKV_H */

@@ -1,0 +1,192 @@
+"""Thin ctypes binding of librlkv: argument marshalling only, one Python function per C entry point.
+
+Every function takes the same arguments as its C counterpart in ``include/rlkv.h`` (torch tensors
+or raw integer addresses for pointers, a torch stream or ``None`` for the stream) and raises
+``RlkvError`` on a negative return code.  Nothing here computes anything: all arithmetic runs in the
+CUDA kernels of the library.  Importing this module fails loudly if the library cannot be loaded;
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librlkv.so")
+
+RLKV_OK, RLKV_EINVAL, RLKV_EFULL, RLKV_EEMPTY, RLKV_ENOMEM, RLKV_ECUDA, RLKV_EKERNEL = 0, -1, -2, -3, -4, -5, -6
+
+# name -> (restype, argtypes); one entry per symbol declared in include/rlkv.h
+_vp, _ci, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+SIGNATURES = {
+    "rlkv_cache_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
+    "rlkv_cache_create": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _sz]),
+    "rlkv_cache_destroy": (_ci, [_vp]),
+    "rlkv_cache_reset": (_ci, [_vp, _vp]),
+    "rlkv_append": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_prefill": (_ci, [_vp, _ci, _vp, _vp, _ci, _vp]),
+    "rlkv_decode_attention": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_step": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "rlkv_step_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "rlkv_length": (_ci, [_vp, _ci, ctypes.POINTER(_ci)]),
+    "rlkv_step_bytes": (_ci, [_vp, _ci, ctypes.POINTER(ctypes.c_uint64)]),
+    "rlkv_debug_export_head": (_ci, [_vp, _ci, _ci, _ci, _vp, _vp, ctypes.POINTER(_ci), _vp]),
+    "rlkv_kernel_status": (_ci, [_vp, ctypes.POINTER(_ci)]),
+    "rlkv_launch_count": (_ci, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
+    "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci]),
+    "rlkv_strerror": (ctypes.c_char_p, [_ci]),
+}
+
+
+class RlkvError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"librlkv error {code}: {text}")
+        self.code = code
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2510_08525_b200.build` "
+            "(nvcc, sm_100a).  There is no fallback implementation.")
+    lib = ctypes.CDLL(LIB_PATH)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)  # AttributeError if the library does not export a declared symbol
+        fn.restype, fn.argtypes = res, args
+    return lib
+
+
+lib = _load()
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise RlkvError(rc, lib.rlkv_strerror(rc).decode())
+
+
+def _ptr(x) -> int:
+    """Address of a torch tensor / numpy array, or the integer itself."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    if isinstance(x, np.ndarray):
+        if not x.flags["C_CONTIGUOUS"]:
+            raise ValueError("array must be contiguous")
+        return x.ctypes.data
+    if not x.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return x.data_ptr()
+
+
+def _stream(s) -> int:
+    if s is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _mask(head_is_full) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(head_is_full, dtype=np.uint8).reshape(-1))
+
+
+def rlkv_cache_size(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window) -> int:
+    m = _mask(head_is_full)
+    if m.size != layers * kv_heads:
+        raise ValueError("head_is_full must have layers*kv_heads entries")
+    out = _sz(0)
+    _check(lib.rlkv_cache_size(layers, kv_heads, q_heads, head_dim, batch, max_len, m.ctypes.data, sink, window,
+                               ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_cache_create(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window,
+                      device_buf=None, device_buf_bytes=0) -> int:
+    """Returns the opaque cache handle (an integer address)."""
+    m = _mask(head_is_full)
+    if m.size != layers * kv_heads:
+        raise ValueError("head_is_full must have layers*kv_heads entries")
+    handle = _vp(0)
+    _check(lib.rlkv_cache_create(ctypes.byref(handle), layers, kv_heads, q_heads, head_dim, batch, max_len,
+                                 m.ctypes.data, sink, window, _ptr(device_buf), device_buf_bytes))
+    return int(handle.value)
+
+
+def rlkv_cache_destroy(cache) -> None:
+    _check(lib.rlkv_cache_destroy(cache))
+
+
+def rlkv_cache_reset(cache, stream=None) -> None:
+    _check(lib.rlkv_cache_reset(cache, _stream(stream)))
+
+
+def rlkv_append(cache, layer, k, v, stream=None) -> None:
+    _check(lib.rlkv_append(cache, layer, _ptr(k), _ptr(v), _stream(stream)))
+
+
+def rlkv_prefill(cache, layer, k, v, n_tokens, stream=None) -> None:
+    _check(lib.rlkv_prefill(cache, layer, _ptr(k), _ptr(v), n_tokens, _stream(stream)))
+
+
+def rlkv_decode_attention(cache, layer, q, out, stream=None) -> None:
+    _check(lib.rlkv_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_step(cache, k, v, q, out, stream=None) -> None:
+    _check(lib.rlkv_step(cache, _ptr(k), _ptr(v), _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_step_host(cache, k_host, v_host, q_host, out_host, stream=None) -> None:
+    _check(lib.rlkv_step_host(cache, _ptr(k_host), _ptr(v_host), _ptr(q_host), _ptr(out_host), _stream(stream)))
+
+
+def rlkv_length(cache, layer) -> int:
+    out = _ci(0)
+    _check(lib.rlkv_length(cache, layer, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_step_bytes(cache, layer) -> int:
+    out = ctypes.c_uint64(0)
+    _check(lib.rlkv_step_bytes(cache, layer, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_debug_export_head(cache, layer, batch_row, kv_head, rows, head_dim):
+    """rows = max_len for a full head, sink+window for a compressed head.
+    Returns (k uint16[rows][D], v uint16[rows][D], token_of_slot int32[rows])."""
+    k = np.empty((rows, head_dim), dtype=np.uint16)
+    v = np.empty((rows, head_dim), dtype=np.uint16)
+    tok = np.empty(rows, dtype=np.int32)
+    got = _ci(0)
+    _check(lib.rlkv_debug_export_head(cache, layer, batch_row, kv_head, k.ctypes.data, v.ctypes.data,
+                                      ctypes.byref(got), tok.ctypes.data))
+    if got.value != rows:
+        raise ValueError(f"head has {got.value} rows, caller expected {rows}")
+    return k, v, tok
+
+
+def rlkv_kernel_status(cache) -> int:
+    out = _ci(0)
+    rc = lib.rlkv_kernel_status(cache, ctypes.byref(out))
+    if rc not in (RLKV_OK, RLKV_EKERNEL):
+        _check(rc)
+    return int(out.value)
+
+
+def rlkv_launch_count(cache) -> int:
+    out = ctypes.c_uint64(0)
+    _check(lib.rlkv_launch_count(cache, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0) -> None:
+    _check(lib.rlkv_set_decode_config(cache, ctas_per_sm, stages))
+
+
+def rlkv_strerror(code: int) -> str:
+    return lib.rlkv_strerror(code).decode()

@@ -1,0 +1,61 @@
+// Fused append / bulk append: writes the new K and V rows of every (batch row, KV head) of one
+// layer into the pool of the head's class and wraps the ring of compressed heads.
+//
+// Compressed-head slot rule: token t lives in row t if t < sink, else in row
+// sink + ((t - sink) mod window) -- a constant-size circular buffer of sink + window rows holding
+// the first `sink` tokens and the most recent `window` tokens (paper, Section 4.3 and Appendix B).
+// In a bulk append only the tokens that survive the whole batch of appends are written, so no two
+// threads ever target the same row and the result equals n successive single appends bit for bit.
+#include "rlkv_internal.cuh"
+
+namespace rlkv {
+namespace {
+
+__global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
+{
+    const int chunks = a.head_dim / 8;  // 16-byte pieces per row
+    const long long per_token = (long long)a.batch * a.kv_heads * chunks;
+    const long long total = per_token * a.n_tokens * 2;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long r = i;
+        const int c = (int)(r % chunks);
+        r /= chunks;
+        const int h = (int)(r % a.kv_heads);
+        r /= a.kv_heads;
+        const int b = (int)(r % a.batch);
+        r /= a.batch;
+        const int tok = (int)(r % a.n_tokens);
+        const int kv = (int)(r / a.n_tokens);  // 0 = K, 1 = V
+
+        const int t = a.t0 + tok;
+        const int slot = a.slot_of_head[h];
+        long long row;
+        if (slot >= 0) {
+            row = a.full_row0 + ((long long)(b * a.n_full + slot) * 2 + kv) * a.rows_full + t;
+        } else {
+            const int n_final = a.t0 + a.n_tokens;
+            if (!(t < a.sink || t >= n_final - a.window)) continue;  // evicted before the batch ends
+            const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
+            row = a.comp_row0 + ((long long)(b * a.n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
+        }
+        const __nv_bfloat16* src = (kv ? a.v : a.k) +
+                                   (((long long)tok * a.batch + b) * a.kv_heads + h) * a.head_dim;
+        const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
+        reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream)
+{
+    const long long total = (long long)a.batch * a.kv_heads * (a.head_dim / 8) * a.n_tokens * 2;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace rlkv

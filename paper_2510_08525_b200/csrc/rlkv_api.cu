@@ -1,0 +1,546 @@
+// Host side of librlkv: argument checks, the two-class cache layout, launches.
+//
+// Device buffer layout (all sections 1024-byte aligned):
+//   pool      rows of head_dim bf16.  Per layer: the full-head region
+//             [batch][n_full(layer)][K|V][rows_full][D], then the compressed-head region
+//             [batch][n_comp(layer)][K|V][rows_comp][D].  rows_full = max_len and
+//             rows_comp = sink+window, each rounded up to the 64-row tile, so a tile never reaches
+//             into a neighbouring head and a compressed head owns a constant number of rows
+//             (the constant-size pool of Section 4.3 of the paper).
+//   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
+//   tickets   int32 [layers][batch*kv_heads]   (split bookkeeping, zero between launches)
+//   status    int32 kernel status word
+//   partials  float [max_grid][2][partial_floats]  (split-KV scratch)
+//   staging   k, v, q, out of one whole step, for rlkv_step_host
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/rlkv.h"
+#include "rlkv_internal.cuh"
+
+namespace rlkv {
+cudaError_t prepare_decode_kernels(int head_dim, int stages);
+}
+
+using namespace rlkv;
+
+namespace {
+
+thread_local char g_cuda_text[256] = "";
+
+int cuda_fail(cudaError_t e, const char* what)
+{
+    snprintf(g_cuda_text, sizeof g_cuda_text, "CUDA error in %s: %s", what, cudaGetErrorString(e));
+    return RLKV_ECUDA;
+}
+#define RLKV_CUDA(call)                                  \
+    do {                                                 \
+        cudaError_t e_ = (call);                         \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Layout {
+    int rows_full = 0, rows_comp = 0;
+    std::vector<int> n_full, n_comp;
+    std::vector<long long> full_row0, comp_row0;  // per layer, in pool rows
+    long long pool_rows = 0;
+    size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
+    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, total = 0;
+    int max_grid = 0;
+};
+
+constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
+
+int check_shape(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                const uint8_t* mask, int sink, int window)
+{
+    if (!mask || layers < 1 || kv_heads < 1 || q_heads < 1 || batch < 1 || max_len < 1) return RLKV_EINVAL;
+    if (q_heads % kv_heads != 0 || q_heads / kv_heads > kMaxGroup) return RLKV_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return RLKV_EINVAL;
+    if (sink < 0 || window < 1) return RLKV_EINVAL;
+    if ((long long)sink + window > (1 << 24) || max_len > (1 << 28)) return RLKV_EINVAL;
+    return RLKV_OK;
+}
+
+int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                const uint8_t* mask, int sink, int window)
+{
+    L.rows_full = (int)align_up((size_t)max_len, kTile);
+    L.rows_comp = (int)align_up((size_t)sink + window, kTile);
+    L.n_full.assign(layers, 0);
+    L.n_comp.assign(layers, 0);
+    L.full_row0.assign(layers, 0);
+    L.comp_row0.assign(layers, 0);
+    long long row = 0;
+    for (int l = 0; l < layers; ++l) {
+        for (int h = 0; h < kv_heads; ++h) (mask[l * kv_heads + h] ? L.n_full[l] : L.n_comp[l])++;
+        L.full_row0[l] = row;
+        row += (long long)batch * L.n_full[l] * 2 * L.rows_full;
+        L.comp_row0[l] = row;
+        row += (long long)batch * L.n_comp[l] * 2 * L.rows_comp;
+    }
+    L.pool_rows = row;
+    if (row >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
+    L.max_grid = 2 * kMaxGridSms;
+    size_t off = 0;
+    L.off_pool = off;
+    off = align_up(off + (size_t)row * head_dim * 2, 1024);
+    L.off_tables = off;
+    off = align_up(off + (size_t)2 * layers * kv_heads * sizeof(int), 1024);
+    L.off_tickets = off;
+    off = align_up(off + (size_t)layers * batch * kv_heads * sizeof(int), 1024);
+    L.off_status = off;
+    off = align_up(off + 64, 1024);
+    L.off_partials = off;
+    off = align_up(off + (size_t)L.max_grid * 2 * partial_floats(head_dim) * sizeof(float), 1024);
+    const size_t kv_step = (size_t)layers * batch * kv_heads * head_dim * 2;
+    const size_t q_step = (size_t)layers * batch * q_heads * head_dim * 2;
+    L.off_k = off;
+    off = align_up(off + kv_step, 1024);
+    L.off_v = off;
+    off = align_up(off + kv_step, 1024);
+    L.off_q = off;
+    off = align_up(off + q_step, 1024);
+    L.off_out = off;
+    off = align_up(off + q_step * 2, 1024);
+    L.total = off;
+    return RLKV_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        if (prev == dev) prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+struct rlkv_cache {
+    int layers, kv_heads, q_heads, head_dim, batch, max_len, sink, window;
+    int device, sm_count;
+    int ctas_per_sm, stages;
+    bool plain;  // debugging cross-check kernel instead of the pipelined one
+    Layout lay;
+    std::vector<uint8_t> is_full;
+    std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
+    std::vector<int> len;                         // [layers]
+    uint8_t* dev_base;
+    bool owns_buffer;
+    CUtensorMap tmap;
+    uint64_t launches;
+};
+
+namespace {
+
+template <typename T>
+T* dev_at(const rlkv_cache* c, size_t off) { return reinterpret_cast<T*>(c->dev_base + off); }
+
+int zero_state(rlkv_cache* c, cudaStream_t s)
+{
+    // pools, tickets and status; tables and the rest need no clearing
+    RLKV_CUDA(cudaMemsetAsync(c->dev_base + c->lay.off_pool, 0, (size_t)c->lay.pool_rows * c->head_dim * 2, s));
+    RLKV_CUDA(cudaMemsetAsync(c->dev_base + c->lay.off_tickets, 0,
+                              c->lay.off_partials - c->lay.off_tickets, s));
+    return RLKV_OK;
+}
+
+int make_tensor_map(rlkv_cache* c)
+{
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    RLKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
+    const cuuint64_t dims[2] = {(cuuint64_t)c->head_dim, (cuuint64_t)c->lay.pool_rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)c->head_dim * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+        &c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->dev_base + c->lay.off_pool, dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_text, sizeof g_cuda_text, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return RLKV_ECUDA;
+    }
+    return RLKV_OK;
+}
+
+bool valid_layer(const rlkv_cache* c, int layer) { return c && layer >= 0 && layer < c->layers; }
+
+int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s)
+{
+    AppendArgs a;
+    a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+    a.full_row0 = c->lay.full_row0[layer];
+    a.comp_row0 = c->lay.comp_row0[layer];
+    a.slot_of_head = dev_at<int>(c, c->lay.off_tables) + (size_t)layer * c->kv_heads;
+    a.k = static_cast<const __nv_bfloat16*>(k);
+    a.v = static_cast<const __nv_bfloat16*>(v);
+    a.n_full = c->lay.n_full[layer];
+    a.n_comp = c->lay.n_comp[layer];
+    a.rows_full = c->lay.rows_full;
+    a.rows_comp = c->lay.rows_comp;
+    a.batch = c->batch;
+    a.kv_heads = c->kv_heads;
+    a.head_dim = c->head_dim;
+    a.t0 = c->len[layer];
+    a.n_tokens = n_tokens;
+    a.sink = c->sink;
+    a.window = c->window;
+    RLKV_CUDA(launch_append(a, s));
+    c->launches++;
+    c->len[layer] += n_tokens;
+    return RLKV_OK;
+}
+
+int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
+{
+    const int n = c->len[layer];
+    const int cap = c->sink + c->window;
+    DecodeArgs a;
+    a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+    a.full_row0 = c->lay.full_row0[layer];
+    a.comp_row0 = c->lay.comp_row0[layer];
+    a.head_of_slot = dev_at<int>(c, c->lay.off_tables) + (size_t)(c->layers + layer) * c->kv_heads;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.out = static_cast<float*>(out);
+    a.partials = dev_at<float>(c, c->lay.off_partials);
+    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
+    a.status = dev_at<int>(c, c->lay.off_status);
+    a.n_full = c->lay.n_full[layer];
+    a.n_comp = c->lay.n_comp[layer];
+    a.rows_full = c->lay.rows_full;
+    a.rows_comp = c->lay.rows_comp;
+    a.len_full = n;
+    a.len_comp = n < cap ? n : cap;
+    a.batch = c->batch;
+    a.group = c->q_heads / c->kv_heads;
+    a.q_heads = c->q_heads;
+    a.tiles_full = (a.len_full + kTile - 1) / kTile;
+    a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
+    const long long total =
+        (long long)c->batch * ((long long)a.n_full * a.tiles_full + (long long)a.n_comp * a.tiles_comp);
+    if (total >= (1ll << 31)) return RLKV_EINVAL;
+    a.total_tiles = (int)total;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
+    // every CTA must own at least one tile (the split bookkeeping assumes no empty ranges)
+    int grid = c->sm_count * (c->plain ? 2 : c->ctas_per_sm);
+    if (grid > c->lay.max_grid) grid = c->lay.max_grid;
+    if (grid > a.total_tiles) grid = a.total_tiles;
+    RLKV_CUDA(launch_decode(a, c->plain ? nullptr : &c->tmap, c->head_dim, grid, c->stages, s));
+    c->launches++;
+    return RLKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rlkv_strerror(int code)
+{
+    switch (code) {
+        case RLKV_OK: return "ok";
+        case RLKV_EINVAL: return "invalid argument";
+        case RLKV_EFULL: return "cache is at max_len";
+        case RLKV_EEMPTY: return "layer holds no token";
+        case RLKV_ENOMEM: return "out of memory or buffer too small";
+        case RLKV_ECUDA: return g_cuda_text[0] ? g_cuda_text : "CUDA error";
+        case RLKV_EKERNEL: return "a kernel gave up on a bounded wait";
+        default: return "unknown error";
+    }
+}
+
+int rlkv_cache_size(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                    const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+{
+    if (!bytes_out) return RLKV_EINVAL;
+    int rc = check_shape(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    Layout L;
+    rc = make_layout(L, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    *bytes_out = L.total;
+    return RLKV_OK;
+}
+
+int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, int head_dim, int batch,
+                      int max_len, const uint8_t* head_is_full, int sink, int window, void* device_buf,
+                      size_t device_buf_bytes)
+{
+    if (!out) return RLKV_EINVAL;
+    *out = nullptr;
+    int rc = check_shape(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    rlkv_cache* c = new (std::nothrow) rlkv_cache();
+    if (!c) return RLKV_ENOMEM;
+    c->layers = layers; c->kv_heads = kv_heads; c->q_heads = q_heads; c->head_dim = head_dim;
+    c->batch = batch; c->max_len = max_len; c->sink = sink; c->window = window;
+    c->dev_base = nullptr; c->owns_buffer = false; c->launches = 0;
+    c->ctas_per_sm = 1;
+    c->stages = head_dim == 128 ? 6 : 8;
+    const char* plain = getenv("RLKV_DECODE_PLAIN");
+    c->plain = plain && plain[0] == '1';
+    rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) { delete c; return rc; }
+    c->is_full.assign(head_is_full, head_is_full + (size_t)layers * kv_heads);
+    c->len.assign(layers, 0);
+    c->slot_of_head.assign((size_t)layers * kv_heads, 0);
+    c->head_of_slot.assign((size_t)layers * kv_heads, 0);
+    for (int l = 0; l < layers; ++l) {
+        int nf = 0, nc = 0;
+        for (int h = 0; h < kv_heads; ++h) {
+            if (c->is_full[l * kv_heads + h]) {
+                c->slot_of_head[l * kv_heads + h] = nf;
+                c->head_of_slot[l * kv_heads + nf] = h;
+                ++nf;
+            } else {
+                c->slot_of_head[l * kv_heads + h] = -(nc + 1);
+                ++nc;
+            }
+        }
+        nc = 0;
+        for (int h = 0; h < kv_heads; ++h)
+            if (!c->is_full[l * kv_heads + h]) c->head_of_slot[l * kv_heads + nf + nc++] = h;
+    }
+    auto fail = [&](int code) {
+        if (c->owns_buffer && c->dev_base) cudaFree(c->dev_base);
+        delete c;
+        return code;
+    };
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
+    e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceGetAttribute"));
+    if (c->sm_count > kMaxGridSms) c->sm_count = kMaxGridSms;
+    if (device_buf) {
+        if ((reinterpret_cast<uintptr_t>(device_buf) & 1023u) != 0) return fail(RLKV_EINVAL);
+        if (device_buf_bytes < c->lay.total) return fail(RLKV_ENOMEM);
+        c->dev_base = static_cast<uint8_t*>(device_buf);
+    } else {
+        void* p = nullptr;
+        e = cudaMalloc(&p, c->lay.total);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(RLKV_ENOMEM);
+        }
+        c->dev_base = static_cast<uint8_t*>(p);
+        c->owns_buffer = true;
+    }
+    rc = zero_state(c, nullptr);
+    if (rc) return fail(rc);
+    const size_t tbytes = (size_t)layers * kv_heads * sizeof(int);
+    e = cudaMemcpy(c->dev_base + c->lay.off_tables, c->slot_of_head.data(), tbytes, cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(c->dev_base + c->lay.off_tables + tbytes, c->head_of_slot.data(), tbytes,
+                       cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaMemcpy(tables)"));
+    rc = make_tensor_map(c);
+    if (rc) return fail(rc);
+    e = prepare_decode_kernels(head_dim, c->stages);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaFuncSetAttribute"));
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceSynchronize"));
+    *out = c;
+    return RLKV_OK;
+}
+
+int rlkv_cache_destroy(rlkv_cache* c)
+{
+    if (!c) return RLKV_EINVAL;
+    int rc = RLKV_OK;
+    if (c->owns_buffer && c->dev_base) {
+        DeviceGuard g(c->device);
+        cudaError_t e = cudaFree(c->dev_base);
+        if (e != cudaSuccess) rc = cuda_fail(e, "cudaFree");
+    }
+    delete c;
+    return rc;
+}
+
+int rlkv_cache_reset(rlkv_cache* c, void* stream)
+{
+    if (!c) return RLKV_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    int rc = zero_state(c, static_cast<cudaStream_t>(stream));
+    if (rc) return rc;
+    std::fill(c->len.begin(), c->len.end(), 0);
+    return RLKV_OK;
+}
+
+int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages)
+{
+    if (!c || ctas_per_sm < 0 || ctas_per_sm > 2 || stages < 0 || stages == 1 || stages > 8) return RLKV_EINVAL;
+    const int cps = ctas_per_sm ? ctas_per_sm : c->ctas_per_sm;
+    const int st = stages ? stages : c->stages;
+    if (decode_smem_bytes(c->head_dim, st) * cps > 227u * 1024u) return RLKV_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    RLKV_CUDA(prepare_decode_kernels(c->head_dim, st));
+    c->ctas_per_sm = cps;
+    c->stages = st;
+    return RLKV_OK;
+}
+
+int rlkv_append(rlkv_cache* c, int layer, const void* k, const void* v, void* stream)
+{
+    return rlkv_prefill(c, layer, k, v, 1, stream);
+}
+
+int rlkv_prefill(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, void* stream)
+{
+    if (!valid_layer(c, layer) || !k || !v || !aligned16(k) || !aligned16(v) || n_tokens < 1) return RLKV_EINVAL;
+    if ((long long)c->len[layer] + n_tokens > c->max_len) return RLKV_EFULL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_append(c, layer, k, v, n_tokens, static_cast<cudaStream_t>(stream));
+}
+
+int rlkv_decode_attention(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (c->len[layer] < 1) return RLKV_EEMPTY;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream));
+}
+
+int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* out, void* stream)
+{
+    if (!c || !k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out))
+        return RLKV_EINVAL;
+    for (int l = 0; l < c->layers; ++l)
+        if (c->len[l] >= c->max_len) return RLKV_EFULL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
+    const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
+    for (int l = 0; l < c->layers; ++l) {
+        int rc = do_append(c, l, static_cast<const __nv_bfloat16*>(k) + l * kv_layer,
+                           static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s);
+        if (rc) return rc;
+        rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
+                       static_cast<float*>(out) + l * q_layer, s);
+        if (rc) return rc;
+    }
+    return RLKV_OK;
+}
+
+int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const void* q_host, void* out_host,
+                   void* stream)
+{
+    if (!c || !k_host || !v_host || !q_host || !out_host) return RLKV_EINVAL;
+    for (int l = 0; l < c->layers; ++l)
+        if (c->len[l] >= c->max_len) return RLKV_EFULL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t kv_bytes = (size_t)c->layers * c->batch * c->kv_heads * c->head_dim * 2;
+    const size_t q_bytes = (size_t)c->layers * c->batch * c->q_heads * c->head_dim * 2;
+    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_k, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_v, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_q, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+    int rc = rlkv_step(c, c->dev_base + c->lay.off_k, c->dev_base + c->lay.off_v, c->dev_base + c->lay.off_q,
+                       c->dev_base + c->lay.off_out, stream);
+    if (rc) return rc;
+    RLKV_CUDA(cudaMemcpyAsync(out_host, c->dev_base + c->lay.off_out, q_bytes * 2, cudaMemcpyDeviceToHost, s));
+    return RLKV_OK;
+}
+
+int rlkv_length(const rlkv_cache* c, int layer, int* len_out)
+{
+    if (!valid_layer(c, layer) || !len_out) return RLKV_EINVAL;
+    *len_out = c->len[layer];
+    return RLKV_OK;
+}
+
+int rlkv_step_bytes(const rlkv_cache* c, int layer, uint64_t* kv_bytes_out)
+{
+    if (!valid_layer(c, layer) || !kv_bytes_out) return RLKV_EINVAL;
+    const uint64_t n = (uint64_t)c->len[layer], cap = (uint64_t)c->sink + c->window;
+    const uint64_t row_pair = (uint64_t)c->head_dim * 2 * 2;  // one K row + one V row
+    const uint64_t rows = (uint64_t)c->lay.n_full[layer] * n + (uint64_t)c->lay.n_comp[layer] * (n < cap ? n : cap);
+    *kv_bytes_out = (uint64_t)c->batch * rows * row_pair;
+    return RLKV_OK;
+}
+
+int rlkv_debug_export_head(rlkv_cache* c, int layer, int b, int h, void* k_host, void* v_host, int* rows_out,
+                           int32_t* token_of_slot)
+{
+    if (!valid_layer(c, layer) || b < 0 || b >= c->batch || h < 0 || h >= c->kv_heads || !k_host || !v_host ||
+        !rows_out || !token_of_slot)
+        return RLKV_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    RLKV_CUDA(cudaDeviceSynchronize());
+    const int slot = c->slot_of_head[layer * c->kv_heads + h];
+    const int n = c->len[layer];
+    long long krow;
+    int rows, stride;
+    if (slot >= 0) {
+        rows = c->max_len;
+        stride = c->lay.rows_full;
+        krow = c->lay.full_row0[layer] + (long long)(b * c->lay.n_full[layer] + slot) * 2 * stride;
+        for (int s = 0; s < rows; ++s) token_of_slot[s] = s < n ? s : -1;
+    } else {
+        rows = c->sink + c->window;
+        stride = c->lay.rows_comp;
+        krow = c->lay.comp_row0[layer] + (long long)(b * c->lay.n_comp[layer] + (-slot - 1)) * 2 * stride;
+        for (int s = 0; s < rows; ++s) {
+            int tok = -1;
+            if (s < c->sink) {
+                if (s < n) tok = s;
+            } else if (n > c->sink) {
+                // newest token t < n with sink + (t - sink) % window == s
+                const int newest = n - 1, r = s - c->sink;
+                const int back = (((newest - c->sink) % c->window) - r + c->window) % c->window;
+                if (newest - back >= c->sink) tok = newest - back;
+            }
+            token_of_slot[s] = tok;
+        }
+    }
+    const size_t bytes = (size_t)rows * c->head_dim * 2;
+    const uint8_t* pool = c->dev_base + c->lay.off_pool;
+    RLKV_CUDA(cudaMemcpy(k_host, pool + (size_t)krow * c->head_dim * 2, bytes, cudaMemcpyDeviceToHost));
+    RLKV_CUDA(cudaMemcpy(v_host, pool + (size_t)(krow + stride) * c->head_dim * 2, bytes, cudaMemcpyDeviceToHost));
+    *rows_out = rows;
+    return RLKV_OK;
+}
+
+int rlkv_kernel_status(rlkv_cache* c, int* status_out)
+{
+    if (!c || !status_out) return RLKV_EINVAL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    RLKV_CUDA(cudaDeviceSynchronize());
+    RLKV_CUDA(cudaMemcpy(status_out, c->dev_base + c->lay.off_status, sizeof(int), cudaMemcpyDeviceToHost));
+    return *status_out == 0 ? RLKV_OK : RLKV_EKERNEL;
+}
+
+int rlkv_launch_count(const rlkv_cache* c, uint64_t* launches_out)
+{
+    if (!c || !launches_out) return RLKV_EINVAL;
+    *launches_out = c->launches;
+    return RLKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+"""Helpers shared by the benchmark and the GPU tests: a small owner object for a cache handle and
+the seeded fill of a cache.  No attention or cache arithmetic happens here -- the fill only moves
+generator output into the library through ``rlkv_prefill``.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import synth
+
+from . import binding as rl
+
+
+class Cache:
+    """Owns one rlkv_cache handle; methods forward to the C entry points of the same name."""
+
+    def __init__(self, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window,
+                 device="cuda:0", device_buf=None):
+        self.layers, self.kv_heads, self.q_heads, self.head_dim = layers, kv_heads, q_heads, head_dim
+        self.batch, self.max_len, self.sink, self.window = batch, max_len, sink, window
+        self.head_is_full = np.asarray(head_is_full, dtype=np.uint8).reshape(-1).copy()
+        self.device = torch.device(device)
+        self._buf = device_buf
+        with torch.cuda.device(self.device):
+            self.handle = rl.rlkv_cache_create(
+                layers, kv_heads, q_heads, head_dim, batch, max_len, self.head_is_full, sink, window,
+                device_buf, 0 if device_buf is None else device_buf.numel() * device_buf.element_size())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            rl.rlkv_cache_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    def is_full(self, layer, head) -> bool:
+        return bool(self.head_is_full[layer * self.kv_heads + head])
+
+    def append(self, layer, k, v):
+        rl.rlkv_append(self.handle, layer, k, v)
+
+    def prefill(self, layer, k, v):
+        rl.rlkv_prefill(self.handle, layer, k, v, k.shape[0])
+
+    def decode(self, layer, q, out=None):
+        if out is None:
+            out = torch.empty((self.batch, self.q_heads, self.head_dim), dtype=torch.float32, device=self.device)
+        rl.rlkv_decode_attention(self.handle, layer, q, out)
+        return out
+
+    def length(self, layer) -> int:
+        return rl.rlkv_length(self.handle, layer)
+
+    def step_bytes(self, layer) -> int:
+        return rl.rlkv_step_bytes(self.handle, layer)
+
+    def export_head(self, layer, b, head):
+        rows = self.max_len if self.is_full(layer, head) else self.sink + self.window
+        return rl.rlkv_debug_export_head(self.handle, layer, b, head, rows, self.head_dim)
+
+    def status(self) -> int:
+        return rl.rlkv_kernel_status(self.handle)
+
+
+def workload_mask(w: synth.Workload) -> np.ndarray:
+    if w.name == "tiny":
+        return np.array([1, 0], dtype=np.uint8)     # KV head 0 full, KV head 1 compressed
+    return synth.head_mask(w.seed, w.layers, w.kv_heads, w.frac_compressed)
+
+
+def make_cache(w: synth.Workload, extra_tokens: int = 64, device="cuda:0") -> Cache:
+    return Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, w.context + extra_tokens,
+                 workload_mask(w), w.sink, w.window, device=device)
+
+
+def fill_cache(cache: Cache, w: synth.Workload, n_tokens: int, chunk_elems: int = 1 << 24) -> None:
+    """Prefill tokens length(layer) .. n_tokens-1 of every layer from the seeded generator."""
+    per_token = w.batch * w.kv_heads * w.head_dim
+    chunk = max(1, chunk_elems // per_token)
+    for layer in range(w.layers):
+        t = cache.length(layer)
+        while t < n_tokens:
+            t1 = min(n_tokens, t + chunk)
+            k = synth.rows(w.seed, synth.STREAM_K, layer, t, t1, w.batch, w.kv_heads, w.head_dim, cache.device)
+            v = synth.rows(w.seed, synth.STREAM_V, layer, t, t1, w.batch, w.kv_heads, w.head_dim, cache.device)
+            cache.prefill(layer, k, v)
+            t = t1
+    torch.cuda.synchronize(cache.device)
+
+
+def step_inputs(w: synth.Workload, t: int, device):
+    """k, v [layers][B][Hkv][D] and q [layers][B][Hq][D] (bf16) for the decode step that appends token t."""
+    k = torch.stack([synth.rows(w.seed, synth.STREAM_K, l, t, t + 1, w.batch, w.kv_heads, w.head_dim, device)[0]
+                     for l in range(w.layers)])
+    v = torch.stack([synth.rows(w.seed, synth.STREAM_V, l, t, t + 1, w.batch, w.kv_heads, w.head_dim, device)[0]
+                     for l in range(w.layers)])
+    q = torch.stack([synth.rows(w.seed, synth.STREAM_Q, l, t, t + 1, w.batch, w.q_heads, w.head_dim, device)[0]
+                     for l in range(w.layers)])
+    return k.contiguous(), v.contiguous(), q.contiguous()

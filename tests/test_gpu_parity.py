@@ -1,0 +1,333 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Cache state is compared bit for bit; attention outputs within the stated bounds
+(max abs error <= 1e-2, mean abs error <= 1e-3, plus max abs error <= 2e-2 * rms(out) per query
+head so the check keeps its teeth at long contexts where |out| ~ 0.02).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle.rlkv_oracle import Oracle
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS, REL_RMS = 1e-2, 1e-3, 2e-2
+
+
+@pytest.fixture(scope="module")
+def rl(cuda_device):
+    import paper_2510_08525_b200.binding as binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def hz(cuda_device):
+    import paper_2510_08525_b200.harness as harness
+    return harness
+
+
+def rand_bf16(shape, seed, device="cpu"):
+    g = torch.Generator().manual_seed(seed)
+    return torch.randn(shape, generator=g, dtype=torch.float32).to(torch.bfloat16).to(device)
+
+
+def check_out(got, want):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    assert np.isfinite(got).all()
+    err = np.abs(got - want)
+    assert err.max() <= MAX_ABS, err.max()
+    assert err.mean() <= MEAN_ABS, err.mean()
+    rms = np.sqrt((want ** 2).mean(axis=-1, keepdims=True))
+    assert (err <= REL_RMS * rms + 1e-6).all(), float((err / (rms + 1e-30)).max())
+
+
+def check_state(cache, oracle, layers=None, rows=None):
+    for l in (range(cache.layers) if layers is None else layers):
+        assert cache.length(l) == oracle.length(l)
+        for b in range(cache.batch):
+            for h in range(cache.kv_heads):
+                gk, gv, gt = cache.export_head(l, b, h)
+                ok, ov, ot = oracle.export_head(l, b, h)
+                np.testing.assert_array_equal(gt, ot)
+                np.testing.assert_array_equal(gk, ok)
+                np.testing.assert_array_equal(gv, ov)
+
+
+def build_pair(hz, layers, Hkv, Hq, D, B, max_len, mask, S, W, dev):
+    cache = hz.Cache(layers, Hkv, Hq, D, B, max_len, mask, S, W, device=dev)
+    oracle = Oracle(layers, Hkv, Hq, D, B, max_len, mask, S, W, threads=8)
+    return cache, oracle
+
+
+def feed(cache, oracle, layer, K, V, bulk):
+    """K, V: bf16 [n][B][Hkv][D] on the CPU."""
+    dev = cache.device
+    if bulk:
+        cache.prefill(layer, K.to(dev), V.to(dev))
+    else:
+        for t in range(K.shape[0]):
+            cache.append(layer, K[t].to(dev), V[t].to(dev))
+    for t in range(K.shape[0]):
+        assert oracle.append(layer, K[t], V[t]) == 0
+
+
+# ------------------------------------------------------------------------------------------ tiny
+@pytest.mark.parametrize("bulk", [False, True])
+def test_tiny_config(rl, hz, cuda_device, bulk):
+    """1 layer, batch 1, 8/2 heads, D 64, KV head 0 full, head 1 compressed 4+60; 512 cached tokens,
+    one append, one decode (n = 513); also checked at n = 512."""
+    w = synth.WORKLOADS["tiny"]
+    mask = hz.workload_mask(w)
+    cache, oracle = build_pair(hz, 1, w.kv_heads, w.q_heads, w.head_dim, 1, 520, mask, w.sink, w.window, cuda_device)
+    K = synth.rows(w.seed, synth.STREAM_K, 0, 0, 513, 1, w.kv_heads, w.head_dim)
+    V = synth.rows(w.seed, synth.STREAM_V, 0, 0, 513, 1, w.kv_heads, w.head_dim)
+    feed(cache, oracle, 0, K[:512], V[:512], bulk)
+    q512 = synth.rows(w.seed, synth.STREAM_Q, 0, 511, 512, 1, w.q_heads, w.head_dim)[0]
+    check_out(cache.decode(0, q512.to(cuda_device)).cpu().numpy(), oracle.decode(0, q512))
+    feed(cache, oracle, 0, K[512:], V[512:], False)
+    q = synth.rows(w.seed, synth.STREAM_Q, 0, 512, 513, 1, w.q_heads, w.head_dim)[0]
+    out = cache.decode(0, q.to(cuda_device))
+    check_out(out.cpu().numpy(), oracle.decode(0, q))
+    check_state(cache, oracle)
+    assert cache.step_bytes(0) == (513 + 64) * 2 * 64 * 2
+    assert cache.status() == 0
+    # determinism: the same call again gives the same bits
+    out2 = cache.decode(0, q.to(cuda_device))
+    assert torch.equal(out, out2)
+
+
+# ------------------------------------------------------------------------------------------ shapes
+SHAPES = [
+    # layers, Hkv, Hq, D, B, S, W, n, mask pattern
+    (1, 2, 8, 64, 1, 4, 60, 1, "10"),
+    (1, 2, 8, 64, 2, 4, 60, 63, "10"),
+    (1, 2, 8, 64, 2, 4, 60, 64, "01"),
+    (1, 2, 8, 64, 2, 4, 60, 65, "10"),
+    (2, 4, 28, 128, 3, 16, 112, 300, "1001" "0110"),
+    (2, 4, 28, 128, 2, 16, 112, 129, "0000" "1111"),
+    (1, 8, 32, 128, 2, 16, 112, 1000, "11011011"),
+    (1, 1, 8, 128, 1, 0, 5, 777, "0"),
+    (1, 1, 1, 64, 5, 3, 200, 450, "1"),
+    (1, 3, 15, 128, 2, 1, 1, 200, "010"),
+    (1, 2, 6, 64, 1, 7, 57, 2000, "10"),
+    (1, 2, 8, 128, 1, 16, 240, 5000, "11"),       # long single rows: every CTA writes partials
+    (3, 2, 4, 128, 4, 130, 62, 193, "100111"),    # sink larger than the window; n == sink + window + 1
+]
+
+
+@pytest.mark.parametrize("bulk", [True, False])
+@pytest.mark.parametrize("shape", SHAPES, ids=[f"s{i}" for i in range(len(SHAPES))])
+def test_shapes_against_oracle(rl, hz, cuda_device, shape, bulk):
+    layers, Hkv, Hq, D, B, S, W, n, pattern = shape
+    if not bulk and n > 1000:
+        pytest.skip("single appends covered at smaller n")
+    mask = [int(c) for c in pattern]
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, n + 3, mask, S, W, cuda_device)
+    for l in range(layers):
+        K, V = rand_bf16((n, B, Hkv, D), 100 + l), rand_bf16((n, B, Hkv, D), 200 + l)
+        feed(cache, oracle, l, K, V, bulk)
+    for l in range(layers):
+        q = rand_bf16((B, Hq, D), 300 + l)
+        out = cache.decode(l, q.to(cuda_device))
+        check_out(out.cpu().numpy(), oracle.decode(l, q))
+    check_state(cache, oracle)
+    assert cache.status() == 0
+
+
+def test_ring_wraps_many_times_and_mixed_append_sizes(rl, hz, cuda_device):
+    """Appends in chunks of 1, 7, 300 ... so the ring wraps inside and across bulk appends; state is
+    compared bit for bit and outputs at several lengths."""
+    layers, Hkv, Hq, D, B, S, W = 1, 2, 4, 64, 2, 16, 48
+    total = 1500
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, total, [0, 1], S, W, cuda_device)
+    K, V = rand_bf16((total, B, Hkv, D), 1), rand_bf16((total, B, Hkv, D), 2)
+    t, sizes, i = 0, [1, 7, 300, 2, 64, 1, 1, 129, 48, 47, 500], 0
+    while t < total:
+        n = min(sizes[i % len(sizes)], total - t)
+        feed(cache, oracle, 0, K[t:t + n], V[t:t + n], bulk=n > 1)
+        t += n
+        i += 1
+        q = rand_bf16((B, Hq, D), 1000 + t)
+        check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), oracle.decode(0, q))
+        check_state(cache, oracle)
+    with pytest.raises(rl.RlkvError) as e:
+        cache.append(0, K[0].to(cuda_device), V[0].to(cuda_device))
+    assert e.value.code == rl.RLKV_EFULL
+    check_state(cache, oracle)          # the refused append changed nothing
+
+
+# ------------------------------------------------------------------------------------------ needles
+def test_planted_needles_at_tile_and_split_boundaries(rl, hz, cuda_device):
+    """One token whose key is aligned with q carries a marker value: the output must be the marker
+    iff the head retains the token.  Positions sweep tile edges and the compressed head's edges."""
+    D, n, S, W, B = 128, 2200, 16, 112, 1
+    base_K, base_V = rand_bf16((n, B, 2, D), 5), rand_bf16((n, B, 2, D), 6)
+    q = rand_bf16((B, 2, D), 7)
+    marker = torch.full((D,), 7.0, dtype=torch.bfloat16)
+    spots = [0, 1, S - 1, S, 63, 64, 65, 127, 128, 1023, 1024, n - W - 1, n - W, n - 2, n - 1]
+    # the flat tile space of this shape is split over many CTAs: add their boundaries too
+    spots += [t for c in range(1, 12) for t in (c * 192 - 1, c * 192)]
+    for t_star in sorted(set(spots)):
+        K, V = base_K.clone(), base_V.clone()
+        for h in range(2):
+            qq = q[0, h].to(torch.float32)
+            K[t_star, 0, h] = (qq / qq.norm() * 100.0).to(torch.bfloat16)
+            V[t_star, 0, h] = marker
+        cache, oracle = build_pair(hz, 1, 2, 2, D, B, n, [1, 0], S, W, cuda_device)
+        feed(cache, oracle, 0, K, V, bulk=True)
+        out = cache.decode(0, q.to(cuda_device)).cpu().numpy()
+        want = oracle.decode(0, q)
+        check_out(out, want)
+        assert np.abs(out[0, 0] - 7.0).max() < 1e-2
+        visible = t_star < S or t_star >= n - W
+        assert (np.abs(out[0, 1] - 7.0).max() < 1e-2) == visible
+        cache.close()
+
+
+# ------------------------------------------------------------------------------------------ budget
+def test_compressed_heads_stay_inside_their_budget(rl, hz, cuda_device):
+    """Caller-provided buffer framed by sentinel guard bands; after many appends and decodes the
+    guards are intact, bytes read per step stop growing with n for compressed heads, and the padding
+    rows of every head are still zero."""
+    layers, Hkv, Hq, D, B, S, W, max_len = 2, 2, 4, 64, 2, 4, 28, 400
+    mask = [0, 1, 0, 0]
+    need = rl.rlkv_cache_size(layers, Hkv, Hq, D, B, max_len, mask, S, W)
+    guard = 4096
+    buf = torch.full((need + 2 * guard + 1024,), 0xA5, dtype=torch.uint8, device=cuda_device)
+    off = (-buf.data_ptr() - guard) % 1024 + guard
+    inner = buf[off:off + need]
+    assert inner.data_ptr() % 1024 == 0
+    cache = hz.Cache(layers, Hkv, Hq, D, B, max_len, mask, S, W, device=cuda_device, device_buf=inner)
+    oracle = Oracle(layers, Hkv, Hq, D, B, max_len, mask, S, W)
+    K, V = rand_bf16((max_len, B, Hkv, D), 8), rand_bf16((max_len, B, Hkv, D), 9)
+    seen = []
+    for l in range(layers):
+        for t0 in range(0, max_len, 50):
+            feed(cache, oracle, l, K[t0:t0 + 50], V[t0:t0 + 50], bulk=(t0 % 100 == 0))
+            q = rand_bf16((B, Hq, D), t0)
+            check_out(cache.decode(l, q.to(cuda_device)).cpu().numpy(), oracle.decode(l, q))
+            if l == 1:
+                seen.append(cache.step_bytes(1))
+    check_state(cache, oracle)
+    torch.cuda.synchronize()
+    assert (buf[:off] == 0xA5).all() and (buf[off + need:] == 0xA5).all()
+    # layer 1 has only compressed heads: bytes per step are constant once n >= S + W
+    assert seen[0] == B * 2 * 32 * 2 * D * 2 and len(set(seen)) == 1
+    # cost model in integers: bytes == B * 2*D*2 * (n_full*n + n_comp*min(n, S+W))
+    assert cache.step_bytes(0) == B * 2 * D * 2 * (1 * max_len + 1 * (S + W))
+    with pytest.raises(rl.RlkvError) as e:
+        cache.append(1, K[0].to(cuda_device), V[0].to(cuda_device))
+    assert e.value.code == rl.RLKV_EFULL      # uniform rule, even for an all-compressed layer
+
+
+# ------------------------------------------------------------------------------------------ errors
+def test_error_paths_leave_state_untouched(rl, hz, cuda_device):
+    D, B, Hkv, Hq = 64, 1, 2, 4
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_cache_create(1, 2, 5, D, B, 10, [1, 0], 1, 1)          # q_heads % kv_heads
+    assert e.value.code == rl.RLKV_EINVAL
+    for bad in (dict(head_dim=96), dict(window=0), dict(sink=-1), dict(q_heads=18)):
+        args = dict(layers=1, kv_heads=2, q_heads=4, head_dim=D, batch=B, max_len=10, head_is_full=[1, 0],
+                    sink=1, window=1)
+        args.update(bad)
+        with pytest.raises(rl.RlkvError) as e:
+            rl.rlkv_cache_create(**args)
+        assert e.value.code == rl.RLKV_EINVAL
+    cache = hz.Cache(1, Hkv, Hq, D, B, 10, [1, 0], 1, 2, device=cuda_device)
+    q = rand_bf16((B, Hq, D), 1, cuda_device)
+    out = torch.zeros((B, Hq, D), dtype=torch.float32, device=cuda_device)
+    with pytest.raises(rl.RlkvError) as e:
+        cache.decode(0, q, out)
+    assert e.value.code == rl.RLKV_EEMPTY
+    k = rand_bf16((B, Hkv, D), 2, cuda_device)
+    for call in (lambda: rl.rlkv_append(cache.handle, 1, k, k), lambda: rl.rlkv_append(cache.handle, -1, k, k),
+                 lambda: rl.rlkv_append(cache.handle, 0, 0, k), lambda: rl.rlkv_append(cache.handle, 0, k.data_ptr() + 2, k),
+                 lambda: rl.rlkv_decode_attention(cache.handle, 0, q, 0),
+                 lambda: rl.rlkv_prefill(cache.handle, 0, k, k, 0)):
+        with pytest.raises(rl.RlkvError) as e:
+            call()
+        assert e.value.code == rl.RLKV_EINVAL
+    big = rand_bf16((11, B, Hkv, D), 3, cuda_device)
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_prefill(cache.handle, 0, big, big, 11)
+    assert e.value.code == rl.RLKV_EFULL
+    assert cache.length(0) == 0 and not out.any()
+    gk, gv, gt = cache.export_head(0, 0, 0)
+    assert not gk.any() and not gv.any() and (gt == -1).all()
+    assert rl.rlkv_strerror(rl.RLKV_EFULL) and cache.status() == 0
+
+
+# ------------------------------------------------------------------------------------------ step API
+def test_step_and_step_host_equal_per_layer_calls(rl, hz, cuda_device):
+    w = synth.WORKLOADS["llama8b"].with_(layers=3, batch=2, context=200)
+    mask = synth.head_mask(w.seed, w.layers, w.kv_heads, 0.4)
+    a = hz.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, 260, mask, w.sink, w.window, device=cuda_device)
+    b = hz.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, 260, mask, w.sink, w.window, device=cuda_device)
+    c = hz.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, 260, mask, w.sink, w.window, device=cuda_device)
+    oracle = Oracle(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, 260, mask, w.sink, w.window, threads=8)
+    for cache in (a, b, c):
+        hz.fill_cache(cache, w, 200)
+    for l in range(w.layers):
+        K = synth.rows(w.seed, synth.STREAM_K, l, 0, 200, w.batch, w.kv_heads, w.head_dim)
+        V = synth.rows(w.seed, synth.STREAM_V, l, 0, 200, w.batch, w.kv_heads, w.head_dim)
+        for t in range(200):
+            oracle.append(l, K[t], V[t])
+    for t in range(200, 203):
+        k, v, q = hz.step_inputs(w, t, cuda_device)
+        out_a = torch.empty((w.layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=cuda_device)
+        for l in range(w.layers):
+            a.append(l, k[l], v[l])
+            a.decode(l, q[l], out_a[l])
+        out_b = torch.empty_like(out_a)
+        rl.rlkv_step(b.handle, k, v, q, out_b)
+        kh, vh, qh = (x.cpu().pin_memory() for x in (k, v, q))
+        out_c = torch.empty(out_a.shape, dtype=torch.float32).pin_memory()
+        rl.rlkv_step_host(c.handle, kh, vh, qh, out_c)
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, out_b) and torch.equal(out_a.cpu(), out_c)
+        for l in range(w.layers):
+            oracle.append(l, k[l].cpu(), v[l].cpu())
+            check_out(out_a[l].cpu().numpy(), oracle.decode(l, q[l].cpu()))
+    check_state(b, oracle)
+    check_state(c, oracle)
+    assert rl.rlkv_launch_count(b.handle) > 0
+
+
+def test_reset_and_config_knobs(rl, hz, cuda_device):
+    D, B, Hkv, Hq, n = 128, 2, 2, 8, 700
+    cache, oracle = build_pair(hz, 1, Hkv, Hq, D, B, n, [1, 0], 16, 112, cuda_device)
+    K, V, q = rand_bf16((n, B, Hkv, D), 1), rand_bf16((n, B, Hkv, D), 2), rand_bf16((B, Hq, D), 3)
+    feed(cache, oracle, 0, K, V, True)
+    want = oracle.decode(0, q)
+    outs = []
+    for cps, st in ((1, 6), (1, 2), (2, 3), (1, 4)):
+        rl.rlkv_set_decode_config(cache.handle, cps, st)
+        outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
+        check_out(outs[-1], want)
+    with pytest.raises(rl.RlkvError):
+        rl.rlkv_set_decode_config(cache.handle, 2, 6)       # does not fit in shared memory twice
+    rl.rlkv_cache_reset(cache.handle)
+    assert cache.length(0) == 0
+    gk, gv, gt = cache.export_head(0, 0, 1)
+    assert not gk.any() and not gv.any() and (gt == -1).all()
+    feed(cache, Oracle(1, Hkv, Hq, D, B, n, [1, 0], 16, 112), 0, K[:100], V[:100], True)
+    o2 = Oracle(1, Hkv, Hq, D, B, n, [1, 0], 16, 112)
+    for t in range(100):
+        o2.append(0, K[t], V[t])
+    check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), o2.decode(0, q))
+
+
+def test_plain_variant_agrees(rl, hz, cuda_device):
+    """The debugging cross-check kernel (no TMA, no tensor cores) against the oracle."""
+    os.environ["RLKV_DECODE_PLAIN"] = "1"
+    try:
+        cache, oracle = build_pair(hz, 1, 4, 28, 128, 2, 1500, [1, 0, 0, 1], 16, 112, cuda_device)
+    finally:
+        del os.environ["RLKV_DECODE_PLAIN"]
+    K, V, q = rand_bf16((1500, 2, 4, 128), 1), rand_bf16((1500, 2, 4, 128), 2), rand_bf16((2, 28, 128), 3)
+    feed(cache, oracle, 0, K, V, True)
+    check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), oracle.decode(0, q))
+    assert cache.status() == 0
