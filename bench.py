@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-attention hot path over a head-mixed KV cache.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama8b|qwen7b|cot|tiny]
+                    [--frac F] [--context C] [--batch B] [--impl ours|reference]
+
+One "step" = for every layer: rlkv_append of one token, then rlkv_decode_attention, over a cache
+that already holds `context` tokens.  Prints ONE JSON line (rank 0).  Inputs are synthetic, seeded,
+bf16 N(0,1); head classes come from a seeded global selection (see synth/).
+
+  value      tokens/s = N * batch * K / (time of K steps, device-timed, max over ranks), inputs
+             resident in HBM (rlkv_step)
+  roofline   the decode kernel: algorithmic K/V bytes per launch / mean launch duration, CUDA
+             events around every rlkv_decode_attention launch of K more steps
+  e2e        the same K steps through rlkv_step_host: pinned host inputs copied in and the result
+             copied out inside the timed region
+  cpu_baseline  the CPU oracle on a bounded sample (rank 0, N=1 only), scaled by bytes
+
+With N > 1 (torchrun) every rank runs the same workload on its own GPU: the path shards by batch
+rows / replicas with no exchange step, so there is no collective on the data path (weak scaling).
+--impl reference times the CPU oracle alone on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import synth
+
+METRIC = "decode-attn tokens/s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------------------------
+def parse_args(argv=None):
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=20)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    p.add_argument("--workload", default="llama8b", choices=sorted(synth.WORKLOADS))
+    p.add_argument("--frac", type=float, default=None, help="override the fraction of compressed KV heads")
+    p.add_argument("--context", type=int, default=None)
+    p.add_argument("--batch", type=int, default=None)
+    p.add_argument("--layers", type=int, default=None)
+    p.add_argument("--ctas-per-sm", type=int, default=0)
+    p.add_argument("--stages", type=int, default=0)
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-e2e", action="store_true")
+    return p.parse_args(argv)
+
+
+def pick_workload(args) -> synth.Workload:
+    w = synth.WORKLOADS[args.workload]
+    kw = {}
+    if args.frac is not None:
+        kw["frac_compressed"] = args.frac
+    if args.context is not None:
+        kw["context"] = args.context
+    if args.batch is not None:
+        kw["batch"] = args.batch
+    if args.layers is not None:
+        kw["layers"] = args.layers
+    return w.with_(**kw) if kw else w
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (earlier pool measurement)"
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """MAX of a per-rank scalar over the process group (identity without a group)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while a timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.rows, self.proc = gpu_index, [], None
+
+    def wait_first_sample(self, timeout=3.0):
+        t0 = time.perf_counter()
+        while self.proc and not self.rows and time.perf_counter() - t0 < timeout:
+            time.sleep(0.01)
+
+    def mark(self):
+        """Index of the next sample: samples from here on belong to what follows."""
+        return len(self.rows)
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) == 7:
+                self.rows.append(parts)
+
+    def __exit__(self, *exc):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=5)
+
+    def summary(self, start=0):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows[start:]:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+def workload_bytes(w: synth.Workload, mask: np.ndarray, n: int) -> int:
+    """K/V bytes one decode step over all layers must read at length n (integer cost model)."""
+    n_full = int(mask.sum())
+    n_comp = mask.size - n_full
+    rows = n_full * n + n_comp * min(n, w.sink + w.window)
+    return w.batch * rows * 2 * w.head_dim * 2
+
+
+def build_oracle_sample(w: synth.Workload, mask: np.ndarray, gen_device, target_bytes=200e6):
+    from oracle.rlkv_oracle import Oracle
+    n = w.context + 1
+    layer_mask = mask[:w.kv_heads]
+    per_row = workload_bytes(w.with_(batch=1, layers=1), layer_mask, n)
+    sb = int(max(1, min(w.batch, target_bytes // max(per_row, 1))))
+    oracle = Oracle(1, w.kv_heads, w.q_heads, w.head_dim, sb, n, layer_mask, w.sink, w.window)
+    chunk = max(1, (1 << 23) // (w.batch * w.kv_heads * w.head_dim))
+    for t0 in range(0, w.context, chunk):
+        t1 = min(w.context, t0 + chunk)
+        k = synth.rows(w.seed, synth.STREAM_K, 0, t0, t1, w.batch, w.kv_heads, w.head_dim, gen_device)[:, :sb].cpu()
+        v = synth.rows(w.seed, synth.STREAM_V, 0, t0, t1, w.batch, w.kv_heads, w.head_dim, gen_device)[:, :sb].cpu()
+        for t in range(t1 - t0):
+            oracle.append(0, k[t].contiguous(), v[t].contiguous())
+    t = w.context
+    k1 = synth.rows(w.seed, synth.STREAM_K, 0, t, t + 1, w.batch, w.kv_heads, w.head_dim)[0, :sb].contiguous()
+    v1 = synth.rows(w.seed, synth.STREAM_V, 0, t, t + 1, w.batch, w.kv_heads, w.head_dim)[0, :sb].contiguous()
+    q = synth.rows(w.seed, synth.STREAM_Q, 0, t, t + 1, w.batch, w.q_heads, w.head_dim)[0, :sb].contiguous()
+    sample_bytes = workload_bytes(w.with_(batch=sb, layers=1), layer_mask, n)
+    desc = f"layer 0, batch rows 0..{sb - 1}, all {w.kv_heads} KV heads, n={n}: {sample_bytes / 1e6:.1f} MB of K/V"
+    return oracle, (k1, v1, q), sample_bytes, desc
+
+
+def time_oracle(oracle, step_in, threads: int, min_seconds: float, min_reps: int = 1):
+    """Median seconds of one oracle decode over the sample (the append is done once, untimed:
+    re-appending would grow the sample)."""
+    k1, v1, q = step_in
+    oracle.set_threads(threads)
+    if oracle.length(0) == oracle.max_len - 1:
+        oracle.append(0, k1, v1)
+    times, t_all = [], time.perf_counter()
+    while len(times) < min_reps or time.perf_counter() - t_all < min_seconds:
+        t0 = time.perf_counter()
+        oracle.decode(0, q)
+        times.append(time.perf_counter() - t0)
+    return statistics.median(times), len(times)
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, w, mask):
+    """--impl reference: the CPU oracle as it stands on the host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle.rlkv_oracle import max_threads
+    gen_dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    oracle, step_in, sample_bytes, desc = build_oracle_sample(w, mask, gen_dev)
+    threads = max_threads()
+    oracle.set_threads(threads)
+    k1, v1, q = step_in
+    oracle.append(0, k1, v1)
+    for _ in range(args.warmup):
+        oracle.decode(0, q)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.decode(0, q)
+    per_sample = (time.perf_counter() - t0) / args.steps
+    total_bytes = workload_bytes(w, mask, w.context + 1)
+    ms_per_step = per_sample * total_bytes / sample_bytes * 1e3
+    value = w.batch / (ms_per_step / 1e3)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": config_dict(w, mask, note="CPU oracle; each step = one decode over the sample, scaled to the "
+                                            "whole workload by K/V bytes"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def config_dict(w, mask, note=None):
+    n_comp = int((mask == 0).sum())
+    cfg = {"workload": w.name, "layers": w.layers, "q_heads": w.q_heads, "kv_heads": w.kv_heads,
+           "head_dim": w.head_dim, "batch_per_gpu": w.batch, "context": w.context,
+           "compressed_heads": f"{n_comp} of {mask.size}", "frac_compressed": w.frac_compressed,
+           "sink": w.sink, "window": w.window, "seed": w.seed,
+           "l2": "inputs larger than L2: every layer's K/V working set exceeds 126 MB and is read once per step"}
+    if note:
+        cfg["note"] = note
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args, w, mask):
+    import torch.distributed as dist
+    from paper_2510_08525_b200 import binding as rl
+    from paper_2510_08525_b200 import harness
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: librlkv has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    K, W = args.steps, args.warmup
+    passes = 3                                    # device-resident, per-launch events, host buffers
+    total_new = passes * (K + W) + 8
+    cache = harness.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, w.context + total_new, mask,
+                          w.sink, w.window, device=dev)
+    if args.ctas_per_sm or args.stages:
+        rl.rlkv_set_decode_config(cache.handle, args.ctas_per_sm, args.stages)
+    harness.fill_cache(cache, w, w.context)
+
+    # inputs of every step, resident on the device (and a pinned host copy for the e2e pass)
+    steps_in = [harness.step_inputs(w, w.context + i, dev) for i in range(total_new - 8)]
+    out = torch.empty((w.layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    nxt = 0
+
+    def device_step(i):
+        k, v, q = steps_in[i]
+        rl.rlkv_step(cache.handle, k, v, q, out, stream)
+
+    # ---- pass 1: device-resident steps (the headline value).  The clock sampler runs from the
+    # warm-up of this pass to the end of the last pass: every sample is taken under load.
+    clocks = ClockSampler(local)
+    clocks.__enter__()
+    clocks.wait_first_sample()
+    for _ in range(W):
+        device_step(nxt); nxt += 1
+    launches0 = rl.rlkv_launch_count(cache.handle)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(); torch.cuda.synchronize()
+    clock_mark = clocks.mark()
+    e0.record(stream)
+    for _ in range(K):
+        device_step(nxt); nxt += 1
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    launches = rl.rlkv_launch_count(cache.handle) - launches0
+    ms_per_step = elapsed_ms / K
+    value = world * w.batch * K / (elapsed_ms / 1e3)
+
+    # ---- pass 2: per-launch CUDA events around every decode-attention launch
+    for _ in range(W):
+        device_step(nxt); nxt += 1
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(K * w.layers)]
+    bytes_launch = []
+    torch.cuda.synchronize()
+    for s in range(K):
+        k, v, q = steps_in[nxt]; nxt += 1
+        for l in range(w.layers):
+            rl.rlkv_append(cache.handle, l, k[l], v[l], stream)
+            a, b = ev[s * w.layers + l]
+            a.record(stream)
+            rl.rlkv_decode_attention(cache.handle, l, q[l], out[l], stream)
+            b.record(stream)
+            bytes_launch.append(rl.rlkv_step_bytes(cache.handle, l))
+    torch.cuda.synchronize()
+    durs = [a.elapsed_time(b) for a, b in ev]
+    peak, peak_src = measured_peak_gbs()
+    achieved = sum(bytes_launch) / (sum(durs) * 1e-3) / 1e9
+    # launches that carry at least one full head are the bandwidth-bound ones; report them separately
+    big = [(by, d) for by, d in zip(bytes_launch, durs) if by > 64e6]
+    roofline = {
+        "bound": "hbm", "kernel": "rlkv::decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": peak_src, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+        "traffic": None, "launches_timed": len(durs), "mean_launch_us": 1e3 * sum(durs) / len(durs),
+        "algorithmic_bytes_per_launch": sum(bytes_launch) / len(bytes_launch),
+        "achieved_launches_over_64MB": (sum(b for b, _ in big) / (sum(d for _, d in big) * 1e-3) / 1e9) if big else None,
+    }
+
+    # ---- pass 3: end to end through rlkv_step_host (pinned host buffers, copies inside the timed region)
+    e2e = None
+    if not args.no_e2e:
+        host_in = []
+        for i in range(nxt, nxt + K + W):
+            host_in.append(tuple(x.cpu().pin_memory() for x in steps_in[i]))
+        out_host = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+        h2d = sum(x.numel() * x.element_size() for x in host_in[0])
+        d2h = out_host.numel() * out_host.element_size()
+        for i in range(W):
+            rl.rlkv_step_host(cache.handle, *host_in[i], out_host, stream)
+        barrier(); torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(W, W + K):
+            rl.rlkv_step_host(cache.handle, *host_in[i], out_host, stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev)
+        e2e = {"value": world * w.batch * K / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K,
+               "checksum": float(out_host.double().abs().sum())}
+    clocks.__exit__()
+    status = cache.status()
+    if status != 0:
+        raise SystemExit(f"a kernel reported status {status}: results are invalid")
+
+    # ---- CPU oracle on a bounded sample (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle.rlkv_oracle import max_threads
+        oracle, step_in, sample_bytes, desc = build_oracle_sample(w, mask, dev)
+        threads = max_threads()
+        sec, reps = time_oracle(oracle, step_in, threads, min_seconds=10.0, min_reps=3)
+        sec1, reps1 = time_oracle(oracle, step_in, 1, min_seconds=5.0, min_reps=1)
+        total_bytes = workload_bytes(w, mask, w.context + 1)
+        cpu = {"value": w.batch / (sec * total_bytes / sample_bytes), "unit": UNIT, "cores": threads,
+               "kind": "oracle", "sample": f"{desc}; median of {reps} decodes, scaled to the step by K/V bytes",
+               "single_thread_value": w.batch / (sec1 * total_bytes / sample_bytes),
+               "oracle_gbs": sample_bytes / sec / 1e9}
+
+    if rank == 0:
+        total_bytes = workload_bytes(w, mask, w.context + 1)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_dict(w, mask),
+            "kv_bytes_per_step": total_bytes,
+            "step_hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
+            "bytes_ratio_vs_uncompressed": total_bytes / (w.batch * w.layers * w.kv_heads * (w.context + 1) * 4 * w.head_dim),
+            "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
+            "clocks": clocks.summary(clock_mark),
+        }
+        print(json.dumps(line), flush=True)
+    cache.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    w = pick_workload(args)
+    mask = synth.workload_mask(w)
+    if args.impl == "reference":
+        run_reference(args, w, mask)
+    else:
+        run_ours(args, w, mask)
+
+
+if __name__ == "__main__":
+    main()

@@ -63,10 +63,7 @@ class Cache:
         return rl.rlkv_kernel_status(self.handle)
 
 
-def workload_mask(w: synth.Workload) -> np.ndarray:
-    if w.name == "tiny":
-        return np.array([1, 0], dtype=np.uint8)     # KV head 0 full, KV head 1 compressed
-    return synth.head_mask(w.seed, w.layers, w.kv_heads, w.frac_compressed)
+workload_mask = synth.workload_mask
 
 
 def make_cache(w: synth.Workload, extra_tokens: int = 64, device="cuda:0") -> Cache:

@@ -18,4 +18,4 @@ from .generator import (  # noqa: F401
     rows,
     unit_rows,
 )
-from .workloads import WORKLOADS, Workload  # noqa: F401
+from .workloads import WORKLOADS, Workload, workload_mask  # noqa: F401

@@ -8,6 +8,8 @@ from __future__ import annotations
 
 from dataclasses import dataclass, replace
 
+import numpy as np
+
 
 @dataclass(frozen=True)
 class Workload:
@@ -39,3 +41,12 @@ WORKLOADS = {
     # long chain-of-thought loop: prompt of 4096 tokens, then 28672 generated steps
     "cot": Workload("cot", 32, 32, 8, 128, 8, 4096, 0.40, 16, 240, 3),
 }
+
+
+def workload_mask(w: Workload) -> "np.ndarray":
+    """uint8[layers*kv_heads], 1 = full cache.  The tiny workload fixes its mask (KV head 0 full,
+    KV head 1 compressed); every other workload draws it from the seeded global selection."""
+    from .generator import head_mask
+    if w.name == "tiny":
+        return np.array([1, 0] * w.layers, dtype=np.uint8)
+    return head_mask(w.seed, w.layers, w.kv_heads, w.frac_compressed)

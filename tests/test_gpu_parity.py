@@ -303,7 +303,7 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     feed(cache, oracle, 0, K, V, True)
     want = oracle.decode(0, q)
     outs = []
-    for cps, st in ((1, 6), (1, 2), (2, 3), (1, 4)):
+    for cps, st in ((1, 6), (1, 2), (2, 2), (1, 4)):
         rl.rlkv_set_decode_config(cache.handle, cps, st)
         outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
         check_out(outs[-1], want)
