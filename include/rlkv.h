@@ -117,9 +117,11 @@ int rlkv_debug_export_head(rlkv_cache* cache, int layer, int batch_row, int kv_h
 int rlkv_kernel_status(rlkv_cache* cache, int* status_out);
 /* Number of kernels this cache has launched so far. */
 int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
-/* Tuning knob for the decode kernel's grid: CTAs per SM (1 or 2) and pipeline stages (2..8);
- * 0 keeps the current value. */
-int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages);
+/* Tuning knobs of the decode kernel: persistent CTAs per SM (1 or 2), TMA pipeline stages (2..8)
+ * and groups of four consumer warps that take tiles in turn (1..3).  0 keeps the current value
+ * (stages: lowered if the new shape no longer fits).  RLKV_EINVAL if the shape does not fit in
+ * shared memory.  Defaults: 1 CTA per SM, 2 groups, as many stages as fit. */
+int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups);
 
 const char* rlkv_strerror(int code);
 

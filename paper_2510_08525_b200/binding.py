@@ -35,7 +35,7 @@ SIGNATURES = {
     "rlkv_debug_export_head": (_ci, [_vp, _ci, _ci, _ci, _vp, _vp, ctypes.POINTER(_ci), _vp]),
     "rlkv_kernel_status": (_ci, [_vp, ctypes.POINTER(_ci)]),
     "rlkv_launch_count": (_ci, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
-    "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci]),
+    "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
 }
 
@@ -184,8 +184,8 @@ def rlkv_launch_count(cache) -> int:
     return int(out.value)
 
 
-def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0) -> None:
-    _check(lib.rlkv_set_decode_config(cache, ctas_per_sm, stages))
+def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0, consumer_groups=0) -> None:
+    _check(lib.rlkv_set_decode_config(cache, ctas_per_sm, stages, consumer_groups))
 
 
 def rlkv_strerror(code: int) -> str:

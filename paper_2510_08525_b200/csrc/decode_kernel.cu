@@ -9,10 +9,12 @@
 // units first, compressed units after).  A persistent grid splits that space evenly: CTA c owns the
 // contiguous range [c*T/P, (c+1)*T/P), so long full-head scans and short compressed-head scans
 // balance to within one tile.  Inside a CTA one producer warp streams tiles HBM -> shared memory
-// with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier pipeline); four consumer warps each
-// take 16 tokens of every tile: S = Q.K^T and O^T += V^T.P^T run on mma.sync m16n8k16 (bf16 in, fp32
-// accumulate) with the G query heads of the group as the M (resp. N) dimension, online softmax in
-// fp32 with warp shuffles.  The path is HBM-bound: the tensor-core work is ~G flop per byte.
+// with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier pipeline); NG groups of four consumer
+// warps take the tiles in turn, each warp 16 tokens of its group's tile: S = Q.K^T and
+// O^T += V^T.P^T run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G query heads of the
+// group as the M (resp. N) dimension, online softmax in fp32 with warp shuffles.  The path is
+// HBM-bound (the tensor-core work is ~G flop per byte); several groups are there only to hide the
+// dependent-issue latency of one tile's softmax chain behind another tile's.
 // When a CTA's range ends inside a unit it writes an (m, l, O) partial; the last CTA to finish a
 // unit (atomic ticket, no spinning) merges the partials with the log-sum-exp rule and writes out.
 #include "rlkv_internal.cuh"
@@ -20,7 +22,6 @@
 namespace rlkv {
 namespace {
 
-constexpr int kThreads = kConsumerThreads + 32;  // 4 consumer warps + 1 producer warp
 constexpr float kNegBig = -1.0e30f;              // finite "minus infinity" for running maxima
 
 // ---------------------------------------------------------------------------------------------
@@ -69,9 +70,26 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+// Byte offset inside a tile row of 16-byte chunk `chunk` of row `row` under the 128-byte swizzle.
+template <int D>
+__device__ __forceinline__ uint32_t swizzled_chunk(int row, int chunk)
+{
+    if (D == 128) return (uint32_t)(((chunk & 8) | ((chunk & 7) ^ ((2 * row + (chunk >> 3)) & 7))) << 4);
+    return (uint32_t)((chunk ^ (row & 7)) << 4);
+}
+template <int NG>
 __device__ __forceinline__ void consumer_sync()
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kConsumerThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"n"(NG * kGroupWarps * 32) : "memory");
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
                                             uint32_t& r3)
@@ -127,48 +145,52 @@ __device__ __forceinline__ void wait_bounded(uint32_t bar, uint32_t parity, vola
 
 // ---------------------------------------------------------------------------------------------
 // Shared-memory carve-up (dynamic shared memory, base aligned to 1024 bytes for the swizzle).
-template <int D>
+template <int D, int NG>
 struct Smem {
-    static constexpr int kTileBytes = kTile * D * 2;       // one K (or V) tile
-    static constexpr int kStageBytes = 2 * kTileBytes;     // K tile then V tile
-    static constexpr int kMergeStride = D + kMergePad;     // floats per head row
-    static constexpr int kMergeFloats = kConsumerWarps * kMaxGroup * kMergeStride;
-    static constexpr int kStatFloats = 2 * kConsumerWarps * kMaxGroup;
-    __host__ __device__ static constexpr size_t bytes(int stages)
+    static constexpr int kWarps = NG * kGroupWarps;         // consumer warps
+    static constexpr int kTileBytes = kTile * D * 2;        // one K (or V) tile
+    static constexpr int kStageBytes = 2 * kTileBytes;      // K tile then V tile
+    static constexpr int kMergeStride = D + kMergePad;      // floats per head row
+    static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
+    __host__ __device__ static constexpr int merge_floats(int group) { return kWarps * group * kMergeStride; }
+    __host__ __device__ static constexpr size_t bytes(int stages, int group)
     {
-        return 1024 /*alignment slack*/ + (size_t)stages * kStageBytes + kMergeFloats * 4 +
+        return 1024 /*alignment slack*/ + (size_t)stages * kStageBytes + merge_floats(group) * 4 +
                kStatFloats * 4 + 2 * 8 * 8 /*barriers*/ + 16 /*flags*/;
     }
 };
 
 // ---------------------------------------------------------------------------------------------
 // End of a segment (the part of one unit a CTA processed).  Input: each consumer warp has put its
-// running max / sum / un-normalised output into the merge area.  The 128 consumer threads merge the
-// four warps; a complete unit is normalised and written out, otherwise the partial goes to the
-// scratch buffer and the last CTA to arrive for that unit merges all partials of the unit.
-template <int D>
+// running max / sum / un-normalised output into the merge area.  The consumer threads merge the
+// warps; a complete unit is normalised and written out, otherwise the partial goes to the scratch
+// buffer and the last CTA to arrive for that unit merges all partials of the unit.
+template <int D, int NG>
 __device__ void finalize_segment(const DecodeArgs& a, const UnitInfo& u, bool complete,
                                  const float* merge, const float* stat_m, const float* stat_l,
-                                 int* s_flag, int ctid, int T, int P)
+                                 int* s_flag, int ctid)
 {
-    constexpr int MS = Smem<D>::kMergeStride;
+    const int T = a.full_tiles, P = a.grid_full;  // the split space of the full units
+    using S = Smem<D, NG>;
+    constexpr int MS = S::kMergeStride;
     constexpr int PF = partial_floats(D);
+    constexpr int NT = S::kWarps * 32;
     const int G = a.group;
-    consumer_sync();  // merge area written by all warps
+    consumer_sync<NG>();  // merge area written by all warps
 
     const int cta = blockIdx.x;
-    const int my_slot = (cta_start(cta, T, P) >= u.first_tile) ? 0 : 1;
+    const int my_slot = (complete || cta_start(cta, T, P) >= u.first_tile) ? 0 : 1;
     float* my_part = a.partials + ((size_t)cta * 2 + my_slot) * PF;
     float* out_rows = a.out + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
 
-    for (int idx = ctid; idx < G * D; idx += kConsumerThreads) {
+    for (int idx = ctid; idx < G * D; idx += NT) {
         const int g = idx / D, d = idx - g * D;
         float M = kNegBig, L = 0.f, O = 0.f;
 #pragma unroll
-        for (int w = 0; w < kConsumerWarps; ++w) {
+        for (int w = 0; w < S::kWarps; ++w) {
             const float mw = stat_m[w * kMaxGroup + g];
             const float lw = stat_l[w * kMaxGroup + g];
-            const float ow = merge[(w * kMaxGroup + g) * MS + d];
+            const float ow = merge[(w * G + g) * MS + d];
             const float Mn = fmaxf(M, mw);
             const float ca = exp2f(M - Mn), cb = exp2f(mw - Mn);
             L = L * ca + lw * cb;
@@ -189,15 +211,15 @@ __device__ void finalize_segment(const DecodeArgs& a, const UnitInfo& u, bool co
         const int first_c = cta_of_tile(u.first_tile, T, P);
         const int last_c = cta_of_tile((long long)u.first_tile + u.tiles - 1, T, P);
         __threadfence();
-        consumer_sync();
+        consumer_sync<NG>();
         if (ctid == 0) {
             const int old = atomicAdd(&a.tickets[u.unit], 1);
             *s_flag = (old == last_c - first_c);
         }
-        consumer_sync();
+        consumer_sync<NG>();
         if (*s_flag) {
             __threadfence();
-            for (int idx = ctid; idx < G * D; idx += kConsumerThreads) {
+            for (int idx = ctid; idx < G * D; idx += NT) {
                 const int g = idx / D;
                 float M = kNegBig, L = 0.f, O = 0.f;
                 for (int c = first_c; c <= last_c; ++c) {
@@ -217,38 +239,36 @@ __device__ void finalize_segment(const DecodeArgs& a, const UnitInfo& u, bool co
             if (ctid == 0) a.tickets[u.unit] = 0;  // ready for the next launch
         }
     }
-    consumer_sync();  // merge area and s_flag may be reused
+    consumer_sync<NG>();  // merge area and s_flag may be reused
 }
 
 // ---------------------------------------------------------------------------------------------
-// The kernel.
-template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+// The kernel.  Warps 0 .. 4*NG-1 are consumers (group = warp / 4), the last warp is the producer.
+template <int D, int NG>
+__global__ void __launch_bounds__(NG * kGroupWarps * 32 + 32, 1)
 decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, const int stages)
 {
-    using S = Smem<D>;
+    using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                                ~static_cast<uintptr_t>(1023));
     uint8_t* stage_base = smem;
     float* merge = reinterpret_cast<float*>(smem + (size_t)stages * S::kStageBytes);
-    float* stat_m = merge + S::kMergeFloats;
-    float* stat_l = stat_m + kConsumerWarps * kMaxGroup;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(stat_l + kConsumerWarps * kMaxGroup);
+    float* stat_m = merge + S::merge_floats(a.group);
+    float* stat_l = stat_m + S::kWarps * kMaxGroup;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(stat_l + S::kWarps * kMaxGroup);
     uint64_t* empty_bar = full_bar + 8;
     int* s_flag = reinterpret_cast<int*>(empty_bar + 8);
     volatile int* s_abort = s_flag + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int T = a.total_tiles, P = gridDim.x;
-    const int start = (int)cta_start(blockIdx.x, T, P);
-    const int end = (int)cta_start(blockIdx.x + 1, T, P);
+    const CtaWork work = cta_work(a, blockIdx.x, gridDim.x);
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
-            mbar_init(smem_u32(empty_bar + s), kConsumerWarps);
+            mbar_init(smem_u32(empty_bar + s), kGroupWarps);
         }
         *s_flag = 0;
         *s_abort = 0;
@@ -256,15 +276,14 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
     }
     __syncthreads();
 
-    if (warp == kConsumerWarps) {
+    if (warp == S::kWarps) {
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
-            int it = 0;
-            for (int x = start; x < end; ++x, ++it) {
-                const UnitInfo u = locate(a, x);
-                const int s = it % stages;
-                const uint32_t par = (uint32_t)(it / stages) & 1u;
+            int s = 0;
+            uint32_t par = 0;
+            for (int v = 0; v < work.total; ++v) {
+                const UnitInfo u = locate(a, work, v);
                 wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status,
                              kStatusEmptyWaitTimeout);
                 const uint32_t fb = smem_u32(full_bar + s);
@@ -272,24 +291,35 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                 const uint32_t dst = smem_u32(stage_base + (size_t)s * S::kStageBytes);
                 const int krow = (int)(u.krow + (long long)u.tile * kTile);
                 const int vrow = krow + u.rows;
-#pragma unroll
-                for (int half = 0; half < D / 64; ++half) {
-                    tma_load_2d(dst + half * (kTile * 128), &tmap, half * 64, krow, fb);
-                    tma_load_2d(dst + S::kTileBytes + half * (kTile * 128), &tmap, half * 64, vrow,
-                                fb);
+                if (D == 128) {  // one contiguous 16 KB box per tile: [64 rows][2 halves][64]
+                    tma_load_3d(dst, &tmap, 0, 0, krow, fb);
+                    tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb);
+                } else {         // one contiguous 8 KB box per tile: [64 rows][64]
+                    tma_load_2d(dst, &tmap, 0, krow, fb);
+                    tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb);
+                }
+                if (++s == stages) {
+                    s = 0;
+                    par ^= 1u;
                 }
             }
         }
     } else {
         // ------------------------------------------------------------------ consumer warps
+        const int grp = warp / kGroupWarps, wig = warp % kGroupWarps;  // tile group, 16-token slice
         const int quad = lane >> 2, tq = lane & 3;  // row inside an 8-row fragment, column pair
         const int ldm_j = lane >> 3, ldm_r = lane & 7;
-        const int ldm_tok = warp * 16 + (ldm_j >> 1) * 8 + ldm_r;  // token row this lane addresses
-        const int ldm_chunk = ldm_j & 1;                           // +1 16-byte chunk for odd matrices
-        int it = 0;
-        for (int x = start; x < end;) {
-            const UnitInfo u = locate(a, x);
-            const int seg_tiles = min(end - x, u.tiles - u.tile);
+        const int ldm_tok = wig * 16 + (ldm_j >> 1) * 8 + ldm_r;  // token row this lane addresses
+        const int ldm_chunk = ldm_j & 1;                          // +1 16-byte chunk for odd matrices
+        // Tile layout in shared memory (written by TMA with the 128-byte swizzle): row r of the tile
+        // starts at r*2*D bytes; its 16-byte chunk c sits at chunk index c ^ (bits 7..9 of the
+        // unswizzled offset), i.e. c ^ ((2r + c/8) & 7) for D = 128 and c ^ (r & 7) for D = 64.
+        const uint32_t row_off = ldm_tok * (2 * D);
+        int s = 0, turn = 0;  // pipeline stage and whose turn the next tile is
+        uint32_t par = 0;
+        for (int v = 0; v < work.total;) {
+            const UnitInfo u = locate(a, work, v);
+            const int seg_tiles = min(work.total - v, u.tiles - u.tile);
 
             // Q as the A operand (rows = query heads of the group, rows >= G are zero)
             uint32_t qa[KS][2];
@@ -307,23 +337,29 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
 #pragma unroll
             for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
 
-            for (int i = 0; i < seg_tiles; ++i, ++it) {
-                const int s = it % stages;
-                const uint32_t par = (uint32_t)(it / stages) & 1u;
-                wait_bounded(smem_u32(full_bar + s), par, s_abort, a.status, kStatusFullWaitTimeout);
-                const int valid = min(kTile, u.len - (u.tile + i) * kTile);
-                if (warp * 16 < valid) {
-                    const uint32_t sK = smem_u32(stage_base + (size_t)s * S::kStageBytes);
+            int valid_left = u.len - u.tile * kTile;  // valid rows from this tile to the unit's end
+            for (int i = 0; i < seg_tiles; ++i, valid_left -= kTile) {
+                const bool mine = (turn == grp);
+                const int cur_s = s;
+                const uint32_t cur_par = par;
+                if (++turn == NG) turn = 0;
+                if (++s == stages) {
+                    s = 0;
+                    par ^= 1u;
+                }
+                if (!mine) continue;
+                wait_bounded(smem_u32(full_bar + cur_s), cur_par, s_abort, a.status, kStatusFullWaitTimeout);
+                const int valid = min(kTile, valid_left);
+                if (wig * 16 < valid && !(a.debug & 1)) {
+                    const uint32_t sK = smem_u32(stage_base + (size_t)cur_s * S::kStageBytes);
                     const uint32_t sV = sK + S::kTileBytes;
-                    const uint32_t row_off = ldm_tok * 128;
                     // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
                     float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
                     float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
                     for (int ks = 0; ks < KS; ++ks) {
                         const int chunk = ks * 2 + ldm_chunk;  // 16-byte chunk along d
-                        const uint32_t addr = sK + (chunk >> 3) * (kTile * 128) + row_off +
-                                              (((chunk & 7) ^ (ldm_tok & 7)) << 4);
+                        const uint32_t addr = sK + row_off + swizzled_chunk<D>(ldm_tok, chunk);
                         uint32_t b0, b1, b2, b3;
                         ldmatrix_x4(addr, b0, b1, b2, b3);
                         if (ks & 1) {
@@ -334,13 +370,13 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                             mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
                         }
                     }
-                    // this lane: head `quad`, tokens warp*16 + {2tq, 2tq+1, 8+2tq, 9+2tq}
+                    // this lane: head `quad`, tokens wig*16 + {2tq, 2tq+1, 8+2tq, 9+2tq}
                     float sc[4];
                     sc[0] = (s0[0] + s2[0]) * a.scale_log2;
                     sc[1] = (s0[1] + s2[1]) * a.scale_log2;
                     sc[2] = (s1[0] + s3[0]) * a.scale_log2;
                     sc[3] = (s1[1] + s3[1]) * a.scale_log2;
-                    const int tok0 = warp * 16 + 2 * tq;
+                    const int tok0 = wig * 16 + 2 * tq;
                     if (tok0 >= valid) sc[0] = -INFINITY;
                     if (tok0 + 1 >= valid) sc[1] = -INFINITY;
                     if (tok0 + 8 >= valid) sc[2] = -INFINITY;
@@ -363,8 +399,7 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
 #pragma unroll
                     for (int mt = 0; mt < KS; ++mt) {
                         const int chunk = mt * 2 + ldm_chunk;
-                        const uint32_t addr = sV + (chunk >> 3) * (kTile * 128) + row_off +
-                                              (((chunk & 7) ^ (ldm_tok & 7)) << 4);
+                        const uint32_t addr = sV + row_off + swizzled_chunk<D>(ldm_tok, chunk);
                         uint32_t v0, v1, v2, v3;
                         ldmatrix_x4_trans(addr, v0, v1, v2, v3);
                         acc[mt][0] *= ca;
@@ -375,7 +410,7 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(empty_bar + s));
+                if (lane == 0) mbar_arrive(smem_u32(empty_bar + cur_s));
             }
 
             // ---- hand the warp's state to the cross-warp merge
@@ -386,147 +421,88 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                 stat_l[warp * kMaxGroup + quad] = l_run;
             }
             {
-                float* mw = merge + (size_t)warp * kMaxGroup * S::kMergeStride;
+                const int G = a.group;
+                float* mw = merge + (size_t)warp * G * S::kMergeStride;
+                const int h0 = 2 * tq, h1 = 2 * tq + 1;
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) {
                     const int d0 = mt * 16 + quad;
-                    mw[(2 * tq) * S::kMergeStride + d0] = acc[mt][0];
-                    mw[(2 * tq + 1) * S::kMergeStride + d0] = acc[mt][1];
-                    mw[(2 * tq) * S::kMergeStride + d0 + 8] = acc[mt][2];
-                    mw[(2 * tq + 1) * S::kMergeStride + d0 + 8] = acc[mt][3];
+                    if (h0 < G) {
+                        mw[h0 * S::kMergeStride + d0] = acc[mt][0];
+                        mw[h0 * S::kMergeStride + d0 + 8] = acc[mt][2];
+                    }
+                    if (h1 < G) {
+                        mw[h1 * S::kMergeStride + d0] = acc[mt][1];
+                        mw[h1 * S::kMergeStride + d0 + 8] = acc[mt][3];
+                    }
                 }
             }
-            finalize_segment<D>(a, u, u.tile == 0 && seg_tiles == u.tiles, merge, stat_m, stat_l,
-                                s_flag, tid, T, P);
-            x += seg_tiles;
+            finalize_segment<D, NG>(a, u, u.tile == 0 && seg_tiles == u.tiles, merge, stat_m, stat_l,
+                                    s_flag, tid);
+            v += seg_tiles;
         }
     }
     __syncthreads();
-    if (warp == kConsumerWarps && lane == 0 && *s_abort) {
+    if (warp == S::kWarps && lane == 0 && *s_abort) {
         // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
         // when the CTA retires
-        const int issued = end - start;
+        const int issued = work.total;
         for (int j = issued > stages ? issued - stages : 0; j < issued; ++j)
             wait_bounded(smem_u32(full_bar + j % stages), (uint32_t)(j / stages) & 1u, s_abort, a.status,
                          kStatusDrainTimeout, false);
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Plain variant without TMA or tensor cores: direct global loads, CUDA-core FMAs, one token at a
-// time per warp.  Same tile space, same partial/ticket protocol.  Kept as the debugging
-// cross-check of the pipelined kernel (RLKV_DECODE_PLAIN=1 at cache creation); never the default.
-template <int D>
-__global__ void __launch_bounds__(kConsumerThreads, 2)
-decode_kernel_plain(const DecodeArgs a)
+template <int D, int NG>
+cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream)
 {
-    using S = Smem<D>;
-    constexpr int DPL = D / 32;  // head_dim elements per lane
-    __shared__ float merge[S::kMergeFloats];
-    __shared__ float stat_m[kConsumerWarps * kMaxGroup];
-    __shared__ float stat_l[kConsumerWarps * kMaxGroup];
-    __shared__ int s_flag;
+    const size_t smem = Smem<D, NG>::bytes(stages, a.group);
+    decode_kernel<D, NG><<<grid, NG * kGroupWarps * 32 + 32, smem, stream>>>(a, tmap, stages);
+    return cudaGetLastError();
+}
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int T = a.total_tiles, P = gridDim.x;
-    const int start = (int)cta_start(blockIdx.x, T, P);
-    const int end = (int)cta_start(blockIdx.x + 1, T, P);
-    const int G = a.group;
-
-    for (int x = start; x < end;) {
-        const UnitInfo u = locate(a, x);
-        const int seg_tiles = min(end - x, u.tiles - u.tile);
-        float qv[kMaxGroup][DPL], acc[kMaxGroup][DPL], m_run[kMaxGroup], l_run[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-            m_run[g] = kNegBig;
-            l_run[g] = 0.f;
-#pragma unroll
-            for (int j = 0; j < DPL; ++j) {
-                acc[g][j] = 0.f;
-                qv[g][j] = g < G ? __bfloat162float(a.q[((size_t)u.b * a.q_heads + (size_t)u.head * G + g) * D +
-                                                        lane * DPL + j])
-                                 : 0.f;
-            }
-        }
-        for (int i = 0; i < seg_tiles; ++i) {
-            const int tile = u.tile + i;
-            const int valid = min(kTile, u.len - tile * kTile);
-            for (int r = warp * 16; r < min(warp * 16 + 16, valid); ++r) {
-                const long long row = u.krow + (long long)tile * kTile + r;
-                const __nv_bfloat16* kp = a.pool + row * D + lane * DPL;
-                const __nv_bfloat16* vp = kp + (long long)u.rows * D;
-                float kf[DPL], vf[DPL];
-#pragma unroll
-                for (int j = 0; j < DPL; ++j) {
-                    kf[j] = __bfloat162float(kp[j]);
-                    vf[j] = __bfloat162float(vp[j]);
-                }
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) {
-                    if (g >= G) break;
-                    float dot = 0.f;
-#pragma unroll
-                    for (int j = 0; j < DPL; ++j) dot += qv[g][j] * kf[j];
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                    const float sc = dot * a.scale_log2;
-                    const float m_new = fmaxf(m_run[g], sc);
-                    const float corr = exp2f(m_run[g] - m_new), p = exp2f(sc - m_new);
-                    l_run[g] = l_run[g] * corr + p;
-                    m_run[g] = m_new;
-#pragma unroll
-                    for (int j = 0; j < DPL; ++j) acc[g][j] = acc[g][j] * corr + p * vf[j];
-                }
-            }
-        }
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-            if (lane == 0) {
-                stat_m[warp * kMaxGroup + g] = m_run[g];
-                stat_l[warp * kMaxGroup + g] = l_run[g];
-            }
-#pragma unroll
-            for (int j = 0; j < DPL; ++j)
-                merge[(warp * kMaxGroup + g) * S::kMergeStride + lane * DPL + j] = acc[g][j];
-        }
-        finalize_segment<D>(a, u, u.tile == 0 && seg_tiles == u.tiles, merge, stat_m, stat_l, &s_flag,
-                            tid, T, P);
-        x += seg_tiles;
-    }
+template <int D, int NG>
+cudaError_t prepare_one()
+{
+    return cudaFuncSetAttribute(decode_kernel<D, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                kMaxDynamicSmem);
 }
 
 }  // namespace
 
-size_t decode_smem_bytes(int head_dim, int stages)
+size_t decode_smem_bytes(int head_dim, int stages, int group, int groups)
 {
-    return head_dim == 128 ? Smem<128>::bytes(stages) : Smem<64>::bytes(stages);
+    if (head_dim == 128)
+        return groups == 1 ? Smem<128, 1>::bytes(stages, group)
+                           : groups == 2 ? Smem<128, 2>::bytes(stages, group) : Smem<128, 3>::bytes(stages, group);
+    return groups == 1 ? Smem<64, 1>::bytes(stages, group)
+                       : groups == 2 ? Smem<64, 2>::bytes(stages, group) : Smem<64, 3>::bytes(stages, group);
 }
 
-cudaError_t prepare_decode_kernels(int head_dim, int stages)
+cudaError_t prepare_decode_kernels(int head_dim)
 {
-    const int bytes = (int)decode_smem_bytes(head_dim, stages);
-    if (head_dim == 128)
-        return cudaFuncSetAttribute(decode_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    return cudaFuncSetAttribute(decode_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    cudaError_t e;
+    if (head_dim == 128) {
+        if ((e = prepare_one<128, 1>()) != cudaSuccess) return e;
+        if ((e = prepare_one<128, 2>()) != cudaSuccess) return e;
+        return prepare_one<128, 3>();
+    }
+    if ((e = prepare_one<64, 1>()) != cudaSuccess) return e;
+    if ((e = prepare_one<64, 2>()) != cudaSuccess) return e;
+    return prepare_one<64, 3>();
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, cudaStream_t stream)
+                          int stages, int groups, cudaStream_t stream)
 {
-    if (tmap == nullptr) {
-        if (head_dim == 128)
-            decode_kernel_plain<128><<<grid, kConsumerThreads, 0, stream>>>(a);
-        else
-            decode_kernel_plain<64><<<grid, kConsumerThreads, 0, stream>>>(a);
-        return cudaGetLastError();
+    if (head_dim == 128) {
+        if (groups == 1) return launch_one<128, 1>(a, *tmap, grid, stages, stream);
+        if (groups == 2) return launch_one<128, 2>(a, *tmap, grid, stages, stream);
+        return launch_one<128, 3>(a, *tmap, grid, stages, stream);
     }
-    const size_t smem = decode_smem_bytes(head_dim, stages);
-    if (head_dim == 128)
-        decode_kernel<128><<<grid, kThreads, smem, stream>>>(a, *tmap, stages);
-    else
-        decode_kernel<64><<<grid, kThreads, smem, stream>>>(a, *tmap, stages);
-    return cudaGetLastError();
+    if (groups == 1) return launch_one<64, 1>(a, *tmap, grid, stages, stream);
+    if (groups == 2) return launch_one<64, 2>(a, *tmap, grid, stages, stream);
+    return launch_one<64, 3>(a, *tmap, grid, stages, stream);
 }
 
 }  // namespace rlkv

@@ -22,10 +22,6 @@
 #include "../../include/rlkv.h"
 #include "rlkv_internal.cuh"
 
-namespace rlkv {
-cudaError_t prepare_decode_kernels(int head_dim, int stages);
-}
-
 using namespace rlkv;
 
 namespace {
@@ -114,6 +110,17 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     return RLKV_OK;
 }
 
+// Most pipeline stages (<= 8) that fit `ctas_per_sm` CTAs of the decode kernel on one SM
+// (228 KB per SM, 1 KB of it reserved per resident CTA).
+int max_stages(int head_dim, int group, int groups, int ctas_per_sm)
+{
+    for (int st = 8; st >= 2; --st) {
+        const size_t one = decode_smem_bytes(head_dim, st, group, groups);
+        if (one <= (size_t)kMaxDynamicSmem && (one + 1024) * ctas_per_sm <= 228u * 1024u) return st;
+    }
+    return 0;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -136,8 +143,7 @@ struct DeviceGuard {
 struct rlkv_cache {
     int layers, kv_heads, q_heads, head_dim, batch, max_len, sink, window;
     int device, sm_count;
-    int ctas_per_sm, stages;
-    bool plain;  // debugging cross-check kernel instead of the pipelined one
+    int ctas_per_sm, stages, groups;  // decode launch shape (rlkv_set_decode_config)
     Layout lay;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -168,14 +174,31 @@ int make_tensor_map(rlkv_cache* c)
     cudaDriverEntryPointQueryResult q;
     RLKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
     if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
-    const cuuint64_t dims[2] = {(cuuint64_t)c->head_dim, (cuuint64_t)c->lay.pool_rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)c->head_dim * 2};
-    const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
-        &c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c->dev_base + c->lay.off_pool, dims, strides, box, estr,
-        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    // The pool as rows of 128-byte pieces so that one box is one contiguous run of memory and still
+    // obeys the 128-byte limit of the swizzled inner dimension:
+    //   head_dim 128: [rows][2 halves][64]  box [64 rows][2][64]  (16 KB)
+    //   head_dim  64: [rows][64]            box [64 rows][64]     ( 8 KB)
+    CUresult r;
+    void* base = c->dev_base + c->lay.off_pool;
+    const CUtensorMapL2promotion l2p = getenv("RLKV_L2P") ? (CUtensorMapL2promotion)atoi(getenv("RLKV_L2P"))
+                                                          : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+    if (c->head_dim == 128) {
+        const cuuint64_t dims[3] = {64, 2, (cuuint64_t)c->lay.pool_rows};
+        const cuuint64_t strides[2] = {128, 256};
+        const cuuint32_t box[3] = {64, 2, (cuuint32_t)kTile};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        r = reinterpret_cast<EncodeTiledFn>(fn)(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box,
+                                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2p,
+                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+        const cuuint64_t dims[2] = {64, (cuuint64_t)c->lay.pool_rows};
+        const cuuint64_t strides[1] = {128};
+        const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
+        const cuuint32_t estr[2] = {1, 1};
+        r = reinterpret_cast<EncodeTiledFn>(fn)(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box,
+                                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2p,
+                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
     if (r != CUDA_SUCCESS) {
         snprintf(g_cuda_text, sizeof g_cuda_text, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
         return RLKV_ECUDA;
@@ -236,16 +259,20 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.q_heads = c->q_heads;
     a.tiles_full = (a.len_full + kTile - 1) / kTile;
     a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
-    const long long total =
-        (long long)c->batch * ((long long)a.n_full * a.tiles_full + (long long)a.n_comp * a.tiles_comp);
-    if (total >= (1ll << 31)) return RLKV_EINVAL;
-    a.total_tiles = (int)total;
+    const long long full_tiles = (long long)c->batch * a.n_full * a.tiles_full;
+    if (full_tiles >= (1ll << 31)) return RLKV_EINVAL;
+    a.full_tiles = (int)full_tiles;
+    a.comp_units = c->batch * a.n_comp;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
-    // every CTA must own at least one tile (the split bookkeeping assumes no empty ranges)
-    int grid = c->sm_count * (c->plain ? 2 : c->ctas_per_sm);
+    { const char* d = getenv("RLKV_DEBUG"); a.debug = d ? atoi(d) : 0; }
+    // persistent grid; no more CTAs than there is work, and every CTA that shares the full tiles
+    // owns at least one of them (the split bookkeeping assumes no empty ranges)
+    int grid = c->sm_count * c->ctas_per_sm;
     if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    if (grid > a.total_tiles) grid = a.total_tiles;
-    RLKV_CUDA(launch_decode(a, c->plain ? nullptr : &c->tmap, c->head_dim, grid, c->stages, s));
+    const int most_work = a.full_tiles > a.comp_units ? a.full_tiles : a.comp_units;
+    if (grid > most_work) grid = most_work;
+    a.grid_full = grid < a.full_tiles ? grid : a.full_tiles;
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
     c->launches++;
     return RLKV_OK;
 }
@@ -295,9 +322,8 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->batch = batch; c->max_len = max_len; c->sink = sink; c->window = window;
     c->dev_base = nullptr; c->owns_buffer = false; c->launches = 0;
     c->ctas_per_sm = 1;
-    c->stages = head_dim == 128 ? 6 : 8;
-    const char* plain = getenv("RLKV_DECODE_PLAIN");
-    c->plain = plain && plain[0] == '1';
+    c->groups = 2;
+    c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
     rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
     if (rc) { delete c; return rc; }
     c->is_full.assign(head_is_full, head_is_full + (size_t)layers * kv_heads);
@@ -354,7 +380,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaMemcpy(tables)"));
     rc = make_tensor_map(c);
     if (rc) return fail(rc);
-    e = prepare_decode_kernels(head_dim, c->stages);
+    e = prepare_decode_kernels(head_dim);
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaFuncSetAttribute"));
     e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceSynchronize"));
@@ -386,17 +412,19 @@ int rlkv_cache_reset(rlkv_cache* c, void* stream)
     return RLKV_OK;
 }
 
-int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages)
+int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consumer_groups)
 {
-    if (!c || ctas_per_sm < 0 || ctas_per_sm > 2 || stages < 0 || stages == 1 || stages > 8) return RLKV_EINVAL;
+    if (!c || ctas_per_sm < 0 || ctas_per_sm > 2 || stages < 0 || stages == 1 || stages > 8 ||
+        consumer_groups < 0 || consumer_groups > kMaxConsumerGroups)
+        return RLKV_EINVAL;
     const int cps = ctas_per_sm ? ctas_per_sm : c->ctas_per_sm;
-    const int st = stages ? stages : c->stages;
-    if (decode_smem_bytes(c->head_dim, st) * cps > 227u * 1024u) return RLKV_EINVAL;
-    DeviceGuard g(c->device);
-    if (!g.ok) return RLKV_ECUDA;
-    RLKV_CUDA(prepare_decode_kernels(c->head_dim, st));
+    const int ng = consumer_groups ? consumer_groups : c->groups;
+    const int most = max_stages(c->head_dim, c->q_heads / c->kv_heads, ng, cps);
+    const int st = stages ? stages : (c->stages < most ? c->stages : most);
+    if (most < 2 || st > most) return RLKV_EINVAL;
     c->ctas_per_sm = cps;
     c->stages = st;
+    c->groups = ng;
     return RLKV_OK;
 }
 

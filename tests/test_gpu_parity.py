@@ -3,8 +3,6 @@ seeded inputs.  Cache state is compared bit for bit; attention outputs within th
 (max abs error <= 1e-2, mean abs error <= 1e-3, plus max abs error <= 2e-2 * rms(out) per query
 head so the check keeps its teeth at long contexts where |out| ~ 0.02).
 """
-import os
-
 import numpy as np
 import pytest
 import torch
@@ -303,12 +301,12 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     feed(cache, oracle, 0, K, V, True)
     want = oracle.decode(0, q)
     outs = []
-    for cps, st in ((1, 6), (1, 2), (2, 2), (1, 4)):
-        rl.rlkv_set_decode_config(cache.handle, cps, st)
+    for cps, st, ng in ((1, 6, 1), (1, 2, 2), (2, 2, 1), (1, 4, 3), (2, 2, 2), (1, 5, 2), (1, 0, 3)):
+        rl.rlkv_set_decode_config(cache.handle, cps, st, ng)
         outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
         check_out(outs[-1], want)
     with pytest.raises(rl.RlkvError):
-        rl.rlkv_set_decode_config(cache.handle, 2, 6)       # does not fit in shared memory twice
+        rl.rlkv_set_decode_config(cache.handle, 2, 6, 1)    # does not fit in shared memory twice
     rl.rlkv_cache_reset(cache.handle)
     assert cache.length(0) == 0
     gk, gv, gt = cache.export_head(0, 0, 1)
@@ -318,16 +316,3 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     for t in range(100):
         o2.append(0, K[t], V[t])
     check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), o2.decode(0, q))
-
-
-def test_plain_variant_agrees(rl, hz, cuda_device):
-    """The debugging cross-check kernel (no TMA, no tensor cores) against the oracle."""
-    os.environ["RLKV_DECODE_PLAIN"] = "1"
-    try:
-        cache, oracle = build_pair(hz, 1, 4, 28, 128, 2, 1500, [1, 0, 0, 1], 16, 112, cuda_device)
-    finally:
-        del os.environ["RLKV_DECODE_PLAIN"]
-    K, V, q = rand_bf16((1500, 2, 4, 128), 1), rand_bf16((1500, 2, 4, 128), 2), rand_bf16((2, 28, 128), 3)
-    feed(cache, oracle, 0, K, V, True)
-    check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), oracle.decode(0, q))
-    assert cache.status() == 0
