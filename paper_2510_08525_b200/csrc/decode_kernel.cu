@@ -264,6 +264,8 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const CtaWork work = cta_work(a, blockIdx.x, gridDim.x);
+    const bool stamp = (a.debug & 4) != 0;
+    if (stamp && tid == 0) a.timeline[blockIdx.x * 4 + 0] = global_timer_ns();
 
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -349,6 +351,7 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                 }
                 if (!mine) continue;
                 wait_bounded(smem_u32(full_bar + cur_s), cur_par, s_abort, a.status, kStatusFullWaitTimeout);
+                if (stamp && tid == 0 && v == 0 && i == 0) a.timeline[blockIdx.x * 4 + 1] = global_timer_ns();
                 const int valid = min(kTile, valid_left);
                 if (wig * 16 < valid && !(a.debug & 1)) {
                     const uint32_t sK = smem_u32(stage_base + (size_t)cur_s * S::kStageBytes);
@@ -437,12 +440,14 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                     }
                 }
             }
+            if (stamp && tid == 0 && v + seg_tiles == work.total) a.timeline[blockIdx.x * 4 + 2] = global_timer_ns();
             finalize_segment<D, NG>(a, u, u.tile == 0 && seg_tiles == u.tiles, merge, stat_m, stat_l,
                                     s_flag, tid);
             v += seg_tiles;
         }
     }
     __syncthreads();
+    if (stamp && tid == 0) a.timeline[blockIdx.x * 4 + 3] = global_timer_ns();
     if (warp == S::kWarps && lane == 0 && *s_abort) {
         // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
         // when the CTA retires

@@ -48,7 +48,7 @@ struct Layout {
     std::vector<long long> full_row0, comp_row0;  // per layer, in pool rows
     long long pool_rows = 0;
     size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
-    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, total = 0;
+    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_timeline = 0, total = 0;
     int max_grid = 0;
 };
 
@@ -106,15 +106,21 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     off = align_up(off + q_step, 1024);
     L.off_out = off;
     off = align_up(off + q_step * 2, 1024);
+    L.off_timeline = off;
+    off = align_up(off + (size_t)L.max_grid * 4 * sizeof(unsigned long long), 1024);
     L.total = off;
     return RLKV_OK;
 }
 
 // Most pipeline stages (<= 8) that fit `ctas_per_sm` CTAs of the decode kernel on one SM
-// (228 KB per SM, 1 KB of it reserved per resident CTA).
+// (228 KB per SM, 1 KB of it reserved per resident CTA).  The stage count is a multiple of the
+// number of consumer groups, so that a given stage is always consumed by the same group: an
+// mbarrier parity wait can only tell two phases apart, and a group that reached a stage a whole
+// phase early would take the wait for the phase before as satisfied.
 int max_stages(int head_dim, int group, int groups, int ctas_per_sm)
 {
     for (int st = 8; st >= 2; --st) {
+        if (st % groups != 0) continue;
         const size_t one = decode_smem_bytes(head_dim, st, group, groups);
         if (one <= (size_t)kMaxDynamicSmem && (one + 1024) * ctas_per_sm <= 228u * 1024u) return st;
     }
@@ -248,6 +254,7 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.partials = dev_at<float>(c, c->lay.off_partials);
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
     a.status = dev_at<int>(c, c->lay.off_status);
+    a.timeline = dev_at<unsigned long long>(c, c->lay.off_timeline);
     a.n_full = c->lay.n_full[layer];
     a.n_comp = c->lay.n_comp[layer];
     a.rows_full = c->lay.rows_full;
@@ -420,8 +427,9 @@ int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consu
     const int cps = ctas_per_sm ? ctas_per_sm : c->ctas_per_sm;
     const int ng = consumer_groups ? consumer_groups : c->groups;
     const int most = max_stages(c->head_dim, c->q_heads / c->kv_heads, ng, cps);
-    const int st = stages ? stages : (c->stages < most ? c->stages : most);
-    if (most < 2 || st > most) return RLKV_EINVAL;
+    int st = stages ? stages : (c->stages < most ? c->stages : most);
+    if (!stages) st -= st % ng;
+    if (most < 2 || st < 2 || st > most || st % ng != 0) return RLKV_EINVAL;
     c->ctas_per_sm = cps;
     c->stages = st;
     c->groups = ng;
@@ -562,6 +570,17 @@ int rlkv_kernel_status(rlkv_cache* c, int* status_out)
     RLKV_CUDA(cudaDeviceSynchronize());
     RLKV_CUDA(cudaMemcpy(status_out, c->dev_base + c->lay.off_status, sizeof(int), cudaMemcpyDeviceToHost));
     return *status_out == 0 ? RLKV_OK : RLKV_EKERNEL;
+}
+
+int rlkv_debug_timeline(rlkv_cache* c, unsigned long long* host_out, int* ctas_out)
+{
+    if (!c || !host_out || !ctas_out) return RLKV_EINVAL;
+    DeviceGuard g(c->device);
+    RLKV_CUDA(cudaDeviceSynchronize());
+    RLKV_CUDA(cudaMemcpy(host_out, c->dev_base + c->lay.off_timeline, (size_t)c->lay.max_grid * 4 * 8,
+                         cudaMemcpyDeviceToHost));
+    *ctas_out = c->lay.max_grid;
+    return RLKV_OK;
 }
 
 int rlkv_launch_count(const rlkv_cache* c, uint64_t* launches_out)

@@ -40,6 +40,7 @@ struct DecodeArgs {
     float* partials;            // [grid][2][partial_floats]
     int* tickets;               // [batch*n_full] for this layer, zero between launches
     int* status;                // device error word
+    unsigned long long* timeline;  // debug: [grid][4] globaltimer stamps
     int n_full, n_comp;         // heads of each class in this layer
     int rows_full, rows_comp;   // allocated rows per head (multiples of kTile)
     int len_full, len_comp;     // valid rows per head right now: n and min(n, sink+window)

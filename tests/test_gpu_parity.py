@@ -301,12 +301,15 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     feed(cache, oracle, 0, K, V, True)
     want = oracle.decode(0, q)
     outs = []
-    for cps, st, ng in ((1, 6, 1), (1, 2, 2), (2, 2, 1), (1, 4, 3), (2, 2, 2), (1, 5, 2), (1, 0, 3)):
+    for cps, st, ng in ((1, 6, 1), (1, 2, 2), (2, 2, 1), (1, 3, 3), (2, 2, 2), (1, 4, 2), (1, 0, 3), (1, 5, 1)):
         rl.rlkv_set_decode_config(cache.handle, cps, st, ng)
         outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
         check_out(outs[-1], want)
-    with pytest.raises(rl.RlkvError):
-        rl.rlkv_set_decode_config(cache.handle, 2, 6, 1)    # does not fit in shared memory twice
+    for bad in ((2, 6, 1),      # does not fit in shared memory twice
+                (1, 5, 2), (1, 4, 3)):   # stages must be a multiple of the consumer groups
+        with pytest.raises(rl.RlkvError) as e:
+            rl.rlkv_set_decode_config(cache.handle, *bad)
+        assert e.value.code == rl.RLKV_EINVAL
     rl.rlkv_cache_reset(cache.handle)
     assert cache.length(0) == 0
     gk, gv, gt = cache.export_head(0, 0, 1)
