@@ -353,7 +353,7 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
                 wait_bounded(smem_u32(full_bar + cur_s), cur_par, s_abort, a.status, kStatusFullWaitTimeout);
                 if (stamp && tid == 0 && v == 0 && i == 0) a.timeline[blockIdx.x * 4 + 1] = global_timer_ns();
                 const int valid = min(kTile, valid_left);
-                if (wig * 16 < valid && !(a.debug & 1)) {
+                if (wig * 16 < valid) {
                     const uint32_t sK = smem_u32(stage_base + (size_t)cur_s * S::kStageBytes);
                     const uint32_t sV = sK + S::kTileBytes;
                     // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
