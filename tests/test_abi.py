@@ -1,0 +1,100 @@
+"""The C-ABI boundary without a GPU: librlkv.so loads, exports every function include/rlkv.h
+declares, the Python binding has one function of the same name for each, and the host-side argument
+checks that need no device answer with the documented codes."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "rlkv.h")
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(rlkv_[a-z0-9_]+)\s*\(", text)
+    return sorted(set(names))
+
+
+@pytest.fixture(scope="module")
+def binding():
+    from paper_2510_08525_b200 import build
+    build.build()
+    import paper_2510_08525_b200.binding as b
+    return b
+
+
+def test_header_declares_the_three_calls_of_the_problem_statement():
+    names = declared_functions()
+    for must in ("rlkv_cache_create", "rlkv_append", "rlkv_decode_attention"):
+        assert must in names
+    assert len(names) >= 10
+
+
+def test_library_exports_every_declared_symbol(binding):
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared_functions():
+        assert hasattr(lib, name), f"librlkv.so does not export {name}"
+
+
+def test_binding_has_the_same_names(binding):
+    for name in declared_functions():
+        assert callable(getattr(binding, name)), name
+        assert name in binding.SIGNATURES
+    assert sorted(binding.SIGNATURES) == declared_functions()
+
+
+def test_error_codes_match_the_header(binding):
+    text = open(HEADER).read()
+    for name, value in re.findall(r"(RLKV_[A-Z]+)\s*=\s*(-?\d+)", text):
+        assert getattr(binding, name) == int(value)
+        assert binding.rlkv_strerror(int(value))
+    assert binding.rlkv_strerror(-99) == "unknown error"
+
+
+def test_host_side_argument_checks_need_no_device(binding):
+    ok = dict(layers=2, kv_heads=2, q_heads=8, head_dim=128, batch=3, max_len=100,
+              head_is_full=[1, 0, 0, 1], sink=4, window=12)
+    size = binding.rlkv_cache_size(**ok)
+    # two full heads of 128 rows (100 rounded up to the tile) and two compressed heads of 64 rows,
+    # K and V, per batch row
+    pool = 3 * (2 * 128 + 2 * 64) * 2 * 128 * 2
+    assert size >= pool
+    # compressed heads cost the same however long the sequence may grow
+    longer = binding.rlkv_cache_size(**{**ok, "max_len": 100 + 64 * 10})
+    assert longer - size == 3 * 2 * 640 * 2 * 128 * 2
+    for bad in (dict(head_dim=96), dict(q_heads=7), dict(q_heads=18), dict(window=0), dict(sink=-1),
+                dict(batch=0), dict(max_len=0)):
+        with pytest.raises(binding.RlkvError) as e:
+            binding.rlkv_cache_size(**{**ok, **bad})
+        assert e.value.code == binding.RLKV_EINVAL
+    with pytest.raises(ValueError):
+        binding.rlkv_cache_size(**{**ok, "head_is_full": [1, 0, 0]})
+    m = np.ones(4, np.uint8)
+    out = ctypes.c_size_t(0)
+    assert binding.lib.rlkv_cache_size(0, 2, 8, 128, 3, 100, m.ctypes.data, 4, 12, ctypes.byref(out)) == binding.RLKV_EINVAL
+    assert binding.lib.rlkv_cache_size(2, 2, 8, 128, 3, 100, None, 4, 12, ctypes.byref(out)) == binding.RLKV_EINVAL
+    assert binding.lib.rlkv_cache_size(2, 2, 8, 128, 3, 100, m.ctypes.data, 4, 12, None) == binding.RLKV_EINVAL
+    # null handles are refused, not dereferenced
+    for call in (lambda: binding.rlkv_length(0, 0), lambda: binding.rlkv_step_bytes(0, 0),
+                 lambda: binding.rlkv_launch_count(0), lambda: binding.rlkv_cache_destroy(0)):
+        with pytest.raises(binding.RlkvError) as e:
+            call()
+        assert e.value.code == binding.RLKV_EINVAL
+
+
+def test_package_fails_loudly_without_the_library(tmp_path):
+    """A copy of the package without librlkv.so must raise on first use: there is no fallback."""
+    import shutil
+    import subprocess
+    import sys
+    pkg = tmp_path / "paper_2510_08525_b200"
+    shutil.copytree(os.path.join(ROOT, "paper_2510_08525_b200"), pkg,
+                    ignore=shutil.ignore_patterns("*.so", "__pycache__"))
+    code = ("import paper_2510_08525_b200 as p\n"
+            "try:\n    p.rlkv_cache_size\nexcept ImportError as e:\n    print('IMPORTERROR', 'no fallback' in str(e))\n")
+    res = subprocess.run([sys.executable, "-c", code], cwd=tmp_path, capture_output=True, text=True)
+    assert "IMPORTERROR True" in res.stdout, res.stdout + res.stderr
