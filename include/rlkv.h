@@ -45,7 +45,8 @@ enum {
     RLKV_EEMPTY = -3, /* decode on a layer that holds no token */
     RLKV_ENOMEM = -4, /* host or device allocation failed, or device_buf too small */
     RLKV_ECUDA = -5,  /* a CUDA call failed; rlkv_strerror(RLKV_ECUDA) carries the CUDA text */
-    RLKV_EKERNEL = -6 /* a kernel gave up on a bounded wait (see rlkv_kernel_status) */
+    RLKV_EKERNEL = -6, /* a kernel gave up on a bounded wait (see rlkv_kernel_status) */
+    RLKV_ESCRATCH = -7 /* rlkv_decode_attention_static_scratch: the static scratch array is too small */
 };
 
 /* Bytes of device memory a cache of this shape needs (pools, index tables, split scratch and the
@@ -86,6 +87,35 @@ int rlkv_prefill(rlkv_cache* cache, int layer, const void* k, const void* v, int
  * q: device bf16 [batch][q_heads][head_dim]; out: device fp32 [batch][q_heads][head_dim].
  * Scores, softmax and accumulation are fp32.  RLKV_EEMPTY if length(layer) == 0. */
 int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out, void* stream);
+
+/* rlkv_decode_attention for callers that must not allocate device memory.  (The paper has no
+ * counterpart: this entry point exists for the integration, not for the method.)
+ *
+ * Who needs it: a host that has handed all device memory to its own pool before this library is
+ * called -- a serving engine that sizes its KV pool to whatever cudaMalloc still grants at
+ * start-up, a plugin running under a framework whose allocator owns the device, code running
+ * where cudaMalloc is forbidden because it would synchronise the device in the middle of a step.
+ * Such a host can give rlkv_cache_create a slice of its pool for the K/V rows, but may not want
+ * the kernel's split-KV work area (tickets and partial results, rewritten by every launch) to
+ * live there.  This call computes exactly what rlkv_decode_attention computes, with the same
+ * kernel, and keeps that work area in an array that is part of the library image instead:
+ * rlkv_static_scratch_bytes() bytes (2 MiB) of device memory on every GPU that loads librlkv,
+ * held until the process exits.  The call itself allocates and frees nothing.
+ *
+ * - A launch that needs more than the array holds (batch * kv_heads tickets plus two partial
+ *   records of 8 * (head_dim + 2) floats per CTA; 2 CTAs per SM at head_dim 128 do not fit) is
+ *   refused with RLKV_ESCRATCH and nothing is launched.
+ * - The first call on a device looks up the array's device address (one runtime query, kept for
+ *   the life of the process; a driver that loads modules lazily gives the array its memory at that
+ *   moment); make that first call at start-up, before starting any stream capture.
+ * - Every cache and every call on a device share the one array, which still holds the previous
+ *   call's contents: each call clears the tickets on `stream` before its launch.  Two such calls
+ *   that overlap on the GPU (different streams, no ordering between them) race on the array and
+ *   give wrong results; order them, or use rlkv_decode_attention for one of them.
+ * Arguments, layouts and the other error codes are those of rlkv_decode_attention. */
+int rlkv_decode_attention_static_scratch(rlkv_cache* cache, int layer, const void* q, void* out,
+                                         void* stream);
+size_t rlkv_static_scratch_bytes(void);
 
 /* One whole decode step: for every layer, append then attend.  Device buffers:
  * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];

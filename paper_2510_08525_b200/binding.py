@@ -17,6 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "librlkv.so")
 
 RLKV_OK, RLKV_EINVAL, RLKV_EFULL, RLKV_EEMPTY, RLKV_ENOMEM, RLKV_ECUDA, RLKV_EKERNEL = 0, -1, -2, -3, -4, -5, -6
+RLKV_ESCRATCH = -7
 
 # name -> (restype, argtypes); one entry per symbol declared in include/rlkv.h
 _vp, _ci, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
@@ -28,6 +29,8 @@ SIGNATURES = {
     "rlkv_append": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_prefill": (_ci, [_vp, _ci, _vp, _vp, _ci, _vp]),
     "rlkv_decode_attention": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_decode_attention_static_scratch": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_static_scratch_bytes": (_sz, []),
     "rlkv_step": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_step_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_length": (_ci, [_vp, _ci, ctypes.POINTER(_ci)]),
@@ -134,6 +137,16 @@ def rlkv_prefill(cache, layer, k, v, n_tokens, stream=None) -> None:
 
 def rlkv_decode_attention(cache, layer, q, out, stream=None) -> None:
     _check(lib.rlkv_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_decode_attention_static_scratch(cache, layer, q, out, stream=None) -> None:
+    """rlkv_decode_attention with the kernel's work area in the library's static device array;
+    the call allocates nothing (see include/rlkv.h for who needs that and for the limits)."""
+    _check(lib.rlkv_decode_attention_static_scratch(cache, layer, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_static_scratch_bytes() -> int:
+    return int(lib.rlkv_static_scratch_bytes())
 
 
 def rlkv_step(cache, k, v, q, out, stream=None) -> None:

@@ -284,6 +284,85 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     return RLKV_OK;
 }
 
+// ---- split-KV scratch that nobody allocates -------------------------------------------------------
+// rlkv_decode_attention_static_scratch keeps the decode kernel's split bookkeeping (tickets) and
+// partial results here instead of in the cache's own buffer.  The array is part of the library
+// image: every GPU that loads librlkv holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = 2u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_scratch_dev[kMaxDevices] = {};  // device address of the array, per device
+
+// Device address of g_static_scratch on `device`, which must be current.  In host code the array's
+// name is only a handle for the runtime, never a pointer a kernel may use: the address has to be
+// asked for, once per device.
+int static_scratch_address(int device, unsigned char** out)
+{
+    if (device < 0 || device >= kMaxDevices) return RLKV_EINVAL;
+    if (!g_static_scratch_dev[device]) {
+        void* p = nullptr;
+        RLKV_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        if (!p) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_static_scratch)");
+        g_static_scratch_dev[device] = static_cast<unsigned char*>(p);
+    }
+    *out = g_static_scratch_dev[device];
+    return RLKV_OK;
+}
+
+// The launch of do_decode with the tickets and partials placed in the static array.
+int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
+{
+    const int n = c->len[layer];
+    const int cap = c->sink + c->window;
+    DecodeArgs a;
+    a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+    a.full_row0 = c->lay.full_row0[layer];
+    a.comp_row0 = c->lay.comp_row0[layer];
+    a.head_of_slot = dev_at<int>(c, c->lay.off_tables) + (size_t)(c->layers + layer) * c->kv_heads;
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.out = static_cast<float*>(out);
+    a.status = dev_at<int>(c, c->lay.off_status);
+    a.timeline = dev_at<unsigned long long>(c, c->lay.off_timeline);
+    a.n_full = c->lay.n_full[layer];
+    a.n_comp = c->lay.n_comp[layer];
+    a.rows_full = c->lay.rows_full;
+    a.rows_comp = c->lay.rows_comp;
+    a.len_full = n;
+    a.len_comp = n < cap ? n : cap;
+    a.batch = c->batch;
+    a.group = c->q_heads / c->kv_heads;
+    a.q_heads = c->q_heads;
+    a.tiles_full = (a.len_full + kTile - 1) / kTile;
+    a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
+    const long long full_tiles = (long long)c->batch * a.n_full * a.tiles_full;
+    if (full_tiles >= (1ll << 31)) return RLKV_EINVAL;
+    a.full_tiles = (int)full_tiles;
+    a.comp_units = c->batch * a.n_comp;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
+    a.debug = 0;
+    int grid = c->sm_count * c->ctas_per_sm;
+    if (grid > c->lay.max_grid) grid = c->lay.max_grid;
+    const int most_work = a.full_tiles > a.comp_units ? a.full_tiles : a.comp_units;
+    if (grid > most_work) grid = most_work;
+    a.grid_full = grid < a.full_tiles ? grid : a.full_tiles;
+
+    // carve the static array: one ticket per (batch row, KV head), then two partial records per CTA
+    const size_t ticket_bytes = align_up((size_t)c->batch * c->kv_heads * sizeof(int), 256);
+    const size_t partial_bytes = (size_t)grid * 2 * partial_floats(c->head_dim) * sizeof(float);
+    if (ticket_bytes + partial_bytes > kStaticScratchBytes) return RLKV_ESCRATCH;
+    unsigned char* base = nullptr;
+    int rc = static_scratch_address(c->device, &base);
+    if (rc) return rc;
+    a.tickets = reinterpret_cast<int*>(base);
+    a.partials = reinterpret_cast<float*>(base + ticket_bytes);
+    // the array still holds whatever the previous call (of any cache) left: tickets must start at 0
+    RLKV_CUDA(cudaMemsetAsync(base, 0, ticket_bytes, s));
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
+    c->launches++;
+    return RLKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -298,6 +377,7 @@ const char* rlkv_strerror(int code)
         case RLKV_ENOMEM: return "out of memory or buffer too small";
         case RLKV_ECUDA: return g_cuda_text[0] ? g_cuda_text : "CUDA error";
         case RLKV_EKERNEL: return "a kernel gave up on a bounded wait";
+        case RLKV_ESCRATCH: return "the launch needs more scratch than the library's static array holds";
         default: return "unknown error";
     }
 }
@@ -458,6 +538,17 @@ int rlkv_decode_attention(rlkv_cache* c, int layer, const void* q, void* out, vo
     if (!g.ok) return RLKV_ECUDA;
     return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream));
 }
+
+int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (c->len[layer] < 1) return RLKV_EEMPTY;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_decode_static_scratch(c, layer, q, out, static_cast<cudaStream_t>(stream));
+}
+
+size_t rlkv_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
 int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* out, void* stream)
 {
