@@ -99,17 +99,18 @@ int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out
  * the kernel's split-KV work area (tickets and partial results, rewritten by every launch) to
  * live there.  This call computes exactly what rlkv_decode_attention computes, with the same
  * kernel, and keeps that work area in an array that is part of the library image instead:
- * rlkv_static_scratch_bytes() bytes (2 MiB) of device memory on every GPU that loads librlkv,
+ * rlkv_static_scratch_bytes() bytes (4 MiB) of device memory on every GPU that loads librlkv,
  * held until the process exits.  The call itself allocates and frees nothing.
  *
  * - A launch that needs more than the array holds (batch * kv_heads tickets plus two partial
- *   records of 8 * (head_dim + 2) floats per CTA; 2 CTAs per SM at head_dim 128 do not fit) is
- *   refused with RLKV_ESCRATCH and nothing is launched.
+ *   records of about (q_heads / kv_heads) * (head_dim + 2) floats per work item of the launch;
+ *   rlkv_debug_schedule tells how many items a launch has) is refused with RLKV_ESCRATCH and
+ *   nothing is launched.  The benchmark shapes (about 900 items of 2 KiB records) fit.
  * - The first call on a device looks up the array's device address (one runtime query, kept for
  *   the life of the process; a driver that loads modules lazily gives the array its memory at that
  *   moment); make that first call at start-up, before starting any stream capture.
  * - Every cache and every call on a device share the one array, which still holds the previous
- *   call's contents: each call clears the tickets on `stream` before its launch.  Two such calls
+ *   call's contents: each call clears the tickets and work-claim counters on `stream` before its launch.  Two such calls
  *   that overlap on the GPU (different streams, no ordering between them) race on the array and
  *   give wrong results; order them, or use rlkv_decode_attention for one of them.
  * Arguments, layouts and the other error codes are those of rlkv_decode_attention. */
@@ -147,11 +148,28 @@ int rlkv_debug_export_head(rlkv_cache* cache, int layer, int batch_row, int kv_h
 int rlkv_kernel_status(rlkv_cache* cache, int* status_out);
 /* Number of kernels this cache has launched so far. */
 int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
-/* Tuning knobs of the decode kernel: persistent CTAs per SM (1 or 2), TMA pipeline stages (2..8)
- * and groups of four consumer warps that take tiles in turn (1..3).  0 keeps the current value
- * (stages: lowered if the new shape no longer fits).  RLKV_EINVAL if the shape does not fit in
- * shared memory.  Defaults: 1 CTA per SM, 2 groups, as many stages as fit. */
-int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups);
+/* Tuning knobs of the decode kernel: persistent CTAs per SM (1 or 2), TMA pipeline stages (2..8, a
+ * multiple of the consumer groups), groups of four consumer warps that take tiles in turn (1..3),
+ * and the size in 64-row tiles of the smallest work items the K/V scan is cut into (2..1024).
+ * 0 keeps the current value (stages: lowered if the new shape no longer fits).  RLKV_EINVAL if the
+ * shape does not fit in shared memory.  Defaults: 1 CTA per SM, 2 groups, as many stages as fit,
+ * 4 tiles.  Results do not depend on these knobs beyond floating-point summation order. */
+int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups,
+                           int item_tiles);
+/* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, eight
+ * 64-bit words: %globaltimer (ns) at CTA start, when its first tile landed, when its last segment
+ * was handed off and at CTA end; the work items, tiles and partial segments it processed; and
+ * %globaltimer when its epilogue warps finished.  words_host != NULL: first synchronises the
+ * device and copies the words of the most recent launch to words_host (host, 8 * 320 words) and
+ * the CTA capacity (320) to *ctas_out; then the switch is applied. */
+int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_host, int* ctas_out);
+/* The work schedule of the decode kernel, host arithmetic only (no GPU): a flat space of `tiles`
+ * tiles is cut for `ctas` CTAs into *n_items_out contiguous items whose sizes shrink geometrically
+ * down to item_tiles.  starts_out (host, optional, starts_cap >= n_items + 1 ints) receives the
+ * first tile of every item and, last, `tiles`.  RLKV_EKERNEL if the schedule's tile->item map
+ * disagrees with the starts (a self-check; never expected). */
+int rlkv_debug_schedule(int tiles, int ctas, int item_tiles, int* n_items_out, int* starts_out,
+                        int starts_cap);
 
 const char* rlkv_strerror(int code);
 

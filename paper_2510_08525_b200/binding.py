@@ -38,7 +38,9 @@ SIGNATURES = {
     "rlkv_debug_export_head": (_ci, [_vp, _ci, _ci, _ci, _vp, _vp, ctypes.POINTER(_ci), _vp]),
     "rlkv_kernel_status": (_ci, [_vp, ctypes.POINTER(_ci)]),
     "rlkv_launch_count": (_ci, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
-    "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci]),
+    "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci, _ci]),
+    "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
+    "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, ctypes.POINTER(_ci), _vp, _ci]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
 }
 
@@ -197,8 +199,26 @@ def rlkv_launch_count(cache) -> int:
     return int(out.value)
 
 
-def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0, consumer_groups=0) -> None:
-    _check(lib.rlkv_set_decode_config(cache, ctas_per_sm, stages, consumer_groups))
+def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0, consumer_groups=0, item_tiles=0) -> None:
+    _check(lib.rlkv_set_decode_config(cache, ctas_per_sm, stages, consumer_groups, item_tiles))
+
+
+def rlkv_debug_trace(cache, enable, read=False):
+    """Switches the decode kernel's trace on or off; with read=True returns uint64[320][8] of the
+    most recent launch (taken before the switch is applied)."""
+    words = np.zeros((320, 8), dtype=np.uint64) if read else None
+    ctas = _ci(0)
+    _check(lib.rlkv_debug_trace(cache, int(enable), _ptr(words), ctypes.byref(ctas)))
+    return words
+
+
+def rlkv_debug_schedule(tiles, ctas, item_tiles):
+    """int32[n_items + 1]: first tile of every work item, then `tiles`."""
+    n = _ci(0)
+    _check(lib.rlkv_debug_schedule(tiles, ctas, item_tiles, ctypes.byref(n), None, 0))
+    starts = np.empty(n.value + 1, dtype=np.int32)
+    _check(lib.rlkv_debug_schedule(tiles, ctas, item_tiles, ctypes.byref(n), starts.ctypes.data, starts.size))
+    return starts
 
 
 def rlkv_strerror(code: int) -> str:

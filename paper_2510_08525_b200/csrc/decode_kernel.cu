@@ -6,17 +6,20 @@
 // (the fused heterogeneous-head kernel Section 4.3 asks for).
 //
 // How: the K/V rows to read are cut into 64-token tiles and laid out as one flat tile space (full
-// units first, compressed units after).  A persistent grid splits that space evenly: CTA c owns the
-// contiguous range [c*T/P, (c+1)*T/P), so long full-head scans and short compressed-head scans
-// balance to within one tile.  Inside a CTA one producer warp streams tiles HBM -> shared memory
+// units first, compressed units after).  The space is cut into contiguous work items whose size
+// shrinks geometrically; a persistent grid takes item c for CTA c and claims further items from an
+// atomic counter, so long full-head scans and short compressed-head scans balance even though some
+// SMs sit on a slower path to memory than others.  Inside a CTA one producer warp streams tiles HBM -> shared memory
 // with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier pipeline); NG groups of four consumer
 // warps take the tiles in turn, each warp 16 tokens of its group's tile: S = Q.K^T and
 // O^T += V^T.P^T run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G query heads of the
 // group as the M (resp. N) dimension, online softmax in fp32 with warp shuffles.  The path is
 // HBM-bound (the tensor-core work is ~G flop per byte); several groups are there only to hide the
 // dependent-issue latency of one tile's softmax chain behind another tile's.
-// When a CTA's range ends inside a unit it writes an (m, l, O) partial; the last CTA to finish a
-// unit (atomic ticket, no spinning) merges the partials with the log-sum-exp rule and writes out.
+// When an item begins or ends inside a unit the CTA writes an (m, l, O) partial; the last CTA to
+// deliver a partial of a unit (atomic ticket, no spinning) merges them with the log-sum-exp rule.
+// Those merges, and the merge of the consumer warps' own states at the end of every segment, run
+// on separate epilogue warps, so the tile stream never waits for a round trip to global memory.
 #include "rlkv_internal.cuh"
 
 namespace rlkv {
@@ -86,10 +89,25 @@ __device__ __forceinline__ uint32_t swizzled_chunk(int row, int chunk)
     if (D == 128) return (uint32_t)(((chunk & 8) | ((chunk & 7) ^ ((2 * row + (chunk >> 3)) & 7))) << 4);
     return (uint32_t)((chunk ^ (row & 7)) << 4);
 }
-template <int NG>
-__device__ __forceinline__ void consumer_sync()
+// Barrier over the epilogue warps (named barrier 2).
+__device__ __forceinline__ void epilogue_sync()
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(NG * kGroupWarps * 32) : "memory");
+    asm volatile("bar.sync 2, %0;" ::"n"(kEpilogueWarps * 32) : "memory");
+}
+// The same barrier, also ORing a flag: every epilogue thread learns whether any of them gave up on
+// a wait, so that they all leave together and the named barrier is never left short.
+__device__ __forceinline__ bool epilogue_or(bool flag)
+{
+    uint32_t any;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 2, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(any)
+        : "r"((uint32_t)flag), "n"(kEpilogueWarps * 32)
+        : "memory");
+    return any != 0;
 }
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
                                             uint32_t& r3)
@@ -120,17 +138,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Wait on an mbarrier phase with a time limit (about one second).  When the limit runs out the
-// kernel records `code` in the status word and raises the CTA-wide abort flag; every later wait
-// then returns at once, so the CTA runs to its end (with meaningless results) instead of hanging.
-__device__ __forceinline__ void wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+// Wait on an mbarrier phase with a time limit (about one second).  Returns true when the phase
+// completed.  When the limit runs out the kernel records `code` in the status word, raises the
+// CTA-wide abort flag and returns false; every later abortable wait of the CTA then gives up at
+// once, so the CTA winds down (with meaningless results) instead of hanging.
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                              int* status, int code, bool abortable = true)
 {
     uint64_t t0 = 0;
     for (uint32_t i = 0;; ++i) {
-        if (mbar_try_wait(bar, parity)) return;
+        if (mbar_try_wait(bar, parity)) return true;
         if (i < 128) continue;
-        if (abortable && *abort_flag) return;
+        if (abortable && *abort_flag) return false;
         __nanosleep(64);
         const uint64_t now = global_timer_ns();
         if (t0 == 0) {
@@ -138,175 +157,133 @@ __device__ __forceinline__ void wait_bounded(uint32_t bar, uint32_t parity, vola
         } else if (now - t0 > 1000000000ull) {
             atomicCAS(status, kStatusOk, code);
             *abort_flag = 1;
-            return;
+            return false;
         }
     }
 }
 
 // ---------------------------------------------------------------------------------------------
+// What the consumer warps tell the epilogue warps about a finished segment (the part of one unit
+// inside one work item).
+struct SegDesc {
+    int out_row;     // first row of the unit's G output rows: b*q_heads + head*G
+    int uid;         // ticket index of the unit
+    int complete;    // the segment is the whole unit: normalise and write out
+    int item, slot;  // where the partial goes otherwise
+    int first_tile;  // flat tile range of the unit
+    int tiles;
+    int stop;        // no more segments: the epilogue warps leave
+};
+
 // Shared-memory carve-up (dynamic shared memory, base aligned to 1024 bytes for the swizzle).
 template <int D, int NG>
 struct Smem {
     static constexpr int kWarps = NG * kGroupWarps;         // consumer warps
+    static constexpr int kThreads = (kWarps + 2 + kEpilogueWarps) * 32;
     static constexpr int kTileBytes = kTile * D * 2;        // one K (or V) tile
     static constexpr int kStageBytes = 2 * kTileBytes;      // K tile then V tile
     static constexpr int kMergeStride = D + kMergePad;      // floats per head row
     static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
+    static constexpr int kBarriers = 2 * 8 + 2 * kItemRing + 2 + 2 * kMergeBuffers;
     __host__ __device__ static constexpr int merge_floats(int group) { return kWarps * group * kMergeStride; }
+    // one hand-off buffer: merge rows, per-warp max and sum, segment descriptor
+    __host__ __device__ static constexpr int buffer_bytes(int group)
+    {
+        return merge_floats(group) * 4 + kStatFloats * 4 + 32;
+    }
     __host__ __device__ static constexpr size_t bytes(int stages, int group)
     {
-        return 1024 /*alignment slack*/ + (size_t)stages * kStageBytes + merge_floats(group) * 4 +
-               kStatFloats * 4 + 2 * 8 * 8 /*barriers*/ + 16 /*flags*/;
+        return (size_t)stages * kStageBytes + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
+               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/;
     }
 };
 
-// ---------------------------------------------------------------------------------------------
-// End of a segment (the part of one unit a CTA processed).  Input: each consumer warp has put its
-// running max / sum / un-normalised output into the merge area.  The consumer threads merge the
-// warps; a complete unit is normalised and written out, otherwise the partial goes to the scratch
-// buffer and the last CTA to arrive for that unit merges all partials of the unit.
-template <int D, int NG>
-__device__ void finalize_segment(const DecodeArgs& a, const UnitInfo& u, bool complete,
-                                 const float* merge, const float* stat_m, const float* stat_l,
-                                 int* s_flag, int ctid)
+// Pool rows of the K and V tile behind flat tile x.
+__device__ __forceinline__ void tile_rows(const DecodeArgs& a, int x, int& krow, int& vrow)
 {
-    const int T = a.full_tiles, P = a.grid_full;  // the split space of the full units
-    using S = Smem<D, NG>;
-    constexpr int MS = S::kMergeStride;
-    constexpr int PF = partial_floats(D);
-    constexpr int NT = S::kWarps * 32;
-    const int G = a.group;
-    consumer_sync<NG>();  // merge area written by all warps
-
-    const int cta = blockIdx.x;
-    const int my_slot = (complete || cta_start(cta, T, P) >= u.first_tile) ? 0 : 1;
-    float* my_part = a.partials + ((size_t)cta * 2 + my_slot) * PF;
-    float* out_rows = a.out + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
-
-    for (int idx = ctid; idx < G * D; idx += NT) {
-        const int g = idx / D, d = idx - g * D;
-        float M = kNegBig, L = 0.f, O = 0.f;
-#pragma unroll
-        for (int w = 0; w < S::kWarps; ++w) {
-            const float mw = stat_m[w * kMaxGroup + g];
-            const float lw = stat_l[w * kMaxGroup + g];
-            const float ow = merge[(w * G + g) * MS + d];
-            const float Mn = fmaxf(M, mw);
-            const float ca = exp2f(M - Mn), cb = exp2f(mw - Mn);
-            L = L * ca + lw * cb;
-            O = O * ca + ow * cb;
-            M = Mn;
-        }
-        if (complete) {
-            out_rows[idx] = O / L;
-        } else {
-            my_part[2 * kMaxGroup + idx] = O;
-            if (d == 0) {
-                my_part[g] = M;
-                my_part[kMaxGroup + g] = L;
-            }
-        }
+    if (x < a.full_tiles) {
+        const int unit = x / a.tiles_full, tile = x - unit * a.tiles_full;
+        krow = (int)(a.full_row0 + (long long)unit * 2 * a.rows_full) + tile * kTile;
+        vrow = krow + a.rows_full;
+    } else {
+        const int y = x - a.full_tiles;
+        const int unit = y / a.tiles_comp, tile = y - unit * a.tiles_comp;
+        krow = (int)(a.comp_row0 + (long long)unit * 2 * a.rows_comp) + tile * kTile;
+        vrow = krow + a.rows_comp;
     }
-    if (!complete) {
-        const int first_c = cta_of_tile(u.first_tile, T, P);
-        const int last_c = cta_of_tile((long long)u.first_tile + u.tiles - 1, T, P);
-        __threadfence();
-        consumer_sync<NG>();
-        if (ctid == 0) {
-            const int old = atomicAdd(&a.tickets[u.unit], 1);
-            *s_flag = (old == last_c - first_c);
-        }
-        consumer_sync<NG>();
-        if (*s_flag) {
-            __threadfence();
-            for (int idx = ctid; idx < G * D; idx += NT) {
-                const int g = idx / D;
-                float M = kNegBig, L = 0.f, O = 0.f;
-                for (int c = first_c; c <= last_c; ++c) {
-                    const int slot = (cta_start(c, T, P) >= u.first_tile) ? 0 : 1;
-                    const float* part = a.partials + ((size_t)c * 2 + slot) * PF;
-                    const float mc = __ldcg(part + g);
-                    const float lc = __ldcg(part + kMaxGroup + g);
-                    const float oc = __ldcg(part + 2 * kMaxGroup + idx);
-                    const float Mn = fmaxf(M, mc);
-                    const float ca = exp2f(M - Mn), cb = exp2f(mc - Mn);
-                    L = L * ca + lc * cb;
-                    O = O * ca + oc * cb;
-                    M = Mn;
-                }
-                out_rows[idx] = O / L;
-            }
-            if (ctid == 0) a.tickets[u.unit] = 0;  // ready for the next launch
-        }
-    }
-    consumer_sync<NG>();  // merge area and s_flag may be reused
 }
 
 // ---------------------------------------------------------------------------------------------
-// The kernel.  Warps 0 .. 4*NG-1 are consumers (group = warp / 4), the last warp is the producer.
+// The kernel.  Warp roles: 0 .. 4*NG-1 consumers (group = warp / 4); then one producer warp (TMA);
+// one claim warp (fetches the next work item from the global counter while the producer streams the
+// current one, so no memory round trip ever sits in the producer's path); kEpilogueWarps epilogue
+// warps (merge the consumer warps' states of a finished segment, write the output or the partial,
+// run the ticket and the merge of split units) so that the consumer warps go straight on to the
+// next segment.  All hand-offs are mbarrier rings in shared memory.
+//
+// Slot i % stages of the tile ring holds the i-th slot the CTA issues; the slot of flat tile x
+// always has i = x (mod NG), so tile x is consumed by group x % NG whatever the CTA did before
+// (results do not depend on which CTA claimed which item) and a stage is always consumed by the
+// same group (stages is a multiple of NG).  Where an item starts on the wrong residue the producer
+// issues an empty slot first.
 template <int D, int NG>
-__global__ void __launch_bounds__(NG * kGroupWarps * 32 + 32, 1)
-decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, const int stages)
+__global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
+decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmap, const int stages)
 {
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                               ~static_cast<uintptr_t>(1023));
+    constexpr int MS = S::kMergeStride;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    const int G = a.group;
     uint8_t* stage_base = smem;
-    float* merge = reinterpret_cast<float*>(smem + (size_t)stages * S::kStageBytes);
-    float* stat_m = merge + S::merge_floats(a.group);
-    float* stat_l = stat_m + S::kWarps * kMaxGroup;
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(stat_l + S::kWarps * kMaxGroup);
+    uint8_t* buffers = smem + (size_t)stages * S::kStageBytes;
+    const int buffer_bytes = S::buffer_bytes(G);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(buffers + (size_t)kMergeBuffers * buffer_bytes);
     uint64_t* empty_bar = full_bar + 8;
-    int* s_flag = reinterpret_cast<int*>(empty_bar + 8);
-    volatile int* s_abort = s_flag + 1;
+    uint64_t* item_full = empty_bar + 8;
+    uint64_t* item_empty = item_full + kItemRing;
+    uint64_t* claim_full = item_empty + kItemRing;
+    uint64_t* claim_empty = claim_full + 1;
+    uint64_t* ep_full = claim_empty + 1;
+    uint64_t* ep_empty = ep_full + kMergeBuffers;
+    int4* item_desc = reinterpret_cast<int4*>(ep_empty + kMergeBuffers);
+    volatile int* claim_slot = reinterpret_cast<volatile int*>(item_desc + kItemRing);
+    volatile int* ep_flag = claim_slot + 1;
+    volatile int* s_abort = claim_slot + 2;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const CtaWork work = cta_work(a, blockIdx.x, gridDim.x);
-    const bool stamp = (a.debug & 4) != 0;
-    if (stamp && tid == 0) a.timeline[blockIdx.x * 4 + 0] = global_timer_ns();
+    const Schedule& sc = a.sched;
+    const bool trace = a.trace_on != 0;
+    unsigned long long* my_trace = a.trace + (size_t)blockIdx.x * kTraceWords;
+    if (trace && tid == 0) my_trace[0] = global_timer_ns();
 
+    if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
+        if (tid == 0) atomicCAS(a.status, kStatusOk, kStatusSmemMisaligned);
+        return;
+    }
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
             mbar_init(smem_u32(empty_bar + s), kGroupWarps);
         }
-        *s_flag = 0;
+        for (int i = 0; i < kItemRing; ++i) {
+            mbar_init(smem_u32(item_full + i), 1);
+            mbar_init(smem_u32(item_empty + i), S::kWarps);
+        }
+        mbar_init(smem_u32(claim_full), 1);
+        mbar_init(smem_u32(claim_empty), 1);
+        for (int i = 0; i < kMergeBuffers; ++i) {
+            mbar_init(smem_u32(ep_full + i), S::kWarps);
+            mbar_init(smem_u32(ep_empty + i), kEpilogueWarps);
+        }
+        *ep_flag = 0;
         *s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    if (warp == S::kWarps) {
-        // ------------------------------------------------------------------ producer warp
-        if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
-            int s = 0;
-            uint32_t par = 0;
-            for (int v = 0; v < work.total; ++v) {
-                const UnitInfo u = locate(a, work, v);
-                wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status,
-                             kStatusEmptyWaitTimeout);
-                const uint32_t fb = smem_u32(full_bar + s);
-                mbar_expect_tx(fb, S::kStageBytes);
-                const uint32_t dst = smem_u32(stage_base + (size_t)s * S::kStageBytes);
-                const int krow = (int)(u.krow + (long long)u.tile * kTile);
-                const int vrow = krow + u.rows;
-                if (D == 128) {  // one contiguous 16 KB box per tile: [64 rows][2 halves][64]
-                    tma_load_3d(dst, &tmap, 0, 0, krow, fb);
-                    tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb);
-                } else {         // one contiguous 8 KB box per tile: [64 rows][64]
-                    tma_load_2d(dst, &tmap, 0, krow, fb);
-                    tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb);
-                }
-                if (++s == stages) {
-                    s = 0;
-                    par ^= 1u;
-                }
-            }
-        }
-    } else {
+    int issued = 0;  // producer: slots issued so far (data or empty)
+    if (warp < S::kWarps) {
         // ------------------------------------------------------------------ consumer warps
         const int grp = warp / kGroupWarps, wig = warp % kGroupWarps;  // tile group, 16-token slice
         const int quad = lane >> 2, tq = lane & 3;  // row inside an 8-row fragment, column pair
@@ -317,152 +294,393 @@ decode_kernel(const DecodeArgs a, const __grid_constant__ CUtensorMap tmap, cons
         // starts at r*2*D bytes; its 16-byte chunk c sits at chunk index c ^ (bits 7..9 of the
         // unswizzled offset), i.e. c ^ ((2r + c/8) & 7) for D = 128 and c ^ (r & 7) for D = 64.
         const uint32_t row_off = ldm_tok * (2 * D);
-        int s = 0, turn = 0;  // pipeline stage and whose turn the next tile is
-        uint32_t par = 0;
-        for (int v = 0; v < work.total;) {
-            const UnitInfo u = locate(a, work, v);
-            const int seg_tiles = min(work.total - v, u.tiles - u.tile);
-
-            // Q as the A operand (rows = query heads of the group, rows >= G are zero)
-            uint32_t qa[KS][2];
-            {
-                const __nv_bfloat16* qrow =
-                    a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * a.group + quad) * D + 2 * tq;
-#pragma unroll
-                for (int ks = 0; ks < KS; ++ks) {
-                    qa[ks][0] = quad < a.group ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
-                    qa[ks][1] = quad < a.group ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
+        int cnt = 0;   // slots seen so far (mirrors the producer's `issued`)
+        int seg = 0;   // segments handed to the epilogue warps so far
+        int di = 0;
+        uint32_t dpar = 0;
+        int n_items = 0, n_tiles = 0, n_partial = 0;  // trace counters
+        bool landed = false, alive = true;
+        while (alive) {
+            if (!wait_bounded(smem_u32(item_full + di), dpar, s_abort, a.status, kStatusItemWaitTimeout)) break;
+            const int4 desc = item_desc[di];
+            const int item = desc.x, x0 = desc.y, x1 = desc.z;
+            if (item >= 0) {
+                ++n_items;
+                // skip the empty slots the producer issued to line the slot counter up with x0
+                for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, ++cnt) {
+                    if (cnt % NG != grp) continue;
+                    const int st = cnt % stages;
+                    alive = wait_bounded(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort, a.status,
+                                         kStatusFullWaitTimeout);
+                    if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
                 }
             }
-            float m_run = kNegBig, l_run = 0.f;
-            float acc[KS][4];
+            for (int x = x0; alive && (item < 0 || x < x1);) {
+                // ---- the segment: tiles [x, x + seg_tiles) of one unit (none for the stop message)
+                UnitInfo u{};
+                int seg_tiles = 0;
+                float m_run = kNegBig, l_run = 0.f;
+                float acc[KS][4];
 #pragma unroll
-            for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
-
-            int valid_left = u.len - u.tile * kTile;  // valid rows from this tile to the unit's end
-            for (int i = 0; i < seg_tiles; ++i, valid_left -= kTile) {
-                const bool mine = (turn == grp);
-                const int cur_s = s;
-                const uint32_t cur_par = par;
-                if (++turn == NG) turn = 0;
-                if (++s == stages) {
-                    s = 0;
-                    par ^= 1u;
-                }
-                if (!mine) continue;
-                wait_bounded(smem_u32(full_bar + cur_s), cur_par, s_abort, a.status, kStatusFullWaitTimeout);
-                if (stamp && tid == 0 && v == 0 && i == 0) a.timeline[blockIdx.x * 4 + 1] = global_timer_ns();
-                const int valid = min(kTile, valid_left);
-                if (wig * 16 < valid) {
-                    const uint32_t sK = smem_u32(stage_base + (size_t)cur_s * S::kStageBytes);
-                    const uint32_t sV = sK + S::kTileBytes;
-                    // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
-                    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-                    float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
+                if (item >= 0) {
+                    u = locate(a, x);
+                    seg_tiles = min(x1 - x, u.tiles - u.tile);
+                    // Q as the A operand (rows = query heads of the group, rows >= G are zero)
+                    uint32_t qa[KS][2];
+                    {
+                        const __nv_bfloat16* qrow =
+                            a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G + quad) * D + 2 * tq;
 #pragma unroll
-                    for (int ks = 0; ks < KS; ++ks) {
-                        const int chunk = ks * 2 + ldm_chunk;  // 16-byte chunk along d
-                        const uint32_t addr = sK + row_off + swizzled_chunk<D>(ldm_tok, chunk);
-                        uint32_t b0, b1, b2, b3;
-                        ldmatrix_x4(addr, b0, b1, b2, b3);
-                        if (ks & 1) {
-                            mma_bf16(s2, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
-                            mma_bf16(s3, qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
-                        } else {
-                            mma_bf16(s0, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
-                            mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+                        for (int ks = 0; ks < KS; ++ks) {
+                            qa[ks][0] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
+                            qa[ks][1] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
                         }
                     }
-                    // this lane: head `quad`, tokens wig*16 + {2tq, 2tq+1, 8+2tq, 9+2tq}
-                    float sc[4];
-                    sc[0] = (s0[0] + s2[0]) * a.scale_log2;
-                    sc[1] = (s0[1] + s2[1]) * a.scale_log2;
-                    sc[2] = (s1[0] + s3[0]) * a.scale_log2;
-                    sc[3] = (s1[1] + s3[1]) * a.scale_log2;
-                    const int tok0 = wig * 16 + 2 * tq;
-                    if (tok0 >= valid) sc[0] = -INFINITY;
-                    if (tok0 + 1 >= valid) sc[1] = -INFINITY;
-                    if (tok0 + 8 >= valid) sc[2] = -INFINITY;
-                    if (tok0 + 9 >= valid) sc[3] = -INFINITY;
-                    // ---- online softmax (log2 domain)
-                    float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                    const float m_new = fmaxf(m_run, mx);
-                    const float corr = exp2f(m_run - m_new);
-                    const float p0 = exp2f(sc[0] - m_new), p1 = exp2f(sc[1] - m_new);
-                    const float p2 = exp2f(sc[2] - m_new), p3 = exp2f(sc[3] - m_new);
-                    l_run = l_run * corr + ((p0 + p1) + (p2 + p3));
-                    m_run = m_new;
-                    // O^T columns of this lane are heads 2tq and 2tq+1: fetch their corrections
-                    const float ca = __shfl_sync(0xffffffffu, corr, tq * 8);
-                    const float cb = __shfl_sync(0xffffffffu, corr, tq * 8 + 4);
-                    const uint32_t pb0 = pack_bf16(p0, p1), pb1 = pack_bf16(p2, p3);
-                    // ---- O^T[d][head] += V^T[d][tok] . P^T[tok][head]
+                    int valid_left = u.len - u.tile * kTile;  // valid rows from this tile to the unit's end
+                    for (int i = 0; alive && i < seg_tiles; ++i, ++cnt, valid_left -= kTile) {
+                        if (cnt % NG != grp) continue;
+                        const int st = cnt % stages;
+                        alive = wait_bounded(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort,
+                                             a.status, kStatusFullWaitTimeout);
+                        if (!alive) break;
+                        if (trace && tid == 0 && !landed) {
+                            my_trace[1] = global_timer_ns();
+                            landed = true;
+                        }
+                        const int valid = min(kTile, valid_left);
+                        if (wig * 16 < valid) {
+                            const uint32_t sK = smem_u32(stage_base + (size_t)st * S::kStageBytes);
+                            const uint32_t sV = sK + S::kTileBytes;
+                            // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
+                            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                            float s2[4] = {0.f, 0.f, 0.f, 0.f}, s3[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                            for (int ks = 0; ks < KS; ++ks) {
+                                const int chunk = ks * 2 + ldm_chunk;  // 16-byte chunk along d
+                                const uint32_t addr = sK + row_off + swizzled_chunk<D>(ldm_tok, chunk);
+                                uint32_t b0, b1, b2, b3;
+                                ldmatrix_x4(addr, b0, b1, b2, b3);
+                                if (ks & 1) {
+                                    mma_bf16(s2, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+                                    mma_bf16(s3, qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+                                } else {
+                                    mma_bf16(s0, qa[ks][0], 0u, qa[ks][1], 0u, b0, b1);
+                                    mma_bf16(s1, qa[ks][0], 0u, qa[ks][1], 0u, b2, b3);
+                                }
+                            }
+                            // this lane: head `quad`, tokens wig*16 + {2tq, 2tq+1, 8+2tq, 9+2tq}
+                            float sc4[4];
+                            sc4[0] = (s0[0] + s2[0]) * a.scale_log2;
+                            sc4[1] = (s0[1] + s2[1]) * a.scale_log2;
+                            sc4[2] = (s1[0] + s3[0]) * a.scale_log2;
+                            sc4[3] = (s1[1] + s3[1]) * a.scale_log2;
+                            const int tok0 = wig * 16 + 2 * tq;
+                            if (tok0 >= valid) sc4[0] = -INFINITY;
+                            if (tok0 + 1 >= valid) sc4[1] = -INFINITY;
+                            if (tok0 + 8 >= valid) sc4[2] = -INFINITY;
+                            if (tok0 + 9 >= valid) sc4[3] = -INFINITY;
+                            // ---- online softmax (log2 domain)
+                            float mx = fmaxf(fmaxf(sc4[0], sc4[1]), fmaxf(sc4[2], sc4[3]));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                            const float m_new = fmaxf(m_run, mx);
+                            const float corr = exp2f(m_run - m_new);
+                            const float p0 = exp2f(sc4[0] - m_new), p1 = exp2f(sc4[1] - m_new);
+                            const float p2 = exp2f(sc4[2] - m_new), p3 = exp2f(sc4[3] - m_new);
+                            l_run = l_run * corr + ((p0 + p1) + (p2 + p3));
+                            m_run = m_new;
+                            // O^T columns of this lane are heads 2tq and 2tq+1: fetch their corrections
+                            const float ca = __shfl_sync(0xffffffffu, corr, tq * 8);
+                            const float cb = __shfl_sync(0xffffffffu, corr, tq * 8 + 4);
+                            const uint32_t pb0 = pack_bf16(p0, p1), pb1 = pack_bf16(p2, p3);
+                            // ---- O^T[d][head] += V^T[d][tok] . P^T[tok][head]
+#pragma unroll
+                            for (int mt = 0; mt < KS; ++mt) {
+                                const int chunk = mt * 2 + ldm_chunk;
+                                const uint32_t addr = sV + row_off + swizzled_chunk<D>(ldm_tok, chunk);
+                                uint32_t v0, v1, v2, v3;
+                                ldmatrix_x4_trans(addr, v0, v1, v2, v3);
+                                acc[mt][0] *= ca;
+                                acc[mt][1] *= cb;
+                                acc[mt][2] *= ca;
+                                acc[mt][3] *= cb;
+                                mma_bf16(acc[mt], v0, v1, v2, v3, pb0, pb1);
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(empty_bar + st));
+                    }
+                    if (!alive) break;
+                }
+
+                // ---- hand the warp's state (or the stop message) to the epilogue warps
+                const int bi = seg % kMergeBuffers;
+                alive = wait_bounded(smem_u32(ep_empty + bi), ((uint32_t)(seg / kMergeBuffers) & 1u) ^ 1u, s_abort,
+                                     a.status, kStatusMergeWaitTimeout);
+                if (!alive) break;
+                uint8_t* buf = buffers + (size_t)bi * buffer_bytes;
+                float* merge = reinterpret_cast<float*>(buf);
+                float* stat_m = merge + S::merge_floats(G);
+                float* stat_l = stat_m + S::kWarps * kMaxGroup;
+                if (item >= 0) {
+                    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+                    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+                    if (tq == 0) {
+                        stat_m[warp * kMaxGroup + quad] = m_run;
+                        stat_l[warp * kMaxGroup + quad] = l_run;
+                    }
+                    float* mw = merge + (size_t)warp * G * MS;
+                    const int h0 = 2 * tq, h1 = 2 * tq + 1;
 #pragma unroll
                     for (int mt = 0; mt < KS; ++mt) {
-                        const int chunk = mt * 2 + ldm_chunk;
-                        const uint32_t addr = sV + row_off + swizzled_chunk<D>(ldm_tok, chunk);
-                        uint32_t v0, v1, v2, v3;
-                        ldmatrix_x4_trans(addr, v0, v1, v2, v3);
-                        acc[mt][0] *= ca;
-                        acc[mt][1] *= cb;
-                        acc[mt][2] *= ca;
-                        acc[mt][3] *= cb;
-                        mma_bf16(acc[mt], v0, v1, v2, v3, pb0, pb1);
+                        const int d0 = mt * 16 + quad;
+                        if (h0 < G) {
+                            mw[h0 * MS + d0] = acc[mt][0];
+                            mw[h0 * MS + d0 + 8] = acc[mt][2];
+                        }
+                        if (h1 < G) {
+                            mw[h1 * MS + d0] = acc[mt][1];
+                            mw[h1 * MS + d0 + 8] = acc[mt][3];
+                        }
                     }
+                }
+                if (warp == 0 && lane == 0) {
+                    SegDesc* sd = reinterpret_cast<SegDesc*>(stat_l + S::kWarps * kMaxGroup);
+                    const bool complete = (u.tile == 0 && seg_tiles == u.tiles);
+                    sd->out_row = u.b * a.q_heads + u.head * G;
+                    sd->uid = u.uid;
+                    sd->complete = complete ? 1 : 0;
+                    sd->item = item;
+                    sd->slot = (x == x0) ? 0 : 1;
+                    sd->first_tile = u.first_tile;
+                    sd->tiles = u.tiles;
+                    sd->stop = item < 0 ? 1 : 0;
+                    n_tiles += seg_tiles;
+                    if (item >= 0 && !complete) ++n_partial;
+                    if (trace) my_trace[2] = global_timer_ns();
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(empty_bar + cur_s));
+                if (lane == 0) mbar_arrive(smem_u32(ep_full + bi));  // release: the warp's rows are visible
+                ++seg;
+                if (item < 0) {
+                    alive = false;  // the stop message was the last thing to do
+                    break;
+                }
+                x += seg_tiles;
             }
-
-            // ---- hand the warp's state to the cross-warp merge
-            l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-            l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-            if (tq == 0) {
-                stat_m[warp * kMaxGroup + quad] = m_run;
-                stat_l[warp * kMaxGroup + quad] = l_run;
+            if (!alive) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(item_empty + di));
+            if (++di == kItemRing) {
+                di = 0;
+                dpar ^= 1u;
             }
-            {
-                const int G = a.group;
-                float* mw = merge + (size_t)warp * G * S::kMergeStride;
-                const int h0 = 2 * tq, h1 = 2 * tq + 1;
-#pragma unroll
-                for (int mt = 0; mt < KS; ++mt) {
-                    const int d0 = mt * 16 + quad;
-                    if (h0 < G) {
-                        mw[h0 * S::kMergeStride + d0] = acc[mt][0];
-                        mw[h0 * S::kMergeStride + d0 + 8] = acc[mt][2];
+        }
+        if (trace && tid == 0) {
+            my_trace[4] = (unsigned long long)n_items;
+            my_trace[5] = (unsigned long long)n_tiles;
+            my_trace[6] = (unsigned long long)n_partial;
+        }
+    } else if (warp == S::kWarps) {
+        // ------------------------------------------------------------------ producer warp
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            int s = 0, di = 0;
+            uint32_t par = 0, dpar = 0, cpar = 0;
+            bool ok = true;
+            int k = blockIdx.x;  // the host launches no more CTAs than there are items
+            while (ok && k < sc.n_items) {
+                mbar_arrive(smem_u32(claim_empty));  // ask the claim warp for the item after this one
+                const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
+                ok = wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout);
+                if (!ok) break;
+                item_desc[di] = make_int4(k, x0, x1, 0);
+                mbar_arrive(smem_u32(item_full + di));  // release: the descriptor is visible to the waiters
+                if (++di == kItemRing) {
+                    di = 0;
+                    dpar ^= 1u;
+                }
+                // empty slots until the slot counter has the residue of x0
+                for (int pad = ((x0 - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
+                    ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
+                    if (!ok) break;
+                    mbar_arrive(smem_u32(full_bar + s));
+                    ++issued;
+                    if (++s == stages) {
+                        s = 0;
+                        par ^= 1u;
                     }
-                    if (h1 < G) {
-                        mw[h1 * S::kMergeStride + d0] = acc[mt][1];
-                        mw[h1 * S::kMergeStride + d0 + 8] = acc[mt][3];
+                }
+                for (int x = x0; ok && x < x1; ++x) {
+                    int krow, vrow;
+                    tile_rows(a, x, krow, vrow);
+                    ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
+                    if (!ok) break;
+                    const uint32_t fb = smem_u32(full_bar + s);
+                    mbar_expect_tx(fb, S::kStageBytes);
+                    const uint32_t dst = smem_u32(stage_base + (size_t)s * S::kStageBytes);
+                    if (D == 128) {  // one contiguous 16 KB box per tile: [64 rows][2 halves][64]
+                        tma_load_3d(dst, &tmap, 0, 0, krow, fb);
+                        tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb);
+                    } else {         // one contiguous 8 KB box per tile: [64 rows][64]
+                        tma_load_2d(dst, &tmap, 0, krow, fb);
+                        tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb);
+                    }
+                    ++issued;
+                    if (++s == stages) {
+                        s = 0;
+                        par ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                ok = wait_bounded(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout);
+                cpar ^= 1u;
+                if (ok) k = *claim_slot;
+            }
+            if (ok && wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout)) {
+                item_desc[di] = make_int4(-1, 0, 0, 0);  // no more work
+                mbar_arrive(smem_u32(item_full + di));
+            }
+        }
+    } else if (warp == S::kWarps + 1) {
+        // ------------------------------------------------------------------ claim warp
+        if (lane == 0) {
+            uint32_t par = 0;
+            for (;;) {
+                if (!wait_bounded(smem_u32(claim_empty), par, s_abort, a.status, kStatusClaimWaitTimeout)) break;
+                par ^= 1u;
+                const int k = sc.P + atomicAdd(&a.counters[0], 1);
+                *claim_slot = k;
+                mbar_arrive(smem_u32(claim_full));
+                if (k >= sc.n_items) break;  // the producer stops asking once it has seen this answer
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps
+        constexpr int NE = kEpilogueWarps * 32;
+        constexpr int D4 = D / 4;
+        const int et = tid - (S::kWarps + 2) * 32;
+        const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+        const size_t slot_stride = (size_t)a.part_items * PF;
+        for (int seg = 0;; ++seg) {
+            const int bi = seg % kMergeBuffers;
+            const bool got = wait_bounded(smem_u32(ep_full + bi), (uint32_t)(seg / kMergeBuffers) & 1u, s_abort,
+                                          a.status, kStatusMergeWaitTimeout);
+            if (epilogue_or(!got)) break;
+            const uint8_t* buf = buffers + (size_t)bi * buffer_bytes;
+            const float* merge = reinterpret_cast<const float*>(buf);
+            const float* stat_m = merge + S::merge_floats(G);
+            const float* stat_l = stat_m + S::kWarps * kMaxGroup;
+            const SegDesc sd = *reinterpret_cast<const SegDesc*>(stat_l + S::kWarps * kMaxGroup);
+            if (sd.stop) break;
+            float* out_rows = a.out + (size_t)sd.out_row * D;
+            float* my_part = a.partials + (size_t)sd.slot * slot_stride + (size_t)sd.item * PF;
+            // merge the consumer warps' states; this thread owns a few 4-float pieces of the G x D rows
+            for (int e = et; e < G * D4; e += NE) {
+                const int g = e / D4, d4 = e - g * D4;
+                float M = kNegBig;
+#pragma unroll
+                for (int w = 0; w < S::kWarps; ++w) M = fmaxf(M, stat_m[w * kMaxGroup + g]);
+                float L = 0.f;
+                float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int w = 0; w < S::kWarps; ++w) {
+                    const float wt = exp2f(stat_m[w * kMaxGroup + g] - M);
+                    const float4 o = *reinterpret_cast<const float4*>(merge + (size_t)(w * G + g) * MS + d4 * 4);
+                    L += stat_l[w * kMaxGroup + g] * wt;
+                    O.x += o.x * wt;
+                    O.y += o.y * wt;
+                    O.z += o.z * wt;
+                    O.w += o.w * wt;
+                }
+                if (sd.complete) {
+                    const float inv = 1.f / L;
+                    *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                } else {
+                    *reinterpret_cast<float4*>(my_part + PH + e * 4) = O;
+                    if (d4 == 0) {
+                        my_part[g] = M;
+                        my_part[G + g] = L;
                     }
                 }
             }
-            if (stamp && tid == 0 && v + seg_tiles == work.total) a.timeline[blockIdx.x * 4 + 2] = global_timer_ns();
-            finalize_segment<D, NG>(a, u, u.tile == 0 && seg_tiles == u.tiles, merge, stat_m, stat_l,
-                                    s_flag, tid);
-            v += seg_tiles;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(ep_empty + bi));  // the buffer may be refilled
+            if (!sd.complete) {
+                const int first_k = item_of_tile(sc, sd.first_tile);
+                const int last_k = item_of_tile(sc, sd.first_tile + sd.tiles - 1);
+                __threadfence();
+                epilogue_sync();
+                if (et == 0) {
+                    const int old = atomicAdd(&a.tickets[sd.uid], 1);
+                    *ep_flag = (old == last_k - first_k);
+                }
+                epilogue_sync();
+                if (*ep_flag) {
+                    // the last partial of the unit has arrived: merge them in item order, so the
+                    // result does not depend on who arrived when
+                    __threadfence();
+                    // the unit's piece of item first_k is that item's first segment only if the item
+                    // starts at or after the unit's first tile; in every later item it is the first
+                    const int slot0 = item_start(sc, first_k) < sd.first_tile ? 1 : 0;
+                    const float* p0 = a.partials + (size_t)slot0 * slot_stride + (size_t)first_k * PF;
+                    const float* p1 = a.partials + (size_t)(first_k + 1) * PF;  // slot 0 of the items after
+                    const int n = last_k - first_k;
+                    for (int e = et; e < G * D4; e += NE) {
+                        const int g = e / D4;
+                        const float m0 = __ldcg(p0 + g);
+                        float M = m0;
+#pragma unroll 8
+                        for (int c = 0; c < n; ++c) M = fmaxf(M, __ldcg(p1 + (size_t)c * PF + g));
+                        float wt = exp2f(m0 - M);
+                        float L = __ldcg(p0 + G + g) * wt;
+                        float4 o = __ldcg(reinterpret_cast<const float4*>(p0 + PH) + e);
+                        float4 O = make_float4(o.x * wt, o.y * wt, o.z * wt, o.w * wt);
+#pragma unroll 8
+                        for (int c = 0; c < n; ++c) {
+                            const float* pc = p1 + (size_t)c * PF;
+                            wt = exp2f(__ldcg(pc + g) - M);
+                            L += __ldcg(pc + G + g) * wt;
+                            o = __ldcg(reinterpret_cast<const float4*>(pc + PH) + e);
+                            O.x += o.x * wt;
+                            O.y += o.y * wt;
+                            O.z += o.z * wt;
+                            O.w += o.w * wt;
+                        }
+                        const float inv = 1.f / L;
+                        *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                    }
+                    if (et == 0) a.tickets[sd.uid] = 0;  // ready for the next launch
+                }
+            }
         }
+        if (trace && et == 0) my_trace[7] = global_timer_ns();
     }
     __syncthreads();
-    if (stamp && tid == 0) a.timeline[blockIdx.x * 4 + 3] = global_timer_ns();
-    if (warp == S::kWarps && lane == 0 && *s_abort) {
-        // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
-        // when the CTA retires
-        const int issued = work.total;
-        for (int j = issued > stages ? issued - stages : 0; j < issued; ++j)
-            wait_bounded(smem_u32(full_bar + j % stages), (uint32_t)(j / stages) & 1u, s_abort, a.status,
-                         kStatusDrainTimeout, false);
+    if (warp == S::kWarps && lane == 0) {
+        if (*s_abort) {
+            // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
+            // when the CTA retires
+            for (int j = issued > stages ? issued - stages : 0; j < issued; ++j)
+                wait_bounded(smem_u32(full_bar + j % stages), (uint32_t)(j / stages) & 1u, s_abort, a.status,
+                             kStatusDrainTimeout, false);
+        }
+        // the last CTA to finish rearms the claim counter for the next launch
+        __threadfence();
+        if (atomicAdd(&a.counters[1], 1) == (int)gridDim.x - 1) {
+            a.counters[0] = 0;
+            a.counters[1] = 0;
+        }
     }
+    if (trace && tid == 0) my_trace[3] = global_timer_ns();
 }
 
 template <int D, int NG>
 cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream)
 {
     const size_t smem = Smem<D, NG>::bytes(stages, a.group);
-    decode_kernel<D, NG><<<grid, NG * kGroupWarps * 32 + 32, smem, stream>>>(a, tmap, stages);
+    decode_kernel<D, NG><<<grid, Smem<D, NG>::kThreads, smem, stream>>>(a, tmap, stages);
     return cudaGetLastError();
 }
 

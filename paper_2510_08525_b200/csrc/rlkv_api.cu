@@ -9,9 +9,10 @@
 //             (the constant-size pool of Section 4.3 of the paper).
 //   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
 //   tickets   int32 [layers][batch*kv_heads]   (split bookkeeping, zero between launches)
-//   status    int32 kernel status word
-//   partials  float [max_grid][2][partial_floats]  (split-KV scratch)
+//   status    int32 kernel status word, then the two work-claim counters (zero between launches)
+//   partials  float [2][max_items][partial_floats]  (split-KV scratch)
 //   staging   k, v, q, out of one whole step, for rlkv_step_host
+//   trace     uint64 [max_grid][8]  (debug trace of the decode kernel)
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
@@ -48,11 +49,25 @@ struct Layout {
     std::vector<long long> full_row0, comp_row0;  // per layer, in pool rows
     long long pool_rows = 0;
     size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
-    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_timeline = 0, total = 0;
-    int max_grid = 0;
+    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_trace = 0, total = 0;
+    int max_grid = 0, max_items = 0;
 };
 
 constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
+constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
+constexpr int kDefaultItemTiles = 4;
+
+// Most work items a decode launch can have when the flat tile space holds at most t_max tiles and
+// the grid at most max_grid CTAs.
+int most_items(long long t_max, int max_grid)
+{
+    int most = 0;
+    for (int p = 1; p <= max_grid; ++p) {  // the bound grows with P except for rounding
+        const int m = max_items((int)t_max, p, kMinItemTiles);
+        if (m > most) most = m;
+    }
+    return most;
+}
 
 int check_shape(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
                 const uint8_t* mask, int sink, int window)
@@ -85,6 +100,17 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     L.pool_rows = row;
     if (row >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
     L.max_grid = 2 * kMaxGridSms;
+    {
+        // the longest flat tile space is reached at max_len by the layer with the most full heads
+        long long t_max = 0;
+        for (int l = 0; l < layers; ++l) {
+            const long long t = (long long)batch * (L.n_full[l] * (long long)(L.rows_full / kTile) +
+                                                    L.n_comp[l] * (long long)(L.rows_comp / kTile));
+            if (t > t_max) t_max = t;
+        }
+        if (t_max >= (1ll << 31)) return RLKV_EINVAL;
+        L.max_items = most_items(t_max, L.max_grid);
+    }
     size_t off = 0;
     L.off_pool = off;
     off = align_up(off + (size_t)row * head_dim * 2, 1024);
@@ -95,7 +121,7 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     L.off_status = off;
     off = align_up(off + 64, 1024);
     L.off_partials = off;
-    off = align_up(off + (size_t)L.max_grid * 2 * partial_floats(head_dim) * sizeof(float), 1024);
+    off = align_up(off + (size_t)L.max_items * 2 * partial_floats(head_dim, q_heads / kv_heads) * sizeof(float), 1024);
     const size_t kv_step = (size_t)layers * batch * kv_heads * head_dim * 2;
     const size_t q_step = (size_t)layers * batch * q_heads * head_dim * 2;
     L.off_k = off;
@@ -106,8 +132,8 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     off = align_up(off + q_step, 1024);
     L.off_out = off;
     off = align_up(off + q_step * 2, 1024);
-    L.off_timeline = off;
-    off = align_up(off + (size_t)L.max_grid * 4 * sizeof(unsigned long long), 1024);
+    L.off_trace = off;
+    off = align_up(off + (size_t)L.max_grid * kTraceWords * sizeof(unsigned long long), 1024);
     L.total = off;
     return RLKV_OK;
 }
@@ -149,7 +175,8 @@ struct DeviceGuard {
 struct rlkv_cache {
     int layers, kv_heads, q_heads, head_dim, batch, max_len, sink, window;
     int device, sm_count;
-    int ctas_per_sm, stages, groups;  // decode launch shape (rlkv_set_decode_config)
+    int ctas_per_sm, stages, groups, item_tiles;  // decode launch shape (rlkv_set_decode_config)
+    int trace_on;
     Layout lay;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -186,8 +213,7 @@ int make_tensor_map(rlkv_cache* c)
     //   head_dim  64: [rows][64]            box [64 rows][64]     ( 8 KB)
     CUresult r;
     void* base = c->dev_base + c->lay.off_pool;
-    const CUtensorMapL2promotion l2p = getenv("RLKV_L2P") ? (CUtensorMapL2promotion)atoi(getenv("RLKV_L2P"))
-                                                          : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+    const CUtensorMapL2promotion l2p = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
     if (c->head_dim == 128) {
         const cuuint64_t dims[3] = {64, 2, (cuuint64_t)c->lay.pool_rows};
         const cuuint64_t strides[2] = {128, 256};
@@ -240,21 +266,20 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
     return RLKV_OK;
 }
 
-int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
+// Everything of a decode launch except where its split-KV work area lives.  Returns the grid size
+// in *grid_out.
+int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, DecodeArgs& a, int* grid_out)
 {
     const int n = c->len[layer];
     const int cap = c->sink + c->window;
-    DecodeArgs a;
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
     a.full_row0 = c->lay.full_row0[layer];
     a.comp_row0 = c->lay.comp_row0[layer];
     a.head_of_slot = dev_at<int>(c, c->lay.off_tables) + (size_t)(c->layers + layer) * c->kv_heads;
     a.q = static_cast<const __nv_bfloat16*>(q);
     a.out = static_cast<float*>(out);
-    a.partials = dev_at<float>(c, c->lay.off_partials);
-    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
     a.status = dev_at<int>(c, c->lay.off_status);
-    a.timeline = dev_at<unsigned long long>(c, c->lay.off_timeline);
+    a.trace = dev_at<unsigned long long>(c, c->lay.off_trace);
     a.n_full = c->lay.n_full[layer];
     a.n_comp = c->lay.n_comp[layer];
     a.rows_full = c->lay.rows_full;
@@ -266,29 +291,44 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.q_heads = c->q_heads;
     a.tiles_full = (a.len_full + kTile - 1) / kTile;
     a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
-    const long long full_tiles = (long long)c->batch * a.n_full * a.tiles_full;
-    if (full_tiles >= (1ll << 31)) return RLKV_EINVAL;
+    a.full_units = c->batch * a.n_full;
+    const long long full_tiles = (long long)a.full_units * a.tiles_full;
+    const long long all_tiles = full_tiles + (long long)c->batch * a.n_comp * a.tiles_comp;
+    if (all_tiles >= (1ll << 31)) return RLKV_EINVAL;
     a.full_tiles = (int)full_tiles;
-    a.comp_units = c->batch * a.n_comp;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
-    { const char* d = getenv("RLKV_DEBUG"); a.debug = d ? atoi(d) : 0; }
-    // persistent grid; no more CTAs than there is work, and every CTA that shares the full tiles
-    // owns at least one of them (the split bookkeeping assumes no empty ranges)
+    a.trace_on = c->trace_on;
+    // persistent grid; the work items of the flat tile space are cut for that many CTAs and no
+    // more CTAs are launched than there are items
     int grid = c->sm_count * c->ctas_per_sm;
     if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    const int most_work = a.full_tiles > a.comp_units ? a.full_tiles : a.comp_units;
-    if (grid > most_work) grid = most_work;
-    a.grid_full = grid < a.full_tiles ? grid : a.full_tiles;
+    a.sched = make_schedule((int)all_tiles, grid, c->item_tiles);
+    if (grid > a.sched.n_items) grid = a.sched.n_items;
+    *grid_out = grid;
+    return RLKV_OK;
+}
+
+int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
+{
+    DecodeArgs a;
+    int grid = 0;
+    int rc = build_decode_args(c, layer, q, out, a, &grid);
+    if (rc) return rc;
+    if (a.sched.n_items > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
+    a.partials = dev_at<float>(c, c->lay.off_partials);
+    a.part_items = c->lay.max_items;
+    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
+    a.counters = dev_at<int>(c, c->lay.off_status) + 4;
     RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
     c->launches++;
     return RLKV_OK;
 }
 
 // ---- split-KV scratch that nobody allocates -------------------------------------------------------
-// rlkv_decode_attention_static_scratch keeps the decode kernel's split bookkeeping (tickets) and
-// partial results here instead of in the cache's own buffer.  The array is part of the library
-// image: every GPU that loads librlkv holds these bytes until the process exits.
-constexpr size_t kStaticScratchBytes = 2u << 20;
+// rlkv_decode_attention_static_scratch keeps the decode kernel's split bookkeeping (work-claim
+// counters, tickets) and partial results here instead of in the cache's own buffer.  The array is
+// part of the library image: every GPU that loads librlkv holds these bytes until the process exits.
+constexpr size_t kStaticScratchBytes = 4u << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
@@ -310,54 +350,29 @@ int static_scratch_address(int device, unsigned char** out)
     return RLKV_OK;
 }
 
-// The launch of do_decode with the tickets and partials placed in the static array.
+// The launch of do_decode with counters, tickets and partials placed in the static array.
 int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
 {
-    const int n = c->len[layer];
-    const int cap = c->sink + c->window;
     DecodeArgs a;
-    a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
-    a.full_row0 = c->lay.full_row0[layer];
-    a.comp_row0 = c->lay.comp_row0[layer];
-    a.head_of_slot = dev_at<int>(c, c->lay.off_tables) + (size_t)(c->layers + layer) * c->kv_heads;
-    a.q = static_cast<const __nv_bfloat16*>(q);
-    a.out = static_cast<float*>(out);
-    a.status = dev_at<int>(c, c->lay.off_status);
-    a.timeline = dev_at<unsigned long long>(c, c->lay.off_timeline);
-    a.n_full = c->lay.n_full[layer];
-    a.n_comp = c->lay.n_comp[layer];
-    a.rows_full = c->lay.rows_full;
-    a.rows_comp = c->lay.rows_comp;
-    a.len_full = n;
-    a.len_comp = n < cap ? n : cap;
-    a.batch = c->batch;
-    a.group = c->q_heads / c->kv_heads;
-    a.q_heads = c->q_heads;
-    a.tiles_full = (a.len_full + kTile - 1) / kTile;
-    a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
-    const long long full_tiles = (long long)c->batch * a.n_full * a.tiles_full;
-    if (full_tiles >= (1ll << 31)) return RLKV_EINVAL;
-    a.full_tiles = (int)full_tiles;
-    a.comp_units = c->batch * a.n_comp;
-    a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
-    a.debug = 0;
-    int grid = c->sm_count * c->ctas_per_sm;
-    if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    const int most_work = a.full_tiles > a.comp_units ? a.full_tiles : a.comp_units;
-    if (grid > most_work) grid = most_work;
-    a.grid_full = grid < a.full_tiles ? grid : a.full_tiles;
-
-    // carve the static array: one ticket per (batch row, KV head), then two partial records per CTA
-    const size_t ticket_bytes = align_up((size_t)c->batch * c->kv_heads * sizeof(int), 256);
-    const size_t partial_bytes = (size_t)grid * 2 * partial_floats(c->head_dim) * sizeof(float);
-    if (ticket_bytes + partial_bytes > kStaticScratchBytes) return RLKV_ESCRATCH;
-    unsigned char* base = nullptr;
-    int rc = static_scratch_address(c->device, &base);
+    int grid = 0;
+    int rc = build_decode_args(c, layer, q, out, a, &grid);
     if (rc) return rc;
-    a.tickets = reinterpret_cast<int*>(base);
-    a.partials = reinterpret_cast<float*>(base + ticket_bytes);
-    // the array still holds whatever the previous call (of any cache) left: tickets must start at 0
-    RLKV_CUDA(cudaMemsetAsync(base, 0, ticket_bytes, s));
+    // carve the static array: the two counters and one ticket per (batch row, KV head), then two
+    // partial records per work item of this launch
+    const size_t head_bytes = align_up((2 + (size_t)c->batch * c->kv_heads) * sizeof(int), 256);
+    const size_t partial_bytes =
+        (size_t)a.sched.n_items * 2 * partial_floats(c->head_dim, a.group) * sizeof(float);
+    if (head_bytes + partial_bytes > kStaticScratchBytes) return RLKV_ESCRATCH;
+    unsigned char* base = nullptr;
+    rc = static_scratch_address(c->device, &base);
+    if (rc) return rc;
+    a.counters = reinterpret_cast<int*>(base);
+    a.tickets = a.counters + 2;
+    a.partials = reinterpret_cast<float*>(base + head_bytes);
+    a.part_items = a.sched.n_items;
+    // the array still holds whatever the previous call (of any cache) left: counters and tickets
+    // must start at zero
+    RLKV_CUDA(cudaMemsetAsync(base, 0, head_bytes, s));
     RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
     c->launches++;
     return RLKV_OK;
@@ -410,6 +425,8 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->dev_base = nullptr; c->owns_buffer = false; c->launches = 0;
     c->ctas_per_sm = 1;
     c->groups = 2;
+    c->item_tiles = kDefaultItemTiles;
+    c->trace_on = 0;
     c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
     rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
     if (rc) { delete c; return rc; }
@@ -499,10 +516,11 @@ int rlkv_cache_reset(rlkv_cache* c, void* stream)
     return RLKV_OK;
 }
 
-int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consumer_groups)
+int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consumer_groups, int item_tiles)
 {
     if (!c || ctas_per_sm < 0 || ctas_per_sm > 2 || stages < 0 || stages == 1 || stages > 8 ||
-        consumer_groups < 0 || consumer_groups > kMaxConsumerGroups)
+        consumer_groups < 0 || consumer_groups > kMaxConsumerGroups ||
+        (item_tiles != 0 && (item_tiles < kMinItemTiles || item_tiles > 1024)))
         return RLKV_EINVAL;
     const int cps = ctas_per_sm ? ctas_per_sm : c->ctas_per_sm;
     const int ng = consumer_groups ? consumer_groups : c->groups;
@@ -513,6 +531,7 @@ int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consu
     c->ctas_per_sm = cps;
     c->stages = st;
     c->groups = ng;
+    if (item_tiles) c->item_tiles = item_tiles;
     return RLKV_OK;
 }
 
@@ -663,14 +682,36 @@ int rlkv_kernel_status(rlkv_cache* c, int* status_out)
     return *status_out == 0 ? RLKV_OK : RLKV_EKERNEL;
 }
 
-int rlkv_debug_timeline(rlkv_cache* c, unsigned long long* host_out, int* ctas_out)
+int rlkv_debug_trace(rlkv_cache* c, int enable, unsigned long long* words_host, int* ctas_out)
 {
-    if (!c || !host_out || !ctas_out) return RLKV_EINVAL;
-    DeviceGuard g(c->device);
-    RLKV_CUDA(cudaDeviceSynchronize());
-    RLKV_CUDA(cudaMemcpy(host_out, c->dev_base + c->lay.off_timeline, (size_t)c->lay.max_grid * 4 * 8,
-                         cudaMemcpyDeviceToHost));
-    *ctas_out = c->lay.max_grid;
+    if (!c) return RLKV_EINVAL;
+    if (words_host) {
+        if (!ctas_out) return RLKV_EINVAL;
+        DeviceGuard g(c->device);
+        if (!g.ok) return RLKV_ECUDA;
+        RLKV_CUDA(cudaDeviceSynchronize());
+        RLKV_CUDA(cudaMemcpy(words_host, c->dev_base + c->lay.off_trace,
+                             (size_t)c->lay.max_grid * kTraceWords * sizeof(unsigned long long),
+                             cudaMemcpyDeviceToHost));
+        *ctas_out = c->lay.max_grid;
+    }
+    c->trace_on = enable ? 1 : 0;
+    return RLKV_OK;
+}
+
+int rlkv_debug_schedule(int tiles, int ctas, int item_tiles, int* n_items_out, int* starts_out, int starts_cap)
+{
+    if (tiles < 1 || ctas < 1 || item_tiles < 1 || !n_items_out) return RLKV_EINVAL;
+    const Schedule sc = make_schedule(tiles, ctas, item_tiles);
+    *n_items_out = sc.n_items;
+    if (starts_out) {
+        if (starts_cap < sc.n_items + 1) return RLKV_ENOMEM;
+        for (int k = 0; k <= sc.n_items; ++k) starts_out[k] = item_start(sc, k);
+        // the inverse map must agree with the starts
+        for (int k = 0; k < sc.n_items; ++k)
+            for (int x = starts_out[k]; x < starts_out[k + 1]; ++x)
+                if (item_of_tile(sc, x) != k) return RLKV_EKERNEL;
+    }
     return RLKV_OK;
 }
 

@@ -166,8 +166,8 @@ def test_planted_needles_at_tile_and_split_boundaries(rl, hz, cuda_device):
     q = rand_bf16((B, 2, D), 7)
     marker = torch.full((D,), 7.0, dtype=torch.bfloat16)
     spots = [0, 1, S - 1, S, 63, 64, 65, 127, 128, 1023, 1024, n - W - 1, n - W, n - 2, n - 1]
-    # the flat tile space of this shape is split over many CTAs: add their boundaries too
-    spots += [t for c in range(1, 12) for t in (c * 192 - 1, c * 192)]
+    # the scan of this shape is cut into work items of 4 tiles (256 tokens): add their boundaries
+    spots += [t for c in range(1, 9) for t in (c * 256 - 1, c * 256)]
     for t_star in sorted(set(spots)):
         K, V = base_K.clone(), base_V.clone()
         for h in range(2):
@@ -301,12 +301,16 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     feed(cache, oracle, 0, K, V, True)
     want = oracle.decode(0, q)
     outs = []
-    for cps, st, ng in ((1, 6, 1), (1, 2, 2), (2, 2, 1), (1, 3, 3), (2, 2, 2), (1, 4, 2), (1, 0, 3), (1, 5, 1)):
-        rl.rlkv_set_decode_config(cache.handle, cps, st, ng)
+    for cps, st, ng, it in ((1, 6, 1, 0), (1, 2, 2, 2), (2, 2, 1, 3), (1, 3, 3, 2), (2, 2, 2, 5), (1, 4, 2, 16),
+                            (1, 0, 3, 7), (1, 5, 1, 1024), (1, 6, 3, 4), (1, 6, 2, 4)):
+        rl.rlkv_set_decode_config(cache.handle, cps, st, ng, it)
         outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
         check_out(outs[-1], want)
+        again = cache.decode(0, q.to(cuda_device)).cpu().numpy()
+        assert np.array_equal(outs[-1], again)      # which CTA claims which item must not matter
     for bad in ((2, 6, 1),      # does not fit in shared memory twice
-                (1, 5, 2), (1, 4, 3)):   # stages must be a multiple of the consumer groups
+                (1, 5, 2), (1, 4, 3),    # stages must be a multiple of the consumer groups
+                (1, 6, 2, 1)):           # work items have at least 2 tiles
         with pytest.raises(rl.RlkvError) as e:
             rl.rlkv_set_decode_config(cache.handle, *bad)
         assert e.value.code == rl.RLKV_EINVAL
@@ -319,3 +323,32 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     for t in range(100):
         o2.append(0, K[t], V[t])
     check_out(cache.decode(0, q.to(cuda_device)).cpu().numpy(), o2.decode(0, q))
+
+
+# ------------------------------------------------------------------------------------------ work claims
+def test_dynamic_work_claims_do_not_change_bits(rl, hz, cuda_device):
+    """A shape with a few hundred work items over all SMs: the items a CTA gets beyond its first are
+    claimed at run time, so repeated calls distribute them differently -- the output bits must not
+    move, and every unit that is split over items must still match the oracle."""
+    layers, Hkv, Hq, D, B, S, W, n = 1, 8, 32, 128, 4, 16, 112, 3001
+    mask = [1, 1, 0, 1, 1, 0, 1, 1]
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, n + 1, mask, S, W, cuda_device)
+    K, V, q = rand_bf16((n, B, Hkv, D), 41), rand_bf16((n, B, Hkv, D), 42), rand_bf16((B, Hq, D), 43)
+    feed(cache, oracle, 0, K, V, True)
+    want = oracle.decode(0, q)
+    qd = q.to(cuda_device)
+    first = cache.decode(0, qd).clone()
+    check_out(first.cpu().numpy(), want)
+    for it in (4, 2, 9):
+        rl.rlkv_set_decode_config(cache.handle, 0, 0, 0, it)
+        ref = cache.decode(0, qd).clone()
+        check_out(ref.cpu().numpy(), want)
+        for _ in range(4):
+            assert torch.equal(cache.decode(0, qd), ref)
+    assert cache.status() == 0
+    # the trace counts what the launch did: every tile was consumed exactly once
+    rl.rlkv_debug_trace(cache.handle, 1)
+    cache.decode(0, qd)
+    words = rl.rlkv_debug_trace(cache.handle, 0, read=True)
+    tiles = B * (6 * ((n + 63) // 64) + 2 * 2)
+    assert int(words[:, 5].sum()) == tiles

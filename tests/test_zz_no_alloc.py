@@ -30,9 +30,10 @@ def rand_bf16(shape, seed, device):
 def test_static_scratch_variant_matches_the_ordinary_call(cuda_device):
     import paper_2510_08525_b200.binding as rl
 
-    # long rows on few units: every CTA ends inside a unit, so tickets and partials are all in use
-    layers, Hkv, Hq, D, B, S, W, n = 2, 4, 16, 128, 2, 16, 112, 3000
-    mask = [1, 0, 1, 1, 0, 1, 1, 0]
+    # long rows on few units: most work items begin or end inside a unit, so counters, tickets and
+    # partials are all in use
+    layers, Hkv, Hq, D, B, S, W, n = 2, 4, 32, 128, 8, 16, 112, 3000
+    mask = [1, 0, 1, 1, 1, 1, 1, 1]
     handle = rl.rlkv_cache_create(layers, Hkv, Hq, D, B, n + 8, mask, S, W)
     try:
         for layer in range(layers):
@@ -47,7 +48,7 @@ def test_static_scratch_variant_matches_the_ordinary_call(cuda_device):
             want.append(out)
         outs = [torch.full((B, Hq, D), float("nan"), dtype=torch.float32, device=cuda_device) for _ in qs]
         # The first call on a device asks the runtime for the array's address; with lazy module
-        # loading that is also the moment the driver gives the array its 2 MiB.  Do it once here,
+        # loading that is also the moment the driver gives the array its 4 MiB.  Do it once here,
         # as a host would at start-up, so that the measurement below sees only the calls themselves.
         first = torch.empty((B, Hq, D), dtype=torch.float32, device=cuda_device)
         rl.rlkv_decode_attention_static_scratch(handle, 0, qs[0], first)
@@ -76,13 +77,14 @@ def test_static_scratch_variant_matches_the_ordinary_call(cuda_device):
             rl.rlkv_decode_attention_static_scratch(handle, layers, qs[0], out)
         assert e.value.code == rl.RLKV_EINVAL
 
-        # 2 CTAs per SM at head_dim 128 need more partial records than the array holds: refused, and
-        # the output buffer is not touched
-        assert rl.rlkv_static_scratch_bytes() == 2 << 20
-        rl.rlkv_set_decode_config(handle, 2, 2, 1)
+        # cut into work items of 2 tiles, layer 1 (4 full heads x 8 rows of 47 tiles) has over 500
+        # items of two 4 KiB partial records each, more than the array holds: refused, and the
+        # output buffer is not touched
+        assert rl.rlkv_static_scratch_bytes() == 4 << 20
+        rl.rlkv_set_decode_config(handle, 0, 0, 0, 2)
         marker = torch.full((B, Hq, D), 123.0, dtype=torch.float32, device=cuda_device)
         with pytest.raises(rl.RlkvError) as e:
-            rl.rlkv_decode_attention_static_scratch(handle, 0, qs[0], marker)
+            rl.rlkv_decode_attention_static_scratch(handle, 1, qs[1], marker)
         assert e.value.code == rl.RLKV_ESCRATCH
         torch.cuda.synchronize()
         assert (marker == 123.0).all()
