@@ -102,10 +102,10 @@ int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out
  * rlkv_static_scratch_bytes() bytes (4 MiB) of device memory on every GPU that loads librlkv,
  * held until the process exits.  The call itself allocates and frees nothing.
  *
- * - A launch that needs more than the array holds (batch * kv_heads tickets plus two partial
- *   records of about (q_heads / kv_heads) * (head_dim + 2) floats per work item of the launch;
- *   rlkv_debug_schedule tells how many items a launch has) is refused with RLKV_ESCRATCH and
- *   nothing is launched.  The benchmark shapes (about 900 items of 2 KiB records) fit.
+ * - A launch that needs more than the array holds (batch * kv_heads tickets plus partial records
+ *   of about (q_heads / kv_heads) * (head_dim + 2) floats each; rlkv_debug_schedule tells how many
+ *   records a launch of a given shape may write) is refused with RLKV_ESCRATCH and nothing is
+ *   launched.
  * - The first call on a device looks up the array's device address (one runtime query, kept for
  *   the life of the process; a driver that loads modules lazily gives the array its memory at that
  *   moment); make that first call at start-up, before starting any stream capture.
@@ -163,13 +163,19 @@ int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int c
  * device and copies the words of the most recent launch to words_host (host, 8 * 320 words) and
  * the CTA capacity (320) to *ctas_out; then the switch is applied. */
 int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_host, int* ctas_out);
-/* The work schedule of the decode kernel, host arithmetic only (no GPU): a flat space of `tiles`
- * tiles is cut for `ctas` CTAs into *n_items_out contiguous items whose sizes shrink geometrically
- * down to item_tiles.  starts_out (host, optional, starts_cap >= n_items + 1 ints) receives the
- * first tile of every item and, last, `tiles`.  RLKV_EKERNEL if the schedule's tile->item map
- * disagrees with the starts (a self-check; never expected). */
-int rlkv_debug_schedule(int tiles, int ctas, int item_tiles, int* n_items_out, int* starts_out,
-                        int starts_cap);
+/* The work schedule of the decode kernel, host arithmetic only (no GPU).  full_units units of
+ * tiles_full 64-row tiles and comp_units units of tiles_comp tiles are laid out as one flat tile
+ * space (in bands: the first half of every full unit, then half of the rest, ... then the rest and
+ * the compressed units) and cut for `ctas` CTAs into *n_items_out contiguous work items whose sizes
+ * shrink geometrically down to item_tiles; *n_slots_out is the number of partial-result records a
+ * launch of this shape may write.  Optional outputs (host; `cap` = ints available in starts_out
+ * and 4-int records available in tile_map_out): starts_out[k] = first flat tile of item k, then
+ * the total; tile_map_out[4x..4x+3] = unit, tile inside the unit, consecutive tiles of the unit
+ * from x on, partial record of the segment holding flat tile x.  RLKV_EKERNEL if the schedule's
+ * own maps disagree with each other (a self-check; never expected). */
+int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas,
+                        int item_tiles, int* n_items_out, int* n_slots_out, int* starts_out,
+                        int* tile_map_out, int cap);
 
 const char* rlkv_strerror(int code);
 

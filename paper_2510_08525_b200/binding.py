@@ -40,7 +40,7 @@ SIGNATURES = {
     "rlkv_launch_count": (_ci, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci, _ci]),
     "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
-    "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, ctypes.POINTER(_ci), _vp, _ci]),
+    "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
 }
 
@@ -212,13 +212,18 @@ def rlkv_debug_trace(cache, enable, read=False):
     return words
 
 
-def rlkv_debug_schedule(tiles, ctas, item_tiles):
-    """int32[n_items + 1]: first tile of every work item, then `tiles`."""
-    n = _ci(0)
-    _check(lib.rlkv_debug_schedule(tiles, ctas, item_tiles, ctypes.byref(n), None, 0))
+def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, tile_map=False):
+    """Returns (starts int32[n_items + 1], n_slots) and, with tile_map=True, also int32[T][4]:
+    unit, tile in unit, run, partial record of every flat tile."""
+    n, slots = _ci(0), _ci(0)
+    args = (full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+    _check(lib.rlkv_debug_schedule(*args, ctypes.byref(n), ctypes.byref(slots), None, None, 0))
+    total = full_units * tiles_full + comp_units * tiles_comp
     starts = np.empty(n.value + 1, dtype=np.int32)
-    _check(lib.rlkv_debug_schedule(tiles, ctas, item_tiles, ctypes.byref(n), starts.ctypes.data, starts.size))
-    return starts
+    tmap = np.empty((total, 4), dtype=np.int32) if tile_map else None
+    _check(lib.rlkv_debug_schedule(*args, ctypes.byref(n), ctypes.byref(slots), starts.ctypes.data, _ptr(tmap),
+                                   max(starts.size, total)))
+    return (starts, int(slots.value), tmap) if tile_map else (starts, int(slots.value))
 
 
 def rlkv_strerror(code: int) -> str:

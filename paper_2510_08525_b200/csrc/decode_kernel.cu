@@ -167,12 +167,11 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
 // inside one work item).
 struct SegDesc {
     int out_row;     // first row of the unit's G output rows: b*q_heads + head*G
-    int uid;         // ticket index of the unit
+    int uid;         // unit index over both classes: the ticket index
     int complete;    // the segment is the whole unit: normalise and write out
-    int item, slot;  // where the partial goes otherwise
-    int first_tile;  // flat tile range of the unit
-    int tiles;
+    int pslot;       // partial record the segment goes to otherwise
     int stop;        // no more segments: the epilogue warps leave
+    int pad[3];
 };
 
 // Shared-memory carve-up (dynamic shared memory, base aligned to 1024 bytes for the swizzle).
@@ -194,21 +193,19 @@ struct Smem {
     __host__ __device__ static constexpr size_t bytes(int stages, int group)
     {
         return (size_t)stages * kStageBytes + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
-               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/;
+               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + 2 * 16 * 4 /*partial lists of a unit*/;
     }
 };
 
 // Pool rows of the K and V tile behind flat tile x.
 __device__ __forceinline__ void tile_rows(const DecodeArgs& a, int x, int& krow, int& vrow)
 {
-    if (x < a.full_tiles) {
-        const int unit = x / a.tiles_full, tile = x - unit * a.tiles_full;
-        krow = (int)(a.full_row0 + (long long)unit * 2 * a.rows_full) + tile * kTile;
+    const TilePos p = tile_pos(a.sched, x);
+    if (p.uid < a.sched.U) {
+        krow = (int)(a.full_row0 + (long long)p.uid * 2 * a.rows_full) + p.tile * kTile;
         vrow = krow + a.rows_full;
     } else {
-        const int y = x - a.full_tiles;
-        const int unit = y / a.tiles_comp, tile = y - unit * a.tiles_comp;
-        krow = (int)(a.comp_row0 + (long long)unit * 2 * a.rows_comp) + tile * kTile;
+        krow = (int)(a.comp_row0 + (long long)(p.uid - a.sched.U) * 2 * a.rows_comp) + p.tile * kTile;
         vrow = krow + a.rows_comp;
     }
 }
@@ -250,6 +247,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     volatile int* claim_slot = reinterpret_cast<volatile int*>(item_desc + kItemRing);
     volatile int* ep_flag = claim_slot + 1;
     volatile int* s_abort = claim_slot + 2;
+    int* ep_slot = const_cast<int*>(claim_slot) + 4;   // [16] first partial record of a unit per band
+    int* ep_count = ep_slot + 16;                      // [16] and how many
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -325,7 +324,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
                 if (item >= 0) {
                     u = locate(a, x);
-                    seg_tiles = min(x1 - x, u.tiles - u.tile);
+                    seg_tiles = min(x1 - x, u.pos.run);
                     // Q as the A operand (rows = query heads of the group, rows >= G are zero)
                     uint32_t qa[KS][2];
                     {
@@ -337,7 +336,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                             qa[ks][1] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
                         }
                     }
-                    int valid_left = u.len - u.tile * kTile;  // valid rows from this tile to the unit's end
+                    int valid_left = u.len - u.pos.tile * kTile;  // valid rows from this tile to the unit's end
                     for (int i = 0; alive && i < seg_tiles; ++i, ++cnt, valid_left -= kTile) {
                         if (cnt % NG != grp) continue;
                         const int st = cnt % stages;
@@ -447,14 +446,11 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 }
                 if (warp == 0 && lane == 0) {
                     SegDesc* sd = reinterpret_cast<SegDesc*>(stat_l + S::kWarps * kMaxGroup);
-                    const bool complete = (u.tile == 0 && seg_tiles == u.tiles);
+                    const bool complete = (u.pos.tile == 0 && seg_tiles == u.tiles);
                     sd->out_row = u.b * a.q_heads + u.head * G;
-                    sd->uid = u.uid;
+                    sd->uid = u.pos.uid;
                     sd->complete = complete ? 1 : 0;
-                    sd->item = item;
-                    sd->slot = (x == x0) ? 0 : 1;
-                    sd->first_tile = u.first_tile;
-                    sd->tiles = u.tiles;
+                    sd->pslot = item < 0 ? 0 : partial_slot(sc, u.pos.band, item, u.pos.uid);
                     sd->stop = item < 0 ? 1 : 0;
                     n_tiles += seg_tiles;
                     if (item >= 0 && !complete) ++n_partial;
@@ -562,7 +558,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         constexpr int D4 = D / 4;
         const int et = tid - (S::kWarps + 2) * 32;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-        const size_t slot_stride = (size_t)a.part_items * PF;
+        constexpr int EPT = (kMaxGroup * D4 + NE - 1) / NE;  // 4-float pieces per thread, at most
+        constexpr int CH = 4;                                // partials fetched together per piece
         for (int seg = 0;; ++seg) {
             const int bi = seg % kMergeBuffers;
             const bool got = wait_bounded(smem_u32(ep_full + bi), (uint32_t)(seg / kMergeBuffers) & 1u, s_abort,
@@ -575,7 +572,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             const SegDesc sd = *reinterpret_cast<const SegDesc*>(stat_l + S::kWarps * kMaxGroup);
             if (sd.stop) break;
             float* out_rows = a.out + (size_t)sd.out_row * D;
-            float* my_part = a.partials + (size_t)sd.slot * slot_stride + (size_t)sd.item * PF;
+            float* my_part = a.partials + (size_t)sd.pslot * PF;
             // merge the consumer warps' states; this thread owns a few 4-float pieces of the G x D rows
             for (int e = et; e < G * D4; e += NE) {
                 const int g = e / D4, d4 = e - g * D4;
@@ -608,48 +605,84 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(ep_empty + bi));  // the buffer may be refilled
             if (!sd.complete) {
-                const int first_k = item_of_tile(sc, sd.first_tile);
-                const int last_k = item_of_tile(sc, sd.first_tile + sd.tiles - 1);
+                // the unit's partial records, band by band (lane r of the first epilogue warp looks up band r)
                 __threadfence();
-                epilogue_sync();
-                if (et == 0) {
-                    const int old = atomicAdd(&a.tickets[sd.uid], 1);
-                    *ep_flag = (old == last_k - first_k);
+                if (et < 32) {
+                    int slot = 0, count = 0;
+                    if (et <= sc.R) unit_partials(sc, sd.uid, et, slot, count);
+                    if (et <= kMaxRounds) {
+                        ep_slot[et] = slot;
+                        ep_count[et] = count;
+                    }
+                    int total = count;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+                    epilogue_sync();  // every thread's partial stores are fenced
+                    if (et == 0) {
+                        const int old = atomicAdd(&a.tickets[sd.uid], 1);
+                        *ep_flag = (old == total - 1);
+                    }
+                } else {
+                    epilogue_sync();
                 }
                 epilogue_sync();
                 if (*ep_flag) {
-                    // the last partial of the unit has arrived: merge them in item order, so the
-                    // result does not depend on who arrived when
+                    // the last partial of the unit has arrived: merge them in a fixed order (band by
+                    // band, item by item), so the result does not depend on who arrived when
                     __threadfence();
-                    // the unit's piece of item first_k is that item's first segment only if the item
-                    // starts at or after the unit's first tile; in every later item it is the first
-                    const int slot0 = item_start(sc, first_k) < sd.first_tile ? 1 : 0;
-                    const float* p0 = a.partials + (size_t)slot0 * slot_stride + (size_t)first_k * PF;
-                    const float* p1 = a.partials + (size_t)(first_k + 1) * PF;  // slot 0 of the items after
-                    const int n = last_k - first_k;
-                    for (int e = et; e < G * D4; e += NE) {
-                        const int g = e / D4;
-                        const float m0 = __ldcg(p0 + g);
-                        float M = m0;
-#pragma unroll 8
-                        for (int c = 0; c < n; ++c) M = fmaxf(M, __ldcg(p1 + (size_t)c * PF + g));
-                        float wt = exp2f(m0 - M);
-                        float L = __ldcg(p0 + G + g) * wt;
-                        float4 o = __ldcg(reinterpret_cast<const float4*>(p0 + PH) + e);
-                        float4 O = make_float4(o.x * wt, o.y * wt, o.z * wt, o.w * wt);
-#pragma unroll 8
-                        for (int c = 0; c < n; ++c) {
-                            const float* pc = p1 + (size_t)c * PF;
-                            wt = exp2f(__ldcg(pc + g) - M);
-                            L += __ldcg(pc + G + g) * wt;
-                            o = __ldcg(reinterpret_cast<const float4*>(pc + PH) + e);
-                            O.x += o.x * wt;
-                            O.y += o.y * wt;
-                            O.z += o.z * wt;
-                            O.w += o.w * wt;
+                    float M[EPT], L[EPT];
+                    float4 O[EPT];
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) {
+                        M[j] = kNegBig;
+                        L[j] = 0.f;
+                        O[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    for (int r = 0; r <= sc.R; ++r) {
+                        const float* pr = a.partials + (size_t)ep_slot[r] * PF;
+                        const int n = ep_count[r];
+                        for (int c0 = 0; c0 < n; c0 += CH) {
+                            float mm[EPT][CH], ll[EPT][CH];
+                            float4 oo[EPT][CH];
+                            // all loads of the chunk first, then the arithmetic
+#pragma unroll
+                            for (int j = 0; j < EPT; ++j) {
+                                const int e = et + j * NE;
+                                const int g = e / D4;
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) {
+                                    const bool on = e < G * D4 && c0 + c < n;
+                                    const float* pc = pr + (size_t)(c0 + c) * PF;
+                                    mm[j][c] = on ? __ldcg(pc + g) : kNegBig;
+                                    ll[j][c] = on ? __ldcg(pc + G + g) : 0.f;
+                                    oo[j][c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e)
+                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < EPT; ++j) {
+#pragma unroll
+                                for (int c = 0; c < CH; ++c) {
+                                    const float Mn = fmaxf(M[j], mm[j][c]);
+                                    const float ca = exp2f(M[j] - Mn), cb = exp2f(mm[j][c] - Mn);
+                                    L[j] = L[j] * ca + ll[j][c] * cb;
+                                    O[j].x = O[j].x * ca + oo[j][c].x * cb;
+                                    O[j].y = O[j].y * ca + oo[j][c].y * cb;
+                                    O[j].z = O[j].z * ca + oo[j][c].z * cb;
+                                    O[j].w = O[j].w * ca + oo[j][c].w * cb;
+                                    M[j] = Mn;
+                                }
+                            }
                         }
-                        const float inv = 1.f / L;
-                        *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                    }
+#pragma unroll
+                    for (int j = 0; j < EPT; ++j) {
+                        const int e = et + j * NE;
+                        if (e < G * D4) {
+                            const float inv = 1.f / L[j];
+                            *reinterpret_cast<float4*>(out_rows + e * 4) =
+                                make_float4(O[j].x * inv, O[j].y * inv, O[j].z * inv, O[j].w * inv);
+                        }
                     }
                     if (et == 0) a.tickets[sd.uid] = 0;  // ready for the next launch
                 }

@@ -10,7 +10,7 @@
 //   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
 //   tickets   int32 [layers][batch*kv_heads]   (split bookkeeping, zero between launches)
 //   status    int32 kernel status word, then the two work-claim counters (zero between launches)
-//   partials  float [2][max_items][partial_floats]  (split-KV scratch)
+//   partials  float [max_slots][partial_floats]  (split-KV scratch)
 //   staging   k, v, q, out of one whole step, for rlkv_step_host
 //   trace     uint64 [max_grid][8]  (debug trace of the decode kernel)
 #include <stdio.h>
@@ -57,13 +57,13 @@ constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up t
 constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
 constexpr int kDefaultItemTiles = 4;
 
-// Most work items a decode launch can have when the flat tile space holds at most t_max tiles and
-// the grid at most max_grid CTAs.
-int most_items(long long t_max, int max_grid)
+// Most partial records a decode launch of this shape can write, over every length up to tf tiles
+// per full unit and every grid up to max_grid CTAs.
+long long most_slots(int U, int tf, int Uc, int tc, int max_grid)
 {
-    int most = 0;
-    for (int p = 1; p <= max_grid; ++p) {  // the bound grows with P except for rounding
-        const int m = max_items((int)t_max, p, kMinItemTiles);
+    long long most = 0;
+    for (int p = 1; p <= max_grid; ++p) {
+        const long long m = max_slots(U, tf, Uc, tc, p, kMinItemTiles);
         if (m > most) most = m;
     }
     return most;
@@ -101,15 +101,18 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     if (row >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
     L.max_grid = 2 * kMaxGridSms;
     {
-        // the longest flat tile space is reached at max_len by the layer with the most full heads
-        long long t_max = 0;
+        // partial records: sized for the layer and length that can need the most of them
+        long long most = 0;
         for (int l = 0; l < layers; ++l) {
             const long long t = (long long)batch * (L.n_full[l] * (long long)(L.rows_full / kTile) +
                                                     L.n_comp[l] * (long long)(L.rows_comp / kTile));
-            if (t > t_max) t_max = t;
+            if (t >= (1ll << 31)) return RLKV_EINVAL;
+            const long long m = most_slots(batch * L.n_full[l], L.rows_full / kTile, batch * L.n_comp[l],
+                                           L.rows_comp / kTile, L.max_grid);
+            if (m > most) most = m;
         }
-        if (t_max >= (1ll << 31)) return RLKV_EINVAL;
-        L.max_items = most_items(t_max, L.max_grid);
+        if (most >= (1ll << 31)) return RLKV_EINVAL;
+        L.max_items = (int)most;
     }
     size_t off = 0;
     L.off_pool = off;
@@ -121,7 +124,7 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     L.off_status = off;
     off = align_up(off + 64, 1024);
     L.off_partials = off;
-    off = align_up(off + (size_t)L.max_items * 2 * partial_floats(head_dim, q_heads / kv_heads) * sizeof(float), 1024);
+    off = align_up(off + (size_t)L.max_items * partial_floats(head_dim, q_heads / kv_heads) * sizeof(float), 1024);
     const size_t kv_step = (size_t)layers * batch * kv_heads * head_dim * 2;
     const size_t q_step = (size_t)layers * batch * q_heads * head_dim * 2;
     L.off_k = off;
@@ -289,20 +292,16 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     a.batch = c->batch;
     a.group = c->q_heads / c->kv_heads;
     a.q_heads = c->q_heads;
-    a.tiles_full = (a.len_full + kTile - 1) / kTile;
-    a.tiles_comp = (a.len_comp + kTile - 1) / kTile;
-    a.full_units = c->batch * a.n_full;
-    const long long full_tiles = (long long)a.full_units * a.tiles_full;
-    const long long all_tiles = full_tiles + (long long)c->batch * a.n_comp * a.tiles_comp;
+    const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
+    const long long all_tiles = (long long)c->batch * ((long long)a.n_full * tiles_full + (long long)a.n_comp * tiles_comp);
     if (all_tiles >= (1ll << 31)) return RLKV_EINVAL;
-    a.full_tiles = (int)full_tiles;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
     a.trace_on = c->trace_on;
     // persistent grid; the work items of the flat tile space are cut for that many CTAs and no
     // more CTAs are launched than there are items
     int grid = c->sm_count * c->ctas_per_sm;
     if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    a.sched = make_schedule((int)all_tiles, grid, c->item_tiles);
+    a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * a.n_comp, tiles_comp, grid, c->item_tiles);
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     *grid_out = grid;
     return RLKV_OK;
@@ -314,9 +313,8 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     int grid = 0;
     int rc = build_decode_args(c, layer, q, out, a, &grid);
     if (rc) return rc;
-    if (a.sched.n_items > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
+    if (a.sched.n_slots > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
     a.partials = dev_at<float>(c, c->lay.off_partials);
-    a.part_items = c->lay.max_items;
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
     a.counters = dev_at<int>(c, c->lay.off_status) + 4;
     RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
@@ -357,11 +355,10 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
     int grid = 0;
     int rc = build_decode_args(c, layer, q, out, a, &grid);
     if (rc) return rc;
-    // carve the static array: the two counters and one ticket per (batch row, KV head), then two
-    // partial records per work item of this launch
+    // carve the static array: the two counters and one ticket per (batch row, KV head), then the
+    // partial records of this launch
     const size_t head_bytes = align_up((2 + (size_t)c->batch * c->kv_heads) * sizeof(int), 256);
-    const size_t partial_bytes =
-        (size_t)a.sched.n_items * 2 * partial_floats(c->head_dim, a.group) * sizeof(float);
+    const size_t partial_bytes = (size_t)a.sched.n_slots * partial_floats(c->head_dim, a.group) * sizeof(float);
     if (head_bytes + partial_bytes > kStaticScratchBytes) return RLKV_ESCRATCH;
     unsigned char* base = nullptr;
     rc = static_scratch_address(c->device, &base);
@@ -369,7 +366,6 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
     a.counters = reinterpret_cast<int*>(base);
     a.tickets = a.counters + 2;
     a.partials = reinterpret_cast<float*>(base + head_bytes);
-    a.part_items = a.sched.n_items;
     // the array still holds whatever the previous call (of any cache) left: counters and tickets
     // must start at zero
     RLKV_CUDA(cudaMemsetAsync(base, 0, head_bytes, s));
@@ -699,18 +695,38 @@ int rlkv_debug_trace(rlkv_cache* c, int enable, unsigned long long* words_host, 
     return RLKV_OK;
 }
 
-int rlkv_debug_schedule(int tiles, int ctas, int item_tiles, int* n_items_out, int* starts_out, int starts_cap)
+int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas, int item_tiles,
+                        int* n_items_out, int* n_slots_out, int* starts_out, int* tile_map_out, int cap)
 {
-    if (tiles < 1 || ctas < 1 || item_tiles < 1 || !n_items_out) return RLKV_EINVAL;
-    const Schedule sc = make_schedule(tiles, ctas, item_tiles);
+    if (full_units < 0 || comp_units < 0 || full_units + comp_units < 1 || tiles_full < 1 || tiles_comp < 1 ||
+        ctas < 1 || item_tiles < 1 || !n_items_out || !n_slots_out)
+        return RLKV_EINVAL;
+    if ((long long)full_units * tiles_full + (long long)comp_units * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
+    const Schedule sc = make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
     *n_items_out = sc.n_items;
+    *n_slots_out = sc.n_slots;
+    if (max_slots(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles) < sc.n_slots) return RLKV_EKERNEL;
     if (starts_out) {
-        if (starts_cap < sc.n_items + 1) return RLKV_ENOMEM;
+        if (cap < sc.n_items + 1) return RLKV_ENOMEM;
         for (int k = 0; k <= sc.n_items; ++k) starts_out[k] = item_start(sc, k);
-        // the inverse map must agree with the starts
-        for (int k = 0; k < sc.n_items; ++k)
+        for (int k = 0; k < sc.n_items; ++k)  // the inverse map must agree with the starts
             for (int x = starts_out[k]; x < starts_out[k + 1]; ++x)
                 if (item_of_tile(sc, x) != k) return RLKV_EKERNEL;
+    }
+    if (tile_map_out) {
+        if (cap < sc.T) return RLKV_ENOMEM;
+        for (int x = 0; x < sc.T; ++x) {
+            const TilePos p = tile_pos(sc, x);
+            tile_map_out[4 * x + 0] = p.uid;
+            tile_map_out[4 * x + 1] = p.tile;
+            tile_map_out[4 * x + 2] = p.run;
+            tile_map_out[4 * x + 3] = partial_slot(sc, p.band, item_of_tile(sc, x), p.uid);
+            // the per-unit list of partial records must contain the record of every tile's segment
+            int slot = 0, count = 0;
+            unit_partials(sc, p.uid, p.band, slot, count);
+            if (tile_map_out[4 * x + 3] < slot || tile_map_out[4 * x + 3] >= slot + count) return RLKV_EKERNEL;
+            if (tile_map_out[4 * x + 3] >= sc.n_slots) return RLKV_EKERNEL;
+        }
     }
     return RLKV_OK;
 }

@@ -40,55 +40,72 @@ __host__ __device__ constexpr int partial_floats(int head_dim, int group) {
 }
 
 // ---- work decomposition -------------------------------------------------------------------------
-// Units are (batch row, head-of-class).  The 64-row tiles of all units form one flat space of T
-// tiles: the FULL units first (unit u owns tiles [u*tiles_full, (u+1)*tiles_full)), then the
-// COMPRESSED units (tiles_comp tiles each: sink + ring rows).  The flat space is cut into work
-// items, contiguous tile ranges, by "factoring": round r hands half of what is left to the P CTAs
-// in P equal items, so items shrink geometrically (few split points while everything is busy,
-// fine grain at the end); once an item would fall under 2*min_sz tiles the rest is cut into items
-// of min_sz tiles.  CTA c starts with item c; later items are claimed from an atomic counter, so a
-// CTA on a slow path to memory simply takes fewer of them.  An item may begin and end inside a
-// unit: such a segment yields an (m, l, O) partial and the last CTA to deliver a partial of a unit
-// merges them.
+// Units are (batch row, head-of-class): U FULL units of tf 64-row tiles each and Uc COMPRESSED
+// units of tc tiles each (sink + ring rows).  Their tiles form one flat space of T tiles, laid out
+// in BANDS: band 0 holds the first half of the tiles of every full unit (unit after unit), band 1
+// half of what is left of every unit, and so on; the last band holds the rest of every full unit
+// and, after them, the compressed units.  The space is cut into work items, contiguous tile
+// ranges, by "factoring": band r < R is handed to the P CTAs in P equal items, so items shrink
+// geometrically (few split points while everything is busy, fine grain at the end); the last band
+// is cut into items of min_sz tiles.  CTA c starts with item c; later items are claimed from an
+// atomic counter, so a CTA on a slow path to memory simply takes fewer of them.
+// A SEGMENT is the part of one unit inside one item (a run of consecutive tiles of the unit).  A
+// segment that is not the whole unit yields an (m, l, O) partial; the last CTA to deliver a
+// partial of a unit merges them.  Because every unit has a slice in every band, every unit ends
+// up with a similar, small number of partials.
 struct Schedule {
-    int T;                      // tiles in the flat space
     int P;                      // CTAs
-    int R;                      // factoring rounds
-    int min_sz;                 // tiles per item in the final section
+    int R;                      // bands handed out in P equal items (the factoring rounds)
+    int min_sz;                 // tiles per item in the last band
     int n_items;
-    int base[kMaxRounds + 1];   // first tile of round r; base[R] = first tile of the final section
-    int len[kMaxRounds];        // tiles handed out in round r
+    int n_slots;                // partial records the launch may write
+    int U, tf, Uc, tc;
+    int T;                      // tiles in the flat space
+    int base[kMaxRounds + 2];   // first flat tile of band r <= R; base[R+1]: first compressed tile
+    int tb[kMaxRounds + 2];     // first tile, inside a full unit, of its slice in band r; tb[R+1] = tf
+    int slot0[kMaxRounds + 1];  // first partial record of band r
 };
 
-inline Schedule make_schedule(int T, int P, int min_sz)
+inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz)
 {
     Schedule s{};
-    s.T = T;
     s.P = P;
     s.min_sz = min_sz;
+    s.U = U;
+    s.tf = U > 0 ? tf : 0;
+    s.Uc = Uc;
+    s.tc = Uc > 0 ? tc : 0;
     int r = 0;
     s.base[0] = 0;
+    s.tb[0] = 0;
     while (r < kMaxRounds) {
-        const int rem = T - s.base[r];
-        const int len = rem / 2;
-        if (len / P < 2 * min_sz) break;
-        s.len[r] = len;
-        s.base[r + 1] = s.base[r] + len;
+        const int bw = (s.tf - s.tb[r]) / 2;
+        if ((long long)U * bw / P < 2 * min_sz) break;
+        s.tb[r + 1] = s.tb[r] + bw;
+        s.base[r + 1] = s.base[r] + U * bw;
+        s.slot0[r] = r * (P + U);
         ++r;
     }
     s.R = r;
-    const int rem = T - s.base[r];
-    s.n_items = r * P + (rem + min_sz - 1) / min_sz;
+    s.slot0[r] = r * (P + U);
+    s.tb[r + 1] = s.tf;
+    s.base[r + 1] = s.base[r] + U * (s.tf - s.tb[r]);
+    s.T = s.base[r + 1] + s.Uc * s.tc;
+    const int n_final = (s.T - s.base[r] + min_sz - 1) / min_sz;
+    s.n_items = r * P + n_final;
+    s.n_slots = s.slot0[r] + n_final + U + Uc;
     return s;
 }
 
-// Upper bound of n_items over every T' <= T with the same P and min_sz.
-inline int max_items(int T, int P, int min_sz)
+// Upper bound of n_slots over every tf' <= tf with everything else the same.
+inline long long max_slots(int U, int tf, int Uc, int tc, int P, int min_sz)
 {
-    const Schedule s = make_schedule(T, P, min_sz);
-    // the final section holds fewer than 4*min_sz*P + 2 tiles unless the rounds ran out first
-    const int by_size = 4 * P + 2, by_rounds = (T >> kMaxRounds) / min_sz + 2;
-    return (s.R + 1) * P + (by_size > by_rounds ? by_size : by_rounds);
+    const Schedule s = make_schedule(U, tf, Uc, tc, P, min_sz);
+    // tiles of the last band: under 4*min_sz*P + 2U unless the rounds ran out first
+    const long long by_size = 4ll * min_sz * P + 2ll * U;
+    const long long by_rounds = (long long)U * ((tf >> kMaxRounds) + 2);
+    const long long last = (by_size > by_rounds ? by_size : by_rounds) + (long long)Uc * tc;
+    return (long long)s.R * (P + U) + last / min_sz + U + Uc + 4;
 }
 
 // First tile of item k (k >= n_items gives T).
@@ -98,7 +115,7 @@ __host__ __device__ inline int item_start(const Schedule& s, int k)
     const int rp = s.R * s.P;
     if (k < rp) {
         const int r = k / s.P, j = k - r * s.P;
-        return s.base[r] + (int)(((long long)j * s.len[r]) / s.P);
+        return s.base[r] + (int)(((long long)j * (s.base[r + 1] - s.base[r])) / s.P);
     }
     return s.base[s.R] + (k - rp) * s.min_sz;
 }
@@ -108,8 +125,70 @@ __host__ __device__ inline int item_of_tile(const Schedule& s, int x)
 {
     for (int r = 0; r < s.R; ++r)
         if (x < s.base[r + 1])
-            return r * s.P + (int)((((long long)(x - s.base[r]) + 1) * s.P - 1) / s.len[r]);
+            return r * s.P + (int)((((long long)(x - s.base[r]) + 1) * s.P - 1) / (s.base[r + 1] - s.base[r]));
     return s.R * s.P + (x - s.base[s.R]) / s.min_sz;
+}
+
+// Where flat tile x lies: the unit (index over both classes, full units first), the tile inside
+// the unit, how many tiles of the unit follow consecutively in the flat space from x on (x
+// included), and the band.
+struct TilePos {
+    int uid, tile, run, band;
+};
+__host__ __device__ inline TilePos tile_pos(const Schedule& s, int x)
+{
+    TilePos p;
+    if (x < s.base[s.R + 1]) {
+        int r = s.R;
+        for (int i = 0; i < s.R; ++i)
+            if (x < s.base[i + 1]) {
+                r = i;
+                break;
+            }
+        const int bw = s.tb[r + 1] - s.tb[r], y = x - s.base[r];
+        const int unit = y / bw, off = y - unit * bw;
+        p.uid = unit;
+        p.tile = s.tb[r] + off;
+        p.run = bw - off;
+        p.band = r;
+    } else {
+        const int y = x - s.base[s.R + 1];
+        const int unit = y / s.tc, off = y - unit * s.tc;
+        p.uid = s.U + unit;
+        p.tile = off;
+        p.run = s.tc - off;
+        p.band = s.R;
+    }
+    return p;
+}
+
+// The partial record of the segment of unit `uid` inside item `item` of band `band`: along a band
+// every new segment raises the item index or the unit index, so their sum numbers the segments.
+__host__ __device__ inline int partial_slot(const Schedule& s, int band, int item, int uid)
+{
+    return s.slot0[band] + (item - band * s.P) + uid;
+}
+
+// The partial records of unit `uid` in band `band`: first record and how many (0 if the unit has
+// no slice there).  Full units have a slice in every band, compressed units only in the last.
+__host__ __device__ inline void unit_partials(const Schedule& s, int uid, int band, int& slot, int& count)
+{
+    int first, width;
+    if (uid < s.U) {
+        width = s.tb[band + 1] - s.tb[band];
+        first = s.base[band] + uid * width;
+    } else {
+        width = band == s.R ? s.tc : 0;
+        first = s.base[s.R + 1] + (uid - s.U) * s.tc;
+    }
+    if (width <= 0) {
+        slot = 0;
+        count = 0;
+        return;
+    }
+    const int kf = item_of_tile(s, first), kl = item_of_tile(s, first + width - 1);
+    slot = partial_slot(s, band, kf, uid);
+    count = kl - kf + 1;
 }
 
 // Everything a decode launch needs about one layer.  Passed by value.
@@ -120,8 +199,7 @@ struct DecodeArgs {
     const int* head_of_slot;    // [kv_heads]: KV head of full slot 0..n_full-1, then of comp slots
     const __nv_bfloat16* q;     // [batch][q_heads][head_dim]
     float* out;                 // [batch][q_heads][head_dim]
-    float* partials;            // [2 slots][part_items][partial_floats]
-    long long part_items;       // items the partial area is laid out for (>= sched.n_items)
+    float* partials;            // [sched.n_slots][partial_floats]
     int* tickets;               // one per unit of this layer, zero between launches
     int* counters;              // [0] items claimed beyond the first P, [1] CTAs finished; zero between launches
     int* status;                // device error word
@@ -130,9 +208,6 @@ struct DecodeArgs {
     int rows_full, rows_comp;   // allocated rows per head (multiples of kTile)
     int len_full, len_comp;     // valid rows per head right now: n and min(n, sink+window)
     int batch, group, q_heads;
-    int tiles_full, tiles_comp; // ceil(len / kTile) per head of each class
-    int full_tiles;             // batch*n_full*tiles_full: where the compressed units start
-    int full_units;             // batch*n_full
     float scale_log2;           // log2(e) / sqrt(head_dim)
     int trace_on;
     Schedule sched;
@@ -150,38 +225,29 @@ struct AppendArgs {
     int sink, window;
 };
 
+// What a consumer needs to know about the unit behind a flat tile.
 struct UnitInfo {
-    int uid;         // unit index over both classes (full units first): the ticket index
-    int tile;        // tile index inside the unit
+    TilePos pos;
     int tiles;       // tiles of the unit
     int len;         // valid rows of the unit
     int b, head;     // batch row, KV head
-    int first_tile;  // flat index of the unit's tile 0
 };
 
-// The unit and tile behind flat tile x.
 __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
 {
     UnitInfo u;
-    if (x < a.full_tiles) {
-        const int unit = x / a.tiles_full;
-        u.uid = unit;
-        u.tile = x - unit * a.tiles_full;
-        u.tiles = a.tiles_full;
+    u.pos = tile_pos(a.sched, x);
+    if (u.pos.uid < a.sched.U) {
+        u.tiles = a.sched.tf;
         u.len = a.len_full;
-        u.b = unit / a.n_full;
-        u.head = a.head_of_slot[unit - u.b * a.n_full];
-        u.first_tile = unit * a.tiles_full;
+        u.b = u.pos.uid / a.n_full;
+        u.head = a.head_of_slot[u.pos.uid - u.b * a.n_full];
     } else {
-        const int y = x - a.full_tiles;
-        const int unit = y / a.tiles_comp;
-        u.uid = a.full_units + unit;
-        u.tile = y - unit * a.tiles_comp;
-        u.tiles = a.tiles_comp;
+        const int unit = u.pos.uid - a.sched.U;
+        u.tiles = a.sched.tc;
         u.len = a.len_comp;
         u.b = unit / a.n_comp;
         u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
-        u.first_tile = a.full_tiles + unit * a.tiles_comp;
     }
     return u;
 }

@@ -1,6 +1,7 @@
-"""Host logic of the decode kernel's work schedule (no GPU): the items partition the flat tile
-space in order, shrink geometrically round by round, end in items of the requested size, and the
-tile -> item map used by the split merge is the inverse of the item starts."""
+"""Host logic of the decode kernel's work schedule (no GPU): the banded flat tile space covers every
+tile of every unit exactly once, the work items partition it in order and shrink geometrically,
+every segment (the part of one unit inside one item) has a partial record of its own, and every
+unit ends up with a small number of them."""
 import numpy as np
 import pytest
 
@@ -13,38 +14,69 @@ def rl():
     return b
 
 
-@pytest.mark.parametrize("tiles,ctas,item", [
-    (1, 148, 4), (3, 148, 4), (5, 1, 2), (147, 148, 4), (148, 148, 4), (1000, 148, 4), (2367, 148, 4),
-    (13209, 148, 4), (13209, 296, 2), (13260, 148, 8), (131072, 148, 4), (524800, 296, 4), (40000, 7, 3),
-    (3000000, 148, 2),
-])
-def test_items_partition_the_tile_space(rl, tiles, ctas, item):
-    starts = rl.rlkv_debug_schedule(tiles, ctas, item)     # the library also checks the inverse map
-    assert starts[0] == 0 and starts[-1] == tiles
+SHAPES = [
+    # full units, tiles each, compressed units, tiles each, CTAs, item tiles
+    (1, 1, 0, 1, 148, 4), (0, 1, 3, 2, 148, 4), (1, 9, 1, 1, 148, 4), (2, 47, 2, 2, 148, 4),
+    (102, 129, 26, 2, 148, 4), (102, 129, 26, 2, 296, 2), (51, 257, 77, 2, 148, 4), (38, 65, 26, 4, 148, 4),
+    (512, 33, 0, 2, 148, 4), (8, 1025, 56, 2, 148, 4), (7, 300, 5, 3, 7, 3), (512, 1025, 0, 2, 296, 4),
+    (24, 47, 8, 2, 148, 9), (3, 2, 200, 2, 148, 2),
+]
+
+
+@pytest.mark.parametrize("U,tf,Uc,tc,ctas,item", SHAPES)
+def test_banded_schedule(rl, U, tf, Uc, tc, ctas, item):
+    starts, n_slots, tmap = rl.rlkv_debug_schedule(U, tf, Uc, tc, ctas, item, tile_map=True)
+    T = U * tf + Uc * tc
+    # ---- items partition the flat space in order
+    assert starts[0] == 0 and starts[-1] == T
     sizes = np.diff(starts)
-    assert (sizes >= 1).all()                               # no empty item, strictly increasing starts
+    assert (sizes >= 1).all()
     n_items = sizes.size
-    # factoring rounds: `ctas` near-equal items of at least 2*item tiles each
     rounds = 0
     while (rounds + 1) * ctas <= n_items and sizes[rounds * ctas:(rounds + 1) * ctas].min() >= 2 * item:
         rounds += 1
-    # the final section: items of exactly `item` tiles (the last one may be shorter)
     tail = sizes[rounds * ctas:]
-    if tail.size:
+    if tail.size:                                           # last band: items of exactly `item` tiles
         assert (tail[:-1] == item).all() and 1 <= tail[-1] <= item
-    # each round hands out half of what is left
-    left = tiles
-    for r in range(rounds):
+    for r in range(rounds):                                 # earlier bands: near-equal items, shrinking
         part = sizes[r * ctas:(r + 1) * ctas]
-        assert part.sum() == left // 2 and part.max() - part.min() <= 1
-        left -= part.sum()
-    assert tail.sum() == left
-    # few items while everything is busy, fine grain at the end
-    assert n_items <= 14 * ctas + 2 or tiles > (1 << 20)
+        assert part.max() - part.min() <= 1
+        if r:
+            assert part.max() <= sizes[(r - 1) * ctas:r * ctas].max()
+    # ---- every tile of every unit exactly once
+    uid, tile, run, slot = tmap[:, 0], tmap[:, 1], tmap[:, 2], tmap[:, 3]
+    want = [(u, t) for u in range(U) for t in range(tf)] + [(U + u, t) for u in range(Uc) for t in range(tc)]
+    assert sorted(zip(uid.tolist(), tile.tolist())) == want
+    # ---- runs: from x on, `run` consecutive flat tiles are consecutive tiles of the same unit, and
+    # the run ends where the unit's slice ends
+    for x in range(T):
+        assert run[x] >= 1
+        if run[x] > 1:
+            assert uid[x + 1] == uid[x] and tile[x + 1] == tile[x] + 1 and run[x + 1] == run[x] - 1
+        elif x + 1 < T:
+            assert (uid[x + 1], tile[x + 1]) != (uid[x], tile[x] + 1) or x + 1 == T
+    # ---- segments and their partial records
+    item_of = np.repeat(np.arange(n_items), sizes)
+    new_seg = np.ones(T, bool)
+    new_seg[1:] = (item_of[1:] != item_of[:-1]) | (uid[1:] != uid[:-1]) | (tile[1:] != tile[:-1] + 1)
+    seg_id = np.cumsum(new_seg) - 1
+    seg_slot = {}
+    for x in range(T):
+        seg_slot.setdefault(int(seg_id[x]), set()).add(int(slot[x]))
+    assert all(len(v) == 1 for v in seg_slot.values())                  # one record per segment
+    slots = [next(iter(v)) for v in seg_slot.values()]
+    assert len(set(slots)) == len(slots)                                # and no two segments share one
+    assert max(slots) < n_slots
+    # ---- every unit is split into few segments: a handful per band, not one per small item
+    per_unit = np.bincount(uid[new_seg], minlength=U + Uc)
+    last_band_tiles = tf / 2 ** rounds + 1
+    per_band = ctas / max(U, 1) + 2                     # a band of a unit spans about P/U items
+    assert per_unit.max() <= rounds * per_band + last_band_tiles / item + 3, (per_unit.max(), rounds)
 
 
 def test_schedule_rejects_bad_arguments(rl):
-    for bad in ((0, 148, 4), (10, 0, 4), (10, 148, 0)):
+    for bad in ((0, 1, 0, 1, 148, 4), (1, 0, 0, 1, 148, 4), (1, 1, 1, 0, 148, 4), (1, 1, 0, 1, 0, 4),
+                (1, 1, 0, 1, 148, 0), (-1, 1, 2, 1, 148, 4)):
         with pytest.raises(rl.RlkvError) as e:
             rl.rlkv_debug_schedule(*bad)
         assert e.value.code == rl.RLKV_EINVAL

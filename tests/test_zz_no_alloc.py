@@ -32,7 +32,7 @@ def test_static_scratch_variant_matches_the_ordinary_call(cuda_device):
 
     # long rows on few units: most work items begin or end inside a unit, so counters, tickets and
     # partials are all in use
-    layers, Hkv, Hq, D, B, S, W, n = 2, 4, 32, 128, 8, 16, 112, 3000
+    layers, Hkv, Hq, D, B, S, W, n = 2, 4, 32, 128, 16, 16, 112, 6000
     mask = [1, 0, 1, 1, 1, 1, 1, 1]
     handle = rl.rlkv_cache_create(layers, Hkv, Hq, D, B, n + 8, mask, S, W)
     try:
@@ -77,9 +77,9 @@ def test_static_scratch_variant_matches_the_ordinary_call(cuda_device):
             rl.rlkv_decode_attention_static_scratch(handle, layers, qs[0], out)
         assert e.value.code == rl.RLKV_EINVAL
 
-        # cut into work items of 2 tiles, layer 1 (4 full heads x 8 rows of 47 tiles) has over 500
-        # items of two 4 KiB partial records each, more than the array holds: refused, and the
-        # output buffer is not touched
+        # cut into work items of 2 tiles, layer 1 (4 full heads x 16 rows of 94 tiles) may write over
+        # 1000 partial records of 4 KiB, more than the array holds: refused, and the output buffer
+        # is not touched
         assert rl.rlkv_static_scratch_bytes() == 4 << 20
         rl.rlkv_set_decode_config(handle, 0, 0, 0, 2)
         marker = torch.full((B, Hq, D), 123.0, dtype=torch.float32, device=cuda_device)
