@@ -156,12 +156,17 @@ int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
  * 4 tiles.  Results do not depend on these knobs beyond floating-point summation order. */
 int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups,
                            int item_tiles);
-/* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, eight
- * 64-bit words: %globaltimer (ns) at CTA start, when its first tile landed, when its last segment
- * was handed off and at CTA end; the work items, tiles and partial segments it processed; and
- * %globaltimer when its epilogue warps finished.  words_host != NULL: first synchronises the
- * device and copies the words of the most recent launch to words_host (host, 8 * 320 words) and
- * the CTA capacity (320) to *ctas_out; then the switch is applied. */
+/* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, 32
+ * 64-bit words: [0..3] %globaltimer (ns) at CTA start, when its first tile landed, when its last
+ * segment was handed off and at CTA end; [4..6] work items, tiles and partial segments it
+ * processed; [7] %globaltimer when its epilogue warps finished; [8..10] ns its first consumer warp
+ * waited for work items, for tiles and for a free hand-off buffer; [11] ns its epilogue warps were
+ * idle; [12..13] split merges its epilogue warps ran at once and the ns they took; [14..15] ns its
+ * producer waited for the next work item's number and for a free descriptor; [16..31] for its
+ * first 16 work items, (%globaltimer << 16) | (item & 0xffff) when the consumers started it.
+ * words_host != NULL: first synchronises the device and copies the words of the most recent launch
+ * to words_host (host, 32 * 320 words) and the CTA capacity (320) to *ctas_out; then the switch is
+ * applied. */
 int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_host, int* ctas_out);
 /* The work schedule of the decode kernel, host arithmetic only (no GPU).  full_units units of
  * tiles_full 64-row tiles and comp_units units of tiles_comp tiles are laid out as one flat tile

@@ -162,6 +162,17 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     }
 }
 
+// wait_bounded that also adds the time spent waiting to *ns when the trace is on (one thread's view).
+__device__ __forceinline__ bool wait_traced(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                            int code, bool on, unsigned long long* ns)
+{
+    if (!on) return wait_bounded(bar, parity, abort_flag, status, code);
+    const uint64_t t = global_timer_ns();
+    const bool ok = wait_bounded(bar, parity, abort_flag, status, code);
+    *ns += global_timer_ns() - t;
+    return ok;
+}
+
 // ---------------------------------------------------------------------------------------------
 // What the consumer warps tell the epilogue warps about a finished segment (the part of one unit
 // inside one work item).
@@ -193,7 +204,8 @@ struct Smem {
     __host__ __device__ static constexpr size_t bytes(int stages, int group)
     {
         return (size_t)stages * kStageBytes + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
-               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + 2 * 16 * 4 /*partial lists of a unit*/;
+               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + 2 * 16 * 4 /*partial lists of a unit*/ +
+               kMaxTodo * 8 /*split merges put off*/;
     }
 };
 
@@ -249,6 +261,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     volatile int* s_abort = claim_slot + 2;
     int* ep_slot = const_cast<int*>(claim_slot) + 4;   // [16] first partial record of a unit per band
     int* ep_count = ep_slot + 16;                      // [16] and how many
+    int2* todo = reinterpret_cast<int2*>(ep_count + 16);  // [kMaxTodo] (unit, first output row)
+    volatile int* todo_count = claim_slot + 3;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -277,6 +291,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         }
         *ep_flag = 0;
         *s_abort = 0;
+        *todo_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -298,12 +313,15 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         int di = 0;
         uint32_t dpar = 0;
         int n_items = 0, n_tiles = 0, n_partial = 0;  // trace counters
+        unsigned long long ns_item = 0, ns_tile = 0, ns_merge = 0;
+        const bool tr0 = trace && tid == 0;
         bool landed = false, alive = true;
         while (alive) {
-            if (!wait_bounded(smem_u32(item_full + di), dpar, s_abort, a.status, kStatusItemWaitTimeout)) break;
+            if (!wait_traced(smem_u32(item_full + di), dpar, s_abort, a.status, kStatusItemWaitTimeout, tr0, &ns_item)) break;
             const int4 desc = item_desc[di];
             const int item = desc.x, x0 = desc.y, x1 = desc.z;
             if (item >= 0) {
+                if (tr0 && n_items < 16) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
                 // skip the empty slots the producer issued to line the slot counter up with x0
                 for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, ++cnt) {
@@ -340,8 +358,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     for (int i = 0; alive && i < seg_tiles; ++i, ++cnt, valid_left -= kTile) {
                         if (cnt % NG != grp) continue;
                         const int st = cnt % stages;
-                        alive = wait_bounded(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort,
-                                             a.status, kStatusFullWaitTimeout);
+                        alive = wait_traced(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort,
+                                            a.status, kStatusFullWaitTimeout, tr0, &ns_tile);
                         if (!alive) break;
                         if (trace && tid == 0 && !landed) {
                             my_trace[1] = global_timer_ns();
@@ -415,8 +433,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
 
                 // ---- hand the warp's state (or the stop message) to the epilogue warps
                 const int bi = seg % kMergeBuffers;
-                alive = wait_bounded(smem_u32(ep_empty + bi), ((uint32_t)(seg / kMergeBuffers) & 1u) ^ 1u, s_abort,
-                                     a.status, kStatusMergeWaitTimeout);
+                alive = wait_traced(smem_u32(ep_empty + bi), ((uint32_t)(seg / kMergeBuffers) & 1u) ^ 1u, s_abort,
+                                    a.status, kStatusMergeWaitTimeout, tr0, &ns_merge);
                 if (!alive) break;
                 uint8_t* buf = buffers + (size_t)bi * buffer_bytes;
                 float* merge = reinterpret_cast<float*>(buf);
@@ -477,6 +495,9 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             my_trace[4] = (unsigned long long)n_items;
             my_trace[5] = (unsigned long long)n_tiles;
             my_trace[6] = (unsigned long long)n_partial;
+            my_trace[8] = ns_item;
+            my_trace[9] = ns_tile;
+            my_trace[10] = ns_merge;
         }
     } else if (warp == S::kWarps) {
         // ------------------------------------------------------------------ producer warp
@@ -485,11 +506,16 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             int s = 0, di = 0;
             uint32_t par = 0, dpar = 0, cpar = 0;
             bool ok = true;
+            unsigned long long ns_claim = 0, ns_ring = 0;
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             while (ok && k < sc.n_items) {
-                mbar_arrive(smem_u32(claim_empty));  // ask the claim warp for the item after this one
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
-                ok = wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout);
+                // ask the claim warp for the next item only shortly before this one is issued in
+                // full: early enough to hide the round trip, late enough that a CTA is never
+                // committed to more than the tiles in its ring plus a few
+                const int x_ask = max(x0, x1 - kClaimAhead);
+                ok = wait_traced(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout, trace,
+                                 &ns_ring);
                 if (!ok) break;
                 item_desc[di] = make_int4(k, x0, x1, 0);
                 mbar_arrive(smem_u32(item_full + di));  // release: the descriptor is visible to the waiters
@@ -509,6 +535,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     }
                 }
                 for (int x = x0; ok && x < x1; ++x) {
+                    if (x == x_ask) mbar_arrive(smem_u32(claim_empty));
                     int krow, vrow;
                     tile_rows(a, x, krow, vrow);
                     ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
@@ -530,13 +557,17 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     }
                 }
                 if (!ok) break;
-                ok = wait_bounded(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout);
+                ok = wait_traced(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout, trace, &ns_claim);
                 cpar ^= 1u;
                 if (ok) k = *claim_slot;
             }
             if (ok && wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout)) {
                 item_desc[di] = make_int4(-1, 0, 0, 0);  // no more work
                 mbar_arrive(smem_u32(item_full + di));
+            }
+            if (trace) {
+                my_trace[14] = ns_claim;
+                my_trace[15] = ns_ring;
             }
         }
     } else if (warp == S::kWarps + 1) {
@@ -560,10 +591,13 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
         constexpr int EPT = (kMaxGroup * D4 + NE - 1) / NE;  // 4-float pieces per thread, at most
         constexpr int CH = 4;                                // partials fetched together per piece
+        unsigned long long ns_idle = 0, ns_final = 0, n_final = 0;
+        int todo_n = 0;  // split merges put off so far (same value in every epilogue thread)
+        const bool tre = trace && et == 0;
         for (int seg = 0;; ++seg) {
             const int bi = seg % kMergeBuffers;
-            const bool got = wait_bounded(smem_u32(ep_full + bi), (uint32_t)(seg / kMergeBuffers) & 1u, s_abort,
-                                          a.status, kStatusMergeWaitTimeout);
+            const bool got = wait_traced(smem_u32(ep_full + bi), (uint32_t)(seg / kMergeBuffers) & 1u, s_abort,
+                                         a.status, kStatusMergeWaitTimeout, tre, &ns_idle);
             if (epilogue_or(!got)) break;
             const uint8_t* buf = buffers + (size_t)bi * buffer_bytes;
             const float* merge = reinterpret_cast<const float*>(buf);
@@ -620,15 +654,21 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     epilogue_sync();  // every thread's partial stores are fenced
                     if (et == 0) {
                         const int old = atomicAdd(&a.tickets[sd.uid], 1);
-                        *ep_flag = (old == total - 1);
+                        *ep_flag = (old == total - 1) ? total : 0;  // the unit's number of partials if this was the last
                     }
                 } else {
                     epilogue_sync();
                 }
                 epilogue_sync();
-                if (*ep_flag) {
+                if (*ep_flag > 0 && *ep_flag <= kMaxFlat && todo_n < kMaxTodo) {
+                    // the last partial of the unit has arrived: the merge waits until this CTA's
+                    // stream has ended, when all its warps are free to do it
+                    if (et == 0) todo[todo_n] = make_int2(sd.uid, sd.out_row);
+                    ++todo_n;
+                } else if (*ep_flag) {
                     // the last partial of the unit has arrived: merge them in a fixed order (band by
                     // band, item by item), so the result does not depend on who arrived when
+                    const uint64_t t_final = tre ? global_timer_ns() : 0;
                     __threadfence();
                     float M[EPT], L[EPT];
                     float4 O[EPT];
@@ -685,12 +725,93 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                         }
                     }
                     if (et == 0) a.tickets[sd.uid] = 0;  // ready for the next launch
+                    if (tre) {
+                        ns_final += global_timer_ns() - t_final;
+                        ++n_final;
+                    }
                 }
             }
         }
-        if (trace && et == 0) my_trace[7] = global_timer_ns();
+        if (et == 0) *todo_count = todo_n;
+        if (tre) {
+            my_trace[7] = global_timer_ns();
+            my_trace[11] = ns_idle;
+            my_trace[12] = n_final;
+            my_trace[13] = ns_final;
+        }
     }
     __syncthreads();
+    // ---- the split merges this CTA put off.  The tile ring is idle now and serves as scratch.
+    // Thread (piece e, lane ul) merges piece e of the units ul, ul + lanes, ...: all partial
+    // records of a unit are fetched together, so a unit costs about one trip to the L2.
+    const int n_todo = *todo_count;
+    if (!*s_abort && n_todo > 0) {
+        constexpr int NT = S::kThreads, D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
+        const int E = G * D4;                        // 4-float pieces of a unit's output rows
+        const int unit_lanes = NT / E > 0 ? NT / E : 1;
+        const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+        int2* lists = reinterpret_cast<int2*>(stage_base);        // [kMaxTodo][NB] (first record, count) per band
+        int* flat = reinterpret_cast<int*>(lists + kMaxTodo * NB);  // [kMaxTodo][kMaxFlat] records in merge order
+        for (int p = tid; p < n_todo * (sc.R + 1); p += NT) {
+            const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
+            int slot = 0, count = 0;
+            unit_partials(sc, todo[i].x, r, slot, count);
+            lists[i * NB + r] = make_int2(slot, count);
+        }
+        __syncthreads();
+        for (int p = tid; p < n_todo * kMaxFlat; p += NT) {
+            const int i = p / kMaxFlat;
+            int j = p - i * kMaxFlat, rec = -1;
+            for (int r = 0; r <= sc.R; ++r) {
+                const int2 l = lists[i * NB + r];
+                if (j < l.y) {
+                    rec = l.x + j;
+                    break;
+                }
+                j -= l.y;
+            }
+            flat[p] = rec;  // -1 past the unit's last record
+        }
+        __syncthreads();
+        __threadfence();
+        const int e = tid % E, ul = tid / E;
+        if (ul < unit_lanes) {
+            const int g = e / D4;
+            for (int i = ul; i < n_todo; i += unit_lanes) {
+                const int* fl = flat + i * kMaxFlat;
+                float M = kNegBig, L = 0.f;
+                float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int c0 = 0; c0 < kMaxFlat && fl[c0] >= 0; c0 += CH) {
+                    float mm[CH], ll[CH];
+                    float4 oo[CH];
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {  // all loads first, then the arithmetic
+                        const int rec = c0 + c < kMaxFlat ? fl[c0 + c] : -1;
+                        const bool on = rec >= 0;
+                        const float* pc = a.partials + (size_t)(on ? rec : 0) * PF;
+                        mm[c] = on ? __ldcg(pc + g) : kNegBig;
+                        ll[c] = on ? __ldcg(pc + G + g) : 0.f;
+                        oo[c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const float Mn = fmaxf(M, mm[c]);
+                        const float ca = exp2f(M - Mn), cb = exp2f(mm[c] - Mn);
+                        L = L * ca + ll[c] * cb;
+                        O.x = O.x * ca + oo[c].x * cb;
+                        O.y = O.y * ca + oo[c].y * cb;
+                        O.z = O.z * ca + oo[c].z * cb;
+                        O.w = O.w * ca + oo[c].w * cb;
+                        M = Mn;
+                    }
+                }
+                const float inv = 1.f / L;
+                *reinterpret_cast<float4*>(a.out + (size_t)todo[i].y * D + e * 4) =
+                    make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+            }
+        }
+        if (tid < n_todo) a.tickets[todo[tid].x] = 0;  // ready for the next launch
+    }
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
             // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
