@@ -205,7 +205,7 @@ struct Smem {
     {
         return (size_t)stages * kStageBytes + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + 2 * 16 * 4 /*partial lists of a unit*/ +
-               kMaxTodo * 8 /*split merges put off*/;
+               kMaxPend * 8 /*partial segments whose tickets are still to be drawn*/;
     }
 };
 
@@ -261,8 +261,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     volatile int* s_abort = claim_slot + 2;
     int* ep_slot = const_cast<int*>(claim_slot) + 4;   // [16] first partial record of a unit per band
     int* ep_count = ep_slot + 16;                      // [16] and how many
-    int2* todo = reinterpret_cast<int2*>(ep_count + 16);  // [kMaxTodo] (unit, first output row)
-    volatile int* todo_count = claim_slot + 3;
+    int2* pend = reinterpret_cast<int2*>(ep_count + 16);  // [kMaxPend] (unit, first output row) of partial segments
+    volatile int* pend_count = claim_slot + 3;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -291,7 +291,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         }
         *ep_flag = 0;
         *s_abort = 0;
-        *todo_count = 0;
+        *pend_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -343,6 +343,26 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 if (item >= 0) {
                     u = locate(a, x);
                     seg_tiles = min(x1 - x, u.pos.run);
+                    if (warp == 0) {
+                        // pull the query rows of the segment after this one into the L1 now, so that
+                        // its start does not wait for them
+                        int xn = x + seg_tiles;
+                        if (xn >= x1) {
+                            const int dn = di + 1 == kItemRing ? 0 : di + 1;
+                            xn = -1;
+                            if (mbar_try_wait(smem_u32(item_full + dn), di + 1 == kItemRing ? dpar ^ 1u : dpar)) {
+                                const int4 next = item_desc[dn];
+                                if (next.x >= 0) xn = next.y;
+                            }
+                        }
+                        if (xn >= 0) {
+                            const UnitInfo un = locate(a, xn);
+                            const char* qn = reinterpret_cast<const char*>(
+                                a.q + ((size_t)un.b * a.q_heads + (size_t)un.head * G) * D);
+                            if (lane * 128 < G * D * 2 + 128)
+                                asm volatile("prefetch.global.L1 [%0];" ::"l"(qn + lane * 128));
+                        }
+                    }
                     // Q as the A operand (rows = query heads of the group, rows >= G are zero)
                     uint32_t qa[KS][2];
                     {
@@ -592,7 +612,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         constexpr int EPT = (kMaxGroup * D4 + NE - 1) / NE;  // 4-float pieces per thread, at most
         constexpr int CH = 4;                                // partials fetched together per piece
         unsigned long long ns_idle = 0, ns_final = 0, n_final = 0;
-        int todo_n = 0;  // split merges put off so far (same value in every epilogue thread)
+        int pend_n = 0;  // partial segments remembered so far (same value in every epilogue thread)
         const bool tre = trace && et == 0;
         for (int seg = 0;; ++seg) {
             const int bi = seg % kMergeBuffers;
@@ -638,7 +658,13 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(ep_empty + bi));  // the buffer may be refilled
-            if (!sd.complete) {
+            if (!sd.complete && pend_n < kMaxPend) {
+                // the partial is on its way to memory; its ticket is drawn when this CTA's stream
+                // has ended, together with all the others, so no round trip to memory sits here
+                if (et == 0) pend[pend_n] = make_int2(sd.uid, sd.out_row);
+                ++pend_n;
+            } else if (!sd.complete) {
+                // no room to remember the segment: draw its ticket now
                 // the unit's partial records, band by band (lane r of the first epilogue warp looks up band r)
                 __threadfence();
                 if (et < 32) {
@@ -654,18 +680,13 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     epilogue_sync();  // every thread's partial stores are fenced
                     if (et == 0) {
                         const int old = atomicAdd(&a.tickets[sd.uid], 1);
-                        *ep_flag = (old == total - 1) ? total : 0;  // the unit's number of partials if this was the last
+                        *ep_flag = (old == total - 1);
                     }
                 } else {
                     epilogue_sync();
                 }
                 epilogue_sync();
-                if (*ep_flag > 0 && *ep_flag <= kMaxFlat && todo_n < kMaxTodo) {
-                    // the last partial of the unit has arrived: the merge waits until this CTA's
-                    // stream has ended, when all its warps are free to do it
-                    if (et == 0) todo[todo_n] = make_int2(sd.uid, sd.out_row);
-                    ++todo_n;
-                } else if (*ep_flag) {
+                if (*ep_flag) {
                     // the last partial of the unit has arrived: merge them in a fixed order (band by
                     // band, item by item), so the result does not depend on who arrived when
                     const uint64_t t_final = tre ? global_timer_ns() : 0;
@@ -732,66 +753,76 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 }
             }
         }
-        if (et == 0) *todo_count = todo_n;
+        __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
+        if (et == 0) *pend_count = pend_n;
         if (tre) {
             my_trace[7] = global_timer_ns();
             my_trace[11] = ns_idle;
-            my_trace[12] = n_final;
-            my_trace[13] = ns_final;
         }
     }
     __syncthreads();
-    // ---- the split merges this CTA put off.  The tile ring is idle now and serves as scratch.
-    // Thread (piece e, lane ul) merges piece e of the units ul, ul + lanes, ...: all partial
-    // records of a unit are fetched together, so a unit costs about one trip to the L2.
-    const int n_todo = *todo_count;
-    if (!*s_abort && n_todo > 0) {
-        constexpr int NT = S::kThreads, D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
+    // ---- tickets and split merges.  Every partial segment of this CTA draws its unit's ticket now,
+    // all at once; where it was the unit's last one, the unit's partials are merged, in a fixed order
+    // (band by band, item by item), so the result does not depend on who arrived when.  Thread
+    // (piece e, lane ul) merges piece e of the units ul, ul + lanes, ...; the partial records of a
+    // unit are fetched 16 at a time, so a typical unit costs one trip to the L2.  The tile ring is
+    // idle now and serves as scratch.
+    const int n_pend = *pend_count;
+    if (trace && tid == 0) my_trace[12] = global_timer_ns();
+    if (!*s_abort && n_pend > 0) {
+        constexpr int NT = S::kThreads, D4 = D / 4, CH = 16, NB = kMaxRounds + 2;
         const int E = G * D4;                        // 4-float pieces of a unit's output rows
         const int unit_lanes = NT / E > 0 ? NT / E : 1;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-        int2* lists = reinterpret_cast<int2*>(stage_base);        // [kMaxTodo][NB] (first record, count) per band
-        int* flat = reinterpret_cast<int*>(lists + kMaxTodo * NB);  // [kMaxTodo][kMaxFlat] records in merge order
-        for (int p = tid; p < n_todo * (sc.R + 1); p += NT) {
+        int2* lists = reinterpret_cast<int2*>(stage_base);  // [kMaxPend][NB]: (first record, count) per band; last: (total, 0)
+        int* last = reinterpret_cast<int*>(lists + kMaxPend * NB);  // [kMaxPend] entries that drew the last ticket
+        int* n_last = last + kMaxPend;
+        if (tid == 0) *n_last = 0;
+        for (int p = tid; p < n_pend * (sc.R + 1); p += NT) {
             const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
             int slot = 0, count = 0;
-            unit_partials(sc, todo[i].x, r, slot, count);
+            unit_partials(sc, pend[i].x, r, slot, count);
             lists[i * NB + r] = make_int2(slot, count);
         }
         __syncthreads();
-        for (int p = tid; p < n_todo * kMaxFlat; p += NT) {
-            const int i = p / kMaxFlat;
-            int j = p - i * kMaxFlat, rec = -1;
-            for (int r = 0; r <= sc.R; ++r) {
-                const int2 l = lists[i * NB + r];
-                if (j < l.y) {
-                    rec = l.x + j;
-                    break;
-                }
-                j -= l.y;
+        for (int i = tid; i < n_pend; i += NT) {
+            int total = 0;
+            for (int r = 0; r <= sc.R; ++r) total += lists[i * NB + r].y;
+            lists[i * NB + NB - 1] = make_int2(total, 0);
+            if (atomicAdd(&a.tickets[pend[i].x], 1) == total - 1) {
+                a.tickets[pend[i].x] = 0;  // ready for the next launch
+                last[atomicAdd(n_last, 1)] = i;
             }
-            flat[p] = rec;  // -1 past the unit's last record
         }
         __syncthreads();
         __threadfence();
+        if (trace && tid == 0) my_trace[13] = global_timer_ns();
         const int e = tid % E, ul = tid / E;
         if (ul < unit_lanes) {
             const int g = e / D4;
-            for (int i = ul; i < n_todo; i += unit_lanes) {
-                const int* fl = flat + i * kMaxFlat;
+            for (int j = ul; j < *n_last; j += unit_lanes) {
+                const int i = last[j];
+                const int2* li = lists + i * NB;
+                const int F = li[NB - 1].x;
                 float M = kNegBig, L = 0.f;
                 float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
-                for (int c0 = 0; c0 < kMaxFlat && fl[c0] >= 0; c0 += CH) {
+                int band = 0, off = 0;  // the record with merge index c0 is record `off` of band `band`
+                for (int c0 = 0; c0 < F; c0 += CH) {
                     float mm[CH], ll[CH];
                     float4 oo[CH];
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {  // all loads first, then the arithmetic
-                        const int rec = c0 + c < kMaxFlat ? fl[c0 + c] : -1;
-                        const bool on = rec >= 0;
-                        const float* pc = a.partials + (size_t)(on ? rec : 0) * PF;
+                        const bool on = c0 + c < F;
+                        if (on)
+                            while (off >= li[band].y) {
+                                off -= li[band].y;
+                                ++band;
+                            }
+                        const float* pc = a.partials + (size_t)(on ? li[band].x + off : 0) * PF;
                         mm[c] = on ? __ldcg(pc + g) : kNegBig;
                         ll[c] = on ? __ldcg(pc + G + g) : 0.f;
                         oo[c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        ++off;
                     }
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {
@@ -806,11 +837,10 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     }
                 }
                 const float inv = 1.f / L;
-                *reinterpret_cast<float4*>(a.out + (size_t)todo[i].y * D + e * 4) =
+                *reinterpret_cast<float4*>(a.out + (size_t)pend[i].y * D + e * 4) =
                     make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
             }
         }
-        if (tid < n_todo) a.tickets[todo[tid].x] = 0;  // ready for the next launch
     }
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {

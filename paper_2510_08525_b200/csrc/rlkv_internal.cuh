@@ -20,7 +20,8 @@ constexpr int kMaxRounds = 10;   // factoring rounds of the work schedule
 constexpr int kItemRing = 4;     // work-item descriptors in flight between producer and consumers
 constexpr int kTraceWords = 32;  // debug trace: 64-bit words per CTA
 constexpr int kMaxTodo = 32;      // split merges a CTA may put off until its stream has ended
-constexpr int kMaxFlat = 192;     // most partial records of a unit whose merge may be put off
+constexpr int kMaxFlat = 128;     // partial records of a unit fetched through the fast path of the final merge
+constexpr int kMaxPend = 48;      // partial segments of a CTA whose tickets are drawn when its stream has ended
 constexpr int kClaimAhead = 3;   // the producer asks for its next work item this many tiles before the current one ends
 
 // Kernel status codes (device error word).
@@ -67,6 +68,8 @@ struct Schedule {
     int base[kMaxRounds + 2];   // first flat tile of band r <= R; base[R+1]: first compressed tile
     int tb[kMaxRounds + 2];     // first tile, inside a full unit, of its slice in band r; tb[R+1] = tf
     int slot0[kMaxRounds + 1];  // first partial record of band r
+    int iq[kMaxRounds];         // band r < R: its P items have iq[r] tiles, the first irem[r] one more
+    int irem[kMaxRounds];
 };
 
 inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz)
@@ -87,6 +90,8 @@ inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz)
         s.tb[r + 1] = s.tb[r] + bw;
         s.base[r + 1] = s.base[r] + U * bw;
         s.slot0[r] = r * (P + U);
+        s.iq[r] = U * bw / P;
+        s.irem[r] = U * bw % P;
         ++r;
     }
     s.R = r;
@@ -118,7 +123,7 @@ __host__ __device__ inline int item_start(const Schedule& s, int k)
     const int rp = s.R * s.P;
     if (k < rp) {
         const int r = k / s.P, j = k - r * s.P;
-        return s.base[r] + (int)(((long long)j * (s.base[r + 1] - s.base[r])) / s.P);
+        return s.base[r] + j * s.iq[r] + (j < s.irem[r] ? j : s.irem[r]);
     }
     return s.base[s.R] + (k - rp) * s.min_sz;
 }
@@ -127,8 +132,10 @@ __host__ __device__ inline int item_start(const Schedule& s, int k)
 __host__ __device__ inline int item_of_tile(const Schedule& s, int x)
 {
     for (int r = 0; r < s.R; ++r)
-        if (x < s.base[r + 1])
-            return r * s.P + (int)((((long long)(x - s.base[r]) + 1) * s.P - 1) / (s.base[r + 1] - s.base[r]));
+        if (x < s.base[r + 1]) {
+            const int y = x - s.base[r], big = s.irem[r] * (s.iq[r] + 1);
+            return r * s.P + (y < big ? y / (s.iq[r] + 1) : s.irem[r] + (y - big) / s.iq[r]);
+        }
     return s.R * s.P + (x - s.base[s.R]) / s.min_sz;
 }
 
