@@ -24,7 +24,8 @@
  *     that step's attention (it is the newest token of the window).
  *   - Physical slot of token t in a compressed head: t if t < sink, else
  *     sink + ((t - sink) mod window).  While length <= sink + window nothing has been evicted.
- *   - Limits: head_dim in {64, 128}; 1 <= q_heads / kv_heads <= 8; sink >= 0; window >= 1.
+ *   - Limits: head_dim in {64, 128}; 1 <= q_heads / kv_heads <= 8; kv_heads <= 128; sink >= 0;
+ *     window >= 1.
  */
 #ifndef RLKV_H
 #define RLKV_H

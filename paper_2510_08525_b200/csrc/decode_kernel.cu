@@ -64,23 +64,38 @@ __device__ __forceinline__ uint64_t global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
-                                            uint32_t bar)
+// L2 policy for data that is read once: K/V tiles stream through the L2 without pushing out the
+// split-KV partials, tickets and query rows that are about to be read again.
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
-                                            uint32_t bar)
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar,
+                                            uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
         : "memory");
+}
+// Untiled bulk copy global -> shared (both addresses 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 // Byte offset inside a tile row of 16-byte chunk `chunk` of row `row` under the 128-byte swizzle.
 template <int D>
@@ -191,7 +206,13 @@ struct Smem {
     static constexpr int kWarps = NG * kGroupWarps;         // consumer warps
     static constexpr int kThreads = (kWarps + 2 + kEpilogueWarps) * 32;
     static constexpr int kTileBytes = kTile * D * 2;        // one K (or V) tile
-    static constexpr int kStageBytes = 2 * kTileBytes;      // K tile then V tile
+    static constexpr int kTilePairBytes = 2 * kTileBytes;   // K tile then V tile
+    // a stage: K tile, V tile, then the G query rows of the tile's unit (filled for the first NG
+    // tiles of a segment), padded so that the next stage starts on a 1024-byte boundary again
+    __host__ __device__ static constexpr int stage_bytes(int group)
+    {
+        return kTilePairBytes + (group * D * 2 + 1023) / 1024 * 1024;
+    }
     static constexpr int kMergeStride = D + kMergePad;      // floats per head row
     static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
     static constexpr int kBarriers = 2 * 8 + 2 * kItemRing + 2 + 2 * kMergeBuffers;
@@ -203,23 +224,98 @@ struct Smem {
     }
     __host__ __device__ static constexpr size_t bytes(int stages, int group)
     {
-        return (size_t)stages * kStageBytes + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
-               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + 2 * 16 * 4 /*partial lists of a unit*/ +
-               kMaxPend * 8 /*partial segments whose tickets are still to be drawn*/;
+        return (size_t)stages * stage_bytes(group) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
+               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
+               kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
+               (sizeof(Schedule) + 15) / 16 * 16;
     }
 };
 
-// Pool rows of the K and V tile behind flat tile x.
-__device__ __forceinline__ void tile_rows(const DecodeArgs& a, int x, int& krow, int& vrow)
+// Merge of split units.  `units` lists (unit, first output row) of n units whose partial records
+// are all in memory; thread t of nt cooperating threads takes 4-float pieces of their G x D output
+// rows.  The records of a unit are merged in a fixed order (band by band, item by item), 16 at a
+// time -- all loads of a batch first, so a typical unit costs one trip to the L2 -- and the
+// arithmetic does not depend on nt, so the result does not depend on who merges or when.
+// `lists` is scratch for (first record, count) per unit and band.
+// (The schedule is passed as a copy in shared memory and everything else by value: a reference to
+// kernel parameters would turn every use into a slow generic load inside this non-inlined function.)
+template <int D, bool kWholeCta>
+__device__ __noinline__ void merge_units(const Schedule& sc, const float* partials, float* out, int G,
+                                         const int2* units, int n, int t, int nt, int2* lists,
+                                         unsigned long long* stamp)
 {
-    const TilePos p = tile_pos(a.sched, x);
-    if (p.uid < a.sched.U) {
-        krow = (int)(a.full_row0 + (long long)p.uid * 2 * a.rows_full) + p.tile * kTile;
-        vrow = krow + a.rows_full;
-    } else {
-        krow = (int)(a.comp_row0 + (long long)(p.uid - a.sched.U) * 2 * a.rows_comp) + p.tile * kTile;
-        vrow = krow + a.rows_comp;
+    constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
+    const int E = G * D4;
+    const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+    for (int p = t; p < n * (sc.R + 1); p += nt) {
+        const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
+        int slot = 0, count = 0;
+        unit_partials(sc, units[i].x, r, slot, count);
+        lists[i * NB + r] = make_int2(slot, count);
     }
+    if (kWholeCta) __syncthreads(); else epilogue_sync();
+    if (stamp && t == 0) stamp[1] = global_timer_ns();
+    __threadfence();
+    if (stamp && t == 0) stamp[0] = global_timer_ns();
+    const bool wide = nt >= E;                  // enough threads for one piece each, of nt / E units at a time
+    const int unit_lanes = wide ? nt / E : 1;
+    const int ul = wide ? t / E : 0;
+    if (ul < unit_lanes) {
+        for (int j = ul; j < n; j += unit_lanes) {
+            const int2* li = lists + j * NB;
+            int F = 0;
+            for (int r = 0; r <= sc.R; ++r) F += li[r].y;
+            for (int e = wide ? t - ul * E : t; e < E; e += wide ? E : nt) {
+                const int g = e / D4;
+                float M = kNegBig, L = 0.f;
+                float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
+                int band = 0, off = 0;  // the record with merge index c0 is record `off` of band `band`
+                for (int c0 = 0; c0 < F; c0 += CH) {
+                    float mm[CH], ll[CH];
+                    float4 oo[CH];
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const bool on = c0 + c < F;
+                        if (on)
+                            while (off >= li[band].y) {
+                                off -= li[band].y;
+                                ++band;
+                            }
+                        const float* pc = partials + (size_t)(on ? li[band].x + off : 0) * PF;
+                        mm[c] = on ? __ldcg(pc + g) : kNegBig;
+                        ll[c] = on ? __ldcg(pc + G + g) : 0.f;
+                        oo[c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        ++off;
+                    }
+                    float Mc = M;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) Mc = fmaxf(Mc, mm[c]);
+                    if (stamp && t == 0 && j == ul && c0 == 0) stamp[2] = global_timer_ns();
+                    const float keep = exp2f(M - Mc);
+                    L *= keep;
+                    O.x *= keep;
+                    O.y *= keep;
+                    O.z *= keep;
+                    O.w *= keep;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const float w = exp2f(mm[c] - Mc);
+                        L += ll[c] * w;
+                        O.x += oo[c].x * w;
+                        O.y += oo[c].y * w;
+                        O.z += oo[c].z * w;
+                        O.w += oo[c].w * w;
+                    }
+                    M = Mc;
+                }
+                if (stamp && t == 0 && j == ul) stamp[3] = global_timer_ns();
+                const float inv = 1.f / L;
+                *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
+                    make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+            }
+        }
+    }
+    if (kWholeCta) __syncthreads(); else epilogue_sync();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -245,7 +341,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     extern __shared__ __align__(1024) uint8_t smem[];
     const int G = a.group;
     uint8_t* stage_base = smem;
-    uint8_t* buffers = smem + (size_t)stages * S::kStageBytes;
+    const int stage_bytes = S::stage_bytes(G);
+    uint8_t* buffers = smem + (size_t)stages * stage_bytes;
     const int buffer_bytes = S::buffer_bytes(G);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(buffers + (size_t)kMergeBuffers * buffer_bytes);
     uint64_t* empty_bar = full_bar + 8;
@@ -259,10 +356,11 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     volatile int* claim_slot = reinterpret_cast<volatile int*>(item_desc + kItemRing);
     volatile int* ep_flag = claim_slot + 1;
     volatile int* s_abort = claim_slot + 2;
-    int* ep_slot = const_cast<int*>(claim_slot) + 4;   // [16] first partial record of a unit per band
-    int* ep_count = ep_slot + 16;                      // [16] and how many
-    int2* pend = reinterpret_cast<int2*>(ep_count + 16);  // [kMaxPend] (unit, first output row) of partial segments
-    volatile int* pend_count = claim_slot + 3;
+    int2* pend = reinterpret_cast<int2*>(const_cast<int*>(claim_slot) + 4);  // [kMaxPend] (unit, first output row)
+    int2* todo = pend + kMaxPend;                                           // [kMaxTodo] units whose partials are all in
+    int2* lists = todo + kMaxTodo;                                          // scratch of merge_units
+    int* todo_count = const_cast<int*>(claim_slot) + 3;
+    Schedule* s_sched = reinterpret_cast<Schedule*>(lists + kMaxTodo * (kMaxRounds + 1));  // copy for merge_units
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -291,7 +389,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         }
         *ep_flag = 0;
         *s_abort = 0;
-        *pend_count = 0;
+        *todo_count = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -321,7 +419,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             const int4 desc = item_desc[di];
             const int item = desc.x, x0 = desc.y, x1 = desc.z;
             if (item >= 0) {
-                if (tr0 && n_items < 16) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
+                if (tr0 && n_items < 12) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
                 // skip the empty slots the producer issued to line the slot counter up with x0
                 for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, ++cnt) {
@@ -343,37 +441,11 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 if (item >= 0) {
                     u = locate(a, x);
                     seg_tiles = min(x1 - x, u.pos.run);
-                    if (warp == 0) {
-                        // pull the query rows of the segment after this one into the L1 now, so that
-                        // its start does not wait for them
-                        int xn = x + seg_tiles;
-                        if (xn >= x1) {
-                            const int dn = di + 1 == kItemRing ? 0 : di + 1;
-                            xn = -1;
-                            if (mbar_try_wait(smem_u32(item_full + dn), di + 1 == kItemRing ? dpar ^ 1u : dpar)) {
-                                const int4 next = item_desc[dn];
-                                if (next.x >= 0) xn = next.y;
-                            }
-                        }
-                        if (xn >= 0) {
-                            const UnitInfo un = locate(a, xn);
-                            const char* qn = reinterpret_cast<const char*>(
-                                a.q + ((size_t)un.b * a.q_heads + (size_t)un.head * G) * D);
-                            if (lane * 128 < G * D * 2 + 128)
-                                asm volatile("prefetch.global.L1 [%0];" ::"l"(qn + lane * 128));
-                        }
-                    }
-                    // Q as the A operand (rows = query heads of the group, rows >= G are zero)
+                    // Q as the A operand (rows = query heads of the group, rows >= G are zero): read from
+                    // the stage of this warp's first tile of the segment, where the producer put the
+                    // unit's query rows
                     uint32_t qa[KS][2];
-                    {
-                        const __nv_bfloat16* qrow =
-                            a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G + quad) * D + 2 * tq;
-#pragma unroll
-                        for (int ks = 0; ks < KS; ++ks) {
-                            qa[ks][0] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
-                            qa[ks][1] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
-                        }
-                    }
+                    bool have_q = false;
                     int valid_left = u.len - u.pos.tile * kTile;  // valid rows from this tile to the unit's end
                     for (int i = 0; alive && i < seg_tiles; ++i, ++cnt, valid_left -= kTile) {
                         if (cnt % NG != grp) continue;
@@ -386,8 +458,19 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                             landed = true;
                         }
                         const int valid = min(kTile, valid_left);
+                        if (!have_q) {
+                            const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
+                                                            stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
+                                                        quad * D + 2 * tq;
+#pragma unroll
+                            for (int ks = 0; ks < KS; ++ks) {
+                                qa[ks][0] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16) : 0u;
+                                qa[ks][1] = quad < G ? *reinterpret_cast<const uint32_t*>(qrow + ks * 16 + 8) : 0u;
+                            }
+                            have_q = true;
+                        }
                         if (wig * 16 < valid) {
-                            const uint32_t sK = smem_u32(stage_base + (size_t)st * S::kStageBytes);
+                            const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
                             const uint32_t sV = sK + S::kTileBytes;
                             // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
                             float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -523,6 +606,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         // ------------------------------------------------------------------ producer warp
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            const uint64_t stream_policy = l2_evict_first_policy();
             int s = 0, di = 0;
             uint32_t par = 0, dpar = 0, cpar = 0;
             bool ok = true;
@@ -554,22 +638,41 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                         par ^= 1u;
                     }
                 }
+                int seg_left = 0, seg_idx = 0, krow = 0, vrow = 0;
+                const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
                     if (x == x_ask) mbar_arrive(smem_u32(claim_empty));
-                    int krow, vrow;
-                    tile_rows(a, x, krow, vrow);
+                    if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
+                        const UnitInfo u = locate(a, x);
+                        seg_left = min(x1 - x, u.pos.run);
+                        seg_idx = 0;
+                        if (u.pos.uid < sc.U) {
+                            krow = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full) + u.pos.tile * kTile;
+                            vrow = krow + a.rows_full;
+                        } else {
+                            krow = (int)(a.comp_row0 + (long long)(u.pos.uid - sc.U) * 2 * a.rows_comp) + u.pos.tile * kTile;
+                            vrow = krow + a.rows_comp;
+                        }
+                        qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
+                    }
                     ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
-                    mbar_expect_tx(fb, S::kStageBytes);
-                    const uint32_t dst = smem_u32(stage_base + (size_t)s * S::kStageBytes);
+                    const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
+                    mbar_expect_tx(fb, S::kTilePairBytes + (with_q ? G * D * 2 : 0));
+                    const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
                     if (D == 128) {  // one contiguous 16 KB box per tile: [64 rows][2 halves][64]
-                        tma_load_3d(dst, &tmap, 0, 0, krow, fb);
-                        tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb);
+                        tma_load_3d(dst, &tmap, 0, 0, krow, fb, stream_policy);
+                        tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb, stream_policy);
                     } else {         // one contiguous 8 KB box per tile: [64 rows][64]
-                        tma_load_2d(dst, &tmap, 0, krow, fb);
-                        tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb);
+                        tma_load_2d(dst, &tmap, 0, krow, fb, stream_policy);
+                        tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb, stream_policy);
                     }
+                    if (with_q) bulk_load(dst + S::kTilePairBytes, qsrc, G * D * 2, fb);
+                    krow += kTile;
+                    vrow += kTile;
+                    ++seg_idx;
+                    --seg_left;
                     ++issued;
                     if (++s == stages) {
                         s = 0;
@@ -609,22 +712,63 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         constexpr int D4 = D / 4;
         const int et = tid - (S::kWarps + 2) * 32;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-        constexpr int EPT = (kMaxGroup * D4 + NE - 1) / NE;  // 4-float pieces per thread, at most
-        constexpr int CH = 4;                                // partials fetched together per piece
-        unsigned long long ns_idle = 0, ns_final = 0, n_final = 0;
-        int pend_n = 0;  // partial segments remembered so far (same value in every epilogue thread)
+        // the copy of the schedule merge_units works from (these warps have nothing else to do yet)
+        for (int i = et; i < (int)(sizeof(Schedule) / sizeof(int)); i += NE)
+            reinterpret_cast<int*>(s_sched)[i] = reinterpret_cast<const int*>(&a.sched)[i];
+        epilogue_sync();
+        unsigned long long ns_idle = 0;
+        int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;
+        // Draws the tickets of the pending partial segments, all at once: where a segment was its
+        // unit's last one the unit goes on the to-do list, merged when the stream has ended (or now,
+        // by these warps alone, if the list is full).
+        auto flush = [&]() {
+            __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
+            epilogue_sync();
+            if (*todo_count + pend_n > kMaxTodo) {
+                merge_units<D, false>(*s_sched, a.partials, a.out, G, todo, *todo_count, et, NE, lists, nullptr);
+                if (et == 0) *todo_count = 0;
+                epilogue_sync();
+            }
+            // 16 lanes per pending segment: lane r counts the unit's partial records in band r
+            for (int base = 0; base < pend_n * 16; base += NE) {  // whole warps take part in the shuffles
+                const int p = base + et, i = p >> 4, r = p & 15;
+                const bool on = p < pend_n * 16;
+                int slot = 0, total = 0;
+                if (on && r <= sc.R) unit_partials(sc, pend[i].x, r, slot, total);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+                if (on && r == 0 && atomicAdd(&a.tickets[pend[i].x], 1) == total - 1) {
+                    a.tickets[pend[i].x] = 0;  // ready for the next launch
+                    todo[atomicAdd(todo_count, 1)] = pend[i];
+                }
+            }
+            epilogue_sync();
+            pend_n = 0;
+        };
         for (int seg = 0;; ++seg) {
             const int bi = seg % kMergeBuffers;
-            const bool got = wait_traced(smem_u32(ep_full + bi), (uint32_t)(seg / kMergeBuffers) & 1u, s_abort,
-                                         a.status, kStatusMergeWaitTimeout, tre, &ns_idle);
+            const uint32_t bar = smem_u32(ep_full + bi), bpar = (uint32_t)(seg / kMergeBuffers) & 1u;
+            // nothing to merge right now: a good moment to draw tickets (the decision is taken by one
+            // thread so that all epilogue threads take the same path)
+            if (pend_n > 0) {
+                if (et == 0) *ep_flag = mbar_try_wait(bar, bpar) ? 0 : 1;
+                epilogue_sync();
+                const bool idle = *ep_flag != 0;
+                epilogue_sync();
+                if (idle || pend_n == kMaxPend) flush();
+            }
+            const bool got = wait_traced(bar, bpar, s_abort, a.status, kStatusMergeWaitTimeout, tre, &ns_idle);
             if (epilogue_or(!got)) break;
             const uint8_t* buf = buffers + (size_t)bi * buffer_bytes;
             const float* merge = reinterpret_cast<const float*>(buf);
             const float* stat_m = merge + S::merge_floats(G);
             const float* stat_l = stat_m + S::kWarps * kMaxGroup;
             const SegDesc sd = *reinterpret_cast<const SegDesc*>(stat_l + S::kWarps * kMaxGroup);
-            if (sd.stop) break;
+            if (sd.stop) {
+                if (pend_n > 0) flush();
+                break;
+            }
             float* out_rows = a.out + (size_t)sd.out_row * D;
             float* my_part = a.partials + (size_t)sd.pslot * PF;
             // merge the consumer warps' states; this thread owns a few 4-float pieces of the G x D rows
@@ -658,190 +802,23 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(ep_empty + bi));  // the buffer may be refilled
-            if (!sd.complete && pend_n < kMaxPend) {
-                // the partial is on its way to memory; its ticket is drawn when this CTA's stream
-                // has ended, together with all the others, so no round trip to memory sits here
+            if (!sd.complete) {
                 if (et == 0) pend[pend_n] = make_int2(sd.uid, sd.out_row);
                 ++pend_n;
-            } else if (!sd.complete) {
-                // no room to remember the segment: draw its ticket now
-                // the unit's partial records, band by band (lane r of the first epilogue warp looks up band r)
-                __threadfence();
-                if (et < 32) {
-                    int slot = 0, count = 0;
-                    if (et <= sc.R) unit_partials(sc, sd.uid, et, slot, count);
-                    if (et <= kMaxRounds) {
-                        ep_slot[et] = slot;
-                        ep_count[et] = count;
-                    }
-                    int total = count;
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-                    epilogue_sync();  // every thread's partial stores are fenced
-                    if (et == 0) {
-                        const int old = atomicAdd(&a.tickets[sd.uid], 1);
-                        *ep_flag = (old == total - 1);
-                    }
-                } else {
-                    epilogue_sync();
-                }
-                epilogue_sync();
-                if (*ep_flag) {
-                    // the last partial of the unit has arrived: merge them in a fixed order (band by
-                    // band, item by item), so the result does not depend on who arrived when
-                    const uint64_t t_final = tre ? global_timer_ns() : 0;
-                    __threadfence();
-                    float M[EPT], L[EPT];
-                    float4 O[EPT];
-#pragma unroll
-                    for (int j = 0; j < EPT; ++j) {
-                        M[j] = kNegBig;
-                        L[j] = 0.f;
-                        O[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    for (int r = 0; r <= sc.R; ++r) {
-                        const float* pr = a.partials + (size_t)ep_slot[r] * PF;
-                        const int n = ep_count[r];
-                        for (int c0 = 0; c0 < n; c0 += CH) {
-                            float mm[EPT][CH], ll[EPT][CH];
-                            float4 oo[EPT][CH];
-                            // all loads of the chunk first, then the arithmetic
-#pragma unroll
-                            for (int j = 0; j < EPT; ++j) {
-                                const int e = et + j * NE;
-                                const int g = e / D4;
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) {
-                                    const bool on = e < G * D4 && c0 + c < n;
-                                    const float* pc = pr + (size_t)(c0 + c) * PF;
-                                    mm[j][c] = on ? __ldcg(pc + g) : kNegBig;
-                                    ll[j][c] = on ? __ldcg(pc + G + g) : 0.f;
-                                    oo[j][c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e)
-                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-                                }
-                            }
-#pragma unroll
-                            for (int j = 0; j < EPT; ++j) {
-#pragma unroll
-                                for (int c = 0; c < CH; ++c) {
-                                    const float Mn = fmaxf(M[j], mm[j][c]);
-                                    const float ca = exp2f(M[j] - Mn), cb = exp2f(mm[j][c] - Mn);
-                                    L[j] = L[j] * ca + ll[j][c] * cb;
-                                    O[j].x = O[j].x * ca + oo[j][c].x * cb;
-                                    O[j].y = O[j].y * ca + oo[j][c].y * cb;
-                                    O[j].z = O[j].z * ca + oo[j][c].z * cb;
-                                    O[j].w = O[j].w * ca + oo[j][c].w * cb;
-                                    M[j] = Mn;
-                                }
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int j = 0; j < EPT; ++j) {
-                        const int e = et + j * NE;
-                        if (e < G * D4) {
-                            const float inv = 1.f / L[j];
-                            *reinterpret_cast<float4*>(out_rows + e * 4) =
-                                make_float4(O[j].x * inv, O[j].y * inv, O[j].z * inv, O[j].w * inv);
-                        }
-                    }
-                    if (et == 0) a.tickets[sd.uid] = 0;  // ready for the next launch
-                    if (tre) {
-                        ns_final += global_timer_ns() - t_final;
-                        ++n_final;
-                    }
-                }
             }
         }
-        __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
-        if (et == 0) *pend_count = pend_n;
         if (tre) {
             my_trace[7] = global_timer_ns();
             my_trace[11] = ns_idle;
         }
     }
     __syncthreads();
-    // ---- tickets and split merges.  Every partial segment of this CTA draws its unit's ticket now,
-    // all at once; where it was the unit's last one, the unit's partials are merged, in a fixed order
-    // (band by band, item by item), so the result does not depend on who arrived when.  Thread
-    // (piece e, lane ul) merges piece e of the units ul, ul + lanes, ...; the partial records of a
-    // unit are fetched 16 at a time, so a typical unit costs one trip to the L2.  The tile ring is
-    // idle now and serves as scratch.
-    const int n_pend = *pend_count;
+    // ---- the units on this CTA's to-do list: merged by all its warps
     if (trace && tid == 0) my_trace[12] = global_timer_ns();
-    if (!*s_abort && n_pend > 0) {
-        constexpr int NT = S::kThreads, D4 = D / 4, CH = 16, NB = kMaxRounds + 2;
-        const int E = G * D4;                        // 4-float pieces of a unit's output rows
-        const int unit_lanes = NT / E > 0 ? NT / E : 1;
-        const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-        int2* lists = reinterpret_cast<int2*>(stage_base);  // [kMaxPend][NB]: (first record, count) per band; last: (total, 0)
-        int* last = reinterpret_cast<int*>(lists + kMaxPend * NB);  // [kMaxPend] entries that drew the last ticket
-        int* n_last = last + kMaxPend;
-        if (tid == 0) *n_last = 0;
-        for (int p = tid; p < n_pend * (sc.R + 1); p += NT) {
-            const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
-            int slot = 0, count = 0;
-            unit_partials(sc, pend[i].x, r, slot, count);
-            lists[i * NB + r] = make_int2(slot, count);
-        }
-        __syncthreads();
-        for (int i = tid; i < n_pend; i += NT) {
-            int total = 0;
-            for (int r = 0; r <= sc.R; ++r) total += lists[i * NB + r].y;
-            lists[i * NB + NB - 1] = make_int2(total, 0);
-            if (atomicAdd(&a.tickets[pend[i].x], 1) == total - 1) {
-                a.tickets[pend[i].x] = 0;  // ready for the next launch
-                last[atomicAdd(n_last, 1)] = i;
-            }
-        }
-        __syncthreads();
-        __threadfence();
-        if (trace && tid == 0) my_trace[13] = global_timer_ns();
-        const int e = tid % E, ul = tid / E;
-        if (ul < unit_lanes) {
-            const int g = e / D4;
-            for (int j = ul; j < *n_last; j += unit_lanes) {
-                const int i = last[j];
-                const int2* li = lists + i * NB;
-                const int F = li[NB - 1].x;
-                float M = kNegBig, L = 0.f;
-                float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
-                int band = 0, off = 0;  // the record with merge index c0 is record `off` of band `band`
-                for (int c0 = 0; c0 < F; c0 += CH) {
-                    float mm[CH], ll[CH];
-                    float4 oo[CH];
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {  // all loads first, then the arithmetic
-                        const bool on = c0 + c < F;
-                        if (on)
-                            while (off >= li[band].y) {
-                                off -= li[band].y;
-                                ++band;
-                            }
-                        const float* pc = a.partials + (size_t)(on ? li[band].x + off : 0) * PF;
-                        mm[c] = on ? __ldcg(pc + g) : kNegBig;
-                        ll[c] = on ? __ldcg(pc + G + g) : 0.f;
-                        oo[c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-                        ++off;
-                    }
-#pragma unroll
-                    for (int c = 0; c < CH; ++c) {
-                        const float Mn = fmaxf(M, mm[c]);
-                        const float ca = exp2f(M - Mn), cb = exp2f(mm[c] - Mn);
-                        L = L * ca + ll[c] * cb;
-                        O.x = O.x * ca + oo[c].x * cb;
-                        O.y = O.y * ca + oo[c].y * cb;
-                        O.z = O.z * ca + oo[c].z * cb;
-                        O.w = O.w * ca + oo[c].w * cb;
-                        M = Mn;
-                    }
-                }
-                const float inv = 1.f / L;
-                *reinterpret_cast<float4*>(a.out + (size_t)pend[i].y * D + e * 4) =
-                    make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
-            }
-        }
-    }
+    if (trace && tid == 0) my_trace[13] = (unsigned long long)*todo_count;
+    if (!*s_abort && *todo_count > 0)
+        merge_units<D, true>(*s_sched, a.partials, a.out, G, todo, *todo_count, tid, S::kThreads, lists,
+                             trace ? my_trace + 28 : nullptr);
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
             // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight

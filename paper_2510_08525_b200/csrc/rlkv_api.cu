@@ -72,7 +72,8 @@ long long most_slots(int U, int tf, int Uc, int tc, int max_grid)
 int check_shape(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
                 const uint8_t* mask, int sink, int window)
 {
-    if (!mask || layers < 1 || kv_heads < 1 || q_heads < 1 || batch < 1 || max_len < 1) return RLKV_EINVAL;
+    if (!mask || layers < 1 || kv_heads < 1 || kv_heads > kMaxKvHeads || q_heads < 1 || batch < 1 || max_len < 1)
+        return RLKV_EINVAL;
     if (q_heads % kv_heads != 0 || q_heads / kv_heads > kMaxGroup) return RLKV_EINVAL;
     if (head_dim != 64 && head_dim != 128) return RLKV_EINVAL;
     if (sink < 0 || window < 1) return RLKV_EINVAL;
@@ -278,7 +279,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
     a.full_row0 = c->lay.full_row0[layer];
     a.comp_row0 = c->lay.comp_row0[layer];
-    a.head_of_slot = dev_at<int>(c, c->lay.off_tables) + (size_t)(c->layers + layer) * c->kv_heads;
+    for (int h = 0; h < c->kv_heads; ++h) a.head_of_slot[h] = (unsigned char)c->head_of_slot[(size_t)layer * c->kv_heads + h];
     a.q = static_cast<const __nv_bfloat16*>(q);
     a.out = static_cast<float*>(out);
     a.status = dev_at<int>(c, c->lay.off_status);

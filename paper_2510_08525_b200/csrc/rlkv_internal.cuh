@@ -10,18 +10,18 @@ namespace rlkv {
 
 constexpr int kTile = 64;        // tokens per K/V tile (one pipeline stage holds a K and a V tile)
 constexpr int kMaxGroup = 8;     // query heads per KV head handled by one tile pass
+constexpr int kMaxKvHeads = 128; // KV heads per layer (their order travels in the kernel arguments)
 constexpr int kGroupWarps = 4;   // consumer warps that share one tile (16 tokens each)
 constexpr int kMaxConsumerGroups = 3;
 constexpr int kMaxDynamicSmem = 227 * 1024;
 constexpr int kMergePad = 4;     // floats of padding per head row in the cross-warp merge area
 constexpr int kEpilogueWarps = 2;  // warps that merge the consumer warps' states and the split partials
-constexpr int kMergeBuffers = 2;   // hand-off buffers between consumer warps and epilogue warps
+constexpr int kMergeBuffers = 1;   // hand-off buffers between consumer warps and epilogue warps
 constexpr int kMaxRounds = 10;   // factoring rounds of the work schedule
 constexpr int kItemRing = 4;     // work-item descriptors in flight between producer and consumers
 constexpr int kTraceWords = 32;  // debug trace: 64-bit words per CTA
-constexpr int kMaxTodo = 32;      // split merges a CTA may put off until its stream has ended
-constexpr int kMaxFlat = 128;     // partial records of a unit fetched through the fast path of the final merge
-constexpr int kMaxPend = 48;      // partial segments of a CTA whose tickets are drawn when its stream has ended
+constexpr int kMaxTodo = 64;      // split merges a CTA may put off until its stream has ended
+constexpr int kMaxPend = 16;      // partial segments of a CTA whose tickets are drawn when its stream has ended
 constexpr int kClaimAhead = 3;   // the producer asks for its next work item this many tiles before the current one ends
 
 // Kernel status codes (device error word).
@@ -206,7 +206,6 @@ struct DecodeArgs {
     const __nv_bfloat16* pool;  // base of the row pool, rows of head_dim bf16
     long long full_row0;        // first pool row of the layer's full-head region
     long long comp_row0;        // first pool row of the layer's compressed-head region
-    const int* head_of_slot;    // [kv_heads]: KV head of full slot 0..n_full-1, then of comp slots
     const __nv_bfloat16* q;     // [batch][q_heads][head_dim]
     float* out;                 // [batch][q_heads][head_dim]
     float* partials;            // [sched.n_slots][partial_floats]
@@ -221,6 +220,7 @@ struct DecodeArgs {
     float scale_log2;           // log2(e) / sqrt(head_dim)
     int trace_on;
     Schedule sched;
+    unsigned char head_of_slot[kMaxKvHeads];  // KV head of full slot 0..n_full-1, then of the compressed slots
 };
 
 struct AppendArgs {
