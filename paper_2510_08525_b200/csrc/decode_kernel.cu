@@ -97,12 +97,14 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-// Byte offset inside a tile row of 16-byte chunk `chunk` of row `row` under the 128-byte swizzle.
+// Byte offset inside a K or V tile of 16-byte chunk `chunk` (along d) of token row `row`.  A tile
+// is stored as D/64 blocks of [64 rows][128 bytes], written by TMA with the 128-byte swizzle: inside a
+// block, chunk c of row r sits at chunk position c ^ (r & 7), so the eight rows of an ldmatrix
+// fragment fall into eight different bank groups.
 template <int D>
-__device__ __forceinline__ uint32_t swizzled_chunk(int row, int chunk)
+__device__ __forceinline__ uint32_t tile_offset(int row, int chunk)
 {
-    if (D == 128) return (uint32_t)(((chunk & 8) | ((chunk & 7) ^ ((2 * row + (chunk >> 3)) & 7))) << 4);
-    return (uint32_t)((chunk ^ (row & 7)) << 4);
+    return (uint32_t)((chunk >> 3) * (kTile * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 // Barrier over the epilogue warps (named barrier 2).
 __device__ __forceinline__ void epilogue_sync()
@@ -177,14 +179,15 @@ __device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, vola
     }
 }
 
-// wait_bounded that also adds the time spent waiting to *ns when the trace is on (one thread's view).
+// wait_bounded that also adds the SM clock cycles spent waiting to *cycles when the trace is on (one
+// thread's view; the cycle counter is cheap to read, unlike %globaltimer).
 __device__ __forceinline__ bool wait_traced(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                            int code, bool on, unsigned long long* ns)
+                                            int code, bool on, unsigned long long* cycles)
 {
     if (!on) return wait_bounded(bar, parity, abort_flag, status, code);
-    const uint64_t t = global_timer_ns();
+    const long long t = clock64();
     const bool ok = wait_bounded(bar, parity, abort_flag, status, code);
-    *ns += global_timer_ns() - t;
+    *cycles += (unsigned long long)(clock64() - t);
     return ok;
 }
 
@@ -402,11 +405,17 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         const int ldm_j = lane >> 3, ldm_r = lane & 7;
         const int ldm_tok = wig * 16 + (ldm_j >> 1) * 8 + ldm_r;  // token row this lane addresses
         const int ldm_chunk = ldm_j & 1;                          // +1 16-byte chunk for odd matrices
-        // Tile layout in shared memory (written by TMA with the 128-byte swizzle): row r of the tile
-        // starts at r*2*D bytes; its 16-byte chunk c sits at chunk index c ^ (bits 7..9 of the
-        // unswizzled offset), i.e. c ^ ((2r + c/8) & 7) for D = 128 and c ^ (r & 7) for D = 64.
-        const uint32_t row_off = ldm_tok * (2 * D);
         int cnt = 0;   // slots seen so far (mirrors the producer's `issued`)
+        int st = 0, turn = 0;  // cnt % stages, cnt % NG
+        uint32_t ph = 0;       // (cnt / stages) & 1
+        auto next_slot = [&]() {
+            ++cnt;
+            if (++turn == NG) turn = 0;
+            if (++st == stages) {
+                st = 0;
+                ph ^= 1u;
+            }
+        };
         int seg = 0;   // segments handed to the epilogue warps so far
         int di = 0;
         uint32_t dpar = 0;
@@ -422,11 +431,9 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 if (tr0 && n_items < 12) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
                 // skip the empty slots the producer issued to line the slot counter up with x0
-                for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, ++cnt) {
-                    if (cnt % NG != grp) continue;
-                    const int st = cnt % stages;
-                    alive = wait_bounded(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort, a.status,
-                                         kStatusFullWaitTimeout);
+                for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
+                    if (turn != grp) continue;
+                    alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
                     if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
                 }
             }
@@ -447,11 +454,10 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     uint32_t qa[KS][2];
                     bool have_q = false;
                     int valid_left = u.len - u.pos.tile * kTile;  // valid rows from this tile to the unit's end
-                    for (int i = 0; alive && i < seg_tiles; ++i, ++cnt, valid_left -= kTile) {
-                        if (cnt % NG != grp) continue;
-                        const int st = cnt % stages;
-                        alive = wait_traced(smem_u32(full_bar + st), (uint32_t)(cnt / stages) & 1u, s_abort,
-                                            a.status, kStatusFullWaitTimeout, tr0, &ns_tile);
+                    for (int i = 0; alive && i < seg_tiles; ++i, next_slot(), valid_left -= kTile) {
+                        if (turn != grp) continue;
+                        alive = wait_traced(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout, tr0,
+                                            &ns_tile);
                         if (!alive) break;
                         if (trace && tid == 0 && !landed) {
                             my_trace[1] = global_timer_ns();
@@ -478,7 +484,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
 #pragma unroll
                             for (int ks = 0; ks < KS; ++ks) {
                                 const int chunk = ks * 2 + ldm_chunk;  // 16-byte chunk along d
-                                const uint32_t addr = sK + row_off + swizzled_chunk<D>(ldm_tok, chunk);
+                                const uint32_t addr = sK + tile_offset<D>(ldm_tok, chunk);
                                 uint32_t b0, b1, b2, b3;
                                 ldmatrix_x4(addr, b0, b1, b2, b3);
                                 if (ks & 1) {
@@ -518,7 +524,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
 #pragma unroll
                             for (int mt = 0; mt < KS; ++mt) {
                                 const int chunk = mt * 2 + ldm_chunk;
-                                const uint32_t addr = sV + row_off + swizzled_chunk<D>(ldm_tok, chunk);
+                                const uint32_t addr = sV + tile_offset<D>(ldm_tok, chunk);
                                 uint32_t v0, v1, v2, v3;
                                 ldmatrix_x4_trans(addr, v0, v1, v2, v3);
                                 acc[mt][0] *= ca;
@@ -661,9 +667,9 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
                     mbar_expect_tx(fb, S::kTilePairBytes + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
-                    if (D == 128) {  // one contiguous 16 KB box per tile: [64 rows][2 halves][64]
-                        tma_load_3d(dst, &tmap, 0, 0, krow, fb, stream_policy);
-                        tma_load_3d(dst + S::kTileBytes, &tmap, 0, 0, vrow, fb, stream_policy);
+                    if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
+                        tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
+                        tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
                     } else {         // one contiguous 8 KB box per tile: [64 rows][64]
                         tma_load_2d(dst, &tmap, 0, krow, fb, stream_policy);
                         tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb, stream_policy);

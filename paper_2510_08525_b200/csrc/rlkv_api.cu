@@ -212,16 +212,19 @@ int make_tensor_map(rlkv_cache* c)
     RLKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
     if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
     // The pool as rows of 128-byte pieces so that one box is one contiguous run of memory and still
-    // obeys the 128-byte limit of the swizzled inner dimension:
-    //   head_dim 128: [rows][2 halves][64]  box [64 rows][2][64]  (16 KB)
+    // obeys the 128-byte limit of the swizzled inner dimension.  For head_dim 128 the two halves of
+    // the rows are the OUTER dimension of the box, so the tile lands in shared memory as two blocks
+    // of [64 rows][128 bytes]: eight consecutive rows of a block are then eight different swizzle
+    // phases (with 256-byte rows only four, and every ldmatrix would take a two-way bank conflict).
+    //   head_dim 128: [2 halves][rows][64]  box [2][64 rows][64]  (16 KB)
     //   head_dim  64: [rows][64]            box [64 rows][64]     ( 8 KB)
     CUresult r;
     void* base = c->dev_base + c->lay.off_pool;
     const CUtensorMapL2promotion l2p = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
     if (c->head_dim == 128) {
-        const cuuint64_t dims[3] = {64, 2, (cuuint64_t)c->lay.pool_rows};
-        const cuuint64_t strides[2] = {128, 256};
-        const cuuint32_t box[3] = {64, 2, (cuuint32_t)kTile};
+        const cuuint64_t dims[3] = {64, (cuuint64_t)c->lay.pool_rows, 2};
+        const cuuint64_t strides[2] = {256, 128};
+        const cuuint32_t box[3] = {64, (cuuint32_t)kTile, 2};
         const cuuint32_t estr[3] = {1, 1, 1};
         r = reinterpret_cast<EncodeTiledFn>(fn)(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box,
                                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2p,
