@@ -428,7 +428,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             const int4 desc = item_desc[di];
             const int item = desc.x, x0 = desc.y, x1 = desc.z;
             if (item >= 0) {
-                if (tr0 && n_items < 12) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
+                if (tr0 && n_items < 11) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
                 // skip the empty slots the producer issued to line the slot counter up with x0
                 for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
@@ -616,7 +616,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             int s = 0, di = 0;
             uint32_t par = 0, dpar = 0, cpar = 0;
             bool ok = true;
-            unsigned long long ns_claim = 0, ns_ring = 0;
+            unsigned long long ns_claim = 0, ns_ring = 0, ns_stage = 0;
+            const long long t_prod = clock64();
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             while (ok && k < sc.n_items) {
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
@@ -661,7 +662,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                         }
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                     }
-                    ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
+                    ok = wait_traced(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout, trace,
+                                     &ns_stage);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
@@ -696,7 +698,8 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             }
             if (trace) {
                 my_trace[14] = ns_claim;
-                my_trace[15] = ns_ring;
+                my_trace[15] = ns_ring + (ns_stage << 32);
+                my_trace[27] = (unsigned long long)(clock64() - t_prod);
             }
         }
     } else if (warp == S::kWarps + 1) {
