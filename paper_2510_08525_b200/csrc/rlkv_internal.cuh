@@ -16,7 +16,7 @@ constexpr int kMaxConsumerGroups = 3;
 constexpr int kMaxDynamicSmem = 227 * 1024;
 constexpr int kMergePad = 4;     // floats of padding per head row in the cross-warp merge area
 constexpr int kEpilogueWarps = 2;  // warps that merge the consumer warps' states and the split partials
-constexpr int kMergeBuffers = 1;   // hand-off buffers between consumer warps and epilogue warps
+constexpr int kMergeBuffers = 2;   // hand-off buffers between consumer warps and epilogue warps
 constexpr int kMaxRounds = 10;   // factoring rounds of the work schedule
 constexpr int kItemRing = 4;     // work-item descriptors in flight between producer and consumers
 constexpr int kTraceWords = 32;  // debug trace: 64-bit words per CTA
