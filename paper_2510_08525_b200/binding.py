@@ -204,9 +204,9 @@ def rlkv_set_decode_config(cache, ctas_per_sm=0, stages=0, consumer_groups=0, it
 
 
 def rlkv_debug_trace(cache, enable, read=False):
-    """Switches the decode kernel's trace on or off; with read=True returns uint64[320][32] of the
+    """Switches the decode kernel's trace on or off; with read=True returns uint64[320][40] of the
     most recent launch (taken before the switch is applied)."""
-    words = np.zeros((320, 32), dtype=np.uint64) if read else None
+    words = np.zeros((320, 40), dtype=np.uint64) if read else None
     ctas = _ci(0)
     _check(lib.rlkv_debug_trace(cache, int(enable), _ptr(words), ctypes.byref(ctas)))
     return words

@@ -230,7 +230,7 @@ struct Smem {
         return (size_t)stages * stage_bytes(group) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
-               (sizeof(Schedule) + 15) / 16 * 16;
+               (sizeof(DecodeArgs) + 15) / 16 * 16;
     }
 };
 
@@ -336,13 +336,13 @@ __device__ __noinline__ void merge_units(const Schedule& sc, const float* partia
 // issues an empty slot first.
 template <int D, int NG>
 __global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
-decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUtensorMap tmap, const int stages)
+decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ CUtensorMap tmap, const int stages)
 {
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     constexpr int MS = S::kMergeStride;
     extern __shared__ __align__(1024) uint8_t smem[];
-    const int G = a.group;
+    const int G = args.group;
     uint8_t* stage_base = smem;
     const int stage_bytes = S::stage_bytes(G);
     uint8_t* buffers = smem + (size_t)stages * stage_bytes;
@@ -363,18 +363,24 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
     int2* todo = pend + kMaxPend;                                           // [kMaxTodo] units whose partials are all in
     int2* lists = todo + kMaxTodo;                                          // scratch of merge_units
     int* todo_count = const_cast<int*>(claim_slot) + 3;
-    Schedule* s_sched = reinterpret_cast<Schedule*>(lists + kMaxTodo * (kMaxRounds + 1));  // copy for merge_units
+    // The arguments, copied to shared memory: the schedule and the head order are looked up with
+    // run-time indices, which is slow on kernel parameters and cheap here.
+    DecodeArgs* s_args = reinterpret_cast<DecodeArgs*>(lists + kMaxTodo * (kMaxRounds + 1));
+    const DecodeArgs& a = *s_args;
+    Schedule* s_sched = &s_args->sched;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
-    const bool trace = a.trace_on != 0;
-    unsigned long long* my_trace = a.trace + (size_t)blockIdx.x * kTraceWords;
+    const bool trace = args.trace_on != 0;
+    unsigned long long* my_trace = args.trace + (size_t)blockIdx.x * kTraceWords;
     if (trace && tid == 0) my_trace[0] = global_timer_ns();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
-        if (tid == 0) atomicCAS(a.status, kStatusOk, kStatusSmemMisaligned);
+        if (tid == 0) atomicCAS(args.status, kStatusOk, kStatusSmemMisaligned);
         return;
     }
+    for (int i = tid; i < (int)(sizeof(DecodeArgs) / sizeof(int)); i += blockDim.x)
+        reinterpret_cast<int*>(s_args)[i] = reinterpret_cast<const int*>(&args)[i];
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
@@ -617,9 +623,11 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
             uint32_t par = 0, dpar = 0, cpar = 0;
             bool ok = true;
             unsigned long long ns_claim = 0, ns_ring = 0, ns_stage = 0;
+            long long cy_expect = 0, cy_tma = 0, cy_q = 0, cy_item = 0, cy_seg = 0;
             const long long t_prod = clock64();
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             while (ok && k < sc.n_items) {
+                const long long ti0 = trace ? clock64() : 0;
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
                 // ask the claim warp for the next item only shortly before this one is issued in
                 // full: early enough to hide the round trip, late enough that a CTA is never
@@ -634,6 +642,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                     di = 0;
                     dpar ^= 1u;
                 }
+                if (trace) cy_item += clock64() - ti0;
                 // empty slots until the slot counter has the residue of x0
                 for (int pad = ((x0 - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
                     ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
@@ -649,6 +658,7 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
                     if (x == x_ask) mbar_arrive(smem_u32(claim_empty));
+                    const long long ts0 = trace ? clock64() : 0;
                     if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
                         const UnitInfo u = locate(a, x);
                         seg_left = min(x1 - x, u.pos.run);
@@ -662,13 +672,16 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                         }
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                     }
+                    if (trace) cy_seg += clock64() - ts0;
                     ok = wait_traced(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout, trace,
                                      &ns_stage);
                     if (!ok) break;
                     const uint32_t fb = smem_u32(full_bar + s);
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
+                    const long long tc0 = trace ? clock64() : 0;
                     mbar_expect_tx(fb, S::kTilePairBytes + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
+                    const long long tc1 = trace ? clock64() : 0;
                     if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
                         tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
                         tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
@@ -676,7 +689,14 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                         tma_load_2d(dst, &tmap, 0, krow, fb, stream_policy);
                         tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb, stream_policy);
                     }
+                    const long long tc2 = trace ? clock64() : 0;
                     if (with_q) bulk_load(dst + S::kTilePairBytes, qsrc, G * D * 2, fb);
+                    if (trace) {
+                        const long long tc3 = clock64();
+                        cy_expect += tc1 - tc0;
+                        cy_tma += tc2 - tc1;
+                        cy_q += tc3 - tc2;
+                    }
                     krow += kTile;
                     vrow += kTile;
                     ++seg_idx;
@@ -700,6 +720,11 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
                 my_trace[14] = ns_claim;
                 my_trace[15] = ns_ring + (ns_stage << 32);
                 my_trace[27] = (unsigned long long)(clock64() - t_prod);
+                my_trace[32] = (unsigned long long)cy_expect;
+                my_trace[33] = (unsigned long long)cy_tma;
+                my_trace[34] = (unsigned long long)cy_q;
+                my_trace[35] = (unsigned long long)cy_item;
+                my_trace[36] = (unsigned long long)cy_seg;
             }
         }
     } else if (warp == S::kWarps + 1) {
@@ -721,10 +746,6 @@ decode_kernel(const __grid_constant__ DecodeArgs a, const __grid_constant__ CUte
         constexpr int D4 = D / 4;
         const int et = tid - (S::kWarps + 2) * 32;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-        // the copy of the schedule merge_units works from (these warps have nothing else to do yet)
-        for (int i = et; i < (int)(sizeof(Schedule) / sizeof(int)); i += NE)
-            reinterpret_cast<int*>(s_sched)[i] = reinterpret_cast<const int*>(&a.sched)[i];
-        epilogue_sync();
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;

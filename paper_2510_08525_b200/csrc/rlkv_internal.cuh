@@ -19,7 +19,7 @@ constexpr int kEpilogueWarps = 2;  // warps that merge the consumer warps' state
 constexpr int kMergeBuffers = 2;   // hand-off buffers between consumer warps and epilogue warps
 constexpr int kMaxRounds = 10;   // factoring rounds of the work schedule
 constexpr int kItemRing = 4;     // work-item descriptors in flight between producer and consumers
-constexpr int kTraceWords = 32;  // debug trace: 64-bit words per CTA
+constexpr int kTraceWords = 40;  // debug trace: 64-bit words per CTA
 constexpr int kMaxTodo = 64;      // split merges a CTA may put off until its stream has ended
 constexpr int kMaxPend = 16;      // partial segments of a CTA whose tickets are drawn when its stream has ended
 constexpr int kClaimAhead = 3;   // the producer asks for its next work item this many tiles before the current one ends

@@ -302,7 +302,7 @@ def test_reset_and_config_knobs(rl, hz, cuda_device):
     want = oracle.decode(0, q)
     outs = []
     for cps, st, ng, it in ((1, 6, 1, 0), (1, 2, 2, 2), (2, 2, 1, 3), (1, 3, 3, 2), (2, 2, 2, 5), (1, 4, 2, 16),
-                            (1, 0, 3, 7), (1, 5, 1, 1024), (1, 3, 3, 4), (1, 6, 2, 4)):
+                            (1, 0, 3, 7), (1, 5, 1, 1024), (1, 3, 3, 4), (1, 4, 2, 4)):
         rl.rlkv_set_decode_config(cache.handle, cps, st, ng, it)
         outs.append(cache.decode(0, q.to(cuda_device)).cpu().numpy())
         check_out(outs[-1], want)
