@@ -242,21 +242,26 @@ struct Smem {
 // `lists` is scratch for (first record, count) per unit and band.
 // (The schedule is passed as a copy in shared memory and everything else by value: a reference to
 // kernel parameters would turn every use into a slow generic load inside this non-inlined function.)
-template <int D, bool kWholeCta>
+// `whole`: all threads of the CTA take part (else the epilogue warps alone).  `dry`: everything but
+// the stores -- run once by the idle epilogue warps at kernel start so that the instructions are in
+// the SM's instruction cache when the merges at the end of the stream need them.
+template <int D>
 __device__ __noinline__ void merge_units(const Schedule& sc, const float* partials, float* out, int G,
-                                         const int2* units, int n, int t, int nt, int2* lists,
-                                         unsigned long long* stamp)
+                                         const int2* units, int n, int t, int nt, int2* lists, bool whole,
+                                         bool dry, unsigned long long* stamp)
 {
     constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
     const int E = G * D4;
     const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+    if (stamp && t == 0) stamp[9] = global_timer_ns();
     for (int p = t; p < n * (sc.R + 1); p += nt) {
         const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
         int slot = 0, count = 0;
         unit_partials(sc, units[i].x, r, slot, count);
         lists[i * NB + r] = make_int2(slot, count);
     }
-    if (kWholeCta) __syncthreads(); else epilogue_sync();
+    if (stamp && t == 0) stamp[10] = global_timer_ns();
+    if (whole) __syncthreads(); else epilogue_sync();
     if (stamp && t == 0) stamp[1] = global_timer_ns();
     __threadfence();
     if (stamp && t == 0) stamp[0] = global_timer_ns();
@@ -313,12 +318,13 @@ __device__ __noinline__ void merge_units(const Schedule& sc, const float* partia
                 }
                 if (stamp && t == 0 && j == ul) stamp[3] = global_timer_ns();
                 const float inv = 1.f / L;
-                *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
-                    make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                if (!dry)
+                    *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
+                        make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
             }
         }
     }
-    if (kWholeCta) __syncthreads(); else epilogue_sync();
+    if (whole) __syncthreads(); else epilogue_sync();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -746,6 +752,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         constexpr int D4 = D / 4;
         const int et = tid - (S::kWarps + 2) * 32;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+        // warm the instruction cache with the merge routine while there is nothing else to do: a dry
+        // run on unit 0 (its partial records hold whatever the last launch left; nothing is stored)
+        if (et == 0) todo[kMaxTodo - 1] = make_int2(0, 0);
+        epilogue_sync();
+        merge_units<D>(*s_sched, a.partials, a.out, G, todo + kMaxTodo - 1, 1, et, NE, lists, false, true, nullptr);
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;
@@ -756,7 +767,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
             epilogue_sync();
             if (*todo_count + pend_n > kMaxTodo) {
-                merge_units<D, false>(*s_sched, a.partials, a.out, G, todo, *todo_count, et, NE, lists, nullptr);
+                merge_units<D>(*s_sched, a.partials, a.out, G, todo, *todo_count, et, NE, lists, false, false, nullptr);
                 if (et == 0) *todo_count = 0;
                 epilogue_sync();
             }
@@ -847,8 +858,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (trace && tid == 0) my_trace[12] = global_timer_ns();
     if (trace && tid == 0) my_trace[13] = (unsigned long long)*todo_count;
     if (!*s_abort && *todo_count > 0)
-        merge_units<D, true>(*s_sched, a.partials, a.out, G, todo, *todo_count, tid, S::kThreads, lists,
-                             trace ? my_trace + 28 : nullptr);
+        merge_units<D>(*s_sched, a.partials, a.out, G, todo, *todo_count, tid, S::kThreads, lists, true, false,
+                       trace ? my_trace + 28 : nullptr);
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
             // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
