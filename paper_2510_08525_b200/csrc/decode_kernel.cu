@@ -235,34 +235,24 @@ struct Smem {
 };
 
 // Merge of split units.  `units` lists (unit, first output row) of n units whose partial records
-// are all in memory; thread t of nt cooperating threads takes 4-float pieces of their G x D output
-// rows.  The records of a unit are merged in a fixed order (band by band, item by item), 16 at a
-// time -- all loads of a batch first, so a typical unit costs one trip to the L2 -- and the
-// arithmetic does not depend on nt, so the result does not depend on who merges or when.
-// `lists` is scratch for (first record, count) per unit and band.
-// (The schedule is passed as a copy in shared memory and everything else by value: a reference to
-// kernel parameters would turn every use into a slow generic load inside this non-inlined function.)
-// `whole`: all threads of the CTA take part (else the epilogue warps alone).  `dry`: everything but
-// the stores -- run once by the idle epilogue warps at kernel start so that the instructions are in
-// the SM's instruction cache when the merges at the end of the stream need them.
+// are all in memory, `lists` their records as (first record, count) per band; thread t of nt
+// cooperating threads takes 4-float pieces of their G x D output rows.  The records of a unit are
+// merged in a fixed order (band by band, item by item), 16 at a time -- all loads of a batch first,
+// so a typical unit costs one trip to the L2 -- and the arithmetic does not depend on nt, so the
+// result does not depend on who merges or when.  `dry`: everything but the stores -- run once by
+// the idle epilogue warps at kernel start so that the instructions are in the SM's instruction
+// cache when the merges at the end of the stream need them.  The caller orders the call after the
+// writes to `units` and `lists`.
+// (Everything comes by value or from shared memory: a reference to kernel parameters would turn
+// every use into a slow generic load inside this non-inlined function.)
 template <int D>
-__device__ __noinline__ void merge_units(const Schedule& sc, const float* partials, float* out, int G,
-                                         const int2* units, int n, int t, int nt, int2* lists, bool whole,
-                                         bool dry, unsigned long long* stamp)
+__device__ __noinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
+                                         const int2* lists, int n, int t, int nt, bool dry,
+                                         unsigned long long* stamp)
 {
     constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
     const int E = G * D4;
     const int PF = partial_floats(D, G), PH = partial_head_floats(G);
-    if (stamp && t == 0) stamp[9] = global_timer_ns();
-    for (int p = t; p < n * (sc.R + 1); p += nt) {
-        const int i = p / (sc.R + 1), r = p - i * (sc.R + 1);
-        int slot = 0, count = 0;
-        unit_partials(sc, units[i].x, r, slot, count);
-        lists[i * NB + r] = make_int2(slot, count);
-    }
-    if (stamp && t == 0) stamp[10] = global_timer_ns();
-    if (whole) __syncthreads(); else epilogue_sync();
-    if (stamp && t == 0) stamp[1] = global_timer_ns();
     __threadfence();
     if (stamp && t == 0) stamp[0] = global_timer_ns();
     const bool wide = nt >= E;                  // enough threads for one piece each, of nt / E units at a time
@@ -272,7 +262,7 @@ __device__ __noinline__ void merge_units(const Schedule& sc, const float* partia
         for (int j = ul; j < n; j += unit_lanes) {
             const int2* li = lists + j * NB;
             int F = 0;
-            for (int r = 0; r <= sc.R; ++r) F += li[r].y;
+            for (int r = 0; r <= R; ++r) F += li[r].y;
             for (int e = wide ? t - ul * E : t; e < E; e += wide ? E : nt) {
                 const int g = e / D4;
                 float M = kNegBig, L = 0.f;
@@ -324,7 +314,6 @@ __device__ __noinline__ void merge_units(const Schedule& sc, const float* partia
             }
         }
     }
-    if (whole) __syncthreads(); else epilogue_sync();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -756,7 +745,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         // run on unit 0 (its partial records hold whatever the last launch left; nothing is stored)
         if (et == 0) todo[kMaxTodo - 1] = make_int2(0, 0);
         epilogue_sync();
-        merge_units<D>(*s_sched, a.partials, a.out, G, todo + kMaxTodo - 1, 1, et, NE, lists, false, true, nullptr);
+        if (et <= kMaxRounds) {
+            int slot = 0, count = 0;
+            if (et <= sc.R) unit_partials(sc, 0, et, slot, count);
+            lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count);
+        }
+        epilogue_sync();
+        merge_units<D>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1, et, NE,
+                       true, nullptr);
+        epilogue_sync();
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;
@@ -767,22 +764,29 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
             epilogue_sync();
             if (*todo_count + pend_n > kMaxTodo) {
-                merge_units<D>(*s_sched, a.partials, a.out, G, todo, *todo_count, et, NE, lists, false, false, nullptr);
+                merge_units<D>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, et, NE, false, nullptr);
+                epilogue_sync();
                 if (et == 0) *todo_count = 0;
                 epilogue_sync();
             }
-            // 16 lanes per pending segment: lane r counts the unit's partial records in band r
+            // 16 lanes per pending segment: lane r looks up the unit's partial records in band r
+            constexpr int NB = kMaxRounds + 1;
             for (int base = 0; base < pend_n * 16; base += NE) {  // whole warps take part in the shuffles
                 const int p = base + et, i = p >> 4, r = p & 15;
                 const bool on = p < pend_n * 16;
-                int slot = 0, total = 0;
-                if (on && r <= sc.R) unit_partials(sc, pend[i].x, r, slot, total);
+                int slot = 0, count = 0;
+                if (on && r <= sc.R) unit_partials(sc, pend[i].x, r, slot, count);
+                int total = count;
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+                int idx = -1;
                 if (on && r == 0 && atomicAdd(&a.tickets[pend[i].x], 1) == total - 1) {
                     a.tickets[pend[i].x] = 0;  // ready for the next launch
-                    todo[atomicAdd(todo_count, 1)] = pend[i];
+                    idx = atomicAdd(todo_count, 1);
+                    todo[idx] = pend[i];
                 }
+                idx = __shfl_sync(0xffffffffu, idx, lane & 16);  // from lane r == 0 of this 16-lane group
+                if (idx >= 0 && r < NB) lists[idx * NB + r] = make_int2(slot, count);
             }
             epilogue_sync();
             pend_n = 0;
@@ -858,7 +862,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (trace && tid == 0) my_trace[12] = global_timer_ns();
     if (trace && tid == 0) my_trace[13] = (unsigned long long)*todo_count;
     if (!*s_abort && *todo_count > 0)
-        merge_units<D>(*s_sched, a.partials, a.out, G, todo, *todo_count, tid, S::kThreads, lists, true, false,
+        merge_units<D>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, tid, S::kThreads, false,
                        trace ? my_trace + 28 : nullptr);
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
