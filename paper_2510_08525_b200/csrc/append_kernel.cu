@@ -13,6 +13,12 @@ namespace {
 
 __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
 {
+    // The next kernel of the stream (the layer's decode launch) may start now: it waits for this
+    // grid to complete before it reads the rows written here.  This grid in turn completes only
+    // after the kernels before it have (the wait at the end), so that whoever waits for it has also
+    // waited for them.
+    grid_dep_launch();
+    if (a.wait_first) grid_dep_wait();
     const int chunks = a.head_dim / 8;  // 16-byte pieces per row
     const long long per_token = (long long)a.batch * a.kv_heads * chunks;
     const long long total = per_token * a.n_tokens * 2;
@@ -44,18 +50,27 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
         const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
         reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
     }
+    grid_dep_wait();
 }
 
 }  // namespace
 
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream)
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream, bool overlap)
 {
     const long long total = (long long)a.batch * a.kv_heads * (a.head_dim / 8) * a.n_tokens * 2;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;
-    append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, append_kernel, a);
 }
 
 }  // namespace rlkv

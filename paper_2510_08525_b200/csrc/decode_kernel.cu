@@ -369,6 +369,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     const bool trace = args.trace_on != 0;
     unsigned long long* my_trace = args.trace + (size_t)blockIdx.x * kTraceWords;
     if (trace && tid == 0) my_trace[0] = global_timer_ns();
+    // The next kernel of the stream may be scheduled as SMs become free.  This kernel itself may have
+    // been started while the kernels before it still run (see launch_decode): everything it does
+    // before a grid_dep_wait() -- fetching tiles that hold only older tokens, the arithmetic on them --
+    // touches nothing those kernels write.
+    if (tid == 0) grid_dep_launch();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
         if (tid == 0) atomicCAS(args.status, kStatusOk, kStatusSmemMisaligned);
@@ -621,6 +626,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             long long cy_expect = 0, cy_tma = 0, cy_q = 0, cy_item = 0, cy_seg = 0;
             const long long t_prod = clock64();
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
+            bool synced = false;  // has waited for the kernels before this one
             while (ok && k < sc.n_items) {
                 const long long ti0 = trace ? clock64() : 0;
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
@@ -658,6 +664,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         const UnitInfo u = locate(a, x);
                         seg_left = min(x1 - x, u.pos.run);
                         seg_idx = 0;
+                        // rows the append launch of this step writes: a compressed unit's ring, the
+                        // last tile of a full unit.  Everything else is older and may be fetched early.
+                        if (!synced && (k != (int)blockIdx.x || u.pos.uid >= sc.U || u.pos.tile + seg_left == u.tiles)) {
+                            grid_dep_wait();
+                            synced = true;
+                        }
                         if (u.pos.uid < sc.U) {
                             krow = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full) + u.pos.tile * kTile;
                             vrow = krow + a.rows_full;
@@ -729,6 +741,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             for (;;) {
                 if (!wait_bounded(smem_u32(claim_empty), par, s_abort, a.status, kStatusClaimWaitTimeout)) break;
                 par ^= 1u;
+                grid_dep_wait();  // the counter belongs to the launch before this one until that has completed
                 const int k = sc.P + atomicAdd(&a.counters[0], 1);
                 *claim_slot = k;
                 mbar_arrive(smem_u32(claim_full));
@@ -754,6 +767,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         merge_units<D>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1, et, NE,
                        true, nullptr);
         epilogue_sync();
+        grid_dep_wait();  // from here on these warps write results, partials and tickets
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;
@@ -873,6 +887,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                              kStatusDrainTimeout, false);
         }
         // the last CTA to finish rearms the claim counter for the next launch
+        grid_dep_wait();
         __threadfence();
         if (atomicAdd(&a.counters[1], 1) == (int)gridDim.x - 1) {
             a.counters[0] = 0;
@@ -883,11 +898,21 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 }
 
 template <int D, int NG>
-cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream)
+cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
+                       bool overlap)
 {
     const size_t smem = Smem<D, NG>::bytes(stages, a.group);
-    decode_kernel<D, NG><<<grid, Smem<D, NG>::kThreads, smem, stream>>>(a, tmap, stages);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(Smem<D, NG>::kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, decode_kernel<D, NG>, a, tmap, stages);
 }
 
 template <int D, int NG>
@@ -922,16 +947,16 @@ cudaError_t prepare_decode_kernels(int head_dim)
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream)
+                          int stages, int groups, cudaStream_t stream, bool overlap)
 {
     if (head_dim == 128) {
-        if (groups == 1) return launch_one<128, 1>(a, *tmap, grid, stages, stream);
-        if (groups == 2) return launch_one<128, 2>(a, *tmap, grid, stages, stream);
-        return launch_one<128, 3>(a, *tmap, grid, stages, stream);
+        if (groups == 1) return launch_one<128, 1>(a, *tmap, grid, stages, stream, overlap);
+        if (groups == 2) return launch_one<128, 2>(a, *tmap, grid, stages, stream, overlap);
+        return launch_one<128, 3>(a, *tmap, grid, stages, stream, overlap);
     }
-    if (groups == 1) return launch_one<64, 1>(a, *tmap, grid, stages, stream);
-    if (groups == 2) return launch_one<64, 2>(a, *tmap, grid, stages, stream);
-    return launch_one<64, 3>(a, *tmap, grid, stages, stream);
+    if (groups == 1) return launch_one<64, 1>(a, *tmap, grid, stages, stream, overlap);
+    if (groups == 2) return launch_one<64, 2>(a, *tmap, grid, stages, stream, overlap);
+    return launch_one<64, 3>(a, *tmap, grid, stages, stream, overlap);
 }
 
 }  // namespace rlkv

@@ -247,7 +247,8 @@ int make_tensor_map(rlkv_cache* c)
 
 bool valid_layer(const rlkv_cache* c, int layer) { return c && layer >= 0 && layer < c->layers; }
 
-int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s)
+int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s,
+              bool overlap = false)
 {
     AppendArgs a;
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
@@ -267,7 +268,10 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
     a.n_tokens = n_tokens;
     a.sink = c->sink;
     a.window = c->window;
-    RLKV_CUDA(launch_append(a, s));
+    // An overlapped append may run beside the decode launch of the layer before it, which never
+    // touches this layer's rows -- unless there is only one layer.
+    a.wait_first = (overlap && c->layers == 1) ? 1 : 0;
+    RLKV_CUDA(launch_append(a, s, overlap));
     c->launches++;
     c->len[layer] += n_tokens;
     return RLKV_OK;
@@ -311,7 +315,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     return RLKV_OK;
 }
 
-int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s)
+int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, bool overlap = false)
 {
     DecodeArgs a;
     int grid = 0;
@@ -321,7 +325,7 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.partials = dev_at<float>(c, c->lay.off_partials);
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
     a.counters = dev_at<int>(c, c->lay.off_status) + 4;
-    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap));
     c->launches++;
     return RLKV_OK;
 }
@@ -373,7 +377,7 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
     // the array still holds whatever the previous call (of any cache) left: counters and tickets
     // must start at zero
     RLKV_CUDA(cudaMemsetAsync(base, 0, head_bytes, s));
-    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s));
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, false));
     c->launches++;
     return RLKV_OK;
 }
@@ -581,11 +585,13 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
     const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
     for (int l = 0; l < c->layers; ++l) {
+        // All inputs of the step are complete before its first launch starts, so every later launch
+        // may overlap the one before it: the kernels wait on the device for exactly what they need.
         int rc = do_append(c, l, static_cast<const __nv_bfloat16*>(k) + l * kv_layer,
-                           static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s);
+                           static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s, l > 0);
         if (rc) return rc;
         rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                       static_cast<float*>(out) + l * q_layer, s);
+                       static_cast<float*>(out) + l * q_layer, s, true);
         if (rc) return rc;
     }
     return RLKV_OK;

@@ -233,6 +233,7 @@ struct AppendArgs {
     int batch, kv_heads, head_dim;
     int t0, n_tokens;           // tokens t0 .. t0+n_tokens-1 are appended
     int sink, window;
+    int wait_first;             // wait for the kernels before this one before writing (see launch_append)
 };
 
 // What a consumer needs to know about the unit behind a flat tile.
@@ -262,10 +263,21 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
     return u;
 }
 
+#ifdef __CUDACC__
+// Programmatic dependent launch: let the next kernel of the stream start / wait until the kernels
+// before this one have completed and their writes are visible (no-ops for ordinary launches).
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Launchers (defined in the .cu files).
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
+// `overlap`: launch with programmatic stream serialization, so that the kernel may start while the
+// kernel before it in the stream is still running; it then waits (griddepcontrol.wait) before it
+// touches anything that kernel may still use.  Only for launches whose inputs are known to be
+// complete (the layers of one rlkv_step after the first launch).
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream, bool overlap);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream);
+                          int stages, int groups, cudaStream_t stream, bool overlap);
 cudaError_t prepare_decode_kernels(int head_dim);
 size_t decode_smem_bytes(int head_dim, int stages, int group, int groups);
 
