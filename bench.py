@@ -61,6 +61,7 @@ def parse_args(argv=None):
     p.add_argument("--ctas-per-sm", type=int, default=0)
     p.add_argument("--stages", type=int, default=0)
     p.add_argument("--groups", type=int, default=0, help="consumer warp groups of the decode kernel")
+    p.add_argument("--item-tiles", type=int, default=0, help="smallest work item of the decode kernel, in 64-row tiles")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     return p.parse_args(argv)
@@ -280,8 +281,8 @@ def run_ours(args, w, mask):
     total_new = passes * (K + W) + 8
     cache = harness.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, w.context + total_new, mask,
                           w.sink, w.window, device=dev)
-    if args.ctas_per_sm or args.stages or args.groups:
-        rl.rlkv_set_decode_config(cache.handle, args.ctas_per_sm, args.stages, args.groups)
+    if args.ctas_per_sm or args.stages or args.groups or args.item_tiles:
+        rl.rlkv_set_decode_config(cache.handle, args.ctas_per_sm, args.stages, args.groups, args.item_tiles)
     harness.fill_cache(cache, w, w.context)
 
     # inputs of every step, resident on the device (and a pinned host copy for the e2e pass)

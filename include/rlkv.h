@@ -154,7 +154,7 @@ int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
  * and the size in 64-row tiles of the smallest work items the K/V scan is cut into (2..1024).
  * 0 keeps the current value (stages: lowered if the new shape no longer fits).  RLKV_EINVAL if the
  * shape does not fit in shared memory.  Defaults: 1 CTA per SM, 2 groups, as many stages as fit,
- * 4 tiles.  Results do not depend on these knobs beyond floating-point summation order. */
+ * 16 tiles.  Results do not depend on these knobs beyond floating-point summation order. */
 int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups,
                            int item_tiles);
 /* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, 32

@@ -55,7 +55,7 @@ struct Layout {
 
 constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
 constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
-constexpr int kDefaultItemTiles = 4;
+constexpr int kDefaultItemTiles = 16;
 
 // Most partial records a decode launch of this shape can write, over every length up to tf tiles
 // per full unit and every grid up to max_grid CTAs.
