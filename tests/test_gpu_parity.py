@@ -352,3 +352,35 @@ def test_dynamic_work_claims_do_not_change_bits(rl, hz, cuda_device):
     words = rl.rlkv_debug_trace(cache.handle, 0, read=True)
     tiles = B * (6 * ((n + 63) // 64) + 2 * 2)
     assert int(words[:, 5].sum()) == tiles
+
+
+# ------------------------------------------------------------------------------------------ decode loop
+@pytest.mark.parametrize("layers", [1, 2])
+def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
+    """A reduced chain-of-thought loop: prompt of 300 tokens, then 700 whole steps through rlkv_step
+    (whose launches overlap one another on the device), sink 16 + window 240 so the ring wraps several
+    times.  Outputs are compared with the oracle every 50 steps and at the end, cache state bit for bit
+    at the end.  One layer is the case where an append may not run beside the decode before it."""
+    Hkv, Hq, D, B, S, W, prompt, steps = 2, 8, 128, 2, 16, 240, 300, 700
+    mask = ([1, 0] + [0, 1])[:2 * layers]
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, cuda_device)
+    for l in range(layers):
+        feed(cache, oracle, l, rand_bf16((prompt, B, Hkv, D), 50 + l), rand_bf16((prompt, B, Hkv, D), 60 + l), True)
+    out = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+    K = rand_bf16((steps, layers, B, Hkv, D), 70)
+    V = rand_bf16((steps, layers, B, Hkv, D), 71)
+    Q = rand_bf16((steps, layers, B, Hq, D), 72)
+    Kd, Vd, Qd = K.to(cuda_device), V.to(cuda_device), Q.to(cuda_device)
+    for t in range(steps):
+        rl.rlkv_step(cache.handle, Kd[t], Vd[t], Qd[t], out)
+        for l in range(layers):
+            assert oracle.append(l, K[t, l], V[t, l]) == 0
+        if t % 50 == 49 or t == steps - 1:
+            got = out.cpu().numpy()
+            for l in range(layers):
+                check_out(got[l], oracle.decode(l, Q[t, l]))
+    check_state(cache, oracle)
+    assert cache.status() == 0
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_step(cache.handle, Kd[0], Vd[0], Qd[0], out)
+    assert e.value.code == rl.RLKV_EFULL
