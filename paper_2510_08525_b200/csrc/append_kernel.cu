@@ -13,12 +13,6 @@ namespace {
 
 __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
 {
-    // The next kernel of the stream (the layer's decode launch) may start now: it waits for this
-    // grid to complete before it reads the rows written here.  This grid in turn completes only
-    // after the kernels before it have (the wait at the end), so that whoever waits for it has also
-    // waited for them.
-    grid_dep_launch();
-    if (a.wait_first) grid_dep_wait();
     const int chunks = a.head_dim / 8;  // 16-byte pieces per row
     const long long per_token = (long long)a.batch * a.kv_heads * chunks;
     const long long total = per_token * a.n_tokens * 2;
@@ -50,27 +44,61 @@ __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
         const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
         reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
     }
-    grid_dep_wait();
+}
+
+// One token for every layer: the same row arithmetic, one more index.
+__global__ void __launch_bounds__(256) append_all_kernel(const __grid_constant__ AppendAllArgs a)
+{
+    const int chunks = a.head_dim / 8;
+    const long long per_layer = (long long)a.batch * a.kv_heads * chunks * 2;
+    const long long total = per_layer * a.n_layers;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long r = i;
+        const int c = (int)(r % chunks);
+        r /= chunks;
+        const int h = (int)(r % a.kv_heads);
+        r /= a.kv_heads;
+        const int b = (int)(r % a.batch);
+        r /= a.batch;
+        const int kv = (int)(r % 2);  // 0 = K, 1 = V
+        const int l = (int)(r / 2);
+        const LayerDesc d = a.layers[l];
+        const int t = a.t0[l];
+        const int slot = a.slot_of_head[l * a.kv_heads + h];
+        long long row;
+        if (slot >= 0) {
+            row = d.full_row0 + ((long long)(b * d.n_full + slot) * 2 + kv) * a.rows_full + t;
+        } else {
+            const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
+            row = d.comp_row0 + ((long long)(b * d.n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
+        }
+        const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.batch + b) * a.kv_heads + h) * a.head_dim;
+        const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
+        reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
+    }
 }
 
 }  // namespace
 
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream, bool overlap)
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream)
 {
     const long long total = (long long)a.batch * a.kv_heads * (a.head_dim / 8) * a.n_tokens * 2;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)blocks);
-    cfg.blockDim = dim3(256);
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, append_kernel, a);
+    append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream)
+{
+    const long long total = (long long)a.n_layers * a.batch * a.kv_heads * (a.head_dim / 8) * 2;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    if (blocks < 1) blocks = 1;
+    append_all_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
+    return cudaGetLastError();
 }
 
 }  // namespace rlkv

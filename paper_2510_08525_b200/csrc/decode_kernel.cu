@@ -369,11 +369,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     const bool trace = args.trace_on != 0;
     unsigned long long* my_trace = args.trace + (size_t)blockIdx.x * kTraceWords;
     if (trace && tid == 0) my_trace[0] = global_timer_ns();
-    // The next kernel of the stream may be scheduled as SMs become free.  This kernel itself may have
-    // been started while the kernels before it still run (see launch_decode): everything it does
-    // before a grid_dep_wait() -- fetching tiles that hold only older tokens, the arithmetic on them --
-    // touches nothing those kernels write.
-    if (tid == 0) grid_dep_launch();
+    // Overlapped launches (the layers of one decode step): the next layer's kernel is scheduled as SMs
+    // become free and touches nothing this one uses.  Only the step's first layer (dep_wait) may be
+    // running before the step's append launch has completed: it fetches and processes tiles that hold
+    // only older tokens, waits (grid_dep_wait) before it touches anything else, and only then lets
+    // the next layer start, which therefore never has to wait.
+    if (tid == 0 && !args.dep_wait) grid_dep_launch();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
         if (tid == 0) atomicCAS(args.status, kStatusOk, kStatusSmemMisaligned);
@@ -666,7 +667,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         seg_idx = 0;
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit.  Everything else is older and may be fetched early.
-                        if (!synced && (k != (int)blockIdx.x || u.pos.uid >= sc.U || u.pos.tile + seg_left == u.tiles)) {
+                        if (a.dep_wait && !synced &&
+                            (k != (int)blockIdx.x || u.pos.uid >= sc.U || u.pos.tile + seg_left == u.tiles)) {
                             grid_dep_wait();
                             synced = true;
                         }
@@ -741,8 +743,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             for (;;) {
                 if (!wait_bounded(smem_u32(claim_empty), par, s_abort, a.status, kStatusClaimWaitTimeout)) break;
                 par ^= 1u;
-                grid_dep_wait();  // the counter belongs to the launch before this one until that has completed
-                const int k = sc.P + atomicAdd(&a.counters[0], 1);
+                // the counter only ever grows; this launch's claims start at claim_base
+                const int k = sc.P + (int)(atomicAdd(a.claim_counter, 1u) - a.claim_base);
                 *claim_slot = k;
                 mbar_arrive(smem_u32(claim_full));
                 if (k >= sc.n_items) break;  // the producer stops asking once it has seen this answer
@@ -767,7 +769,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         merge_units<D>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1, et, NE,
                        true, nullptr);
         epilogue_sync();
-        grid_dep_wait();  // from here on these warps write results, partials and tickets
+        if (a.dep_wait) {  // from here on these warps write results, partials and tickets
+            grid_dep_wait();
+            if (et == 0) grid_dep_launch();
+        }
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)
         const bool tre = trace && et == 0;
@@ -885,13 +890,6 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             for (int j = issued > stages ? issued - stages : 0; j < issued; ++j)
                 wait_bounded(smem_u32(full_bar + j % stages), (uint32_t)(j / stages) & 1u, s_abort, a.status,
                              kStatusDrainTimeout, false);
-        }
-        // the last CTA to finish rearms the claim counter for the next launch
-        grid_dep_wait();
-        __threadfence();
-        if (atomicAdd(&a.counters[1], 1) == (int)gridDim.x - 1) {
-            a.counters[0] = 0;
-            a.counters[1] = 0;
         }
     }
     if (trace && tid == 0) my_trace[3] = global_timer_ns();

@@ -9,8 +9,10 @@
 //             (the constant-size pool of Section 4.3 of the paper).
 //   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
 //   tickets   int32 [layers][batch*kv_heads]   (split bookkeeping, zero between launches)
-//   status    int32 kernel status word, then the two work-claim counters (zero between launches)
-//   partials  float [max_slots][partial_floats]  (split-KV scratch)
+//   tables    then LayerDesc[layers] (where each layer's regions start; for the step's append launch)
+//   status    int32 kernel status word, then two work-claim counters (they only grow; consecutive
+//             launches of a step alternate between them)
+//   partials  float [2][max_slots][partial_floats]  (split-KV scratch; the two halves alternate too)
 //   staging   k, v, q, out of one whole step, for rlkv_step_host
 //   trace     uint64 [max_grid][8]  (debug trace of the decode kernel)
 #include <stdio.h>
@@ -48,6 +50,7 @@ struct Layout {
     std::vector<int> n_full, n_comp;
     std::vector<long long> full_row0, comp_row0;  // per layer, in pool rows
     long long pool_rows = 0;
+    size_t off_layer_desc = 0;
     size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
     size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_trace = 0, total = 0;
     int max_grid = 0, max_items = 0;
@@ -55,7 +58,7 @@ struct Layout {
 
 constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
 constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
-constexpr int kDefaultItemTiles = 16;
+constexpr int kDefaultItemTiles = 32;
 
 // Most partial records a decode launch of this shape can write, over every length up to tf tiles
 // per full unit and every grid up to max_grid CTAs.
@@ -119,13 +122,15 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     L.off_pool = off;
     off = align_up(off + (size_t)row * head_dim * 2, 1024);
     L.off_tables = off;
-    off = align_up(off + (size_t)2 * layers * kv_heads * sizeof(int), 1024);
+    off = align_up(off + (size_t)2 * layers * kv_heads * sizeof(int), 16);
+    L.off_layer_desc = off;
+    off = align_up(off + (size_t)layers * sizeof(LayerDesc), 1024);
     L.off_tickets = off;
     off = align_up(off + (size_t)layers * batch * kv_heads * sizeof(int), 1024);
     L.off_status = off;
     off = align_up(off + 64, 1024);
     L.off_partials = off;
-    off = align_up(off + (size_t)L.max_items * partial_floats(head_dim, q_heads / kv_heads) * sizeof(float), 1024);
+    off = align_up(off + (size_t)2 * L.max_items * partial_floats(head_dim, q_heads / kv_heads) * sizeof(float), 1024);
     const size_t kv_step = (size_t)layers * batch * kv_heads * head_dim * 2;
     const size_t q_step = (size_t)layers * batch * q_heads * head_dim * 2;
     L.off_k = off;
@@ -181,6 +186,7 @@ struct rlkv_cache {
     int device, sm_count;
     int ctas_per_sm, stages, groups, item_tiles;  // decode launch shape (rlkv_set_decode_config)
     int trace_on;
+    unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
     Layout lay;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -247,8 +253,7 @@ int make_tensor_map(rlkv_cache* c)
 
 bool valid_layer(const rlkv_cache* c, int layer) { return c && layer >= 0 && layer < c->layers; }
 
-int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s,
-              bool overlap = false)
+int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s)
 {
     AppendArgs a;
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
@@ -268,10 +273,7 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
     a.n_tokens = n_tokens;
     a.sink = c->sink;
     a.window = c->window;
-    // An overlapped append may run beside the decode launch of the layer before it, which never
-    // touches this layer's rows -- unless there is only one layer.
-    a.wait_first = (overlap && c->layers == 1) ? 1 : 0;
-    RLKV_CUDA(launch_append(a, s, overlap));
+    RLKV_CUDA(launch_append(a, s));
     c->launches++;
     c->len[layer] += n_tokens;
     return RLKV_OK;
@@ -309,23 +311,36 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     // more CTAs are launched than there are items
     int grid = c->sm_count * c->ctas_per_sm;
     if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * a.n_comp, tiles_comp, grid, c->item_tiles);
+    // smallest work item: the configured size, less where the launch is too small to give every CTA
+    // one item of that size
+    int item_tiles = (int)(all_tiles / (1ll * grid));
+    if (item_tiles > c->item_tiles) item_tiles = c->item_tiles;
+    if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
+    a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * a.n_comp, tiles_comp, grid, item_tiles);
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     *grid_out = grid;
     return RLKV_OK;
 }
 
-int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, bool overlap = false)
+// `half`: which half of the scratch memory (partials, claim counter) the launch uses; `overlap` and
+// `dep_wait` as in launch_decode.
+int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, int half = 0, bool overlap = false,
+              bool dep_wait = false, int* grid_out = nullptr)
 {
     DecodeArgs a;
     int grid = 0;
     int rc = build_decode_args(c, layer, q, out, a, &grid);
     if (rc) return rc;
     if (a.sched.n_slots > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
-    a.partials = dev_at<float>(c, c->lay.off_partials);
+    a.partials = dev_at<float>(c, c->lay.off_partials) +
+                 (size_t)half * c->lay.max_items * partial_floats(c->head_dim, a.group);
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
-    a.counters = dev_at<int>(c, c->lay.off_status) + 4;
+    a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4 + half;
+    a.claim_base = c->claims[half];
+    a.dep_wait = dep_wait ? 1 : 0;
     RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap));
+    c->claims[half] += (unsigned int)a.sched.n_items;  // every CTA claims until it is told there is no more
+    if (grid_out) *grid_out = grid;
     c->launches++;
     return RLKV_OK;
 }
@@ -365,14 +380,16 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
     if (rc) return rc;
     // carve the static array: the two counters and one ticket per (batch row, KV head), then the
     // partial records of this launch
-    const size_t head_bytes = align_up((2 + (size_t)c->batch * c->kv_heads) * sizeof(int), 256);
+    const size_t head_bytes = align_up((2 + (size_t)c->batch * c->kv_heads) * sizeof(int), 256);  // claim counter, tickets
     const size_t partial_bytes = (size_t)a.sched.n_slots * partial_floats(c->head_dim, a.group) * sizeof(float);
     if (head_bytes + partial_bytes > kStaticScratchBytes) return RLKV_ESCRATCH;
     unsigned char* base = nullptr;
     rc = static_scratch_address(c->device, &base);
     if (rc) return rc;
-    a.counters = reinterpret_cast<int*>(base);
-    a.tickets = a.counters + 2;
+    a.claim_counter = reinterpret_cast<unsigned int*>(base);
+    a.claim_base = 0;
+    a.dep_wait = 0;
+    a.tickets = reinterpret_cast<int*>(base) + 2;
     a.partials = reinterpret_cast<float*>(base + head_bytes);
     // the array still holds whatever the previous call (of any cache) left: counters and tickets
     // must start at zero
@@ -431,6 +448,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->groups = 2;
     c->item_tiles = kDefaultItemTiles;
     c->trace_on = 0;
+    c->claims[0] = c->claims[1] = 0;
     c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
     rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
     if (rc) { delete c; return rc; }
@@ -485,6 +503,13 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     if (e == cudaSuccess)
         e = cudaMemcpy(c->dev_base + c->lay.off_tables + tbytes, c->head_of_slot.data(), tbytes,
                        cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        std::vector<LayerDesc> desc(layers);
+        for (int l = 0; l < layers; ++l)
+            desc[l] = LayerDesc{c->lay.full_row0[l], c->lay.comp_row0[l], c->lay.n_full[l], c->lay.n_comp[l]};
+        e = cudaMemcpy(c->dev_base + c->lay.off_layer_desc, desc.data(), desc.size() * sizeof(LayerDesc),
+                       cudaMemcpyHostToDevice);
+    }
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaMemcpy(tables)"));
     rc = make_tensor_map(c);
     if (rc) return fail(rc);
@@ -517,6 +542,7 @@ int rlkv_cache_reset(rlkv_cache* c, void* stream)
     int rc = zero_state(c, static_cast<cudaStream_t>(stream));
     if (rc) return rc;
     std::fill(c->len.begin(), c->len.end(), 0);
+    c->claims[0] = c->claims[1] = 0;  // zero_state has cleared the counters on the device
     return RLKV_OK;
 }
 
@@ -584,14 +610,51 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
+    if (c->layers <= kMaxStepLayers) {
+        // One launch appends the new token to every layer.  All inputs of the step are complete
+        // before that launch starts, so the decode launches may overlap one another: consecutive
+        // layers alternate between the two halves of the scratch memory, and the first one waits on
+        // the device for the append launch before it reads rows that launch writes.
+        AppendAllArgs aa;
+        aa.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+        aa.layers = dev_at<LayerDesc>(c, c->lay.off_layer_desc);
+        aa.slot_of_head = dev_at<int>(c, c->lay.off_tables);
+        aa.k = static_cast<const __nv_bfloat16*>(k);
+        aa.v = static_cast<const __nv_bfloat16*>(v);
+        aa.n_layers = c->layers;
+        aa.rows_full = c->lay.rows_full;
+        aa.rows_comp = c->lay.rows_comp;
+        aa.batch = c->batch;
+        aa.kv_heads = c->kv_heads;
+        aa.head_dim = c->head_dim;
+        aa.sink = c->sink;
+        aa.window = c->window;
+        for (int l = 0; l < c->layers; ++l) aa.t0[l] = c->len[l];
+        RLKV_CUDA(launch_append_all(aa, s));
+        c->launches++;
+        for (int l = 0; l < c->layers; ++l) c->len[l] += 1;
+        // Launch l and launch l-2 share a half of the scratch memory, so launch l must not start before
+        // launch l-2 has completed.  An overlapped launch starts when every CTA of launch l-1 has
+        // started; if launch l-1 puts exactly one CTA on every SM (and a CTA takes a whole SM: its
+        // registers see to that), all of them having started means that no CTA of launch l-2 is left.
+        // After a smaller launch the next one is an ordinary launch, which waits for everything.
+        bool prev_fills_gpu = true;  // the append launch is followed by an overlapped launch that waits on the device
+        for (int l = 0; l < c->layers; ++l) {
+            int grid = 0;
+            const bool overlap = prev_fills_gpu;
+            int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
+                               static_cast<float*>(out) + l * q_layer, s, l & 1, overlap, overlap && l == 0, &grid);
+            if (rc) return rc;
+            prev_fills_gpu = (grid == c->sm_count && c->ctas_per_sm == 1);
+        }
+        return RLKV_OK;
+    }
     for (int l = 0; l < c->layers; ++l) {
-        // All inputs of the step are complete before its first launch starts, so every later launch
-        // may overlap the one before it: the kernels wait on the device for exactly what they need.
         int rc = do_append(c, l, static_cast<const __nv_bfloat16*>(k) + l * kv_layer,
-                           static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s, l > 0);
+                           static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s);
         if (rc) return rc;
         rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                       static_cast<float*>(out) + l * q_layer, s, true);
+                       static_cast<float*>(out) + l * q_layer, s);
         if (rc) return rc;
     }
     return RLKV_OK;

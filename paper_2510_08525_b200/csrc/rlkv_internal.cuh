@@ -11,6 +11,7 @@ namespace rlkv {
 constexpr int kTile = 64;        // tokens per K/V tile (one pipeline stage holds a K and a V tile)
 constexpr int kMaxGroup = 8;     // query heads per KV head handled by one tile pass
 constexpr int kMaxKvHeads = 128; // KV heads per layer (their order travels in the kernel arguments)
+constexpr int kMaxStepLayers = 128;  // layers whose appends rlkv_step does in one launch
 constexpr int kGroupWarps = 4;   // consumer warps that share one tile (16 tokens each)
 constexpr int kMaxConsumerGroups = 3;
 constexpr int kMaxDynamicSmem = 227 * 1024;
@@ -210,7 +211,10 @@ struct DecodeArgs {
     float* out;                 // [batch][q_heads][head_dim]
     float* partials;            // [sched.n_slots][partial_floats]
     int* tickets;               // one per unit of this layer, zero between launches
-    int* counters;              // [0] items claimed beyond the first P, [1] CTAs finished; zero between launches
+    unsigned int* claim_counter;  // items claimed beyond the first P, over all launches so far (never reset)
+    unsigned int claim_base;      // its value when this launch starts: every launch adds exactly sched.n_items
+    int dep_wait;               // the launch may start before the kernel that wrote this step's new rows has
+                                // completed: wait for it before touching what it writes (see launch_decode)
     int* status;                // device error word
     unsigned long long* trace;  // debug: [grid][kTraceWords]
     int n_full, n_comp;         // heads of each class in this layer
@@ -233,7 +237,6 @@ struct AppendArgs {
     int batch, kv_heads, head_dim;
     int t0, n_tokens;           // tokens t0 .. t0+n_tokens-1 are appended
     int sink, window;
-    int wait_first;             // wait for the kernels before this one before writing (see launch_append)
 };
 
 // What a consumer needs to know about the unit behind a flat tile.
@@ -271,11 +274,28 @@ __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.w
 #endif
 
 // Launchers (defined in the .cu files).
-// `overlap`: launch with programmatic stream serialization, so that the kernel may start while the
-// kernel before it in the stream is still running; it then waits (griddepcontrol.wait) before it
-// touches anything that kernel may still use.  Only for launches whose inputs are known to be
-// complete (the layers of one rlkv_step after the first launch).
-cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream, bool overlap);
+// `overlap` (launch_decode): launch with programmatic stream serialization, so that the kernel may
+// start while the kernel before it in the stream is still running.  Only for the decode launches of
+// one rlkv_step, whose inputs are complete before the step's first launch: consecutive layers use
+// different halves of the scratch memory and touch nothing of each other, and the first layer's
+// launch (dep_wait) waits on the device for the step's append launch before it reads new rows.
+cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
+
+// The appends of one token to every layer, in one launch (rlkv_step).
+struct LayerDesc {
+    long long full_row0, comp_row0;  // first pool row of the layer's full-head / compressed-head region
+    int n_full, n_comp;
+};
+struct AppendAllArgs {
+    __nv_bfloat16* pool;
+    const LayerDesc* layers;    // device, [n_layers]
+    const int* slot_of_head;    // device, [n_layers][kv_heads]
+    const __nv_bfloat16* k;     // [n_layers][batch][kv_heads][head_dim]
+    const __nv_bfloat16* v;
+    int n_layers, rows_full, rows_comp, batch, kv_heads, head_dim, sink, window;
+    int t0[kMaxStepLayers];     // token index appended to each layer
+};
+cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
                           int stages, int groups, cudaStream_t stream, bool overlap);
 cudaError_t prepare_decode_kernels(int head_dim);
