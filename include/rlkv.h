@@ -121,8 +121,8 @@ size_t rlkv_static_scratch_bytes(void);
 
 /* One whole decode step: for every layer, append then attend.  Device buffers:
  * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];
- * out fp32 [layers][batch][q_heads][head_dim].  The results equal those of the per-layer calls in
- * order.  Because all inputs are there before the first launch, the step is issued as one append
+ * out fp32 [layers][batch][q_heads][head_dim].  The results are those of the per-layer calls in
+ * order (up to floating-point summation order: the step cuts the work into larger items).  Because all inputs are there before the first launch, the step is issued as one append
  * launch for all layers followed by the layers' attention launches, which overlap on the device
  * (programmatic dependent launch): every buffer must be complete when the call is made and stay
  * untouched until the work on `stream` has finished.  RLKV_EFULL (nothing done) if any layer is at
@@ -159,7 +159,7 @@ int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
  * launch too small to give every CTA one such item uses smaller ones).
  * 0 keeps the current value (stages: lowered if the new shape no longer fits).  RLKV_EINVAL if the
  * shape does not fit in shared memory.  Defaults: 1 CTA per SM, 2 groups, as many stages as fit,
- * 32 tiles.  Results do not depend on these knobs beyond floating-point summation order. */
+ * 32 tiles inside rlkv_step (whose launches overlap) and 8 tiles for a launch on its own.  Results do not depend on these knobs beyond floating-point summation order. */
 int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups,
                            int item_tiles);
 /* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, 32

@@ -58,7 +58,8 @@ struct Layout {
 
 constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
 constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
-constexpr int kDefaultItemTiles = 32;
+constexpr int kDefaultItemTiles = 32;        // launches of rlkv_step, which overlap: coarse items, few partials
+constexpr int kDefaultItemTilesAlone = 8;    // a launch on its own: finer items for an even finish
 
 // Most partial records a decode launch of this shape can write, over every length up to tf tiles
 // per full unit and every grid up to max_grid CTAs.
@@ -185,6 +186,7 @@ struct rlkv_cache {
     int layers, kv_heads, q_heads, head_dim, batch, max_len, sink, window;
     int device, sm_count;
     int ctas_per_sm, stages, groups, item_tiles;  // decode launch shape (rlkv_set_decode_config)
+    int item_tiles_alone;                         // item_tiles of launches outside rlkv_step
     int trace_on;
     unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
     Layout lay;
@@ -281,7 +283,8 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
 
 // Everything of a decode launch except where its split-KV work area lives.  Returns the grid size
 // in *grid_out.
-int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, DecodeArgs& a, int* grid_out)
+int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, DecodeArgs& a, int* grid_out,
+                      bool in_step = false)
 {
     const int n = c->len[layer];
     const int cap = c->sink + c->window;
@@ -314,7 +317,8 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     // smallest work item: the configured size, less where the launch is too small to give every CTA
     // one item of that size
     int item_tiles = (int)(all_tiles / (1ll * grid));
-    if (item_tiles > c->item_tiles) item_tiles = c->item_tiles;
+    const int most = in_step ? c->item_tiles : c->item_tiles_alone;
+    if (item_tiles > most) item_tiles = most;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * a.n_comp, tiles_comp, grid, item_tiles);
     if (grid > a.sched.n_items) grid = a.sched.n_items;
@@ -329,7 +333,7 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
 {
     DecodeArgs a;
     int grid = 0;
-    int rc = build_decode_args(c, layer, q, out, a, &grid);
+    int rc = build_decode_args(c, layer, q, out, a, &grid, overlap);
     if (rc) return rc;
     if (a.sched.n_slots > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
     a.partials = dev_at<float>(c, c->lay.off_partials) +
@@ -447,6 +451,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->ctas_per_sm = 1;
     c->groups = 2;
     c->item_tiles = kDefaultItemTiles;
+    c->item_tiles_alone = kDefaultItemTilesAlone;
     c->trace_on = 0;
     c->claims[0] = c->claims[1] = 0;
     c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
@@ -561,7 +566,7 @@ int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consu
     c->ctas_per_sm = cps;
     c->stages = st;
     c->groups = ng;
-    if (item_tiles) c->item_tiles = item_tiles;
+    if (item_tiles) c->item_tiles = c->item_tiles_alone = item_tiles;
     return RLKV_OK;
 }
 

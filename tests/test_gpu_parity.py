@@ -285,7 +285,8 @@ def test_step_and_step_host_equal_per_layer_calls(rl, hz, cuda_device):
         out_c = torch.empty(out_a.shape, dtype=torch.float32).pin_memory()
         rl.rlkv_step_host(c.handle, kh, vh, qh, out_c)
         torch.cuda.synchronize()
-        assert torch.equal(out_a, out_b) and torch.equal(out_a.cpu(), out_c)
+        # the step and the per-layer calls may cut the work differently: same values up to summation order
+        assert torch.allclose(out_a, out_b, atol=1e-4, rtol=0) and torch.equal(out_b.cpu(), out_c)
         for l in range(w.layers):
             oracle.append(l, k[l].cpu(), v[l].cpu())
             check_out(out_a[l].cpu().numpy(), oracle.decode(l, q[l].cpu()))
