@@ -189,6 +189,9 @@ struct rlkv_cache {
     int item_tiles_alone;                         // item_tiles of launches outside rlkv_step
     int trace_on;
     unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
+    cudaStream_t copy_stream;      // rlkv_step_host: copies that run beside the kernels
+    cudaEvent_t ev_start, ev_done; // order copy_stream after / before the caller's stream
+    cudaEvent_t ev_in[4], ev_out[4];  // per chunk of layers: its q has arrived / its results are ready
     Layout lay;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -200,6 +203,18 @@ struct rlkv_cache {
 };
 
 namespace {
+
+void destroy_copy_objects(rlkv_cache* c)
+{
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->ev_start) cudaEventDestroy(c->ev_start);
+    if (c->ev_done) cudaEventDestroy(c->ev_done);
+    for (int i = 0; i < 4; ++i) {
+        if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+        if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+    }
+    c->copy_stream = nullptr;
+}
 
 template <typename T>
 T* dev_at(const rlkv_cache* c, size_t off) { return reinterpret_cast<T*>(c->dev_base + off); }
@@ -403,6 +418,56 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
     return RLKV_OK;
 }
 
+// The launches of one decode step on device buffers (k, v, q, out as in rlkv_step).
+// step_append: one launch appends the new token to every layer.  step_decode: the decode launches of
+// layers [l0, l1).  All inputs of the step are complete before its first launch starts, so the decode
+// launches may overlap one another: consecutive layers alternate between the two halves of the
+// scratch memory, and the first layer's launch waits on the device for the append launch before it
+// reads rows that launch writes.
+// Launch l and launch l-2 share a half of the scratch memory, so launch l must not start before
+// launch l-2 has completed.  An overlapped launch starts when every CTA of launch l-1 has started; if
+// launch l-1 puts exactly one CTA on every SM (and a CTA takes a whole SM: its registers see to that),
+// all of them having started means that no CTA of launch l-2 is left.  After a smaller launch, or
+// after anything but a kernel of this step in the stream (`fresh`), the next launch is an ordinary
+// one, which waits for everything before it.
+int step_append(rlkv_cache* c, const void* k, const void* v, cudaStream_t s)
+{
+    AppendAllArgs aa;
+    aa.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+    aa.layers = dev_at<LayerDesc>(c, c->lay.off_layer_desc);
+    aa.slot_of_head = dev_at<int>(c, c->lay.off_tables);
+    aa.k = static_cast<const __nv_bfloat16*>(k);
+    aa.v = static_cast<const __nv_bfloat16*>(v);
+    aa.n_layers = c->layers;
+    aa.rows_full = c->lay.rows_full;
+    aa.rows_comp = c->lay.rows_comp;
+    aa.batch = c->batch;
+    aa.kv_heads = c->kv_heads;
+    aa.head_dim = c->head_dim;
+    aa.sink = c->sink;
+    aa.window = c->window;
+    for (int l = 0; l < c->layers; ++l) aa.t0[l] = c->len[l];
+    RLKV_CUDA(launch_append_all(aa, s));
+    c->launches++;
+    for (int l = 0; l < c->layers; ++l) c->len[l] += 1;
+    return RLKV_OK;
+}
+
+int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStream_t s, bool fresh)
+{
+    const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
+    bool prev_ok = !fresh;  // right after the append launch an overlapped launch is fine: it waits on the device
+    for (int l = l0; l < l1; ++l) {
+        int grid = 0;
+        const bool overlap = prev_ok;
+        int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
+                           static_cast<float*>(out) + l * q_layer, s, l & 1, overlap, overlap && l == 0, &grid);
+        if (rc) return rc;
+        prev_ok = (grid == c->sm_count && c->ctas_per_sm == 1);
+    }
+    return RLKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -454,6 +519,9 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->item_tiles_alone = kDefaultItemTilesAlone;
     c->trace_on = 0;
     c->claims[0] = c->claims[1] = 0;
+    c->copy_stream = nullptr;
+    c->ev_start = c->ev_done = nullptr;
+    for (int i = 0; i < 4; ++i) c->ev_in[i] = c->ev_out[i] = nullptr;
     c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
     rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
     if (rc) { delete c; return rc; }
@@ -478,6 +546,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
             if (!c->is_full[l * kv_heads + h]) c->head_of_slot[l * kv_heads + nf + nc++] = h;
     }
     auto fail = [&](int code) {
+        destroy_copy_objects(c);
         if (c->owns_buffer && c->dev_base) cudaFree(c->dev_base);
         delete c;
         return code;
@@ -520,6 +589,14 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     if (rc) return fail(rc);
     e = prepare_decode_kernels(head_dim);
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaFuncSetAttribute"));
+    e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done, cudaEventDisableTiming);
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaStreamCreate/cudaEventCreate"));
     e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceSynchronize"));
     *out = c;
@@ -530,6 +607,10 @@ int rlkv_cache_destroy(rlkv_cache* c)
 {
     if (!c) return RLKV_EINVAL;
     int rc = RLKV_OK;
+    {
+        DeviceGuard g(c->device);
+        destroy_copy_objects(c);
+    }
     if (c->owns_buffer && c->dev_base) {
         DeviceGuard g(c->device);
         cudaError_t e = cudaFree(c->dev_base);
@@ -616,43 +697,9 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
     const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
     if (c->layers <= kMaxStepLayers) {
-        // One launch appends the new token to every layer.  All inputs of the step are complete
-        // before that launch starts, so the decode launches may overlap one another: consecutive
-        // layers alternate between the two halves of the scratch memory, and the first one waits on
-        // the device for the append launch before it reads rows that launch writes.
-        AppendAllArgs aa;
-        aa.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
-        aa.layers = dev_at<LayerDesc>(c, c->lay.off_layer_desc);
-        aa.slot_of_head = dev_at<int>(c, c->lay.off_tables);
-        aa.k = static_cast<const __nv_bfloat16*>(k);
-        aa.v = static_cast<const __nv_bfloat16*>(v);
-        aa.n_layers = c->layers;
-        aa.rows_full = c->lay.rows_full;
-        aa.rows_comp = c->lay.rows_comp;
-        aa.batch = c->batch;
-        aa.kv_heads = c->kv_heads;
-        aa.head_dim = c->head_dim;
-        aa.sink = c->sink;
-        aa.window = c->window;
-        for (int l = 0; l < c->layers; ++l) aa.t0[l] = c->len[l];
-        RLKV_CUDA(launch_append_all(aa, s));
-        c->launches++;
-        for (int l = 0; l < c->layers; ++l) c->len[l] += 1;
-        // Launch l and launch l-2 share a half of the scratch memory, so launch l must not start before
-        // launch l-2 has completed.  An overlapped launch starts when every CTA of launch l-1 has
-        // started; if launch l-1 puts exactly one CTA on every SM (and a CTA takes a whole SM: its
-        // registers see to that), all of them having started means that no CTA of launch l-2 is left.
-        // After a smaller launch the next one is an ordinary launch, which waits for everything.
-        bool prev_fills_gpu = true;  // the append launch is followed by an overlapped launch that waits on the device
-        for (int l = 0; l < c->layers; ++l) {
-            int grid = 0;
-            const bool overlap = prev_fills_gpu;
-            int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                               static_cast<float*>(out) + l * q_layer, s, l & 1, overlap, overlap && l == 0, &grid);
-            if (rc) return rc;
-            prev_fills_gpu = (grid == c->sm_count && c->ctas_per_sm == 1);
-        }
-        return RLKV_OK;
+        int rc = step_append(c, k, v, s);
+        if (rc) return rc;
+        return step_decode(c, 0, c->layers, q, out, s, false);
     }
     for (int l = 0; l < c->layers; ++l) {
         int rc = do_append(c, l, static_cast<const __nv_bfloat16*>(k) + l * kv_layer,
@@ -676,13 +723,58 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t kv_bytes = (size_t)c->layers * c->batch * c->kv_heads * c->head_dim * 2;
     const size_t q_bytes = (size_t)c->layers * c->batch * c->q_heads * c->head_dim * 2;
-    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_k, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
-    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_v, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
-    RLKV_CUDA(cudaMemcpyAsync(c->dev_base + c->lay.off_q, q_host, q_bytes, cudaMemcpyHostToDevice, s));
-    int rc = rlkv_step(c, c->dev_base + c->lay.off_k, c->dev_base + c->lay.off_v, c->dev_base + c->lay.off_q,
-                       c->dev_base + c->lay.off_out, stream);
+    uint8_t* dk = c->dev_base + c->lay.off_k;
+    uint8_t* dv = c->dev_base + c->lay.off_v;
+    uint8_t* dq = c->dev_base + c->lay.off_q;
+    uint8_t* dout = c->dev_base + c->lay.off_out;
+    const int chunks = c->layers >= 8 ? 4 : 1;
+    if (chunks == 1 || c->layers > kMaxStepLayers) {
+        RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
+        RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
+        RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+        int rc = rlkv_step(c, dk, dv, dq, dout, stream);
+        if (rc) return rc;
+        RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * 2, cudaMemcpyDeviceToHost, s));
+        return RLKV_OK;
+    }
+    // The layers go in four chunks.  The caller's stream carries k, v, the first chunk's q, the
+    // kernels and the last chunk's results; a second stream brings in the q of the later chunks
+    // and takes out the results of the earlier ones while the kernels run.
+    const size_t q_layer = q_bytes / c->layers;
+    // a short first chunk (little to copy before the first kernel can start) and a short last one
+    // (little to copy after the last kernel has ended)
+    const int L = c->layers, head = L / 16 > 0 ? L / 16 : 1, tail = L / 8 > 0 ? L / 8 : 1;
+    const int bounds[5] = {0, head, head + (L - head - tail) / 2, L - tail, L};
+    auto first = [&](int i) { return bounds[i]; };
+    RLKV_CUDA(cudaEventRecord(c->ev_start, s));  // the staging buffers are free once earlier work on s is done
+    RLKV_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_start, 0));
+    RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
+    RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_layer * first(1), cudaMemcpyHostToDevice, s));
+    for (int i = 1; i < chunks; ++i) {
+        const size_t o = q_layer * first(i), n = q_layer * (first(i + 1) - first(i));
+        RLKV_CUDA(cudaMemcpyAsync(dq + o, static_cast<const uint8_t*>(q_host) + o, n, cudaMemcpyHostToDevice,
+                                  c->copy_stream));
+        RLKV_CUDA(cudaEventRecord(c->ev_in[i], c->copy_stream));
+    }
+    int rc = step_append(c, dk, dv, s);
     if (rc) return rc;
-    RLKV_CUDA(cudaMemcpyAsync(out_host, c->dev_base + c->lay.off_out, q_bytes * 2, cudaMemcpyDeviceToHost, s));
+    for (int i = 0; i < chunks; ++i) {
+        if (i > 0) RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_in[i], 0));
+        rc = step_decode(c, first(i), first(i + 1), dq, dout, s, i > 0);
+        if (rc) return rc;
+        const size_t o = 2 * q_layer * first(i), n = 2 * q_layer * (first(i + 1) - first(i));
+        if (i + 1 < chunks) {
+            RLKV_CUDA(cudaEventRecord(c->ev_out[i], s));
+            RLKV_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_out[i], 0));
+            RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost,
+                                      c->copy_stream));
+        } else {
+            RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost, s));
+        }
+    }
+    RLKV_CUDA(cudaEventRecord(c->ev_done, c->copy_stream));  // whoever waits for s also waits for the side copies
+    RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_done, 0));
     return RLKV_OK;
 }
 
