@@ -130,10 +130,14 @@ size_t rlkv_static_scratch_bytes(void);
 int rlkv_step(rlkv_cache* cache, const void* k, const void* v, const void* q, void* out,
               void* stream);
 
-/* The same step with HOST buffers of the same shapes: inputs are copied host->device and the
- * result device->host on `stream` inside the call (pinned host memory makes the copies
- * asynchronous).  The call returns once the work is enqueued; synchronise `stream` before reading
- * out_host. */
+/* The same step with HOST buffers of the same shapes (pinned memory makes the copies
+ * asynchronous).  Inputs are copied host->device and results device->host inside the call, on two
+ * streams of the library's own that run beside the kernels on `stream`: this call's inputs come in
+ * while the kernels of the call before still run (the device staging area exists twice), and the
+ * results of the first layers go out while the last layers are still computed.  The call returns
+ * once the work is enqueued; work enqueued on `stream` afterwards waits for the results to have
+ * arrived, so synchronising `stream` is enough before reading out_host.  The host input buffers
+ * must stay untouched until then. */
 int rlkv_step_host(rlkv_cache* cache, const void* k_host, const void* v_host, const void* q_host,
                    void* out_host, void* stream);
 

@@ -13,7 +13,7 @@
 //   status    int32 kernel status word, then two work-claim counters (they only grow; consecutive
 //             launches of a step alternate between them)
 //   partials  float [2][max_slots][partial_floats]  (split-KV scratch; the two halves alternate too)
-//   staging   k, v, q, out of one whole step, for rlkv_step_host
+//   staging   k, v, q (twice: calls alternate) and out of one whole step, for rlkv_step_host
 //   trace     uint64 [max_grid][8]  (debug trace of the decode kernel)
 #include <stdio.h>
 #include <stdlib.h>
@@ -52,7 +52,7 @@ struct Layout {
     long long pool_rows = 0;
     size_t off_layer_desc = 0;
     size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
-    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_trace = 0, total = 0;
+    size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_in2 = 0, off_trace = 0, total = 0;
     int max_grid = 0, max_items = 0;
 };
 
@@ -142,6 +142,8 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     off = align_up(off + q_step, 1024);
     L.off_out = off;
     off = align_up(off + q_step * 2, 1024);
+    L.off_in2 = off;  // second copy of the k, v, q staging (same internal layout as the first)
+    off = align_up(off + (L.off_out - L.off_k), 1024);
     L.off_trace = off;
     off = align_up(off + (size_t)L.max_grid * kTraceWords * sizeof(unsigned long long), 1024);
     L.total = off;
@@ -189,9 +191,10 @@ struct rlkv_cache {
     int item_tiles_alone;                         // item_tiles of launches outside rlkv_step
     int trace_on;
     unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
-    cudaStream_t copy_stream;      // rlkv_step_host: copies that run beside the kernels
-    cudaEvent_t ev_start, ev_done; // order copy_stream after / before the caller's stream
-    cudaEvent_t ev_in[4], ev_out[4];  // per chunk of layers: its q has arrived / its results are ready
+    cudaStream_t in_stream, out_stream;  // rlkv_step_host: copies that run beside the kernels
+    cudaEvent_t ev_step[2], ev_done;     // kernels of a call done with staging copy p / results copied out
+    cudaEvent_t ev_in[4], ev_out[4];     // per chunk of layers: its inputs have arrived / its results are ready
+    unsigned long long host_steps;       // rlkv_step_host calls so far
     Layout lay;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -206,14 +209,16 @@ namespace {
 
 void destroy_copy_objects(rlkv_cache* c)
 {
-    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
-    if (c->ev_start) cudaEventDestroy(c->ev_start);
+    if (c->in_stream) cudaStreamDestroy(c->in_stream);
+    if (c->out_stream) cudaStreamDestroy(c->out_stream);
+    if (c->ev_step[0]) cudaEventDestroy(c->ev_step[0]);
+    if (c->ev_step[1]) cudaEventDestroy(c->ev_step[1]);
     if (c->ev_done) cudaEventDestroy(c->ev_done);
     for (int i = 0; i < 4; ++i) {
         if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
         if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
     }
-    c->copy_stream = nullptr;
+    c->in_stream = c->out_stream = nullptr;
 }
 
 template <typename T>
@@ -519,8 +524,9 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->item_tiles_alone = kDefaultItemTilesAlone;
     c->trace_on = 0;
     c->claims[0] = c->claims[1] = 0;
-    c->copy_stream = nullptr;
-    c->ev_start = c->ev_done = nullptr;
+    c->in_stream = c->out_stream = nullptr;
+    c->ev_step[0] = c->ev_step[1] = c->ev_done = nullptr;
+    c->host_steps = 0;
     for (int i = 0; i < 4; ++i) c->ev_in[i] = c->ev_out[i] = nullptr;
     c->stages = max_stages(head_dim, q_heads / kv_heads, c->groups, c->ctas_per_sm);
     rc = make_layout(c->lay, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
@@ -589,8 +595,10 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     if (rc) return fail(rc);
     e = prepare_decode_kernels(head_dim);
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaFuncSetAttribute"));
-    e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
-    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming);
+    e = cudaStreamCreateWithFlags(&c->in_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->out_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_step[0], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_step[1], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_done, cudaEventDisableTiming);
     for (int i = 0; i < 4 && e == cudaSuccess; ++i) {
         e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming);
@@ -723,12 +731,12 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t kv_bytes = (size_t)c->layers * c->batch * c->kv_heads * c->head_dim * 2;
     const size_t q_bytes = (size_t)c->layers * c->batch * c->q_heads * c->head_dim * 2;
-    uint8_t* dk = c->dev_base + c->lay.off_k;
-    uint8_t* dv = c->dev_base + c->lay.off_v;
-    uint8_t* dq = c->dev_base + c->lay.off_q;
-    uint8_t* dout = c->dev_base + c->lay.off_out;
     const int chunks = c->layers >= 8 ? 4 : 1;
     if (chunks == 1 || c->layers > kMaxStepLayers) {
+        uint8_t* dk = c->dev_base + c->lay.off_k;
+        uint8_t* dv = c->dev_base + c->lay.off_v;
+        uint8_t* dq = c->dev_base + c->lay.off_q;
+        uint8_t* dout = c->dev_base + c->lay.off_out;
         RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
         RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
         RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
@@ -737,43 +745,48 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
         RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * 2, cudaMemcpyDeviceToHost, s));
         return RLKV_OK;
     }
-    // The layers go in four chunks.  The caller's stream carries k, v, the first chunk's q, the
-    // kernels and the last chunk's results; a second stream brings in the q of the later chunks
-    // and takes out the results of the earlier ones while the kernels run.
+    // Inputs come in on one side stream, results go out on another, both beside the kernels on the
+    // caller's stream.  The input staging area exists twice and calls alternate between the copies,
+    // so this call's inputs can be copied in while the kernels of the call before still read theirs.
+    // The layers go in four chunks: a short first one (little to wait for before the first kernel),
+    // a short last one (little to copy out after the last kernel).
+    const int p = (int)(c->host_steps++ & 1);
+    const size_t in_bytes = c->lay.off_out - c->lay.off_k;          // k, v, q of one copy
+    uint8_t* dk = c->dev_base + c->lay.off_k + (p ? c->lay.off_in2 - c->lay.off_k : 0);
+    uint8_t* dv = dk + (c->lay.off_v - c->lay.off_k);
+    uint8_t* dq = dk + (c->lay.off_q - c->lay.off_k);
+    uint8_t* dout = c->dev_base + c->lay.off_out;
+    (void)in_bytes;
     const size_t q_layer = q_bytes / c->layers;
-    // a short first chunk (little to copy before the first kernel can start) and a short last one
-    // (little to copy after the last kernel has ended)
     const int L = c->layers, head = L / 16 > 0 ? L / 16 : 1, tail = L / 8 > 0 ? L / 8 : 1;
     const int bounds[5] = {0, head, head + (L - head - tail) / 2, L - tail, L};
-    auto first = [&](int i) { return bounds[i]; };
-    RLKV_CUDA(cudaEventRecord(c->ev_start, s));  // the staging buffers are free once earlier work on s is done
-    RLKV_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_start, 0));
-    RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
-    RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
-    RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_layer * first(1), cudaMemcpyHostToDevice, s));
-    for (int i = 1; i < chunks; ++i) {
-        const size_t o = q_layer * first(i), n = q_layer * (first(i + 1) - first(i));
+    // inputs: this copy of the staging area was last read by the kernels of the call before last
+    RLKV_CUDA(cudaStreamWaitEvent(c->in_stream, c->ev_step[p], 0));
+    RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, c->in_stream));
+    RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, c->in_stream));
+    for (int i = 0; i < chunks; ++i) {
+        const size_t o = q_layer * bounds[i], n = q_layer * (bounds[i + 1] - bounds[i]);
         RLKV_CUDA(cudaMemcpyAsync(dq + o, static_cast<const uint8_t*>(q_host) + o, n, cudaMemcpyHostToDevice,
-                                  c->copy_stream));
-        RLKV_CUDA(cudaEventRecord(c->ev_in[i], c->copy_stream));
+                                  c->in_stream));
+        RLKV_CUDA(cudaEventRecord(c->ev_in[i], c->in_stream));
     }
+    // kernels
+    RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_in[0], 0));
     int rc = step_append(c, dk, dv, s);
     if (rc) return rc;
     for (int i = 0; i < chunks; ++i) {
         if (i > 0) RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_in[i], 0));
-        rc = step_decode(c, first(i), first(i + 1), dq, dout, s, i > 0);
+        rc = step_decode(c, bounds[i], bounds[i + 1], dq, dout, s, i > 0);
         if (rc) return rc;
-        const size_t o = 2 * q_layer * first(i), n = 2 * q_layer * (first(i + 1) - first(i));
-        if (i + 1 < chunks) {
-            RLKV_CUDA(cudaEventRecord(c->ev_out[i], s));
-            RLKV_CUDA(cudaStreamWaitEvent(c->copy_stream, c->ev_out[i], 0));
-            RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost,
-                                      c->copy_stream));
-        } else {
-            RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost, s));
-        }
+        RLKV_CUDA(cudaEventRecord(c->ev_out[i], s));
+        // results of the chunk
+        const size_t o = 2 * q_layer * bounds[i], n = 2 * q_layer * (bounds[i + 1] - bounds[i]);
+        RLKV_CUDA(cudaStreamWaitEvent(c->out_stream, c->ev_out[i], 0));
+        RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost,
+                                  c->out_stream));
     }
-    RLKV_CUDA(cudaEventRecord(c->ev_done, c->copy_stream));  // whoever waits for s also waits for the side copies
+    RLKV_CUDA(cudaEventRecord(c->ev_step[p], s));             // this call's kernels are done with their inputs
+    RLKV_CUDA(cudaEventRecord(c->ev_done, c->out_stream));   // whoever waits for s also waits for the results
     RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_done, 0));
     return RLKV_OK;
 }
