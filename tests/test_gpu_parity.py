@@ -385,3 +385,34 @@ def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
     with pytest.raises(rl.RlkvError) as e:
         rl.rlkv_step(cache.handle, Kd[0], Vd[0], Qd[0], out)
     assert e.value.code == rl.RLKV_EFULL
+
+
+def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):
+    """Nine layers, so that rlkv_step_host brings inputs in and takes results out in chunks on its side
+    streams, and consecutive calls alternate between its two input staging areas: five steps in a row
+    without synchronising in between, every result compared with rlkv_step on a twin cache and with
+    the oracle."""
+    layers, Hkv, Hq, D, B, S, W, n0, steps = 9, 2, 4, 64, 2, 4, 28, 150, 5
+    mask = [1, 0] * layers
+    a = hz.Cache(layers, Hkv, Hq, D, B, n0 + steps, mask, S, W, device=cuda_device)
+    b, oracle = build_pair(hz, layers, Hkv, Hq, D, B, n0 + steps, mask, S, W, cuda_device)
+    for l in range(layers):
+        K, V = rand_bf16((n0, B, Hkv, D), 80 + l), rand_bf16((n0, B, Hkv, D), 90 + l)
+        a.prefill(l, K.to(cuda_device), V.to(cuda_device))
+        feed(b, oracle, l, K, V, True)
+    ins = [(rand_bf16((layers, B, Hkv, D), 100 + t).pin_memory(), rand_bf16((layers, B, Hkv, D), 110 + t).pin_memory(),
+            rand_bf16((layers, B, Hq, D), 120 + t).pin_memory()) for t in range(steps)]
+    outs = [torch.empty((layers, B, Hq, D), dtype=torch.float32).pin_memory() for _ in range(steps)]
+    for t in range(steps):                                   # back to back: copies and kernels of
+        rl.rlkv_step_host(a.handle, *ins[t], outs[t])        # neighbouring calls overlap
+    torch.cuda.synchronize()
+    for t in range(steps):
+        k, v, q = (x.to(cuda_device) for x in ins[t])
+        ref = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+        rl.rlkv_step(b.handle, k, v, q, ref)
+        assert torch.allclose(ref.cpu(), outs[t], atol=1e-4, rtol=0)
+        for l in range(layers):
+            oracle.append(l, ins[t][0][l], ins[t][1][l])
+            check_out(outs[t][l].numpy(), oracle.decode(l, ins[t][2][l]))
+    check_state(a, oracle)
+    assert a.status() == 0 and b.status() == 0
