@@ -5,21 +5,23 @@
 // full head, the sink + ring rows for a compressed head.  One launch serves both head classes
 // (the fused heterogeneous-head kernel Section 4.3 asks for).
 //
-// How: the K/V rows to read are cut into 64-token tiles and laid out as one flat tile space (full
-// units first, compressed units after).  The space is cut into contiguous work items whose size
-// shrinks geometrically; a persistent grid takes item c for CTA c and claims further items from an
-// atomic counter, so long full-head scans and short compressed-head scans balance even though some
-// SMs sit on a slower path to memory than others.  Inside a CTA one producer warp streams tiles HBM -> shared memory
-// with TMA (cp.async.bulk.tensor, 128-byte swizzle, mbarrier pipeline); NG groups of four consumer
-// warps take the tiles in turn, each warp 16 tokens of its group's tile: S = Q.K^T and
-// O^T += V^T.P^T run on mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G query heads of the
-// group as the M (resp. N) dimension, online softmax in fp32 with warp shuffles.  The path is
-// HBM-bound (the tensor-core work is ~G flop per byte); several groups are there only to hide the
-// dependent-issue latency of one tile's softmax chain behind another tile's.
+// How: the K/V rows to read are cut into 64-token tiles and laid out as one flat tile space, which
+// is cut into contiguous work items whose size shrinks geometrically (rlkv_internal.cuh); a
+// persistent grid takes item c for CTA c and claims further items from an atomic counter, so long
+// full-head scans and short compressed-head scans balance even though some SMs sit on a slower path
+// to memory than others.  Inside a CTA one producer warp streams tiles HBM -> shared memory with TMA
+// (cp.async.bulk.tensor, 128-byte swizzle, mbarrier pipeline); NG groups of four consumer warps take
+// the tiles in turn, each warp 16 tokens of its group's tile: S = Q.K^T and O^T += V^T.P^T run on
+// mma.sync m16n8k16 (bf16 in, fp32 accumulate) with the G query heads of the group as the M (resp. N)
+// dimension, online softmax in fp32 with warp shuffles.  The path is HBM-bound (the tensor-core work
+// is ~G flop per byte).
 // When an item begins or ends inside a unit the CTA writes an (m, l, O) partial; the last CTA to
 // deliver a partial of a unit (atomic ticket, no spinning) merges them with the log-sum-exp rule.
-// Those merges, and the merge of the consumer warps' own states at the end of every segment, run
-// on separate epilogue warps, so the tile stream never waits for a round trip to global memory.
+// The merge of the consumer warps' own states at the end of every segment and the tickets run on
+// separate epilogue warps, so the tile stream never waits for a round trip to global memory; the
+// merges of split units run on all warps once the CTA's stream has ended.
+// The decode launches of one step overlap on the device (programmatic dependent launch): see the
+// kernel's first lines and launch_decode.
 #include "rlkv_internal.cuh"
 
 namespace rlkv {
@@ -362,7 +364,6 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     // run-time indices, which is slow on kernel parameters and cheap here.
     DecodeArgs* s_args = reinterpret_cast<DecodeArgs*>(lists + kMaxTodo * (kMaxRounds + 1));
     const DecodeArgs& a = *s_args;
-    Schedule* s_sched = &s_args->sched;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
