@@ -29,7 +29,8 @@
  * Parity pins (tests/test_oracle_pins.py): all-full == library causal attention's
  * last row; sink+window >= n == full; brute-force masked softmax; ring invariants;
  * closed forms; planted needle; Table 3's "theoretical" column for the retained-token
- * count.  The paper prints no numeric attention values, so beyond those pins the
+ * count; the mixed form of Eq. 1 has its own pins, listed at rlkv_oracle_decode_mixed.
+ * The paper prints no numeric attention values, so beyond those pins the
  * numeric output is "parity unpinned" by any printed example.
  */
 #include <math.h>
@@ -256,6 +257,89 @@ int rlkv_oracle_decode(const oracle_t *o, int layer, const uint16_t *q, float *o
                 if (s && rows) attend_one(o, layer, b, j, q, out, s, rows);
         free(s);
         free(rows);
+    }
+    return fail ? -4 : 0;
+}
+
+/* ---- mixed attention with gating adapters (Section 3.1, Eq. 1) ----------------------------
+ * The form attention takes while the gates are trained and while samples are generated for that
+ * training: every head keeps its full cache, and head h of layer l carries a gate alpha in [0, 1].
+ *   out_full_attn  = softmax over all n tokens                     (mask M_causal, last row)
+ *   out_local_attn = softmax over {t < sink} U {t >= n - window}   (mask M_local, last row)
+ *   out_mix_attn   = alpha * out_full_attn + (1 - alpha) * out_local_attn
+ * The gate belongs to the KV head; its G query heads share it.  Scores, both softmaxes and the
+ * mix run in acc_t; the query's own token (the last one appended) is inside the window.
+ * Pins (tests/test_oracle_pins.py): alpha = 1 against rlkv_oracle_decode on the same cache;
+ * alpha = 0 against rlkv_oracle_decode on a cache that holds the same history in compressed
+ * heads; a masked softmax written out with boolean mask matrices in numpy; n <= sink + window
+ * (both branches equal, so alpha drops out). */
+static void attend_masked(const oracle_t *o, int layer, int b, int j, const uint16_t *q, int local,
+                          acc_t *res, acc_t *p)
+{
+    int D = o->head_dim, G = o->q_heads / o->kv_heads, h = j / G, n = o->len[layer];
+    size_t u = unit_index(o, layer, b, h);
+    const uint16_t *qj = q + ((size_t)b * o->q_heads + j) * D;
+    acc_t scale = (acc_t)1 / (acc_t)sqrt((double)D);
+    acc_t m = -INFINITY;
+    for (int t = 0; t < n; ++t) {
+        int keep = !local || t < o->sink || t >= n - o->window;
+        p[t] = -INFINITY;
+        if (!keep) continue;
+        const uint16_t *kr = o->k[u] + (size_t)t * D;
+        acc_t dot = 0;
+        for (int d = 0; d < D; ++d) dot += (acc_t)bf16_to_float(qj[d]) * (acc_t)bf16_to_float(kr[d]);
+        p[t] = dot * scale;
+        if (p[t] > m) m = p[t];
+    }
+    acc_t l = 0;
+    for (int t = 0; t < n; ++t) {
+        if (p[t] == -INFINITY) { p[t] = 0; continue; }
+        p[t] = sizeof(acc_t) == sizeof(float) ? (acc_t)expf((float)(p[t] - m)) : (acc_t)exp((double)(p[t] - m));
+        l += p[t];
+    }
+    for (int d = 0; d < D; ++d) {
+        acc_t a = 0;
+        for (int t = 0; t < n; ++t)
+            if (p[t] != 0) a += p[t] * (acc_t)bf16_to_float(o->v[u][(size_t)t * D + d]);
+        res[d] = a / l;
+    }
+}
+
+/* q: bf16 bits [batch][q_heads][head_dim]; alpha: float [kv_heads], the gates of this layer;
+ * out: float [batch][q_heads][head_dim].
+ * Returns 0, -3 if the layer is empty, -5 if a head of the layer is compressed (its cache no
+ * longer holds what out_full_attn needs), -6 if a gate lies outside [0, 1]. */
+int rlkv_oracle_decode_mixed(const oracle_t *o, int layer, const uint16_t *q, const float *alpha, float *out)
+{
+    if (layer < 0 || layer >= o->layers) return -2;
+    int n = o->len[layer], D = o->head_dim, G = o->q_heads / o->kv_heads;
+    if (n < 1) return -3;
+    for (int h = 0; h < o->kv_heads; ++h) {
+        if (!o->is_full[layer * o->kv_heads + h]) return -5;
+        if (!(alpha[h] >= 0.0f && alpha[h] <= 1.0f)) return -6;
+    }
+    int fail = 0;
+#pragma omp parallel num_threads(o->threads)
+    {
+        acc_t *p = malloc((size_t)n * sizeof(acc_t));
+        acc_t *full = malloc((size_t)D * sizeof(acc_t)), *loc = malloc((size_t)D * sizeof(acc_t));
+        if (!p || !full || !loc) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp for collapse(2) schedule(dynamic, 1)
+        for (int b = 0; b < o->batch; ++b)
+            for (int j = 0; j < o->q_heads; ++j) {
+                if (!p || !full || !loc) continue;
+                acc_t a = (acc_t)alpha[j / G];
+                attend_masked(o, layer, b, j, q, 0, full, p);
+                attend_masked(o, layer, b, j, q, 1, loc, p);
+                float *oj = out + ((size_t)b * o->q_heads + j) * D;
+                for (int d = 0; d < D; ++d) oj[d] = (float)(a * full[d] + ((acc_t)1 - a) * loc[d]);
+            }
+        free(p);
+        free(full);
+        free(loc);
     }
     return fail ? -4 : 0;
 }

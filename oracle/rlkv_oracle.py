@@ -52,6 +52,8 @@ def _lib(acc: str) -> ctypes.CDLL:
         lib.rlkv_oracle_append.argtypes = [vp, ci, vp, vp]
         lib.rlkv_oracle_decode.restype = ci
         lib.rlkv_oracle_decode.argtypes = [vp, ci, vp, vp]
+        lib.rlkv_oracle_decode_mixed.restype = ci
+        lib.rlkv_oracle_decode_mixed.argtypes = [vp, ci, vp, vp, vp]
         lib.rlkv_oracle_retained.restype = ci
         lib.rlkv_oracle_retained.argtypes = [vp, ci, ci]
         lib.rlkv_oracle_export_head.restype = ci
@@ -129,6 +131,21 @@ class Oracle:
         rc = self._lib.rlkv_oracle_decode(self._h, layer, q.ctypes.data, out.ctypes.data)
         if rc != 0:
             raise RuntimeError(f"rlkv_oracle_decode failed: {rc}")
+        return out
+
+    def decode_mixed(self, layer: int, q, alpha) -> np.ndarray:
+        """Eq. 1: alpha[h] * full attention + (1 - alpha[h]) * sink+window attention; every head of
+        the layer must be full.  alpha: [kv_heads] floats in [0, 1]."""
+        q = _bits(q)
+        if q.size != self.batch * self.q_heads * self.head_dim:
+            raise ValueError("q must be [batch][q_heads][head_dim]")
+        alpha = np.ascontiguousarray(np.asarray(alpha, dtype=np.float32).reshape(-1))
+        if alpha.size != self.kv_heads:
+            raise ValueError("alpha must have kv_heads entries")
+        out = np.empty((self.batch, self.q_heads, self.head_dim), dtype=np.float32)
+        rc = self._lib.rlkv_oracle_decode_mixed(self._h, layer, q.ctypes.data, alpha.ctypes.data, out.ctypes.data)
+        if rc != 0:
+            raise RuntimeError(f"rlkv_oracle_decode_mixed failed: {rc}")
         return out
 
     def retained(self, layer: int, head: int) -> int:

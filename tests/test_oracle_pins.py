@@ -286,3 +286,116 @@ def test_layers_keep_separate_lengths_and_masks():
     assert [o.retained(0, 0), o.retained(0, 1), o.retained(1, 0), o.retained(1, 1)] == [6, 3, 3, 3]
     with pytest.raises(RuntimeError):
         Oracle(1, 1, 1, D, 1, 4, [1], 0, 1).decode(0, rand_bf16((1, 1, D), 1))   # empty layer
+
+
+# ---------------------------------------------------------------------------- mixed attention, Eq. 1
+def mask_matrices(n, S, W):
+    """M_causal and M_local of Section 3.1 as boolean [n][n] matrices (row = query position):
+    causal = every earlier token and the query's own; local = causal AND (one of the first S tokens
+    OR one of the W most recent, the query's own included)."""
+    i, j = np.arange(n)[:, None], np.arange(n)[None, :]
+    causal = j <= i
+    local = causal & ((j < S) | (j > i - W))
+    return causal, local
+
+
+@pytest.mark.parametrize("acc", ["f32", "f64"])
+@pytest.mark.parametrize("S,W,n", [(4, 8, 40), (0, 5, 23), (3, 1, 17), (16, 64, 200)])
+def test_mixed_equals_masked_softmax_with_mask_matrices(acc, S, W, n):
+    """Eq. 1 computed for EVERY position with explicit mask matrices in float64 numpy; the decode
+    step is the last row."""
+    Hq, Hkv, D, B = 6, 2, 16, 2
+    G = Hq // Hkv
+    K, V, Q = rand_bf16((n, B, Hkv, D), 71), rand_bf16((n, B, Hkv, D), 72), rand_bf16((n, B, Hq, D), 73)
+    alpha = np.array([0.3, 0.85], np.float32)
+    o = Oracle(1, Hkv, Hq, D, B, n, [1, 1], S, W, acc=acc)
+    fill(o, 0, K, V)
+    out = o.decode_mixed(0, Q[-1], alpha)
+    causal, local = mask_matrices(n, S, W)
+    for b in range(B):
+        for j in range(Hq):
+            h = j // G
+            q2, k2, v2 = (f32(Q[:, b, j]).astype(np.float64), f32(K[:, b, h]).astype(np.float64),
+                          f32(V[:, b, h]).astype(np.float64))
+            s = q2 @ k2.T / np.sqrt(D)                               # [n][n]
+            rows = []
+            for m in (causal, local):
+                sm = np.where(m, s, -np.inf)
+                p = np.exp(sm - sm.max(axis=1, keepdims=True))
+                rows.append(((p / p.sum(axis=1, keepdims=True)) @ v2)[-1])
+            want = float(alpha[h]) * rows[0] + (1.0 - float(alpha[h])) * rows[1]
+            np.testing.assert_allclose(out[b, j], want, atol=2e-5 if acc == "f32" else 3e-7, rtol=0)
+
+
+def test_mixed_gate_one_is_full_attention_and_gate_zero_is_the_compressed_head():
+    """alpha = 1 must give what a full head gives and alpha = 0 what a compressed head gives
+    (Section 3.3: at inference the gate picks one branch) -- through rlkv_oracle_decode, whose own
+    pins are above.  A swapped gate or a window off by one fails here."""
+    Hq, Hkv, D, B, S, W, n = 8, 2, 32, 2, 4, 12, 61
+    K, V, q = rand_bf16((n, B, Hkv, D), 74), rand_bf16((n, B, Hkv, D), 75), rand_bf16((B, Hq, D), 76)
+    full = Oracle(1, Hkv, Hq, D, B, n, [1, 1], S, W)
+    comp = Oracle(1, Hkv, Hq, D, B, n, [0, 0], S, W)
+    fill(full, 0, K, V)
+    fill(comp, 0, K, V)
+    np.testing.assert_allclose(full.decode_mixed(0, q, [1.0, 1.0]), full.decode(0, q), atol=1e-6, rtol=0)
+    np.testing.assert_allclose(full.decode_mixed(0, q, [0.0, 0.0]), comp.decode(0, q), atol=1e-6, rtol=0)
+    mixed = full.decode_mixed(0, q, [1.0, 0.0])                     # head 0 full, head 1 local
+    G = Hq // Hkv
+    np.testing.assert_allclose(mixed[:, :G], full.decode(0, q)[:, :G], atol=1e-6, rtol=0)
+    np.testing.assert_allclose(mixed[:, G:], comp.decode(0, q)[:, G:], atol=1e-6, rtol=0)
+    # the two branches differ here, so the checks above can tell them apart
+    assert np.abs(full.decode(0, q) - comp.decode(0, q)).max() > 1e-2
+    # in between: the straight line between the two branches, gate by gate
+    a = np.array([0.25, 0.6], np.float32)
+    want = np.repeat(a, G)[None, :, None] * full.decode(0, q) + np.repeat(1 - a, G)[None, :, None] * comp.decode(0, q)
+    np.testing.assert_allclose(full.decode_mixed(0, q, a), want, atol=2e-6, rtol=0)
+
+
+def test_mixed_short_sequence_does_not_depend_on_the_gate():
+    """While n <= sink + window the local mask hides nothing, both branches agree and the gate
+    drops out of Eq. 1."""
+    Hq, Hkv, D, B, S, W = 4, 2, 32, 1, 4, 28
+    for n in (1, 3, 4, 5, 32):
+        K, V, q = rand_bf16((n, B, Hkv, D), 77), rand_bf16((n, B, Hkv, D), 78), rand_bf16((B, Hq, D), 79)
+        o = Oracle(1, Hkv, Hq, D, B, 64, [1, 1], S, W)
+        fill(o, 0, K, V)
+        ref = o.decode(0, q)
+        for a in ([0.0, 1.0], [0.5, 0.123]):
+            np.testing.assert_allclose(o.decode_mixed(0, q, a), ref, atol=1e-6, rtol=0)
+
+
+def test_mixed_planted_needle_is_seen_only_through_the_full_branch():
+    """One token in the evicted middle carries a key aligned with the query and a marker value: the
+    full branch returns (almost exactly) the marker, the local branch cannot see it, so the output
+    is alpha * marker + (1 - alpha) * local."""
+    Hq, Hkv, D, B, S, W, n = 2, 1, 32, 1, 2, 6, 50
+    K, V = rand_bf16((n, B, Hkv, D), 80) * 0.1, rand_bf16((n, B, Hkv, D), 81)
+    q = torch.zeros((B, Hq, D), dtype=torch.bfloat16)
+    q[..., 0] = 16.0
+    K[20, 0, 0, :] = 0
+    K[20, 0, 0, 0] = 64.0                                     # score 16*64/sqrt(32) = 181 above the rest
+    V[20, 0, 0, :] = 7.0
+    o = Oracle(1, Hkv, Hq, D, B, n, [1], S, W)
+    c = Oracle(1, Hkv, Hq, D, B, n, [0], S, W)
+    fill(o, 0, K, V)
+    fill(c, 0, K, V)
+    local = c.decode(0, q)
+    assert np.abs(local - 7.0).min() > 1.0
+    out = o.decode_mixed(0, q, [0.75])
+    np.testing.assert_allclose(out, 0.75 * 7.0 + 0.25 * local, atol=1e-5, rtol=0)
+
+
+def test_mixed_refuses_compressed_heads_and_gates_outside_the_unit_interval():
+    Hq, Hkv, D, B = 4, 2, 16, 1
+    K, V, q = rand_bf16((9, B, Hkv, D), 82), rand_bf16((9, B, Hkv, D), 83), rand_bf16((B, Hq, D), 84)
+    o = Oracle(1, Hkv, Hq, D, B, 16, [1, 0], 2, 3)
+    fill(o, 0, K, V)
+    with pytest.raises(RuntimeError, match="-5"):
+        o.decode_mixed(0, q, [0.5, 0.5])
+    o = Oracle(1, Hkv, Hq, D, B, 16, [1, 1], 2, 3)
+    with pytest.raises(RuntimeError, match="-3"):
+        o.decode_mixed(0, q, [0.5, 0.5])
+    fill(o, 0, K, V)
+    for bad in ([1.5, 0.5], [0.5, -0.1], [float("nan"), 0.5]):
+        with pytest.raises(RuntimeError, match="-6"):
+            o.decode_mixed(0, q, bad)
