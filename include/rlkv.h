@@ -119,6 +119,25 @@ int rlkv_decode_attention_static_scratch(rlkv_cache* cache, int layer, const voi
                                          void* stream);
 size_t rlkv_static_scratch_bytes(void);
 
+/* Mixed attention with gating adapters, the decode step of sample generation while the gates are
+ * trained (Section 3.1, Eq. 1; Appendix B names custom decode kernels for it):
+ *   out = alpha[h] * out_full_attn + (1 - alpha[h]) * out_local_attn        for q head j, h = j / G
+ * where out_full_attn is attention over all length(layer) tokens of KV head h and out_local_attn
+ * attention over its first `sink` tokens and its `window` most recent ones (the token appended last
+ * included) -- what the head would see if it were compressed.  While length <= sink + window the two
+ * branches are equal.  alpha = 1 gives rlkv_decode_attention's result for a full head, alpha = 0 the
+ * result of a compressed head with the same history.
+ * Every head of the layer must be a full head (the full branch needs every token): RLKV_EINVAL
+ * otherwise.  q: device bf16 [batch][q_heads][head_dim]; alpha: DEVICE fp32 [kv_heads], the gates of
+ * this layer, read when the kernel runs and used as they are (the paper keeps them in [0, 1]; the
+ * library does not check); out: device fp32 [batch][q_heads][head_dim].  One launch: the K/V rows are
+ * streamed once for the full branch, the sink and window rows a second time for the local branch
+ * (sink + window rows per head, normally out of the L2), and each branch adds its weighted result
+ * into `out`, which the call clears on `stream` first.  K and V rows are assumed finite.
+ * RLKV_EEMPTY if length(layer) == 0. */
+int rlkv_decode_mixed_attention(rlkv_cache* cache, int layer, const void* q, const float* alpha,
+                                void* out, void* stream);
+
 /* One whole decode step: for every layer, append then attend.  Device buffers:
  * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];
  * out fp32 [layers][batch][q_heads][head_dim].  The results are those of the per-layer calls in
@@ -166,16 +185,19 @@ int rlkv_launch_count(const rlkv_cache* cache, uint64_t* launches_out);
  * 32 tiles inside rlkv_step (whose launches overlap) and 8 tiles for a launch on its own.  Results do not depend on these knobs beyond floating-point summation order. */
 int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int consumer_groups,
                            int item_tiles);
-/* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, 32
+/* Debug trace of the decode kernel.  enable != 0: later decode launches record, per CTA, 40
  * 64-bit words: [0..3] %globaltimer (ns) at CTA start, when its first tile landed, when its last
  * segment was handed off and at CTA end; [4..6] work items, tiles and partial segments it
- * processed; [7] %globaltimer when its epilogue warps finished; [8..10] ns its first consumer warp
- * waited for work items, for tiles and for a free hand-off buffer; [11] ns its epilogue warps were
- * idle; [12..13] split merges its epilogue warps ran at once and the ns they took; [14..15] ns its
- * producer waited for the next work item's number and for a free descriptor; [16..31] for its
- * first 16 work items, (%globaltimer << 16) | (item & 0xffff) when the consumers started it.
+ * processed; [7] %globaltimer when its epilogue warps finished; [8..10] SM cycles its first consumer
+ * warp waited for work items, for tiles and for a free hand-off buffer; [11] cycles its epilogue
+ * warps were idle; [12..13] %globaltimer when the CTA's stream had ended and how many split units
+ * it then merged; [14..15] cycles its producer waited for the next work item's number, and for a
+ * free descriptor (low half) and a free stage (high half); [16..26] for its first 11 work items,
+ * (%globaltimer << 16) | (item & 0xffff) when the consumers started it; [27] cycles the producer
+ * ran; [28..31] %globaltimer stamps inside the final merge; [32..36] producer cycles spent arming
+ * barriers, issuing tile copies, issuing query copies, publishing items and locating segments.
  * words_host != NULL: first synchronises the device and copies the words of the most recent launch
- * to words_host (host, 32 * 320 words) and the CTA capacity (320) to *ctas_out; then the switch is
+ * to words_host (host, 40 * 320 words) and the CTA capacity (320) to *ctas_out; then the switch is
  * applied. */
 int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_host, int* ctas_out);
 /* The work schedule of the decode kernel, host arithmetic only (no GPU).  full_units units of

@@ -31,6 +31,7 @@ SIGNATURES = {
     "rlkv_decode_attention": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_decode_attention_static_scratch": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_static_scratch_bytes": (_sz, []),
+    "rlkv_decode_mixed_attention": (_ci, [_vp, _ci, _vp, _vp, _vp, _vp]),
     "rlkv_step": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_step_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_length": (_ci, [_vp, _ci, ctypes.POINTER(_ci)]),
@@ -149,6 +150,12 @@ def rlkv_decode_attention_static_scratch(cache, layer, q, out, stream=None) -> N
 
 def rlkv_static_scratch_bytes() -> int:
     return int(lib.rlkv_static_scratch_bytes())
+
+
+def rlkv_decode_mixed_attention(cache, layer, q, alpha, out, stream=None) -> None:
+    """Eq. 1: alpha[h] * full attention + (1 - alpha[h]) * sink+window attention over a layer whose
+    heads are all full.  alpha: device fp32 [kv_heads]."""
+    _check(lib.rlkv_decode_mixed_attention(cache, layer, _ptr(q), _ptr(alpha), _ptr(out), _stream(stream)))
 
 
 def rlkv_step(cache, k, v, q, out, stream=None) -> None:

@@ -247,10 +247,14 @@ struct Smem {
 // writes to `units` and `lists`.
 // (Everything comes by value or from shared memory: a reference to kernel parameters would turn
 // every use into a slow generic load inside this non-inlined function.)
-template <int D>
+// MIXED (Eq. 1 of the paper): a unit's rows are shared by its full and its local unit; each adds
+// its result times its weight (the head's gate alpha for the full unit u < U, 1 - alpha for the
+// local one) to rows the host cleared.  Two addends on zero commute, so the sum does not depend
+// on their order.
+template <int D, bool MIXED>
 __device__ __noinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
                                          const int2* lists, int n, int t, int nt, bool dry,
-                                         unsigned long long* stamp)
+                                         unsigned long long* stamp, const float* alpha, int U, int q_heads)
 {
     constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
     const int E = G * D4;
@@ -309,8 +313,18 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
                     M = Mc;
                 }
                 if (stamp && t == 0 && j == ul) stamp[3] = global_timer_ns();
-                const float inv = 1.f / L;
-                if (!dry)
+                float inv = 1.f / L;
+                if (MIXED) {
+                    const float gate = __ldg(alpha + (units[j].y % q_heads) / G);
+                    inv *= units[j].x < U ? gate : 1.f - gate;
+                    if (!dry) {
+                        float* o = out + (size_t)units[j].y * D + e * 4;
+                        atomicAdd(o, O.x * inv);
+                        atomicAdd(o + 1, O.y * inv);
+                        atomicAdd(o + 2, O.z * inv);
+                        atomicAdd(o + 3, O.w * inv);
+                    }
+                } else if (!dry)
                     *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
                         make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
             }
@@ -331,7 +345,11 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
 // (results do not depend on which CTA claimed which item) and a stage is always consumed by the
 // same group (stages is a multiple of NG).  Where an item starts on the wrong residue the producer
 // issues an empty slot first.
-template <int D, int NG>
+//
+// MIXED: the mixed attention of Eq. 1.  The schedule's second class holds, for every full unit, a
+// LOCAL unit over the same head's sink and window rows; its tiles start at whatever row the window
+// starts (a TMA box may start at any row) and are masked past their valid rows.
+template <int D, int NG, bool MIXED>
 __global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
 decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ CUtensorMap tmap, const int stages)
 {
@@ -454,8 +472,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
                 if (item >= 0) {
-                    u = locate(a, x);
+                    u = locate<MIXED>(a, x);
                     seg_tiles = min(x1 - x, u.pos.run);
+                    const bool local_unit = MIXED && u.pos.uid >= sc.U;
                     // Q as the A operand (rows = query heads of the group, rows >= G are zero): read from
                     // the stage of this warp's first tile of the segment, where the producer put the
                     // unit's query rows
@@ -471,7 +490,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             my_trace[1] = global_timer_ns();
                             landed = true;
                         }
-                        const int valid = min(kTile, valid_left);
+                        int valid = min(kTile, valid_left);
+                        if (local_unit) {
+                            int row;
+                            local_tile(a, u.pos.tile + i, row, valid);
+                        }
                         if (!have_q) {
                             const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
                                                             stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
@@ -658,14 +681,16 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     }
                 }
                 int seg_left = 0, seg_idx = 0, krow = 0, vrow = 0;
+                int local_row0 = -1, local_next = 0;  // MIXED, inside a local unit: first row of its head, next tile
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
                     if (x == x_ask) mbar_arrive(smem_u32(claim_empty));
                     const long long ts0 = trace ? clock64() : 0;
                     if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
-                        const UnitInfo u = locate(a, x);
+                        const UnitInfo u = locate<MIXED>(a, x);
                         seg_left = min(x1 - x, u.pos.run);
                         seg_idx = 0;
+                        local_row0 = -1;
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit.  Everything else is older and may be fetched early.
                         if (a.dep_wait && !synced &&
@@ -676,11 +701,20 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         if (u.pos.uid < sc.U) {
                             krow = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full) + u.pos.tile * kTile;
                             vrow = krow + a.rows_full;
+                        } else if (MIXED) {
+                            local_row0 = (int)(a.full_row0 + (long long)(u.pos.uid - sc.U) * 2 * a.rows_full);
+                            local_next = u.pos.tile;
                         } else {
                             krow = (int)(a.comp_row0 + (long long)(u.pos.uid - sc.U) * 2 * a.rows_comp) + u.pos.tile * kTile;
                             vrow = krow + a.rows_comp;
                         }
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
+                    }
+                    if (MIXED && local_row0 >= 0) {
+                        int row, valid;
+                        local_tile(a, local_next++, row, valid);
+                        krow = local_row0 + row;
+                        vrow = krow + a.rows_full;
                     }
                     if (trace) cy_seg += clock64() - ts0;
                     ok = wait_traced(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout, trace,
@@ -767,8 +801,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count);
         }
         epilogue_sync();
-        merge_units<D>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1, et, NE,
-                       true, nullptr);
+        merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1,
+                              et, NE, true, nullptr, a.alpha, sc.U, a.q_heads);
         epilogue_sync();
         if (a.dep_wait) {  // from here on these warps write results, partials and tickets
             grid_dep_wait();
@@ -784,7 +818,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             __threadfence();  // this thread's partial stores are visible before any ticket is drawn for them
             epilogue_sync();
             if (*todo_count + pend_n > kMaxTodo) {
-                merge_units<D>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, et, NE, false, nullptr);
+                merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, et, NE, false, nullptr, a.alpha,
+                                      sc.U, a.q_heads);
                 epilogue_sync();
                 if (et == 0) *todo_count = 0;
                 epilogue_sync();
@@ -836,6 +871,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             }
             float* out_rows = a.out + (size_t)sd.out_row * D;
             float* my_part = a.partials + (size_t)sd.pslot * PF;
+            float weight = 1.f;  // MIXED: the gate's share of this unit in its output rows
+            if (MIXED) {
+                const float gate = __ldg(a.alpha + (sd.out_row % a.q_heads) / G);
+                weight = sd.uid < sc.U ? gate : 1.f - gate;
+            }
             // merge the consumer warps' states; this thread owns a few 4-float pieces of the G x D rows
             for (int e = et; e < G * D4; e += NE) {
                 const int g = e / D4, d4 = e - g * D4;
@@ -854,7 +894,13 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     O.z += o.z * wt;
                     O.w += o.w * wt;
                 }
-                if (sd.complete) {
+                if (sd.complete && MIXED) {
+                    const float inv = weight / L;
+                    atomicAdd(out_rows + e * 4, O.x * inv);
+                    atomicAdd(out_rows + e * 4 + 1, O.y * inv);
+                    atomicAdd(out_rows + e * 4 + 2, O.z * inv);
+                    atomicAdd(out_rows + e * 4 + 3, O.w * inv);
+                } else if (sd.complete) {
                     const float inv = 1.f / L;
                     *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
                 } else {
@@ -882,8 +928,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (trace && tid == 0) my_trace[12] = global_timer_ns();
     if (trace && tid == 0) my_trace[13] = (unsigned long long)*todo_count;
     if (!*s_abort && *todo_count > 0)
-        merge_units<D>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, tid, S::kThreads, false,
-                       trace ? my_trace + 28 : nullptr);
+        merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, tid, S::kThreads, false,
+                              trace ? my_trace + 28 : nullptr, a.alpha, sc.U, a.q_heads);
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
             // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight
@@ -896,7 +942,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (trace && tid == 0) my_trace[3] = global_timer_ns();
 }
 
-template <int D, int NG>
+template <int D, int NG, bool MIXED>
 cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
                        bool overlap)
 {
@@ -911,13 +957,16 @@ cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, i
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<D, NG>, a, tmap, stages);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<D, NG, MIXED>, a, tmap, stages);
 }
 
 template <int D, int NG>
 cudaError_t prepare_one()
 {
-    return cudaFuncSetAttribute(decode_kernel<D, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    const cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, NG, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                               kMaxDynamicSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_kernel<D, NG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kMaxDynamicSmem);
 }
 
@@ -945,17 +994,25 @@ cudaError_t prepare_decode_kernels(int head_dim)
     return prepare_one<64, 3>();
 }
 
+template <int D, int NG>
+static cudaError_t launch_either(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
+                          bool overlap, bool mixed)
+{
+    return mixed ? launch_one<D, NG, true>(a, tmap, grid, stages, stream, overlap)
+                 : launch_one<D, NG, false>(a, tmap, grid, stages, stream, overlap);
+}
+
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream, bool overlap)
+                          int stages, int groups, cudaStream_t stream, bool overlap, bool mixed)
 {
     if (head_dim == 128) {
-        if (groups == 1) return launch_one<128, 1>(a, *tmap, grid, stages, stream, overlap);
-        if (groups == 2) return launch_one<128, 2>(a, *tmap, grid, stages, stream, overlap);
-        return launch_one<128, 3>(a, *tmap, grid, stages, stream, overlap);
+        if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mixed);
+        if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mixed);
+        return launch_either<128, 3>(a, *tmap, grid, stages, stream, overlap, mixed);
     }
-    if (groups == 1) return launch_one<64, 1>(a, *tmap, grid, stages, stream, overlap);
-    if (groups == 2) return launch_one<64, 2>(a, *tmap, grid, stages, stream, overlap);
-    return launch_one<64, 3>(a, *tmap, grid, stages, stream, overlap);
+    if (groups == 1) return launch_either<64, 1>(a, *tmap, grid, stages, stream, overlap, mixed);
+    if (groups == 2) return launch_either<64, 2>(a, *tmap, grid, stages, stream, overlap, mixed);
+    return launch_either<64, 3>(a, *tmap, grid, stages, stream, overlap, mixed);
 }
 
 }  // namespace rlkv

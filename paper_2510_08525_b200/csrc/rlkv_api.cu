@@ -8,7 +8,8 @@
 //             into a neighbouring head and a compressed head owns a constant number of rows
 //             (the constant-size pool of Section 4.3 of the paper).
 //   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
-//   tickets   int32 [layers][batch*kv_heads]   (split bookkeeping, zero between launches)
+//   tickets   int32 [layers][2*batch*kv_heads] (split bookkeeping, zero between launches; the second
+//             half of a layer's tickets serves the local units of a mixed-attention launch)
 //   tables    then LayerDesc[layers] (where each layer's regions start; for the step's append launch)
 //   status    int32 kernel status word, then two work-claim counters (they only grow; consecutive
 //             launches of a step alternate between them)
@@ -115,6 +116,12 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
             const long long m = most_slots(batch * L.n_full[l], L.rows_full / kTile, batch * L.n_comp[l],
                                            L.rows_comp / kTile, L.max_grid);
             if (m > most) most = m;
+            if (L.n_comp[l] == 0) {  // a layer rlkv_decode_mixed_attention accepts: a local unit beside every full unit
+                const int local_tiles = (sink + kTile - 1) / kTile + (window + kTile - 1) / kTile;
+                const long long mm = most_slots(batch * L.n_full[l], L.rows_full / kTile, batch * L.n_full[l], local_tiles,
+                                                L.max_grid);
+                if (mm > most) most = mm;
+            }
         }
         if (most >= (1ll << 31)) return RLKV_EINVAL;
         L.max_items = (int)most;
@@ -127,7 +134,7 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     L.off_layer_desc = off;
     off = align_up(off + (size_t)layers * sizeof(LayerDesc), 1024);
     L.off_tickets = off;
-    off = align_up(off + (size_t)layers * batch * kv_heads * sizeof(int), 1024);
+    off = align_up(off + (size_t)layers * 2 * batch * kv_heads * sizeof(int), 1024);
     L.off_status = off;
     off = align_up(off + 64, 1024);
     L.off_partials = off;
@@ -303,8 +310,10 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
 
 // Everything of a decode launch except where its split-KV work area lives.  Returns the grid size
 // in *grid_out.
+// `alpha` != null: a mixed-attention launch (every head of the layer is full): the second class of
+// units are the local units, one per (batch row, head), over the head's sink and window rows.
 int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, DecodeArgs& a, int* grid_out,
-                      bool in_step = false)
+                      bool in_step = false, const float* alpha = nullptr)
 {
     const int n = c->len[layer];
     const int cap = c->sink + c->window;
@@ -325,8 +334,15 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     a.batch = c->batch;
     a.group = c->q_heads / c->kv_heads;
     a.q_heads = c->q_heads;
-    const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
-    const long long all_tiles = (long long)c->batch * ((long long)a.n_full * tiles_full + (long long)a.n_comp * tiles_comp);
+    a.alpha = alpha;
+    a.local_sink = n < c->sink ? n : c->sink;
+    a.local_sink_tiles = (a.local_sink + kTile - 1) / kTile;
+    a.local_win0 = n - c->window > c->sink ? n - c->window : c->sink;  // first token of the window
+    a.local_win_len = n > a.local_win0 ? n - a.local_win0 : 0;
+    const int tiles_full = (a.len_full + kTile - 1) / kTile;
+    const int tiles_comp = alpha ? a.local_sink_tiles + (a.local_win_len + kTile - 1) / kTile : (a.len_comp + kTile - 1) / kTile;
+    const int second_class = alpha ? a.n_full : a.n_comp;  // units per batch row beside the full ones
+    const long long all_tiles = (long long)c->batch * ((long long)a.n_full * tiles_full + (long long)second_class * tiles_comp);
     if (all_tiles >= (1ll << 31)) return RLKV_EINVAL;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
     a.trace_on = c->trace_on;
@@ -340,7 +356,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     const int most = in_step ? c->item_tiles : c->item_tiles_alone;
     if (item_tiles > most) item_tiles = most;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
-    a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * a.n_comp, tiles_comp, grid, item_tiles);
+    a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * second_class, tiles_comp, grid, item_tiles);
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     *grid_out = grid;
     return RLKV_OK;
@@ -349,20 +365,22 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
 // `half`: which half of the scratch memory (partials, claim counter) the launch uses; `overlap` and
 // `dep_wait` as in launch_decode.
 int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, int half = 0, bool overlap = false,
-              bool dep_wait = false, int* grid_out = nullptr)
+              bool dep_wait = false, int* grid_out = nullptr, const float* alpha = nullptr)
 {
     DecodeArgs a;
     int grid = 0;
-    int rc = build_decode_args(c, layer, q, out, a, &grid, overlap);
+    int rc = build_decode_args(c, layer, q, out, a, &grid, overlap, alpha);
     if (rc) return rc;
-    if (a.sched.n_slots > c->lay.max_items) return RLKV_EINVAL;  // cannot happen: the scratch is sized for it
+    if (a.sched.n_slots > c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
+    // mixed attention: both units of a head add into `out`
+    if (alpha) RLKV_CUDA(cudaMemsetAsync(out, 0, (size_t)c->batch * c->q_heads * c->head_dim * sizeof(float), s));
     a.partials = dev_at<float>(c, c->lay.off_partials) +
                  (size_t)half * c->lay.max_items * partial_floats(c->head_dim, a.group);
-    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * c->batch * c->kv_heads;
+    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * 2 * c->batch * c->kv_heads;
     a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4 + half;
     a.claim_base = c->claims[half];
     a.dep_wait = dep_wait ? 1 : 0;
-    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap));
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap, alpha != nullptr));
     c->claims[half] += (unsigned int)a.sched.n_items;  // every CTA claims until it is told there is no more
     if (grid_out) *grid_out = grid;
     c->launches++;
@@ -692,6 +710,17 @@ int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q
 }
 
 size_t rlkv_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+int rlkv_decode_mixed_attention(rlkv_cache* c, int layer, const void* q, const float* alpha, void* out, void* stream)
+{
+    if (!valid_layer(c, layer) || !q || !alpha || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(alpha) & 3u) != 0) return RLKV_EINVAL;
+    if (c->lay.n_comp[layer] != 0) return RLKV_EINVAL;  // the full branch needs every token of every head
+    if (c->len[layer] < 1) return RLKV_EEMPTY;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream), 0, false, false, nullptr, alpha);
+}
 
 int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* out, void* stream)
 {

@@ -223,6 +223,13 @@ struct DecodeArgs {
     int batch, group, q_heads;
     float scale_log2;           // log2(e) / sqrt(head_dim)
     int trace_on;
+    // Mixed attention (paper, Eq. 1; MIXED kernels only).  Every head of the layer is full; beside
+    // the FULL unit of each (batch row, head) the schedule's second class holds a LOCAL unit over
+    // the same rows restricted to the sink and the window: tiles 0 .. local_sink_tiles-1 cover rows
+    // [0, local_sink), the tiles after them rows [local_win0, local_win0 + local_win_len).  Both
+    // units add their weighted result into `out`, which the host clears before the launch.
+    const float* alpha;         // gates of the layer's KV heads (device, [kv_heads]); null otherwise
+    int local_sink, local_sink_tiles, local_win0, local_win_len;
     Schedule sched;
     unsigned char head_of_slot[kMaxKvHeads];  // KV head of full slot 0..n_full-1, then of the compressed slots
 };
@@ -247,6 +254,7 @@ struct UnitInfo {
     int b, head;     // batch row, KV head
 };
 
+template <bool MIXED = false>
 __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
 {
     UnitInfo u;
@@ -256,6 +264,12 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
         u.len = a.len_full;
         u.b = u.pos.uid / a.n_full;
         u.head = a.head_of_slot[u.pos.uid - u.b * a.n_full];
+    } else if (MIXED) {  // the local unit of full unit uid - U
+        const int unit = u.pos.uid - a.sched.U;
+        u.tiles = a.sched.tc;
+        u.len = 0;       // its tiles' rows come from local_tile
+        u.b = unit / a.n_full;
+        u.head = a.head_of_slot[unit - u.b * a.n_full];
     } else {
         const int unit = u.pos.uid - a.sched.U;
         u.tiles = a.sched.tc;
@@ -264,6 +278,21 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
         u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
     }
     return u;
+}
+
+// Mixed attention: tile `tile` of a local unit holds rows [row, row + valid) of its head; what
+// follows them in the 64-row box is fetched and masked.
+__device__ inline void local_tile(const DecodeArgs& a, int tile, int& row, int& valid)
+{
+    if (tile < a.local_sink_tiles) {
+        row = tile * kTile;
+        valid = a.local_sink - row;
+    } else {
+        const int off = (tile - a.local_sink_tiles) * kTile;
+        row = a.local_win0 + off;
+        valid = a.local_win_len - off;
+    }
+    if (valid > kTile) valid = kTile;
 }
 
 #ifdef __CUDACC__
@@ -297,7 +326,7 @@ struct AppendAllArgs {
 };
 cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream, bool overlap);
+                          int stages, int groups, cudaStream_t stream, bool overlap, bool mixed = false);
 cudaError_t prepare_decode_kernels(int head_dim);
 size_t decode_smem_bytes(int head_dim, int stages, int group, int groups);
 

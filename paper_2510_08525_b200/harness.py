@@ -49,6 +49,13 @@ class Cache:
         rl.rlkv_decode_attention(self.handle, layer, q, out)
         return out
 
+    def decode_mixed(self, layer, q, alpha, out=None):
+        """alpha: fp32 [kv_heads] on the cache's device."""
+        if out is None:
+            out = torch.empty((self.batch, self.q_heads, self.head_dim), dtype=torch.float32, device=self.device)
+        rl.rlkv_decode_mixed_attention(self.handle, layer, q, alpha, out)
+        return out
+
     def length(self, layer) -> int:
         return rl.rlkv_length(self.handle, layer)
 
