@@ -64,6 +64,7 @@ def parse_args(argv=None):
     p.add_argument("--item-tiles", type=int, default=0, help="smallest work item of the decode kernel, in 64-row tiles")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
+    p.add_argument("--no-mixed", action="store_true", help="skip the mixed-attention (Eq. 1) side measurement")
     return p.parse_args(argv)
 
 
@@ -402,6 +403,43 @@ def run_ours(args, w, mask):
         e2e = {"value": world * w.batch * K / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K,
                "checksum": float(out_host.double().abs().sum())}
+    # ---- side measurement: mixed attention (Eq. 1) on a 4-layer all-full cache of the same shape.  Every
+    # layer's K/V rows exceed the L2 and the launches cycle through the layers, so each launch reads from HBM.
+    mixed = None
+    if not args.no_mixed and rank == 0:
+        ml, reps = 4, max(K, 8)
+        n = w.context + 1
+        mw = w.with_(layers=ml, frac_compressed=0.0)
+        mcache = harness.Cache(ml, w.kv_heads, w.q_heads, w.head_dim, w.batch, n + 8, np.ones(ml * w.kv_heads, np.uint8),
+                               w.sink, w.window, device=dev)
+        harness.fill_cache(mcache, mw, n)
+        alpha = torch.rand(w.kv_heads, dtype=torch.float32, device=dev)
+        q = steps_in[0][2]
+        mout = torch.empty((ml, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+        times = {}
+        for name, call in (("plain", lambda l: rl.rlkv_decode_attention(mcache.handle, l, q[l % w.layers], mout[l], stream)),
+                           ("mixed", lambda l: rl.rlkv_decode_mixed_attention(mcache.handle, l, q[l % w.layers], alpha,
+                                                                              mout[l], stream))):
+            for i in range(2 * ml):
+                call(i % ml)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(reps * ml):
+                call(i % ml)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            times[name] = e0.elapsed_time(e1) / (reps * ml)
+        full_bytes = w.batch * w.kv_heads * n * 4 * w.head_dim
+        local_rows = min(n, w.sink) + min(w.window, max(n - w.sink, 0))
+        mixed = {"workload": f"{ml} all-full layers of the {w.name} shape, n = {n}, launches back to back (not overlapped)",
+                 "launch_us": 1e3 * times["mixed"], "plain_launch_us": 1e3 * times["plain"],
+                 "algorithmic_bytes_per_launch": full_bytes,
+                 "achieved_gbs": full_bytes / (times["mixed"] * 1e-3) / 1e9,
+                 "plain_gbs": full_bytes / (times["plain"] * 1e-3) / 1e9,
+                 "local_branch_rows_reread": local_rows, "launches_timed": reps * ml}
+        if mcache.status() != 0:
+            raise SystemExit("a mixed-attention kernel reported a status: results are invalid")
+        mcache.close()
     clocks.__exit__()
     status = cache.status()
     if status != 0:
@@ -431,6 +469,7 @@ def run_ours(args, w, mask):
             "step_hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
             "bytes_ratio_vs_uncompressed": total_bytes / (w.batch * w.layers * w.kv_heads * (w.context + 1) * 4 * w.head_dim),
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
+            "mixed_attention": mixed,
             "clocks": clocks.summary(clock_mark),
         }
         print(json.dumps(line), flush=True)

@@ -122,3 +122,38 @@ def test_mixed_attention_argument_checks(rl, hz, cuda_device):
     # one token: softmax over one row is that row of V, whatever the gate
     np.testing.assert_allclose(out.cpu().numpy()[0, :4], np.tile(k[0, 0].float().cpu().numpy(), (4, 1)), atol=1e-6)
     cache.close()
+
+
+@pytest.mark.parametrize("name,layers", [("llama8b", 3), ("qwen7b", 2)])
+def test_mixed_attention_full_size_sampled_units(rl, hz, cuda_device, name, layers):
+    """The benchmark's shapes (every head full, a few layers of them) with the launch the benchmark's
+    side measurement times: sampled (layer, batch row, KV head) units against the oracle, which
+    regenerates the unit's K/V history from the addressable generator."""
+    w = synth.WORKLOADS[name].with_(layers=layers, frac_compressed=0.0)
+    n = w.context + 1
+    mask = np.ones(layers * w.kv_heads, np.uint8)
+    cache = hz.Cache(layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, n + 8, mask, w.sink, w.window,
+                     device=cuda_device)
+    hz.fill_cache(cache, w, n)
+    g = torch.Generator().manual_seed(5)
+    alpha = torch.rand((layers, w.kv_heads), generator=g, dtype=torch.float32)
+    a_dev = alpha.to(cuda_device)
+    q = hz.step_inputs(w, n - 1, cuda_device)[2]
+    outs = [cache.decode_mixed(l, q[l], a_dev[l]) for l in range(layers)]
+    torch.cuda.synchronize()
+    assert cache.status() == 0
+    q = q.cpu()
+    rng = np.random.default_rng(77)
+    G = w.group
+    for _ in range(6):
+        layer, b, h = int(rng.integers(layers)), int(rng.integers(w.batch)), int(rng.integers(w.kv_heads))
+        o = Oracle(1, 1, G, w.head_dim, 1, n, [1], w.sink, w.window)
+        K = synth.unit_rows(w.seed, synth.STREAM_K, layer, 0, n, w.batch, w.kv_heads, w.head_dim, b, h)
+        V = synth.unit_rows(w.seed, synth.STREAM_V, layer, 0, n, w.batch, w.kv_heads, w.head_dim, b, h)
+        kb, vb = K.view(torch.int16).numpy().view(np.uint16), V.view(torch.int16).numpy().view(np.uint16)
+        for t in range(n):
+            o.append(0, kb[t], vb[t])
+        want = o.decode_mixed(0, q[layer, b, h * G:(h + 1) * G].contiguous(), [float(alpha[layer, h])])[0]
+        check_out(outs[layer][b, h * G:(h + 1) * G].cpu().numpy(), want)
+    cache.close()
+    torch.cuda.empty_cache()
