@@ -160,6 +160,63 @@ int rlkv_step(rlkv_cache* cache, const void* k, const void* v, const void* q, vo
 int rlkv_step_host(rlkv_cache* cache, const void* k_host, const void* v_host, const void* q_host,
                    void* out_host, void* stream);
 
+/* ---- the paged, ragged cache: the serving layout --------------------------------------------------
+ * Section 4.3 of the paper serves requests of different lengths with continuous batching: the full
+ * heads live in a paged pool, the compressed heads in a fixed-size pool with one constant-size
+ * buffer per request, and the memory the compressed heads no longer need admits more requests.
+ * rlkv_paged is that layout: max_seqs REQUEST SLOTS, each with its own length (per layer); the
+ * full heads of all slots share n_pages PAGES of 64 tokens, handed out from one free list as
+ * sequences grow and taken back when a slot is closed (page p of a sequence is page p of every full
+ * head of every layer, as in the usual block table); every slot owns a sink + window ring per
+ * compressed head.  What is computed per sequence is exactly what the lock-step cache computes for a
+ * batch row (same slot rule, same attention); the calls name the request slots they act on, so a
+ * decode step can serve any subset of the open slots, each at its own length.
+ * Limits: max_seq_len <= 65536 tokens; at most min(max_seqs, 256) sequences per call; the other
+ * shape limits of rlkv_cache_create.  Device memory: rlkv_paged_size bytes, library- or caller-owned
+ * as for rlkv_cache_create.  Errors leave the cache unchanged. */
+typedef struct rlkv_paged rlkv_paged;
+int rlkv_paged_size(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                    int max_seq_len, const uint8_t* head_is_full, int sink, int window,
+                    size_t* bytes_out);
+int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim,
+                      int max_seqs, int n_pages, int max_seq_len, const uint8_t* head_is_full,
+                      int sink, int window, void* device_buf, size_t device_buf_bytes);
+int rlkv_paged_destroy(rlkv_paged* cache);
+/* Takes a free request slot (length 0 in every layer): RLKV_EFULL if all max_seqs are open. */
+int rlkv_paged_seq_open(rlkv_paged* cache, int* slot_out);
+/* Closes a slot: its pages go back to the free list.  The caller makes sure no work that uses the
+ * slot is still in flight (host bookkeeping only, nothing is enqueued). */
+int rlkv_paged_seq_close(rlkv_paged* cache, int slot);
+/* One token for each of n sequences of one layer.  slots: HOST int[n], open slots, none twice;
+ * k, v: device bf16 [n][kv_heads][head_dim], entry i for slots[i].  A sequence whose token opens a
+ * page takes one from the free list.  RLKV_EFULL (nothing appended for any sequence) if a sequence
+ * is at max_seq_len or the free list cannot serve every new page. */
+int rlkv_paged_append(rlkv_paged* cache, int layer, const int* slots, int n, const void* k,
+                      const void* v, void* stream);
+/* n_tokens tokens for one sequence, exactly n_tokens single appends.  k, v: device bf16
+ * [n_tokens][kv_heads][head_dim]. */
+int rlkv_paged_prefill(rlkv_paged* cache, int layer, int slot, const void* k, const void* v,
+                       int n_tokens, void* stream);
+/* Decode attention for n sequences of one layer, each over its own length, one launch for both
+ * head classes and all lengths.  q: device bf16 [n][q_heads][head_dim]; out: device fp32
+ * [n][q_heads][head_dim]; entry i belongs to slots[i] (HOST int[n]).  RLKV_EEMPTY if a listed
+ * sequence holds no token in this layer. */
+int rlkv_paged_decode_attention(rlkv_paged* cache, int layer, const int* slots, int n,
+                                const void* q, void* out, void* stream);
+int rlkv_paged_length(const rlkv_paged* cache, int layer, int slot, int* len_out);
+/* Pages on the free list and pages in total. */
+int rlkv_paged_pages(const rlkv_paged* cache, int* free_out, int* total_out);
+/* Bytes of K and V rows the next rlkv_paged_decode_attention on these slots must read. */
+int rlkv_paged_step_bytes(const rlkv_paged* cache, int layer, const int* slots, int n,
+                          uint64_t* kv_bytes_out);
+/* One head of one sequence copied to the host (synchronises the device).  A full head: its
+ * length(layer, slot) rows in token order, gathered page by page (k_host, v_host hold up to
+ * max_seq_len rows); a compressed head: its sink + window physical rows, as
+ * rlkv_debug_export_head. */
+int rlkv_paged_debug_export_head(rlkv_paged* cache, int layer, int slot, int kv_head, void* k_host,
+                                 void* v_host, int* rows_out, int32_t* token_of_slot_host);
+int rlkv_paged_kernel_status(rlkv_paged* cache, int* status_out);
+
 /* ---- introspection (host-side bookkeeping; no GPU work unless stated) ---- */
 int rlkv_length(const rlkv_cache* cache, int layer, int* len_out);
 /* Bytes of K and V rows the next rlkv_decode_attention on `layer` must read:

@@ -43,6 +43,19 @@ SIGNATURES = {
     "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
     "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
+    "rlkv_paged_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
+    "rlkv_paged_create": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _sz]),
+    "rlkv_paged_destroy": (_ci, [_vp]),
+    "rlkv_paged_seq_open": (_ci, [_vp, ctypes.POINTER(_ci)]),
+    "rlkv_paged_seq_close": (_ci, [_vp, _ci]),
+    "rlkv_paged_append": (_ci, [_vp, _ci, _vp, _ci, _vp, _vp, _vp]),
+    "rlkv_paged_prefill": (_ci, [_vp, _ci, _ci, _vp, _vp, _ci, _vp]),
+    "rlkv_paged_decode_attention": (_ci, [_vp, _ci, _vp, _ci, _vp, _vp, _vp]),
+    "rlkv_paged_length": (_ci, [_vp, _ci, _ci, ctypes.POINTER(_ci)]),
+    "rlkv_paged_pages": (_ci, [_vp, ctypes.POINTER(_ci), ctypes.POINTER(_ci)]),
+    "rlkv_paged_step_bytes": (_ci, [_vp, _ci, _vp, _ci, ctypes.POINTER(ctypes.c_uint64)]),
+    "rlkv_paged_debug_export_head": (_ci, [_vp, _ci, _ci, _ci, _vp, _vp, ctypes.POINTER(_ci), _vp]),
+    "rlkv_paged_kernel_status": (_ci, [_vp, ctypes.POINTER(_ci)]),
 }
 
 
@@ -235,3 +248,95 @@ def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, it
 
 def rlkv_strerror(code: int) -> str:
     return lib.rlkv_strerror(code).decode()
+
+
+# ---- the paged, ragged cache -------------------------------------------------------------------
+def _slots(slots) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(slots, dtype=np.int32).reshape(-1))
+
+
+def rlkv_paged_size(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window) -> int:
+    m = _mask(head_is_full)
+    if m.size != layers * kv_heads:
+        raise ValueError("head_is_full must have layers*kv_heads entries")
+    out = _sz(0)
+    _check(lib.rlkv_paged_size(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, m.ctypes.data, sink,
+                               window, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_paged_create(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window,
+                      device_buf=None, device_buf_bytes=0) -> int:
+    m = _mask(head_is_full)
+    if m.size != layers * kv_heads:
+        raise ValueError("head_is_full must have layers*kv_heads entries")
+    handle = _vp(0)
+    _check(lib.rlkv_paged_create(ctypes.byref(handle), layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
+                                 m.ctypes.data, sink, window, _ptr(device_buf), device_buf_bytes))
+    return int(handle.value)
+
+
+def rlkv_paged_destroy(cache) -> None:
+    _check(lib.rlkv_paged_destroy(cache))
+
+
+def rlkv_paged_seq_open(cache) -> int:
+    slot = _ci(-1)
+    _check(lib.rlkv_paged_seq_open(cache, ctypes.byref(slot)))
+    return int(slot.value)
+
+
+def rlkv_paged_seq_close(cache, slot) -> None:
+    _check(lib.rlkv_paged_seq_close(cache, slot))
+
+
+def rlkv_paged_append(cache, layer, slots, k, v, stream=None) -> None:
+    s = _slots(slots)
+    _check(lib.rlkv_paged_append(cache, layer, s.ctypes.data, s.size, _ptr(k), _ptr(v), _stream(stream)))
+
+
+def rlkv_paged_prefill(cache, layer, slot, k, v, n_tokens, stream=None) -> None:
+    _check(lib.rlkv_paged_prefill(cache, layer, slot, _ptr(k), _ptr(v), n_tokens, _stream(stream)))
+
+
+def rlkv_paged_decode_attention(cache, layer, slots, q, out, stream=None) -> None:
+    s = _slots(slots)
+    _check(lib.rlkv_paged_decode_attention(cache, layer, s.ctypes.data, s.size, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_paged_length(cache, layer, slot) -> int:
+    out = _ci(0)
+    _check(lib.rlkv_paged_length(cache, layer, slot, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_paged_pages(cache):
+    """(pages on the free list, pages in total)."""
+    free, total = _ci(0), _ci(0)
+    _check(lib.rlkv_paged_pages(cache, ctypes.byref(free), ctypes.byref(total)))
+    return int(free.value), int(total.value)
+
+
+def rlkv_paged_step_bytes(cache, layer, slots) -> int:
+    s = _slots(slots)
+    out = ctypes.c_uint64(0)
+    _check(lib.rlkv_paged_step_bytes(cache, layer, s.ctypes.data, s.size, ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_paged_debug_export_head(cache, layer, slot, kv_head, max_rows, head_dim):
+    """Returns (k, v, token_of_slot) as numpy arrays (uint16 bf16 bits [rows][head_dim], int32 [rows])."""
+    k = np.zeros((max_rows, head_dim), dtype=np.uint16)
+    v = np.zeros((max_rows, head_dim), dtype=np.uint16)
+    tok = np.full(max_rows, -1, dtype=np.int32)
+    rows = _ci(0)
+    _check(lib.rlkv_paged_debug_export_head(cache, layer, slot, kv_head, k.ctypes.data, v.ctypes.data, ctypes.byref(rows),
+                                            tok.ctypes.data))
+    n = int(rows.value)
+    return k[:n], v[:n], tok[:n]
+
+
+def rlkv_paged_kernel_status(cache) -> int:
+    out = _ci(0)
+    _check(lib.rlkv_paged_kernel_status(cache, ctypes.byref(out)))
+    return int(out.value)

@@ -79,7 +79,56 @@ __global__ void __launch_bounds__(256) append_all_kernel(const __grid_constant__
     }
 }
 
+// Paged cache.  A full head's token t goes to row t % 64 of the sequence's page t / 64; a compressed
+// head's to its ring slot (request slot instead of batch row).  The thread that writes the first piece
+// of the row of the layer's first full head also records the page in the device page table (every
+// token of a page and every layer write the same value there).
+__global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant__ PagedAppendArgs a)
+{
+    const int chunks = a.head_dim / 8;
+    const long long total = (long long)a.n * a.kv_heads * chunks * 2;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        long long r = i;
+        const int c = (int)(r % chunks);
+        r /= chunks;
+        const int h = (int)(r % a.kv_heads);
+        r /= a.kv_heads;
+        const int e = (int)(r % a.n);   // entry of k, v
+        const int kv = (int)(r / a.n);  // 0 = K, 1 = V
+        const int seq = a.prefill ? a.slot[0] : a.slot[e];
+        const int t = a.prefill ? a.t0 + e : a.t[e];
+        const int page = a.page[a.prefill ? t / kTile - a.first_page : e];
+        const int slot = a.slot_of_head[h];
+        long long row;
+        if (slot >= 0) {
+            row = a.full_row0 + (((long long)slot * a.n_pages + page) * 2 + kv) * kTile + t % kTile;
+            if (slot == 0 && c == 0 && kv == 0) a.page_table[(size_t)seq * a.table_stride + t / kTile] = page;
+        } else {
+            if (a.prefill) {
+                const int n_final = a.t0 + a.n;
+                if (!(t < a.sink || t >= n_final - a.window)) continue;  // evicted before the batch ends
+            }
+            const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
+            row = a.comp_row0 + (((long long)seq * a.n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
+        }
+        const __nv_bfloat16* src = (kv ? a.v : a.k) + ((long long)e * a.kv_heads + h) * a.head_dim;
+        const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
+        reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_paged_append(const PagedAppendArgs& a, cudaStream_t stream)
+{
+    const long long total = (long long)a.n * a.kv_heads * (a.head_dim / 8) * 2;
+    long long blocks = (total + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks < 1) blocks = 1;
+    paged_append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream)
 {

@@ -220,19 +220,21 @@ struct Smem {
     }
     static constexpr int kMergeStride = D + kMergePad;      // floats per head row
     static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
-    static constexpr int kBarriers = 2 * 8 + 2 * kItemRing + 2 + 2 * kMergeBuffers;
+    static constexpr int kBarriers = 2 * 8 + 2 * kItemRing + 2 + 2 * kMergeBuffers + 2;  // the last two: page look-ups
     __host__ __device__ static constexpr int merge_floats(int group) { return kWarps * group * kMergeStride; }
     // one hand-off buffer: merge rows, per-warp max and sum, segment descriptor
     __host__ __device__ static constexpr int buffer_bytes(int group)
     {
         return merge_floats(group) * 4 + kStatFloats * 4 + 32;
     }
-    __host__ __device__ static constexpr size_t bytes(int stages, int group)
+    // paged cache only: the page-table entries of the segment being streamed, the PagedArgs
+    static constexpr int kPagedBytes = (kMaxSeqPages + 4) * 4 + (int)((sizeof(PagedArgs) + 15) / 16 * 16);
+    __host__ __device__ static constexpr size_t bytes(int stages, int group, int mode = kModePlain)
     {
         return (size_t)stages * stage_bytes(group) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
-               (sizeof(DecodeArgs) + 15) / 16 * 16;
+               (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged ? kPagedBytes : 0);
     }
 };
 
@@ -349,10 +351,28 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
 // MIXED: the mixed attention of Eq. 1.  The schedule's second class holds, for every full unit, a
 // LOCAL unit over the same head's sink and window rows; its tiles start at whatever row the window
 // starts (a TMA box may start at any row) and are masked past their valid rows.
-template <int D, int NG, bool MIXED>
+//
+// kModePaged: the paged cache.  Units keep the uniform layout (every full unit is given the tiles of
+// the longest sequence); producer and consumers both leave out a unit's tiles past its own length and
+// realign the slot counter at every segment, and the producer looks a full unit's rows up in the
+// sequence's page table, whose entries for a segment it fetches with one bulk copy.
+struct NoPagedArgs {};
+template <int MODE>
+struct ExtraArgs {
+    typedef NoPagedArgs type;
+};
+template <>
+struct ExtraArgs<kModePaged> {
+    typedef PagedArgs type;
+};
+
+template <int D, int NG, int MODE>
 __global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
-decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ CUtensorMap tmap, const int stages)
+decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ CUtensorMap tmap, const int stages,
+              const __grid_constant__ typename ExtraArgs<MODE>::type extra)
 {
+    constexpr bool MIXED = MODE == kModeMixed;
+    constexpr bool PAGED = MODE == kModePaged;
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     constexpr int MS = S::kMergeStride;
@@ -370,7 +390,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     uint64_t* claim_empty = claim_full + 1;
     uint64_t* ep_full = claim_empty + 1;
     uint64_t* ep_empty = ep_full + kMergeBuffers;
-    int4* item_desc = reinterpret_cast<int4*>(ep_empty + kMergeBuffers);
+    uint64_t* page_bar = ep_empty + kMergeBuffers;  // [2], the second one unused
+    int4* item_desc = reinterpret_cast<int4*>(page_bar + 2);
     volatile int* claim_slot = reinterpret_cast<volatile int*>(item_desc + kItemRing);
     volatile int* ep_flag = claim_slot + 1;
     volatile int* s_abort = claim_slot + 2;
@@ -382,6 +403,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     // run-time indices, which is slow on kernel parameters and cheap here.
     DecodeArgs* s_args = reinterpret_cast<DecodeArgs*>(lists + kMaxTodo * (kMaxRounds + 1));
     const DecodeArgs& a = *s_args;
+    // paged cache: lengths and request slots of the batch, then the page ids of one segment
+    PagedArgs* s_paged = reinterpret_cast<PagedArgs*>(reinterpret_cast<uint8_t*>(s_args) + (sizeof(DecodeArgs) + 15) / 16 * 16);
+    int* s_pages = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(s_paged) + (sizeof(PagedArgs) + 15) / 16 * 16);
+    const PagedArgs* pg = PAGED ? s_paged : nullptr;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -401,6 +426,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     }
     for (int i = tid; i < (int)(sizeof(DecodeArgs) / sizeof(int)); i += blockDim.x)
         reinterpret_cast<int*>(s_args)[i] = reinterpret_cast<const int*>(&args)[i];
+    if (PAGED)
+        for (int i = tid; i < (int)(sizeof(PagedArgs) / sizeof(int)); i += blockDim.x)
+            reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
@@ -412,6 +440,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         }
         mbar_init(smem_u32(claim_full), 1);
         mbar_init(smem_u32(claim_empty), 1);
+        mbar_init(smem_u32(page_bar), 1);
         for (int i = 0; i < kMergeBuffers; ++i) {
             mbar_init(smem_u32(ep_full + i), S::kWarps);
             mbar_init(smem_u32(ep_empty + i), kEpilogueWarps);
@@ -424,6 +453,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     __syncthreads();
 
     int issued = 0;  // producer: slots issued so far (data or empty)
+    int page_lost_par = -1;  // producer, paged cache: phase of a page look-up it gave up waiting for
     if (warp < S::kWarps) {
         // ------------------------------------------------------------------ consumer warps
         const int grp = warp / kGroupWarps, wig = warp % kGroupWarps;  // tile group, 16-token slice
@@ -457,7 +487,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 if (tr0 && n_items < 11) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
                 // skip the empty slots the producer issued to line the slot counter up with x0
-                for (int pad = ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
+                for (int pad = PAGED ? 0 : ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
                     if (turn != grp) continue;
                     alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
                     if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
@@ -472,16 +502,26 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
                 if (item >= 0) {
-                    u = locate<MIXED>(a, x);
+                    u = locate<MODE>(a, x, pg);
                     seg_tiles = min(x1 - x, u.pos.run);
                     const bool local_unit = MIXED && u.pos.uid >= sc.U;
+                    int seg_eff = seg_tiles;  // tiles of the segment that exist
+                    if (PAGED) {
+                        seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
+                        // tiles left out shift the slot counter against x: skip the producer's empty slots
+                        for (int pad = seg_eff > 0 ? ((x - cnt) % NG + NG) % NG : 0; alive && pad > 0; --pad, next_slot()) {
+                            if (turn != grp) continue;
+                            alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
+                            if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
+                        }
+                    }
                     // Q as the A operand (rows = query heads of the group, rows >= G are zero): read from
                     // the stage of this warp's first tile of the segment, where the producer put the
                     // unit's query rows
                     uint32_t qa[KS][2];
                     bool have_q = false;
                     int valid_left = u.len - u.pos.tile * kTile;  // valid rows from this tile to the unit's end
-                    for (int i = 0; alive && i < seg_tiles; ++i, next_slot(), valid_left -= kTile) {
+                    for (int i = 0; alive && i < seg_eff; ++i, next_slot(), valid_left -= kTile) {
                         if (turn != grp) continue;
                         alive = wait_traced(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout, tr0,
                                             &ns_tile);
@@ -652,6 +692,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             const long long t_prod = clock64();
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             bool synced = false;  // has waited for the kernels before this one
+            uint32_t ppar = 0;    // PAGED: phase of the page look-up barrier
             while (ok && k < sc.n_items) {
                 const long long ti0 = trace ? clock64() : 0;
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
@@ -670,7 +711,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 }
                 if (trace) cy_item += clock64() - ti0;
                 // empty slots until the slot counter has the residue of x0
-                for (int pad = ((x0 - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
+                for (int pad = PAGED ? 0 : ((x0 - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
                     ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
                     if (!ok) break;
                     mbar_arrive(smem_u32(full_bar + s));
@@ -682,15 +723,70 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 }
                 int seg_left = 0, seg_idx = 0, krow = 0, vrow = 0;
                 int local_row0 = -1, local_next = 0;  // MIXED, inside a local unit: first row of its head, next tile
+                // PAGED: tiles of the segment past the unit's own length (not issued); first pool row of the
+                // full head's pages (-1: a compressed unit); page-table index of s_pages[0]; next tile
+                int seg_skip = 0, paged_row0 = -1, page_base = 0, paged_tile = 0;
+                bool asked = false;
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
-                    if (x == x_ask) mbar_arrive(smem_u32(claim_empty));
+                    if (PAGED) {
+                        if (!asked && x >= x_ask) {
+                            mbar_arrive(smem_u32(claim_empty));
+                            asked = true;
+                        }
+                    } else if (x == x_ask) {
+                        mbar_arrive(smem_u32(claim_empty));
+                    }
                     const long long ts0 = trace ? clock64() : 0;
                     if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
-                        const UnitInfo u = locate<MIXED>(a, x);
+                        const UnitInfo u = locate<MODE>(a, x, pg);
                         seg_left = min(x1 - x, u.pos.run);
                         seg_idx = 0;
                         local_row0 = -1;
+                        if (PAGED) {
+                            const int seg_eff = max(0, min(seg_left, (u.len + kTile - 1) / kTile - u.pos.tile));
+                            seg_skip = seg_left - seg_eff;
+                            seg_left = seg_eff;
+                            if (seg_eff == 0) {  // nothing of this unit here
+                                x += seg_skip - 1;
+                                continue;
+                            }
+                            // empty slots until the slot counter has the residue of x
+                            for (int pad = ((x - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
+                                ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
+                                if (!ok) break;
+                                mbar_arrive(smem_u32(full_bar + s));
+                                ++issued;
+                                if (++s == stages) {
+                                    s = 0;
+                                    par ^= 1u;
+                                }
+                            }
+                            if (!ok) break;
+                            paged_tile = u.pos.tile;
+                            if (u.pos.uid < sc.U) {
+                                // the segment's page-table entries, widened to 16-byte pieces, in one bulk copy
+                                const int first = u.pos.tile & ~3, last = (u.pos.tile + seg_eff + 3) & ~3;
+                                const int* src = pg->page_table + (size_t)pg->seq_slot[u.b] * pg->table_stride + first;
+                                mbar_expect_tx(smem_u32(page_bar), (uint32_t)(last - first) * 4u);
+                                bulk_load(smem_u32(s_pages), src, (uint32_t)(last - first) * 4u, smem_u32(page_bar));
+                                ok = wait_bounded(smem_u32(page_bar), ppar, s_abort, a.status, kStatusPageWaitTimeout);
+                                if (!ok) {
+                                    page_lost_par = (int)ppar;
+                                    break;
+                                }
+                                ppar ^= 1u;
+                                page_base = first;
+                                paged_row0 = (int)(a.full_row0 + (long long)(u.pos.uid - u.b * a.n_full) * pg->n_pages * 2 * kTile);
+                            } else {
+                                paged_row0 = -1;
+                                const int c = u.pos.uid - sc.U - u.b * a.n_comp;
+                                krow = (int)(a.comp_row0 + ((long long)pg->seq_slot[u.b] * a.n_comp + c) * 2 * a.rows_comp) +
+                                       u.pos.tile * kTile;
+                                vrow = krow + a.rows_comp;
+                            }
+                            qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
+                        } else {
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit.  Everything else is older and may be fetched early.
                         if (a.dep_wait && !synced &&
@@ -709,6 +805,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             vrow = krow + a.rows_comp;
                         }
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
+                        }
+                    }
+                    if (PAGED && paged_row0 >= 0) {
+                        krow = paged_row0 + s_pages[paged_tile++ - page_base] * (2 * kTile);
+                        vrow = krow + kTile;
                     }
                     if (MIXED && local_row0 >= 0) {
                         int row, valid;
@@ -750,8 +851,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         s = 0;
                         par ^= 1u;
                     }
+                    if (PAGED && seg_left == 0) x += seg_skip;  // the unit's tiles that do not exist
                 }
                 if (!ok) break;
+                if (PAGED && !asked) mbar_arrive(smem_u32(claim_empty));
                 ok = wait_traced(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout, trace, &ns_claim);
                 cpar ^= 1u;
                 if (ok) k = *claim_slot;
@@ -937,16 +1040,18 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             for (int j = issued > stages ? issued - stages : 0; j < issued; ++j)
                 wait_bounded(smem_u32(full_bar + j % stages), (uint32_t)(j / stages) & 1u, s_abort, a.status,
                              kStatusDrainTimeout, false);
+            if (PAGED && page_lost_par >= 0)
+                wait_bounded(smem_u32(page_bar), (uint32_t)page_lost_par, s_abort, a.status, kStatusDrainTimeout, false);
         }
     }
     if (trace && tid == 0) my_trace[3] = global_timer_ns();
 }
 
-template <int D, int NG, bool MIXED>
+template <int D, int NG, int MODE>
 cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
-                       bool overlap)
+                       bool overlap, const typename ExtraArgs<MODE>::type& extra)
 {
-    const size_t smem = Smem<D, NG>::bytes(stages, a.group);
+    const size_t smem = Smem<D, NG>::bytes(stages, a.group, MODE);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(Smem<D, NG>::kThreads);
@@ -957,28 +1062,30 @@ cudaError_t launch_one(const DecodeArgs& a, const CUtensorMap& tmap, int grid, i
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<D, NG, MIXED>, a, tmap, stages);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<D, NG, MODE>, a, tmap, stages, extra);
 }
 
 template <int D, int NG>
 cudaError_t prepare_one()
 {
-    const cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, NG, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                               kMaxDynamicSmem);
+    cudaError_t e = cudaFuncSetAttribute(decode_kernel<D, NG, kModePlain>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         kMaxDynamicSmem);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(decode_kernel<D, NG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(decode_kernel<D, NG, kModeMixed>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(decode_kernel<D, NG, kModePaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kMaxDynamicSmem);
 }
 
 }  // namespace
 
-size_t decode_smem_bytes(int head_dim, int stages, int group, int groups)
+size_t decode_smem_bytes(int head_dim, int stages, int group, int groups, int mode)
 {
     if (head_dim == 128)
-        return groups == 1 ? Smem<128, 1>::bytes(stages, group)
-                           : groups == 2 ? Smem<128, 2>::bytes(stages, group) : Smem<128, 3>::bytes(stages, group);
-    return groups == 1 ? Smem<64, 1>::bytes(stages, group)
-                       : groups == 2 ? Smem<64, 2>::bytes(stages, group) : Smem<64, 3>::bytes(stages, group);
+        return groups == 1 ? Smem<128, 1>::bytes(stages, group, mode)
+                           : groups == 2 ? Smem<128, 2>::bytes(stages, group, mode) : Smem<128, 3>::bytes(stages, group, mode);
+    return groups == 1 ? Smem<64, 1>::bytes(stages, group, mode)
+                       : groups == 2 ? Smem<64, 2>::bytes(stages, group, mode) : Smem<64, 3>::bytes(stages, group, mode);
 }
 
 cudaError_t prepare_decode_kernels(int head_dim)
@@ -996,23 +1103,25 @@ cudaError_t prepare_decode_kernels(int head_dim)
 
 template <int D, int NG>
 static cudaError_t launch_either(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
-                          bool overlap, bool mixed)
+                                 bool overlap, int mode, const PagedArgs* paged)
 {
-    return mixed ? launch_one<D, NG, true>(a, tmap, grid, stages, stream, overlap)
-                 : launch_one<D, NG, false>(a, tmap, grid, stages, stream, overlap);
+    if (mode == kModePaged) return launch_one<D, NG, kModePaged>(a, tmap, grid, stages, stream, overlap, *paged);
+    if (mode == kModeMixed) return launch_one<D, NG, kModeMixed>(a, tmap, grid, stages, stream, overlap, NoPagedArgs{});
+    return launch_one<D, NG, kModePlain>(a, tmap, grid, stages, stream, overlap, NoPagedArgs{});
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream, bool overlap, bool mixed)
+                          int stages, int groups, cudaStream_t stream, bool overlap, int mode, const PagedArgs* paged)
 {
+    if (mode == kModePaged && !paged) return cudaErrorInvalidValue;
     if (head_dim == 128) {
-        if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mixed);
-        if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mixed);
-        return launch_either<128, 3>(a, *tmap, grid, stages, stream, overlap, mixed);
+        if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+        if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+        return launch_either<128, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged);
     }
-    if (groups == 1) return launch_either<64, 1>(a, *tmap, grid, stages, stream, overlap, mixed);
-    if (groups == 2) return launch_either<64, 2>(a, *tmap, grid, stages, stream, overlap, mixed);
-    return launch_either<64, 3>(a, *tmap, grid, stages, stream, overlap, mixed);
+    if (groups == 1) return launch_either<64, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+    if (groups == 2) return launch_either<64, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+    return launch_either<64, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged);
 }
 
 }  // namespace rlkv

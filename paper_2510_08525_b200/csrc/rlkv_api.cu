@@ -23,28 +23,15 @@
 #include <new>
 #include <vector>
 
-#include "../../include/rlkv.h"
-#include "rlkv_internal.cuh"
+#include "rlkv_host.cuh"
 
 using namespace rlkv;
 
-namespace {
-
+namespace rlkv {
 thread_local char g_cuda_text[256] = "";
-
-int cuda_fail(cudaError_t e, const char* what)
-{
-    snprintf(g_cuda_text, sizeof g_cuda_text, "CUDA error in %s: %s", what, cudaGetErrorString(e));
-    return RLKV_ECUDA;
 }
-#define RLKV_CUDA(call)                                  \
-    do {                                                 \
-        cudaError_t e_ = (call);                         \
-        if (e_ != cudaSuccess) return cuda_fail(e_, #call); \
-    } while (0)
 
-size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+namespace {
 
 struct Layout {
     int rows_full = 0, rows_comp = 0;
@@ -57,22 +44,8 @@ struct Layout {
     int max_grid = 0, max_items = 0;
 };
 
-constexpr int kMaxGridSms = 160;  // scratch is sized for 2 CTAs on each of up to 160 SMs
-constexpr int kMinItemTiles = 2;  // smallest work item rlkv_set_decode_config accepts (sizes the scratch)
 constexpr int kDefaultItemTiles = 32;        // launches of rlkv_step, which overlap: coarse items, few partials
 constexpr int kDefaultItemTilesAlone = 8;    // a launch on its own: finer items for an even finish
-
-// Most partial records a decode launch of this shape can write, over every length up to tf tiles
-// per full unit and every grid up to max_grid CTAs.
-long long most_slots(int U, int tf, int Uc, int tc, int max_grid)
-{
-    long long most = 0;
-    for (int p = 1; p <= max_grid; ++p) {
-        const long long m = max_slots(U, tf, Uc, tc, p, kMinItemTiles);
-        if (m > most) most = m;
-    }
-    return most;
-}
 
 int check_shape(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
                 const uint8_t* mask, int sink, int window)
@@ -157,38 +130,6 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
     return RLKV_OK;
 }
 
-// Most pipeline stages (<= 8) that fit `ctas_per_sm` CTAs of the decode kernel on one SM
-// (228 KB per SM, 1 KB of it reserved per resident CTA).  The stage count is a multiple of the
-// number of consumer groups, so that a given stage is always consumed by the same group: an
-// mbarrier parity wait can only tell two phases apart, and a group that reached a stage a whole
-// phase early would take the wait for the phase before as satisfied.
-int max_stages(int head_dim, int group, int groups, int ctas_per_sm)
-{
-    for (int st = 8; st >= 2; --st) {
-        if (st % groups != 0) continue;
-        const size_t one = decode_smem_bytes(head_dim, st, group, groups);
-        if (one <= (size_t)kMaxDynamicSmem && (one + 1024) * ctas_per_sm <= 228u * 1024u) return st;
-    }
-    return 0;
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceGuard(int dev)
-    {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-        if (prev == dev) prev = -1;
-    }
-    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
-};
-
 }  // namespace
 
 struct rlkv_cache {
@@ -242,42 +183,7 @@ int zero_state(rlkv_cache* c, cudaStream_t s)
 
 int make_tensor_map(rlkv_cache* c)
 {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    RLKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-    if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
-    // The pool as rows of 128-byte pieces so that one box is one contiguous run of memory and still
-    // obeys the 128-byte limit of the swizzled inner dimension.  For head_dim 128 the two halves of
-    // the rows are the OUTER dimension of the box, so the tile lands in shared memory as two blocks
-    // of [64 rows][128 bytes]: eight consecutive rows of a block are then eight different swizzle
-    // phases (with 256-byte rows only four, and every ldmatrix would take a two-way bank conflict).
-    //   head_dim 128: [2 halves][rows][64]  box [2][64 rows][64]  (16 KB)
-    //   head_dim  64: [rows][64]            box [64 rows][64]     ( 8 KB)
-    CUresult r;
-    void* base = c->dev_base + c->lay.off_pool;
-    const CUtensorMapL2promotion l2p = CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-    if (c->head_dim == 128) {
-        const cuuint64_t dims[3] = {64, (cuuint64_t)c->lay.pool_rows, 2};
-        const cuuint64_t strides[2] = {256, 128};
-        const cuuint32_t box[3] = {64, (cuuint32_t)kTile, 2};
-        const cuuint32_t estr[3] = {1, 1, 1};
-        r = reinterpret_cast<EncodeTiledFn>(fn)(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box,
-                                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2p,
-                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    } else {
-        const cuuint64_t dims[2] = {64, (cuuint64_t)c->lay.pool_rows};
-        const cuuint64_t strides[1] = {128};
-        const cuuint32_t box[2] = {64, (cuuint32_t)kTile};
-        const cuuint32_t estr[2] = {1, 1};
-        r = reinterpret_cast<EncodeTiledFn>(fn)(&c->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box,
-                                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, l2p,
-                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    }
-    if (r != CUDA_SUCCESS) {
-        snprintf(g_cuda_text, sizeof g_cuda_text, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
-        return RLKV_ECUDA;
-    }
-    return RLKV_OK;
+    return encode_pool_tensor_map(&c->tmap, c->dev_base + c->lay.off_pool, c->lay.pool_rows, c->head_dim);
 }
 
 bool valid_layer(const rlkv_cache* c, int layer) { return c && layer >= 0 && layer < c->layers; }
@@ -380,7 +286,7 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4 + half;
     a.claim_base = c->claims[half];
     a.dep_wait = dep_wait ? 1 : 0;
-    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap, alpha != nullptr));
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap, alpha ? kModeMixed : kModePlain));
     c->claims[half] += (unsigned int)a.sched.n_items;  // every CTA claims until it is told there is no more
     if (grid_out) *grid_out = grid;
     c->launches++;

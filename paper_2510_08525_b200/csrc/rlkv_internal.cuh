@@ -23,6 +23,8 @@ constexpr int kItemRing = 4;     // work-item descriptors in flight between prod
 constexpr int kTraceWords = 40;  // debug trace: 64-bit words per CTA
 constexpr int kMaxTodo = 64;      // split merges a CTA may put off until its stream has ended
 constexpr int kMaxPend = 16;      // partial segments of a CTA whose tickets are drawn when its stream has ended
+constexpr int kMaxPagedBatch = 256;   // sequences one launch over the paged cache may serve
+constexpr int kMaxSeqPages = 1024;    // 64-token pages one sequence may hold (65536 tokens)
 constexpr int kClaimAhead = 3;   // the producer asks for its next work item this many tiles before the current one ends
 
 // Kernel status codes (device error word).
@@ -34,7 +36,15 @@ enum : int {
     kStatusItemWaitTimeout = 4,   // a wait on the work-item ring ran out
     kStatusClaimWaitTimeout = 5,  // a wait between producer and claim warp ran out
     kStatusMergeWaitTimeout = 6,  // a wait between consumer warps and epilogue warps ran out
-    kStatusSmemMisaligned = 7     // dynamic shared memory does not start on a 1024-byte boundary
+    kStatusSmemMisaligned = 7,    // dynamic shared memory does not start on a 1024-byte boundary
+    kStatusPageWaitTimeout = 8    // the producer gave up waiting for page-table entries
+};
+
+// What a decode kernel is compiled for.
+enum : int {
+    kModePlain = 0,   // the lock-step cache: full and compressed heads, one length for the whole batch
+    kModeMixed = 1,   // mixed attention (Eq. 1) over a lock-step cache whose heads are all full
+    kModePaged = 2    // the paged cache: one length per sequence, full heads in 64-token pages
 };
 
 // One record of split-KV partial results: running max and sum (log2 domain) of the G query heads
@@ -234,6 +244,23 @@ struct DecodeArgs {
     unsigned char head_of_slot[kMaxKvHeads];  // KV head of full slot 0..n_full-1, then of the compressed slots
 };
 
+// Paged cache (kModePaged kernels): what DecodeArgs cannot say.  The launch serves `batch` sequences;
+// entry b of q and out belongs to request slot seq_slot[b], which holds seq_len[b] tokens in this
+// layer.  Units are laid out as for the lock-step cache with every full unit given the tiles of the
+// LONGEST sequence; a unit's tiles past its own length are skipped by producer and consumers alike.
+// Full heads: token t of slot s lives in page page_table[s * table_stride + t / 64], row t % 64; page
+// p of full-head slot f of the layer starts at pool row full_row0 + ((f * n_pages + p) * 2) * 64 (K
+// rows, then the 64 V rows).  Compressed heads: the ring of request slot s and compressed-head slot
+// c starts at pool row comp_row0 + ((s * n_comp + c) * 2) * rows_comp.
+struct PagedArgs {
+    const int* page_table;
+    int table_stride;  // entries per request slot, a multiple of 4
+    int n_pages;       // physical pages per full head
+    int cap;           // sink + window
+    int seq_len[kMaxPagedBatch];
+    unsigned short seq_slot[kMaxPagedBatch];
+};
+
 struct AppendArgs {
     __nv_bfloat16* pool;
     long long full_row0, comp_row0;
@@ -254,9 +281,10 @@ struct UnitInfo {
     int b, head;     // batch row, KV head
 };
 
-template <bool MIXED = false>
-__device__ inline UnitInfo locate(const DecodeArgs& a, int x)
+template <int MODE = kModePlain>
+__device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* pg = nullptr)
 {
+    constexpr bool MIXED = MODE == kModeMixed;
     UnitInfo u;
     u.pos = tile_pos(a.sched, x);
     if (u.pos.uid < a.sched.U) {
@@ -276,6 +304,10 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x)
         u.len = a.len_comp;
         u.b = unit / a.n_comp;
         u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
+    }
+    if (MODE == kModePaged) {  // this sequence's own length
+        const int n = pg->seq_len[u.b];
+        u.len = u.pos.uid < a.sched.U ? n : (n < pg->cap ? n : pg->cap);
     }
     return u;
 }
@@ -326,8 +358,32 @@ struct AppendAllArgs {
 };
 cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream, bool overlap, bool mixed = false);
+                          int stages, int groups, cudaStream_t stream, bool overlap, int mode = kModePlain,
+                          const PagedArgs* paged = nullptr);
 cudaError_t prepare_decode_kernels(int head_dim);
-size_t decode_smem_bytes(int head_dim, int stages, int group, int groups);
+size_t decode_smem_bytes(int head_dim, int stages, int group, int groups, int mode = kModePlain);
+
+// Paged cache: one token for each of n sequences of one layer / n_tokens tokens of one sequence.
+// Entry i of k, v ([n][kv_heads][head_dim]) is token t[i] of request slot slot[i] (append) or token
+// t0 + i of request slot slot[0] (prefill); page[j] is the physical page of page index
+// first_page + j of the sequence (append: j = i, the page of token t[i]).  The kernel also records
+// the pages in the device page table.
+constexpr int kMaxAppendPages = 512;
+struct PagedAppendArgs {
+    __nv_bfloat16* pool;
+    int* page_table;
+    long long full_row0, comp_row0;
+    const int* slot_of_head;    // [kv_heads]: >= 0 full slot, < 0: -(comp slot + 1)
+    const __nv_bfloat16* k;
+    const __nv_bfloat16* v;
+    int n_full, n_comp, rows_comp, n_pages, table_stride;
+    int kv_heads, head_dim, sink, window;
+    int prefill;                // 0: n sequences, one token each; 1: one sequence, n tokens from t0
+    int n, t0, first_page;
+    int page[kMaxAppendPages];
+    int t[kMaxPagedBatch];
+    unsigned short slot[kMaxPagedBatch];
+};
+cudaError_t launch_paged_append(const PagedAppendArgs& a, cudaStream_t stream);
 
 }  // namespace rlkv

@@ -1,0 +1,518 @@
+// Host side of the paged, ragged cache of librlkv (rlkv_paged_* in include/rlkv.h): request slots
+// with their own lengths, full heads in 64-token pages handed out from one free list, compressed
+// heads in a constant-size ring per request slot (the serving layout of Section 4.3 of the paper:
+// a paged pool for the full heads beside a fixed-size pool for the compressed ones).
+//
+// Device buffer (sections 1024-byte aligned):
+//   pool        rows of head_dim bf16.  Per layer: the full-head region
+//               [n_full(layer)][n_pages][K|V][64][D] -- page p of a sequence is page p of every full
+//               head of every layer -- then the compressed-head region
+//               [max_seqs][n_comp(layer)][K|V][rows_comp][D]
+//   tables      int32 slot_of_head[layers][kv_heads]
+//   page table  int32 [max_seqs][table_stride]   (written by the append kernels)
+//   tickets     int32 [kMaxPagedBatch * kv_heads]
+//   status      int32 kernel status word, then the work-claim counter
+//   partials    float [max_slots][partial_floats]
+// Lengths, the page table's mirror and the free list live on the host.
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "rlkv_host.cuh"
+
+using namespace rlkv;
+
+struct rlkv_paged {
+    int layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, table_stride, sink, window;
+    int device, sm_count, stages, groups, item_tiles;
+    int rows_comp, max_batch, max_items, max_grid;
+    long long pool_rows;
+    std::vector<uint8_t> is_full;
+    std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
+    std::vector<int> n_full, n_comp;
+    std::vector<long long> full_row0, comp_row0;
+    std::vector<int> len;         // [layers][max_seqs]
+    std::vector<int> table;       // [max_seqs][table_stride], -1 = no page
+    std::vector<int> free_pages;  // stack of physical pages
+    std::vector<uint8_t> open;    // [max_seqs]
+    size_t off_pool, off_tables, off_page_table, off_tickets, off_status, off_partials, total;
+    unsigned int claims;
+    uint8_t* dev_base;
+    bool owns_buffer;
+    CUtensorMap tmap;
+    uint64_t launches;
+};
+
+namespace {
+
+constexpr int kPagedItemTiles = 8;
+
+int check_paged_shape(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                      int max_seq_len, const uint8_t* mask, int sink, int window)
+{
+    if (!mask || layers < 1 || kv_heads < 1 || kv_heads > kMaxKvHeads || q_heads < 1 || max_seqs < 1 ||
+        max_seqs > 65535 || n_pages < 1 || max_seq_len < 1)
+        return RLKV_EINVAL;
+    if (q_heads % kv_heads != 0 || q_heads / kv_heads > kMaxGroup) return RLKV_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return RLKV_EINVAL;
+    if (sink < 0 || window < 1 || (long long)sink + window > (1 << 24)) return RLKV_EINVAL;
+    if (max_seq_len > kMaxSeqPages * kTile) return RLKV_EINVAL;
+    return RLKV_OK;
+}
+
+// Fills the shape-dependent fields of `p` (no device work).
+int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
+{
+    p.table_stride = (int)align_up((size_t)(max_seq_len + kTile - 1) / kTile, 4);
+    p.rows_comp = (int)align_up((size_t)p.sink + p.window, kTile);
+    p.max_batch = p.max_seqs < kMaxPagedBatch ? p.max_seqs : kMaxPagedBatch;
+    p.max_grid = 2 * kMaxGridSms;
+    p.is_full.assign(mask, mask + (size_t)p.layers * p.kv_heads);
+    p.slot_of_head.assign((size_t)p.layers * p.kv_heads, 0);
+    p.head_of_slot.assign((size_t)p.layers * p.kv_heads, 0);
+    p.n_full.assign(p.layers, 0);
+    p.n_comp.assign(p.layers, 0);
+    p.full_row0.assign(p.layers, 0);
+    p.comp_row0.assign(p.layers, 0);
+    long long row = 0, most = 0;
+    for (int l = 0; l < p.layers; ++l) {
+        int nf = 0, nc = 0;
+        for (int h = 0; h < p.kv_heads; ++h)
+            if (mask[l * p.kv_heads + h]) p.slot_of_head[l * p.kv_heads + h] = nf++;
+            else p.slot_of_head[l * p.kv_heads + h] = -(++nc);
+        for (int h = 0; h < p.kv_heads; ++h) {
+            const int s = p.slot_of_head[l * p.kv_heads + h];
+            p.head_of_slot[l * p.kv_heads + (s >= 0 ? s : nf + (-s - 1))] = h;
+        }
+        p.n_full[l] = nf;
+        p.n_comp[l] = nc;
+        p.full_row0[l] = row;
+        row += (long long)nf * p.n_pages * 2 * kTile;
+        p.comp_row0[l] = row;
+        row += (long long)p.max_seqs * nc * 2 * p.rows_comp;
+        const long long t = (long long)p.max_batch * ((long long)nf * p.table_stride + (long long)nc * (p.rows_comp / kTile));
+        if (t >= (1ll << 31)) return RLKV_EINVAL;
+        const long long m = most_slots(p.max_batch * nf, p.table_stride, p.max_batch * nc, p.rows_comp / kTile, p.max_grid);
+        if (m > most) most = m;
+    }
+    if (row >= (1ll << 31) || most >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
+    p.pool_rows = row;
+    p.max_items = (int)most;
+    size_t off = 0;
+    p.off_pool = off;
+    off = align_up(off + (size_t)row * p.head_dim * 2, 1024);
+    p.off_tables = off;
+    off = align_up(off + (size_t)p.layers * p.kv_heads * sizeof(int), 1024);
+    p.off_page_table = off;
+    off = align_up(off + (size_t)p.max_seqs * p.table_stride * sizeof(int), 1024);
+    p.off_tickets = off;
+    off = align_up(off + (size_t)kMaxPagedBatch * p.kv_heads * sizeof(int), 1024);
+    p.off_status = off;
+    off = align_up(off + 64, 1024);
+    p.off_partials = off;
+    off = align_up(off + (size_t)p.max_items * partial_floats(p.head_dim, p.q_heads / p.kv_heads) * sizeof(float), 1024);
+    p.total = off;
+    return RLKV_OK;
+}
+
+template <typename T>
+T* dev_at(const rlkv_paged* p, size_t off) { return reinterpret_cast<T*>(p->dev_base + off); }
+
+bool valid_layer(const rlkv_paged* p, int layer) { return p && layer >= 0 && layer < p->layers; }
+bool valid_slot(const rlkv_paged* p, int slot) { return slot >= 0 && slot < p->max_seqs && p->open[slot]; }
+
+// The request slots of a call: all open, no slot twice.
+int check_slots(const rlkv_paged* p, const int* slots, int n)
+{
+    if (!slots || n < 1 || n > p->max_batch) return RLKV_EINVAL;
+    std::vector<uint8_t> seen(p->max_seqs, 0);
+    for (int i = 0; i < n; ++i) {
+        if (!valid_slot(p, slots[i]) || seen[slots[i]]) return RLKV_EINVAL;
+        seen[slots[i]] = 1;
+    }
+    return RLKV_OK;
+}
+
+int* len_of(rlkv_paged* p, int layer) { return p->len.data() + (size_t)layer * p->max_seqs; }
+const int* len_of(const rlkv_paged* p, int layer) { return p->len.data() + (size_t)layer * p->max_seqs; }
+
+void fill_append_args(rlkv_paged* p, int layer, const void* k, const void* v, PagedAppendArgs& a)
+{
+    a.pool = dev_at<__nv_bfloat16>(p, p->off_pool);
+    a.page_table = dev_at<int>(p, p->off_page_table);
+    a.full_row0 = p->full_row0[layer];
+    a.comp_row0 = p->comp_row0[layer];
+    a.slot_of_head = dev_at<int>(p, p->off_tables) + (size_t)layer * p->kv_heads;
+    a.k = static_cast<const __nv_bfloat16*>(k);
+    a.v = static_cast<const __nv_bfloat16*>(v);
+    a.n_full = p->n_full[layer];
+    a.n_comp = p->n_comp[layer];
+    a.rows_comp = p->rows_comp;
+    a.n_pages = p->n_pages;
+    a.table_stride = p->table_stride;
+    a.kv_heads = p->kv_heads;
+    a.head_dim = p->head_dim;
+    a.sink = p->sink;
+    a.window = p->window;
+}
+
+}  // namespace
+
+extern "C" {
+
+int rlkv_paged_size(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages, int max_seq_len,
+                    const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+{
+    if (!bytes_out) return RLKV_EINVAL;
+    int rc = check_paged_shape(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window);
+    if (rc) return rc;
+    rlkv_paged p{};
+    p.layers = layers; p.kv_heads = kv_heads; p.q_heads = q_heads; p.head_dim = head_dim;
+    p.max_seqs = max_seqs; p.n_pages = n_pages; p.sink = sink; p.window = window;
+    rc = make_paged_layout(p, head_is_full, max_seq_len);
+    if (rc) return rc;
+    *bytes_out = p.total;
+    return RLKV_OK;
+}
+
+int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                      int max_seq_len, const uint8_t* head_is_full, int sink, int window, void* device_buf,
+                      size_t device_buf_bytes)
+{
+    if (!out) return RLKV_EINVAL;
+    *out = nullptr;
+    int rc = check_paged_shape(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window);
+    if (rc) return rc;
+    rlkv_paged* p = new (std::nothrow) rlkv_paged();
+    if (!p) return RLKV_ENOMEM;
+    p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
+    p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window;
+    p->claims = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false;
+    rc = make_paged_layout(*p, head_is_full, max_seq_len);
+    if (rc) { delete p; return rc; }
+    p->len.assign((size_t)layers * max_seqs, 0);
+    p->table.assign((size_t)max_seqs * p->table_stride, -1);
+    p->open.assign(max_seqs, 0);
+    p->free_pages.resize(n_pages);
+    for (int i = 0; i < n_pages; ++i) p->free_pages[i] = n_pages - 1 - i;  // page 0 is handed out first
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    if (e != cudaSuccess) { delete p; return cuda_fail(e, "device query"); }
+    p->groups = 2;
+    p->item_tiles = kPagedItemTiles;
+    p->stages = max_stages(head_dim, q_heads / kv_heads, p->groups, 1, kModePaged);
+    if (p->stages < 2) { delete p; return RLKV_EINVAL; }
+    if (device_buf) {
+        if ((reinterpret_cast<uintptr_t>(device_buf) & 1023u) != 0 || device_buf_bytes < p->total) { delete p; return RLKV_ENOMEM; }
+        p->dev_base = static_cast<uint8_t*>(device_buf);
+    } else {
+        void* mem = nullptr;
+        e = cudaMalloc(&mem, p->total);
+        if (e != cudaSuccess) { cudaGetLastError(); delete p; return RLKV_ENOMEM; }
+        p->dev_base = static_cast<uint8_t*>(mem);
+        p->owns_buffer = true;
+    }
+    auto fail = [&](int code) {
+        if (p->owns_buffer) cudaFree(p->dev_base);
+        delete p;
+        return code;
+    };
+    // pools zero-filled (rows never written stay finite), tickets / status / counter start at zero
+    e = cudaMemset(p->dev_base + p->off_pool, 0, (size_t)p->pool_rows * head_dim * 2);
+    if (e == cudaSuccess) e = cudaMemset(p->dev_base + p->off_page_table, 0, p->off_partials - p->off_page_table);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->dev_base + p->off_tables, p->slot_of_head.data(), p->slot_of_head.size() * sizeof(int),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = prepare_decode_kernels(head_dim);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "rlkv_paged_create"));
+    rc = encode_pool_tensor_map(&p->tmap, p->dev_base + p->off_pool, p->pool_rows, head_dim);
+    if (rc) return fail(rc);
+    *out = p;
+    return RLKV_OK;
+}
+
+int rlkv_paged_destroy(rlkv_paged* p)
+{
+    if (!p) return RLKV_EINVAL;
+    DeviceGuard g(p->device);
+    cudaDeviceSynchronize();
+    if (p->owns_buffer) cudaFree(p->dev_base);
+    delete p;
+    return RLKV_OK;
+}
+
+int rlkv_paged_seq_open(rlkv_paged* p, int* slot_out)
+{
+    if (!p || !slot_out) return RLKV_EINVAL;
+    for (int s = 0; s < p->max_seqs; ++s)
+        if (!p->open[s]) {
+            p->open[s] = 1;
+            *slot_out = s;
+            return RLKV_OK;
+        }
+    return RLKV_EFULL;
+}
+
+int rlkv_paged_seq_close(rlkv_paged* p, int slot)
+{
+    if (!p || !valid_slot(p, slot)) return RLKV_EINVAL;
+    int* row = p->table.data() + (size_t)slot * p->table_stride;
+    for (int i = p->table_stride - 1; i >= 0; --i)
+        if (row[i] >= 0) {
+            p->free_pages.push_back(row[i]);
+            row[i] = -1;
+        }
+    for (int l = 0; l < p->layers; ++l) len_of(p, l)[slot] = 0;
+    p->open[slot] = 0;
+    return RLKV_OK;
+}
+
+int rlkv_paged_append(rlkv_paged* p, int layer, const int* slots, int n, const void* k, const void* v, void* stream)
+{
+    if (!valid_layer(p, layer) || !k || !v || !aligned16(k) || !aligned16(v)) return RLKV_EINVAL;
+    int rc = check_slots(p, slots, n);
+    if (rc) return rc;
+    int* len = len_of(p, layer);
+    // every sequence must have room and, where its token opens a page, a free page: checked before
+    // anything changes
+    int need = 0;
+    for (int i = 0; i < n; ++i) {
+        const int t = len[slots[i]];
+        if (t / kTile >= p->table_stride) return RLKV_EFULL;
+        if (p->table[(size_t)slots[i] * p->table_stride + t / kTile] < 0) ++need;
+    }
+    if (need > (int)p->free_pages.size()) return RLKV_EFULL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    PagedAppendArgs a;
+    fill_append_args(p, layer, k, v, a);
+    a.prefill = 0;
+    a.n = n;
+    a.t0 = 0;
+    a.first_page = 0;
+    for (int i = 0; i < n; ++i) {
+        const int s = slots[i], t = len[s];
+        int& entry = p->table[(size_t)s * p->table_stride + t / kTile];
+        if (entry < 0) {
+            entry = p->free_pages.back();
+            p->free_pages.pop_back();
+        }
+        a.slot[i] = (unsigned short)s;
+        a.t[i] = t;
+        a.page[i] = entry;
+    }
+    RLKV_CUDA(launch_paged_append(a, static_cast<cudaStream_t>(stream)));
+    for (int i = 0; i < n; ++i) len[slots[i]] += 1;
+    p->launches++;
+    return RLKV_OK;
+}
+
+int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const void* v, int n_tokens, void* stream)
+{
+    if (!valid_layer(p, layer) || !valid_slot(p, slot) || !k || !v || !aligned16(k) || !aligned16(v) || n_tokens < 1)
+        return RLKV_EINVAL;
+    int* len = len_of(p, layer);
+    const int t0 = len[slot];
+    if (((long long)t0 + n_tokens + kTile - 1) / kTile > p->table_stride) return RLKV_EFULL;
+    const int first = t0 / kTile, last = (t0 + n_tokens - 1) / kTile;
+    int* row = p->table.data() + (size_t)slot * p->table_stride;
+    int need = 0;
+    for (int i = first; i <= last; ++i)
+        if (row[i] < 0) ++need;
+    if (need > (int)p->free_pages.size()) return RLKV_EFULL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    for (int i = first; i <= last; ++i)
+        if (row[i] < 0) {
+            row[i] = p->free_pages.back();
+            p->free_pages.pop_back();
+        }
+    // launches of at most kMaxAppendPages pages each: every launch equals that many single appends,
+    // bit for bit, and the launches run in order, so the whole equals n_tokens single appends
+    const size_t row_elems = (size_t)p->kv_heads * p->head_dim;
+    for (int done = 0; done < n_tokens;) {
+        const int t = t0 + done;
+        const int page0 = t / kTile;
+        int count = n_tokens - done;
+        const int room = (page0 + kMaxAppendPages) * kTile - t;  // tokens up to the end of the last page the args can name
+        if (count > room) count = room;
+        PagedAppendArgs a;
+        fill_append_args(p, layer, static_cast<const __nv_bfloat16*>(k) + (size_t)done * row_elems,
+                         static_cast<const __nv_bfloat16*>(v) + (size_t)done * row_elems, a);
+        a.prefill = 1;
+        a.n = count;
+        a.t0 = t;
+        a.first_page = page0;
+        a.slot[0] = (unsigned short)slot;
+        for (int i = page0; i <= (t + count - 1) / kTile; ++i) a.page[i - page0] = row[i];
+        RLKV_CUDA(launch_paged_append(a, static_cast<cudaStream_t>(stream)));
+        p->launches++;
+        done += count;
+    }
+    len[slot] = t0 + n_tokens;
+    return RLKV_OK;
+}
+
+int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int n, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(p, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    int rc = check_slots(p, slots, n);
+    if (rc) return rc;
+    const int* len = len_of(p, layer);
+    int longest = 0;
+    for (int i = 0; i < n; ++i) {
+        if (len[slots[i]] < 1) return RLKV_EEMPTY;
+        if (len[slots[i]] > longest) longest = len[slots[i]];
+    }
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    const int cap = p->sink + p->window;
+    DecodeArgs a;
+    memset(&a, 0, sizeof a);
+    a.pool = dev_at<__nv_bfloat16>(p, p->off_pool);
+    a.full_row0 = p->full_row0[layer];
+    a.comp_row0 = p->comp_row0[layer];
+    for (int h = 0; h < p->kv_heads; ++h) a.head_of_slot[h] = (unsigned char)p->head_of_slot[(size_t)layer * p->kv_heads + h];
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.out = static_cast<float*>(out);
+    a.status = dev_at<int>(p, p->off_status);
+    a.trace = nullptr;
+    a.trace_on = 0;
+    a.n_full = p->n_full[layer];
+    a.n_comp = p->n_comp[layer];
+    a.rows_full = 0;
+    a.rows_comp = p->rows_comp;
+    a.len_full = longest;
+    a.len_comp = longest < cap ? longest : cap;
+    a.batch = n;
+    a.group = p->q_heads / p->kv_heads;
+    a.q_heads = p->q_heads;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)p->head_dim);
+    a.alpha = nullptr;
+    const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
+    // the tiles that exist (the schedule also spans the ones that do not) decide the item size
+    long long real_tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        const int t = len[slots[i]];
+        real_tiles += (long long)a.n_full * ((t + kTile - 1) / kTile) + (long long)a.n_comp * (((t < cap ? t : cap) + kTile - 1) / kTile);
+    }
+    int grid = p->sm_count;
+    if (grid > p->max_grid) grid = p->max_grid;
+    int item_tiles = (int)(real_tiles / grid);
+    if (item_tiles > p->item_tiles) item_tiles = p->item_tiles;
+    if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
+    a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
+    if (grid > a.sched.n_items) grid = a.sched.n_items;
+    if (a.sched.n_slots > p->max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
+    a.partials = dev_at<float>(p, p->off_partials);
+    a.tickets = dev_at<int>(p, p->off_tickets);
+    a.claim_counter = dev_at<unsigned int>(p, p->off_status) + 4;
+    a.claim_base = p->claims;
+    a.dep_wait = 0;
+    PagedArgs pa;
+    pa.page_table = dev_at<int>(p, p->off_page_table);
+    pa.table_stride = p->table_stride;
+    pa.n_pages = p->n_pages;
+    pa.cap = cap;
+    for (int i = 0; i < kMaxPagedBatch; ++i) {
+        pa.seq_len[i] = i < n ? len[slots[i]] : 0;
+        pa.seq_slot[i] = (unsigned short)(i < n ? slots[i] : 0);
+    }
+    RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, static_cast<cudaStream_t>(stream), false,
+                            kModePaged, &pa));
+    p->claims += (unsigned int)a.sched.n_items;
+    p->launches++;
+    return RLKV_OK;
+}
+
+int rlkv_paged_length(const rlkv_paged* p, int layer, int slot, int* len_out)
+{
+    if (!valid_layer(p, layer) || !valid_slot(p, slot) || !len_out) return RLKV_EINVAL;
+    *len_out = len_of(p, layer)[slot];
+    return RLKV_OK;
+}
+
+int rlkv_paged_pages(const rlkv_paged* p, int* free_out, int* total_out)
+{
+    if (!p || !free_out || !total_out) return RLKV_EINVAL;
+    *free_out = (int)p->free_pages.size();
+    *total_out = p->n_pages;
+    return RLKV_OK;
+}
+
+int rlkv_paged_step_bytes(const rlkv_paged* p, int layer, const int* slots, int n, uint64_t* kv_bytes_out)
+{
+    if (!valid_layer(p, layer) || !kv_bytes_out) return RLKV_EINVAL;
+    int rc = check_slots(p, slots, n);
+    if (rc) return rc;
+    const int cap = p->sink + p->window;
+    uint64_t rows = 0;
+    for (int i = 0; i < n; ++i) {
+        const int t = len_of(p, layer)[slots[i]];
+        rows += (uint64_t)p->n_full[layer] * t + (uint64_t)p->n_comp[layer] * (t < cap ? t : cap);
+    }
+    *kv_bytes_out = rows * 2 * p->head_dim * 2;
+    return RLKV_OK;
+}
+
+int rlkv_paged_debug_export_head(rlkv_paged* p, int layer, int slot, int kv_head, void* k_host, void* v_host,
+                                 int* rows_out, int32_t* token_of_slot_host)
+{
+    if (!valid_layer(p, layer) || !valid_slot(p, slot) || kv_head < 0 || kv_head >= p->kv_heads || !k_host || !v_host ||
+        !rows_out || !token_of_slot_host)
+        return RLKV_EINVAL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    RLKV_CUDA(cudaDeviceSynchronize());
+    const int n = len_of(p, layer)[slot], D = p->head_dim;
+    const int s = p->slot_of_head[(size_t)layer * p->kv_heads + kv_head];
+    const uint8_t* pool = p->dev_base + p->off_pool;
+    const size_t row_bytes = (size_t)D * 2;
+    if (s >= 0) {  // a full head: its n tokens in token order, page by page
+        for (int t0 = 0; t0 < n; t0 += kTile) {
+            const int page = p->table[(size_t)slot * p->table_stride + t0 / kTile];
+            if (page < 0) return RLKV_EKERNEL;
+            const int cnt = n - t0 < kTile ? n - t0 : kTile;
+            const long long krow = p->full_row0[layer] + ((long long)s * p->n_pages + page) * 2 * kTile;
+            RLKV_CUDA(cudaMemcpy(static_cast<uint8_t*>(k_host) + t0 * row_bytes, pool + krow * row_bytes, cnt * row_bytes,
+                                 cudaMemcpyDeviceToHost));
+            RLKV_CUDA(cudaMemcpy(static_cast<uint8_t*>(v_host) + t0 * row_bytes, pool + (krow + kTile) * row_bytes,
+                                 cnt * row_bytes, cudaMemcpyDeviceToHost));
+        }
+        for (int t = 0; t < n; ++t) token_of_slot_host[t] = t;
+        *rows_out = n;
+    } else {       // a compressed head: the physical ring
+        const int cap = p->sink + p->window;
+        const long long krow = p->comp_row0[layer] + ((long long)slot * p->n_comp[layer] + (-s - 1)) * 2 * p->rows_comp;
+        RLKV_CUDA(cudaMemcpy(k_host, pool + krow * row_bytes, cap * row_bytes, cudaMemcpyDeviceToHost));
+        RLKV_CUDA(cudaMemcpy(v_host, pool + (krow + p->rows_comp) * row_bytes, cap * row_bytes, cudaMemcpyDeviceToHost));
+        for (int r = 0; r < cap; ++r) {
+            int tok = -1;
+            if (r < p->sink) {
+                if (r < n) tok = r;
+            } else if (n > p->sink) {
+                // the newest token t >= sink with sink + (t - sink) % window == r
+                const int newest = n - 1, back = ((newest - p->sink) - (r - p->sink)) % p->window;
+                const int cand = newest - (back < 0 ? back + p->window : back);
+                if (cand >= p->sink) tok = cand;
+            }
+            token_of_slot_host[r] = tok;
+        }
+        *rows_out = cap;
+    }
+    return RLKV_OK;
+}
+
+int rlkv_paged_kernel_status(rlkv_paged* p, int* status_out)
+{
+    if (!p || !status_out) return RLKV_EINVAL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    RLKV_CUDA(cudaDeviceSynchronize());
+    RLKV_CUDA(cudaMemcpy(status_out, p->dev_base + p->off_status, sizeof(int), cudaMemcpyDeviceToHost));
+    return RLKV_OK;
+}
+
+}  // extern "C"

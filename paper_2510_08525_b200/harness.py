@@ -102,3 +102,58 @@ def step_inputs(w: synth.Workload, t: int, device):
     q = torch.stack([synth.rows(w.seed, synth.STREAM_Q, l, t, t + 1, w.batch, w.q_heads, w.head_dim, device)[0]
                      for l in range(w.layers)])
     return k.contiguous(), v.contiguous(), q.contiguous()
+
+
+class PagedCache:
+    """Owns an rlkv_paged handle (request slots with their own lengths, paged full heads)."""
+
+    def __init__(self, layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window,
+                 device="cuda:0"):
+        self.layers, self.kv_heads, self.q_heads, self.head_dim = layers, kv_heads, q_heads, head_dim
+        self.max_seqs, self.n_pages, self.max_seq_len, self.sink, self.window = max_seqs, n_pages, max_seq_len, sink, window
+        self.device = torch.device(device)
+        self.mask = np.asarray(head_is_full, dtype=np.uint8).reshape(layers, kv_heads)
+        with torch.cuda.device(self.device):
+            self.handle = rl.rlkv_paged_create(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
+                                               self.mask, sink, window)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            rl.rlkv_paged_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    def open_seq(self) -> int:
+        return rl.rlkv_paged_seq_open(self.handle)
+
+    def close_seq(self, slot) -> None:
+        rl.rlkv_paged_seq_close(self.handle, slot)
+
+    def append(self, layer, slots, k, v):
+        rl.rlkv_paged_append(self.handle, layer, slots, k, v)
+
+    def prefill(self, layer, slot, k, v):
+        rl.rlkv_paged_prefill(self.handle, layer, slot, k, v, k.shape[0])
+
+    def decode(self, layer, slots, q, out=None):
+        if out is None:
+            out = torch.empty((len(slots), self.q_heads, self.head_dim), dtype=torch.float32, device=self.device)
+        rl.rlkv_paged_decode_attention(self.handle, layer, slots, q, out)
+        return out
+
+    def length(self, layer, slot) -> int:
+        return rl.rlkv_paged_length(self.handle, layer, slot)
+
+    def pages(self):
+        return rl.rlkv_paged_pages(self.handle)
+
+    def step_bytes(self, layer, slots) -> int:
+        return rl.rlkv_paged_step_bytes(self.handle, layer, slots)
+
+    def export_head(self, layer, slot, head):
+        rows = max(self.max_seq_len, self.sink + self.window)
+        return rl.rlkv_paged_debug_export_head(self.handle, layer, slot, head, rows, self.head_dim)
+
+    def status(self) -> int:
+        return rl.rlkv_paged_kernel_status(self.handle)

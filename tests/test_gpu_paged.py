@@ -1,0 +1,227 @@
+"""GPU parity of the paged, ragged cache (rlkv_paged_*): every sequence must come out exactly as a
+batch row of its own would -- the oracle is one single-sequence oracle per request slot.  Cache
+state is compared bit for bit (full heads gathered page by page in token order, compressed heads as
+their physical ring), attention outputs within the bounds of the other parity tests.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle.rlkv_oracle import Oracle
+from test_gpu_parity import check_out, rand_bf16
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def rl(cuda_device):
+    import paper_2510_08525_b200.binding as binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def hz(cuda_device):
+    import paper_2510_08525_b200.harness as harness
+    return harness
+
+
+class Seq:
+    """One request: its slot in the cache under test and its own oracle."""
+
+    def __init__(self, cache, seed, max_len):
+        self.cache, self.seed = cache, seed
+        self.slot = cache.open_seq()
+        self.oracle = Oracle(cache.layers, cache.kv_heads, cache.q_heads, cache.head_dim, 1, max_len,
+                             cache.mask.reshape(-1), cache.sink, cache.window, threads=4)
+        self.n = 0
+
+    def rows(self, layer, t0, t1, what):
+        return rand_bf16((t1 - t0, self.cache.kv_heads, self.cache.head_dim),
+                         (self.seed * 131 + layer) * 100003 + t0 * 7 + what)
+
+    def prefill(self, n, dev):
+        for layer in range(self.cache.layers):
+            K, V = self.rows(layer, self.n, self.n + n, 0), self.rows(layer, self.n, self.n + n, 1)
+            self.cache.prefill(layer, self.slot, K.to(dev), V.to(dev))
+            for t in range(n):
+                assert self.oracle.append(layer, K[t], V[t]) == 0
+        self.n += n
+
+
+def append_all(cache, seqs, dev):
+    """One token for every sequence of `seqs`, every layer, in one call per layer."""
+    for layer in range(cache.layers):
+        ks = [s.rows(layer, s.n, s.n + 1, 0) for s in seqs]
+        vs = [s.rows(layer, s.n, s.n + 1, 1) for s in seqs]
+        cache.append(layer, [s.slot for s in seqs], torch.cat(ks).to(dev), torch.cat(vs).to(dev))
+        for s, k, v in zip(seqs, ks, vs):
+            assert s.oracle.append(layer, k[0], v[0]) == 0
+    for s in seqs:
+        s.n += 1
+
+
+def check_decode(cache, seqs, dev, seed, layers=None):
+    for layer in (range(cache.layers) if layers is None else layers):
+        q = rand_bf16((len(seqs), cache.q_heads, cache.head_dim), seed + layer)
+        out = cache.decode(layer, [s.slot for s in seqs], q.to(dev))
+        again = cache.decode(layer, [s.slot for s in seqs], q.to(dev))
+        assert torch.equal(out, again)                       # the same call, the same bits
+        out = out.cpu().numpy()
+        for i, s in enumerate(seqs):
+            check_out(out[i], s.oracle.decode(layer, q[i:i + 1])[0])
+
+
+def check_state(cache, seqs):
+    for s in seqs:
+        for layer in range(cache.layers):
+            assert cache.length(layer, s.slot) == s.oracle.length(layer) == s.n
+            for h in range(cache.kv_heads):
+                gk, gv, gt = cache.export_head(layer, s.slot, h)
+                ok, ov, ot = s.oracle.export_head(layer, 0, h)
+                rows = s.n if cache.mask[layer, h] else cache.sink + cache.window
+                assert len(gt) == rows
+                np.testing.assert_array_equal(gt, ot[:rows])
+                np.testing.assert_array_equal(gk, ok[:rows])
+                np.testing.assert_array_equal(gv, ov[:rows])
+
+
+SHAPES = [
+    # layers, Hkv, Hq, D, S, W, mask, lengths
+    (1, 2, 8, 64, 4, 60, "10", [1]),
+    (1, 2, 8, 64, 4, 60, "01", [63, 64, 65]),
+    (2, 2, 8, 64, 4, 12, "1001", [5, 200, 17, 129]),
+    (1, 4, 28, 128, 16, 112, "1001", [300, 1, 128, 1000, 77]),
+    (2, 8, 32, 128, 16, 112, "11011011" "00100001", [900, 64, 2500, 130]),
+    (1, 1, 8, 128, 0, 5, "0", [777, 3]),
+    (1, 2, 4, 128, 100, 200, "11", [1500, 299, 301]),
+    (1, 4, 16, 128, 16, 64, "0000", [400, 90]),
+]
+
+
+@pytest.mark.parametrize("layers,Hkv,Hq,D,S,W,mask,lens", SHAPES)
+def test_ragged_batch_matches_one_oracle_per_sequence(rl, hz, cuda_device, layers, Hkv, Hq, D, S, W, mask, lens):
+    mask = [int(c) for c in mask]
+    max_len = max(lens) + 8
+    pages = sum((n + 2 + 63) // 64 for n in lens) + 2
+    cache = hz.PagedCache(layers, Hkv, Hq, D, len(lens) + 1, pages, max_len, mask, S, W, device=cuda_device)
+    seqs = []
+    for i, n in enumerate(lens):
+        s = Seq(cache, i + 1, max_len)
+        if n > 1:
+            s.prefill(n - 1, cuda_device)
+        seqs.append(s)
+    append_all(cache, seqs, cuda_device)                     # the decode step's own token, for everyone
+    check_decode(cache, seqs, cuda_device, 500)
+    check_state(cache, seqs)
+    # a subset, in another order, after one more token for that subset only
+    sub = seqs[::-1][: max(1, len(seqs) // 2)]
+    append_all(cache, sub, cuda_device)
+    check_decode(cache, sub, cuda_device, 600)
+    check_state(cache, seqs)
+    want = sum(int(cache.mask[0].sum()) * s.n + int((1 - cache.mask[0]).sum()) * min(s.n, S + W) for s in sub) * 4 * D
+    assert cache.step_bytes(0, [s.slot for s in sub]) == want
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_continuous_batching_slots_and_pages_are_reused(rl, hz, cuda_device):
+    """Requests arrive, grow token by token across page boundaries, finish and hand their pages to
+    newcomers; every step is checked for the sequences alive at that moment."""
+    layers, Hkv, Hq, D, S, W = 2, 4, 16, 128, 8, 56
+    mask = [1, 0, 1, 1, 0, 1, 0, 0]
+    cache = hz.PagedCache(layers, Hkv, Hq, D, 4, 12, 400, mask, S, W, device=cuda_device)
+    assert cache.pages() == (12, 12)
+    a, b = Seq(cache, 1, 400), Seq(cache, 2, 400)
+    a.prefill(120, cuda_device)                              # 2 pages
+    b.prefill(190, cuda_device)                              # 3 pages
+    assert cache.pages() == (7, 12)
+    live = [a, b]
+    for step in range(12):                                   # a: 120 -> 132 (3rd page at 128), b: 190 -> 202 (4th at 192)
+        append_all(cache, live, cuda_device)
+        if step in (0, 7, 8, 11):
+            check_decode(cache, live, cuda_device, 700 + step)
+    assert cache.pages() == (5, 12)
+    check_state(cache, live)
+    # b finishes; c takes its slot and its pages
+    slot_b = b.slot
+    cache.close_seq(b.slot)
+    assert cache.pages() == (9, 12)
+    c = Seq(cache, 3, 400)
+    assert c.slot == slot_b
+    c.prefill(300, cuda_device)                              # 5 pages, four of them b's old ones
+    assert cache.pages() == (4, 12)
+    live = [c, a]
+    for step in range(5):
+        append_all(cache, live, cuda_device)
+    check_decode(cache, live, cuda_device, 800)
+    check_state(cache, live)
+    # the free list runs dry: refused, and nothing has changed for anybody
+    d = Seq(cache, 4, 400)
+    with pytest.raises(rl.RlkvError) as e:
+        d.cache.prefill(0, d.slot, rand_bf16((4 * 64 + 1, Hkv, D), 9).to(cuda_device),
+                        rand_bf16((4 * 64 + 1, Hkv, D), 10).to(cuda_device))
+    assert e.value.code == rl.RLKV_EFULL
+    assert cache.pages() == (4, 12) and cache.length(0, d.slot) == 0
+    check_decode(cache, live, cuda_device, 900)
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_paged_argument_checks(rl, hz, cuda_device):
+    Hkv, Hq, D = 2, 8, 64
+    cache = hz.PagedCache(1, Hkv, Hq, D, 2, 2, 128, [1, 0], 4, 12, device=cuda_device)
+    k = rand_bf16((2, Hkv, D), 1).to(cuda_device)
+    q = rand_bf16((2, Hq, D), 2).to(cuda_device)
+    out = torch.full((2, Hq, D), 3.0, dtype=torch.float32, device=cuda_device)
+    s0, s1 = cache.open_seq(), cache.open_seq()
+    with pytest.raises(rl.RlkvError) as e:                   # no third slot
+        cache.open_seq()
+    assert e.value.code == rl.RLKV_EFULL
+    for bad in ([s0, s0], [5], [-1], []):
+        with pytest.raises(rl.RlkvError) as e:
+            rl.rlkv_paged_append(cache.handle, 0, bad, k, k)
+        assert e.value.code == rl.RLKV_EINVAL
+    with pytest.raises(rl.RlkvError) as e:                   # nothing cached yet
+        rl.rlkv_paged_decode_attention(cache.handle, 0, [s0, s1], q, out)
+    assert e.value.code == rl.RLKV_EEMPTY
+    cache.append(0, [s0, s1], k, k)
+    assert cache.pages() == (0, 2)
+    cache.close_seq(s1)
+    with pytest.raises(rl.RlkvError) as e:                   # a closed slot
+        rl.rlkv_paged_append(cache.handle, 0, [s1], k, k)
+    assert e.value.code == rl.RLKV_EINVAL
+    for _ in range(127):
+        cache.append(0, [s0], k[:1], k[:1])
+    assert cache.length(0, s0) == 128
+    with pytest.raises(rl.RlkvError) as e:                   # at max_seq_len
+        cache.append(0, [s0], k[:1], k[:1])
+    assert e.value.code == rl.RLKV_EFULL
+    assert cache.length(0, s0) == 128
+    torch.cuda.synchronize()
+    assert (out == 3.0).all()
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_many_ragged_sequences_at_a_serving_shape(rl, hz, cuda_device):
+    """48 requests of 40 .. 5000 tokens over 8/32 heads of 128 with a mixed mask: sampled sequences
+    against their oracles (the long ones split over many work items, the short ones lie inside one)."""
+    layers, Hkv, Hq, D, S, W = 1, 8, 32, 128, 16, 112
+    mask = [1, 1, 0, 1, 1, 0, 1, 1]
+    rng = np.random.default_rng(3)
+    lens = [int(x) for x in rng.integers(40, 5000, size=48)]
+    lens[5], lens[17] = 64 * 70, 1
+    pages = sum((n + 63) // 64 for n in lens) + 4
+    cache = hz.PagedCache(layers, Hkv, Hq, D, 64, pages, 5200, mask, S, W, device=cuda_device)
+    seqs = []
+    for i, n in enumerate(lens):
+        s = Seq(cache, 50 + i, n + 2)
+        s.prefill(n, cuda_device)
+        seqs.append(s)
+    q = rand_bf16((len(seqs), Hq, D), 4242)
+    out = cache.decode(0, [s.slot for s in seqs], q.to(cuda_device)).cpu().numpy()
+    assert np.isfinite(out).all()
+    for i in [0, 5, 17, 23, 31, 47, int(np.argmax(lens)), int(np.argmin(lens))]:
+        check_out(out[i], seqs[i].oracle.decode(0, q[i:i + 1])[0])
+    assert cache.status() == 0
+    cache.close()
