@@ -65,6 +65,7 @@ def parse_args(argv=None):
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     p.add_argument("--no-mixed", action="store_true", help="skip the mixed-attention (Eq. 1) side measurement")
+    p.add_argument("--no-paged", action="store_true", help="skip the paged, ragged cache side measurement")
     return p.parse_args(argv)
 
 
@@ -440,6 +441,46 @@ def run_ours(args, w, mask):
         if mcache.status() != 0:
             raise SystemExit("a mixed-attention kernel reported a status: results are invalid")
         mcache.close()
+    # ---- side measurement: the paged, ragged cache on the first 4 layers of the workload's mask: the
+    # same batch once with every sequence at the workload's length and once with lengths spread from
+    # a quarter to seven quarters of it (same total), launches cycling through the layers
+    paged = None
+    if not args.no_paged and rank == 0:
+        pl, reps = min(4, w.layers), max(K, 8)
+        n = w.context + 1
+        pmask = mask[:pl * w.kv_heads]
+        spread = [max(1, int(round(n * (0.25 + 1.5 * i / max(1, w.batch - 1))))) for i in range(w.batch)]
+        paged = {"workload": f"first {pl} layers of the {w.name} mask, {w.batch} sequences, launches back to back"}
+        for name, lens in (("uniform", [n] * w.batch), ("ragged", spread)):
+            pages = sum((x + 63) // 64 for x in lens) + 2
+            pc = harness.PagedCache(pl, w.kv_heads, w.q_heads, w.head_dim, w.batch, pages, max(lens) + 64, pmask,
+                                    w.sink, w.window, device=dev)
+            slots = [pc.open_seq() for _ in lens]
+            for i, x in enumerate(lens):
+                for l in range(pl):
+                    for t0 in range(0, x, 4096):
+                        t1 = min(x, t0 + 4096)
+                        kk = synth.rows(w.seed + 1 + i, synth.STREAM_K, l, t0, t1, 1, w.kv_heads, w.head_dim, dev)
+                        vv = synth.rows(w.seed + 1 + i, synth.STREAM_V, l, t0, t1, 1, w.kv_heads, w.head_dim, dev)
+                        pc.prefill(l, slots[i], kk.reshape(t1 - t0, w.kv_heads, w.head_dim),
+                                   vv.reshape(t1 - t0, w.kv_heads, w.head_dim))
+            q = steps_in[0][2]
+            pout = torch.empty((pl, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
+            for i in range(2 * pl):
+                rl.rlkv_paged_decode_attention(pc.handle, i % pl, slots, q[i % pl], pout[i % pl], stream)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(reps * pl):
+                rl.rlkv_paged_decode_attention(pc.handle, i % pl, slots, q[i % pl], pout[i % pl], stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = 1e3 * e0.elapsed_time(e1) / (reps * pl)
+            nbytes = sum(pc.step_bytes(l, slots) for l in range(pl)) / pl
+            paged[name] = {"launch_us": us, "algorithmic_bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
+                           "lengths": [min(lens), max(lens)], "launches_timed": reps * pl}
+            if pc.status() != 0:
+                raise SystemExit("a paged decode kernel reported a status: results are invalid")
+            pc.close()
     clocks.__exit__()
     status = cache.status()
     if status != 0:
@@ -469,7 +510,7 @@ def run_ours(args, w, mask):
             "step_hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
             "bytes_ratio_vs_uncompressed": total_bytes / (w.batch * w.layers * w.kv_heads * (w.context + 1) * 4 * w.head_dim),
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
-            "mixed_attention": mixed,
+            "mixed_attention": mixed, "paged_cache": paged,
             "clocks": clocks.summary(clock_mark),
         }
         print(json.dumps(line), flush=True)
