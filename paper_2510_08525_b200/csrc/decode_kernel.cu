@@ -508,6 +508,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     int seg_eff = seg_tiles;  // tiles of the segment that exist
                     if (PAGED) {
                         seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
+                        if (seg_eff == 0) {  // nothing of this unit here: no tiles, no record
+                            x += seg_tiles;
+                            continue;
+                        }
                         // tiles left out shift the slot counter against x: skip the producer's empty slots
                         for (int pad = seg_eff > 0 ? ((x - cnt) % NG + NG) % NG : 0; alive && pad > 0; --pad, next_slot()) {
                             if (turn != grp) continue;
@@ -644,7 +648,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 }
                 if (warp == 0 && lane == 0) {
                     SegDesc* sd = reinterpret_cast<SegDesc*>(stat_l + S::kWarps * kMaxGroup);
-                    const bool complete = (u.pos.tile == 0 && seg_tiles == u.tiles);
+                    // the whole unit (paged cache: all of its tiles that exist) in one segment
+                    const bool complete = u.pos.tile == 0 && (PAGED ? seg_tiles >= (u.len + kTile - 1) / kTile
+                                                                    : seg_tiles == u.tiles);
                     sd->out_row = u.b * a.q_heads + u.head * G;
                     sd->uid = u.pos.uid;
                     sd->complete = complete ? 1 : 0;
@@ -933,7 +939,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 const int p = base + et, i = p >> 4, r = p & 15;
                 const bool on = p < pend_n * 16;
                 int slot = 0, count = 0;
-                if (on && r <= sc.R) unit_partials(sc, pend[i].x, r, slot, count);
+                if (on && r <= sc.R) {
+                    if (PAGED) unit_partials(sc, pend[i].x, r, slot, count, paged_unit_tiles(a, pg, pend[i].x));
+                    else unit_partials(sc, pend[i].x, r, slot, count);
+                }
                 int total = count;
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);

@@ -192,14 +192,18 @@ __host__ __device__ inline int partial_slot(const Schedule& s, int band, int ite
 
 // The partial records of unit `uid` in band `band`: first record and how many (0 if the unit has
 // no slice there).  Full units have a slice in every band, compressed units only in the last.
-__host__ __device__ inline void unit_partials(const Schedule& s, int uid, int band, int& slot, int& count)
+// `tiles`: how many of the unit's tiles exist (paged cache: a sequence shorter than the longest one
+// of the call); segments that hold none of them deliver no record.
+__host__ __device__ inline void unit_partials(const Schedule& s, int uid, int band, int& slot, int& count,
+                                              int tiles = 0x7fffffff)
 {
     int first, width;
     if (uid < s.U) {
         width = s.tb[band + 1] - s.tb[band];
         first = s.base[band] + uid * width;
+        if (width > tiles - s.tb[band]) width = tiles - s.tb[band];
     } else {
-        width = band == s.R ? s.tc : 0;
+        width = band == s.R ? (s.tc < tiles ? s.tc : tiles) : 0;
         first = s.base[s.R + 1] + (uid - s.U) * s.tc;
     }
     if (width <= 0) {
@@ -310,6 +314,19 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.len = u.pos.uid < a.sched.U ? n : (n < pg->cap ? n : pg->cap);
     }
     return u;
+}
+
+// Paged cache: how many tiles of unit `uid` exist.
+__device__ inline int paged_unit_tiles(const DecodeArgs& a, const PagedArgs* pg, int uid)
+{
+    int n;
+    if (uid < a.sched.U) {
+        n = pg->seq_len[uid / a.n_full];
+    } else {
+        n = pg->seq_len[(uid - a.sched.U) / a.n_comp];
+        if (n > pg->cap) n = pg->cap;
+    }
+    return (n + kTile - 1) / kTile;
 }
 
 // Mixed attention: tile `tile` of a local unit holds rows [row, row + valid) of its head; what
