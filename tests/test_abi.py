@@ -98,3 +98,31 @@ def test_package_fails_loudly_without_the_library(tmp_path):
             "try:\n    p.rlkv_cache_size\nexcept ImportError as e:\n    print('IMPORTERROR', 'no fallback' in str(e))\n")
     res = subprocess.run([sys.executable, "-c", code], cwd=tmp_path, capture_output=True, text=True)
     assert "IMPORTERROR True" in res.stdout, res.stdout + res.stderr
+
+
+def test_paged_size_and_argument_checks_need_no_device(binding):
+    """rlkv_paged_size is host arithmetic: the page pool grows with n_pages and with the number of
+    full heads only, the ring pool with max_seqs and the number of compressed heads only, and
+    neither with max_seq_len (beyond the page table)."""
+    ok = dict(layers=2, kv_heads=2, q_heads=8, head_dim=128, max_seqs=3, n_pages=10, max_seq_len=1000,
+              head_is_full=[1, 0, 0, 1], sink=4, window=60)
+    size = binding.rlkv_paged_size(**ok)
+    page_bytes = 2 * 64 * 128 * 2                       # K and V rows of one page of one full head
+    ring_bytes = 2 * 64 * 128 * 2                       # sink + window = 64 rows, K and V
+    assert size >= 2 * (10 * page_bytes + 3 * ring_bytes)
+    more_pages = binding.rlkv_paged_size(**{**ok, "n_pages": 10 + 1000})
+    assert more_pages - size == 2 * 1000 * page_bytes   # one full head per layer
+    # request slots beyond the 256 a launch can serve cost their rings and page-table rows, no scratch
+    a, b = (binding.rlkv_paged_size(**{**ok, "max_seqs": m}) for m in (300, 300 + 256))
+    assert b - a == 2 * 256 * ring_bytes + 256 * 16 * 4     # 1000 tokens = 16 page-table entries
+    for bad in (dict(head_dim=96), dict(q_heads=7), dict(window=0), dict(sink=-1), dict(max_seqs=0), dict(n_pages=0),
+                dict(max_seq_len=0), dict(max_seq_len=65537), dict(max_seqs=70000)):
+        with pytest.raises(binding.RlkvError) as e:
+            binding.rlkv_paged_size(**{**ok, **bad})
+        assert e.value.code == binding.RLKV_EINVAL
+    for call in (lambda: binding.rlkv_paged_seq_open(0), lambda: binding.rlkv_paged_seq_close(0, 0),
+                 lambda: binding.rlkv_paged_pages(0), lambda: binding.rlkv_paged_length(0, 0, 0),
+                 lambda: binding.rlkv_paged_destroy(0)):
+        with pytest.raises(binding.RlkvError) as e:
+            call()
+        assert e.value.code == binding.RLKV_EINVAL
