@@ -407,7 +407,7 @@ def run_ours(args, w, mask):
     # ---- side measurement: mixed attention (Eq. 1) on a 4-layer all-full cache of the same shape.  Every
     # layer's K/V rows exceed the L2 and the launches cycle through the layers, so each launch reads from HBM.
     mixed = None
-    if not args.no_mixed and rank == 0:
+    if not args.no_mixed and world == 1:
         ml, reps = 4, max(K, 8)
         n = w.context + 1
         mw = w.with_(layers=ml, frac_compressed=0.0)
@@ -445,7 +445,7 @@ def run_ours(args, w, mask):
     # same batch once with every sequence at the workload's length and once with lengths spread from
     # a quarter to seven quarters of it (same total), launches cycling through the layers
     paged = None
-    if not args.no_paged and rank == 0:
+    if not args.no_paged and world == 1:
         pl, reps = min(4, w.layers), max(K, 8)
         n = w.context + 1
         pmask = mask[:pl * w.kv_heads]

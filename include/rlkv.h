@@ -216,6 +216,18 @@ int rlkv_paged_step_bytes(const rlkv_paged* cache, int layer, const int* slots, 
 int rlkv_paged_debug_export_head(rlkv_paged* cache, int layer, int slot, int kv_head, void* k_host,
                                  void* v_host, int* rows_out, int32_t* token_of_slot_host);
 int rlkv_paged_kernel_status(rlkv_paged* cache, int* status_out);
+/* The split bookkeeping of a paged decode launch, host arithmetic only (no GPU): n sequences of
+ * lens[i] tokens (host int[n]) over n_full full and n_comp compressed heads, cap = sink + window,
+ * cut for `ctas` CTAs into work items of at least item_tiles tiles.  For every unit (sequence i,
+ * head slot f: index i * n_full + f; then the compressed units, i * n_comp + c after all full ones)
+ * delivered_out counts the partial records the kernel's walk over the work items delivers,
+ * expected_out the number its tickets wait for, complete_out the segments that hold the whole unit
+ * and write its result directly (host int[n * (n_full + n_comp)] each).  A unit is served
+ * correctly iff complete == 1 and delivered == 0, or complete == 0 and delivered == expected >= 1.
+ * RLKV_EKERNEL if two segments of a unit would share a partial record. */
+int rlkv_debug_paged_schedule(const int* lens, int n, int n_full, int n_comp, int cap, int ctas,
+                              int item_tiles, int* n_items_out, int* delivered_out,
+                              int* expected_out, int* complete_out);
 
 /* ---- introspection (host-side bookkeeping; no GPU work unless stated) ---- */
 int rlkv_length(const rlkv_cache* cache, int layer, int* len_out);

@@ -56,6 +56,7 @@ SIGNATURES = {
     "rlkv_paged_step_bytes": (_ci, [_vp, _ci, _vp, _ci, ctypes.POINTER(ctypes.c_uint64)]),
     "rlkv_paged_debug_export_head": (_ci, [_vp, _ci, _ci, _ci, _vp, _vp, ctypes.POINTER(_ci), _vp]),
     "rlkv_paged_kernel_status": (_ci, [_vp, ctypes.POINTER(_ci)]),
+    "rlkv_debug_paged_schedule": (_ci, [_vp, _ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), _vp, _vp, _vp]),
 }
 
 
@@ -340,3 +341,15 @@ def rlkv_paged_kernel_status(cache) -> int:
     out = _ci(0)
     _check(lib.rlkv_paged_kernel_status(cache, ctypes.byref(out)))
     return int(out.value)
+
+
+def rlkv_debug_paged_schedule(lens, n_full, n_comp, cap, ctas, item_tiles):
+    """Returns (n_items, delivered, expected, complete), the last three int32 arrays per unit."""
+    ln = _slots(lens)
+    units = ln.size * (n_full + n_comp)
+    delivered, expected, complete = (np.zeros(units, dtype=np.int32) for _ in range(3))
+    n_items = _ci(0)
+    _check(lib.rlkv_debug_paged_schedule(ln.ctypes.data, ln.size, n_full, n_comp, cap, ctas, item_tiles,
+                                         ctypes.byref(n_items), delivered.ctypes.data, expected.ctypes.data,
+                                         complete.ctypes.data))
+    return int(n_items.value), delivered, expected, complete

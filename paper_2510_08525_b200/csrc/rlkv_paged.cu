@@ -505,6 +505,61 @@ int rlkv_paged_debug_export_head(rlkv_paged* p, int layer, int slot, int kv_head
     return RLKV_OK;
 }
 
+int rlkv_debug_paged_schedule(const int* lens, int n, int n_full, int n_comp, int cap, int ctas, int item_tiles,
+                              int* n_items_out, int* delivered_out, int* expected_out, int* complete_out)
+{
+    if (!lens || n < 1 || n > kMaxPagedBatch || n_full < 0 || n_comp < 0 || n_full + n_comp < 1 || cap < 1 || ctas < 1 ||
+        item_tiles < 1 || !n_items_out || !delivered_out || !expected_out || !complete_out)
+        return RLKV_EINVAL;
+    int longest = 0;
+    for (int i = 0; i < n; ++i) {
+        if (lens[i] < 1) return RLKV_EINVAL;
+        if (lens[i] > longest) longest = lens[i];
+    }
+    const int tf = (longest + kTile - 1) / kTile, tc = ((longest < cap ? longest : cap) + kTile - 1) / kTile;
+    const Schedule sc = make_schedule(n * n_full, tf, n * n_comp, tc, ctas, item_tiles);
+    const int units = n * (n_full + n_comp);
+    auto unit_tiles = [&](int uid) {  // tiles of the unit that exist
+        int len = uid < sc.U ? lens[uid / n_full] : lens[(uid - sc.U) / n_comp];
+        if (uid >= sc.U && len > cap) len = cap;
+        return (len + kTile - 1) / kTile;
+    };
+    std::vector<int> last_slot(units, -1);
+    for (int u = 0; u < units; ++u) delivered_out[u] = complete_out[u] = 0;
+    // what the kernel does: walk every work item segment by segment
+    for (int k = 0; k < sc.n_items; ++k) {
+        const int x1 = item_start(sc, k + 1);
+        for (int x = item_start(sc, k); x < x1;) {
+            const TilePos pos = tile_pos(sc, x);
+            const int seg_tiles = x1 - x < pos.run ? x1 - x : pos.run;
+            const int exist = unit_tiles(pos.uid) - pos.tile;
+            if (exist > 0) {
+                if (pos.tile == 0 && seg_tiles >= unit_tiles(pos.uid)) {
+                    complete_out[pos.uid]++;
+                } else {
+                    const int slot = partial_slot(sc, pos.band, k, pos.uid);
+                    if (slot < 0 || slot >= sc.n_slots || slot <= last_slot[pos.uid]) return RLKV_EKERNEL;
+                    last_slot[pos.uid] = slot;
+                    delivered_out[pos.uid]++;
+                }
+            }
+            x += seg_tiles;
+        }
+    }
+    // what the tickets expect: the records of every band, clipped to the tiles that exist
+    for (int u = 0; u < units; ++u) {
+        int total = 0;
+        for (int r = 0; r <= sc.R; ++r) {
+            int slot = 0, count = 0;
+            unit_partials(sc, u, r, slot, count, unit_tiles(u));
+            total += count;
+        }
+        expected_out[u] = total;
+    }
+    *n_items_out = sc.n_items;
+    return RLKV_OK;
+}
+
 int rlkv_paged_kernel_status(rlkv_paged* p, int* status_out)
 {
     if (!p || !status_out) return RLKV_EINVAL;

@@ -95,6 +95,7 @@ SHAPES = [
     (1, 1, 8, 128, 0, 5, "0", [777, 3]),
     (1, 2, 4, 128, 100, 200, "11", [1500, 299, 301]),
     (1, 4, 16, 128, 16, 64, "0000", [400, 90]),
+    (1, 2, 4, 64, 16, 112, "10", [40000, 100]),   # 625 pages: the prompt goes in over two prefill launches
 ]
 
 

@@ -80,3 +80,35 @@ def test_schedule_rejects_bad_arguments(rl):
         with pytest.raises(rl.RlkvError) as e:
             rl.rlkv_debug_schedule(*bad)
         assert e.value.code == rl.RLKV_EINVAL
+
+
+def test_paged_launch_tickets_match_the_segments_that_exist():
+    """Paged cache: sequences shorter than the longest one of a call own only the first tiles of
+    their (uniformly sized) units.  Whatever the lengths, grid and item size, every unit must either
+    be written directly by the one segment that holds all of its tiles, or receive exactly as many
+    partial records as its tickets wait for -- otherwise its merge would never run, or run early."""
+    import paper_2510_08525_b200.binding as rl
+    rng = np.random.default_rng(11)
+    cases = 0
+    for trial in range(300):
+        n = int(rng.integers(1, 40))
+        hi = int(rng.choice([70, 700, 5000, 40000]))
+        lens = rng.integers(1, hi + 1, size=n)
+        if trial % 3 == 0:
+            lens[rng.integers(n)] = hi                      # one long sequence beside short ones
+        if trial % 7 == 0:
+            lens[:] = int(lens[0])                          # a uniform batch
+        n_full, n_comp = int(rng.integers(0, 5)), int(rng.integers(0, 4))
+        if n_full + n_comp == 0:
+            n_full = 1
+        cap = int(rng.choice([5, 64, 128, 200, 384]))
+        ctas = int(rng.choice([1, 7, 148, 160]))
+        item_tiles = int(rng.choice([2, 3, 8, 32]))
+        n_items, delivered, expected, complete = rl.rlkv_debug_paged_schedule(lens, n_full, n_comp, cap, ctas, item_tiles)
+        assert n_items >= 1
+        direct = complete == 1
+        assert ((complete == 0) | direct).all()
+        assert (delivered[direct] == 0).all()
+        assert (delivered[~direct] == expected[~direct]).all() and (delivered[~direct] >= 1).all()
+        cases += len(delivered)
+    assert cases > 10000
