@@ -22,6 +22,10 @@
 // merges of split units run on all warps once the CTA's stream has ended.
 // The decode launches of one step overlap on the device (programmatic dependent launch): see the
 // kernel's first lines and launch_decode.
+// The kernel is compiled in three modes: the lock-step cache (above), mixed attention with gating
+// adapters (paper, Eq. 1: a second class of "local" units over the sink and window rows, both
+// classes adding their weighted result), and the paged cache (one length per sequence, full-head
+// rows looked up in a page table); see the notes above decode_kernel.
 #include "rlkv_internal.cuh"
 
 namespace rlkv {

@@ -15,7 +15,7 @@
 //             launches of a step alternate between them)
 //   partials  float [2][max_slots][partial_floats]  (split-KV scratch; the two halves alternate too)
 //   staging   k, v, q (twice: calls alternate) and out of one whole step, for rlkv_step_host
-//   trace     uint64 [max_grid][8]  (debug trace of the decode kernel)
+//   trace     uint64 [max_grid][40]  (debug trace of the decode kernel)
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
