@@ -138,6 +138,13 @@ size_t rlkv_static_scratch_bytes(void);
 int rlkv_decode_mixed_attention(rlkv_cache* cache, int layer, const void* q, const float* alpha,
                                 void* out, void* stream);
 
+/* Output element type of rlkv_decode_attention, rlkv_decode_attention_static_scratch, rlkv_step and
+ * rlkv_step_host from now on: on != 0 stores results as bf16 (the fp32 result rounded to nearest
+ * even when it is stored; `out` buffers then hold bf16 elements of the same shape, half the bytes),
+ * on == 0 (the default) as fp32.  The arithmetic does not change.  rlkv_decode_mixed_attention adds
+ * its two branches up in the fp32 output buffer and returns RLKV_EINVAL while bf16 output is on. */
+int rlkv_set_output_bf16(rlkv_cache* cache, int on);
+
 /* One whole decode step: for every layer, append then attend.  Device buffers:
  * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];
  * out fp32 [layers][batch][q_heads][head_dim].  The results are those of the per-layer calls in
@@ -203,6 +210,8 @@ int rlkv_paged_prefill(rlkv_paged* cache, int layer, int slot, const void* k, co
  * sequence holds no token in this layer. */
 int rlkv_paged_decode_attention(rlkv_paged* cache, int layer, const int* slots, int n,
                                 const void* q, void* out, void* stream);
+/* As rlkv_set_output_bf16, for rlkv_paged_decode_attention. */
+int rlkv_paged_set_output_bf16(rlkv_paged* cache, int on);
 int rlkv_paged_length(const rlkv_paged* cache, int layer, int slot, int* len_out);
 /* Pages on the free list and pages in total. */
 int rlkv_paged_pages(const rlkv_paged* cache, int* free_out, int* total_out);

@@ -31,6 +31,8 @@ SIGNATURES = {
     "rlkv_decode_attention": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_decode_attention_static_scratch": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_static_scratch_bytes": (_sz, []),
+    "rlkv_set_output_bf16": (_ci, [_vp, _ci]),
+    "rlkv_paged_set_output_bf16": (_ci, [_vp, _ci]),
     "rlkv_decode_mixed_attention": (_ci, [_vp, _ci, _vp, _vp, _vp, _vp]),
     "rlkv_step": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_step_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
@@ -170,6 +172,14 @@ def rlkv_decode_mixed_attention(cache, layer, q, alpha, out, stream=None) -> Non
     """Eq. 1: alpha[h] * full attention + (1 - alpha[h]) * sink+window attention over a layer whose
     heads are all full.  alpha: device fp32 [kv_heads]."""
     _check(lib.rlkv_decode_mixed_attention(cache, layer, _ptr(q), _ptr(alpha), _ptr(out), _stream(stream)))
+
+
+def rlkv_set_output_bf16(cache, on) -> None:
+    _check(lib.rlkv_set_output_bf16(cache, int(bool(on))))
+
+
+def rlkv_paged_set_output_bf16(cache, on) -> None:
+    _check(lib.rlkv_paged_set_output_bf16(cache, int(bool(on))))
 
 
 def rlkv_step(cache, k, v, q, out, stream=None) -> None:

@@ -260,7 +260,7 @@ struct Smem {
 template <int D, bool MIXED>
 __device__ __noinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
                                          const int2* lists, int n, int t, int nt, bool dry,
-                                         unsigned long long* stamp, const float* alpha, int U, int q_heads)
+                                         unsigned long long* stamp, const float* alpha, int U, int q_heads, int out_bf16)
 {
     constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
     const int E = G * D4;
@@ -330,9 +330,14 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
                         atomicAdd(o + 2, O.z * inv);
                         atomicAdd(o + 3, O.w * inv);
                     }
-                } else if (!dry)
-                    *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
-                        make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                } else if (!dry) {
+                    if (out_bf16)
+                        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)units[j].y * D + e * 4) =
+                            make_uint2(pack_bf16(O.x * inv, O.y * inv), pack_bf16(O.z * inv, O.w * inv));
+                    else
+                        *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
+                            make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                }
             }
         }
     }
@@ -915,7 +920,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         }
         epilogue_sync();
         merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1,
-                              et, NE, true, nullptr, a.alpha, sc.U, a.q_heads);
+                              et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
         epilogue_sync();
         if (a.dep_wait) {  // from here on these warps write results, partials and tickets
             grid_dep_wait();
@@ -932,7 +937,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             epilogue_sync();
             if (*todo_count + pend_n > kMaxTodo) {
                 merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, et, NE, false, nullptr, a.alpha,
-                                      sc.U, a.q_heads);
+                                      sc.U, a.q_heads, a.out_bf16);
                 epilogue_sync();
                 if (et == 0) *todo_count = 0;
                 epilogue_sync();
@@ -1018,7 +1023,11 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     atomicAdd(out_rows + e * 4 + 3, O.w * inv);
                 } else if (sd.complete) {
                     const float inv = 1.f / L;
-                    *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                    if (a.out_bf16)
+                        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.out) + (size_t)sd.out_row * D + e * 4) =
+                            make_uint2(pack_bf16(O.x * inv, O.y * inv), pack_bf16(O.z * inv, O.w * inv));
+                    else
+                        *reinterpret_cast<float4*>(out_rows + e * 4) = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
                 } else {
                     *reinterpret_cast<float4*>(my_part + PH + e * 4) = O;
                     if (d4 == 0) {
@@ -1045,7 +1054,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (trace && tid == 0) my_trace[13] = (unsigned long long)*todo_count;
     if (!*s_abort && *todo_count > 0)
         merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo, lists, *todo_count, tid, S::kThreads, false,
-                              trace ? my_trace + 28 : nullptr, a.alpha, sc.U, a.q_heads);
+                              trace ? my_trace + 28 : nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
     if (warp == S::kWarps && lane == 0) {
         if (*s_abort) {
             // a wait ran out somewhere in this CTA: make sure none of its copies is still in flight

@@ -138,6 +138,7 @@ struct rlkv_cache {
     int ctas_per_sm, stages, groups, item_tiles;  // decode launch shape (rlkv_set_decode_config)
     int item_tiles_alone;                         // item_tiles of launches outside rlkv_step
     int trace_on;
+    int out_bf16;            // results are stored as bf16 instead of fp32 (rlkv_set_output_bf16)
     unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
     cudaStream_t in_stream, out_stream;  // rlkv_step_host: copies that run beside the kernels
     cudaEvent_t ev_step[2], ev_done;     // kernels of a call done with staging copy p / results copied out
@@ -252,6 +253,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     if (all_tiles >= (1ll << 31)) return RLKV_EINVAL;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
     a.trace_on = c->trace_on;
+    a.out_bf16 = c->out_bf16;
     // persistent grid; the work items of the flat tile space are cut for that many CTAs and no
     // more CTAs are launched than there are items
     int grid = c->sm_count * c->ctas_per_sm;
@@ -390,7 +392,8 @@ int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStr
         int grid = 0;
         const bool overlap = prev_ok;
         int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                           static_cast<float*>(out) + l * q_layer, s, l & 1, overlap, overlap && l == 0, &grid);
+                           static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, overlap,
+                           overlap && l == 0, &grid);
         if (rc) return rc;
         prev_ok = (grid == c->sm_count && c->ctas_per_sm == 1);
     }
@@ -447,6 +450,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->item_tiles = kDefaultItemTiles;
     c->item_tiles_alone = kDefaultItemTilesAlone;
     c->trace_on = 0;
+    c->out_bf16 = 0;
     c->claims[0] = c->claims[1] = 0;
     c->in_stream = c->out_stream = nullptr;
     c->ev_step[0] = c->ev_step[1] = c->ev_done = nullptr;
@@ -617,11 +621,19 @@ int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q
 
 size_t rlkv_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
+int rlkv_set_output_bf16(rlkv_cache* c, int on)
+{
+    if (!c) return RLKV_EINVAL;
+    c->out_bf16 = on ? 1 : 0;
+    return RLKV_OK;
+}
+
 int rlkv_decode_mixed_attention(rlkv_cache* c, int layer, const void* q, const float* alpha, void* out, void* stream)
 {
     if (!valid_layer(c, layer) || !q || !alpha || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
     if ((reinterpret_cast<uintptr_t>(alpha) & 3u) != 0) return RLKV_EINVAL;
     if (c->lay.n_comp[layer] != 0) return RLKV_EINVAL;  // the full branch needs every token of every head
+    if (c->out_bf16) return RLKV_EINVAL;                // the two branches are added up in fp32
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
@@ -649,7 +661,7 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
                            static_cast<const __nv_bfloat16*>(v) + l * kv_layer, 1, s);
         if (rc) return rc;
         rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                       static_cast<float*>(out) + l * q_layer, s);
+                       static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s);
         if (rc) return rc;
     }
     return RLKV_OK;
@@ -677,7 +689,7 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
         RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
         int rc = rlkv_step(c, dk, dv, dq, dout, stream);
         if (rc) return rc;
-        RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * 2, cudaMemcpyDeviceToHost, s));
+        RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * (c->out_bf16 ? 1 : 2), cudaMemcpyDeviceToHost, s));
         return RLKV_OK;
     }
     // Inputs come in on one side stream, results go out on another, both beside the kernels on the
@@ -715,7 +727,8 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
         if (rc) return rc;
         RLKV_CUDA(cudaEventRecord(c->ev_out[i], s));
         // results of the chunk
-        const size_t o = 2 * q_layer * bounds[i], n = 2 * q_layer * (bounds[i + 1] - bounds[i]);
+        const size_t ob = c->out_bf16 ? 1 : 2;  // bytes of a result element / bytes of a query element
+        const size_t o = ob * q_layer * bounds[i], n = ob * q_layer * (bounds[i + 1] - bounds[i]);
         RLKV_CUDA(cudaStreamWaitEvent(c->out_stream, c->ev_out[i], 0));
         RLKV_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(out_host) + o, dout + o, n, cudaMemcpyDeviceToHost,
                                   c->out_stream));

@@ -222,7 +222,7 @@ struct DecodeArgs {
     long long full_row0;        // first pool row of the layer's full-head region
     long long comp_row0;        // first pool row of the layer's compressed-head region
     const __nv_bfloat16* q;     // [batch][q_heads][head_dim]
-    float* out;                 // [batch][q_heads][head_dim]
+    float* out;                 // [batch][q_heads][head_dim]; bf16 elements instead of fp32 if out_bf16
     float* partials;            // [sched.n_slots][partial_floats]
     int* tickets;               // one per unit of this layer, zero between launches
     unsigned int* claim_counter;  // items claimed beyond the first P, over all launches so far (never reset)
@@ -237,6 +237,7 @@ struct DecodeArgs {
     int batch, group, q_heads;
     float scale_log2;           // log2(e) / sqrt(head_dim)
     int trace_on;
+    int out_bf16;               // results are rounded to bf16 (nearest even) when they are stored
     // Mixed attention (paper, Eq. 1; MIXED kernels only).  Every head of the layer is full; beside
     // the FULL unit of each (batch row, head) the schedule's second class holds a LOCAL unit over
     // the same rows restricted to the sink and the window: tiles 0 .. local_sink_tiles-1 cover rows

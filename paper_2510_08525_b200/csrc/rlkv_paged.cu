@@ -28,6 +28,7 @@ struct rlkv_paged {
     int layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, table_stride, sink, window;
     int device, sm_count, stages, groups, item_tiles;
     int rows_comp, max_batch, max_items, max_grid;
+    int out_bf16;
     long long pool_rows;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -189,7 +190,7 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
     if (!p) return RLKV_ENOMEM;
     p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
     p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window;
-    p->claims = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false;
+    p->claims = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
     rc = make_paged_layout(*p, head_is_full, max_seq_len);
     if (rc) { delete p; return rc; }
     p->len.assign((size_t)layers * max_seqs, 0);
@@ -391,6 +392,7 @@ int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int 
     a.q_heads = p->q_heads;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)p->head_dim);
     a.alpha = nullptr;
+    a.out_bf16 = p->out_bf16;
     const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
     // the tiles that exist (the schedule also spans the ones that do not) decide the item size
     long long real_tiles = 0;
@@ -424,6 +426,13 @@ int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int 
                             kModePaged, &pa));
     p->claims += (unsigned int)a.sched.n_items;
     p->launches++;
+    return RLKV_OK;
+}
+
+int rlkv_paged_set_output_bf16(rlkv_paged* p, int on)
+{
+    if (!p) return RLKV_EINVAL;
+    p->out_bf16 = on ? 1 : 0;
     return RLKV_OK;
 }
 

@@ -226,3 +226,22 @@ def test_many_ragged_sequences_at_a_serving_shape(rl, hz, cuda_device):
         check_out(out[i], seqs[i].oracle.decode(0, q[i:i + 1])[0])
     assert cache.status() == 0
     cache.close()
+
+
+def test_paged_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
+    Hkv, Hq, D, S, W = 4, 16, 128, 16, 48
+    cache = hz.PagedCache(1, Hkv, Hq, D, 3, 40, 1000, [1, 0, 1, 1], S, W, device=cuda_device)
+    seqs = [Seq(cache, i + 1, 1000) for i in range(3)]
+    for s, n in zip(seqs, (900, 33, 257)):
+        s.prefill(n, cuda_device)
+    q = rand_bf16((3, Hq, D), 77).to(cuda_device)
+    slots = [s.slot for s in seqs]
+    want = cache.decode(0, slots, q)
+    rl.rlkv_paged_set_output_bf16(cache.handle, 1)
+    got = torch.zeros((3, Hq, D), dtype=torch.bfloat16, device=cuda_device)
+    rl.rlkv_paged_decode_attention(cache.handle, 0, slots, q, got)
+    assert torch.equal(got, want.to(torch.bfloat16))
+    rl.rlkv_paged_set_output_bf16(cache.handle, 0)
+    assert torch.equal(cache.decode(0, slots, q), want)
+    assert cache.status() == 0
+    cache.close()

@@ -416,3 +416,53 @@ def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):
             check_out(outs[t][l].numpy(), oracle.decode(l, ins[t][2][l]))
     check_state(a, oracle)
     assert a.status() == 0 and b.status() == 0
+
+
+# ------------------------------------------------------------------------------------------ bf16 output
+def test_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
+    """rlkv_set_output_bf16: the same arithmetic, results rounded to nearest even when stored -- so
+    the bf16 result must equal the fp32 result of the same call converted by torch, bit for bit, for
+    the per-layer call, the whole step on device buffers and the step on host buffers."""
+    layers, Hkv, Hq, D, B, S, W, n = 8, 4, 16, 128, 3, 16, 48, 700
+    mask = synth.head_mask(5, layers, Hkv, 0.4)
+    caches = []
+    for _ in range(2):
+        c = hz.Cache(layers, Hkv, Hq, D, B, n + 8, mask, S, W, device=cuda_device)
+        for l in range(layers):
+            c.prefill(l, rand_bf16((n, B, Hkv, D), 10 + l, cuda_device), rand_bf16((n, B, Hkv, D), 50 + l, cuda_device))
+        caches.append(c)
+    f32, b16 = caches
+    rl.rlkv_set_output_bf16(b16.handle, 1)
+    q = rand_bf16((layers, B, Hq, D), 90, cuda_device)
+    # per-layer call
+    want = f32.decode(0, q[0])
+    got = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=cuda_device)
+    rl.rlkv_decode_attention(b16.handle, 0, q[0], got)
+    assert torch.equal(got, want.to(torch.bfloat16))
+    # whole step, device buffers
+    k, v = rand_bf16((layers, B, Hkv, D), 91, cuda_device), rand_bf16((layers, B, Hkv, D), 92, cuda_device)
+    want = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+    got = torch.zeros((layers, B, Hq, D), dtype=torch.bfloat16, device=cuda_device)
+    rl.rlkv_step(f32.handle, k, v, q, want)
+    rl.rlkv_step(b16.handle, k, v, q, got)
+    assert torch.equal(got, want.to(torch.bfloat16))
+    # whole step, host buffers
+    kh, vh, qh = (x.cpu().pin_memory() for x in (k, v, q))
+    want_h = torch.empty((layers, B, Hq, D), dtype=torch.float32).pin_memory()
+    got_h = torch.zeros((layers, B, Hq, D), dtype=torch.bfloat16).pin_memory()
+    rl.rlkv_step_host(f32.handle, kh, vh, qh, want_h)
+    rl.rlkv_step_host(b16.handle, kh, vh, qh, got_h)
+    torch.cuda.synchronize()
+    assert torch.equal(got_h, want_h.to(torch.bfloat16))
+    # mixed attention adds up in fp32: refused while bf16 output is on; back to fp32, the cache works as before
+    allf = hz.Cache(1, Hkv, Hq, D, B, 16, np.ones(Hkv, np.uint8), S, W, device=cuda_device)
+    allf.append(0, k[0], v[0])
+    rl.rlkv_set_output_bf16(allf.handle, 1)
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_decode_mixed_attention(allf.handle, 0, q[0], torch.ones(Hkv, device=cuda_device), want[0])
+    assert e.value.code == rl.RLKV_EINVAL
+    rl.rlkv_set_output_bf16(b16.handle, 0)
+    assert torch.equal(b16.decode(1, q[1]), f32.decode(1, q[1]))
+    assert f32.status() == 0 and b16.status() == 0
+    for c in caches + [allf]:
+        c.close()
