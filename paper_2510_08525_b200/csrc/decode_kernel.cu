@@ -916,7 +916,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         if (et <= kMaxRounds) {
             int slot = 0, count = 0;
             if (et <= sc.R) unit_partials(sc, 0, et, slot, count);
-            lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count);
+            // two records per band at most: one batch of loads warms the same instructions as many
+            lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count < 2 ? count : 2);
         }
         epilogue_sync();
         merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1,

@@ -46,6 +46,7 @@ struct Layout {
 
 constexpr int kDefaultItemTiles = 32;        // launches of rlkv_step, which overlap: coarse items, few partials
 constexpr int kDefaultItemTilesAlone = 8;    // a launch on its own: finer items for an even finish
+constexpr int kMaxFanIn = 32;                // most pieces a full unit is cut into when the schedule has no bands
 
 int check_shape(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
                 const uint8_t* mask, int sink, int window)
@@ -265,6 +266,15 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     if (item_tiles > most) item_tiles = most;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * second_class, tiles_comp, grid, item_tiles);
+    // A launch too small for the schedule to form bands cuts every full unit into tiles_full / item_tiles
+    // pieces, all merged by one CTA at the end: with a few long rows that fan-in, not the bytes, sets
+    // the time.  Larger items (fewer CTAs, each streaming longer) bound it.
+    // Inside a step only where the launch would not fill the GPU anyway: a full grid overlaps with its
+    // neighbours, which hides the merge better than larger items avoid it.
+    if (a.sched.R == 0 && a.n_full > 0 && tiles_full > kMaxFanIn * item_tiles && (!in_step || a.sched.n_items < grid)) {
+        item_tiles = (tiles_full + kMaxFanIn - 1) / kMaxFanIn;
+        a.sched = make_schedule(c->batch * a.n_full, tiles_full, c->batch * second_class, tiles_comp, grid, item_tiles);
+    }
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     *grid_out = grid;
     return RLKV_OK;
@@ -273,11 +283,11 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
 // `half`: which half of the scratch memory (partials, claim counter) the launch uses; `overlap` and
 // `dep_wait` as in launch_decode.
 int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, int half = 0, bool overlap = false,
-              bool dep_wait = false, int* grid_out = nullptr, const float* alpha = nullptr)
+              bool dep_wait = false, int* grid_out = nullptr, const float* alpha = nullptr, bool in_step = false)
 {
     DecodeArgs a;
     int grid = 0;
-    int rc = build_decode_args(c, layer, q, out, a, &grid, overlap, alpha);
+    int rc = build_decode_args(c, layer, q, out, a, &grid, in_step, alpha);
     if (rc) return rc;
     if (a.sched.n_slots > c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
     // mixed attention: both units of a head add into `out`
@@ -393,7 +403,7 @@ int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStr
         const bool overlap = prev_ok;
         int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
                            static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, overlap,
-                           overlap && l == 0, &grid);
+                           overlap && l == 0, &grid, nullptr, true);
         if (rc) return rc;
         prev_ok = (grid == c->sm_count && c->ctas_per_sm == 1);
     }
