@@ -910,19 +910,23 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         const int et = tid - (S::kWarps + 2) * 32;
         const int PF = partial_floats(D, G), PH = partial_head_floats(G);
         // warm the instruction cache with the merge routine while there is nothing else to do: a dry
-        // run on unit 0 (its partial records hold whatever the last launch left; nothing is stored)
-        if (et == 0) todo[kMaxTodo - 1] = make_int2(0, 0);
-        epilogue_sync();
-        if (et <= kMaxRounds) {
-            int slot = 0, count = 0;
-            if (et <= sc.R) unit_partials(sc, 0, et, slot, count);
-            // two records per band at most: one batch of loads warms the same instructions as many
-            lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count < 2 ? count : 2);
+        // run on unit 0 (its partial records hold whatever the last launch left; nothing is stored).
+        // Not in a launch so small that a CTA's stream is a few tiles: there the first segment would
+        // wait for the dry run's trip to memory.
+        if (sc.n_items > 2 * sc.P) {
+            if (et == 0) todo[kMaxTodo - 1] = make_int2(0, 0);
+            epilogue_sync();
+            if (et <= kMaxRounds) {
+                int slot = 0, count = 0;
+                if (et <= sc.R) unit_partials(sc, 0, et, slot, count);
+                // two records per band at most: one batch of loads warms the same instructions as many
+                lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count < 2 ? count : 2);
+            }
+            epilogue_sync();
+            merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1),
+                                  1, et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
+            epilogue_sync();
         }
-        epilogue_sync();
-        merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1), 1,
-                              et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
-        epilogue_sync();
         if (a.dep_wait) {  // from here on these warps write results, partials and tickets
             grid_dep_wait();
             if (et == 0) grid_dep_launch();

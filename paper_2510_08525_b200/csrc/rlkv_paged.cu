@@ -49,6 +49,7 @@ struct rlkv_paged {
 namespace {
 
 constexpr int kPagedItemTiles = 8;
+constexpr int kPagedMaxFanIn = 32;
 
 int check_paged_shape(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
                       int max_seq_len, const uint8_t* mask, int sink, int window)
@@ -406,6 +407,12 @@ int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int 
     if (item_tiles > p->item_tiles) item_tiles = p->item_tiles;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
+    // a launch too small for bands: no full unit in more than kPagedMaxFanIn pieces (their merge by one
+    // CTA, not the bytes, would set the time)
+    if (a.sched.R == 0 && a.n_full > 0 && tiles_full > kPagedMaxFanIn * item_tiles) {
+        item_tiles = (tiles_full + kPagedMaxFanIn - 1) / kPagedMaxFanIn;
+        a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
+    }
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     if (a.sched.n_slots > p->max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
     a.partials = dev_at<float>(p, p->off_partials);
