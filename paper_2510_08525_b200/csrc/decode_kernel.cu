@@ -427,6 +427,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     // running before the step's append launch has completed: it fetches and processes tiles that hold
     // only older tokens, waits (grid_dep_wait) before it touches anything else, and only then lets
     // the next layer start, which therefore never has to wait.
+    // dep_wait == 2: a launch that follows one too small to fill the GPU.  The host starts it this way
+    // only where the launch two before it has completed, so it works freely; but the NEXT launch shares
+    // its scratch half with the launch before this one, which may still be running: an otherwise idle
+    // thread of every CTA waits for that launch and only then lets the next one start.
     if (tid == 0 && !args.dep_wait) grid_dep_launch();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
@@ -804,7 +808,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         } else {
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit.  Everything else is older and may be fetched early.
-                        if (a.dep_wait && !synced &&
+                        if (a.dep_wait == 1 && !synced &&
                             (k != (int)blockIdx.x || u.pos.uid >= sc.U || u.pos.tile + seg_left == u.tiles)) {
                             grid_dep_wait();
                             synced = true;
@@ -902,6 +906,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 mbar_arrive(smem_u32(claim_full));
                 if (k >= sc.n_items) break;  // the producer stops asking once it has seen this answer
             }
+        } else if (lane == 1 && a.dep_wait == 2) {
+            grid_dep_wait();    // the launch before this one has completed ...
+            grid_dep_launch();  // ... so the next one, which shares its scratch half, may start
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps
@@ -927,7 +934,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                   1, et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
             epilogue_sync();
         }
-        if (a.dep_wait) {  // from here on these warps write results, partials and tickets
+        if (a.dep_wait == 1) {  // from here on these warps write results, partials and tickets
             grid_dep_wait();
             if (et == 0) grid_dep_launch();
         }

@@ -283,7 +283,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
 // `half`: which half of the scratch memory (partials, claim counter) the launch uses; `overlap` and
 // `dep_wait` as in launch_decode.
 int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, int half = 0, bool overlap = false,
-              bool dep_wait = false, int* grid_out = nullptr, const float* alpha = nullptr, bool in_step = false)
+              int dep_wait = 0, int* grid_out = nullptr, const float* alpha = nullptr, bool in_step = false)
 {
     DecodeArgs a;
     int grid = 0;
@@ -297,7 +297,7 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * 2 * c->batch * c->kv_heads;
     a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4 + half;
     a.claim_base = c->claims[half];
-    a.dep_wait = dep_wait ? 1 : 0;
+    a.dep_wait = dep_wait;
     RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, overlap, alpha ? kModeMixed : kModePlain));
     c->claims[half] += (unsigned int)a.sched.n_items;  // every CTA claims until it is told there is no more
     if (grid_out) *grid_out = grid;
@@ -397,15 +397,33 @@ int step_append(rlkv_cache* c, const void* k, const void* v, cudaStream_t s)
 int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStream_t s, bool fresh)
 {
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
-    bool prev_ok = !fresh;  // right after the append launch an overlapped launch is fine: it waits on the device
+    // What the launch before this one in the stream was: an ordinary launch (it started after
+    // everything before it had completed: the append launch, or a decode launch after a stream wait),
+    // an overlapped launch that lets its successor start at once, or an overlapped launch that lets
+    // its successor start only after its own predecessor has completed (dep_wait 1 or 2).
+    enum { kOrdinary, kFree, kWaits } prev = kOrdinary;
+    bool prev_full = false;  // it put one CTA on every SM
     for (int l = l0; l < l1; ++l) {
-        int grid = 0;
-        const bool overlap = prev_ok;
+        int grid = 0, dep_wait = 0;
+        bool overlap;
+        if (l == l0) {
+            // right after the append launch an overlapped launch is fine: it waits on the device for it
+            overlap = !fresh;
+            dep_wait = overlap && l == 0 ? 1 : 0;
+        } else if (prev_full) {
+            overlap = true;  // all CTAs of the launch before have started: none of the one before that is left
+        } else if (prev != kFree) {
+            overlap = true;  // the launch two back had completed when the launch before let this one start
+            dep_wait = 2;    // and this one keeps the next launch back until the launch before has completed
+        } else {
+            overlap = false;
+        }
         int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                           static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, overlap,
-                           overlap && l == 0, &grid, nullptr, true);
+                           static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, overlap, dep_wait,
+                           &grid, nullptr, true);
         if (rc) return rc;
-        prev_ok = (grid == c->sm_count && c->ctas_per_sm == 1);
+        prev = !overlap ? kOrdinary : (dep_wait ? kWaits : kFree);
+        prev_full = (grid == c->sm_count && c->ctas_per_sm == 1);
     }
     return RLKV_OK;
 }

@@ -227,8 +227,10 @@ struct DecodeArgs {
     int* tickets;               // one per unit of this layer, zero between launches
     unsigned int* claim_counter;  // items claimed beyond the first P, over all launches so far (never reset)
     unsigned int claim_base;      // its value when this launch starts: every launch adds exactly sched.n_items
-    int dep_wait;               // the launch may start before the kernel that wrote this step's new rows has
-                                // completed: wait for it before touching what it writes (see launch_decode)
+    int dep_wait;               // 1: the launch may start before the kernel that wrote this step's new rows has
+                                // completed: wait for it before touching what it writes (see launch_decode);
+                                // 2: the launch may start while the two launches before it still run: wait for
+                                // the one before it prior to any claim and any write (see decode_kernel)
     int* status;                // device error word
     unsigned long long* trace;  // debug: [grid][kTraceWords]
     int n_full, n_comp;         // heads of each class in this layer

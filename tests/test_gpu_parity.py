@@ -387,6 +387,39 @@ def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
     assert e.value.code == rl.RLKV_EFULL
 
 
+def test_step_mixes_tiny_and_gpu_filling_launches(rl, hz, cuda_device):
+    """Seven layers whose launches alternate between a few work items and more than one per SM (all
+    heads compressed, one full head, all full): inside rlkv_step a launch after a small one starts
+    beside it and holds its own successor back, a launch after a GPU-filling one starts as SMs free
+    up.  60 consecutive steps, every layer against the oracle at several of them, and the step's
+    results equal to the per-layer calls on a twin cache."""
+    Hkv, Hq, D, B, S, W, prompt, steps = 4, 16, 128, 6, 8, 56, 3000, 60
+    mask = [0, 0, 0, 0,  1, 1, 1, 1,  0, 1, 0, 0,  0, 0, 0, 0,  0, 0, 0, 0,  1, 1, 1, 1,  1, 0, 0, 1]
+    layers = len(mask) // Hkv
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, cuda_device)
+    twin = hz.Cache(layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, device=cuda_device)
+    for l in range(layers):
+        K, V = rand_bf16((prompt, B, Hkv, D), 150 + l), rand_bf16((prompt, B, Hkv, D), 160 + l)
+        feed(cache, oracle, l, K, V, True)
+        twin.prefill(l, K.to(cuda_device), V.to(cuda_device))
+    out = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+    K, V = rand_bf16((steps, layers, B, Hkv, D), 170), rand_bf16((steps, layers, B, Hkv, D), 171)
+    Q = rand_bf16((steps, layers, B, Hq, D), 172)
+    Kd, Vd, Qd = K.to(cuda_device), V.to(cuda_device), Q.to(cuda_device)
+    for t in range(steps):
+        rl.rlkv_step(cache.handle, Kd[t], Vd[t], Qd[t], out)
+        for l in range(layers):
+            assert oracle.append(l, K[t, l], V[t, l]) == 0
+            twin.append(l, Kd[t, l], Vd[t, l])
+        if t in (0, 1, 2, 31, steps - 1):
+            got = out.cpu().numpy()
+            for l in range(layers):
+                check_out(got[l], oracle.decode(l, Q[t, l]))
+                np.testing.assert_allclose(got[l], twin.decode(l, Qd[t, l]).cpu().numpy(), atol=1e-4, rtol=0)
+    check_state(cache, oracle)
+    assert cache.status() == 0 and twin.status() == 0
+
+
 def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):
     """Nine layers, so that rlkv_step_host brings inputs in and takes results out in chunks on its side
     streams, and consecutive calls alternate between its two input staging areas: five steps in a row
