@@ -368,9 +368,12 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
 // Launch l and launch l-2 share a half of the scratch memory, so launch l must not start before
 // launch l-2 has completed.  An overlapped launch starts when every CTA of launch l-1 has started; if
 // launch l-1 puts exactly one CTA on every SM (and a CTA takes a whole SM: its registers see to that),
-// all of them having started means that no CTA of launch l-2 is left.  After a smaller launch, or
-// after anything but a kernel of this step in the stream (`fresh`), the next launch is an ordinary
-// one, which waits for everything before it.
+// all of them having started means that no CTA of launch l-2 is left.  After a smaller launch l-1
+// the launch is still overlapped if launch l-2 is known to have completed by the time launch l-1 lets
+// launch l start (launch l-1 was an ordinary launch, or held launch l back itself); launch l then
+// holds launch l+1 back until launch l-1 has completed (dep_wait 2 in decode_kernel).  Otherwise, and
+// after anything but a kernel of this step in the stream (`fresh`), the launch is an ordinary one,
+// which waits for everything before it.
 int step_append(rlkv_cache* c, const void* k, const void* v, cudaStream_t s)
 {
     AppendAllArgs aa;

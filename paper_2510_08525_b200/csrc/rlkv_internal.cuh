@@ -359,7 +359,8 @@ __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.w
 // start while the kernel before it in the stream is still running.  Only for the decode launches of
 // one rlkv_step, whose inputs are complete before the step's first launch: consecutive layers use
 // different halves of the scratch memory and touch nothing of each other, and the first layer's
-// launch (dep_wait) waits on the device for the step's append launch before it reads new rows.
+// launch (dep_wait 1) waits on the device for the step's append launch before it reads new rows; a
+// launch after one too small to fill the GPU (dep_wait 2) keeps the next launch back instead.
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
 
 // The appends of one token to every layer, in one launch (rlkv_step).
