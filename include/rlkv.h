@@ -178,7 +178,7 @@ int rlkv_step_host(rlkv_cache* cache, const void* k_host, const void* v_host, co
  * compressed head.  What is computed per sequence is exactly what the lock-step cache computes for a
  * batch row (same slot rule, same attention); the calls name the request slots they act on, so a
  * decode step can serve any subset of the open slots, each at its own length.
- * Limits: max_seq_len <= 65536 tokens; at most min(max_seqs, 256) sequences per call; the other
+ * Limits: max_seq_len <= 65536 tokens; at most min(max_seqs, 512) sequences per call; the other
  * shape limits of rlkv_cache_create.  Device memory: rlkv_paged_size bytes, library- or caller-owned
  * as for rlkv_cache_create.  Errors leave the cache unchanged. */
 typedef struct rlkv_paged rlkv_paged;

@@ -23,7 +23,7 @@ constexpr int kItemRing = 4;     // work-item descriptors in flight between prod
 constexpr int kTraceWords = 40;  // debug trace: 64-bit words per CTA
 constexpr int kMaxTodo = 64;      // split merges a CTA may put off until its stream has ended
 constexpr int kMaxPend = 16;      // partial segments of a CTA whose tickets are drawn when its stream has ended
-constexpr int kMaxPagedBatch = 256;   // sequences one launch over the paged cache may serve
+constexpr int kMaxPagedBatch = 512;   // sequences one launch over the paged cache may serve
 constexpr int kMaxSeqPages = 1024;    // 64-token pages one sequence may hold (65536 tokens)
 constexpr int kClaimAhead = 3;   // the producer asks for its next work item this many tiles before the current one ends
 

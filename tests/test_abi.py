@@ -112,8 +112,8 @@ def test_paged_size_and_argument_checks_need_no_device(binding):
     assert size >= 2 * (10 * page_bytes + 3 * ring_bytes)
     more_pages = binding.rlkv_paged_size(**{**ok, "n_pages": 10 + 1000})
     assert more_pages - size == 2 * 1000 * page_bytes   # one full head per layer
-    # request slots beyond the 256 a launch can serve cost their rings and page-table rows, no scratch
-    a, b = (binding.rlkv_paged_size(**{**ok, "max_seqs": m}) for m in (300, 300 + 256))
+    # request slots beyond the 512 a launch can serve cost their rings and page-table rows, no scratch
+    a, b = (binding.rlkv_paged_size(**{**ok, "max_seqs": m}) for m in (600, 600 + 256))
     assert b - a == 2 * 256 * ring_bytes + 256 * 16 * 4     # 1000 tokens = 16 page-table entries
     for bad in (dict(head_dim=96), dict(q_heads=7), dict(window=0), dict(sink=-1), dict(max_seqs=0), dict(n_pages=0),
                 dict(max_seq_len=0), dict(max_seq_len=65537), dict(max_seqs=70000)):

@@ -245,3 +245,29 @@ def test_paged_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
     assert torch.equal(cache.decode(0, slots, q), want)
     assert cache.status() == 0
     cache.close()
+
+
+def test_four_hundred_sequences_in_one_call(rl, hz, cuda_device):
+    """More requests than the paper's largest serving batch (375, Table 3) in one append and one decode
+    call: 400 sequences of 1 .. 260 tokens, one full and one compressed head."""
+    Hkv, Hq, D, S, W, n = 2, 4, 64, 4, 28, 400
+    rng = np.random.default_rng(8)
+    lens = [int(x) for x in rng.integers(1, 261, size=n)]
+    pages = sum((x + 1 + 63) // 64 for x in lens) + 1
+    cache = hz.PagedCache(1, Hkv, Hq, D, n, pages, 300, [1, 0], S, W, device=cuda_device)
+    seqs = []
+    for i, x in enumerate(lens):
+        s = Seq(cache, 1000 + i, 300)
+        if x > 1:
+            s.prefill(x - 1, cuda_device)
+        seqs.append(s)
+    append_all(cache, seqs, cuda_device)
+    q = rand_bf16((n, Hq, D), 31)
+    out = cache.decode(0, [s.slot for s in seqs], q.to(cuda_device)).cpu().numpy()
+    for i, s in enumerate(seqs):
+        check_out(out[i], s.oracle.decode(0, q[i:i + 1])[0])
+    with pytest.raises(rl.RlkvError) as e:                   # 513 would be too many for one call
+        rl.rlkv_paged_decode_attention(cache.handle, 0, list(range(400)) + list(range(113)), q.to(cuda_device), out)
+    assert e.value.code == rl.RLKV_EINVAL
+    assert cache.status() == 0
+    cache.close()
