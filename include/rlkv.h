@@ -210,7 +210,18 @@ int rlkv_paged_prefill(rlkv_paged* cache, int layer, int slot, const void* k, co
  * sequence holds no token in this layer. */
 int rlkv_paged_decode_attention(rlkv_paged* cache, int layer, const int* slots, int n,
                                 const void* q, void* out, void* stream);
-/* As rlkv_set_output_bf16, for rlkv_paged_decode_attention. */
+/* One whole decode step for n sequences: one token appended to every layer of each, then every
+ * layer's attention.  k, v: device bf16 [layers][n][kv_heads][head_dim]; q: device bf16
+ * [layers][n][q_heads][head_dim]; out: device fp32 [layers][n][q_heads][head_dim]; entry i of the
+ * second dimension belongs to slots[i] (HOST int[n]).  Results are those of rlkv_paged_append and
+ * rlkv_paged_decode_attention layer by layer (up to floating-point summation order).  As in rlkv_step
+ * all inputs are there before the first launch, so the step is one append launch for all layers and
+ * the layers' attention launches, overlapped on the device; the buffers must be complete at the call
+ * and stay untouched until the work on `stream` has finished.  Every listed sequence must have the
+ * same length in all layers (RLKV_EINVAL otherwise); RLKV_EFULL as for rlkv_paged_append. */
+int rlkv_paged_step(rlkv_paged* cache, const int* slots, int n, const void* k, const void* v,
+                    const void* q, void* out, void* stream);
+/* As rlkv_set_output_bf16, for rlkv_paged_decode_attention and rlkv_paged_step. */
 int rlkv_paged_set_output_bf16(rlkv_paged* cache, int on);
 int rlkv_paged_length(const rlkv_paged* cache, int layer, int slot, int* len_out);
 /* Pages on the free list and pages in total. */

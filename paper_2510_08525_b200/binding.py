@@ -53,6 +53,7 @@ SIGNATURES = {
     "rlkv_paged_append": (_ci, [_vp, _ci, _vp, _ci, _vp, _vp, _vp]),
     "rlkv_paged_prefill": (_ci, [_vp, _ci, _ci, _vp, _vp, _ci, _vp]),
     "rlkv_paged_decode_attention": (_ci, [_vp, _ci, _vp, _ci, _vp, _vp, _vp]),
+    "rlkv_paged_step": (_ci, [_vp, _vp, _ci, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_paged_length": (_ci, [_vp, _ci, _ci, ctypes.POINTER(_ci)]),
     "rlkv_paged_pages": (_ci, [_vp, ctypes.POINTER(_ci), ctypes.POINTER(_ci)]),
     "rlkv_paged_step_bytes": (_ci, [_vp, _ci, _vp, _ci, ctypes.POINTER(ctypes.c_uint64)]),
@@ -313,6 +314,11 @@ def rlkv_paged_prefill(cache, layer, slot, k, v, n_tokens, stream=None) -> None:
 def rlkv_paged_decode_attention(cache, layer, slots, q, out, stream=None) -> None:
     s = _slots(slots)
     _check(lib.rlkv_paged_decode_attention(cache, layer, s.ctypes.data, s.size, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_paged_step(cache, slots, k, v, q, out, stream=None) -> None:
+    s = _slots(slots)
+    _check(lib.rlkv_paged_step(cache, s.ctypes.data, s.size, _ptr(k), _ptr(v), _ptr(q), _ptr(out), _stream(stream)))
 
 
 def rlkv_paged_length(cache, layer, slot) -> int:

@@ -86,10 +86,12 @@ __global__ void __launch_bounds__(256) append_all_kernel(const __grid_constant__
 __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant__ PagedAppendArgs a)
 {
     const int chunks = a.head_dim / 8;
-    const long long total = (long long)a.n * a.kv_heads * chunks * 2;
+    const long long per_layer = (long long)a.n * a.kv_heads * chunks * 2;
+    const long long total = per_layer * a.n_layers;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (long long)gridDim.x * blockDim.x) {
-        long long r = i;
+        const int l = (int)(i / per_layer);
+        long long r = i - l * per_layer;
         const int c = (int)(r % chunks);
         r /= chunks;
         const int h = (int)(r % a.kv_heads);
@@ -99,10 +101,17 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
         const int seq = a.prefill ? a.slot[0] : a.slot[e];
         const int t = a.prefill ? a.t0 + e : a.t[e];
         const int page = a.page[a.prefill ? t / kTile - a.first_page : e];
-        const int slot = a.slot_of_head[h];
+        const int slot = a.slot_of_head[l * a.kv_heads + h];
+        long long full_row0 = a.full_row0, comp_row0 = a.comp_row0;
+        int n_comp = a.n_comp;
+        if (a.n_layers > 1) {
+            full_row0 = a.layers[l].full_row0;
+            comp_row0 = a.layers[l].comp_row0;
+            n_comp = a.layers[l].n_comp;
+        }
         long long row;
         if (slot >= 0) {
-            row = a.full_row0 + (((long long)slot * a.n_pages + page) * 2 + kv) * kTile + t % kTile;
+            row = full_row0 + (((long long)slot * a.n_pages + page) * 2 + kv) * kTile + t % kTile;
             if (slot == 0 && c == 0 && kv == 0) a.page_table[(size_t)seq * a.table_stride + t / kTile] = page;
         } else {
             if (a.prefill) {
@@ -110,9 +119,9 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
                 if (!(t < a.sink || t >= n_final - a.window)) continue;  // evicted before the batch ends
             }
             const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
-            row = a.comp_row0 + (((long long)seq * a.n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
+            row = comp_row0 + (((long long)seq * n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
         }
-        const __nv_bfloat16* src = (kv ? a.v : a.k) + ((long long)e * a.kv_heads + h) * a.head_dim;
+        const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.n + e) * a.kv_heads + h) * a.head_dim;
         const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
         reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
     }
@@ -122,7 +131,7 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
 
 cudaError_t launch_paged_append(const PagedAppendArgs& a, cudaStream_t stream)
 {
-    const long long total = (long long)a.n * a.kv_heads * (a.head_dim / 8) * 2;
+    const long long total = (long long)a.n_layers * a.n * a.kv_heads * (a.head_dim / 8) * 2;
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;

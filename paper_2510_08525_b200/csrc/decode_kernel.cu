@@ -770,6 +770,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 x += seg_skip - 1;
                                 continue;
                             }
+                            // the step's append launch writes page-table entries and rows this launch reads:
+                            // the first layer's launch waits for it before its first look-up
+                            if (a.dep_wait == 1 && !synced) {
+                                grid_dep_wait();
+                                synced = true;
+                            }
                             // empty slots until the slot counter has the residue of x
                             for (int pad = ((x - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
                                 ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);

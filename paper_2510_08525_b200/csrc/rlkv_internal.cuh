@@ -389,6 +389,9 @@ size_t decode_smem_bytes(int head_dim, int stages, int group, int groups, int mo
 // t0 + i of request slot slot[0] (prefill); page[j] is the physical page of page index
 // first_page + j of the sequence (append: j = i, the page of token t[i]).  The kernel also records
 // the pages in the device page table.
+// With n_layers > 1 (rlkv_paged_step) the launch appends the same token positions to every layer: k, v
+// are [n_layers][n][kv_heads][head_dim], slot_of_head is the table of layer 0 of [n_layers][kv_heads],
+// and each layer's regions come from `layers`.
 constexpr int kMaxAppendPages = 512;
 struct PagedAppendArgs {
     __nv_bfloat16* pool;
@@ -401,6 +404,8 @@ struct PagedAppendArgs {
     int kv_heads, head_dim, sink, window;
     int prefill;                // 0: n sequences, one token each; 1: one sequence, n tokens from t0
     int n, t0, first_page;
+    int n_layers;               // 1 unless the launch serves every layer
+    const LayerDesc* layers;    // device, [n_layers]; unused when n_layers == 1
     int page[kMaxAppendPages];
     int t[kMaxPagedBatch];
     unsigned short slot[kMaxPagedBatch];

@@ -10,9 +10,12 @@
 //               [max_seqs][n_comp(layer)][K|V][rows_comp][D]
 //   tables      int32 slot_of_head[layers][kv_heads]
 //   page table  int32 [max_seqs][table_stride]   (written by the append kernels)
-//   tickets     int32 [kMaxPagedBatch * kv_heads]
-//   status      int32 kernel status word, then the work-claim counter
-//   partials    float [max_slots][partial_floats]
+//   layer desc  LayerDesc[layers]  (where each layer's regions start; for the step's append launch)
+//   tickets     int32 [2][kMaxPagedBatch * kv_heads]
+//   status      int32 kernel status word, then two work-claim counters
+//   partials    float [2][max_slots][partial_floats]
+//               (tickets, counters and partials exist twice: the overlapped launches of
+//               rlkv_paged_step alternate between the halves)
 // Lengths, the page table's mirror and the free list live on the host.
 #include <stdlib.h>
 #include <string.h>
@@ -38,8 +41,8 @@ struct rlkv_paged {
     std::vector<int> table;       // [max_seqs][table_stride], -1 = no page
     std::vector<int> free_pages;  // stack of physical pages
     std::vector<uint8_t> open;    // [max_seqs]
-    size_t off_pool, off_tables, off_page_table, off_tickets, off_status, off_partials, total;
-    unsigned int claims;
+    size_t off_pool, off_tables, off_layer_desc, off_page_table, off_tickets, off_status, off_partials, total;
+    unsigned int claims[2];
     uint8_t* dev_base;
     bool owns_buffer;
     CUtensorMap tmap;
@@ -48,7 +51,8 @@ struct rlkv_paged {
 
 namespace {
 
-constexpr int kPagedItemTiles = 8;
+constexpr int kPagedItemTiles = 8;       // smallest work item of a launch on its own
+constexpr int kPagedItemTilesStep = 32;  // and of the overlapped launches of rlkv_paged_step
 constexpr int kPagedMaxFanIn = 32;
 
 int check_paged_shape(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
@@ -107,14 +111,16 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
     off = align_up(off + (size_t)row * p.head_dim * 2, 1024);
     p.off_tables = off;
     off = align_up(off + (size_t)p.layers * p.kv_heads * sizeof(int), 1024);
+    p.off_layer_desc = off;
+    off = align_up(off + (size_t)p.layers * sizeof(LayerDesc), 1024);
     p.off_page_table = off;
     off = align_up(off + (size_t)p.max_seqs * p.table_stride * sizeof(int), 1024);
     p.off_tickets = off;
-    off = align_up(off + (size_t)kMaxPagedBatch * p.kv_heads * sizeof(int), 1024);
+    off = align_up(off + (size_t)2 * kMaxPagedBatch * p.kv_heads * sizeof(int), 1024);
     p.off_status = off;
     off = align_up(off + 64, 1024);
     p.off_partials = off;
-    off = align_up(off + (size_t)p.max_items * partial_floats(p.head_dim, p.q_heads / p.kv_heads) * sizeof(float), 1024);
+    off = align_up(off + (size_t)2 * p.max_items * partial_floats(p.head_dim, p.q_heads / p.kv_heads) * sizeof(float), 1024);
     p.total = off;
     return RLKV_OK;
 }
@@ -158,6 +164,8 @@ void fill_append_args(rlkv_paged* p, int layer, const void* k, const void* v, Pa
     a.head_dim = p->head_dim;
     a.sink = p->sink;
     a.window = p->window;
+    a.n_layers = 1;
+    a.layers = nullptr;
 }
 
 }  // namespace
@@ -191,7 +199,7 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
     if (!p) return RLKV_ENOMEM;
     p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
     p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window;
-    p->claims = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
+    p->claims[0] = p->claims[1] = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
     rc = make_paged_layout(*p, head_is_full, max_seq_len);
     if (rc) { delete p; return rc; }
     p->len.assign((size_t)layers * max_seqs, 0);
@@ -227,6 +235,11 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
     if (e == cudaSuccess)
         e = cudaMemcpy(p->dev_base + p->off_tables, p->slot_of_head.data(), p->slot_of_head.size() * sizeof(int),
                        cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) {
+        std::vector<LayerDesc> desc(layers);
+        for (int l = 0; l < layers; ++l) desc[l] = LayerDesc{p->full_row0[l], p->comp_row0[l], p->n_full[l], p->n_comp[l]};
+        e = cudaMemcpy(p->dev_base + p->off_layer_desc, desc.data(), desc.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice);
+    }
     if (e == cudaSuccess) e = prepare_decode_kernels(head_dim);
     if (e != cudaSuccess) return fail(cuda_fail(e, "rlkv_paged_create"));
     rc = encode_pool_tensor_map(&p->tmap, p->dev_base + p->off_pool, p->pool_rows, head_dim);
@@ -357,19 +370,16 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
     return RLKV_OK;
 }
 
-int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int n, const void* q, void* out, void* stream)
+// One decode launch (arguments checked by the caller).  `half`: which copy of tickets, claim counter
+// and partials; `overlap`, `dep_wait`: as for the lock-step cache (launch_decode, decode_kernel);
+// `in_step`: the launch belongs to rlkv_paged_step (coarser items: its neighbours hide its tail).
+static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const void* q, void* out, cudaStream_t stream,
+                        int half, bool overlap, int dep_wait, bool in_step, int* grid_out)
 {
-    if (!valid_layer(p, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
-    int rc = check_slots(p, slots, n);
-    if (rc) return rc;
     const int* len = len_of(p, layer);
     int longest = 0;
-    for (int i = 0; i < n; ++i) {
-        if (len[slots[i]] < 1) return RLKV_EEMPTY;
+    for (int i = 0; i < n; ++i)
         if (len[slots[i]] > longest) longest = len[slots[i]];
-    }
-    DeviceGuard g(p->device);
-    if (!g.ok) return RLKV_ECUDA;
     const int cap = p->sink + p->window;
     DecodeArgs a;
     memset(&a, 0, sizeof a);
@@ -404,22 +414,23 @@ int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int 
     int grid = p->sm_count;
     if (grid > p->max_grid) grid = p->max_grid;
     int item_tiles = (int)(real_tiles / grid);
-    if (item_tiles > p->item_tiles) item_tiles = p->item_tiles;
+    const int most = in_step ? kPagedItemTilesStep : p->item_tiles;
+    if (item_tiles > most) item_tiles = most;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
     // a launch too small for bands: no full unit in more than kPagedMaxFanIn pieces (their merge by one
     // CTA, not the bytes, would set the time)
-    if (a.sched.R == 0 && a.n_full > 0 && tiles_full > kPagedMaxFanIn * item_tiles) {
+    if (a.sched.R == 0 && a.n_full > 0 && tiles_full > kPagedMaxFanIn * item_tiles && (!in_step || a.sched.n_items < grid)) {
         item_tiles = (tiles_full + kPagedMaxFanIn - 1) / kPagedMaxFanIn;
         a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
     }
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     if (a.sched.n_slots > p->max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
-    a.partials = dev_at<float>(p, p->off_partials);
-    a.tickets = dev_at<int>(p, p->off_tickets);
-    a.claim_counter = dev_at<unsigned int>(p, p->off_status) + 4;
-    a.claim_base = p->claims;
-    a.dep_wait = 0;
+    a.partials = dev_at<float>(p, p->off_partials) + (size_t)half * p->max_items * partial_floats(p->head_dim, a.group);
+    a.tickets = dev_at<int>(p, p->off_tickets) + (size_t)half * kMaxPagedBatch * p->kv_heads;
+    a.claim_counter = dev_at<unsigned int>(p, p->off_status) + 4 + half;
+    a.claim_base = p->claims[half];
+    a.dep_wait = dep_wait;
     PagedArgs pa;
     pa.page_table = dev_at<int>(p, p->off_page_table);
     pa.table_stride = p->table_stride;
@@ -429,12 +440,99 @@ int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int 
         pa.seq_len[i] = i < n ? len[slots[i]] : 0;
         pa.seq_slot[i] = (unsigned short)(i < n ? slots[i] : 0);
     }
-    RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, static_cast<cudaStream_t>(stream), false,
-                            kModePaged, &pa));
-    p->claims += (unsigned int)a.sched.n_items;
+    RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, stream, overlap, kModePaged, &pa));
+    p->claims[half] += (unsigned int)a.sched.n_items;
     p->launches++;
+    if (grid_out) *grid_out = grid;
     return RLKV_OK;
 }
+
+int rlkv_paged_decode_attention(rlkv_paged* p, int layer, const int* slots, int n, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(p, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    int rc = check_slots(p, slots, n);
+    if (rc) return rc;
+    for (int i = 0; i < n; ++i)
+        if (len_of(p, layer)[slots[i]] < 1) return RLKV_EEMPTY;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return paged_decode(p, layer, slots, n, q, out, static_cast<cudaStream_t>(stream), 0, false, 0, false, nullptr);
+}
+
+int rlkv_paged_step(rlkv_paged* p, const int* slots, int n, const void* k, const void* v, const void* q, void* out,
+                    void* stream)
+{
+    if (!p || !k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    int rc = check_slots(p, slots, n);
+    if (rc) return rc;
+    // one append launch for all layers needs every listed sequence at the same length in every layer
+    // (which is how a decode loop leaves them); room and pages are checked before anything changes
+    int need = 0;
+    for (int i = 0; i < n; ++i) {
+        const int t = len_of(p, 0)[slots[i]];
+        for (int l = 1; l < p->layers; ++l)
+            if (len_of(p, l)[slots[i]] != t) return RLKV_EINVAL;
+        if (t / kTile >= p->table_stride) return RLKV_EFULL;
+        if (p->table[(size_t)slots[i] * p->table_stride + t / kTile] < 0) ++need;
+    }
+    if (need > (int)p->free_pages.size()) return RLKV_EFULL;
+    if (p->layers > kMaxStepLayers) return RLKV_EINVAL;
+    DeviceGuard g(p->device);
+    if (!g.ok) return RLKV_ECUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    PagedAppendArgs aa;
+    fill_append_args(p, 0, k, v, aa);
+    aa.prefill = 0;
+    aa.n = n;
+    aa.t0 = 0;
+    aa.first_page = 0;
+    aa.n_layers = p->layers;
+    aa.layers = dev_at<LayerDesc>(p, p->off_layer_desc);
+    for (int i = 0; i < n; ++i) {
+        const int sl = slots[i], t = len_of(p, 0)[sl];
+        int& entry = p->table[(size_t)sl * p->table_stride + t / kTile];
+        if (entry < 0) {
+            entry = p->free_pages.back();
+            p->free_pages.pop_back();
+        }
+        aa.slot[i] = (unsigned short)sl;
+        aa.t[i] = t;
+        aa.page[i] = entry;
+    }
+    RLKV_CUDA(launch_paged_append(aa, s));
+    p->launches++;
+    for (int l = 0; l < p->layers; ++l)
+        for (int i = 0; i < n; ++i) len_of(p, l)[slots[i]] += 1;
+    // the layers' decode launches, overlapped as in rlkv_step: see step_decode in rlkv_api.cu for why
+    // each of the three cases is safe
+    const size_t q_layer = (size_t)n * p->q_heads * p->head_dim;
+    enum { kOrdinary, kFree, kWaits } prev = kOrdinary;
+    bool prev_full = false;
+    for (int l = 0; l < p->layers; ++l) {
+        int grid = 0, dep_wait = 0;
+        bool overlap;
+        if (l == 0) {
+            overlap = true;  // waits on the device for the append launch
+            dep_wait = 1;
+        } else if (prev_full) {
+            overlap = true;
+        } else if (prev != kFree) {
+            overlap = true;
+            dep_wait = 2;
+        } else {
+            overlap = false;
+        }
+        rc = paged_decode(p, l, slots, n, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
+                          static_cast<uint8_t*>(out) + l * q_layer * (p->out_bf16 ? 2 : 4), s, l & 1, overlap, dep_wait, true,
+                          &grid);
+        if (rc) return rc;
+        prev = !overlap ? kOrdinary : (dep_wait ? kWaits : kFree);
+        prev_full = grid == p->sm_count;
+    }
+    return RLKV_OK;
+}
+
+
 
 int rlkv_paged_set_output_bf16(rlkv_paged* p, int on)
 {

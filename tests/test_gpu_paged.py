@@ -271,3 +271,50 @@ def test_four_hundred_sequences_in_one_call(rl, hz, cuda_device):
     assert e.value.code == rl.RLKV_EINVAL
     assert cache.status() == 0
     cache.close()
+
+
+@pytest.mark.parametrize("shape", ["small", "filling"])
+def test_paged_step_equals_the_per_layer_calls(rl, hz, cuda_device, shape):
+    """rlkv_paged_step (one append launch for all layers, the layers' attention launches overlapped)
+    over consecutive steps that cross page boundaries: every sequence against its oracle, and the page
+    accounting as the per-layer calls would leave it.  'small': launches of a few work items, each
+    started beside the one before; 'filling': launches with more than one item per SM."""
+    if shape == "small":
+        layers, Hkv, Hq, D, S, W, lens = 5, 2, 8, 64, 4, 28, [60, 1, 126, 200]
+        mask = [1, 0, 0, 0, 1, 1, 0, 1, 1, 0]
+    else:
+        layers, Hkv, Hq, D, S, W, lens = 3, 8, 32, 128, 16, 112, [3000, 1500, 2900, 700, 2047, 3100, 2500, 1000]
+        mask = [1] * 8 + [1, 1, 0, 1, 1, 0, 1, 1] + [0] * 8
+    steps = 6
+    pages = sum((n + steps + 63) // 64 for n in lens) + 1
+    cache = hz.PagedCache(layers, Hkv, Hq, D, len(lens), pages, max(lens) + 64, mask, S, W, device=cuda_device)
+    seqs = []
+    for i, n in enumerate(lens):
+        s = Seq(cache, 300 + i, max(lens) + 64)
+        s.prefill(n, cuda_device)
+        seqs.append(s)
+    slots = [s.slot for s in seqs]
+    out = torch.empty((layers, len(seqs), Hq, D), dtype=torch.float32, device=cuda_device)
+    for step in range(steps):
+        ks = torch.stack([torch.cat([s.rows(l, s.n, s.n + 1, 0) for s in seqs]) for l in range(layers)])
+        vs = torch.stack([torch.cat([s.rows(l, s.n, s.n + 1, 1) for s in seqs]) for l in range(layers)])
+        q = rand_bf16((layers, len(seqs), Hq, D), 2000 + step)
+        rl.rlkv_paged_step(cache.handle, slots, ks.to(cuda_device), vs.to(cuda_device), q.to(cuda_device), out)
+        for i, s in enumerate(seqs):
+            for l in range(layers):
+                assert s.oracle.append(l, ks[l, i], vs[l, i]) == 0
+            s.n += 1
+        got = out.cpu().numpy()
+        for l in range(layers):
+            for i, s in enumerate(seqs):
+                check_out(got[l, i], s.oracle.decode(l, q[l, i:i + 1])[0])
+    check_state(cache, seqs)
+    assert cache.pages()[0] == pages - sum((s.n + 63) // 64 for s in seqs)
+    # a sequence that is ahead in one layer cannot take part in a whole step
+    k1 = rand_bf16((1, Hkv, D), 5).to(cuda_device)
+    cache.append(0, [slots[0]], k1, k1)
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_paged_step(cache.handle, slots, ks.to(cuda_device), vs.to(cuda_device), q.to(cuda_device), out)
+    assert e.value.code == rl.RLKV_EINVAL
+    assert cache.status() == 0
+    cache.close()
