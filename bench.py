@@ -452,8 +452,8 @@ def run_ours(args, w, mask):
         spread = [max(1, int(round(n * (0.25 + 1.5 * i / max(1, w.batch - 1))))) for i in range(w.batch)]
         paged = {"workload": f"first {pl} layers of the {w.name} mask, {w.batch} sequences, launches back to back"}
         for name, lens in (("uniform", [n] * w.batch), ("ragged", spread)):
-            pages = sum((x + 63) // 64 for x in lens) + 2
-            pc = harness.PagedCache(pl, w.kv_heads, w.q_heads, w.head_dim, w.batch, pages, max(lens) + 64, pmask,
+            pages = sum((x + 63) // 64 for x in lens) + 2 + 2 * len(lens)
+            pc = harness.PagedCache(pl, w.kv_heads, w.q_heads, w.head_dim, w.batch, pages, max(lens) + 128, pmask,
                                     w.sink, w.window, device=dev)
             slots = [pc.open_seq() for _ in lens]
             for i, x in enumerate(lens):
@@ -478,6 +478,21 @@ def run_ours(args, w, mask):
             nbytes = sum(pc.step_bytes(l, slots) for l in range(pl)) / pl
             paged[name] = {"launch_us": us, "algorithmic_bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
                            "lengths": [min(lens), max(lens)], "launches_timed": reps * pl}
+            # the same layers through rlkv_paged_step (one token appended per step, launches overlapped)
+            kk, vv = steps_in[0][0][:pl].contiguous(), steps_in[0][1][:pl].contiguous()
+            qq = q[:pl].contiguous()
+            for i in range(3):
+                rl.rlkv_paged_step(pc.handle, slots, kk, vv, qq, pout, stream)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for i in range(reps):
+                rl.rlkv_paged_step(pc.handle, slots, kk, vv, qq, pout, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = 1e3 * e0.elapsed_time(e1) / (reps * pl)
+            nbytes = sum(pc.step_bytes(l, slots) for l in range(pl)) / pl
+            paged[name]["in_step_us_per_layer"] = us
+            paged[name]["in_step_gbs"] = nbytes / (us * 1e-6) / 1e9
             if pc.status() != 0:
                 raise SystemExit("a paged decode kernel reported a status: results are invalid")
             pc.close()
