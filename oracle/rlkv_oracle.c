@@ -53,6 +53,9 @@ typedef struct {
     uint16_t **k, **v;       /* [layers*batch*kv_heads] -> rows*head_dim bf16 bits */
     int32_t **token_of_slot; /* compressed heads: [cap], -1 = empty; NULL for full heads */
     int threads;
+    /* 8-bit storage of the full heads (rlkv_oracle_set_fp8): their k, v entries hold E4M3 codes */
+    int fp8;
+    float *k_scale, *v_scale; /* [layers*kv_heads] */
 } oracle_t;
 
 static float bf16_to_float(uint16_t b)
@@ -61,6 +64,44 @@ static float bf16_to_float(uint16_t b)
     float f;
     memcpy(&f, &u, sizeof f);
     return f;
+}
+
+/* ---- 8-bit K/V for the full heads (the paper's Limitations and Future Work: head-level
+ * compression "can be combined with" KV-cache quantisation; no format is given there).
+ * Reading taken: the OCP 8-bit floating-point format E4M3 -- 1 sign bit, 4 exponent bits with bias
+ * 7, 3 mantissa bits; exponent field 0 holds the subnormals m/8 * 2^-6; there are no infinities and
+ * only exponent 15 with mantissa 7 is NaN, so the largest finite value is 1.75 * 2^8 = 448 -- with
+ * one scale per (layer, KV head) for K and one for V, given by the caller:
+ *     code  = E4M3( fl32( fl32(x) * fl32(1 / scale) ) )    round to nearest, ties to even,
+ *                                                           magnitudes above 448 saturate to 448
+ *     x_hat = value(code) * scale
+ * and attention runs on x_hat as before.  Compressed heads keep their 16-bit rows.
+ * Pins: every code's value against torch.float8_e4m3fn; the encoder against torch's cast on a
+ * sweep that holds every midpoint between neighbouring codes; closed forms. */
+float rlkv_oracle_e4m3_value(uint8_t code)
+{
+    int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    float mag;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) mag = ldexpf((float)m / 8.0f, -6);
+    else mag = ldexpf(1.0f + (float)m / 8.0f, e - 7);
+    return sign ? -mag : mag;
+}
+
+/* Nearest code by search over the 127 finite magnitudes (they grow with the code). */
+uint8_t rlkv_oracle_e4m3_encode(float x)
+{
+    if (x != x) return 0x7f;
+    uint8_t sign = signbit(x) ? 0x80 : 0;
+    double a = fabs((double)x);
+    if (a >= 448.0) return sign | 0x7e;
+    int lo = 0;
+    for (int c = 0; c <= 0x7e; ++c)
+        if ((double)rlkv_oracle_e4m3_value((uint8_t)c) <= a) lo = c;
+    double below = a - (double)rlkv_oracle_e4m3_value((uint8_t)lo);
+    double above = (double)rlkv_oracle_e4m3_value((uint8_t)(lo + 1)) - a;
+    int c = below < above ? lo : (above < below ? lo + 1 : ((lo & 1) ? lo + 1 : lo));
+    return sign | (uint8_t)c;
 }
 
 static size_t unit_index(const oracle_t *o, int layer, int b, int h)
@@ -91,6 +132,8 @@ void rlkv_oracle_destroy(oracle_t *o)
     free(o->token_of_slot);
     free(o->is_full);
     free(o->len);
+    free(o->k_scale);
+    free(o->v_scale);
     free(o);
 }
 
@@ -133,6 +176,37 @@ oracle_t *rlkv_oracle_create(int layers, int kv_heads, int q_heads, int head_dim
     return o;
 }
 
+/* Switches the full heads to 8-bit storage.  k_scale, v_scale: [layers*kv_heads], positive and finite.
+ * Only while the cache is empty.  Returns 0, -7 otherwise. */
+int rlkv_oracle_set_fp8(oracle_t *o, const float *k_scale, const float *v_scale)
+{
+    size_t heads = (size_t)o->layers * o->kv_heads;
+    for (int l = 0; l < o->layers; ++l)
+        if (o->len[l] != 0) return -7;
+    for (size_t i = 0; i < heads; ++i)
+        if (!(k_scale[i] > 0) || !(v_scale[i] > 0) || isinf(k_scale[i]) || isinf(v_scale[i])) return -7;
+    free(o->k_scale);
+    free(o->v_scale);
+    o->k_scale = malloc(heads * sizeof(float));
+    o->v_scale = malloc(heads * sizeof(float));
+    if (!o->k_scale || !o->v_scale) return -4;
+    memcpy(o->k_scale, k_scale, heads * sizeof(float));
+    memcpy(o->v_scale, v_scale, heads * sizeof(float));
+    o->fp8 = 1;
+    return 0;
+}
+
+/* The 16 stored bits of one element as a number: a bf16 value, or for a full head in 8-bit storage
+ * the E4M3 code's value times the head's scale. */
+static acc_t stored(const oracle_t *o, int layer, int h, uint16_t bits, int is_v)
+{
+    if (o->fp8 && o->is_full[layer * o->kv_heads + h]) {
+        float scale = (is_v ? o->v_scale : o->k_scale)[layer * o->kv_heads + h];
+        return (acc_t)rlkv_oracle_e4m3_value((uint8_t)bits) * (acc_t)scale;
+    }
+    return (acc_t)bf16_to_float(bits);
+}
+
 void rlkv_oracle_set_threads(oracle_t *o, int threads) { o->threads = threads < 1 ? 1 : threads; }
 
 int rlkv_oracle_length(const oracle_t *o, int layer)
@@ -166,6 +240,14 @@ int rlkv_oracle_append(oracle_t *o, int layer, const uint16_t *k, const uint16_t
             } else {
                 row = slot_of_token(o, t);
                 o->token_of_slot[u][row] = t;
+            }
+            if (o->fp8 && o->is_full[layer * o->kv_heads + h]) {
+                float ik = 1.0f / o->k_scale[layer * o->kv_heads + h], iv = 1.0f / o->v_scale[layer * o->kv_heads + h];
+                for (int d = 0; d < D; ++d) {
+                    o->k[u][(size_t)row * D + d] = rlkv_oracle_e4m3_encode(bf16_to_float(ks[d]) * ik);
+                    o->v[u][(size_t)row * D + d] = rlkv_oracle_e4m3_encode(bf16_to_float(vs[d]) * iv);
+                }
+                continue;
             }
             memcpy(o->k[u] + (size_t)row * D, ks, D * sizeof(uint16_t));
             memcpy(o->v[u] + (size_t)row * D, vs, D * sizeof(uint16_t));
@@ -217,7 +299,7 @@ static void attend_one(const oracle_t *o, int layer, int b, int j, const uint16_
     for (int i = 0; i < cnt; ++i) {
         const uint16_t *kr = o->k[u] + (size_t)rows[i] * D;
         acc_t dot = 0;
-        for (int d = 0; d < D; ++d) dot += (acc_t)bf16_to_float(qj[d]) * (acc_t)bf16_to_float(kr[d]);
+        for (int d = 0; d < D; ++d) dot += (acc_t)bf16_to_float(qj[d]) * stored(o, layer, h, kr[d], 0);
         s[i] = dot * scale;
         if (s[i] > m) m = s[i];
     }
@@ -230,7 +312,7 @@ static void attend_one(const oracle_t *o, int layer, int b, int j, const uint16_
     float *oj = out + ((size_t)b * o->q_heads + j) * D;
     for (int d = 0; d < D; ++d) {
         acc_t a = 0;
-        for (int i = 0; i < cnt; ++i) a += s[i] * (acc_t)bf16_to_float(o->v[u][(size_t)rows[i] * D + d]);
+        for (int i = 0; i < cnt; ++i) a += s[i] * stored(o, layer, h, o->v[u][(size_t)rows[i] * D + d], 1);
         oj[d] = (float)(a / l);
     }
 }
@@ -314,6 +396,7 @@ int rlkv_oracle_decode_mixed(const oracle_t *o, int layer, const uint16_t *q, co
     if (layer < 0 || layer >= o->layers) return -2;
     int n = o->len[layer], D = o->head_dim, G = o->q_heads / o->kv_heads;
     if (n < 1) return -3;
+    if (o->fp8) return -7; /* the training-time form keeps 16-bit rows */
     for (int h = 0; h < o->kv_heads; ++h) {
         if (!o->is_full[layer * o->kv_heads + h]) return -5;
         if (!(alpha[h] >= 0.0f && alpha[h] <= 1.0f)) return -6;

@@ -58,6 +58,12 @@ def _lib(acc: str) -> ctypes.CDLL:
         lib.rlkv_oracle_retained.argtypes = [vp, ci, ci]
         lib.rlkv_oracle_export_head.restype = ci
         lib.rlkv_oracle_export_head.argtypes = [vp, ci, ci, ci, vp, vp, vp]
+        lib.rlkv_oracle_set_fp8.restype = ci
+        lib.rlkv_oracle_set_fp8.argtypes = [vp, vp, vp]
+        lib.rlkv_oracle_e4m3_value.restype = ctypes.c_float
+        lib.rlkv_oracle_e4m3_value.argtypes = [ctypes.c_uint8]
+        lib.rlkv_oracle_e4m3_encode.restype = ctypes.c_uint8
+        lib.rlkv_oracle_e4m3_encode.argtypes = [ctypes.c_float]
         lib.rlkv_oracle_max_threads.restype = ci
         lib.rlkv_oracle_acc_bytes.restype = ci
         assert lib.rlkv_oracle_acc_bytes() == (4 if acc == "f32" else 8)
@@ -67,6 +73,16 @@ def _lib(acc: str) -> ctypes.CDLL:
 
 def max_threads() -> int:
     return int(_lib("f32").rlkv_oracle_max_threads())
+
+
+def e4m3_value(code: int) -> float:
+    """Value of an OCP E4M3 code (nan for 0x7f / 0xff)."""
+    return float(_lib("f32").rlkv_oracle_e4m3_value(int(code) & 0xff))
+
+
+def e4m3_encode(x: float) -> int:
+    """Nearest E4M3 code of a float32 (ties to even, saturating at +-448, NaN -> 0x7f)."""
+    return int(_lib("f32").rlkv_oracle_e4m3_encode(float(np.float32(x))))
 
 
 def _bits(a) -> np.ndarray:
@@ -112,6 +128,18 @@ class Oracle:
     def set_threads(self, threads: int) -> None:
         self.threads = int(threads)
         self._lib.rlkv_oracle_set_threads(self._h, int(threads))
+
+    def set_fp8(self, k_scale, v_scale) -> None:
+        """Full heads store E4M3 codes from now on (only while the cache is empty).  k_scale,
+        v_scale: [layers][kv_heads] positive floats."""
+        ks = np.ascontiguousarray(np.asarray(k_scale, dtype=np.float32).reshape(-1))
+        vs = np.ascontiguousarray(np.asarray(v_scale, dtype=np.float32).reshape(-1))
+        if ks.size != self.layers * self.kv_heads or vs.size != ks.size:
+            raise ValueError("k_scale, v_scale must have layers*kv_heads entries")
+        rc = self._lib.rlkv_oracle_set_fp8(self._h, ks.ctypes.data, vs.ctypes.data)
+        if rc != 0:
+            raise RuntimeError(f"rlkv_oracle_set_fp8 failed: {rc}")
+        self.fp8 = True
 
     def length(self, layer: int) -> int:
         return int(self._lib.rlkv_oracle_length(self._h, layer))

@@ -399,3 +399,79 @@ def test_mixed_refuses_compressed_heads_and_gates_outside_the_unit_interval():
     for bad in ([1.5, 0.5], [0.5, -0.1], [float("nan"), 0.5]):
         with pytest.raises(RuntimeError, match="-6"):
             o.decode_mixed(0, q, bad)
+
+
+# ---------------------------------------------------------------------------- 8-bit K/V (E4M3)
+def test_e4m3_values_of_all_codes_match_the_library_type():
+    from oracle.rlkv_oracle import e4m3_value
+    codes = torch.arange(256, dtype=torch.uint8)
+    want = codes.view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    got = np.array([e4m3_value(int(c)) for c in codes], dtype=np.float32)
+    assert np.isnan(got[[0x7f, 0xff]]).all() and np.isnan(want[[0x7f, 0xff]]).all()
+    ok = ~np.isnan(want)
+    np.testing.assert_array_equal(got[ok], want[ok])
+    # what the format's definition fixes, written out: largest finite, smallest normal, smallest subnormal
+    assert e4m3_value(0x7e) == 448.0 and e4m3_value(0x08) == 2.0 ** -6 and e4m3_value(0x01) == 2.0 ** -9
+    assert e4m3_value(0x38) == 1.0 and e4m3_value(0xb8) == -1.0 and e4m3_value(0x80) == 0.0
+
+
+def test_e4m3_encoder_matches_the_library_cast_on_every_code_midpoint_and_neighbour():
+    """Every representable value, every midpoint between neighbours (the ties) and points just beside
+    them, both signs, against torch's float32 -> float8_e4m3fn cast, which rounds to nearest even.
+    Above 464 torch's cast gives NaN where this format's users saturate: there the reading (448) is
+    checked as such."""
+    from oracle.rlkv_oracle import e4m3_encode, e4m3_value
+    vals = np.array([e4m3_value(c) for c in range(0x7f)], dtype=np.float64)
+    pts = [vals, (vals[:-1] + vals[1:]) / 2]
+    pts += [np.nextafter(p.astype(np.float32), np.float32(np.inf)).astype(np.float64) for p in list(pts)]
+    pts += [np.nextafter(p.astype(np.float32), np.float32(-np.inf)).astype(np.float64) for p in pts[:2]]
+    x = np.concatenate(pts + [np.array([449.0, 463.9, 464.0, 1e-12, 0.3, 0.7, 3.14159, 100.0, 447.9])])
+    x = np.concatenate([x, -x]).astype(np.float32)
+    x = x[np.abs(x) <= 464.0]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = np.array([e4m3_encode(float(v)) for v in x], dtype=np.uint8)
+    zero = (want & 0x7f) == 0                                  # +0 / -0: compare the magnitude only
+    np.testing.assert_array_equal(got[~zero], want[~zero])
+    assert ((got[zero] & 0x7f) == 0).all()
+    for big in (464.1, 480.0, 1e6, 3e38):
+        assert e4m3_encode(big) == 0x7e and e4m3_encode(-big) == 0xfe
+    assert e4m3_encode(float("nan")) == 0x7f
+    # decoding an encoded code gives the code back
+    for c in list(range(0x7f)) + list(range(0x81, 0xff)):
+        assert e4m3_encode(e4m3_value(c)) == c
+
+
+def test_fp8_full_heads_equal_plain_attention_over_the_dequantised_rows():
+    """With 8-bit storage the oracle must give exactly what the 16-bit oracle gives on rows that were
+    quantised and dequantised beforehand with the library type (values chosen so that x_hat is a
+    bf16 number: scale a power of two); compressed heads are untouched."""
+    Hq, Hkv, D, B, S, W, n = 8, 2, 32, 2, 4, 12, 90
+    K, V, q = rand_bf16((n, B, Hkv, D), 301), rand_bf16((n, B, Hkv, D), 302), rand_bf16((B, Hq, D), 303)
+    ks, vs = np.array([0.5, 2.0], np.float32), np.array([0.25, 1.0], np.float32)
+    a = Oracle(1, Hkv, Hq, D, B, n, [1, 0], S, W)
+    a.set_fp8(ks, vs)
+    fill(a, 0, K, V)
+
+    def roundtrip(x, scale):      # e4m3 has 3 mantissa bits: value * 2^k is exact in bf16
+        return ((x.float() / scale).to(torch.float8_e4m3fn).float() * scale).to(torch.bfloat16)
+
+    K2, V2 = K.clone(), V.clone()
+    K2[:, :, 0], V2[:, :, 0] = roundtrip(K[:, :, 0], 0.5), roundtrip(V[:, :, 0], 0.25)
+    b = Oracle(1, Hkv, Hq, D, B, n, [1, 0], S, W)
+    fill(b, 0, K2, V2)
+    np.testing.assert_array_equal(a.decode(0, q), b.decode(0, q))
+    # the full head's stored entries are the codes; the compressed head's rows are the bf16 bits
+    k_codes, v_codes, _ = a.export_head(0, 1, 0)
+    want = (K[:, 1, 0].float() / 0.5).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    np.testing.assert_array_equal(k_codes[:n], want)
+    assert np.abs(a.decode(0, q) - Oracle_decode_plain(K, V, q, Hkv, Hq, D, B, n, S, W)).max() > 1e-4   # it does quantise
+    with pytest.raises(RuntimeError, match="-7"):
+        a.set_fp8(ks, vs)                                       # only while empty
+    with pytest.raises(RuntimeError, match="-7"):
+        Oracle(1, Hkv, Hq, D, B, n, [1, 0], S, W).set_fp8([0.0, 1.0], vs)
+
+
+def Oracle_decode_plain(K, V, q, Hkv, Hq, D, B, n, S, W):
+    o = Oracle(1, Hkv, Hq, D, B, n, [1, 0], S, W)
+    fill(o, 0, K, V)
+    return o.decode(0, q)
