@@ -189,6 +189,25 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
                       int max_seqs, int n_pages, int max_seq_len, const uint8_t* head_is_full,
                       int sink, int window, void* device_buf, size_t device_buf_bytes);
 int rlkv_paged_destroy(rlkv_paged* cache);
+/* The paged cache with the full heads' pages held in 8 bits.  (The paper names KV-cache quantisation
+ * as the direction to combine head-level compression with and fixes no format; this is the format
+ * taken.)  Every K and V element of a full head is stored as an OCP E4M3 code (1 sign, 4 exponent bits
+ * with bias 7, 3 mantissa bits, largest finite value 448, no infinities):
+ *     code = E4M3(x * (1 / scale))   round to nearest even, magnitudes above 448 saturate;
+ *     attention then runs on value(code) * scale
+ * with one scale per (layer, KV head) for K and one for V: k_scale, v_scale, HOST float
+ * [layers][kv_heads], positive and finite, copied (a scale of max|x| / 448 uses the whole range;
+ * 1 is fine for activations of order one).  The full heads then cost half the bytes per token, to
+ * store and to read; compressed heads keep their 16-bit rings.  head_dim must be 128.  Every other
+ * call works as on a cache from rlkv_paged_create; rlkv_paged_debug_export_head returns a full
+ * head's codes, one per 16-bit element. */
+int rlkv_paged_size_fp8(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                        int max_seq_len, const uint8_t* head_is_full, int sink, int window,
+                        size_t* bytes_out);
+int rlkv_paged_create_fp8(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim,
+                          int max_seqs, int n_pages, int max_seq_len, const uint8_t* head_is_full,
+                          int sink, int window, const float* k_scale, const float* v_scale,
+                          void* device_buf, size_t device_buf_bytes);
 /* Takes a free request slot (length 0 in every layer): RLKV_EFULL if all max_seqs are open. */
 int rlkv_paged_seq_open(rlkv_paged* cache, int* slot_out);
 /* Closes a slot: its pages go back to the free list.  The caller makes sure no work that uses the

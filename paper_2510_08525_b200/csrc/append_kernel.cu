@@ -6,6 +6,8 @@
 // the first `sink` tokens and the most recent `window` tokens (paper, Section 4.3 and Appendix B).
 // In a bulk append only the tokens that survive the whole batch of appends are written, so no two
 // threads ever target the same row and the result equals n successive single appends bit for bit.
+#include <cuda_fp8.h>
+
 #include "rlkv_internal.cuh"
 
 namespace rlkv {
@@ -110,6 +112,28 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
             n_comp = a.layers[l].n_comp;
         }
         long long row;
+        if (slot >= 0 && a.pool8) {
+            // 8-bit pages: code = E4M3(x * (1 / scale)), round to nearest even, saturating.  A page is
+            // the K codes [64 tokens][128] followed by the V codes transposed [128][64 tokens].
+            const long long page0 = a.n_layers > 1 ? a.layers[l].page0_8 : a.page0_8;
+            unsigned char* pg = a.pool8 + (page0 + (long long)slot * a.n_pages + page) * (2 * kTile * 128);
+            const float inv = (kv ? a.v_inv : a.k_inv)[l * a.kv_heads + h];
+            const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.n + e) * a.kv_heads + h) * a.head_dim + c * 8;
+            const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src));
+            const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(&bits);
+            alignas(8) unsigned char code[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                code[j] = (unsigned char)__nv_cvt_float_to_fp8(__bfloat162float(x[j]) * inv, __NV_SATFINITE, __NV_E4M3);
+            if (kv == 0) {
+                *reinterpret_cast<uint2*>(pg + (t % kTile) * 128 + c * 8) = *reinterpret_cast<const uint2*>(code);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) pg[kTile * 128 + (c * 8 + j) * kTile + t % kTile] = code[j];
+            }
+            if (slot == 0 && c == 0 && kv == 0) a.page_table[(size_t)seq * a.table_stride + t / kTile] = page;
+            continue;
+        }
         if (slot >= 0) {
             row = full_row0 + (((long long)slot * a.n_pages + page) * 2 + kv) * kTile + t % kTile;
             if (slot == 0 && c == 0 && kv == 0) a.page_table[(size_t)seq * a.table_stride + t / kTile] = page;

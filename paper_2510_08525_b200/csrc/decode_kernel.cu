@@ -26,6 +26,8 @@
 // adapters (paper, Eq. 1: a second class of "local" units over the sink and window rows, both
 // classes adding their weighted result), and the paged cache (one length per sequence, full-head
 // rows looked up in a page table); see the notes above decode_kernel.
+#include <cuda_fp16.h>
+
 #include "rlkv_internal.cuh"
 
 namespace rlkv {
@@ -155,6 +157,32 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Four E4M3 codes (one 32-bit register, lowest byte first) as two f16x2 registers: codes 0, 1 and
+// codes 2, 3.  Every E4M3 value is an f16 value, so the conversion is exact.
+__device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t codes, uint32_t& lo, uint32_t& hi)
+{
+    asm volatile(
+        "{\n\t.reg .b16 a, b;\n\t"
+        "mov.b32 {a, b}, %2;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
+        "cvt.rn.f16x2.e4m3x2 %1, b;\n\t}"
+        : "=r"(lo), "=r"(hi)
+        : "r"(codes));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
+{
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -238,7 +266,7 @@ struct Smem {
         return (size_t)stages * stage_bytes(group) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
-               (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged ? kPagedBytes : 0);
+               (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0);
     }
 };
 
@@ -374,6 +402,10 @@ template <>
 struct ExtraArgs<kModePaged> {
     typedef PagedArgs type;
 };
+template <>
+struct ExtraArgs<kModePagedFp8> {
+    typedef PagedFp8Args type;  // starts with a PagedArgs
+};
 
 template <int D, int NG, int MODE>
 __global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
@@ -381,7 +413,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
               const __grid_constant__ typename ExtraArgs<MODE>::type extra)
 {
     constexpr bool MIXED = MODE == kModeMixed;
-    constexpr bool PAGED = MODE == kModePaged;
+    constexpr bool PAGED = MODE == kModePaged || MODE == kModePagedFp8;
+    constexpr bool FP8 = MODE == kModePagedFp8;  // the full heads' pages hold E4M3 codes (head_dim 128 only)
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     constexpr int MS = S::kMergeStride;
@@ -518,6 +551,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     u = locate<MODE>(a, x, pg);
                     seg_tiles = min(x1 - x, u.pos.run);
                     const bool local_unit = MIXED && u.pos.uid >= sc.U;
+                    const bool fp8_unit = FP8 && u.pos.uid < sc.U;  // a full head whose pages hold E4M3 codes
                     int seg_eff = seg_tiles;  // tiles of the segment that exist
                     if (PAGED) {
                         seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
@@ -552,6 +586,23 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             int row;
                             local_tile(a, u.pos.tile + i, row, valid);
                         }
+                        if (FP8 && fp8_unit && !have_q) {
+                            // the contraction index may be permuted as long as both operands agree: against
+                            // codes fetched four consecutive d per lane, Q goes in as f16 with k-halves
+                            // (d 4tq, 4tq+1) and (d 4tq+2, 4tq+3) of every 16
+                            const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
+                                                            stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
+                                                        quad * D + 4 * tq;
+#pragma unroll
+                            for (int ks = 0; ks < KS; ++ks) {
+                                const uint2 raw = quad < G ? *reinterpret_cast<const uint2*>(qrow + ks * 16) : make_uint2(0u, 0u);
+                                const float2 f0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                                const float2 f1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                                qa[ks][0] = pack_f16(f0.x, f0.y);
+                                qa[ks][1] = pack_f16(f1.x, f1.y);
+                            }
+                            have_q = true;
+                        }
                         if (!have_q) {
                             const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
                                                             stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
@@ -563,7 +614,80 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             }
                             have_q = true;
                         }
-                        if (wig * 16 < valid) {
+                        if (FP8 && fp8_unit) {
+                            if (wig * 16 < valid) {
+                                // a stage of an 8-bit page: K codes [64 tokens][128 B] with the 128-byte swizzle,
+                                // then V codes transposed [128 d][64 B] with the 64-byte swizzle
+                                const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
+                                const uint32_t sV = sK + kTile * 128;
+                                // ---- S = Q.K^T.  ldmatrix row i of token set s is token 4(i/2) + 2s + (i%2) of
+                                // the warp's 16, so that this lane ends up with four consecutive tokens
+                                const int lj = lane >> 3, li = lane & 7;
+                                const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
+                                float sA[4] = {0.f, 0.f, 0.f, 0.f}, sB[4] = {0.f, 0.f, 0.f, 0.f};
+                                float sA2[4] = {0.f, 0.f, 0.f, 0.f}, sB2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                                for (int kp = 0; kp < KS / 2; ++kp) {
+                                    const int chunk = 2 * kp + (lj >> 1);  // 16 codes along d
+                                    uint32_t r0, r1, r2, r3, b0, b1;
+                                    ldmatrix_x4(sK + ktok * 128 + ((chunk ^ (ktok & 7)) << 4), r0, r1, r2, r3);
+                                    e4m3x4_to_f16x2x2(r0, b0, b1);
+                                    mma_f16(sA, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
+                                    e4m3x4_to_f16x2x2(r1, b0, b1);
+                                    mma_f16(sB, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
+                                    e4m3x4_to_f16x2x2(r2, b0, b1);
+                                    mma_f16(sA2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                    e4m3x4_to_f16x2x2(r3, b0, b1);
+                                    mma_f16(sB2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                }
+                                // this lane: head `quad`, tokens wig*16 + 4tq + {0, 1, 2, 3}; K's scale joins the softmax scale
+                                const float sl2 = a.scale_log2 * pg->k_scale[u.head];
+                                float sc4[4];
+                                sc4[0] = (sA[0] + sA2[0]) * sl2;
+                                sc4[1] = (sA[1] + sA2[1]) * sl2;
+                                sc4[2] = (sB[0] + sB2[0]) * sl2;
+                                sc4[3] = (sB[1] + sB2[1]) * sl2;
+                                const int tok0 = wig * 16 + 4 * tq;
+                                if (tok0 >= valid) sc4[0] = -INFINITY;
+                                if (tok0 + 1 >= valid) sc4[1] = -INFINITY;
+                                if (tok0 + 2 >= valid) sc4[2] = -INFINITY;
+                                if (tok0 + 3 >= valid) sc4[3] = -INFINITY;
+                                float mx = fmaxf(fmaxf(sc4[0], sc4[1]), fmaxf(sc4[2], sc4[3]));
+                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                                const float m_new = fmaxf(m_run, mx);
+                                const float corr = exp2f(m_run - m_new);
+                                const float p0 = exp2f(sc4[0] - m_new), p1 = exp2f(sc4[1] - m_new);
+                                const float p2 = exp2f(sc4[2] - m_new), p3 = exp2f(sc4[3] - m_new);
+                                l_run = l_run * corr + ((p0 + p1) + (p2 + p3));
+                                m_run = m_new;
+                                const float ca = __shfl_sync(0xffffffffu, corr, tq * 8);
+                                const float cb = __shfl_sync(0xffffffffu, corr, tq * 8 + 4);
+                                const uint32_t pb0 = pack_f16(p0, p1), pb1 = pack_f16(p2, p3);
+                                // ---- O^T[d][head] += V^T[d][tok] . P^T[tok][head]: V^T rows come straight out of
+                                // the transposed page, four consecutive tokens per lane
+#pragma unroll
+                                for (int mp = 0; mp < KS / 2; ++mp) {
+                                    const int vd = 16 * (2 * mp + (lj >> 1)) + 8 * (lj & 1) + li;
+                                    uint32_t r0, r1, r2, r3, a0, a1, a2, a3;
+                                    ldmatrix_x4(sV + vd * 64 + ((wig ^ ((vd >> 1) & 3)) << 4), r0, r1, r2, r3);
+                                    e4m3x4_to_f16x2x2(r0, a0, a2);
+                                    e4m3x4_to_f16x2x2(r1, a1, a3);
+                                    acc[2 * mp][0] *= ca;
+                                    acc[2 * mp][1] *= cb;
+                                    acc[2 * mp][2] *= ca;
+                                    acc[2 * mp][3] *= cb;
+                                    mma_f16(acc[2 * mp], a0, a1, a2, a3, pb0, pb1);
+                                    e4m3x4_to_f16x2x2(r2, a0, a2);
+                                    e4m3x4_to_f16x2x2(r3, a1, a3);
+                                    acc[2 * mp + 1][0] *= ca;
+                                    acc[2 * mp + 1][1] *= cb;
+                                    acc[2 * mp + 1][2] *= ca;
+                                    acc[2 * mp + 1][3] *= cb;
+                                    mma_f16(acc[2 * mp + 1], a0, a1, a2, a3, pb0, pb1);
+                                }
+                            }
+                        } else if (wig * 16 < valid) {
                             const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
                             const uint32_t sV = sK + S::kTileBytes;
                             // ---- S = Q.K^T for this warp's 16 tokens (two 8-token column blocks)
@@ -637,6 +761,16 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 float* merge = reinterpret_cast<float*>(buf);
                 float* stat_m = merge + S::merge_floats(G);
                 float* stat_l = stat_m + S::kWarps * kMaxGroup;
+                if (FP8 && item >= 0 && u.pos.uid < sc.U) {  // the rows were value(code): V's scale goes in here
+                    const float vs = pg->v_scale[u.head];
+#pragma unroll
+                    for (int mt = 0; mt < KS; ++mt) {
+                        acc[mt][0] *= vs;
+                        acc[mt][1] *= vs;
+                        acc[mt][2] *= vs;
+                        acc[mt][3] *= vs;
+                    }
+                }
                 if (item >= 0) {
                     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
                     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -802,7 +936,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 }
                                 ppar ^= 1u;
                                 page_base = first;
-                                paged_row0 = (int)(a.full_row0 + (long long)(u.pos.uid - u.b * a.n_full) * pg->n_pages * 2 * kTile);
+                                // 16-bit pages: the first pool row of the head's pages; 8-bit pages: its first page
+                                paged_row0 = FP8 ? pg->page0_8 + (u.pos.uid - u.b * a.n_full) * pg->n_pages
+                                                 : (int)(a.full_row0 + (long long)(u.pos.uid - u.b * a.n_full) * pg->n_pages * 2 * kTile);
                             } else {
                                 paged_row0 = -1;
                                 const int c = u.pos.uid - sc.U - u.b * a.n_comp;
@@ -833,8 +969,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         }
                     }
                     if (PAGED && paged_row0 >= 0) {
-                        krow = paged_row0 + s_pages[paged_tile++ - page_base] * (2 * kTile);
-                        vrow = krow + kTile;
+                        if (FP8) {  // the page itself; its row coordinates in the two 8-bit maps follow below
+                            krow = paged_row0 + s_pages[paged_tile++ - page_base];
+                        } else {
+                            krow = paged_row0 + s_pages[paged_tile++ - page_base] * (2 * kTile);
+                            vrow = krow + kTile;
+                        }
                     }
                     if (MIXED && local_row0 >= 0) {
                         int row, valid;
@@ -849,10 +989,19 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     const uint32_t fb = smem_u32(full_bar + s);
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
                     const long long tc0 = trace ? clock64() : 0;
-                    mbar_expect_tx(fb, S::kTilePairBytes + (with_q ? G * D * 2 : 0));
+                    const bool page8 = FP8 && paged_row0 >= 0;  // a 16 KB page of codes instead of two 16-bit tiles
+                    mbar_expect_tx(fb, (page8 ? S::kTilePairBytes / 2 : S::kTilePairBytes) + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
                     const long long tc1 = trace ? clock64() : 0;
-                    if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
+                    if constexpr (FP8) {
+                        if (page8) {  // a page is 128 rows of the K map (64 of them K codes) and 256 rows of the V map
+                            tma_load_2d(dst, &extra.map_k, 0, krow * 128, fb, stream_policy);
+                            tma_load_2d(dst + kTile * 128, &extra.map_v, 0, krow * 256 + 128, fb, stream_policy);
+                        } else {
+                            tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
+                            tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
+                        }
+                    } else if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
                         tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
                         tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
                     } else {         // one contiguous 8 KB box per tile: [64 rows][64]
@@ -1113,6 +1262,11 @@ cudaError_t prepare_one()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(decode_kernel<D, NG, kModeMixed>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
     if (e != cudaSuccess) return e;
+    if (D == 128 && NG == 2) {  // 8-bit pages: head_dim 128, two consumer groups only
+        e = cudaFuncSetAttribute(decode_kernel<128, 2, kModePagedFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kMaxDynamicSmem);
+        if (e != cudaSuccess) return e;
+    }
     return cudaFuncSetAttribute(decode_kernel<D, NG, kModePaged>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 kMaxDynamicSmem);
 }
@@ -1151,9 +1305,14 @@ static cudaError_t launch_either(const DecodeArgs& a, const CUtensorMap& tmap, i
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
-                          int stages, int groups, cudaStream_t stream, bool overlap, int mode, const PagedArgs* paged)
+                          int stages, int groups, cudaStream_t stream, bool overlap, int mode, const PagedArgs* paged,
+                          const PagedFp8Args* paged8)
 {
     if (mode == kModePaged && !paged) return cudaErrorInvalidValue;
+    if (mode == kModePagedFp8) {
+        if (!paged8 || head_dim != 128 || groups != 2) return cudaErrorInvalidValue;
+        return launch_one<128, 2, kModePagedFp8>(a, *tmap, grid, stages, stream, overlap, *paged8);
+    }
     if (head_dim == 128) {
         if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged);
         if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged);

@@ -112,4 +112,30 @@ inline int encode_pool_tensor_map(CUtensorMap* tmap, void* base, long long rows,
     return RLKV_OK;
 }
 
+// Tensor map over `rows` rows of row_bytes (64 or 128) bytes at `base`, boxes of box_rows whole rows,
+// swizzled over the row width: the two views of the paged cache's 8-bit pool.
+inline int encode_byte_rows_tensor_map(CUtensorMap* tmap, void* base, int row_bytes, long long rows, int box_rows)
+{
+    typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    RLKV_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (!fn || q != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)row_bytes, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+        tmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(g_cuda_text, sizeof g_cuda_text, "cuTensorMapEncodeTiled (8-bit pool) failed with CUresult %d", (int)r);
+        return RLKV_ECUDA;
+    }
+    return RLKV_OK;
+}
+
 }  // namespace rlkv

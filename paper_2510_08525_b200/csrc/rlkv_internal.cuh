@@ -44,7 +44,8 @@ enum : int {
 enum : int {
     kModePlain = 0,   // the lock-step cache: full and compressed heads, one length for the whole batch
     kModeMixed = 1,   // mixed attention (Eq. 1) over a lock-step cache whose heads are all full
-    kModePaged = 2    // the paged cache: one length per sequence, full heads in 64-token pages
+    kModePaged = 2,   // the paged cache: one length per sequence, full heads in 64-token pages
+    kModePagedFp8 = 3 // the paged cache with the full heads' pages held as 8-bit E4M3 codes
 };
 
 // One record of split-KV partial results: running max and sum (log2 domain) of the G query heads
@@ -264,8 +265,20 @@ struct PagedArgs {
     int table_stride;  // entries per request slot, a multiple of 4
     int n_pages;       // physical pages per full head
     int cap;           // sink + window
+    // 8-bit pages (kModePagedFp8): a page is 16 KB, K codes [64 tokens][128] then V codes TRANSPOSED
+    // [128][64 tokens]; page p of full-head slot f of the layer is page page0_8 + f * n_pages + p of the
+    // 8-bit pool.  x_hat = value(code) * scale with one scale per KV head (indexed by head) for K, V.
+    int page0_8;
+    float k_scale[kMaxKvHeads], v_scale[kMaxKvHeads];
     int seq_len[kMaxPagedBatch];
     unsigned short seq_slot[kMaxPagedBatch];
+};
+// The two tensor maps over the 8-bit pool: rows of 128 bytes with boxes of 64 rows (a page's K codes),
+// rows of 64 bytes with boxes of 128 rows (a page's transposed V codes).
+struct alignas(64) PagedFp8Args {
+    PagedArgs pa;
+    alignas(64) CUtensorMap map_k;
+    alignas(64) CUtensorMap map_v;
 };
 
 struct AppendArgs {
@@ -312,7 +325,7 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.b = unit / a.n_comp;
         u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
     }
-    if (MODE == kModePaged) {  // this sequence's own length
+    if (MODE == kModePaged || MODE == kModePagedFp8) {  // this sequence's own length
         const int n = pg->seq_len[u.b];
         u.len = u.pos.uid < a.sched.U ? n : (n < pg->cap ? n : pg->cap);
     }
@@ -367,6 +380,7 @@ cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
 struct LayerDesc {
     long long full_row0, comp_row0;  // first pool row of the layer's full-head / compressed-head region
     int n_full, n_comp;
+    long long page0_8;               // paged cache with 8-bit pages: first page of the layer in the 8-bit pool
 };
 struct AppendAllArgs {
     __nv_bfloat16* pool;
@@ -380,7 +394,7 @@ struct AppendAllArgs {
 cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
                           int stages, int groups, cudaStream_t stream, bool overlap, int mode = kModePlain,
-                          const PagedArgs* paged = nullptr);
+                          const PagedArgs* paged = nullptr, const PagedFp8Args* paged8 = nullptr);
 cudaError_t prepare_decode_kernels(int head_dim);
 size_t decode_smem_bytes(int head_dim, int stages, int group, int groups, int mode = kModePlain);
 
@@ -406,6 +420,12 @@ struct PagedAppendArgs {
     int n, t0, first_page;
     int n_layers;               // 1 unless the launch serves every layer
     const LayerDesc* layers;    // device, [n_layers]; unused when n_layers == 1
+    // 8-bit pages of the full heads (null: 16-bit rows): the pool, 1 / scale per head of the first layer
+    // served ([n_layers][kv_heads]), the layer's first page when n_layers == 1
+    unsigned char* pool8;
+    const float* k_inv;
+    const float* v_inv;
+    long long page0_8;
     int page[kMaxAppendPages];
     int t[kMaxPagedBatch];
     unsigned short slot[kMaxPagedBatch];

@@ -8,6 +8,10 @@
 //               [n_full(layer)][n_pages][K|V][64][D] -- page p of a sequence is page p of every full
 //               head of every layer -- then the compressed-head region
 //               [max_seqs][n_comp(layer)][K|V][rows_comp][D]
+//   pool8       only with 8-bit pages (rlkv_paged_create_fp8): the full heads' pages as E4M3 codes,
+//               per layer [n_full(layer)][n_pages] pages of 16 KB (K codes [64][128], then V codes
+//               transposed [128][64]); the 16-bit pool then holds the compressed-head regions only
+//   scales      float 1/k_scale, 1/v_scale [layers][kv_heads] (8-bit pages only)
 //   tables      int32 slot_of_head[layers][kv_heads]
 //   page table  int32 [max_seqs][table_stride]   (written by the append kernels)
 //   layer desc  LayerDesc[layers]  (where each layer's regions start; for the step's append launch)
@@ -32,6 +36,12 @@ struct rlkv_paged {
     int device, sm_count, stages, groups, item_tiles;
     int rows_comp, max_batch, max_items, max_grid;
     int out_bf16;
+    int fp8;                      // the full heads' pages hold E4M3 codes
+    std::vector<float> k_scale, v_scale;  // [layers*kv_heads]
+    std::vector<long long> page0_8;       // first page of each layer in the 8-bit pool
+    long long pages8;                      // pages of the 8-bit pool
+    size_t off_pool8, off_scales;
+    CUtensorMap map_k, map_v;
     long long pool_rows;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -82,6 +92,8 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
     p.n_comp.assign(p.layers, 0);
     p.full_row0.assign(p.layers, 0);
     p.comp_row0.assign(p.layers, 0);
+    p.page0_8.assign(p.layers, 0);
+    p.pages8 = 0;
     long long row = 0, most = 0;
     for (int l = 0; l < p.layers; ++l) {
         int nf = 0, nc = 0;
@@ -95,7 +107,12 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
         p.n_full[l] = nf;
         p.n_comp[l] = nc;
         p.full_row0[l] = row;
-        row += (long long)nf * p.n_pages * 2 * kTile;
+        if (p.fp8) {
+            p.page0_8[l] = p.pages8;
+            p.pages8 += (long long)nf * p.n_pages;
+        } else {
+            row += (long long)nf * p.n_pages * 2 * kTile;
+        }
         p.comp_row0[l] = row;
         row += (long long)p.max_seqs * nc * 2 * p.rows_comp;
         const long long t = (long long)p.max_batch * ((long long)nf * p.table_stride + (long long)nc * (p.rows_comp / kTile));
@@ -104,11 +121,16 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
         if (m > most) most = m;
     }
     if (row >= (1ll << 31) || most >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
+    if (p.pages8 * 256 >= (1ll << 31)) return RLKV_EINVAL;              // a page is 256 rows of the V map
     p.pool_rows = row;
     p.max_items = (int)most;
     size_t off = 0;
     p.off_pool = off;
     off = align_up(off + (size_t)row * p.head_dim * 2, 1024);
+    p.off_pool8 = off;
+    off = align_up(off + (size_t)p.pages8 * 2 * kTile * 128, 1024);
+    p.off_scales = off;
+    off = align_up(off + (p.fp8 ? (size_t)2 * p.layers * p.kv_heads * sizeof(float) : 0), 1024);
     p.off_tables = off;
     off = align_up(off + (size_t)p.layers * p.kv_heads * sizeof(int), 1024);
     p.off_layer_desc = off;
@@ -166,40 +188,70 @@ void fill_append_args(rlkv_paged* p, int layer, const void* k, const void* v, Pa
     a.window = p->window;
     a.n_layers = 1;
     a.layers = nullptr;
+    a.pool8 = p->fp8 ? p->dev_base + p->off_pool8 : nullptr;
+    a.k_inv = dev_at<float>(p, p->off_scales) + (size_t)layer * p->kv_heads;
+    a.v_inv = a.k_inv + (size_t)p->layers * p->kv_heads;
+    a.page0_8 = p->page0_8[layer];
 }
 
 }  // namespace
 
 extern "C" {
 
-int rlkv_paged_size(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages, int max_seq_len,
-                    const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+static int paged_size(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages, int max_seq_len,
+                      const uint8_t* head_is_full, int sink, int window, int fp8, size_t* bytes_out)
 {
     if (!bytes_out) return RLKV_EINVAL;
     int rc = check_paged_shape(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window);
     if (rc) return rc;
+    if (fp8 && head_dim != 128) return RLKV_EINVAL;
     rlkv_paged p{};
     p.layers = layers; p.kv_heads = kv_heads; p.q_heads = q_heads; p.head_dim = head_dim;
-    p.max_seqs = max_seqs; p.n_pages = n_pages; p.sink = sink; p.window = window;
+    p.max_seqs = max_seqs; p.n_pages = n_pages; p.sink = sink; p.window = window; p.fp8 = fp8;
     rc = make_paged_layout(p, head_is_full, max_seq_len);
     if (rc) return rc;
     *bytes_out = p.total;
     return RLKV_OK;
 }
 
-int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
-                      int max_seq_len, const uint8_t* head_is_full, int sink, int window, void* device_buf,
-                      size_t device_buf_bytes)
+int rlkv_paged_size(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages, int max_seq_len,
+                    const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+{
+    return paged_size(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window, 0,
+                      bytes_out);
+}
+
+int rlkv_paged_size_fp8(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages, int max_seq_len,
+                        const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+{
+    return paged_size(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window, 1,
+                      bytes_out);
+}
+
+static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                        int max_seq_len, const uint8_t* head_is_full, int sink, int window, const float* k_scale,
+                        const float* v_scale, void* device_buf, size_t device_buf_bytes)
 {
     if (!out) return RLKV_EINVAL;
     *out = nullptr;
     int rc = check_paged_shape(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window);
     if (rc) return rc;
+    const int fp8 = k_scale != nullptr;
+    if (fp8) {
+        if (!v_scale || head_dim != 128) return RLKV_EINVAL;
+        for (int i = 0; i < layers * kv_heads; ++i)
+            if (!(k_scale[i] > 0.f) || !(v_scale[i] > 0.f) || k_scale[i] > 3.0e38f || v_scale[i] > 3.0e38f) return RLKV_EINVAL;
+    }
     rlkv_paged* p = new (std::nothrow) rlkv_paged();
     if (!p) return RLKV_ENOMEM;
     p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
     p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window;
     p->claims[0] = p->claims[1] = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
+    p->fp8 = fp8;
+    if (fp8) {
+        p->k_scale.assign(k_scale, k_scale + (size_t)layers * kv_heads);
+        p->v_scale.assign(v_scale, v_scale + (size_t)layers * kv_heads);
+    }
     rc = make_paged_layout(*p, head_is_full, max_seq_len);
     if (rc) { delete p; return rc; }
     p->len.assign((size_t)layers * max_seqs, 0);
@@ -212,7 +264,7 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
     if (e != cudaSuccess) { delete p; return cuda_fail(e, "device query"); }
     p->groups = 2;
     p->item_tiles = kPagedItemTiles;
-    p->stages = max_stages(head_dim, q_heads / kv_heads, p->groups, 1, kModePaged);
+    p->stages = max_stages(head_dim, q_heads / kv_heads, p->groups, 1, fp8 ? kModePagedFp8 : kModePaged);
     if (p->stages < 2) { delete p; return RLKV_EINVAL; }
     if (device_buf) {
         if ((reinterpret_cast<uintptr_t>(device_buf) & 1023u) != 0 || device_buf_bytes < p->total) { delete p; return RLKV_ENOMEM; }
@@ -231,21 +283,54 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
     };
     // pools zero-filled (rows never written stay finite), tickets / status / counter start at zero
     e = cudaMemset(p->dev_base + p->off_pool, 0, (size_t)p->pool_rows * head_dim * 2);
+    if (e == cudaSuccess && fp8) e = cudaMemset(p->dev_base + p->off_pool8, 0, (size_t)p->pages8 * 2 * kTile * 128);
+    if (e == cudaSuccess && fp8) {
+        // the kernels multiply by 1 / scale: one IEEE division per head, here
+        std::vector<float> inv((size_t)2 * layers * kv_heads);
+        for (int i = 0; i < layers * kv_heads; ++i) {
+            inv[i] = 1.0f / k_scale[i];
+            inv[(size_t)layers * kv_heads + i] = 1.0f / v_scale[i];
+        }
+        e = cudaMemcpy(p->dev_base + p->off_scales, inv.data(), inv.size() * sizeof(float), cudaMemcpyHostToDevice);
+    }
     if (e == cudaSuccess) e = cudaMemset(p->dev_base + p->off_page_table, 0, p->off_partials - p->off_page_table);
     if (e == cudaSuccess)
         e = cudaMemcpy(p->dev_base + p->off_tables, p->slot_of_head.data(), p->slot_of_head.size() * sizeof(int),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         std::vector<LayerDesc> desc(layers);
-        for (int l = 0; l < layers; ++l) desc[l] = LayerDesc{p->full_row0[l], p->comp_row0[l], p->n_full[l], p->n_comp[l]};
+        for (int l = 0; l < layers; ++l) desc[l] = LayerDesc{p->full_row0[l], p->comp_row0[l], p->n_full[l], p->n_comp[l], p->page0_8[l]};
         e = cudaMemcpy(p->dev_base + p->off_layer_desc, desc.data(), desc.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = prepare_decode_kernels(head_dim);
     if (e != cudaSuccess) return fail(cuda_fail(e, "rlkv_paged_create"));
-    rc = encode_pool_tensor_map(&p->tmap, p->dev_base + p->off_pool, p->pool_rows, head_dim);
+    // (a pool without rows -- every head full and in 8-bit pages -- still gets a one-row map: it is never used)
+    rc = encode_pool_tensor_map(&p->tmap, p->dev_base + p->off_pool, p->pool_rows > 0 ? p->pool_rows : 1, head_dim);
     if (rc) return fail(rc);
+    if (fp8 && p->pages8 > 0) {
+        rc = encode_byte_rows_tensor_map(&p->map_k, p->dev_base + p->off_pool8, 128, p->pages8 * 128, kTile);
+        if (!rc) rc = encode_byte_rows_tensor_map(&p->map_v, p->dev_base + p->off_pool8, 64, p->pages8 * 256, 128);
+        if (rc) return fail(rc);
+    }
     *out = p;
     return RLKV_OK;
+}
+
+int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                      int max_seq_len, const uint8_t* head_is_full, int sink, int window, void* device_buf,
+                      size_t device_buf_bytes)
+{
+    return paged_create(out, layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window,
+                        nullptr, nullptr, device_buf, device_buf_bytes);
+}
+
+int rlkv_paged_create_fp8(rlkv_paged** out, int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
+                          int max_seq_len, const uint8_t* head_is_full, int sink, int window, const float* k_scale,
+                          const float* v_scale, void* device_buf, size_t device_buf_bytes)
+{
+    if (!k_scale || !v_scale) return RLKV_EINVAL;
+    return paged_create(out, layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window,
+                        k_scale, v_scale, device_buf, device_buf_bytes);
 }
 
 int rlkv_paged_destroy(rlkv_paged* p)
@@ -440,7 +525,21 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
         pa.seq_len[i] = i < n ? len[slots[i]] : 0;
         pa.seq_slot[i] = (unsigned short)(i < n ? slots[i] : 0);
     }
-    RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, stream, overlap, kModePaged, &pa));
+    pa.page0_8 = (int)p->page0_8[layer];
+    for (int h = 0; h < kMaxKvHeads; ++h) {
+        pa.k_scale[h] = p->fp8 && h < p->kv_heads ? p->k_scale[(size_t)layer * p->kv_heads + h] : 1.f;
+        pa.v_scale[h] = p->fp8 && h < p->kv_heads ? p->v_scale[(size_t)layer * p->kv_heads + h] : 1.f;
+    }
+    if (p->fp8) {
+        PagedFp8Args p8;
+        p8.pa = pa;
+        p8.map_k = p->map_k;
+        p8.map_v = p->map_v;
+        RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, stream, overlap, kModePagedFp8, nullptr,
+                                &p8));
+    } else {
+        RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, stream, overlap, kModePaged, &pa));
+    }
     p->claims[half] += (unsigned int)a.sched.n_items;
     p->launches++;
     if (grid_out) *grid_out = grid;
@@ -565,9 +664,10 @@ int rlkv_paged_step_bytes(const rlkv_paged* p, int layer, const int* slots, int 
     uint64_t rows = 0;
     for (int i = 0; i < n; ++i) {
         const int t = len_of(p, layer)[slots[i]];
-        rows += (uint64_t)p->n_full[layer] * t + (uint64_t)p->n_comp[layer] * (t < cap ? t : cap);
+        // a row of a full head in 8-bit pages is half the bytes: counted as half a row
+        rows += (uint64_t)p->n_full[layer] * t * (p->fp8 ? 1 : 2) + (uint64_t)p->n_comp[layer] * (t < cap ? t : cap) * 2;
     }
-    *kv_bytes_out = rows * 2 * p->head_dim * 2;
+    *kv_bytes_out = rows * p->head_dim * 2;
     return RLKV_OK;
 }
 
@@ -584,7 +684,26 @@ int rlkv_paged_debug_export_head(rlkv_paged* p, int layer, int slot, int kv_head
     const int s = p->slot_of_head[(size_t)layer * p->kv_heads + kv_head];
     const uint8_t* pool = p->dev_base + p->off_pool;
     const size_t row_bytes = (size_t)D * 2;
-    if (s >= 0) {  // a full head: its n tokens in token order, page by page
+    if (s >= 0 && p->fp8) {  // a full head in 8-bit pages: its codes, one per 16-bit element of the output
+        std::vector<uint8_t> page_bytes((size_t)2 * kTile * 128);
+        uint16_t* kh = static_cast<uint16_t*>(k_host);
+        uint16_t* vh = static_cast<uint16_t*>(v_host);
+        for (int t0 = 0; t0 < n; t0 += kTile) {
+            const int page = p->table[(size_t)slot * p->table_stride + t0 / kTile];
+            if (page < 0) return RLKV_EKERNEL;
+            const int cnt = n - t0 < kTile ? n - t0 : kTile;
+            const uint8_t* src = p->dev_base + p->off_pool8 +
+                                 (size_t)(p->page0_8[layer] + (long long)s * p->n_pages + page) * page_bytes.size();
+            RLKV_CUDA(cudaMemcpy(page_bytes.data(), src, page_bytes.size(), cudaMemcpyDeviceToHost));
+            for (int t = 0; t < cnt; ++t)
+                for (int d = 0; d < D; ++d) {
+                    kh[(size_t)(t0 + t) * D + d] = page_bytes[(size_t)t * 128 + d];
+                    vh[(size_t)(t0 + t) * D + d] = page_bytes[(size_t)kTile * 128 + (size_t)d * kTile + t];  // transposed
+                }
+        }
+        for (int t = 0; t < n; ++t) token_of_slot_host[t] = t;
+        *rows_out = n;
+    } else if (s >= 0) {  // a full head: its n tokens in token order, page by page
         for (int t0 = 0; t0 < n; t0 += kTile) {
             const int page = p->table[(size_t)slot * p->table_stride + t0 / kTile];
             if (page < 0) return RLKV_EKERNEL;

@@ -108,14 +108,18 @@ class PagedCache:
     """Owns an rlkv_paged handle (request slots with their own lengths, paged full heads)."""
 
     def __init__(self, layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len, head_is_full, sink, window,
-                 device="cuda:0"):
+                 device="cuda:0", k_scale=None, v_scale=None):
         self.layers, self.kv_heads, self.q_heads, self.head_dim = layers, kv_heads, q_heads, head_dim
         self.max_seqs, self.n_pages, self.max_seq_len, self.sink, self.window = max_seqs, n_pages, max_seq_len, sink, window
         self.device = torch.device(device)
         self.mask = np.asarray(head_is_full, dtype=np.uint8).reshape(layers, kv_heads)
         with torch.cuda.device(self.device):
-            self.handle = rl.rlkv_paged_create(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
-                                               self.mask, sink, window)
+            if k_scale is None:
+                self.handle = rl.rlkv_paged_create(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
+                                                   self.mask, sink, window)
+            else:      # the full heads' pages as E4M3 codes
+                self.handle = rl.rlkv_paged_create_fp8(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
+                                                       self.mask, sink, window, k_scale, v_scale)
 
     def close(self):
         if getattr(self, "handle", None):

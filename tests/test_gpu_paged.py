@@ -28,11 +28,13 @@ def hz(cuda_device):
 class Seq:
     """One request: its slot in the cache under test and its own oracle."""
 
-    def __init__(self, cache, seed, max_len):
+    def __init__(self, cache, seed, max_len, scales=None):
         self.cache, self.seed = cache, seed
         self.slot = cache.open_seq()
         self.oracle = Oracle(cache.layers, cache.kv_heads, cache.q_heads, cache.head_dim, 1, max_len,
                              cache.mask.reshape(-1), cache.sink, cache.window, threads=4)
+        if scales is not None:                                # the full heads in 8-bit storage
+            self.oracle.set_fp8(*scales)
         self.n = 0
 
     def rows(self, layer, t0, t1, what):
@@ -318,3 +320,75 @@ def test_paged_step_equals_the_per_layer_calls(rl, hz, cuda_device, shape):
     assert e.value.code == rl.RLKV_EINVAL
     assert cache.status() == 0
     cache.close()
+
+
+# ------------------------------------------------------------------------------------------ 8-bit pages
+FP8_SHAPES = [
+    # layers, Hkv, Hq, S, W, mask, lengths
+    (1, 2, 8, 4, 60, "10", [1, 63, 64, 65]),
+    (2, 4, 28, 16, 112, "1001" "0111", [300, 1, 128, 1000, 77]),
+    (1, 8, 32, 16, 112, "11111111", [900, 64, 2500]),
+    (1, 1, 8, 0, 5, "1", [777, 3]),
+    (1, 4, 16, 16, 64, "0000", [400, 90]),
+    (1, 2, 8, 16, 112, "11", [9000, 4100]),              # long rows: split over many work items
+]
+
+
+@pytest.mark.parametrize("layers,Hkv,Hq,S,W,mask,lens", FP8_SHAPES)
+def test_fp8_pages_match_the_quantising_oracle(rl, hz, cuda_device, layers, Hkv, Hq, S, W, mask, lens):
+    """rlkv_paged_create_fp8: the codes in the pages equal the oracle's bit for bit (K in token order,
+    V transposed back), compressed heads keep their 16-bit rings, outputs within the usual bounds of
+    the oracle's attention over the dequantised rows.  Scales differ per head and are no powers of two."""
+    D = 128
+    mask = [int(c) for c in mask]
+    rng = np.random.default_rng(17)
+    ks = rng.uniform(0.004, 0.02, size=layers * Hkv).astype(np.float32)      # N(0,1) inputs reach about 4.5: some saturate
+    vs = rng.uniform(0.02, 1.5, size=layers * Hkv).astype(np.float32)
+    max_len = max(lens) + 8
+    pages = sum((n + 2 + 63) // 64 for n in lens) + 2
+    cache = hz.PagedCache(layers, Hkv, Hq, D, len(lens) + 1, pages, max_len, mask, S, W, device=cuda_device,
+                          k_scale=ks, v_scale=vs)
+    seqs = []
+    for i, n in enumerate(lens):
+        s = Seq(cache, i + 1, max_len, scales=(ks, vs))
+        if n > 1:
+            s.prefill(n - 1, cuda_device)
+        seqs.append(s)
+    append_all(cache, seqs, cuda_device)
+    check_decode(cache, seqs, cuda_device, 500)
+    check_state(cache, seqs)
+    n_full = int(cache.mask[0].sum())
+    want = sum(n_full * s.n * 2 * D + (Hkv - n_full) * min(s.n, S + W) * 4 * D for s in seqs)
+    assert cache.step_bytes(0, [s.slot for s in seqs]) == want       # half the bytes per row of a full head
+    # whole steps on the same cache
+    slots = [s.slot for s in seqs]
+    out = torch.empty((layers, len(seqs), Hq, D), dtype=torch.float32, device=cuda_device)
+    for step in range(3):
+        kk = torch.stack([torch.cat([s.rows(l, s.n, s.n + 1, 0) for s in seqs]) for l in range(layers)])
+        vv = torch.stack([torch.cat([s.rows(l, s.n, s.n + 1, 1) for s in seqs]) for l in range(layers)])
+        q = rand_bf16((layers, len(seqs), Hq, D), 3000 + step)
+        rl.rlkv_paged_step(cache.handle, slots, kk.to(cuda_device), vv.to(cuda_device), q.to(cuda_device), out)
+        for i, s in enumerate(seqs):
+            for l in range(layers):
+                assert s.oracle.append(l, kk[l, i], vv[l, i]) == 0
+            s.n += 1
+        got = out.cpu().numpy()
+        for l in range(layers):
+            for i, s in enumerate(seqs):
+                check_out(got[l, i], s.oracle.decode(l, q[l, i:i + 1])[0])
+    check_state(cache, seqs)
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_fp8_argument_checks(rl, hz, cuda_device):
+    ok = dict(layers=1, kv_heads=2, q_heads=8, head_dim=128, max_seqs=2, n_pages=4, max_seq_len=128,
+              head_is_full=[1, 0], sink=4, window=12, k_scale=[1.0, 1.0], v_scale=[1.0, 1.0])
+    for bad in (dict(head_dim=64), dict(k_scale=[0.0, 1.0]), dict(v_scale=[1.0, -2.0]), dict(k_scale=[float("nan"), 1.0]),
+                dict(v_scale=[float("inf"), 1.0])):
+        with pytest.raises(rl.RlkvError) as e:
+            rl.rlkv_paged_create_fp8(**{**ok, **bad})
+        assert e.value.code == rl.RLKV_EINVAL
+    h = rl.rlkv_paged_create_fp8(**ok)
+    assert rl.rlkv_paged_size_fp8(1, 2, 8, 128, 2, 4, 128, [1, 0], 4, 12) < rl.rlkv_paged_size(1, 2, 8, 128, 2, 4, 128, [1, 0], 4, 12)
+    rl.rlkv_paged_destroy(h)
