@@ -451,10 +451,14 @@ def run_ours(args, w, mask):
         pmask = mask[:pl * w.kv_heads]
         spread = [max(1, int(round(n * (0.25 + 1.5 * i / max(1, w.batch - 1))))) for i in range(w.batch)]
         paged = {"workload": f"first {pl} layers of the {w.name} mask, {w.batch} sequences, launches back to back"}
-        for name, lens in (("uniform", [n] * w.batch), ("ragged", spread)):
+        variants = [("uniform", [n] * w.batch, False), ("ragged", spread, False)]
+        if w.head_dim == 128:
+            variants.append(("uniform_fp8", [n] * w.batch, True))   # the full heads' pages as E4M3 codes
+        for name, lens, fp8 in variants:
             pages = sum((x + 63) // 64 for x in lens) + 2 + 2 * len(lens)
+            scales = np.full(pl * w.kv_heads, 1.0 / 64, np.float32) if fp8 else None   # N(0,1) inputs stay well inside +-448
             pc = harness.PagedCache(pl, w.kv_heads, w.q_heads, w.head_dim, w.batch, pages, max(lens) + 128, pmask,
-                                    w.sink, w.window, device=dev)
+                                    w.sink, w.window, device=dev, k_scale=scales, v_scale=scales)
             slots = [pc.open_seq() for _ in lens]
             for i, x in enumerate(lens):
                 for l in range(pl):
