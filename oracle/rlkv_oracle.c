@@ -53,7 +53,7 @@ typedef struct {
     uint16_t **k, **v;       /* [layers*batch*kv_heads] -> rows*head_dim bf16 bits */
     int32_t **token_of_slot; /* compressed heads: [cap], -1 = empty; NULL for full heads */
     int threads;
-    /* 8-bit storage of the full heads (rlkv_oracle_set_fp8): their k, v entries hold E4M3 codes */
+    /* 8-bit storage (rlkv_oracle_set_fp8): the k, v entries of every head hold E4M3 codes */
     int fp8;
     float *k_scale, *v_scale; /* [layers*kv_heads] */
 } oracle_t;
@@ -66,7 +66,7 @@ static float bf16_to_float(uint16_t b)
     return f;
 }
 
-/* ---- 8-bit K/V for the full heads (the paper's Limitations and Future Work: head-level
+/* ---- 8-bit K/V (the paper's Limitations and Future Work: head-level
  * compression "can be combined with" KV-cache quantisation; no format is given there).
  * Reading taken: the OCP 8-bit floating-point format E4M3 -- 1 sign bit, 4 exponent bits with bias
  * 7, 3 mantissa bits; exponent field 0 holds the subnormals m/8 * 2^-6; there are no infinities and
@@ -75,7 +75,8 @@ static float bf16_to_float(uint16_t b)
  *     code  = E4M3( fl32( fl32(x) * fl32(1 / scale) ) )    round to nearest, ties to even,
  *                                                           magnitudes above 448 saturate to 448
  *     x_hat = value(code) * scale
- * and attention runs on x_hat as before.  Compressed heads keep their 16-bit rows.
+ * and attention runs on x_hat as before.  Every head is stored this way, full heads and the sink +
+ * window rings of compressed heads alike (one storage format per cache).
  * Pins: every code's value against torch.float8_e4m3fn; the encoder against torch's cast on a
  * sweep that holds every midpoint between neighbouring codes; closed forms. */
 float rlkv_oracle_e4m3_value(uint8_t code)
@@ -176,7 +177,7 @@ oracle_t *rlkv_oracle_create(int layers, int kv_heads, int q_heads, int head_dim
     return o;
 }
 
-/* Switches the full heads to 8-bit storage.  k_scale, v_scale: [layers*kv_heads], positive and finite.
+/* Switches the cache to 8-bit storage.  k_scale, v_scale: [layers*kv_heads], positive and finite.
  * Only while the cache is empty.  Returns 0, -7 otherwise. */
 int rlkv_oracle_set_fp8(oracle_t *o, const float *k_scale, const float *v_scale)
 {
@@ -196,11 +197,11 @@ int rlkv_oracle_set_fp8(oracle_t *o, const float *k_scale, const float *v_scale)
     return 0;
 }
 
-/* The 16 stored bits of one element as a number: a bf16 value, or for a full head in 8-bit storage
- * the E4M3 code's value times the head's scale. */
+/* The 16 stored bits of one element as a number: a bf16 value, or in 8-bit storage the E4M3 code's
+ * value times the head's scale. */
 static acc_t stored(const oracle_t *o, int layer, int h, uint16_t bits, int is_v)
 {
-    if (o->fp8 && o->is_full[layer * o->kv_heads + h]) {
+    if (o->fp8) {
         float scale = (is_v ? o->v_scale : o->k_scale)[layer * o->kv_heads + h];
         return (acc_t)rlkv_oracle_e4m3_value((uint8_t)bits) * (acc_t)scale;
     }
@@ -241,7 +242,7 @@ int rlkv_oracle_append(oracle_t *o, int layer, const uint16_t *k, const uint16_t
                 row = slot_of_token(o, t);
                 o->token_of_slot[u][row] = t;
             }
-            if (o->fp8 && o->is_full[layer * o->kv_heads + h]) {
+            if (o->fp8) {
                 float ik = 1.0f / o->k_scale[layer * o->kv_heads + h], iv = 1.0f / o->v_scale[layer * o->kv_heads + h];
                 for (int d = 0; d < D; ++d) {
                     o->k[u][(size_t)row * D + d] = rlkv_oracle_e4m3_encode(bf16_to_float(ks[d]) * ik);

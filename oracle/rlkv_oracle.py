@@ -130,7 +130,7 @@ class Oracle:
         self._lib.rlkv_oracle_set_threads(self._h, int(threads))
 
     def set_fp8(self, k_scale, v_scale) -> None:
-        """Full heads store E4M3 codes from now on (only while the cache is empty).  k_scale,
+        """Every head stores E4M3 codes from now on (only while the cache is empty).  k_scale,
         v_scale: [layers][kv_heads] positive floats."""
         ks = np.ascontiguousarray(np.asarray(k_scale, dtype=np.float32).reshape(-1))
         vs = np.ascontiguousarray(np.asarray(v_scale, dtype=np.float32).reshape(-1))

@@ -441,10 +441,10 @@ def test_e4m3_encoder_matches_the_library_cast_on_every_code_midpoint_and_neighb
         assert e4m3_encode(e4m3_value(c)) == c
 
 
-def test_fp8_full_heads_equal_plain_attention_over_the_dequantised_rows():
+def test_fp8_storage_equals_plain_attention_over_the_dequantised_rows():
     """With 8-bit storage the oracle must give exactly what the 16-bit oracle gives on rows that were
-    quantised and dequantised beforehand with the library type (values chosen so that x_hat is a
-    bf16 number: scale a power of two); compressed heads are untouched."""
+    quantised and dequantised beforehand with the library type (scales are powers of two, so that
+    x_hat is a bf16 number) -- for a full head and for a compressed head's ring alike."""
     Hq, Hkv, D, B, S, W, n = 8, 2, 32, 2, 4, 12, 90
     K, V, q = rand_bf16((n, B, Hkv, D), 301), rand_bf16((n, B, Hkv, D), 302), rand_bf16((B, Hq, D), 303)
     ks, vs = np.array([0.5, 2.0], np.float32), np.array([0.25, 1.0], np.float32)
@@ -456,14 +456,18 @@ def test_fp8_full_heads_equal_plain_attention_over_the_dequantised_rows():
         return ((x.float() / scale).to(torch.float8_e4m3fn).float() * scale).to(torch.bfloat16)
 
     K2, V2 = K.clone(), V.clone()
-    K2[:, :, 0], V2[:, :, 0] = roundtrip(K[:, :, 0], 0.5), roundtrip(V[:, :, 0], 0.25)
+    for h in range(Hkv):
+        K2[:, :, h], V2[:, :, h] = roundtrip(K[:, :, h], float(ks[h])), roundtrip(V[:, :, h], float(vs[h]))
     b = Oracle(1, Hkv, Hq, D, B, n, [1, 0], S, W)
     fill(b, 0, K2, V2)
     np.testing.assert_array_equal(a.decode(0, q), b.decode(0, q))
-    # the full head's stored entries are the codes; the compressed head's rows are the bf16 bits
+    # the stored entries are the codes: the full head's in token order, the ring's in slot order
     k_codes, v_codes, _ = a.export_head(0, 1, 0)
     want = (K[:, 1, 0].float() / 0.5).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
     np.testing.assert_array_equal(k_codes[:n], want)
+    ring_k, ring_v, tok = a.export_head(0, 1, 1)
+    want = (V[tok, 1, 1].float() / 1.0).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    np.testing.assert_array_equal(ring_v, want)
     assert np.abs(a.decode(0, q) - Oracle_decode_plain(K, V, q, Hkv, Hq, D, B, n, S, W)).max() > 1e-4   # it does quantise
     with pytest.raises(RuntimeError, match="-7"):
         a.set_fp8(ks, vs)                                       # only while empty
