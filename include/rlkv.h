@@ -189,18 +189,17 @@ int rlkv_paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads, i
                       int max_seqs, int n_pages, int max_seq_len, const uint8_t* head_is_full,
                       int sink, int window, void* device_buf, size_t device_buf_bytes);
 int rlkv_paged_destroy(rlkv_paged* cache);
-/* The paged cache with the full heads' pages held in 8 bits.  (The paper names KV-cache quantisation
- * as the direction to combine head-level compression with and fixes no format; this is the format
- * taken.)  Every K and V element of a full head is stored as an OCP E4M3 code (1 sign, 4 exponent bits
+/* The paged cache held in 8 bits.  (The paper names KV-cache quantisation as the direction to
+ * combine head-level compression with and fixes no format; this is the format taken.)  Every K and
+ * V element -- of the full heads' pages and of the compressed heads' rings -- is stored as an OCP E4M3 code (1 sign, 4 exponent bits
  * with bias 7, 3 mantissa bits, largest finite value 448, no infinities):
  *     code = E4M3(x * (1 / scale))   round to nearest even, magnitudes above 448 saturate;
  *     attention then runs on value(code) * scale
  * with one scale per (layer, KV head) for K and one for V: k_scale, v_scale, HOST float
  * [layers][kv_heads], positive and finite, copied (a scale of max|x| / 448 uses the whole range;
- * 1 is fine for activations of order one).  The full heads then cost half the bytes per token, to
- * store and to read; compressed heads keep their 16-bit rings.  head_dim must be 128.  Every other
- * call works as on a cache from rlkv_paged_create; rlkv_paged_debug_export_head returns a full
- * head's codes, one per 16-bit element. */
+ * 1 is fine for activations of order one).  The cache then costs half the bytes per token, to store
+ * and to read.  head_dim must be 128.  Every other call works as on a cache from rlkv_paged_create;
+ * rlkv_paged_debug_export_head returns the codes, one per 16-bit element. */
 int rlkv_paged_size_fp8(int layers, int kv_heads, int q_heads, int head_dim, int max_seqs, int n_pages,
                         int max_seq_len, const uint8_t* head_is_full, int sink, int window,
                         size_t* bytes_out);

@@ -112,11 +112,28 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
             n_comp = a.layers[l].n_comp;
         }
         long long row;
-        if (slot >= 0 && a.pool8) {
+        if (a.pool8) {
             // 8-bit pages: code = E4M3(x * (1 / scale)), round to nearest even, saturating.  A page is
-            // the K codes [64 tokens][128] followed by the V codes transposed [128][64 tokens].
-            const long long page0 = a.n_layers > 1 ? a.layers[l].page0_8 : a.page0_8;
-            unsigned char* pg = a.pool8 + (page0 + (long long)slot * a.n_pages + page) * (2 * kTile * 128);
+            // the K codes [64 rows][128] followed by the V codes transposed [128][64 rows]; a full head's
+            // token t is row t % 64 of the sequence's page t / 64, a compressed head's ring row r is row
+            // r % 64 of page r / 64 of its ring.
+            long long page_index;
+            int prow;
+            if (slot >= 0) {
+                const long long page0 = a.n_layers > 1 ? a.layers[l].page0_8 : a.page0_8;
+                page_index = page0 + (long long)slot * a.n_pages + page;
+                prow = t % kTile;
+            } else {
+                if (a.prefill) {
+                    const int n_final = a.t0 + a.n;
+                    if (!(t < a.sink || t >= n_final - a.window)) continue;  // evicted before the batch ends
+                }
+                const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
+                const long long ring0 = a.n_layers > 1 ? a.layers[l].ring0_8 : a.ring0_8;
+                page_index = ring0 + ((long long)seq * n_comp + (-slot - 1)) * a.ring_tiles + phys / kTile;
+                prow = phys % kTile;
+            }
+            unsigned char* pg = a.pool8 + page_index * (2 * kTile * 128);
             const float inv = (kv ? a.v_inv : a.k_inv)[l * a.kv_heads + h];
             const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.n + e) * a.kv_heads + h) * a.head_dim + c * 8;
             const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src));
@@ -126,10 +143,10 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
             for (int j = 0; j < 8; ++j)
                 code[j] = (unsigned char)__nv_cvt_float_to_fp8(__bfloat162float(x[j]) * inv, __NV_SATFINITE, __NV_E4M3);
             if (kv == 0) {
-                *reinterpret_cast<uint2*>(pg + (t % kTile) * 128 + c * 8) = *reinterpret_cast<const uint2*>(code);
+                *reinterpret_cast<uint2*>(pg + prow * 128 + c * 8) = *reinterpret_cast<const uint2*>(code);
             } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) pg[kTile * 128 + (c * 8 + j) * kTile + t % kTile] = code[j];
+                for (int j = 0; j < 8; ++j) pg[kTile * 128 + (c * 8 + j) * kTile + prow] = code[j];
             }
             if (slot == 0 && c == 0 && kv == 0) a.page_table[(size_t)seq * a.table_stride + t / kTile] = page;
             continue;

@@ -246,9 +246,14 @@ struct Smem {
     static constexpr int kTilePairBytes = 2 * kTileBytes;   // K tile then V tile
     // a stage: K tile, V tile, then the G query rows of the tile's unit (filled for the first NG
     // tiles of a segment), padded so that the next stage starts on a 1024-byte boundary again
-    __host__ __device__ static constexpr int stage_bytes(int group)
+    // (8-bit pages: a stage is one 16 KB page of codes, K then V transposed, and the query rows)
+    __host__ __device__ static constexpr int tile_pair_bytes(int mode)
     {
-        return kTilePairBytes + (group * D * 2 + 1023) / 1024 * 1024;
+        return mode == kModePagedFp8 ? kTilePairBytes / 2 : kTilePairBytes;
+    }
+    __host__ __device__ static constexpr int stage_bytes(int group, int mode = kModePlain)
+    {
+        return tile_pair_bytes(mode) + (group * D * 2 + 1023) / 1024 * 1024;
     }
     static constexpr int kMergeStride = D + kMergePad;      // floats per head row
     static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
@@ -263,7 +268,7 @@ struct Smem {
     static constexpr int kPagedBytes = (kMaxSeqPages + 4) * 4 + (int)((sizeof(PagedArgs) + 15) / 16 * 16);
     __host__ __device__ static constexpr size_t bytes(int stages, int group, int mode = kModePlain)
     {
-        return (size_t)stages * stage_bytes(group) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
+        return (size_t)stages * stage_bytes(group, mode) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
                (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0);
@@ -421,7 +426,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     extern __shared__ __align__(1024) uint8_t smem[];
     const int G = args.group;
     uint8_t* stage_base = smem;
-    const int stage_bytes = S::stage_bytes(G);
+    const int stage_bytes = S::stage_bytes(G, MODE);
+    constexpr int kPairBytes = S::tile_pair_bytes(MODE);  // the query rows of a stage follow its K/V data
     uint8_t* buffers = smem + (size_t)stages * stage_bytes;
     const int buffer_bytes = S::buffer_bytes(G);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(buffers + (size_t)kMergeBuffers * buffer_bytes);
@@ -551,7 +557,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     u = locate<MODE>(a, x, pg);
                     seg_tiles = min(x1 - x, u.pos.run);
                     const bool local_unit = MIXED && u.pos.uid >= sc.U;
-                    const bool fp8_unit = FP8 && u.pos.uid < sc.U;  // a full head whose pages hold E4M3 codes
+                    const bool fp8_unit = FP8;  // every unit of an 8-bit cache is pages of E4M3 codes
                     int seg_eff = seg_tiles;  // tiles of the segment that exist
                     if (PAGED) {
                         seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
@@ -591,7 +597,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             // codes fetched four consecutive d per lane, Q goes in as f16 with k-halves
                             // (d 4tq, 4tq+1) and (d 4tq+2, 4tq+3) of every 16
                             const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
-                                                            stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
+                                                            stage_base + (size_t)st * stage_bytes + kPairBytes) +
                                                         quad * D + 4 * tq;
 #pragma unroll
                             for (int ks = 0; ks < KS; ++ks) {
@@ -605,7 +611,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         }
                         if (!have_q) {
                             const __nv_bfloat16* qrow = reinterpret_cast<const __nv_bfloat16*>(
-                                                            stage_base + (size_t)st * stage_bytes + S::kTilePairBytes) +
+                                                            stage_base + (size_t)st * stage_bytes + kPairBytes) +
                                                         quad * D + 2 * tq;
 #pragma unroll
                             for (int ks = 0; ks < KS; ++ks) {
@@ -761,7 +767,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 float* merge = reinterpret_cast<float*>(buf);
                 float* stat_m = merge + S::merge_floats(G);
                 float* stat_l = stat_m + S::kWarps * kMaxGroup;
-                if (FP8 && item >= 0 && u.pos.uid < sc.U) {  // the rows were value(code): V's scale goes in here
+                if (FP8 && item >= 0) {  // the rows were value(code): V's scale goes in here
                     const float vs = pg->v_scale[u.head];
 #pragma unroll
                     for (int mt = 0; mt < KS; ++mt) {
@@ -878,7 +884,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 int local_row0 = -1, local_next = 0;  // MIXED, inside a local unit: first row of its head, next tile
                 // PAGED: tiles of the segment past the unit's own length (not issued); first pool row of the
                 // full head's pages (-1: a compressed unit); page-table index of s_pages[0]; next tile
-                int seg_skip = 0, paged_row0 = -1, page_base = 0, paged_tile = 0;
+                int seg_skip = 0, paged_row0 = -1, page_base = 0, paged_tile = 0, ring_next = 0;
                 bool asked = false;
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
@@ -942,9 +948,13 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             } else {
                                 paged_row0 = -1;
                                 const int c = u.pos.uid - sc.U - u.b * a.n_comp;
-                                krow = (int)(a.comp_row0 + ((long long)pg->seq_slot[u.b] * a.n_comp + c) * 2 * a.rows_comp) +
-                                       u.pos.tile * kTile;
-                                vrow = krow + a.rows_comp;
+                                if (FP8) {  // the ring's pages follow one another
+                                    ring_next = pg->ring0_8 + (pg->seq_slot[u.b] * a.n_comp + c) * pg->ring_tiles + u.pos.tile;
+                                } else {
+                                    krow = (int)(a.comp_row0 + ((long long)pg->seq_slot[u.b] * a.n_comp + c) * 2 * a.rows_comp) +
+                                           u.pos.tile * kTile;
+                                    vrow = krow + a.rows_comp;
+                                }
                             }
                             qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                         } else {
@@ -968,6 +978,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                         }
                     }
+                    if (FP8 && paged_row0 < 0) krow = ring_next++;
                     if (PAGED && paged_row0 >= 0) {
                         if (FP8) {  // the page itself; its row coordinates in the two 8-bit maps follow below
                             krow = paged_row0 + s_pages[paged_tile++ - page_base];
@@ -989,18 +1000,13 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     const uint32_t fb = smem_u32(full_bar + s);
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
                     const long long tc0 = trace ? clock64() : 0;
-                    const bool page8 = FP8 && paged_row0 >= 0;  // a 16 KB page of codes instead of two 16-bit tiles
-                    mbar_expect_tx(fb, (page8 ? S::kTilePairBytes / 2 : S::kTilePairBytes) + (with_q ? G * D * 2 : 0));
+                    mbar_expect_tx(fb, kPairBytes + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
                     const long long tc1 = trace ? clock64() : 0;
                     if constexpr (FP8) {
-                        if (page8) {  // a page is 128 rows of the K map (64 of them K codes) and 256 rows of the V map
-                            tma_load_2d(dst, &extra.map_k, 0, krow * 128, fb, stream_policy);
-                            tma_load_2d(dst + kTile * 128, &extra.map_v, 0, krow * 256 + 128, fb, stream_policy);
-                        } else {
-                            tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
-                            tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
-                        }
+                        // page krow: 128 rows of the K map (the first 64 are its K codes), 256 rows of the V map
+                        tma_load_2d(dst, &extra.map_k, 0, krow * 128, fb, stream_policy);
+                        tma_load_2d(dst + kTile * 128, &extra.map_v, 0, krow * 256 + 128, fb, stream_policy);
                     } else if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
                         tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
                         tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
@@ -1009,7 +1015,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb, stream_policy);
                     }
                     const long long tc2 = trace ? clock64() : 0;
-                    if (with_q) bulk_load(dst + S::kTilePairBytes, qsrc, G * D * 2, fb);
+                    if (with_q) bulk_load(dst + kPairBytes, qsrc, G * D * 2, fb);
                     if (trace) {
                         const long long tc3 = clock64();
                         cy_expect += tc1 - tc0;

@@ -267,8 +267,10 @@ struct PagedArgs {
     int cap;           // sink + window
     // 8-bit pages (kModePagedFp8): a page is 16 KB, K codes [64 tokens][128] then V codes TRANSPOSED
     // [128][64 tokens]; page p of full-head slot f of the layer is page page0_8 + f * n_pages + p of the
-    // 8-bit pool.  x_hat = value(code) * scale with one scale per KV head (indexed by head) for K, V.
-    int page0_8;
+    // 8-bit pool; the ring of request slot s and compressed-head slot c is the ring_tiles pages from
+    // ring0_8 + (s * n_comp + c) * ring_tiles on (ring row r in page r / 64, row r % 64).
+    // x_hat = value(code) * scale with one scale per KV head (indexed by head) for K, V.
+    int page0_8, ring0_8, ring_tiles;
     float k_scale[kMaxKvHeads], v_scale[kMaxKvHeads];
     int seq_len[kMaxPagedBatch];
     unsigned short seq_slot[kMaxPagedBatch];
@@ -380,7 +382,8 @@ cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
 struct LayerDesc {
     long long full_row0, comp_row0;  // first pool row of the layer's full-head / compressed-head region
     int n_full, n_comp;
-    long long page0_8;               // paged cache with 8-bit pages: first page of the layer in the 8-bit pool
+    long long page0_8, ring0_8;      // paged cache with 8-bit pages: the layer's first full-head page and first
+                                     // ring page in the 8-bit pool
 };
 struct AppendAllArgs {
     __nv_bfloat16* pool;
@@ -425,7 +428,8 @@ struct PagedAppendArgs {
     unsigned char* pool8;
     const float* k_inv;
     const float* v_inv;
-    long long page0_8;
+    long long page0_8, ring0_8;
+    int ring_tiles;             // pages per ring
     int page[kMaxAppendPages];
     int t[kMaxPagedBatch];
     unsigned short slot[kMaxPagedBatch];

@@ -8,9 +8,10 @@
 //               [n_full(layer)][n_pages][K|V][64][D] -- page p of a sequence is page p of every full
 //               head of every layer -- then the compressed-head region
 //               [max_seqs][n_comp(layer)][K|V][rows_comp][D]
-//   pool8       only with 8-bit pages (rlkv_paged_create_fp8): the full heads' pages as E4M3 codes,
-//               per layer [n_full(layer)][n_pages] pages of 16 KB (K codes [64][128], then V codes
-//               transposed [128][64]); the 16-bit pool then holds the compressed-head regions only
+//   pool8       only with 8-bit storage (rlkv_paged_create_fp8; the 16-bit pool is then empty): pages of
+//               16 KB (K codes [64 rows][128], then V codes transposed [128][64 rows]); per layer the
+//               full heads' pages [n_full(layer)][n_pages], then the rings
+//               [max_seqs][n_comp(layer)][rows_comp / 64]
 //   scales      float 1/k_scale, 1/v_scale [layers][kv_heads] (8-bit pages only)
 //   tables      int32 slot_of_head[layers][kv_heads]
 //   page table  int32 [max_seqs][table_stride]   (written by the append kernels)
@@ -38,7 +39,7 @@ struct rlkv_paged {
     int out_bf16;
     int fp8;                      // the full heads' pages hold E4M3 codes
     std::vector<float> k_scale, v_scale;  // [layers*kv_heads]
-    std::vector<long long> page0_8;       // first page of each layer in the 8-bit pool
+    std::vector<long long> page0_8, ring0_8;  // first full-head page / first ring page of each layer in the 8-bit pool
     long long pages8;                      // pages of the 8-bit pool
     size_t off_pool8, off_scales;
     CUtensorMap map_k, map_v;
@@ -93,6 +94,7 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
     p.full_row0.assign(p.layers, 0);
     p.comp_row0.assign(p.layers, 0);
     p.page0_8.assign(p.layers, 0);
+    p.ring0_8.assign(p.layers, 0);
     p.pages8 = 0;
     long long row = 0, most = 0;
     for (int l = 0; l < p.layers; ++l) {
@@ -110,11 +112,14 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
         if (p.fp8) {
             p.page0_8[l] = p.pages8;
             p.pages8 += (long long)nf * p.n_pages;
+            p.ring0_8[l] = p.pages8;
+            p.pages8 += (long long)p.max_seqs * nc * (p.rows_comp / kTile);
+            p.comp_row0[l] = row;
         } else {
             row += (long long)nf * p.n_pages * 2 * kTile;
+            p.comp_row0[l] = row;
+            row += (long long)p.max_seqs * nc * 2 * p.rows_comp;
         }
-        p.comp_row0[l] = row;
-        row += (long long)p.max_seqs * nc * 2 * p.rows_comp;
         const long long t = (long long)p.max_batch * ((long long)nf * p.table_stride + (long long)nc * (p.rows_comp / kTile));
         if (t >= (1ll << 31)) return RLKV_EINVAL;
         const long long m = most_slots(p.max_batch * nf, p.table_stride, p.max_batch * nc, p.rows_comp / kTile, p.max_grid);
@@ -192,6 +197,8 @@ void fill_append_args(rlkv_paged* p, int layer, const void* k, const void* v, Pa
     a.k_inv = dev_at<float>(p, p->off_scales) + (size_t)layer * p->kv_heads;
     a.v_inv = a.k_inv + (size_t)p->layers * p->kv_heads;
     a.page0_8 = p->page0_8[layer];
+    a.ring0_8 = p->ring0_8[layer];
+    a.ring_tiles = p->rows_comp / kTile;
 }
 
 }  // namespace
@@ -299,7 +306,7 @@ static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads,
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         std::vector<LayerDesc> desc(layers);
-        for (int l = 0; l < layers; ++l) desc[l] = LayerDesc{p->full_row0[l], p->comp_row0[l], p->n_full[l], p->n_comp[l], p->page0_8[l]};
+        for (int l = 0; l < layers; ++l) desc[l] = LayerDesc{p->full_row0[l], p->comp_row0[l], p->n_full[l], p->n_comp[l], p->page0_8[l], p->ring0_8[l]};
         e = cudaMemcpy(p->dev_base + p->off_layer_desc, desc.data(), desc.size() * sizeof(LayerDesc), cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = prepare_decode_kernels(head_dim);
@@ -526,6 +533,8 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
         pa.seq_slot[i] = (unsigned short)(i < n ? slots[i] : 0);
     }
     pa.page0_8 = (int)p->page0_8[layer];
+    pa.ring0_8 = (int)p->ring0_8[layer];
+    pa.ring_tiles = p->rows_comp / kTile;
     for (int h = 0; h < kMaxKvHeads; ++h) {
         pa.k_scale[h] = p->fp8 && h < p->kv_heads ? p->k_scale[(size_t)layer * p->kv_heads + h] : 1.f;
         pa.v_scale[h] = p->fp8 && h < p->kv_heads ? p->v_scale[(size_t)layer * p->kv_heads + h] : 1.f;
@@ -664,10 +673,9 @@ int rlkv_paged_step_bytes(const rlkv_paged* p, int layer, const int* slots, int 
     uint64_t rows = 0;
     for (int i = 0; i < n; ++i) {
         const int t = len_of(p, layer)[slots[i]];
-        // a row of a full head in 8-bit pages is half the bytes: counted as half a row
-        rows += (uint64_t)p->n_full[layer] * t * (p->fp8 ? 1 : 2) + (uint64_t)p->n_comp[layer] * (t < cap ? t : cap) * 2;
+        rows += (uint64_t)p->n_full[layer] * t + (uint64_t)p->n_comp[layer] * (t < cap ? t : cap);
     }
-    *kv_bytes_out = rows * p->head_dim * 2;
+    *kv_bytes_out = rows * 2 * p->head_dim * (p->fp8 ? 1 : 2);  // a K row and a V row of codes or of bf16
     return RLKV_OK;
 }
 
@@ -716,6 +724,33 @@ int rlkv_paged_debug_export_head(rlkv_paged* p, int layer, int slot, int kv_head
         }
         for (int t = 0; t < n; ++t) token_of_slot_host[t] = t;
         *rows_out = n;
+    } else if (p->fp8) {  // a compressed head in 8-bit storage: the codes of its physical ring
+        const int cap = p->sink + p->window, ring_tiles = p->rows_comp / kTile;
+        std::vector<uint8_t> page_bytes((size_t)2 * kTile * 128);
+        uint16_t* kh = static_cast<uint16_t*>(k_host);
+        uint16_t* vh = static_cast<uint16_t*>(v_host);
+        for (int r0 = 0; r0 < cap; r0 += kTile) {
+            const long long page = p->ring0_8[layer] + ((long long)slot * p->n_comp[layer] + (-s - 1)) * ring_tiles + r0 / kTile;
+            RLKV_CUDA(cudaMemcpy(page_bytes.data(), p->dev_base + p->off_pool8 + (size_t)page * page_bytes.size(),
+                                 page_bytes.size(), cudaMemcpyDeviceToHost));
+            for (int r = 0; r < kTile && r0 + r < cap; ++r)
+                for (int d = 0; d < D; ++d) {
+                    kh[(size_t)(r0 + r) * D + d] = page_bytes[(size_t)r * 128 + d];
+                    vh[(size_t)(r0 + r) * D + d] = page_bytes[(size_t)kTile * 128 + (size_t)d * kTile + r];
+                }
+        }
+        for (int r = 0; r < cap; ++r) {
+            int tok = -1;
+            if (r < p->sink) {
+                if (r < n) tok = r;
+            } else if (n > p->sink) {
+                const int newest = n - 1, back = ((newest - p->sink) - (r - p->sink)) % p->window;
+                const int cand = newest - (back < 0 ? back + p->window : back);
+                if (cand >= p->sink) tok = cand;
+            }
+            token_of_slot_host[r] = tok;
+        }
+        *rows_out = cap;
     } else {       // a compressed head: the physical ring
         const int cap = p->sink + p->window;
         const long long krow = p->comp_row0[layer] + ((long long)slot * p->n_comp[layer] + (-s - 1)) * 2 * p->rows_comp;

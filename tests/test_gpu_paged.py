@@ -336,13 +336,13 @@ FP8_SHAPES = [
 
 @pytest.mark.parametrize("layers,Hkv,Hq,S,W,mask,lens", FP8_SHAPES)
 def test_fp8_pages_match_the_quantising_oracle(rl, hz, cuda_device, layers, Hkv, Hq, S, W, mask, lens):
-    """rlkv_paged_create_fp8: the codes in the pages equal the oracle's bit for bit (K in token order,
-    V transposed back), compressed heads keep their 16-bit rings, outputs within the usual bounds of
-    the oracle's attention over the dequantised rows.  Scales differ per head and are no powers of two."""
+    """rlkv_paged_create_fp8: the codes in the pages and in the rings equal the oracle's bit for bit (K
+    in row order, V transposed back), outputs within the usual bounds of the oracle's attention over
+    the dequantised rows.  Scales differ per head and are no powers of two."""
     D = 128
     mask = [int(c) for c in mask]
     rng = np.random.default_rng(17)
-    ks = rng.uniform(0.004, 0.02, size=layers * Hkv).astype(np.float32)      # N(0,1) inputs reach about 4.5: some saturate
+    ks = rng.uniform(0.008, 0.05, size=layers * Hkv).astype(np.float32)      # N(0,1) inputs reach about 4.5: some saturate
     vs = rng.uniform(0.02, 1.5, size=layers * Hkv).astype(np.float32)
     max_len = max(lens) + 8
     pages = sum((n + 2 + 63) // 64 for n in lens) + 2
@@ -358,8 +358,8 @@ def test_fp8_pages_match_the_quantising_oracle(rl, hz, cuda_device, layers, Hkv,
     check_decode(cache, seqs, cuda_device, 500)
     check_state(cache, seqs)
     n_full = int(cache.mask[0].sum())
-    want = sum(n_full * s.n * 2 * D + (Hkv - n_full) * min(s.n, S + W) * 4 * D for s in seqs)
-    assert cache.step_bytes(0, [s.slot for s in seqs]) == want       # half the bytes per row of a full head
+    want = sum((n_full * s.n + (Hkv - n_full) * min(s.n, S + W)) * 2 * D for s in seqs)
+    assert cache.step_bytes(0, [s.slot for s in seqs]) == want       # a K row and a V row of codes: 2 * D bytes
     # whole steps on the same cache
     slots = [s.slot for s in seqs]
     out = torch.empty((layers, len(seqs), Hq, D), dtype=torch.float32, device=cuda_device)
