@@ -160,7 +160,7 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1)
 {
-    asm volatile(
+    asm(  // no side effects: the compiler may schedule it among the conversions around it
         "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
         "{%8,%9}, {%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
@@ -170,7 +170,7 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1,
 // codes 2, 3.  Every E4M3 value is an f16 value, so the conversion is exact.
 __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t codes, uint32_t& lo, uint32_t& hi)
 {
-    asm volatile(
+    asm(
         "{\n\t.reg .b16 a, b;\n\t"
         "mov.b32 {a, b}, %2;\n\t"
         "cvt.rn.f16x2.e4m3x2 %0, a;\n\t"
@@ -622,8 +622,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         }
                         if (FP8 && fp8_unit) {
                             if (wig * 16 < valid) {
-                                // a stage of an 8-bit page: K codes [64 tokens][128 B] with the 128-byte swizzle,
-                                // then V codes transposed [128 d][64 B] with the 64-byte swizzle
+                                // a stage of an 8-bit page, 128 rows of 128 bytes under the 128-byte swizzle: K codes
+                                // [64 tokens][128], then V codes transposed [128 d][64 tokens], two d per row
                                 const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
                                 const uint32_t sV = sK + kTile * 128;
                                 // ---- S = Q.K^T.  ldmatrix row i of token set s is token 4(i/2) + 2s + (i%2) of
@@ -632,11 +632,18 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
                                 float sA[4] = {0.f, 0.f, 0.f, 0.f}, sB[4] = {0.f, 0.f, 0.f, 0.f};
                                 float sA2[4] = {0.f, 0.f, 0.f, 0.f}, sB2[4] = {0.f, 0.f, 0.f, 0.f};
+                                // all fragments of K first, then the arithmetic: the loads' latencies overlap
+                                uint32_t kf[KS / 2][4];
 #pragma unroll
                                 for (int kp = 0; kp < KS / 2; ++kp) {
                                     const int chunk = 2 * kp + (lj >> 1);  // 16 codes along d
-                                    uint32_t r0, r1, r2, r3, b0, b1;
-                                    ldmatrix_x4(sK + ktok * 128 + ((chunk ^ (ktok & 7)) << 4), r0, r1, r2, r3);
+                                    ldmatrix_x4(sK + ktok * 128 + ((chunk ^ (ktok & 7)) << 4), kf[kp][0], kf[kp][1], kf[kp][2],
+                                                kf[kp][3]);
+                                }
+#pragma unroll
+                                for (int kp = 0; kp < KS / 2; ++kp) {
+                                    const uint32_t r0 = kf[kp][0], r1 = kf[kp][1], r2 = kf[kp][2], r3 = kf[kp][3];
+                                    uint32_t b0, b1;
                                     e4m3x4_to_f16x2x2(r0, b0, b1);
                                     mma_f16(sA, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
                                     e4m3x4_to_f16x2x2(r1, b0, b1);
@@ -645,6 +652,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                     mma_f16(sA2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
                                     e4m3x4_to_f16x2x2(r3, b0, b1);
                                     mma_f16(sB2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                }
+                                // the fragments of V are fetched now, under the softmax
+                                uint32_t vf[KS / 2][4];
+#pragma unroll
+                                for (int mp = 0; mp < KS / 2; ++mp) {
+                                    // row d of the transposed block is half of 128-byte row d / 2 of the stage
+                                    const int vd = 16 * (2 * mp + (lj >> 1)) + 8 * (lj & 1) + li, vr = vd >> 1;
+                                    ldmatrix_x4(sV + vr * 128 + ((((vd & 1) * 4 + wig) ^ (vr & 7)) << 4), vf[mp][0], vf[mp][1],
+                                                vf[mp][2], vf[mp][3]);
                                 }
                                 // this lane: head `quad`, tokens wig*16 + 4tq + {0, 1, 2, 3}; K's scale joins the softmax scale
                                 const float sl2 = a.scale_log2 * pg->k_scale[u.head];
@@ -674,9 +690,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 // the transposed page, four consecutive tokens per lane
 #pragma unroll
                                 for (int mp = 0; mp < KS / 2; ++mp) {
-                                    const int vd = 16 * (2 * mp + (lj >> 1)) + 8 * (lj & 1) + li;
-                                    uint32_t r0, r1, r2, r3, a0, a1, a2, a3;
-                                    ldmatrix_x4(sV + vd * 64 + ((wig ^ ((vd >> 1) & 3)) << 4), r0, r1, r2, r3);
+                                    const uint32_t r0 = vf[mp][0], r1 = vf[mp][1], r2 = vf[mp][2], r3 = vf[mp][3];
+                                    uint32_t a0, a1, a2, a3;
                                     e4m3x4_to_f16x2x2(r0, a0, a2);
                                     e4m3x4_to_f16x2x2(r1, a1, a3);
                                     acc[2 * mp][0] *= ca;
@@ -1004,9 +1019,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
                     const long long tc1 = trace ? clock64() : 0;
                     if constexpr (FP8) {
-                        // page krow: 128 rows of the K map (the first 64 are its K codes), 256 rows of the V map
+                        // page krow in one box of 128 rows of 128 bytes: 64 rows of K codes, then the transposed V
+                        // codes, two d per row
                         tma_load_2d(dst, &extra.map_k, 0, krow * 128, fb, stream_policy);
-                        tma_load_2d(dst + kTile * 128, &extra.map_v, 0, krow * 256 + 128, fb, stream_policy);
                     } else if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
                         tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
                         tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);

@@ -113,7 +113,7 @@ inline int encode_pool_tensor_map(CUtensorMap* tmap, void* base, long long rows,
 }
 
 // Tensor map over `rows` rows of row_bytes (64 or 128) bytes at `base`, boxes of box_rows whole rows,
-// swizzled over the row width: the two views of the paged cache's 8-bit pool.
+// swizzled over the row width: the view of the paged cache's 8-bit pool (128-byte rows, a page per box).
 inline int encode_byte_rows_tensor_map(CUtensorMap* tmap, void* base, int row_bytes, long long rows, int box_rows)
 {
     typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -275,12 +275,11 @@ struct PagedArgs {
     int seq_len[kMaxPagedBatch];
     unsigned short seq_slot[kMaxPagedBatch];
 };
-// The two tensor maps over the 8-bit pool: rows of 128 bytes with boxes of 64 rows (a page's K codes),
-// rows of 64 bytes with boxes of 128 rows (a page's transposed V codes).
+// The tensor map over the 8-bit pool: rows of 128 bytes, boxes of 128 rows = one page (64 rows of K
+// codes, then the transposed V codes, two d per row).
 struct alignas(64) PagedFp8Args {
     PagedArgs pa;
     alignas(64) CUtensorMap map_k;
-    alignas(64) CUtensorMap map_v;
 };
 
 struct AppendArgs {

@@ -42,7 +42,7 @@ struct rlkv_paged {
     std::vector<long long> page0_8, ring0_8;  // first full-head page / first ring page of each layer in the 8-bit pool
     long long pages8;                      // pages of the 8-bit pool
     size_t off_pool8, off_scales;
-    CUtensorMap map_k, map_v;
+    CUtensorMap map_k;  // the 8-bit pool as rows of 128 bytes, one page per box
     long long pool_rows;
     std::vector<uint8_t> is_full;
     std::vector<int> slot_of_head, head_of_slot;  // [layers*kv_heads]
@@ -126,7 +126,7 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
         if (m > most) most = m;
     }
     if (row >= (1ll << 31) || most >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
-    if (p.pages8 * 256 >= (1ll << 31)) return RLKV_EINVAL;              // a page is 256 rows of the V map
+    if (p.pages8 * 128 >= (1ll << 31)) return RLKV_EINVAL;              // a page is 128 rows of the 8-bit map
     p.pool_rows = row;
     p.max_items = (int)most;
     size_t off = 0;
@@ -315,8 +315,7 @@ static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads,
     rc = encode_pool_tensor_map(&p->tmap, p->dev_base + p->off_pool, p->pool_rows > 0 ? p->pool_rows : 1, head_dim);
     if (rc) return fail(rc);
     if (fp8 && p->pages8 > 0) {
-        rc = encode_byte_rows_tensor_map(&p->map_k, p->dev_base + p->off_pool8, 128, p->pages8 * 128, kTile);
-        if (!rc) rc = encode_byte_rows_tensor_map(&p->map_v, p->dev_base + p->off_pool8, 64, p->pages8 * 256, 128);
+        rc = encode_byte_rows_tensor_map(&p->map_k, p->dev_base + p->off_pool8, 128, p->pages8 * 128, 2 * kTile);
         if (rc) return fail(rc);
     }
     *out = p;
@@ -543,7 +542,6 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
         PagedFp8Args p8;
         p8.pa = pa;
         p8.map_k = p->map_k;
-        p8.map_v = p->map_v;
         RLKV_CUDA(launch_decode(a, &p->tmap, p->head_dim, grid, p->stages, p->groups, stream, overlap, kModePagedFp8, nullptr,
                                 &p8));
     } else {
