@@ -126,3 +126,18 @@ def test_paged_size_and_argument_checks_need_no_device(binding):
         with pytest.raises(binding.RlkvError) as e:
             call()
         assert e.value.code == binding.RLKV_EINVAL
+
+
+def test_paged_fp8_size_is_half_the_pool(binding):
+    """8-bit storage: a page of a full head and a 64-row ring tile are 16 KB (K codes and transposed V
+    codes) where the 16-bit cache needs 32 KB; the rest of the buffer is the same."""
+    ok = dict(layers=2, kv_heads=2, q_heads=8, head_dim=128, max_seqs=600, n_pages=10, max_seq_len=1000,
+              head_is_full=[1, 0, 0, 1], sink=4, window=60)
+    page16, page8 = 2 * 64 * 128 * 2, 2 * 64 * 128
+    for grow, unit in ((dict(n_pages=10 + 1000), 2 * 1000), (dict(max_seqs=600 + 256), 2 * 256)):
+        d16 = binding.rlkv_paged_size(**{**ok, **grow}) - binding.rlkv_paged_size(**ok)
+        d8 = binding.rlkv_paged_size_fp8(**{**ok, **grow}) - binding.rlkv_paged_size_fp8(**ok)
+        assert d16 - d8 == unit * (page16 - page8)
+    with pytest.raises(binding.RlkvError) as e:
+        binding.rlkv_paged_size_fp8(**{**ok, "head_dim": 64})
+    assert e.value.code == binding.RLKV_EINVAL
