@@ -15,6 +15,9 @@ bf16 N(0,1); head classes come from a seeded global selection (see synth/).
   e2e        the same K steps through rlkv_step_host: pinned host inputs copied in and the result
              copied out inside the timed region
   cpu_baseline  the CPU oracle on a bounded sample (rank 0, N=1 only), scaled by bytes
+  mixed_attention, paged_cache   side measurements at N=1 (not part of `value`): the mixed-attention
+             call of Eq. 1 beside the plain call on all-full layers; the paged cache with uniform and
+             with ragged lengths, per launch and through rlkv_paged_step, and its 8-bit variant
 
 With N > 1 (torchrun) every rank runs the same workload on its own GPU: the path shards by batch
 rows / replicas with no exchange step, so there is no collective on the data path (weak scaling).
