@@ -246,11 +246,9 @@ struct Smem {
     static constexpr int kTilePairBytes = 2 * kTileBytes;   // K tile then V tile
     // a stage: K tile, V tile, then the G query rows of the tile's unit (filled for the first NG
     // tiles of a segment), padded so that the next stage starts on a 1024-byte boundary again
-    // (8-bit pages: a stage is one 16 KB page of codes, K then V transposed, and the query rows)
-    __host__ __device__ static constexpr int tile_pair_bytes(int mode)
-    {
-        return mode == kModePagedFp8 ? kTilePairBytes / 2 : kTilePairBytes;
-    }
+    // (8-bit pages: a stage is TWO consecutive 16 KB pages of a unit, tiles 2p and 2p + 1, each K codes
+    // then V codes transposed: the per-stage costs are then paid per 128 tokens)
+    __host__ __device__ static constexpr int tile_pair_bytes(int /*mode*/) { return kTilePairBytes; }
     __host__ __device__ static constexpr int stage_bytes(int group, int mode = kModePlain)
     {
         return tile_pair_bytes(mode) + (group * D * 2 + 1023) / 1024 * 1024;
@@ -578,7 +576,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     uint32_t qa[KS][2];
                     bool have_q = false;
                     int valid_left = u.len - u.pos.tile * kTile;  // valid rows from this tile to the unit's end
-                    for (int i = 0; alive && i < seg_eff; ++i, next_slot(), valid_left -= kTile) {
+                    int step = 1;  // tiles in the slot (8-bit pages: two where the unit has an even-odd pair here)
+                    for (int i = 0; alive && i < seg_eff; i += step, next_slot(), valid_left -= step * kTile) {
+                        if (FP8) step = ((u.pos.tile + i) & 1) ? 1 : min(2, seg_eff - i);
                         if (turn != grp) continue;
                         alive = wait_traced(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout, tr0,
                                             &ns_tile);
@@ -621,10 +621,14 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             have_q = true;
                         }
                         if (FP8 && fp8_unit) {
+                            for (int sb = 0; sb < step; ++sb) {
+                            const int valid = min(kTile, valid_left - sb * kTile);  // of this tile of the slot
                             if (wig * 16 < valid) {
-                                // a stage of an 8-bit page, 128 rows of 128 bytes under the 128-byte swizzle: K codes
-                                // [64 tokens][128], then V codes transposed [128 d][64 tokens], two d per row
-                                const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
+                                // an 8-bit page, 128 rows of 128 bytes under the 128-byte swizzle: K codes
+                                // [64 tokens][128], then V codes transposed [128 d][64 tokens], two d per row;
+                                // an even tile's page is the first of the stage, an odd tile's the second
+                                const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes) +
+                                                    ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128);
                                 const uint32_t sV = sK + kTile * 128;
                                 // ---- S = Q.K^T.  ldmatrix row i of token set s is token 4(i/2) + 2s + (i%2) of
                                 // the warp's 16, so that this lane ends up with four consecutive tokens
@@ -707,6 +711,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                     acc[2 * mp + 1][3] *= cb;
                                     mma_f16(acc[2 * mp + 1], a0, a1, a2, a3, pb0, pb1);
                                 }
+                            }
                             }
                         } else if (wig * 16 < valid) {
                             const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
@@ -993,14 +998,22 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                         }
                     }
-                    if (FP8 && paged_row0 < 0) krow = ring_next++;
-                    if (PAGED && paged_row0 >= 0) {
-                        if (FP8) {  // the page itself; its row coordinates in the two 8-bit maps follow below
-                            krow = paged_row0 + s_pages[paged_tile++ - page_base];
+                    // 8-bit pages: the slot holds tiles 2p and 2p + 1 of the unit where the segment has both,
+                    // else the one it has, each in its own half of the stage
+                    int n_sub = 1, pg0 = 0, pg1 = 0;
+                    if (FP8) {
+                        n_sub = (paged_tile & 1) ? 1 : min(2, seg_left);
+                        if (paged_row0 >= 0) {
+                            pg0 = paged_row0 + s_pages[paged_tile - page_base];
+                            if (n_sub == 2) pg1 = paged_row0 + s_pages[paged_tile + 1 - page_base];
                         } else {
-                            krow = paged_row0 + s_pages[paged_tile++ - page_base] * (2 * kTile);
-                            vrow = krow + kTile;
+                            pg0 = ring_next;
+                            pg1 = ring_next + 1;
+                            ring_next += n_sub;
                         }
+                    } else if (PAGED && paged_row0 >= 0) {
+                        krow = paged_row0 + s_pages[paged_tile++ - page_base] * (2 * kTile);
+                        vrow = krow + kTile;
                     }
                     if (MIXED && local_row0 >= 0) {
                         int row, valid;
@@ -1015,13 +1028,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     const uint32_t fb = smem_u32(full_bar + s);
                     const bool with_q = seg_idx < NG;  // each consumer group reads q at its first tile of the segment
                     const long long tc0 = trace ? clock64() : 0;
-                    mbar_expect_tx(fb, kPairBytes + (with_q ? G * D * 2 : 0));
+                    mbar_expect_tx(fb, (FP8 ? n_sub * (kPairBytes / 2) : kPairBytes) + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
                     const long long tc1 = trace ? clock64() : 0;
                     if constexpr (FP8) {
-                        // page krow in one box of 128 rows of 128 bytes: 64 rows of K codes, then the transposed V
+                        // a page in one box of 128 rows of 128 bytes: 64 rows of K codes, then the transposed V
                         // codes, two d per row
-                        tma_load_2d(dst, &extra.map_k, 0, krow * 128, fb, stream_policy);
+                        tma_load_2d(dst + (paged_tile & 1) * (kPairBytes / 2), &extra.map_k, 0, pg0 * 128, fb, stream_policy);
+                        if (n_sub == 2) tma_load_2d(dst + kPairBytes / 2, &extra.map_k, 0, pg1 * 128, fb, stream_policy);
+                        paged_tile += n_sub;
                     } else if (D == 128) {  // one box per tile, 16 KB contiguous in memory: [2 halves][64 rows][64]
                         tma_load_3d(dst, &tmap, 0, krow, 0, fb, stream_policy);
                         tma_load_3d(dst + S::kTileBytes, &tmap, 0, vrow, 0, fb, stream_policy);
@@ -1040,7 +1055,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     krow += kTile;
                     vrow += kTile;
                     ++seg_idx;
-                    --seg_left;
+                    seg_left -= n_sub;
+                    x += n_sub - 1;
                     ++issued;
                     if (++s == stages) {
                         s = 0;
