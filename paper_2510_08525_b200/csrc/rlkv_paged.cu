@@ -505,7 +505,8 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
     int grid = p->sm_count;
     if (grid > p->max_grid) grid = p->max_grid;
     int item_tiles = (int)(real_tiles / grid);
-    const int most = in_step ? kPagedItemTilesStep : p->item_tiles;
+    // (a tile of 8-bit pages is half the bytes, so the same grain in time is twice the tiles)
+    const int most = (in_step ? kPagedItemTilesStep : p->item_tiles) * (p->fp8 ? 2 : 1);
     if (item_tiles > most) item_tiles = most;
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     a.sched = make_schedule(n * a.n_full, tiles_full, n * a.n_comp, tiles_comp, grid, item_tiles);
