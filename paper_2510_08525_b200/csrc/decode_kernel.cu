@@ -621,97 +621,116 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             have_q = true;
                         }
                         if (FP8 && fp8_unit) {
-                            for (int sb = 0; sb < step; ++sb) {
-                            const int valid = min(kTile, valid_left - sb * kTile);  // of this tile of the slot
-                            if (wig * 16 < valid) {
-                                // an 8-bit page, 128 rows of 128 bytes under the 128-byte swizzle: K codes
-                                // [64 tokens][128], then V codes transposed [128 d][64 tokens], two d per row;
-                                // an even tile's page is the first of the stage, an odd tile's the second
-                                const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes) +
-                                                    ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128);
-                                const uint32_t sV = sK + kTile * 128;
-                                // ---- S = Q.K^T.  ldmatrix row i of token set s is token 4(i/2) + 2s + (i%2) of
-                                // the warp's 16, so that this lane ends up with four consecutive tokens
-                                const int lj = lane >> 3, li = lane & 7;
-                                const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
-                                float sA[4] = {0.f, 0.f, 0.f, 0.f}, sB[4] = {0.f, 0.f, 0.f, 0.f};
-                                float sA2[4] = {0.f, 0.f, 0.f, 0.f}, sB2[4] = {0.f, 0.f, 0.f, 0.f};
-                                // all fragments of K first, then the arithmetic: the loads' latencies overlap
-                                uint32_t kf[KS / 2][4];
+                            // The slot's tiles (two where the unit has an even-odd pair here): an 8-bit page is 128
+                            // rows of 128 bytes under the 128-byte swizzle, K codes [64 tokens][128], then V codes
+                            // transposed [128 d][64 tokens], two d per row; an even tile's page is the first of
+                            // the stage, an odd tile's the second.  The scores of both tiles go through ONE
+                            // softmax update: one maximum, one correction of the accumulators per 128 tokens.
+                            const int lj = lane >> 3, li = lane & 7;
+                            // ldmatrix row i of token set s is token 4(i/2) + 2s + (i%2) of the warp's 16, so that
+                            // this lane ends up with four consecutive tokens
+                            const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
+                            const uint32_t stage0 = smem_u32(stage_base + (size_t)st * stage_bytes);
+                            const float sl2 = a.scale_log2 * pg->k_scale[u.head];  // K's scale joins the softmax scale
+                            float sc8[2][4];
+                            bool active[2];
 #pragma unroll
-                                for (int kp = 0; kp < KS / 2; ++kp) {
-                                    const int chunk = 2 * kp + (lj >> 1);  // 16 codes along d
-                                    ldmatrix_x4(sK + ktok * 128 + ((chunk ^ (ktok & 7)) << 4), kf[kp][0], kf[kp][1], kf[kp][2],
-                                                kf[kp][3]);
-                                }
+                            for (int sb = 0; sb < 2; ++sb) {
+                                const int valid_sb = min(kTile, valid_left - sb * kTile);  // of this tile of the slot
+                                active[sb] = sb < step && wig * 16 < valid_sb;
+                                sc8[sb][0] = sc8[sb][1] = sc8[sb][2] = sc8[sb][3] = -INFINITY;
+                                if (active[sb]) {
+                                    const uint32_t sK = stage0 + ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128);
+                                    // ---- S = Q.K^T: all fragments of K first, then the arithmetic
+                                    float sA[4] = {0.f, 0.f, 0.f, 0.f}, sB[4] = {0.f, 0.f, 0.f, 0.f};
+                                    float sA2[4] = {0.f, 0.f, 0.f, 0.f}, sB2[4] = {0.f, 0.f, 0.f, 0.f};
+                                    uint32_t kf[KS / 2][4];
 #pragma unroll
-                                for (int kp = 0; kp < KS / 2; ++kp) {
-                                    const uint32_t r0 = kf[kp][0], r1 = kf[kp][1], r2 = kf[kp][2], r3 = kf[kp][3];
-                                    uint32_t b0, b1;
-                                    e4m3x4_to_f16x2x2(r0, b0, b1);
-                                    mma_f16(sA, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                                    e4m3x4_to_f16x2x2(r1, b0, b1);
-                                    mma_f16(sB, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                                    e4m3x4_to_f16x2x2(r2, b0, b1);
-                                    mma_f16(sA2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
-                                    e4m3x4_to_f16x2x2(r3, b0, b1);
-                                    mma_f16(sB2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
-                                }
-                                // the fragments of V are fetched now, under the softmax
-                                uint32_t vf[KS / 2][4];
+                                    for (int kp = 0; kp < KS / 2; ++kp) {
+                                        const int chunk = 2 * kp + (lj >> 1);  // 16 codes along d
+                                        ldmatrix_x4(sK + ktok * 128 + ((chunk ^ (ktok & 7)) << 4), kf[kp][0], kf[kp][1],
+                                                    kf[kp][2], kf[kp][3]);
+                                    }
 #pragma unroll
-                                for (int mp = 0; mp < KS / 2; ++mp) {
-                                    // row d of the transposed block is half of 128-byte row d / 2 of the stage
-                                    const int vd = 16 * (2 * mp + (lj >> 1)) + 8 * (lj & 1) + li, vr = vd >> 1;
-                                    ldmatrix_x4(sV + vr * 128 + ((((vd & 1) * 4 + wig) ^ (vr & 7)) << 4), vf[mp][0], vf[mp][1],
-                                                vf[mp][2], vf[mp][3]);
+                                    for (int kp = 0; kp < KS / 2; ++kp) {
+                                        uint32_t b0, b1;
+                                        e4m3x4_to_f16x2x2(kf[kp][0], b0, b1);
+                                        mma_f16(sA, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
+                                        e4m3x4_to_f16x2x2(kf[kp][1], b0, b1);
+                                        mma_f16(sB, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
+                                        e4m3x4_to_f16x2x2(kf[kp][2], b0, b1);
+                                        mma_f16(sA2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                        e4m3x4_to_f16x2x2(kf[kp][3], b0, b1);
+                                        mma_f16(sB2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                    }
+                                    // this lane: head `quad`, tokens wig*16 + 4tq + {0, 1, 2, 3} of the tile
+                                    sc8[sb][0] = (sA[0] + sA2[0]) * sl2;
+                                    sc8[sb][1] = (sA[1] + sA2[1]) * sl2;
+                                    sc8[sb][2] = (sB[0] + sB2[0]) * sl2;
+                                    sc8[sb][3] = (sB[1] + sB2[1]) * sl2;
+                                    const int tok0 = wig * 16 + 4 * tq;
+                                    if (tok0 >= valid_sb) sc8[sb][0] = -INFINITY;
+                                    if (tok0 + 1 >= valid_sb) sc8[sb][1] = -INFINITY;
+                                    if (tok0 + 2 >= valid_sb) sc8[sb][2] = -INFINITY;
+                                    if (tok0 + 3 >= valid_sb) sc8[sb][3] = -INFINITY;
                                 }
-                                // this lane: head `quad`, tokens wig*16 + 4tq + {0, 1, 2, 3}; K's scale joins the softmax scale
-                                const float sl2 = a.scale_log2 * pg->k_scale[u.head];
-                                float sc4[4];
-                                sc4[0] = (sA[0] + sA2[0]) * sl2;
-                                sc4[1] = (sA[1] + sA2[1]) * sl2;
-                                sc4[2] = (sB[0] + sB2[0]) * sl2;
-                                sc4[3] = (sB[1] + sB2[1]) * sl2;
-                                const int tok0 = wig * 16 + 4 * tq;
-                                if (tok0 >= valid) sc4[0] = -INFINITY;
-                                if (tok0 + 1 >= valid) sc4[1] = -INFINITY;
-                                if (tok0 + 2 >= valid) sc4[2] = -INFINITY;
-                                if (tok0 + 3 >= valid) sc4[3] = -INFINITY;
-                                float mx = fmaxf(fmaxf(sc4[0], sc4[1]), fmaxf(sc4[2], sc4[3]));
+                            }
+                            if (active[0] || active[1]) {  // uniform over the warp
+                                // ---- one online-softmax update for the slot (log2 domain)
+                                float mx = fmaxf(fmaxf(fmaxf(sc8[0][0], sc8[0][1]), fmaxf(sc8[0][2], sc8[0][3])),
+                                                 fmaxf(fmaxf(sc8[1][0], sc8[1][1]), fmaxf(sc8[1][2], sc8[1][3])));
                                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                                 const float m_new = fmaxf(m_run, mx);
                                 const float corr = exp2f(m_run - m_new);
-                                const float p0 = exp2f(sc4[0] - m_new), p1 = exp2f(sc4[1] - m_new);
-                                const float p2 = exp2f(sc4[2] - m_new), p3 = exp2f(sc4[3] - m_new);
-                                l_run = l_run * corr + ((p0 + p1) + (p2 + p3));
+                                float pr[2][4];
+                                float psum = 0.f;
+#pragma unroll
+                                for (int sb = 0; sb < 2; ++sb) {
+                                    pr[sb][0] = exp2f(sc8[sb][0] - m_new);
+                                    pr[sb][1] = exp2f(sc8[sb][1] - m_new);
+                                    pr[sb][2] = exp2f(sc8[sb][2] - m_new);
+                                    pr[sb][3] = exp2f(sc8[sb][3] - m_new);
+                                    psum += (pr[sb][0] + pr[sb][1]) + (pr[sb][2] + pr[sb][3]);
+                                }
+                                l_run = l_run * corr + psum;
                                 m_run = m_new;
+                                // O^T columns of this lane are heads 2tq and 2tq+1: fetch their corrections
                                 const float ca = __shfl_sync(0xffffffffu, corr, tq * 8);
                                 const float cb = __shfl_sync(0xffffffffu, corr, tq * 8 + 4);
-                                const uint32_t pb0 = pack_f16(p0, p1), pb1 = pack_f16(p2, p3);
-                                // ---- O^T[d][head] += V^T[d][tok] . P^T[tok][head]: V^T rows come straight out of
-                                // the transposed page, four consecutive tokens per lane
 #pragma unroll
-                                for (int mp = 0; mp < KS / 2; ++mp) {
-                                    const uint32_t r0 = vf[mp][0], r1 = vf[mp][1], r2 = vf[mp][2], r3 = vf[mp][3];
-                                    uint32_t a0, a1, a2, a3;
-                                    e4m3x4_to_f16x2x2(r0, a0, a2);
-                                    e4m3x4_to_f16x2x2(r1, a1, a3);
-                                    acc[2 * mp][0] *= ca;
-                                    acc[2 * mp][1] *= cb;
-                                    acc[2 * mp][2] *= ca;
-                                    acc[2 * mp][3] *= cb;
-                                    mma_f16(acc[2 * mp], a0, a1, a2, a3, pb0, pb1);
-                                    e4m3x4_to_f16x2x2(r2, a0, a2);
-                                    e4m3x4_to_f16x2x2(r3, a1, a3);
-                                    acc[2 * mp + 1][0] *= ca;
-                                    acc[2 * mp + 1][1] *= cb;
-                                    acc[2 * mp + 1][2] *= ca;
-                                    acc[2 * mp + 1][3] *= cb;
-                                    mma_f16(acc[2 * mp + 1], a0, a1, a2, a3, pb0, pb1);
+                                for (int mt = 0; mt < KS; ++mt) {
+                                    acc[mt][0] *= ca;
+                                    acc[mt][1] *= cb;
+                                    acc[mt][2] *= ca;
+                                    acc[mt][3] *= cb;
                                 }
-                            }
+                                // ---- O^T[d][head] += V^T[d][tok] . P^T[tok][head], tile by tile: V^T rows come
+                                // straight out of the transposed page, four consecutive tokens per lane
+#pragma unroll
+                                for (int sb = 0; sb < 2; ++sb) {
+                                    if (!active[sb]) continue;
+                                    const uint32_t sV = stage0 + ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128) + kTile * 128;
+                                    const uint32_t pb0 = pack_f16(pr[sb][0], pr[sb][1]), pb1 = pack_f16(pr[sb][2], pr[sb][3]);
+                                    uint32_t vf[KS / 2][4];
+#pragma unroll
+                                    for (int mp = 0; mp < KS / 2; ++mp) {
+                                        // row d of the transposed block is half of 128-byte row d / 2 of the page
+                                        const int vd = 16 * (2 * mp + (lj >> 1)) + 8 * (lj & 1) + li, vr = vd >> 1;
+                                        ldmatrix_x4(sV + vr * 128 + ((((vd & 1) * 4 + wig) ^ (vr & 7)) << 4), vf[mp][0], vf[mp][1],
+                                                    vf[mp][2], vf[mp][3]);
+                                    }
+#pragma unroll
+                                    for (int mp = 0; mp < KS / 2; ++mp) {
+                                        uint32_t a0, a1, a2, a3;
+                                        e4m3x4_to_f16x2x2(vf[mp][0], a0, a2);
+                                        e4m3x4_to_f16x2x2(vf[mp][1], a1, a3);
+                                        mma_f16(acc[2 * mp], a0, a1, a2, a3, pb0, pb1);
+                                        e4m3x4_to_f16x2x2(vf[mp][2], a0, a2);
+                                        e4m3x4_to_f16x2x2(vf[mp][3], a1, a3);
+                                        mma_f16(acc[2 * mp + 1], a0, a1, a2, a3, pb0, pb1);
+                                    }
+                                }
                             }
                         } else if (wig * 16 < valid) {
                             const uint32_t sK = smem_u32(stage_base + (size_t)st * stage_bytes);
