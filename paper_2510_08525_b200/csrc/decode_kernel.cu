@@ -178,6 +178,14 @@ __device__ __forceinline__ void e4m3x4_to_f16x2x2(uint32_t codes, uint32_t& lo, 
         : "=r"(lo), "=r"(hi)
         : "r"(codes));
 }
+// Transposes an 8x8 matrix of 16-bit elements held one row per quad of lanes (lane l: row l / 4,
+// columns 2(l % 4) and 2(l % 4) + 1): afterwards the lane holds the same positions of the transpose.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
 {
     __half2 v = __floats2half2_rn(lo, hi);
@@ -548,6 +556,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 UnitInfo u{};
                 int seg_tiles = 0;
                 float m_run = kNegBig, l_run = 0.f;
+                // 8-bit pages: the first product has the tokens as rows and the heads as columns, so a lane
+                // keeps the running maximum and sum of heads 2tq (m_run, l_run) and 2tq + 1 (these)
+                float m_run1 = kNegBig, l_run1 = 0.f;
                 float acc[KS][4];
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
@@ -632,6 +643,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
                             const uint32_t stage0 = smem_u32(stage_base + (size_t)st * stage_bytes);
                             const float sl2 = a.scale_log2 * pg->k_scale[u.head];  // K's scale joins the softmax scale
+                            // scores of this lane per tile: [0], [1] token row `quad` of set A, heads 2tq and 2tq+1;
+                            // [2], [3] token row `quad` of set B, the same heads
                             float sc8[2][4];
                             bool active[2];
 #pragma unroll
@@ -641,9 +654,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 sc8[sb][0] = sc8[sb][1] = sc8[sb][2] = sc8[sb][3] = -INFINITY;
                                 if (active[sb]) {
                                     const uint32_t sK = stage0 + ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128);
-                                    // ---- S = Q.K^T: all fragments of K first, then the arithmetic
-                                    float sA[4] = {0.f, 0.f, 0.f, 0.f}, sB[4] = {0.f, 0.f, 0.f, 0.f};
-                                    float sA2[4] = {0.f, 0.f, 0.f, 0.f}, sB2[4] = {0.f, 0.f, 0.f, 0.f};
+                                    // ---- S^T = K.Q^T: the 16 tokens are the rows (set A rows 0-7, set B rows 8-15),
+                                    // the query heads the 8 columns -- one MMA per 16 d, where the heads as rows
+                                    // would take two, half of them padding.  All fragments of K first.
+                                    float se[4] = {0.f, 0.f, 0.f, 0.f}, so[4] = {0.f, 0.f, 0.f, 0.f};
                                     uint32_t kf[KS / 2][4];
 #pragma unroll
                                     for (int kp = 0; kp < KS / 2; ++kp) {
@@ -653,51 +667,52 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                     }
 #pragma unroll
                                     for (int kp = 0; kp < KS / 2; ++kp) {
-                                        uint32_t b0, b1;
-                                        e4m3x4_to_f16x2x2(kf[kp][0], b0, b1);
-                                        mma_f16(sA, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                                        e4m3x4_to_f16x2x2(kf[kp][1], b0, b1);
-                                        mma_f16(sB, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, b0, b1);
-                                        e4m3x4_to_f16x2x2(kf[kp][2], b0, b1);
-                                        mma_f16(sA2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
-                                        e4m3x4_to_f16x2x2(kf[kp][3], b0, b1);
-                                        mma_f16(sB2, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, b0, b1);
+                                        uint32_t a0, a1, a2, a3;
+                                        e4m3x4_to_f16x2x2(kf[kp][0], a0, a2);  // set A, chunk 2kp
+                                        e4m3x4_to_f16x2x2(kf[kp][1], a1, a3);  // set B, chunk 2kp
+                                        mma_f16(se, a0, a1, a2, a3, qa[2 * kp][0], qa[2 * kp][1]);
+                                        e4m3x4_to_f16x2x2(kf[kp][2], a0, a2);  // set A, chunk 2kp + 1
+                                        e4m3x4_to_f16x2x2(kf[kp][3], a1, a3);  // set B, chunk 2kp + 1
+                                        mma_f16(so, a0, a1, a2, a3, qa[2 * kp + 1][0], qa[2 * kp + 1][1]);
                                     }
-                                    // this lane: head `quad`, tokens wig*16 + 4tq + {0, 1, 2, 3} of the tile
-                                    sc8[sb][0] = (sA[0] + sA2[0]) * sl2;
-                                    sc8[sb][1] = (sA[1] + sA2[1]) * sl2;
-                                    sc8[sb][2] = (sB[0] + sB2[0]) * sl2;
-                                    sc8[sb][3] = (sB[1] + sB2[1]) * sl2;
-                                    const int tok0 = wig * 16 + 4 * tq;
-                                    if (tok0 >= valid_sb) sc8[sb][0] = -INFINITY;
-                                    if (tok0 + 1 >= valid_sb) sc8[sb][1] = -INFINITY;
-                                    if (tok0 + 2 >= valid_sb) sc8[sb][2] = -INFINITY;
-                                    if (tok0 + 3 >= valid_sb) sc8[sb][3] = -INFINITY;
+                                    sc8[sb][0] = (se[0] + so[0]) * sl2;
+                                    sc8[sb][1] = (se[1] + so[1]) * sl2;
+                                    sc8[sb][2] = (se[2] + so[2]) * sl2;
+                                    sc8[sb][3] = (se[3] + so[3]) * sl2;
+                                    // row `quad` of set A is token 4(quad/2) + quad%2 of the warp's 16, of set B two on
+                                    const int tokA = wig * 16 + 4 * (quad >> 1) + (quad & 1);
+                                    if (tokA >= valid_sb) sc8[sb][0] = sc8[sb][1] = -INFINITY;
+                                    if (tokA + 2 >= valid_sb) sc8[sb][2] = sc8[sb][3] = -INFINITY;
                                 }
                             }
                             if (active[0] || active[1]) {  // uniform over the warp
-                                // ---- one online-softmax update for the slot (log2 domain)
-                                float mx = fmaxf(fmaxf(fmaxf(sc8[0][0], sc8[0][1]), fmaxf(sc8[0][2], sc8[0][3])),
-                                                 fmaxf(fmaxf(sc8[1][0], sc8[1][1]), fmaxf(sc8[1][2], sc8[1][3])));
-                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                                const float m_new = fmaxf(m_run, mx);
-                                const float corr = exp2f(m_run - m_new);
+                                // ---- one online-softmax update for the slot (log2 domain): the maxima of heads 2tq
+                                // and 2tq+1 over this lane's tokens, then over the quads
+                                float mx0 = fmaxf(fmaxf(sc8[0][0], sc8[0][2]), fmaxf(sc8[1][0], sc8[1][2]));
+                                float mx1 = fmaxf(fmaxf(sc8[0][1], sc8[0][3]), fmaxf(sc8[1][1], sc8[1][3]));
+#pragma unroll
+                                for (int o = 4; o < 32; o <<= 1) {
+                                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, o));
+                                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, o));
+                                }
+                                const float mn0 = fmaxf(m_run, mx0), mn1 = fmaxf(m_run1, mx1);
+                                const float ca = exp2f(m_run - mn0), cb = exp2f(m_run1 - mn1);
                                 float pr[2][4];
-                                float psum = 0.f;
+                                float ps0 = 0.f, ps1 = 0.f;
 #pragma unroll
                                 for (int sb = 0; sb < 2; ++sb) {
-                                    pr[sb][0] = exp2f(sc8[sb][0] - m_new);
-                                    pr[sb][1] = exp2f(sc8[sb][1] - m_new);
-                                    pr[sb][2] = exp2f(sc8[sb][2] - m_new);
-                                    pr[sb][3] = exp2f(sc8[sb][3] - m_new);
-                                    psum += (pr[sb][0] + pr[sb][1]) + (pr[sb][2] + pr[sb][3]);
+                                    pr[sb][0] = exp2f(sc8[sb][0] - mn0);
+                                    pr[sb][1] = exp2f(sc8[sb][1] - mn1);
+                                    pr[sb][2] = exp2f(sc8[sb][2] - mn0);
+                                    pr[sb][3] = exp2f(sc8[sb][3] - mn1);
+                                    ps0 += pr[sb][0] + pr[sb][2];
+                                    ps1 += pr[sb][1] + pr[sb][3];
                                 }
-                                l_run = l_run * corr + psum;
-                                m_run = m_new;
-                                // O^T columns of this lane are heads 2tq and 2tq+1: fetch their corrections
-                                const float ca = __shfl_sync(0xffffffffu, corr, tq * 8);
-                                const float cb = __shfl_sync(0xffffffffu, corr, tq * 8 + 4);
+                                l_run = l_run * ca + ps0;
+                                l_run1 = l_run1 * cb + ps1;
+                                m_run = mn0;
+                                m_run1 = mn1;
+                                // O^T columns of this lane are heads 2tq and 2tq+1: its own corrections
 #pragma unroll
                                 for (int mt = 0; mt < KS; ++mt) {
                                     acc[mt][0] *= ca;
@@ -711,7 +726,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 for (int sb = 0; sb < 2; ++sb) {
                                     if (!active[sb]) continue;
                                     const uint32_t sV = stage0 + ((u.pos.tile + i + sb) & 1) * (2 * kTile * 128) + kTile * 128;
-                                    const uint32_t pb0 = pack_f16(pr[sb][0], pr[sb][1]), pb1 = pack_f16(pr[sb][2], pr[sb][3]);
+                                    // P is held tokens x heads; the second product wants it heads x tokens
+                                    const uint32_t pb0 = movmatrix_trans(pack_f16(pr[sb][0], pr[sb][1]));
+                                    const uint32_t pb1 = movmatrix_trans(pack_f16(pr[sb][2], pr[sb][3]));
                                     uint32_t vf[KS / 2][4];
 #pragma unroll
                                     for (int mp = 0; mp < KS / 2; ++mp) {
@@ -816,13 +833,27 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         acc[mt][3] *= vs;
                     }
                 }
-                if (item >= 0) {
+                if (FP8 && item >= 0) {  // sums over the lanes that hold the other tokens (same tq, other quads)
+#pragma unroll
+                    for (int o = 4; o < 32; o <<= 1) {
+                        l_run += __shfl_xor_sync(0xffffffffu, l_run, o);
+                        l_run1 += __shfl_xor_sync(0xffffffffu, l_run1, o);
+                    }
+                    if (quad == 0) {
+                        stat_m[warp * kMaxGroup + 2 * tq] = m_run;
+                        stat_l[warp * kMaxGroup + 2 * tq] = l_run;
+                        stat_m[warp * kMaxGroup + 2 * tq + 1] = m_run1;
+                        stat_l[warp * kMaxGroup + 2 * tq + 1] = l_run1;
+                    }
+                } else if (item >= 0) {
                     l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
                     l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
                     if (tq == 0) {
                         stat_m[warp * kMaxGroup + quad] = m_run;
                         stat_l[warp * kMaxGroup + quad] = l_run;
                     }
+                }
+                if (item >= 0) {
                     float* mw = merge + (size_t)warp * G * MS;
                     const int h0 = 2 * tq, h1 = 2 * tq + 1;
 #pragma unroll
