@@ -456,7 +456,7 @@ def run_ours(args, w, mask):
         paged = {"workload": f"first {pl} layers of the {w.name} mask, {w.batch} sequences, launches back to back"}
         variants = [("uniform", [n] * w.batch, False), ("ragged", spread, False)]
         if w.head_dim == 128:
-            variants.append(("uniform_fp8", [n] * w.batch, True))   # the full heads' pages as E4M3 codes
+            variants.append(("uniform_fp8", [n] * w.batch, True))   # every K/V row as an E4M3 code
         for name, lens, fp8 in variants:
             pages = sum((x + 63) // 64 for x in lens) + 2 + 2 * len(lens)
             scales = np.full(pl * w.kv_heads, 1.0 / 64, np.float32) if fp8 else None   # N(0,1) inputs stay well inside +-448

@@ -11,7 +11,10 @@
  *
  * Conventions
  *   - Every function returns 0 (RLKV_OK) or a negative RLKV_E* code; nothing throws, exits or
- *     prints.  A call that returns an error leaves the cache state untouched.
+ *     prints.  A call that returns RLKV_EINVAL, RLKV_EFULL, RLKV_EEMPTY, RLKV_ENOMEM or
+ *     RLKV_ESCRATCH has changed nothing: these are found before anything is enqueued.  RLKV_ECUDA
+ *     means a CUDA call failed part-way (normally the context is lost with it): lengths and cache
+ *     contents are then unspecified and the cache should be destroyed.
  *   - "device" pointers are CUDA device memory on the GPU that was current at rlkv_cache_create;
  *     "host" pointers are ordinary host memory.  The caller owns every buffer it passes in.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All GPU work is
@@ -57,7 +60,7 @@ enum {
 int rlkv_cache_size(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
                     const uint8_t* head_is_full, int sink, int window, size_t* bytes_out);
 
-/* Two-class cache layout (Section 4.3: "dual KV pool").  device_buf == NULL: the library
+/* Two-class cache layout (the two KV pools of Section 4.3).  device_buf == NULL: the library
  * cudaMallocs the memory and frees it in rlkv_cache_destroy.  Otherwise the caller provides
  * device_buf (1024-byte aligned, >= rlkv_cache_size bytes) and keeps it alive until destroy.
  * The pools are zero-filled, head_is_full is copied, all lengths start at 0.  Synchronous. */
@@ -69,8 +72,8 @@ int rlkv_cache_destroy(rlkv_cache* cache);
 /* All lengths back to 0 and the pools re-zeroed (asynchronous on `stream`). */
 int rlkv_cache_reset(rlkv_cache* cache, void* stream);
 
-/* Fused append (Section 4.3 circular buffer; Appendix B "first ... sink tokens and the recent ...
- * local tokens").  k, v: device bf16 [batch][kv_heads][head_dim] -- all KV heads; the caller does
+/* Fused append (Section 4.3: circular buffer; Appendix B: the first sink tokens and the most
+ * recent local tokens are kept).  k, v: device bf16 [batch][kv_heads][head_dim] -- all KV heads; the caller does
  * not need to know their classes.  Token t = length(layer) goes to row t of a full head and to
  * slot(t) of a compressed head; then length(layer) = t + 1.  Copies are bit-exact.
  * RLKV_EFULL if length(layer) == max_len. */
@@ -83,8 +86,9 @@ int rlkv_prefill(rlkv_cache* cache, int layer, const void* k, const void* v, int
                  void* stream);
 
 /* Split-KV decode attention over the heterogeneous heads of one layer, one launch for both head
- * classes (Section 3.3: compressed heads "still use full attention but with compressed KV cache";
- * Section 4.3 asks for exactly this fused heterogeneous-head kernel).
+ * classes (Section 3.3, last paragraph: a compressed head runs the same full attention, only over
+ * the rows its smaller cache retains; Section 4.3 names a fused kernel for heterogeneous heads as
+ * what would close the gap to the cost model).
  * q: device bf16 [batch][q_heads][head_dim]; out: device fp32 [batch][q_heads][head_dim].
  * Scores, softmax and accumulation are fp32.  RLKV_EEMPTY if length(layer) == 0. */
 int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out, void* stream);
@@ -109,7 +113,9 @@ int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out
  *   launched.
  * - The first call on a device looks up the array's device address (one runtime query, kept for
  *   the life of the process; a driver that loads modules lazily gives the array its memory at that
- *   moment); make that first call at start-up, before starting any stream capture.
+ *   moment); make that first call at start-up, before starting any stream capture.  Two host
+ *   threads may make their first calls on one device at the same time: both look the address up,
+ *   get the same answer, and the slot that keeps it is written atomically.
  * - Every cache and every call on a device share the one array, which still holds the previous
  *   call's contents: each call clears the tickets and work-claim counters on `stream` before its launch.  Two such calls
  *   that overlap on the GPU (different streams, no ordering between them) race on the array and
@@ -320,6 +326,18 @@ int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_ho
 int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas,
                         int item_tiles, int* n_items_out, int* n_slots_out, int* starts_out,
                         int* tile_map_out, int cap);
+
+/* How rlkv_step and rlkv_paged_step order the decode launches of one step, host arithmetic only (no
+ * GPU).  For launch l of n_launches in a row (follows_append != 0: the first one directly follows the
+ * step's append launch in the stream): overlap_out[l] = 1 if it is launched so that it may start
+ * while launch l - 1 still runs; dep_wait_out[l] = what it waits for on the device before it lets
+ * launch l + 1 start (0: nothing -- it is an ordinary launch, whose predecessor has completed before
+ * it starts; 1: the append launch; 2: launch l - 1); scratch_copy_out[l] = which of the two copies
+ * of the split-KV scratch it uses.  Launches l and l - 2 share a copy; they are never in flight
+ * together because launch l - 1 holds launch l back until launch l - 2 has completed.  (host int
+ * [n_launches] each) */
+int rlkv_debug_step_plan(int n_launches, int follows_append, int* overlap_out, int* dep_wait_out,
+                         int* scratch_copy_out);
 
 const char* rlkv_strerror(int code);
 

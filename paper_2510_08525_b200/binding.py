@@ -44,6 +44,7 @@ SIGNATURES = {
     "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci, _ci]),
     "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
     "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
+    "rlkv_debug_step_plan": (_ci, [_ci, _ci, _vp, _vp, _vp]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
     "rlkv_paged_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
     "rlkv_paged_create": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _sz]),
@@ -258,6 +259,13 @@ def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, it
     _check(lib.rlkv_debug_schedule(*args, ctypes.byref(n), ctypes.byref(slots), starts.ctypes.data, _ptr(tmap),
                                    max(starts.size, total)))
     return (starts, int(slots.value), tmap) if tile_map else (starts, int(slots.value))
+
+
+def rlkv_debug_step_plan(n_launches, follows_append=True):
+    """Returns (overlap, dep_wait, scratch_copy), int32[n_launches] each."""
+    arrs = [np.zeros(n_launches, dtype=np.int32) for _ in range(3)]
+    _check(lib.rlkv_debug_step_plan(n_launches, int(follows_append), *[a.ctypes.data for a in arrs]))
+    return tuple(arrs)
 
 
 def rlkv_strerror(code: int) -> str:

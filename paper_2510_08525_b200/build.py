@@ -11,7 +11,11 @@ LIB = os.path.join(PKG, "librlkv.so")
 SOURCES = ["rlkv_api.cu", "rlkv_paged.cu", "append_kernel.cu", "decode_kernel.cu"]
 HEADERS = ["rlkv_internal.cuh", "rlkv_host.cuh", os.path.join("..", "..", "include", "rlkv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math", "-Xcompiler", "-fPIC", "-shared"]
+              "-Xcompiler", "-fPIC"]
+# Fast-math (approximate exp2 and division, flush-to-zero) is wanted in the decode kernel's softmax and
+# nowhere else: the append kernel's quantiser and the host arithmetic keep IEEE behaviour.
+EXTRA_FLAGS = {"decode_kernel.cu": ["--use_fast_math"]}
+OBJ_DIR = os.path.join(PKG, "_build")
 
 
 def _stale() -> bool:
@@ -27,13 +31,27 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not force and not _stale():
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-          [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    objs, procs = [], []
+    for src in SOURCES:                       # one object per source, compiled side by side
+        obj = os.path.join(OBJ_DIR, src.replace(".cu", ".o"))
+        cmd = [nvcc] + NVCC_FLAGS + EXTRA_FLAGS.get(src, []) + (["-Xptxas", "-v"] if verbose else []) + \
+              ["-c", os.path.join(CSRC, src), "-o", obj]
+        procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+        objs.append(obj)
+    failed = False
+    for src, proc in procs:
+        out, _ = proc.communicate()
+        if verbose or proc.returncode != 0:
+            sys.stderr.write(out)
+        failed = failed or proc.returncode != 0
+    if failed:
         raise RuntimeError("nvcc failed building librlkv.so")
+    res = subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a"] + objs + ["-o", LIB],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed linking librlkv.so")
     return LIB
 
 

@@ -425,7 +425,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 {
     constexpr bool MIXED = MODE == kModeMixed;
     constexpr bool PAGED = MODE == kModePaged || MODE == kModePagedFp8;
-    constexpr bool FP8 = MODE == kModePagedFp8;  // the full heads' pages hold E4M3 codes (head_dim 128 only)
+    constexpr bool FP8 = MODE == kModePagedFp8;  // pages and rings hold E4M3 codes (head_dim 128 only)
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     constexpr int MS = S::kMergeStride;
@@ -468,14 +468,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     unsigned long long* my_trace = args.trace + (size_t)blockIdx.x * kTraceWords;
     if (trace && tid == 0) my_trace[0] = global_timer_ns();
     // Overlapped launches (the layers of one decode step): the next layer's kernel is scheduled as SMs
-    // become free and touches nothing this one uses.  Only the step's first layer (dep_wait) may be
-    // running before the step's append launch has completed: it fetches and processes tiles that hold
-    // only older tokens, waits (grid_dep_wait) before it touches anything else, and only then lets
-    // the next layer start, which therefore never has to wait.
-    // dep_wait == 2: a launch that follows one too small to fill the GPU.  The host starts it this way
-    // only where the launch two before it has completed, so it works freely; but the NEXT launch shares
-    // its scratch half with the launch before this one, which may still be running: an otherwise idle
-    // thread of every CTA waits for that launch and only then lets the next one start.
+    // become free and uses the other copy of the scratch memory, so it touches nothing this one uses.
+    // A launch lets its successor start (launch_dependents) only once its own predecessor has completed:
+    // two launches that share a scratch copy are then never in flight together.
+    //   dep_wait == 0: an ordinary launch; its predecessor completed before it started.
+    //   dep_wait == 1: the step's first decode launch, which may run beside the step's append launch: it
+    //     fetches and processes tiles that hold only older tokens, waits (grid_dep_wait) before it touches
+    //     anything else, and only then lets the next layer start.
+    //   dep_wait == 2: any later launch of the step, which may run beside its predecessor: an otherwise
+    //     idle thread of every CTA waits for the predecessor and only then lets the next launch start.
     if (tid == 0 && !args.dep_wait) grid_dep_launch();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
@@ -1150,7 +1151,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             }
         } else if (lane == 1 && a.dep_wait == 2) {
             grid_dep_wait();    // the launch before this one has completed ...
-            grid_dep_launch();  // ... so the next one, which shares its scratch half, may start
+            grid_dep_launch();  // ... so the next one, which shares that launch's scratch copy, may start
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps

@@ -20,6 +20,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <new>
 #include <vector>
 
@@ -313,7 +314,9 @@ constexpr size_t kStaticScratchBytes = 4u << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_static_scratch_dev[kMaxDevices] = {};  // device address of the array, per device
+// device address of the array, per device; two host threads that make their first call on a device at
+// the same time both ask the runtime and store the same answer
+std::atomic<unsigned char*> g_static_scratch_dev[kMaxDevices];
 
 // Device address of g_static_scratch on `device`, which must be current.  In host code the array's
 // name is only a handle for the runtime, never a pointer a kernel may use: the address has to be
@@ -321,13 +324,15 @@ unsigned char* g_static_scratch_dev[kMaxDevices] = {};  // device address of the
 int static_scratch_address(int device, unsigned char** out)
 {
     if (device < 0 || device >= kMaxDevices) return RLKV_EINVAL;
-    if (!g_static_scratch_dev[device]) {
+    unsigned char* known = g_static_scratch_dev[device].load(std::memory_order_acquire);
+    if (!known) {
         void* p = nullptr;
         RLKV_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
         if (!p) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_static_scratch)");
-        g_static_scratch_dev[device] = static_cast<unsigned char*>(p);
+        known = static_cast<unsigned char*>(p);
+        g_static_scratch_dev[device].store(known, std::memory_order_release);
     }
-    *out = g_static_scratch_dev[device];
+    *out = known;
     return RLKV_OK;
 }
 
@@ -363,17 +368,11 @@ int do_decode_static_scratch(rlkv_cache* c, int layer, const void* q, void* out,
 // step_append: one launch appends the new token to every layer.  step_decode: the decode launches of
 // layers [l0, l1).  All inputs of the step are complete before its first launch starts, so the decode
 // launches may overlap one another: consecutive layers alternate between the two halves of the
-// scratch memory, and the first layer's launch waits on the device for the append launch before it
-// reads rows that launch writes.
-// Launch l and launch l-2 share a half of the scratch memory, so launch l must not start before
-// launch l-2 has completed.  An overlapped launch starts when every CTA of launch l-1 has started; if
-// launch l-1 puts exactly one CTA on every SM (and a CTA takes a whole SM: its registers see to that),
-// all of them having started means that no CTA of launch l-2 is left.  After a smaller launch l-1
-// the launch is still overlapped if launch l-2 is known to have completed by the time launch l-1 lets
-// launch l start (launch l-1 was an ordinary launch, or held launch l back itself); launch l then
-// holds launch l+1 back until launch l-1 has completed (dep_wait 2 in decode_kernel).  Otherwise, and
-// after anything but a kernel of this step in the stream (`fresh`), the launch is an ordinary one,
-// which waits for everything before it.
+// scratch memory, the first layer's launch waits on the device for the append launch before it reads
+// rows that launch writes, and every later launch lets its successor start only after its own
+// predecessor has completed (step_launch_mode in rlkv_host.cuh), so two launches that share a half are
+// never in flight together.  After anything but a kernel of this step in the stream (`fresh`) the
+// first launch is an ordinary one, which waits for everything before it.
 int step_append(rlkv_cache* c, const void* k, const void* v, cudaStream_t s)
 {
     AppendAllArgs aa;
@@ -400,33 +399,12 @@ int step_append(rlkv_cache* c, const void* k, const void* v, cudaStream_t s)
 int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStream_t s, bool fresh)
 {
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
-    // What the launch before this one in the stream was: an ordinary launch (it started after
-    // everything before it had completed: the append launch, or a decode launch after a stream wait),
-    // an overlapped launch that lets its successor start at once, or an overlapped launch that lets
-    // its successor start only after its own predecessor has completed (dep_wait 1 or 2).
-    enum { kOrdinary, kFree, kWaits } prev = kOrdinary;
-    bool prev_full = false;  // it put one CTA on every SM
     for (int l = l0; l < l1; ++l) {
-        int grid = 0, dep_wait = 0;
-        bool overlap;
-        if (l == l0) {
-            // right after the append launch an overlapped launch is fine: it waits on the device for it
-            overlap = !fresh;
-            dep_wait = overlap && l == 0 ? 1 : 0;
-        } else if (prev_full) {
-            overlap = true;  // all CTAs of the launch before have started: none of the one before that is left
-        } else if (prev != kFree) {
-            overlap = true;  // the launch two back had completed when the launch before let this one start
-            dep_wait = 2;    // and this one keeps the next launch back until the launch before has completed
-        } else {
-            overlap = false;
-        }
+        const StepLaunchMode m = step_launch_mode(l == l0, !fresh && l == 0);
         int rc = do_decode(c, l, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                           static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, overlap, dep_wait,
-                           &grid, nullptr, true);
+                           static_cast<uint8_t*>(out) + l * q_layer * (c->out_bf16 ? 2 : 4), s, l & 1, m.overlap, m.dep_wait,
+                           nullptr, nullptr, true);
         if (rc) return rc;
-        prev = !overlap ? kOrdinary : (dep_wait ? kWaits : kFree);
-        prev_full = (grid == c->sm_count && c->ctas_per_sm == 1);
     }
     return RLKV_OK;
 }
@@ -889,6 +867,18 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
             if (tile_map_out[4 * x + 3] < slot || tile_map_out[4 * x + 3] >= slot + count) return RLKV_EKERNEL;
             if (tile_map_out[4 * x + 3] >= sc.n_slots) return RLKV_EKERNEL;
         }
+    }
+    return RLKV_OK;
+}
+
+int rlkv_debug_step_plan(int n_launches, int follows_append, int* overlap_out, int* dep_wait_out, int* scratch_copy_out)
+{
+    if (n_launches < 1 || !overlap_out || !dep_wait_out || !scratch_copy_out) return RLKV_EINVAL;
+    for (int l = 0; l < n_launches; ++l) {
+        const StepLaunchMode m = step_launch_mode(l == 0, follows_append != 0);
+        overlap_out[l] = m.overlap ? 1 : 0;
+        dep_wait_out[l] = m.dep_wait;
+        scratch_copy_out[l] = l & 1;
     }
     return RLKV_OK;
 }

@@ -56,6 +56,35 @@ inline int max_stages(int head_dim, int group, int groups, int ctas_per_sm, int 
     return 0;
 }
 
+// How the decode launches of one step follow one another in the stream.  Consecutive launches use
+// different copies of the split-KV scratch (partial records, claim counter, and in the paged cache the
+// tickets), so launch l may run beside launch l-1; it shares its copy with launch l-2 and must not start
+// before that one has completed.  The device guarantees it: a launch is started in one of three ways,
+//   ordinary   (overlap 0, dep_wait 0): it starts when everything before it in the stream has completed,
+//              and lets its successor start at once;
+//   dep_wait 1 (the launch right after the step's append launch): it may start beside the append launch,
+//              waits for it before it touches what that launch writes, and only then lets its successor
+//              start;
+//   dep_wait 2 (every other launch): it may start beside its predecessor; an otherwise idle thread of
+//              each of its CTAs waits (griddepcontrol.wait) until the predecessor has completed and only
+//              then executes griddepcontrol.launch_dependents.
+// A launch with the programmatic-serialization attribute starts once every CTA of its predecessor has
+// executed launch_dependents or exited; in all three cases that happens only after the predecessor's own
+// predecessor has completed.  So at most two decode launches are ever in flight and launch l never runs
+// beside launch l-2, however the block scheduler places CTAs.
+// `first`: the first decode launch of this run of launches; `after_append`: it directly follows the
+// step's append launch in the stream (otherwise something else precedes it, e.g. a wait for a copy).
+struct StepLaunchMode {
+    bool overlap;
+    int dep_wait;
+};
+inline StepLaunchMode step_launch_mode(bool first, bool after_append)
+{
+    if (!first) return StepLaunchMode{true, 2};
+    if (after_append) return StepLaunchMode{true, 1};
+    return StepLaunchMode{false, 0};
+}
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;

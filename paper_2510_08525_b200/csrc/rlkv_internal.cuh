@@ -45,7 +45,7 @@ enum : int {
     kModePlain = 0,   // the lock-step cache: full and compressed heads, one length for the whole batch
     kModeMixed = 1,   // mixed attention (Eq. 1) over a lock-step cache whose heads are all full
     kModePaged = 2,   // the paged cache: one length per sequence, full heads in 64-token pages
-    kModePagedFp8 = 3 // the paged cache with the full heads' pages held as 8-bit E4M3 codes
+    kModePagedFp8 = 3 // the paged cache with every K/V row (pages and rings) held as 8-bit E4M3 codes
 };
 
 // One record of split-KV partial results: running max and sum (log2 domain) of the G query heads
@@ -228,10 +228,9 @@ struct DecodeArgs {
     int* tickets;               // one per unit of this layer, zero between launches
     unsigned int* claim_counter;  // items claimed beyond the first P, over all launches so far (never reset)
     unsigned int claim_base;      // its value when this launch starts: every launch adds exactly sched.n_items
-    int dep_wait;               // 1: the launch may start before the kernel that wrote this step's new rows has
-                                // completed: wait for it before touching what it writes (see launch_decode);
-                                // 2: the launch may start while the two launches before it still run: wait for
-                                // the one before it prior to any claim and any write (see decode_kernel)
+    int dep_wait;               // how the launch is ordered against its predecessor in the stream (see the
+                                // first lines of decode_kernel and step_launch_mode): 0 ordinary, 1 it may run
+                                // beside the step's append launch, 2 it may run beside the decode launch before it
     int* status;                // device error word
     unsigned long long* trace;  // debug: [grid][kTraceWords]
     int n_full, n_comp;         // heads of each class in this layer
@@ -371,10 +370,9 @@ __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.w
 // Launchers (defined in the .cu files).
 // `overlap` (launch_decode): launch with programmatic stream serialization, so that the kernel may
 // start while the kernel before it in the stream is still running.  Only for the decode launches of
-// one rlkv_step, whose inputs are complete before the step's first launch: consecutive layers use
-// different halves of the scratch memory and touch nothing of each other, and the first layer's
-// launch (dep_wait 1) waits on the device for the step's append launch before it reads new rows; a
-// launch after one too small to fill the GPU (dep_wait 2) keeps the next launch back instead.
+// one step, whose inputs are complete before the step's first launch: consecutive layers use
+// different copies of the scratch memory and touch nothing of each other; DecodeArgs::dep_wait says
+// what the kernel waits for on the device.
 cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream);
 
 // The appends of one token to every layer, in one launch (rlkv_step).
@@ -422,7 +420,7 @@ struct PagedAppendArgs {
     int n, t0, first_page;
     int n_layers;               // 1 unless the launch serves every layer
     const LayerDesc* layers;    // device, [n_layers]; unused when n_layers == 1
-    // 8-bit pages of the full heads (null: 16-bit rows): the pool, 1 / scale per head of the first layer
+    // 8-bit storage (null: 16-bit rows): the pool of pages and rings, 1 / scale per head of the first layer
     // served ([n_layers][kv_heads]), the layer's first page when n_layers == 1
     unsigned char* pool8;
     const float* k_inv;

@@ -34,10 +34,11 @@ using namespace rlkv;
 
 struct rlkv_paged {
     int layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, table_stride, sink, window;
+    int max_seq_len;              // most tokens a sequence may hold (the page table is laid out for a few more)
     int device, sm_count, stages, groups, item_tiles;
     int rows_comp, max_batch, max_items, max_grid;
     int out_bf16;
-    int fp8;                      // the full heads' pages hold E4M3 codes
+    int fp8;                      // K/V rows (pages and rings) are held as E4M3 codes
     std::vector<float> k_scale, v_scale;  // [layers*kv_heads]
     std::vector<long long> page0_8, ring0_8;  // first full-head page / first ring page of each layer in the 8-bit pool
     long long pages8;                      // pages of the 8-bit pool
@@ -252,7 +253,7 @@ static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads,
     rlkv_paged* p = new (std::nothrow) rlkv_paged();
     if (!p) return RLKV_ENOMEM;
     p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
-    p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window;
+    p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window; p->max_seq_len = max_seq_len;
     p->claims[0] = p->claims[1] = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
     p->fp8 = fp8;
     if (fp8) {
@@ -386,7 +387,7 @@ int rlkv_paged_append(rlkv_paged* p, int layer, const int* slots, int n, const v
     int need = 0;
     for (int i = 0; i < n; ++i) {
         const int t = len[slots[i]];
-        if (t / kTile >= p->table_stride) return RLKV_EFULL;
+        if (t >= p->max_seq_len) return RLKV_EFULL;
         if (p->table[(size_t)slots[i] * p->table_stride + t / kTile] < 0) ++need;
     }
     if (need > (int)p->free_pages.size()) return RLKV_EFULL;
@@ -421,7 +422,7 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
         return RLKV_EINVAL;
     int* len = len_of(p, layer);
     const int t0 = len[slot];
-    if (((long long)t0 + n_tokens + kTile - 1) / kTile > p->table_stride) return RLKV_EFULL;
+    if ((long long)t0 + n_tokens > p->max_seq_len) return RLKV_EFULL;
     const int first = t0 / kTile, last = (t0 + n_tokens - 1) / kTile;
     int* row = p->table.data() + (size_t)slot * p->table_stride;
     int need = 0;
@@ -579,7 +580,7 @@ int rlkv_paged_step(rlkv_paged* p, const int* slots, int n, const void* k, const
         const int t = len_of(p, 0)[slots[i]];
         for (int l = 1; l < p->layers; ++l)
             if (len_of(p, l)[slots[i]] != t) return RLKV_EINVAL;
-        if (t / kTile >= p->table_stride) return RLKV_EFULL;
+        if (t >= p->max_seq_len) return RLKV_EFULL;
         if (p->table[(size_t)slots[i] * p->table_stride + t / kTile] < 0) ++need;
     }
     if (need > (int)p->free_pages.size()) return RLKV_EFULL;
@@ -610,31 +611,14 @@ int rlkv_paged_step(rlkv_paged* p, const int* slots, int n, const void* k, const
     p->launches++;
     for (int l = 0; l < p->layers; ++l)
         for (int i = 0; i < n; ++i) len_of(p, l)[slots[i]] += 1;
-    // the layers' decode launches, overlapped as in rlkv_step: see step_decode in rlkv_api.cu for why
-    // each of the three cases is safe
+    // the layers' decode launches, overlapped as in rlkv_step (step_launch_mode in rlkv_host.cuh)
     const size_t q_layer = (size_t)n * p->q_heads * p->head_dim;
-    enum { kOrdinary, kFree, kWaits } prev = kOrdinary;
-    bool prev_full = false;
     for (int l = 0; l < p->layers; ++l) {
-        int grid = 0, dep_wait = 0;
-        bool overlap;
-        if (l == 0) {
-            overlap = true;  // waits on the device for the append launch
-            dep_wait = 1;
-        } else if (prev_full) {
-            overlap = true;
-        } else if (prev != kFree) {
-            overlap = true;
-            dep_wait = 2;
-        } else {
-            overlap = false;
-        }
+        const StepLaunchMode m = step_launch_mode(l == 0, true);
         rc = paged_decode(p, l, slots, n, static_cast<const __nv_bfloat16*>(q) + l * q_layer,
-                          static_cast<uint8_t*>(out) + l * q_layer * (p->out_bf16 ? 2 : 4), s, l & 1, overlap, dep_wait, true,
-                          &grid);
+                          static_cast<uint8_t*>(out) + l * q_layer * (p->out_bf16 ? 2 : 4), s, l & 1, m.overlap, m.dep_wait, true,
+                          nullptr);
         if (rc) return rc;
-        prev = !overlap ? kOrdinary : (dep_wait ? kWaits : kFree);
-        prev_full = grid == p->sm_count;
     }
     return RLKV_OK;
 }

@@ -117,7 +117,7 @@ class PagedCache:
             if k_scale is None:
                 self.handle = rl.rlkv_paged_create(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
                                                    self.mask, sink, window)
-            else:      # the full heads' pages as E4M3 codes
+            else:      # every K/V row (pages and rings) as E4M3 codes
                 self.handle = rl.rlkv_paged_create_fp8(layers, kv_heads, q_heads, head_dim, max_seqs, n_pages, max_seq_len,
                                                        self.mask, sink, window, k_scale, v_scale)
 

@@ -33,7 +33,7 @@ class Seq:
         self.slot = cache.open_seq()
         self.oracle = Oracle(cache.layers, cache.kv_heads, cache.q_heads, cache.head_dim, 1, max_len,
                              cache.mask.reshape(-1), cache.sink, cache.window, threads=4)
-        if scales is not None:                                # the full heads in 8-bit storage
+        if scales is not None:                                # all heads in 8-bit storage
             self.oracle.set_fp8(*scales)
         self.n = 0
 
@@ -202,6 +202,44 @@ def test_paged_argument_checks(rl, hz, cuda_device):
     assert cache.length(0, s0) == 128
     torch.cuda.synchronize()
     assert (out == 3.0).all()
+    assert cache.status() == 0
+    cache.close()
+
+
+def test_max_seq_len_is_the_limit_even_with_pages_to_spare(rl, hz, cuda_device):
+    """max_seq_len = 100 is no multiple of the page (64) nor of the table's padding (256 tokens), and
+    the free list holds far more pages than one sequence can use: append, prefill and step must all
+    refuse token 100 with RLKV_EFULL and leave lengths, page table and free list as they were."""
+    Hkv, Hq, D = 2, 4, 64
+    cache = hz.PagedCache(2, Hkv, Hq, D, 2, 16, 100, [1, 0, 0, 1], 4, 12, device=cuda_device)
+    s0, s1 = cache.open_seq(), cache.open_seq()
+    k = rand_bf16((100, Hkv, D), 5).to(cuda_device)
+    with pytest.raises(rl.RlkvError) as e:                   # 101 tokens at once
+        rl.rlkv_paged_prefill(cache.handle, 0, s0, torch.cat([k, k[:1]]), torch.cat([k, k[:1]]), 101)
+    assert e.value.code == rl.RLKV_EFULL and cache.length(0, s0) == 0 and cache.pages() == (16, 16)
+    for layer in range(2):
+        cache.prefill(layer, s0, k[:99], k[:99])
+        cache.prefill(layer, s1, k[:40], k[:40])
+    assert cache.pages() == (16 - 2 - 1, 16)
+    with pytest.raises(rl.RlkvError) as e:                   # 99 + 2 > 100
+        rl.rlkv_paged_prefill(cache.handle, 0, s0, k[:2], k[:2], 2)
+    assert e.value.code == rl.RLKV_EFULL and cache.length(0, s0) == 99
+    q = rand_bf16((2, 2, Hq, D), 6).to(cuda_device)
+    out = torch.empty((2, 2, Hq, D), dtype=torch.float32, device=cuda_device)
+    kv = k[:4].reshape(2, 2, Hkv, D).contiguous()
+    rl.rlkv_paged_step(cache.handle, [s0, s1], kv, kv, q, out)   # token 99 of s0: the last one allowed
+    assert [cache.length(l, s0) for l in range(2)] == [100, 100] and cache.length(0, s1) == 41
+    free = cache.pages()
+    with pytest.raises(rl.RlkvError) as e:
+        rl.rlkv_paged_step(cache.handle, [s0, s1], kv, kv, q, out)
+    assert e.value.code == rl.RLKV_EFULL
+    with pytest.raises(rl.RlkvError) as e:                   # nothing appended for s1 either
+        rl.rlkv_paged_append(cache.handle, 1, [s1, s0], kv[0], kv[0])
+    assert e.value.code == rl.RLKV_EFULL
+    assert [cache.length(l, s) for l in range(2) for s in (s0, s1)] == [100, 41, 100, 41]
+    assert cache.pages() == free
+    rows = cache.export_head(0, s0, 0)                       # a buffer of max_seq_len rows is enough
+    assert rows[0].shape[0] == 100
     assert cache.status() == 0
     cache.close()
 

@@ -112,3 +112,34 @@ def test_paged_launch_tickets_match_the_segments_that_exist():
         assert (delivered[~direct] == expected[~direct]).all() and (delivered[~direct] >= 1).all()
         cases += len(delivered)
     assert cases > 10000
+
+
+@pytest.mark.parametrize("n,follows_append", [(1, True), (2, True), (7, True), (32, True), (5, False), (128, False)])
+def test_two_launches_sharing_a_scratch_copy_are_never_in_flight_together(rl, n, follows_append):
+    """The decode launches of a step alternate between two copies of the split-KV scratch.  Replay
+    the launch rules with the slowest possible completions: a launch starts when it is allowed to
+    and completes only when something waits for it.  Launch l must never start before launch l - 2
+    (the other user of its scratch copy) has completed."""
+    overlap, dep_wait, copy = rl.rlkv_debug_step_plan(n, follows_append)
+    assert list(copy) == [l & 1 for l in range(n)]
+    assert dep_wait[0] == (1 if follows_append else 0) and overlap[0] == (1 if follows_append else 0)
+    # earliest moment launch l can start, in terms of which earlier launches must have COMPLETED by then
+    must_be_complete = []
+    for l in range(n):
+        if not overlap[l]:
+            done = set(range(l))                     # an ordinary launch waits for everything before it
+        elif l == 0:
+            done = set()
+        else:
+            # it starts once launch l - 1 has executed launch_dependents: at its own start if that
+            # launch waits for nothing (then it was an ordinary launch, which implies its predecessors
+            # were complete), else after the launch before it has completed
+            prev_done = must_be_complete[l - 1]
+            done = set(prev_done)
+            if dep_wait[l - 1] == 0:
+                assert not overlap[l - 1], "a launch that triggers at once must itself be an ordinary launch"
+            elif dep_wait[l - 1] == 2:
+                done |= set(range(l - 1))            # launch l - 2 complete, and by induction all before it
+        must_be_complete.append(done)
+        if l >= 2:
+            assert l - 2 in done, f"launch {l} may start while launch {l - 2} still uses scratch copy {copy[l]}"
