@@ -327,6 +327,14 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
                         int item_tiles, int* n_items_out, int* n_slots_out, int* starts_out,
                         int* tile_map_out, int cap);
 
+/* Measurement aid (synchronous; no cache involved): reads `bytes` of device memory at device_buf
+ * (16-byte aligned, at least 32 KiB; contents irrelevant) `launches` times with the mechanism the
+ * decode kernel's producer uses -- bulk asynchronous copies into a ring of shared-memory stages, one
+ * persistent CTA per SM -- and nobody consuming the data.  *ms_out = mean time of one pass in
+ * milliseconds (CUDA events, after one untimed pass): bytes / that is the read-only bandwidth the
+ * decode kernel could at best reach on this GPU.  RLKV_EKERNEL if a wait inside the kernel ran out. */
+int rlkv_debug_read_bandwidth(const void* device_buf, size_t bytes, int launches, float* ms_out);
+
 /* How rlkv_step and rlkv_paged_step order the decode launches of one step, host arithmetic only (no
  * GPU).  For launch l of n_launches in a row (follows_append != 0: the first one directly follows the
  * step's append launch in the stream): overlap_out[l] = 1 if it is launched so that it may start

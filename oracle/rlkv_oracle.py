@@ -22,13 +22,16 @@ _LIBS = {"f32": os.path.join(_HERE, "librlkv_oracle_f32.so"),
 _loaded: dict = {}
 
 
+CC = "gcc"
+CFLAGS = ["-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-fno-fast-math", "-ffp-contract=off"]
+
+
 def build(force: bool = False) -> None:
     """Compile both builds of the oracle with gcc (plain C, -O2, OpenMP over (b, q head))."""
     for acc, path in _LIBS.items():
         if not force and os.path.exists(path) and os.path.getmtime(path) >= os.path.getmtime(_SRC):
             continue
-        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp",
-               "-fno-fast-math", "-ffp-contract=off"]
+        cmd = [CC] + CFLAGS
         if acc == "f64":
             cmd.append("-DRLKV_ORACLE_ACC=double")
         cmd += [_SRC, "-o", path, "-lm"]

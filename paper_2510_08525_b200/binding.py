@@ -45,6 +45,7 @@ SIGNATURES = {
     "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
     "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
     "rlkv_debug_step_plan": (_ci, [_ci, _ci, _vp, _vp, _vp]),
+    "rlkv_debug_read_bandwidth": (_ci, [_vp, _sz, _ci, ctypes.POINTER(ctypes.c_float)]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
     "rlkv_paged_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
     "rlkv_paged_create": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _sz]),
@@ -259,6 +260,13 @@ def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, it
     _check(lib.rlkv_debug_schedule(*args, ctypes.byref(n), ctypes.byref(slots), starts.ctypes.data, _ptr(tmap),
                                    max(starts.size, total)))
     return (starts, int(slots.value), tmap) if tile_map else (starts, int(slots.value))
+
+
+def rlkv_debug_read_bandwidth(buf, nbytes, launches=4) -> float:
+    """Mean milliseconds of one read-only pass over nbytes of device memory at buf."""
+    ms = ctypes.c_float(0)
+    _check(lib.rlkv_debug_read_bandwidth(_ptr(buf), int(nbytes), int(launches), ctypes.byref(ms)))
+    return float(ms.value)
 
 
 def rlkv_debug_step_plan(n_launches, follows_append=True):

@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librlkv.so")
-SOURCES = ["rlkv_api.cu", "rlkv_paged.cu", "append_kernel.cu", "decode_kernel.cu"]
+SOURCES = ["rlkv_api.cu", "rlkv_paged.cu", "append_kernel.cu", "decode_kernel.cu", "probe_kernel.cu"]
 HEADERS = ["rlkv_internal.cuh", "rlkv_host.cuh", os.path.join("..", "..", "include", "rlkv.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]

@@ -104,6 +104,15 @@ def step_inputs(w: synth.Workload, t: int, device):
     return k.contiguous(), v.contiguous(), q.contiguous()
 
 
+def step_inputs_block(w: synth.Workload, t0: int, t1: int, device):
+    """The inputs of the decode steps that append tokens t0 .. t1-1, generated in one go:
+    k, v [t1-t0][layers][B][Hkv][D] and q [t1-t0][layers][B][Hq][D]; entry i equals step_inputs(w, t0 + i)."""
+    def one(stream_id, heads):
+        return torch.stack([synth.rows(w.seed, stream_id, l, t0, t1, w.batch, heads, w.head_dim, device)
+                            for l in range(w.layers)], dim=1).contiguous()
+    return one(synth.STREAM_K, w.kv_heads), one(synth.STREAM_V, w.kv_heads), one(synth.STREAM_Q, w.q_heads)
+
+
 class PagedCache:
     """Owns an rlkv_paged handle (request slots with their own lengths, paged full heads)."""
 

@@ -77,46 +77,127 @@ def test_full_size_sampled_units(cuda_device, name):
     torch.cuda.empty_cache()
 
 
+def check_unit(cache, w, mask, layer, b, h, n, q_rows, got_rows):
+    """One sampled unit against an oracle of its own: the oracle regenerates the unit's n-token history
+    from the addressable generator; exported rows bit for bit, the G output rows within the bounds."""
+    o = unit_oracle(w, mask, layer, b, h, n)
+    for got, ref in zip(cache.export_head(layer, b, h), o.export_head(0, 0, 0)):
+        np.testing.assert_array_equal(got[:len(ref)] if got.ndim == 1 else got[:ref.shape[0]], ref)
+    want = o.decode(0, q_rows)[0]
+    err = np.abs(got_rows - want)
+    rms = np.sqrt((want.astype(np.float64) ** 2).mean(axis=-1, keepdims=True))
+    assert err.max() <= 1e-2 and err.mean() <= 1e-3, (layer, b, h, n, float(err.max()), float(err.mean()))
+    assert (err <= 2e-2 * rms + 1e-6).all(), (layer, b, h, n, float((err / rms).max()))
+
+
 def test_full_size_decode_loop_sampled_units(cuda_device):
-    """The long chain-of-thought loop at its full shape (32 layers, batch 8, 40 % of the heads
-    compressed, sink 16 + window 240, room for 32768 tokens): a 4096-token prompt, then 300 whole
-    steps through rlkv_step, so that every ring has wrapped.  Sampled units are checked after the last
-    step: exported rows bit for bit, output rows within the stated bounds."""
+    """The long chain-of-thought loop exactly as the benchmark runs it (32 layers, batch 8, 40 % of the
+    heads compressed, sink 16 + window 240): a 4096-token prompt, then every one of the 28672 steps
+    through rlkv_step with fresh seeded inputs, to n = 32768; the rings wrap about 136 times.  72
+    sampled (step, layer, batch row, KV head) units -- at steps spread over the loop, the last one
+    included -- are checked when their step has run: the unit's exported rows bit for bit against an
+    oracle that regenerates its history, its output rows within the stated bounds."""
     from paper_2510_08525_b200 import binding as rl
     from paper_2510_08525_b200 import harness
     w = synth.WORKLOADS["cot"]
     mask = synth.workload_mask(w)
-    max_len, steps = 32768, 300
+    steps = 28672
+    n_end = w.context + steps
     free, _ = torch.cuda.mem_get_info()
-    need = rl.rlkv_cache_size(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, max_len, mask, w.sink, w.window)
-    if free < need + (4 << 30):
+    need = rl.rlkv_cache_size(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, n_end, mask, w.sink, w.window)
+    if free < need + (6 << 30):
         pytest.skip("not enough free device memory for the full-size cache")
-    cache = harness.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, max_len, mask, w.sink, w.window,
+    cache = harness.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, n_end, mask, w.sink, w.window,
                           device=cuda_device)
     harness.fill_cache(cache, w, w.context)
     out = torch.empty((w.layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=cuda_device)
-    for t in range(w.context, w.context + steps):
-        k, v, q = harness.step_inputs(w, t, cuda_device)
-        rl.rlkv_step(cache.handle, k, v, q, out)
-    torch.cuda.synchronize()
-    assert cache.status() == 0
-    n = w.context + steps
-    assert all(cache.length(l) == n for l in range(w.layers))
-    res, q = out.cpu().numpy(), q.cpu()
-    assert np.isfinite(res).all()
     rng = np.random.default_rng(99)
     comp, full = np.flatnonzero(mask == 0), np.flatnonzero(mask == 1)
-    picks = list(rng.choice(full, 4, replace=False)) + list(rng.choice(comp, 4, replace=False))
+    # sampled steps (token index appended): the first, the ones that fill and first wrap the ring of a
+    # prompt that long, a spread over the loop, and the last 8 (steady state at n = 32768)
+    sample_steps = sorted(set([w.context, w.context + 1, w.context + w.window - 1, w.context + w.window]
+                              + [int(x) for x in rng.integers(w.context, n_end - 8, size=28)]
+                              + list(range(n_end - 4, n_end))))
+    samples = {}
+    for t in sample_steps:
+        picks = [rng.choice(full), rng.choice(comp)]
+        samples[t] = [(int(f) // w.kv_heads, int(rng.integers(w.batch)), int(f) % w.kv_heads) for f in picks]
+    assert sum(len(v) for v in samples.values()) >= 64
+    G, checked = w.group, 0
+    t = w.context
+    while t < n_end:
+        t1 = min(n_end, t + 256)
+        k, v, q = harness.step_inputs_block(w, t, t1, cuda_device)
+        for i in range(t1 - t):
+            rl.rlkv_step(cache.handle, k[i], v[i], q[i], out)
+            if t + i in samples:
+                torch.cuda.synchronize()
+                res, qc = out.cpu().numpy(), q[i].cpu()
+                for layer, b, h in samples[t + i]:
+                    check_unit(cache, w, mask, layer, b, h, t + i + 1, qc[layer, b, h * G:(h + 1) * G].contiguous(),
+                               res[layer, b, h * G:(h + 1) * G])
+                    checked += 1
+        torch.cuda.synchronize()
+        t = t1
+    assert checked >= 64
+    assert cache.status() == 0
+    assert all(cache.length(l) == n_end for l in range(w.layers))
+    assert np.isfinite(out.cpu().numpy()).all()
+    with pytest.raises(rl.RlkvError) as e:                  # the cache is exactly full
+        rl.rlkv_step(cache.handle, k[0], v[0], q[0], out)
+    assert e.value.code == rl.RLKV_EFULL
+    cache.close()
+    torch.cuda.empty_cache()
+
+
+# The corners of the compression x context x batch sweep the benchmark times: a few layers of each
+# (the mask is drawn for all 32 layers, the first `layers` are held, as the sweep does).
+CORNERS = [
+    # context, batch, fraction compressed, layers held
+    (65536, 8, 0.0, 3),
+    (65536, 8, 0.8, 6),
+    (32768, 32, 0.6, 3),
+    (8192, 64, 0.2, 3),
+    (65536, 1, 0.4, 8),
+    (2048, 64, 0.8, 8),
+]
+
+
+@pytest.mark.parametrize("context,batch,frac,layers", CORNERS)
+def test_sweep_corners_sampled_units(cuda_device, context, batch, frac, layers):
+    from paper_2510_08525_b200 import binding as rl
+    from paper_2510_08525_b200 import harness
+    w32 = synth.WORKLOADS["llama8b"].with_(context=context, batch=batch, frac_compressed=frac)
+    w = w32.with_(layers=layers)
+    mask = synth.workload_mask(w32)[:layers * w.kv_heads]
+    free, _ = torch.cuda.mem_get_info()
+    need = rl.rlkv_cache_size(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, w.context + 8, mask, w.sink, w.window)
+    if free < need + (6 << 30):
+        pytest.skip("not enough free device memory for this corner")
+    cache = harness.Cache(w.layers, w.kv_heads, w.q_heads, w.head_dim, w.batch, w.context + 8, mask, w.sink, w.window,
+                          device=cuda_device)
+    harness.fill_cache(cache, w, w.context)
+    out = torch.empty((w.layers, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=cuda_device)
+    n = w.context
+    for step in range(2):                                   # two steps: n = context + 1 and context + 2
+        k, v, q = harness.step_inputs(w, n, cuda_device)
+        rl.rlkv_step(cache.handle, k, v, q, out)
+        n += 1
+    torch.cuda.synchronize()
+    assert cache.status() == 0
+    res, qc = out.cpu().numpy(), q.cpu()
+    assert np.isfinite(res).all()
+    total = sum(cache.step_bytes(l) for l in range(w.layers))
+    n_full = int(mask.sum())
+    assert total == w.batch * (n_full * n + (mask.size - n_full) * (w.sink + w.window)) * 4 * w.head_dim
+    rng = np.random.default_rng(context + batch)
+    units = {(0, 0, 0), (w.layers - 1, w.batch - 1, w.kv_heads - 1)}
+    for cls in (np.flatnonzero(mask == 1), np.flatnonzero(mask == 0)):
+        for flat in rng.choice(cls, min(3, len(cls)), replace=False) if len(cls) else []:
+            units.add((int(flat) // w.kv_heads, int(rng.integers(w.batch)), int(flat) % w.kv_heads))
     G = w.group
-    for flat in picks:
-        layer, h, b = int(flat) // w.kv_heads, int(flat) % w.kv_heads, int(rng.integers(w.batch))
-        o = unit_oracle(w, mask, layer, b, h, n)
-        for got, ref in zip(cache.export_head(layer, b, h), o.export_head(0, 0, 0)):
-            np.testing.assert_array_equal(got[:len(ref)] if got.ndim == 1 else got[:ref.shape[0]], ref)
-        want = o.decode(0, q[layer, b, h * G:(h + 1) * G].contiguous())[0]
-        err = np.abs(res[layer, b, h * G:(h + 1) * G] - want)
-        rms = np.sqrt((want.astype(np.float64) ** 2).mean(axis=-1, keepdims=True))
-        assert err.max() <= 1e-2 and err.mean() <= 1e-3
-        assert (err <= 2e-2 * rms + 1e-6).all(), (layer, b, h, float((err / rms).max()))
+    for layer, b, h in sorted(units):
+        check_unit(cache, w, mask, layer, b, h, n, qc[layer, b, h * G:(h + 1) * G].contiguous(),
+                   res[layer, b, h * G:(h + 1) * G])
     cache.close()
     torch.cuda.empty_cache()

@@ -219,6 +219,24 @@ def test_compressed_heads_stay_inside_their_budget(rl, hz, cuda_device):
     with pytest.raises(rl.RlkvError) as e:
         cache.append(1, K[0].to(cuda_device), V[0].to(cuda_device))
     assert e.value.code == rl.RLKV_EFULL      # uniform rule, even for an all-compressed layer
+    # The pool starts the buffer: per layer the full heads' region [batch][full head][K|V][rows_full][D],
+    # then the compressed heads' [batch][compressed head][K|V][rows_comp][D], rows rounded up to the
+    # 64-row tile.  Every row past a head's budget (rows 400.. of a full head, rows 32.. of a ring) must
+    # still hold the zeros it was created with: a write that strays out of a ring lands there first.
+    rows_full, rows_comp, cap = 448, 64, S + W
+    pool = inner.view(torch.bfloat16)
+    row = 0
+    heads_seen = 0
+    for l in range(layers):
+        n_full = sum(mask[l * Hkv:(l + 1) * Hkv])
+        for rows, count, used in ((rows_full, B * n_full, max_len), (rows_comp, B * (Hkv - n_full), cap)):
+            for _ in range(2 * count):                       # K block and V block of every head
+                block = pool[row * D:(row + rows) * D].view(rows, D)
+                assert block[:used].any()                    # the head's own rows were written ...
+                assert not block[used:].any()                # ... and nothing beyond them
+                row += rows
+                heads_seen += 1
+    assert heads_seen == 2 * B * layers * Hkv
 
 
 # ------------------------------------------------------------------------------------------ errors
@@ -387,6 +405,39 @@ def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
     assert e.value.code == rl.RLKV_EFULL
 
 
+def test_reduced_loop_of_4000_steps_checked_at_every_step(rl, hz, cuda_device):
+    """The long decode loop at a reduced shape (2 layers, batch 2, 8/2 heads, prompt 300, sink 16 +
+    window 240, 4000 steps: the rings wrap 16 times).  At EVERY step the outputs of both layers are
+    compared with the oracle and the rings of the compressed heads bit for bit; the whole cache state
+    every 250 steps and at the end."""
+    layers, Hkv, Hq, D, B, S, W, prompt, steps = 2, 2, 8, 128, 2, 16, 240, 300, 4000
+    mask = [1, 0, 0, 1]
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, cuda_device)
+    for l in range(layers):
+        feed(cache, oracle, l, rand_bf16((prompt, B, Hkv, D), 250 + l), rand_bf16((prompt, B, Hkv, D), 260 + l), True)
+    out = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+    block = 500
+    for t0 in range(0, steps, block):
+        K = rand_bf16((block, layers, B, Hkv, D), 270 + t0)
+        V = rand_bf16((block, layers, B, Hkv, D), 271 + t0)
+        Q = rand_bf16((block, layers, B, Hq, D), 272 + t0)
+        Kd, Vd, Qd = K.to(cuda_device), V.to(cuda_device), Q.to(cuda_device)
+        for i in range(block):
+            rl.rlkv_step(cache.handle, Kd[i], Vd[i], Qd[i], out)
+            got = out.cpu().numpy()
+            for l in range(layers):
+                assert oracle.append(l, K[i, l], V[i, l]) == 0
+                check_out(got[l], oracle.decode(l, Q[i, l]))
+                h = mask[l * Hkv:(l + 1) * Hkv].index(0)     # the layer's compressed head
+                for b in range(B):
+                    for g_, o_ in zip(cache.export_head(l, b, h), oracle.export_head(l, b, h)):
+                        np.testing.assert_array_equal(g_, o_)
+            if (t0 + i) % 250 == 249:
+                check_state(cache, oracle)
+    check_state(cache, oracle)
+    assert cache.length(0) == prompt + steps and cache.status() == 0
+
+
 def test_step_mixes_tiny_and_gpu_filling_launches(rl, hz, cuda_device):
     """Seven layers whose launches alternate between a few work items and more than one per SM (all
     heads compressed, one full head, all full): inside rlkv_step a launch after a small one starts
@@ -465,13 +516,33 @@ def test_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
             c.prefill(l, rand_bf16((n, B, Hkv, D), 10 + l, cuda_device), rand_bf16((n, B, Hkv, D), 50 + l, cuda_device))
         caches.append(c)
     f32, b16 = caches
+    oracle = Oracle(layers, Hkv, Hq, D, B, n + 8, mask, S, W, threads=8)
+    for l in range(layers):
+        Kc, Vc = rand_bf16((n, B, Hkv, D), 10 + l), rand_bf16((n, B, Hkv, D), 50 + l)
+        for t in range(n):
+            assert oracle.append(l, Kc[t], Vc[t]) == 0
     rl.rlkv_set_output_bf16(b16.handle, 1)
     q = rand_bf16((layers, B, Hq, D), 90, cuda_device)
+
+    def check_bf16(got, want):
+        """bf16 results against the oracle's fp32 ones: the usual bounds, widened by the half ulp that
+        the final rounding to bf16 may add (2^-9 of the value)."""
+        got, want = got.float().cpu().numpy().astype(np.float64), np.asarray(want, np.float64)
+        err = np.abs(got - want)
+        half_ulp = np.abs(want) * 2.0 ** -8
+        rms = np.sqrt((want ** 2).mean(axis=-1, keepdims=True))
+        assert np.isfinite(got).all()
+        assert (err <= MAX_ABS + half_ulp).all() and err.mean() <= MEAN_ABS + half_ulp.mean()
+        assert (err <= REL_RMS * rms + half_ulp + 1e-6).all()
+
     # per-layer call
     want = f32.decode(0, q[0])
     got = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=cuda_device)
     rl.rlkv_decode_attention(b16.handle, 0, q[0], got)
     assert torch.equal(got, want.to(torch.bfloat16))
+    ref0 = oracle.decode(0, q[0].cpu())
+    check_out(want.cpu().numpy(), ref0)
+    check_bf16(got, ref0)
     # whole step, device buffers
     k, v = rand_bf16((layers, B, Hkv, D), 91, cuda_device), rand_bf16((layers, B, Hkv, D), 92, cuda_device)
     want = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
@@ -479,6 +550,11 @@ def test_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
     rl.rlkv_step(f32.handle, k, v, q, want)
     rl.rlkv_step(b16.handle, k, v, q, got)
     assert torch.equal(got, want.to(torch.bfloat16))
+    for l in range(layers):                                  # both against the oracle, every layer
+        assert oracle.append(l, k[l].cpu(), v[l].cpu()) == 0
+        ref = oracle.decode(l, q[l].cpu())
+        check_out(want[l].cpu().numpy(), ref)
+        check_bf16(got[l], ref)
     # whole step, host buffers
     kh, vh, qh = (x.cpu().pin_memory() for x in (k, v, q))
     want_h = torch.empty((layers, B, Hq, D), dtype=torch.float32).pin_memory()
