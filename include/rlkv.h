@@ -154,13 +154,21 @@ int rlkv_set_output_bf16(rlkv_cache* cache, int on);
 /* One whole decode step: for every layer, append then attend.  Device buffers:
  * k, v bf16 [layers][batch][kv_heads][head_dim]; q bf16 [layers][batch][q_heads][head_dim];
  * out fp32 [layers][batch][q_heads][head_dim].  The results are those of the per-layer calls in
- * order (up to floating-point summation order: the step cuts the work into larger items).  Because all inputs are there before the first launch, the step is issued as one append
- * launch for all layers followed by the layers' attention launches, which overlap on the device
- * (programmatic dependent launch): every buffer must be complete when the call is made and stay
- * untouched until the work on `stream` has finished.  RLKV_EFULL (nothing done) if any layer is at
- * max_len. */
+ * order (up to floating-point summation order: the step cuts the work differently).  Because all
+ * inputs are there before the first launch, the step is issued as one append launch for all layers
+ * and ONE attention launch over the K/V rows of every layer (the units of all layers form one flat
+ * tile space, so a step of many small layers costs what its bytes cost, not a launch per layer);
+ * where the layers hold different numbers of tokens, or the shape has more than 128 layers or 4096
+ * (layer, KV head) pairs, it is one attention launch per layer, overlapped on the device (programmatic
+ * dependent launch).  Every buffer must be complete when the call is made and stay untouched until
+ * the work on `stream` has finished.  RLKV_EFULL (nothing done) if any layer is at max_len. */
 int rlkv_step(rlkv_cache* cache, const void* k, const void* v, const void* q, void* out,
               void* stream);
+/* How rlkv_step issues the attention of a step from now on: 0 (the default) lets the library choose as
+ * described above, 1 forces one launch per layer, 2 one launch for the whole step (RLKV_EINVAL if
+ * the shape does not allow it; a step whose layers differ in length still falls back to one launch
+ * per layer).  Results do not depend on it beyond floating-point summation order. */
+int rlkv_set_step_mode(rlkv_cache* cache, int mode);
 
 /* The same step with HOST buffers of the same shapes (pinned memory makes the copies
  * asynchronous).  Inputs are copied host->device and results device->host inside the call, on two
@@ -318,14 +326,16 @@ int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_ho
  * space (in bands: the first half of every full unit, then half of the rest, ... then the rest and
  * the compressed units) and cut for `ctas` CTAs into *n_items_out contiguous work items whose sizes
  * shrink geometrically down to item_tiles; *n_slots_out is the number of partial-result records a
- * launch of this shape may write.  Optional outputs (host; `cap` = ints available in starts_out
+ * launch of this shape may write.  whole_step != 0: the schedule rlkv_step uses for one launch over
+ * all layers instead (most full units whole, unit after unit, in one equal item per CTA; the rest and
+ * the compressed units unit after unit in items of item_tiles tiles, fewer where the step is small).  Optional outputs (host; `cap` = ints available in starts_out
  * and 4-int records available in tile_map_out): starts_out[k] = first flat tile of item k, then
  * the total; tile_map_out[4x..4x+3] = unit, tile inside the unit, consecutive tiles of the unit
  * from x on, partial record of the segment holding flat tile x.  RLKV_EKERNEL if the schedule's
  * own maps disagree with each other (a self-check; never expected). */
 int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas,
-                        int item_tiles, int* n_items_out, int* n_slots_out, int* starts_out,
-                        int* tile_map_out, int cap);
+                        int item_tiles, int whole_step, int* n_items_out, int* n_slots_out,
+                        int* starts_out, int* tile_map_out, int cap);
 
 /* Measurement aid (synchronous; no cache involved): reads `bytes` of device memory at device_buf
  * (16-byte aligned, at least 32 KiB; contents irrelevant) `launches` times with the mechanism the

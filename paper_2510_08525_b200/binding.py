@@ -43,7 +43,8 @@ SIGNATURES = {
     "rlkv_launch_count": (_ci, [_vp, ctypes.POINTER(ctypes.c_uint64)]),
     "rlkv_set_decode_config": (_ci, [_vp, _ci, _ci, _ci, _ci]),
     "rlkv_debug_trace": (_ci, [_vp, _ci, _vp, ctypes.POINTER(_ci)]),
-    "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
+    "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
+    "rlkv_set_step_mode": (_ci, [_vp, _ci]),
     "rlkv_debug_step_plan": (_ci, [_ci, _ci, _vp, _vp, _vp]),
     "rlkv_debug_read_bandwidth": (_ci, [_vp, _sz, _ci, ctypes.POINTER(ctypes.c_float)]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
@@ -248,11 +249,15 @@ def rlkv_debug_trace(cache, enable, read=False):
     return words
 
 
-def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, tile_map=False):
+def rlkv_set_step_mode(cache, mode) -> None:
+    _check(lib.rlkv_set_step_mode(cache, int(mode)))
+
+
+def rlkv_debug_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, tile_map=False, whole_step=False):
     """Returns (starts int32[n_items + 1], n_slots) and, with tile_map=True, also int32[T][4]:
     unit, tile in unit, run, partial record of every flat tile."""
     n, slots = _ci(0), _ci(0)
-    args = (full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+    args = (full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, int(whole_step))
     _check(lib.rlkv_debug_schedule(*args, ctypes.byref(n), ctypes.byref(slots), None, None, 0))
     total = full_units * tiles_full + comp_units * tiles_comp
     starts = np.empty(n.value + 1, dtype=np.int32)

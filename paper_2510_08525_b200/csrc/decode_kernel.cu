@@ -22,10 +22,11 @@
 // merges of split units run on all warps once the CTA's stream has ended.
 // The decode launches of one step overlap on the device (programmatic dependent launch): see the
 // kernel's first lines and launch_decode.
-// The kernel is compiled in three modes: the lock-step cache (above), mixed attention with gating
+// The kernel is compiled in several modes: the lock-step cache (above), mixed attention with gating
 // adapters (paper, Eq. 1: a second class of "local" units over the sink and window rows, both
-// classes adding their weighted result), and the paged cache (one length per sequence, full-head
-// rows looked up in a page table); see the notes above decode_kernel.
+// classes adding their weighted result), the paged cache (one length per sequence, full-head
+// rows looked up in a page table; also with 8-bit pages), and the whole decode step in one launch
+// (the units of every layer in one flat tile space); see the notes above decode_kernel.
 #include <cuda_fp16.h>
 
 #include "rlkv_internal.cuh"
@@ -272,12 +273,15 @@ struct Smem {
     }
     // paged cache only: the page-table entries of the segment being streamed, the PagedArgs
     static constexpr int kPagedBytes = (kMaxSeqPages + 4) * 4 + (int)((sizeof(PagedArgs) + 15) / 16 * 16);
+    // whole-step launches only: the StepArgs and the KV head of every slot of every layer
+    static constexpr int kStepBytes = (int)((sizeof(StepArgs) + 15) / 16 * 16) + kMaxStepHeads;
     __host__ __device__ static constexpr size_t bytes(int stages, int group, int mode = kModePlain)
     {
         return (size_t)stages * stage_bytes(group, mode) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
-               (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0);
+               (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0) +
+               (mode == kModeStep ? kStepBytes : 0);
     }
 };
 
@@ -400,6 +404,10 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
 // LOCAL unit over the same head's sink and window rows; its tiles start at whatever row the window
 // starts (a TMA box may start at any row) and are masked past their valid rows.
 //
+// kModeStep: a whole decode step.  The full units of all layers are one list and so are the compressed
+// units (every layer holds the same number of tokens); a unit's layer, rows, query and output rows are
+// looked up in the StepArgs.  Everything else is the lock-step kernel.
+//
 // kModePaged: the paged cache.  Units keep the uniform layout (every full unit is given the tiles of
 // the longest sequence); producer and consumers both leave out a unit's tiles past its own length and
 // realign the slot counter at every segment, and the producer looks a full unit's rows up in the
@@ -417,6 +425,10 @@ template <>
 struct ExtraArgs<kModePagedFp8> {
     typedef PagedFp8Args type;  // starts with a PagedArgs
 };
+template <>
+struct ExtraArgs<kModeStep> {
+    typedef StepArgs type;
+};
 
 template <int D, int NG, int MODE>
 __global__ void __launch_bounds__(Smem<D, NG>::kThreads, 1)
@@ -426,6 +438,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     constexpr bool MIXED = MODE == kModeMixed;
     constexpr bool PAGED = MODE == kModePaged || MODE == kModePagedFp8;
     constexpr bool FP8 = MODE == kModePagedFp8;  // pages and rings hold E4M3 codes (head_dim 128 only)
+    constexpr bool STEP = MODE == kModeStep;
     using S = Smem<D, NG>;
     constexpr int KS = D / 16;  // k-steps of Q.K^T; also 16-row slabs of O^T
     constexpr int MS = S::kMergeStride;
@@ -461,6 +474,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     PagedArgs* s_paged = reinterpret_cast<PagedArgs*>(reinterpret_cast<uint8_t*>(s_args) + (sizeof(DecodeArgs) + 15) / 16 * 16);
     int* s_pages = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(s_paged) + (sizeof(PagedArgs) + 15) / 16 * 16);
     const PagedArgs* pg = PAGED ? s_paged : nullptr;
+    // whole-step launch: the layer tables and the KV head of every slot, at the same place
+    const StepArgs* stp = STEP ? reinterpret_cast<const StepArgs*>(s_paged) : nullptr;
+    unsigned char* s_heads = reinterpret_cast<unsigned char*>(s_paged) + (sizeof(StepArgs) + 15) / 16 * 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -488,6 +504,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     if (PAGED)
         for (int i = tid; i < (int)(sizeof(PagedArgs) / sizeof(int)); i += blockDim.x)
             reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+    if constexpr (STEP) {
+        for (int i = tid; i < (int)(sizeof(StepArgs) / sizeof(int)); i += blockDim.x)
+            reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+        for (int i = tid; i < extra.n_layers * extra.kv_heads; i += blockDim.x)  // written at cache creation
+            s_heads[i] = (unsigned char)__ldg(extra.head_of_slot + i);
+    }
     if (tid == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
@@ -564,7 +586,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
                 if (item >= 0) {
-                    u = locate<MODE>(a, x, pg);
+                    u = locate<MODE>(a, x, pg, stp, s_heads);
                     seg_tiles = min(x1 - x, u.pos.run);
                     const bool local_unit = MIXED && u.pos.uid >= sc.U;
                     const bool fp8_unit = FP8;  // every unit of an 8-bit cache is pages of E4M3 codes
@@ -956,6 +978,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 // PAGED: tiles of the segment past the unit's own length (not issued); first pool row of the
                 // full head's pages (-1: a compressed unit); page-table index of s_pages[0]; next tile
                 int seg_skip = 0, paged_row0 = -1, page_base = 0, paged_tile = 0, ring_next = 0;
+                int cur_tile = 0, newest_tile = -1;  // lock-step cache: the tile about to be issued, the full unit's last tile
                 bool asked = false;
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
@@ -969,7 +992,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     }
                     const long long ts0 = trace ? clock64() : 0;
                     if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
-                        const UnitInfo u = locate<MODE>(a, x, pg);
+                        const UnitInfo u = locate<MODE>(a, x, pg, stp, s_heads);
                         seg_left = min(x1 - x, u.pos.run);
                         seg_idx = 0;
                         local_row0 = -1;
@@ -1030,21 +1053,20 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                         } else {
                         // rows the append launch of this step writes: a compressed unit's ring, the
-                        // last tile of a full unit.  Everything else is older and may be fetched early.
-                        if (a.dep_wait == 1 && !synced &&
-                            (k != (int)blockIdx.x || u.pos.uid >= sc.U || u.pos.tile + seg_left == u.tiles)) {
+                        // last tile of a full unit (waited for when that tile's turn comes, below).
+                        // Everything else is older and may be fetched early.
+                        if (a.dep_wait == 1 && !synced && (k != (int)blockIdx.x || u.pos.uid >= sc.U)) {
                             grid_dep_wait();
                             synced = true;
                         }
-                        if (u.pos.uid < sc.U) {
-                            krow = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full) + u.pos.tile * kTile;
-                            vrow = krow + a.rows_full;
-                        } else if (MIXED) {
-                            local_row0 = (int)(a.full_row0 + (long long)(u.pos.uid - sc.U) * 2 * a.rows_full);
+                        cur_tile = u.pos.tile;
+                        newest_tile = u.pos.uid < sc.U ? u.tiles - 1 : -1;
+                        if (MIXED && u.pos.uid >= sc.U) {
+                            local_row0 = u.row0;
                             local_next = u.pos.tile;
                         } else {
-                            krow = (int)(a.comp_row0 + (long long)(u.pos.uid - sc.U) * 2 * a.rows_comp) + u.pos.tile * kTile;
-                            vrow = krow + a.rows_comp;
+                            krow = u.row0 + u.pos.tile * kTile;
+                            vrow = krow + u.vrows;
                         }
                         qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
                         }
@@ -1071,6 +1093,13 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         local_tile(a, local_next++, row, valid);
                         krow = local_row0 + row;
                         vrow = krow + a.rows_full;
+                    }
+                    if (!PAGED) {
+                        if (a.dep_wait == 1 && !synced && cur_tile == newest_tile) {  // the tile that holds this step's token
+                            grid_dep_wait();
+                            synced = true;
+                        }
+                        ++cur_tile;
                     }
                     if (trace) cy_seg += clock64() - ts0;
                     ok = wait_traced(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout, trace,
@@ -1350,6 +1379,8 @@ cudaError_t prepare_one()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(decode_kernel<D, NG, kModeMixed>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(decode_kernel<D, NG, kModeStep>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynamicSmem);
+    if (e != cudaSuccess) return e;
     if (D == 128 && NG == 2) {  // 8-bit pages: head_dim 128, two consumer groups only
         e = cudaFuncSetAttribute(decode_kernel<128, 2, kModePagedFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kMaxDynamicSmem);
@@ -1385,30 +1416,32 @@ cudaError_t prepare_decode_kernels(int head_dim)
 
 template <int D, int NG>
 static cudaError_t launch_either(const DecodeArgs& a, const CUtensorMap& tmap, int grid, int stages, cudaStream_t stream,
-                                 bool overlap, int mode, const PagedArgs* paged)
+                                 bool overlap, int mode, const PagedArgs* paged, const StepArgs* step)
 {
     if (mode == kModePaged) return launch_one<D, NG, kModePaged>(a, tmap, grid, stages, stream, overlap, *paged);
+    if (mode == kModeStep) return launch_one<D, NG, kModeStep>(a, tmap, grid, stages, stream, overlap, *step);
     if (mode == kModeMixed) return launch_one<D, NG, kModeMixed>(a, tmap, grid, stages, stream, overlap, NoPagedArgs{});
     return launch_one<D, NG, kModePlain>(a, tmap, grid, stages, stream, overlap, NoPagedArgs{});
 }
 
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
                           int stages, int groups, cudaStream_t stream, bool overlap, int mode, const PagedArgs* paged,
-                          const PagedFp8Args* paged8)
+                          const PagedFp8Args* paged8, const StepArgs* step)
 {
     if (mode == kModePaged && !paged) return cudaErrorInvalidValue;
+    if (mode == kModeStep && !step) return cudaErrorInvalidValue;
     if (mode == kModePagedFp8) {
         if (!paged8 || head_dim != 128 || groups != 2) return cudaErrorInvalidValue;
         return launch_one<128, 2, kModePagedFp8>(a, *tmap, grid, stages, stream, overlap, *paged8);
     }
     if (head_dim == 128) {
-        if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged);
-        if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged);
-        return launch_either<128, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+        if (groups == 1) return launch_either<128, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
+        if (groups == 2) return launch_either<128, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
+        return launch_either<128, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
     }
-    if (groups == 1) return launch_either<64, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged);
-    if (groups == 2) return launch_either<64, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged);
-    return launch_either<64, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged);
+    if (groups == 1) return launch_either<64, 1>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
+    if (groups == 2) return launch_either<64, 2>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
+    return launch_either<64, 3>(a, *tmap, grid, stages, stream, overlap, mode, paged, step);
 }
 
 }  // namespace rlkv

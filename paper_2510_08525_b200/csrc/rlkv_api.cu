@@ -43,6 +43,7 @@ struct Layout {
     size_t off_pool = 0, off_tables = 0, off_tickets = 0, off_status = 0, off_partials = 0;
     size_t off_k = 0, off_v = 0, off_q = 0, off_out = 0, off_in2 = 0, off_trace = 0, total = 0;
     int max_grid = 0, max_items = 0;
+    bool step_in_one_launch = false;  // the shape allows rlkv_step to serve all layers with one decode launch
 };
 
 constexpr int kDefaultItemTiles = 32;        // launches of rlkv_step, which overlap: coarse items, few partials
@@ -98,6 +99,23 @@ int make_layout(Layout& L, int layers, int kv_heads, int q_heads, int head_dim, 
                 if (mm > most) most = mm;
             }
         }
+        // a whole step in one launch (step_schedule) uses both halves of the scratch as one: its prefix
+        // gives every CTA and every full unit at most one record, the rest is cut into items of at least
+        // kMinItemTiles tiles while the step is small and of kDefaultItemTiles tiles once it is large
+        {
+            long long U = 0, Uc = 0;
+            for (int l = 0; l < layers; ++l) {
+                U += (long long)batch * L.n_full[l];
+                Uc += (long long)batch * L.n_comp[l];
+            }
+            const long long T = U * (L.rows_full / kTile) + Uc * (L.rows_comp / kTile);
+            const long long small = (long long)L.max_grid * kDefaultItemTiles / kMinItemTiles + 1;  // T < grid * 32
+            const long long large = T / kDefaultItemTiles + 1;
+            const long long fused = 2ll * L.max_grid + 2 * U + Uc + (small > large ? small : large) + 8;
+            L.step_in_one_launch = layers <= kMaxStepLayers && layers * kv_heads <= kMaxStepHeads && T < (1ll << 31) &&
+                                   fused < (1ll << 31);
+            if (L.step_in_one_launch && (fused + 1) / 2 > most) most = (fused + 1) / 2;
+        }
         if (most >= (1ll << 31)) return RLKV_EINVAL;
         L.max_items = (int)most;
     }
@@ -141,6 +159,8 @@ struct rlkv_cache {
     int item_tiles_alone;                         // item_tiles of launches outside rlkv_step
     int trace_on;
     int out_bf16;            // results are stored as bf16 instead of fp32 (rlkv_set_output_bf16)
+    int step_mode;           // rlkv_step: 0 chooses, 1 one decode launch per layer, 2 one for the whole step
+    StepArgs step_args;      // the layer tables of a whole-step launch
     unsigned int claims[2];  // value of each work-claim counter after the launches issued so far
     cudaStream_t in_stream, out_stream;  // rlkv_step_host: copies that run beside the kernels
     cudaEvent_t ev_step[2], ev_done;     // kernels of a call done with staging copy p / results copied out
@@ -306,6 +326,83 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     return RLKV_OK;
 }
 
+// The schedule of a whole step in one launch: U full units of tf tiles and Uc compressed units of tc
+// tiles over all layers, for `grid` CTAs.  Two thirds of the full units go to the whole-unit prefix
+// (one static item per CTA, units streamed in one piece), as long as what remains still gives every
+// CTA a few items to claim, so that CTAs on a slower path to memory end together with the others.
+Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_most)
+{
+    const long long all_tiles = (long long)U * tf + (long long)Uc * tc;
+    int item_tiles = (int)(all_tiles / grid);
+    if (item_tiles > item_most) item_tiles = item_most;
+    if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
+    int U0 = 0;
+    if (U > 0) {
+        const long long rest_wanted = 4ll * grid * item_tiles;  // tiles left to the claimed items
+        long long most = U - (rest_wanted - (long long)Uc * tc + tf - 1) / tf;
+        if (most > U) most = U;
+        U0 = (int)(2ll * U / 3);
+        if (U0 > most) U0 = most > 0 ? (int)most : 0;
+    }
+    return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0);
+}
+
+// One decode launch for every layer of a step (all layers hold the same number of tokens).  q, out:
+// the step's [layers][batch][q_heads][head_dim] arrays.  `after_append`: the launch directly follows the
+// step's append launch and may start beside it.
+int do_decode_step(rlkv_cache* c, const void* q, void* out, cudaStream_t s, bool after_append)
+{
+    const int n = c->len[0];
+    const int cap = c->sink + c->window;
+    DecodeArgs a;
+    memset(&a, 0, sizeof a);
+    a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
+    a.q = static_cast<const __nv_bfloat16*>(q);
+    a.out = static_cast<float*>(out);
+    a.status = dev_at<int>(c, c->lay.off_status);
+    a.trace = dev_at<unsigned long long>(c, c->lay.off_trace);
+    a.rows_full = c->lay.rows_full;
+    a.rows_comp = c->lay.rows_comp;
+    a.len_full = n;
+    a.len_comp = n < cap ? n : cap;
+    a.batch = c->batch * c->layers;
+    a.group = c->q_heads / c->kv_heads;
+    a.q_heads = c->q_heads;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
+    a.trace_on = c->trace_on;
+    a.out_bf16 = c->out_bf16;
+    const StepArgs& st = c->step_args;
+    const int U = st.full_base[c->layers], Uc = st.comp_base[c->layers];
+    const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
+    if ((long long)U * tiles_full + (long long)Uc * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
+    int grid = c->sm_count * c->ctas_per_sm;
+    if (grid > c->lay.max_grid) grid = c->lay.max_grid;
+    a.sched = step_schedule(U, tiles_full, Uc, tiles_comp, grid, c->item_tiles);
+    if (grid > a.sched.n_items) grid = a.sched.n_items;
+    if (a.sched.n_slots > 2 * c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
+    a.partials = dev_at<float>(c, c->lay.off_partials);                // both halves as one
+    a.tickets = dev_at<int>(c, c->lay.off_tickets);                    // one per unit of the step
+    a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4;
+    a.claim_base = c->claims[0];
+    a.dep_wait = after_append ? 1 : 0;
+    RLKV_CUDA(launch_decode(a, &c->tmap, c->head_dim, grid, c->stages, c->groups, s, after_append, kModeStep, nullptr, nullptr,
+                            &st));
+    c->claims[0] += (unsigned int)a.sched.n_items;
+    c->launches++;
+    return RLKV_OK;
+}
+
+// Whether rlkv_step serves all layers with one decode launch: the shape must allow it and every layer
+// must hold the same number of tokens; left to the library (step_mode 0) it is chosen always -- one
+// flat tile space over all layers has no per-layer start-up, tail or merge phase to hide.
+bool step_uses_one_launch(const rlkv_cache* c)
+{
+    if (c->step_mode == 1 || !c->lay.step_in_one_launch) return false;
+    for (int l = 1; l < c->layers; ++l)
+        if (c->len[l] != c->len[0]) return false;
+    return true;
+}
+
 // ---- split-KV scratch that nobody allocates -------------------------------------------------------
 // rlkv_decode_attention_static_scratch keeps the decode kernel's split bookkeeping (work-claim
 // counters, tickets) and partial results here instead of in the cache's own buffer.  The array is
@@ -460,6 +557,7 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->item_tiles_alone = kDefaultItemTilesAlone;
     c->trace_on = 0;
     c->out_bf16 = 0;
+    c->step_mode = 0;
     c->claims[0] = c->claims[1] = 0;
     c->in_stream = c->out_stream = nullptr;
     c->ev_step[0] = c->ev_step[1] = c->ev_done = nullptr;
@@ -528,6 +626,21 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
                        cudaMemcpyHostToDevice);
     }
     if (e != cudaSuccess) return fail(cuda_fail(e, "cudaMemcpy(tables)"));
+    {
+        StepArgs& st = c->step_args;
+        memset(&st, 0, sizeof st);
+        st.head_of_slot = reinterpret_cast<const int*>(c->dev_base + c->lay.off_tables + tbytes);
+        st.n_layers = layers;
+        st.kv_heads = kv_heads;
+        st.batch = batch;
+        if (c->lay.step_in_one_launch)
+            for (int l = 0; l < layers; ++l) {
+                st.full_base[l + 1] = st.full_base[l] + batch * c->lay.n_full[l];
+                st.comp_base[l + 1] = st.comp_base[l] + batch * c->lay.n_comp[l];
+                st.full_row0[l] = (int)c->lay.full_row0[l];
+                st.comp_row0[l] = (int)c->lay.comp_row0[l];
+            }
+    }
     rc = make_tensor_map(c);
     if (rc) return fail(rc);
     e = prepare_decode_kernels(head_dim);
@@ -630,6 +743,14 @@ int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q
 
 size_t rlkv_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
+int rlkv_set_step_mode(rlkv_cache* c, int mode)
+{
+    if (!c || mode < 0 || mode > 2) return RLKV_EINVAL;
+    if (mode == 2 && !c->lay.step_in_one_launch) return RLKV_EINVAL;
+    c->step_mode = mode;
+    return RLKV_OK;
+}
+
 int rlkv_set_output_bf16(rlkv_cache* c, int on)
 {
     if (!c) return RLKV_EINVAL;
@@ -661,8 +782,10 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
     const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
     if (c->layers <= kMaxStepLayers) {
+        const bool one_launch = step_uses_one_launch(c);  // asked before the append moves the lengths
         int rc = step_append(c, k, v, s);
         if (rc) return rc;
+        if (one_launch) return do_decode_step(c, q, out, s, true);
         return step_decode(c, 0, c->layers, q, out, s, false);
     }
     for (int l = 0; l < c->layers; ++l) {
@@ -836,16 +959,18 @@ int rlkv_debug_trace(rlkv_cache* c, int enable, unsigned long long* words_host, 
 }
 
 int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas, int item_tiles,
-                        int* n_items_out, int* n_slots_out, int* starts_out, int* tile_map_out, int cap)
+                        int whole_step, int* n_items_out, int* n_slots_out, int* starts_out, int* tile_map_out, int cap)
 {
     if (full_units < 0 || comp_units < 0 || full_units + comp_units < 1 || tiles_full < 1 || tiles_comp < 1 ||
         ctas < 1 || item_tiles < 1 || !n_items_out || !n_slots_out)
         return RLKV_EINVAL;
     if ((long long)full_units * tiles_full + (long long)comp_units * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
-    const Schedule sc = make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
+    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+                                   : make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
     *n_items_out = sc.n_items;
     *n_slots_out = sc.n_slots;
-    if (max_slots(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles) < sc.n_slots) return RLKV_EKERNEL;
+    if (!whole_step && max_slots(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles) < sc.n_slots)
+        return RLKV_EKERNEL;
     if (starts_out) {
         if (cap < sc.n_items + 1) return RLKV_ENOMEM;
         for (int k = 0; k <= sc.n_items; ++k) starts_out[k] = item_start(sc, k);
@@ -863,7 +988,7 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
             tile_map_out[4 * x + 3] = partial_slot(sc, p.band, item_of_tile(sc, x), p.uid);
             // the per-unit list of partial records must contain the record of every tile's segment
             int slot = 0, count = 0;
-            unit_partials(sc, p.uid, p.band, slot, count);
+            unit_partials(sc, p.uid, p.band < 0 ? 0 : p.band, slot, count);
             if (tile_map_out[4 * x + 3] < slot || tile_map_out[4 * x + 3] >= slot + count) return RLKV_EKERNEL;
             if (tile_map_out[4 * x + 3] >= sc.n_slots) return RLKV_EKERNEL;
         }

@@ -12,6 +12,7 @@ constexpr int kTile = 64;        // tokens per K/V tile (one pipeline stage hold
 constexpr int kMaxGroup = 8;     // query heads per KV head handled by one tile pass
 constexpr int kMaxKvHeads = 128; // KV heads per layer (their order travels in the kernel arguments)
 constexpr int kMaxStepLayers = 128;  // layers whose appends rlkv_step does in one launch
+constexpr int kMaxStepHeads = 4096;  // layers * kv_heads that one whole-step decode launch may serve
 constexpr int kGroupWarps = 4;   // consumer warps that share one tile (16 tokens each)
 constexpr int kMaxConsumerGroups = 3;
 constexpr int kMaxDynamicSmem = 227 * 1024;
@@ -45,7 +46,8 @@ enum : int {
     kModePlain = 0,   // the lock-step cache: full and compressed heads, one length for the whole batch
     kModeMixed = 1,   // mixed attention (Eq. 1) over a lock-step cache whose heads are all full
     kModePaged = 2,   // the paged cache: one length per sequence, full heads in 64-token pages
-    kModePagedFp8 = 3 // the paged cache with every K/V row (pages and rings) held as 8-bit E4M3 codes
+    kModePagedFp8 = 3, // the paged cache with every K/V row (pages and rings) held as 8-bit E4M3 codes
+    kModeStep = 4     // the lock-step cache, every layer of a decode step in one launch
 };
 
 // One record of split-KV partial results: running max and sum (log2 domain) of the G query heads
@@ -69,6 +71,11 @@ __host__ __device__ constexpr int partial_floats(int head_dim, int group) {
 // segment that is not the whole unit yields an (m, l, O) partial; the last CTA to deliver a
 // partial of a unit merges them.  Because every unit has a slice in every band, every unit ends
 // up with a similar, small number of partials.
+// A launch with many more units than CTAs (a whole decode step in one launch) puts a PREFIX in front
+// of the bands: the first U0 full units lie there whole, unit after unit, and are cut into P equal
+// items (items 0 .. P-1, one per CTA), so most units are streamed in one piece by one CTA and only
+// the units an item boundary falls into are split.  The remaining U - U0 units follow in bands as
+// above (`rounds` = 0: in one band, i.e. unit after unit, cut into items of min_sz tiles).
 struct Schedule {
     int P;                      // CTAs
     int R;                      // bands handed out in P equal items (the factoring rounds)
@@ -77,6 +84,9 @@ struct Schedule {
     int n_slots;                // partial records the launch may write
     int U, tf, Uc, tc;
     int T;                      // tiles in the flat space
+    int U0;                     // full units in the whole-unit prefix (0: no prefix)
+    int x0, k0, s0;             // first flat tile, first item and first partial record after the prefix
+    int pq, prem;               // the prefix's P items have pq tiles, the first prem one more
     int base[kMaxRounds + 2];   // first flat tile of band r <= R; base[R+1]: first compressed tile
     int tb[kMaxRounds + 2];     // first tile, inside a full unit, of its slice in band r; tb[R+1] = tf
     int slot0[kMaxRounds + 1];  // first partial record of band r
@@ -84,7 +94,7 @@ struct Schedule {
     int irem[kMaxRounds];
 };
 
-inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz)
+inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz, int U0 = 0, int rounds = kMaxRounds)
 {
     Schedule s{};
     s.P = P;
@@ -93,31 +103,40 @@ inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz)
     s.tf = U > 0 ? tf : 0;
     s.Uc = Uc;
     s.tc = Uc > 0 ? tc : 0;
+    if (U0 > U) U0 = U;
+    if (U0 < 0 || (long long)U0 * s.tf < P) U0 = 0;  // every prefix item holds at least one tile
+    s.U0 = U0;
+    s.x0 = U0 * s.tf;
+    s.k0 = U0 > 0 ? P : 0;
+    s.s0 = U0 > 0 ? P + U0 : 0;
+    s.pq = U0 > 0 ? s.x0 / P : 0;
+    s.prem = U0 > 0 ? s.x0 % P : 0;
+    const int Ub = U - U0;  // full units laid out in bands
     int r = 0;
-    s.base[0] = 0;
+    s.base[0] = s.x0;
     s.tb[0] = 0;
-    while (r < kMaxRounds) {
+    while (r < rounds && r < kMaxRounds) {
         const int bw = (s.tf - s.tb[r]) / 2;
-        if ((long long)U * bw / P < 2 * min_sz) break;
+        if ((long long)Ub * bw / P < 2 * min_sz) break;
         s.tb[r + 1] = s.tb[r] + bw;
-        s.base[r + 1] = s.base[r] + U * bw;
-        s.slot0[r] = r * (P + U);
-        s.iq[r] = U * bw / P;
-        s.irem[r] = U * bw % P;
+        s.base[r + 1] = s.base[r] + Ub * bw;
+        s.slot0[r] = s.s0 + r * (P + Ub);
+        s.iq[r] = Ub * bw / P;
+        s.irem[r] = Ub * bw % P;
         ++r;
     }
     s.R = r;
-    s.slot0[r] = r * (P + U);
+    s.slot0[r] = s.s0 + r * (P + Ub);
     s.tb[r + 1] = s.tf;
-    s.base[r + 1] = s.base[r] + U * (s.tf - s.tb[r]);
+    s.base[r + 1] = s.base[r] + Ub * (s.tf - s.tb[r]);
     s.T = s.base[r + 1] + s.Uc * s.tc;
     const int n_final = (s.T - s.base[r] + min_sz - 1) / min_sz;
-    s.n_items = r * P + n_final;
-    s.n_slots = s.slot0[r] + n_final + U + Uc;
+    s.n_items = s.k0 + r * P + n_final;
+    s.n_slots = s.slot0[r] + n_final + Ub + Uc;
     return s;
 }
 
-// Upper bound of n_slots over every tf' <= tf with everything else the same.
+// Upper bound of n_slots over every tf' <= tf with everything else the same (no prefix).
 inline long long max_slots(int U, int tf, int Uc, int tc, int P, int min_sz)
 {
     const Schedule s = make_schedule(U, tf, Uc, tc, P, min_sz);
@@ -132,6 +151,8 @@ inline long long max_slots(int U, int tf, int Uc, int tc, int P, int min_sz)
 __host__ __device__ inline int item_start(const Schedule& s, int k)
 {
     if (k >= s.n_items) return s.T;
+    if (k < s.k0) return k * s.pq + (k < s.prem ? k : s.prem);
+    k -= s.k0;
     const int rp = s.R * s.P;
     if (k < rp) {
         const int r = k / s.P, j = k - r * s.P;
@@ -143,24 +164,33 @@ __host__ __device__ inline int item_start(const Schedule& s, int k)
 // The item that holds flat tile x.
 __host__ __device__ inline int item_of_tile(const Schedule& s, int x)
 {
+    if (x < s.x0) {
+        const int big = s.prem * (s.pq + 1);
+        return x < big ? x / (s.pq + 1) : s.prem + (x - big) / s.pq;
+    }
     for (int r = 0; r < s.R; ++r)
         if (x < s.base[r + 1]) {
             const int y = x - s.base[r], big = s.irem[r] * (s.iq[r] + 1);
-            return r * s.P + (y < big ? y / (s.iq[r] + 1) : s.irem[r] + (y - big) / s.iq[r]);
+            return s.k0 + r * s.P + (y < big ? y / (s.iq[r] + 1) : s.irem[r] + (y - big) / s.iq[r]);
         }
-    return s.R * s.P + (x - s.base[s.R]) / s.min_sz;
+    return s.k0 + s.R * s.P + (x - s.base[s.R]) / s.min_sz;
 }
 
 // Where flat tile x lies: the unit (index over both classes, full units first), the tile inside
 // the unit, how many tiles of the unit follow consecutively in the flat space from x on (x
-// included), and the band.
+// included), and the band (-1: the whole-unit prefix).
 struct TilePos {
     int uid, tile, run, band;
 };
 __host__ __device__ inline TilePos tile_pos(const Schedule& s, int x)
 {
     TilePos p;
-    if (x < s.base[s.R + 1]) {
+    if (x < s.x0) {
+        p.uid = x / s.tf;
+        p.tile = x - p.uid * s.tf;
+        p.run = s.tf - p.tile;
+        p.band = -1;
+    } else if (x < s.base[s.R + 1]) {
         int r = s.R;
         for (int i = 0; i < s.R; ++i)
             if (x < s.base[i + 1]) {
@@ -169,7 +199,7 @@ __host__ __device__ inline TilePos tile_pos(const Schedule& s, int x)
             }
         const int bw = s.tb[r + 1] - s.tb[r], y = x - s.base[r];
         const int unit = y / bw, off = y - unit * bw;
-        p.uid = unit;
+        p.uid = s.U0 + unit;
         p.tile = s.tb[r] + off;
         p.run = bw - off;
         p.band = r;
@@ -185,23 +215,30 @@ __host__ __device__ inline TilePos tile_pos(const Schedule& s, int x)
 }
 
 // The partial record of the segment of unit `uid` inside item `item` of band `band`: along a band
-// every new segment raises the item index or the unit index, so their sum numbers the segments.
+// (and along the prefix) every new segment raises the item index or the unit index, so their sum
+// numbers the segments.
 __host__ __device__ inline int partial_slot(const Schedule& s, int band, int item, int uid)
 {
-    return s.slot0[band] + (item - band * s.P) + uid;
+    if (band < 0) return item + uid;
+    return s.slot0[band] + (item - s.k0 - band * s.P) + (uid - s.U0);
 }
 
-// The partial records of unit `uid` in band `band`: first record and how many (0 if the unit has
-// no slice there).  Full units have a slice in every band, compressed units only in the last.
+// The partial records of unit `uid` in band `band` >= 0: first record and how many (0 if the unit
+// has no slice there).  Full units outside the prefix have a slice in every band, compressed units
+// only in the last; a unit of the prefix reports its records under band 0 and none elsewhere.
 // `tiles`: how many of the unit's tiles exist (paged cache: a sequence shorter than the longest one
 // of the call); segments that hold none of them deliver no record.
 __host__ __device__ inline void unit_partials(const Schedule& s, int uid, int band, int& slot, int& count,
                                               int tiles = 0x7fffffff)
 {
     int first, width;
-    if (uid < s.U) {
+    const bool prefix = uid < s.U0;
+    if (prefix) {
+        width = band == 0 ? (s.tf < tiles ? s.tf : tiles) : 0;
+        first = uid * s.tf;
+    } else if (uid < s.U) {
         width = s.tb[band + 1] - s.tb[band];
-        first = s.base[band] + uid * width;
+        first = s.base[band] + (uid - s.U0) * width;
         if (width > tiles - s.tb[band]) width = tiles - s.tb[band];
     } else {
         width = band == s.R ? (s.tc < tiles ? s.tc : tiles) : 0;
@@ -213,7 +250,7 @@ __host__ __device__ inline void unit_partials(const Schedule& s, int uid, int ba
         return;
     }
     const int kf = item_of_tile(s, first), kl = item_of_tile(s, first + width - 1);
-    slot = partial_slot(s, band, kf, uid);
+    slot = partial_slot(s, prefix ? -1 : band, kf, uid);
     count = kl - kf + 1;
 }
 
@@ -281,6 +318,19 @@ struct alignas(64) PagedFp8Args {
     alignas(64) CUtensorMap map_k;
 };
 
+// A whole decode step in one launch (kModeStep kernels): what DecodeArgs cannot say.  Every layer holds
+// the same number of tokens.  The full units of all layers form one list, layer after layer (inside a
+// layer: batch row, then full-head slot), and so do the compressed units; q and out are the step's
+// [layers][batch][q_heads][head_dim] arrays, so "batch row" l * batch + b addresses them directly.
+struct StepArgs {
+    const int* head_of_slot;            // device, int [n_layers][kv_heads]: KV head of each slot (full slots first)
+    int n_layers, kv_heads, batch;
+    int full_base[kMaxStepLayers + 1];  // first full unit of layer l = batch * (full heads of the layers before it)
+    int comp_base[kMaxStepLayers + 1];  // first compressed unit of layer l, counted from the first compressed unit
+    int full_row0[kMaxStepLayers];      // first pool row of the layer's full-head / compressed-head region
+    int comp_row0[kMaxStepLayers];
+};
+
 struct AppendArgs {
     __nv_bfloat16* pool;
     long long full_row0, comp_row0;
@@ -293,37 +343,79 @@ struct AppendArgs {
     int sink, window;
 };
 
-// What a consumer needs to know about the unit behind a flat tile.
+// What producer and consumers need to know about the unit behind a flat tile.
 struct UnitInfo {
     TilePos pos;
     int tiles;       // tiles of the unit
     int len;         // valid rows of the unit
-    int b, head;     // batch row, KV head
+    int b, head;     // batch row (whole-step launch: layer * batch + batch row), KV head
+    int row0;        // lock-step cache: first pool row of the unit's K rows; its V rows start `vrows` further on
+    int vrows;
 };
 
+// The layer a unit of a whole-step launch belongs to: the last l with base[l] <= unit.
+__device__ inline int step_layer(const int* base, int n_layers, int unit)
+{
+    int lo = 0, hi = n_layers - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (base[mid] <= unit) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+
+// `st`, `heads`: whole-step launches only -- the layer tables and the KV head of every slot
+// ([layer][kv_heads] bytes), both in shared memory.
 template <int MODE = kModePlain>
-__device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* pg = nullptr)
+__device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* pg = nullptr, const StepArgs* st = nullptr,
+                                  const unsigned char* heads = nullptr)
 {
     constexpr bool MIXED = MODE == kModeMixed;
     UnitInfo u;
     u.pos = tile_pos(a.sched, x);
+    u.row0 = 0;
+    u.vrows = 0;
+    if (MODE == kModeStep) {
+        const bool full = u.pos.uid < a.sched.U;
+        const int unit = full ? u.pos.uid : u.pos.uid - a.sched.U;
+        const int* base = full ? st->full_base : st->comp_base;
+        const int l = step_layer(base, st->n_layers, unit);
+        const int local = unit - base[l];
+        const int nf = (st->full_base[l + 1] - st->full_base[l]) / st->batch;
+        const int per_row = full ? nf : st->kv_heads - nf;  // units of this class per batch row of the layer
+        const int b = local / per_row, slot = local - b * per_row;
+        u.tiles = full ? a.sched.tf : a.sched.tc;
+        u.len = full ? a.len_full : a.len_comp;
+        u.b = l * st->batch + b;
+        u.head = heads[l * st->kv_heads + (full ? slot : nf + slot)];
+        u.vrows = full ? a.rows_full : a.rows_comp;
+        u.row0 = (full ? st->full_row0[l] : st->comp_row0[l]) + local * 2 * u.vrows;
+        return u;
+    }
     if (u.pos.uid < a.sched.U) {
         u.tiles = a.sched.tf;
         u.len = a.len_full;
         u.b = u.pos.uid / a.n_full;
         u.head = a.head_of_slot[u.pos.uid - u.b * a.n_full];
+        u.vrows = a.rows_full;
+        u.row0 = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full);
     } else if (MIXED) {  // the local unit of full unit uid - U
         const int unit = u.pos.uid - a.sched.U;
         u.tiles = a.sched.tc;
         u.len = 0;       // its tiles' rows come from local_tile
         u.b = unit / a.n_full;
         u.head = a.head_of_slot[unit - u.b * a.n_full];
+        u.vrows = a.rows_full;
+        u.row0 = (int)(a.full_row0 + (long long)unit * 2 * a.rows_full);
     } else {
         const int unit = u.pos.uid - a.sched.U;
         u.tiles = a.sched.tc;
         u.len = a.len_comp;
         u.b = unit / a.n_comp;
         u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
+        u.vrows = a.rows_comp;
+        u.row0 = (int)(a.comp_row0 + (long long)unit * 2 * a.rows_comp);
     }
     if (MODE == kModePaged || MODE == kModePagedFp8) {  // this sequence's own length
         const int n = pg->seq_len[u.b];
@@ -394,7 +486,8 @@ struct AppendAllArgs {
 cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeArgs& a, const CUtensorMap* tmap, int head_dim, int grid,
                           int stages, int groups, cudaStream_t stream, bool overlap, int mode = kModePlain,
-                          const PagedArgs* paged = nullptr, const PagedFp8Args* paged8 = nullptr);
+                          const PagedArgs* paged = nullptr, const PagedFp8Args* paged8 = nullptr,
+                          const StepArgs* step = nullptr);
 cudaError_t prepare_decode_kernels(int head_dim);
 size_t decode_smem_bytes(int head_dim, int stages, int group, int groups, int mode = kModePlain);
 

@@ -374,8 +374,9 @@ def test_dynamic_work_claims_do_not_change_bits(rl, hz, cuda_device):
 
 
 # ------------------------------------------------------------------------------------------ decode loop
+@pytest.mark.parametrize("step_mode", [1, 2], ids=["launch_per_layer", "one_launch"])
 @pytest.mark.parametrize("layers", [1, 2])
-def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
+def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers, step_mode):
     """A reduced chain-of-thought loop: prompt of 300 tokens, then 700 whole steps through rlkv_step
     (whose launches overlap one another on the device), sink 16 + window 240 so the ring wraps several
     times.  Outputs are compared with the oracle every 50 steps and at the end, cache state bit for bit
@@ -383,6 +384,7 @@ def test_long_decode_loop_through_rlkv_step(rl, hz, cuda_device, layers):
     Hkv, Hq, D, B, S, W, prompt, steps = 2, 8, 128, 2, 16, 240, 300, 700
     mask = ([1, 0] + [0, 1])[:2 * layers]
     cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, cuda_device)
+    rl.rlkv_set_step_mode(cache.handle, step_mode)
     for l in range(layers):
         feed(cache, oracle, l, rand_bf16((prompt, B, Hkv, D), 50 + l), rand_bf16((prompt, B, Hkv, D), 60 + l), True)
     out = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
@@ -438,16 +440,19 @@ def test_reduced_loop_of_4000_steps_checked_at_every_step(rl, hz, cuda_device):
     assert cache.length(0) == prompt + steps and cache.status() == 0
 
 
-def test_step_mixes_tiny_and_gpu_filling_launches(rl, hz, cuda_device):
-    """Seven layers whose launches alternate between a few work items and more than one per SM (all
-    heads compressed, one full head, all full): inside rlkv_step a launch after a small one starts
-    beside it and holds its own successor back, a launch after a GPU-filling one starts as SMs free
-    up.  60 consecutive steps, every layer against the oracle at several of them, and the step's
-    results equal to the per-layer calls on a twin cache."""
+@pytest.mark.parametrize("step_mode", [1, 2], ids=["launch_per_layer", "one_launch"])
+def test_step_mixes_tiny_and_gpu_filling_launches(rl, hz, cuda_device, step_mode):
+    """Seven layers that alternate between a few work items and more than one per SM (all heads
+    compressed, one full head, all full).  With one launch per layer every launch of the step starts
+    beside its predecessor and holds its own successor back until that predecessor has completed; with
+    one launch for the step the layers' units share one flat tile space.  60 consecutive steps, every
+    layer against the oracle at several of them, and the step's results equal to the per-layer calls on
+    a twin cache."""
     Hkv, Hq, D, B, S, W, prompt, steps = 4, 16, 128, 6, 8, 56, 3000, 60
     mask = [0, 0, 0, 0,  1, 1, 1, 1,  0, 1, 0, 0,  0, 0, 0, 0,  0, 0, 0, 0,  1, 1, 1, 1,  1, 0, 0, 1]
     layers = len(mask) // Hkv
     cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, cuda_device)
+    rl.rlkv_set_step_mode(cache.handle, step_mode)
     twin = hz.Cache(layers, Hkv, Hq, D, B, prompt + steps, mask, S, W, device=cuda_device)
     for l in range(layers):
         K, V = rand_bf16((prompt, B, Hkv, D), 150 + l), rand_bf16((prompt, B, Hkv, D), 160 + l)
@@ -466,9 +471,76 @@ def test_step_mixes_tiny_and_gpu_filling_launches(rl, hz, cuda_device):
             got = out.cpu().numpy()
             for l in range(layers):
                 check_out(got[l], oracle.decode(l, Q[t, l]))
-                np.testing.assert_allclose(got[l], twin.decode(l, Qd[t, l]).cpu().numpy(), atol=1e-4, rtol=0)
+                # the two cut the rows differently, so P is rounded to bf16 against different running
+                # maxima: the difference is rounding noise (a few 1e-5 per element at this length)
+                np.testing.assert_allclose(got[l], twin.decode(l, Qd[t, l]).cpu().numpy(), atol=5e-4, rtol=0)
     check_state(cache, oracle)
     assert cache.status() == 0 and twin.status() == 0
+
+
+def test_one_launch_step_against_launch_per_layer_and_oracle(rl, hz, cuda_device):
+    """rlkv_step as one attention launch over all layers against the same step with one launch per layer
+    and against the oracle, on shapes where the whole-step schedule has a prefix of whole units (many
+    units), where it has none (few tiles), with layers that hold no full or no compressed head, and
+    with head_dim 64.  A step whose layers hold different numbers of tokens falls back to one launch per
+    layer and is still right.  Planted needles: in every layer one batch row's newest token (written by
+    the step's own append launch, which the attention launch may start beside) and its first token carry
+    markers that must show in the output."""
+    cases = [
+        # layers, Hkv, Hq, D, B, S, W, n, fraction compressed
+        (6, 4, 16, 128, 8, 16, 48, 3000, 0.4),
+        (5, 2, 8, 64, 2, 4, 60, 150, 0.5),
+        (3, 8, 32, 128, 1, 16, 112, 5000, 0.8),
+        (4, 4, 4, 128, 3, 8, 24, 700, 0.0),
+        (4, 4, 28, 128, 3, 8, 24, 700, 1.0),
+    ]
+    for ci, (layers, Hkv, Hq, D, B, S, W, n, frac) in enumerate(cases):
+        mask = synth.head_mask(40 + ci, layers, Hkv, frac)
+        a, oracle = build_pair(hz, layers, Hkv, Hq, D, B, n + 8, mask, S, W, cuda_device)
+        b = hz.Cache(layers, Hkv, Hq, D, B, n + 8, mask, S, W, device=cuda_device)
+        rl.rlkv_set_step_mode(a.handle, 2)
+        rl.rlkv_set_step_mode(b.handle, 1)
+        for l in range(layers):
+            K, V = rand_bf16((n, B, Hkv, D), 500 + 10 * ci + l), rand_bf16((n, B, Hkv, D), 600 + 10 * ci + l)
+            feed(a, oracle, l, K, V, True)
+            b.prefill(l, K.to(cuda_device), V.to(cuda_device))
+        out_a = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+        out_b = torch.empty_like(out_a)
+        for t in range(3):
+            k, v = rand_bf16((layers, B, Hkv, D), 700 + t), rand_bf16((layers, B, Hkv, D), 710 + t)
+            q = rand_bf16((layers, B, Hq, D), 720 + t)
+            if t == 1:                                       # needles: the token appended now, row 0 of every layer
+                for l in range(layers):
+                    for h in range(Hkv):
+                        qq = q[l, 0, h * (Hq // Hkv)].to(torch.float32)
+                        k[l, 0, h] = (qq / qq.norm() * 100.0).to(torch.bfloat16)
+                        v[l, 0, h] = 5.0
+            kd, vd, qd = k.to(cuda_device), v.to(cuda_device), q.to(cuda_device)
+            rl.rlkv_step(a.handle, kd, vd, qd, out_a)
+            rl.rlkv_step(b.handle, kd, vd, qd, out_b)
+            got = out_a.cpu().numpy()
+            assert torch.allclose(out_a, out_b, atol=5e-4, rtol=0)   # different cuts: rounding noise only
+            for l in range(layers):
+                assert oracle.append(l, k[l], v[l]) == 0
+                check_out(got[l], oracle.decode(l, q[l]))
+            if t == 1:
+                G = Hq // Hkv
+                assert np.abs(got[:, 0, ::G] - 5.0).max() < 1e-2     # the first query head of every group saw its needle
+        check_state(a, oracle)
+        # different lengths: one more token for layer 0 only, then a step
+        k1, v1 = rand_bf16((B, Hkv, D), 800), rand_bf16((B, Hkv, D), 801)
+        a.append(0, k1.to(cuda_device), v1.to(cuda_device))
+        oracle.append(0, k1, v1)
+        k, v, q = rand_bf16((layers, B, Hkv, D), 802), rand_bf16((layers, B, Hkv, D), 803), rand_bf16((layers, B, Hq, D), 804)
+        rl.rlkv_step(a.handle, k.to(cuda_device), v.to(cuda_device), q.to(cuda_device), out_a)
+        got = out_a.cpu().numpy()
+        for l in range(layers):
+            assert oracle.append(l, k[l], v[l]) == 0
+            check_out(got[l], oracle.decode(l, q[l]))
+        check_state(a, oracle)
+        assert a.status() == 0 and b.status() == 0
+        a.close()
+        b.close()
 
 
 def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):

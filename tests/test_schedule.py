@@ -74,6 +74,67 @@ def test_banded_schedule(rl, U, tf, Uc, tc, ctas, item):
     assert per_unit.max() <= rounds * per_band + last_band_tiles / item + 3, (per_unit.max(), rounds)
 
 
+STEP_SHAPES = [
+    # full units, tiles each, compressed units, tiles each, CTAs, largest item
+    (3280, 129, 816, 2, 148, 32),       # 32 layers x batch 16, 205 of 256 heads full, n = 8193
+    (1232, 65, 816, 4, 148, 32),        # batch 8, n = 4097, 16 + 240 rings
+    (205, 33, 51, 2, 148, 32),          # batch 1, n = 2049: fewer tiles than 32 per CTA
+    (51, 129, 205, 2, 148, 32),         # 80 % compressed
+    (8, 1025, 248, 2, 148, 32),         # very few, very long full units
+    (0, 1, 256, 2, 148, 32),            # no full unit at all
+    (2, 3, 2, 1, 148, 32), (300, 1, 0, 1, 148, 32), (149, 2, 0, 1, 148, 2), (1000, 7, 24, 3, 7, 5),
+]
+
+
+@pytest.mark.parametrize("U,tf,Uc,tc,ctas,item", STEP_SHAPES)
+def test_whole_step_schedule(rl, U, tf, Uc, tc, ctas, item):
+    """The schedule of a whole decode step in one launch: most full units lie whole, unit after unit,
+    in one static item per CTA (the prefix); the remaining units follow unit after unit in small items.
+    Every tile exactly once, items in order, one partial record per segment, none shared; units of the
+    prefix are split only where an item boundary falls into them."""
+    starts, n_slots, tmap = rl.rlkv_debug_schedule(U, tf, Uc, tc, ctas, item, tile_map=True, whole_step=True)
+    T = U * tf + Uc * tc
+    assert starts[0] == 0 and starts[-1] == T
+    sizes = np.diff(starts)
+    assert (sizes >= 1).all()
+    n_items = sizes.size
+    uid, tile, run, slot = tmap[:, 0], tmap[:, 1], tmap[:, 2], tmap[:, 3]
+    want = [(u, t) for u in range(U) for t in range(tf)] + [(U + u, t) for u in range(Uc) for t in range(tc)]
+    assert list(zip(uid.tolist(), tile.tolist())) == want          # unit after unit, tile after tile
+    for x in range(T - 1):
+        if run[x] > 1:
+            assert uid[x + 1] == uid[x] and run[x + 1] == run[x] - 1
+    # the prefix: the first `ctas` items are near-equal and hold whole units except at their borders;
+    # the items after it are small
+    small = min(item, max(2, T // ctas))
+    prefix_items = ctas if n_items > ctas and sizes[:ctas].min() > small else 0
+    if prefix_items:
+        part = sizes[:ctas]
+        assert part.max() - part.min() <= 1
+        x0 = int(starts[ctas])
+        assert x0 % tf == 0 and x0 // tf <= (2 * U) // 3 + 1       # whole units, at most two thirds of them
+        assert T - x0 >= 4 * ctas * small - tf                     # enough left for every CTA to claim a few items
+        rest = sizes[ctas:]
+        assert (rest[:-1] == small).all() and 1 <= rest[-1] <= small
+    else:
+        assert (sizes[:-1] == small).all()
+    item_of = np.repeat(np.arange(n_items), sizes)
+    new_seg = np.ones(T, bool)
+    new_seg[1:] = (item_of[1:] != item_of[:-1]) | (uid[1:] != uid[:-1])
+    seg_id = np.cumsum(new_seg) - 1
+    seg_slot = {}
+    for x in range(T):
+        seg_slot.setdefault(int(seg_id[x]), set()).add(int(slot[x]))
+    assert all(len(v) == 1 for v in seg_slot.values())
+    slots = [next(iter(v)) for v in seg_slot.values()]
+    assert len(set(slots)) == len(slots) and max(slots) < n_slots
+    per_unit = np.bincount(uid[new_seg], minlength=U + Uc)
+    if prefix_items:                                               # a prefix unit: one piece, or one more per item border inside it
+        n_prefix = int(starts[ctas]) // tf
+        assert per_unit[:n_prefix].max() <= 1 + -(-tf // int(sizes[:ctas].min()))
+        assert (per_unit[:n_prefix] == 1).sum() >= n_prefix - 2 * ctas
+
+
 def test_schedule_rejects_bad_arguments(rl):
     for bad in ((0, 1, 0, 1, 148, 4), (1, 0, 0, 1, 148, 4), (1, 1, 1, 0, 148, 4), (1, 1, 0, 1, 0, 4),
                 (1, 1, 0, 1, 148, 0), (-1, 1, 2, 1, 148, 4)):
