@@ -156,28 +156,63 @@ def barrier():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while a timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU while a timed region runs: through NVML
+    every 2 ms where the Python bindings are there (read-only queries), else through nvidia-smi."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
     def __init__(self, gpu_index: int):
-        self.gpu, self.rows, self.proc = gpu_index, [], None
+        self.gpu, self.rows, self.proc, self.thread, self.stop, self.how = gpu_index, [], None, None, False, None
 
     def wait_first_sample(self, timeout=3.0):
         t0 = time.perf_counter()
-        while self.proc and not self.rows and time.perf_counter() - t0 < timeout:
+        while self.thread and not self.rows and time.perf_counter() - t0 < timeout:
             time.sleep(0.01)
 
     def mark(self):
         """Index of the next sample: samples from here on belong to what follows."""
         return len(self.rows)
 
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            uuid = torch.cuda.get_device_properties(self.gpu).uuid
+            return pynvml, pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+        except Exception:
+            return pynvml, pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
+
     def __enter__(self):
+        try:
+            nv, h = self._nvml_handle()
+            nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+            mx = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+            bits = [(nv.nvmlClocksEventReasonHwSlowdown, 0), (nv.nvmlClocksEventReasonHwThermalSlowdown, 1),
+                    (nv.nvmlClocksEventReasonSwThermalSlowdown, 2), (nv.nvmlClocksEventReasonSwPowerCap, 3)]
+
+            def loop():
+                while not self.stop:
+                    try:
+                        sm = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                        reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                        row = [str(sm), str(mx), ""] + ["Active" if reasons & bit else "Not Active" for bit, _ in bits]
+                        self.rows.append(row)
+                    except Exception:
+                        pass
+                    time.sleep(0.002)
+            self.how = "nvml, every 2 ms"
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+            return self
+        except Exception:
+            pass
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                  "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.how = "nvidia-smi -lms 20"
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -191,28 +226,29 @@ class ClockSampler:
                 self.rows.append(parts)
 
     def __exit__(self, *exc):
+        self.stop = True
         if self.proc:
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=5)
             except subprocess.TimeoutExpired:
                 self.proc.kill()
+        if self.thread:
             self.thread.join(timeout=5)
 
     def summary(self, start=0, end=None):
         sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in self.rows[start:end]:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
             except ValueError:
                 continue
-            for name, val in zip(names, r[3:]):
+            for name, val in zip(self.NAMES, r[3:]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "reasons": sorted(reasons), "samples": len(sm), "how": self.how}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -564,7 +600,7 @@ def run_ours(args, w, mask):
     clocks.wait_first_sample()
 
     # ---- pass 1: device-resident steps (the headline value), one event between consecutive steps
-    cache, steps_in, res = timed_steps(rl, harness, w, mask, dev, stream, K, W, clocks, tune, extra_tokens=2 * (K + W))
+    cache, steps_in, res = timed_steps(rl, harness, w, mask, dev, stream, K, W, clocks, tune, extra_tokens=2 * (K + W) + 24)
     out = res.pop("out")
     median_ms = max_over_ranks(res["ms_per_step"], dev)
     mean_ms = max_over_ranks(res["ms_per_step_mean"], dev)
@@ -599,31 +635,84 @@ def run_ours(args, w, mask):
     probe_ms = rl.rlkv_debug_read_bandwidth(probe, probe.numel(), 6)
     read_only_gbs = probe.numel() / (probe_ms * 1e-3) / 1e9
     del probe
-    # The decode launches of the timed region (pass 1): K * layers of them between the first and the
-    # last event on the launching stream, overlapping one another as rlkv_step issues them.  Their
-    # average duration is taken as the whole region divided by their number, which charges them the
-    # append launches too.
-    n_launch = K * w.layers
+    # The decode launches of the timed region (pass 1): every step is one append launch and the step's
+    # decode launches (one over all layers, or one per layer where the step had to fall back), between
+    # the first and the last event on the launching stream.  Their average duration is taken as the
+    # whole region divided by their number, which charges them the append launches too.
+    n_launch = launches - K
     step_bytes = res["kv_bytes_per_step"]
-    mean_launch_ms = mean_ms / w.layers
-    achieved = step_bytes / w.layers / (mean_launch_ms * 1e-3) / 1e9
+    mean_launch_ms = mean_ms * K / n_launch
+    bytes_per_launch = step_bytes * K / n_launch
+    achieved = bytes_per_launch / (mean_launch_ms * 1e-3) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "rlkv::decode_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "bound": "hbm", "kernel": "rlkv::decode_kernel (whole-step mode)" if n_launch == K else "rlkv::decode_kernel",
+        "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_source": peak_src, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
         # ncu capture of a 4-layer cut of the workload (same kernel, same per-layer shape), scaled to
         # the mean launch of this run by the algorithmic bytes; null if the kernel has changed since
-        "traffic": None if ratio is None else ratio * step_bytes / w.layers,
+        "traffic": None if ratio is None else ratio * bytes_per_launch,
         "launches_timed": n_launch, "mean_launch_us": 1e3 * mean_launch_ms,
-        "algorithmic_bytes_per_launch": step_bytes / w.layers,
-        "how": "CUDA events on the launching stream around the timed region; launches overlap inside a step "
-               "(programmatic dependent launch), so duration = region / launches",
+        "algorithmic_bytes_per_launch": bytes_per_launch,
+        "how": "CUDA events on the launching stream around the timed region (K steps, each one append launch "
+               "and its decode launches); duration = region / decode launches",
         "read_only_stream": {"gbs": read_only_gbs, "frac_of_it": achieved / read_only_gbs,
                              "how": "rlkv_debug_read_bandwidth: 2 GiB read by bulk copies into shared memory, "
                                     "no consumer, measured in this run"},
         "isolated": {"achieved": isolated, "frac": isolated / peak, "frac_of_nominal_8000": isolated / NOMINAL_HBM_GBS,
                      "mean_launch_us": 1e3 * sum(durs) / len(durs), "launches_timed": len(durs),
-                     "how": "every rlkv_decode_attention launch of K more steps timed alone between two events"},
+                     "how": "the per-layer call: every rlkv_decode_attention launch of K more steps timed alone "
+                            "between two events"},
     }
+
+    # ---- the per-layer calls as a model forward would issue them: before every layer a stand-in kernel
+    # (a ~30 us device copy of the bench's own buffers) that consumes the layer before's output and
+    # writes this layer's k, v, q at its end, then the append and the attention call.  Once with ordinary
+    # launches (rlkv_append, rlkv_decode_attention), once with the overlapped calls and an overlapping
+    # stand-in, once with rlkv_layer_step_overlapped (append and attention in one launch).  Attention time per layer = (chain - the same chain without the attention calls) / layers.
+    per_layer = None
+    if world == 1:
+        kv_e, q_e = w.batch * w.kv_heads * w.head_dim, w.batch * w.q_heads * w.head_dim
+        stage = torch.zeros(2 * kv_e + q_e, dtype=torch.bfloat16, device=dev)
+        kb, vb, qb = stage[:kv_e], stage[kv_e:2 * kv_e], stage[2 * kv_e:]
+        kk, vv, qq = more[0]
+        srcs = [torch.cat([kk[l].reshape(-1), vv[l].reshape(-1), qq[l].reshape(-1)]) for l in range(w.layers)]
+        work_src = torch.ones(96 << 20, dtype=torch.uint8, device=dev)
+        work_dst = torch.empty_like(work_src)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 4
+
+        def chain(overlap, attention):
+            for l in range(w.layers):
+                rl.rlkv_debug_standin(work_dst, work_src, work_src.numel(), out[l - 1] if l else None, stage, srcs[l],
+                                      stage.numel() * 2, 1 if overlap else 0, stream)
+                if attention and overlap == 2:
+                    rl.rlkv_layer_step_overlapped(cache.handle, l, kb, vb, qb, out[l], stream)
+                elif attention and overlap:
+                    rl.rlkv_append_overlapped(cache.handle, l, kb, vb, stream)
+                    rl.rlkv_decode_attention_overlapped(cache.handle, l, qb, out[l], stream)
+                elif attention:
+                    rl.rlkv_append(cache.handle, l, kb, vb, stream)
+                    rl.rlkv_decode_attention(cache.handle, l, qb, out[l], stream)
+
+        per_layer = {"workload": f"{w.name}: every layer = stand-in kernel (96 MiB device copy, writes the layer's k, v, q at "
+                                 f"its end), append, attention; {reps} passes over the {w.layers} layers",
+                     "kv_bytes_per_layer": step_bytes / w.layers}
+        for name, overlap in (("ordinary", 0), ("overlapped", 1), ("overlapped_one_launch", 2)):
+            t = {}
+            for attention in (False, True):
+                chain(overlap, attention)
+                torch.cuda.synchronize()
+                e0.record(stream)
+                for _ in range(reps):
+                    chain(overlap, attention)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                t[attention] = 1e3 * e0.elapsed_time(e1) / (reps * w.layers)
+            us = t[True] - t[False]
+            gbs = step_bytes / w.layers / (us * 1e-6) / 1e9
+            per_layer[name] = {"standin_us": t[False], "chain_us_per_layer": t[True], "attention_us_per_layer": us,
+                               "gbs": gbs, "frac_of_measured_copy": gbs / peak, "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS}
+        del work_src, work_dst
 
     # ---- pass 3: end to end through rlkv_step_host (pinned host buffers, copies inside the timed region)
     e2e = None
@@ -822,7 +911,7 @@ def run_ours(args, w, mask):
             "step_hbm_gbs": total_bytes / (median_ms * 1e-3) / 1e9,
             "bytes_ratio_vs_uncompressed": total_bytes / (w.batch * w.layers * w.kv_heads * (w.context + W + 1 + K // 2) * 4 * w.head_dim),
             "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "gpu_launches": launches,
-            "configs": configs, "mixed_attention": mixed, "paged_cache": paged,
+            "per_layer_calls": per_layer, "configs": configs, "mixed_attention": mixed, "paged_cache": paged,
             "clocks": main_clocks,
         }
         print(json.dumps(line), flush=True)

@@ -93,6 +93,37 @@ int rlkv_prefill(rlkv_cache* cache, int layer, const void* k, const void* v, int
  * Scores, softmax and accumulation are fp32.  RLKV_EEMPTY if length(layer) == 0. */
 int rlkv_decode_attention(rlkv_cache* cache, int layer, const void* q, void* out, void* stream);
 
+/* The per-layer calls for a model forward that wants them to overlap with the kernels around them.
+ * (An integration call: the paper runs attention once per layer inside the model forward, Section 4.3
+ * and Appendix B, and says nothing about how launches are ordered.)  A forward pass cannot use
+ * rlkv_step: layer l + 1's q, k, v exist only after layer l's output has gone through its projections.
+ * These two calls compute exactly what rlkv_append / rlkv_decode_attention compute, but are launched
+ * with programmatic stream serialization, so they may START while the kernel before them on `stream`
+ * is still running, and they let the kernel after them start early in turn:
+ *   - the append executes griddepcontrol.wait before it reads k and v;
+ *   - the attention launch sets up, and fetches K/V tiles that hold only older tokens (as many as its
+ *     tile ring holds), before it waits; the query rows, the newest token's rows, the compressed
+ *     heads' rings, the split-KV scratch and `out` are touched only after the wait.
+ * So q, k and v may be written by the kernel directly before the call.  Requirements on the caller:
+ * every kernel on `stream` that is itself launched with programmatic stream serialization must execute
+ * griddepcontrol.wait (cudaGridDependencySynchronize) before it completes -- the usual way to use the
+ * attribute -- so that a kernel's completion implies the completion of everything before it; a kernel
+ * after the attention call that is launched that way must wait before it reads `out`.  After an
+ * ordinary launch the calls behave like their ordinary counterparts.  Arguments, layouts, results and
+ * error codes are those of rlkv_append and rlkv_decode_attention. */
+int rlkv_append_overlapped(rlkv_cache* cache, int layer, const void* k, const void* v, void* stream);
+int rlkv_decode_attention_overlapped(rlkv_cache* cache, int layer, const void* q, void* out,
+                                     void* stream);
+/* Both of them in ONE launch: the layer's step.  The attention launch appends the token itself --
+ * the CTA that reads the tile a head's new token belongs to copies the caller's K and V rows there
+ * first (bit for bit, after its wait), so no second kernel sits between the producer of k, v, q and
+ * the attention.  Result and cache state are those of rlkv_append followed by
+ * rlkv_decode_attention; the launch overlaps with its neighbours as described above.  k, v: device
+ * bf16 [batch][kv_heads][head_dim]; q, out as for rlkv_decode_attention.  RLKV_EFULL if the layer is
+ * at max_len. */
+int rlkv_layer_step_overlapped(rlkv_cache* cache, int layer, const void* k, const void* v,
+                               const void* q, void* out, void* stream);
+
 /* rlkv_decode_attention for callers that must not allocate device memory.  (The paper has no
  * counterpart: this entry point exists for the integration, not for the method.)
  *
@@ -344,6 +375,17 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
  * milliseconds (CUDA events, after one untimed pass): bytes / that is the read-only bandwidth the
  * decode kernel could at best reach on this GPU.  RLKV_EKERNEL if a wait inside the kernel ran out. */
 int rlkv_debug_read_bandwidth(const void* device_buf, size_t bytes, int launches, float* ms_out);
+
+/* Measurement and test aid: a stand-in for the kernels a model runs between two attention calls.
+ * One launch on `stream` that (1) copies `bytes` bytes from src to dst (device buffers of the caller;
+ * work that depends on nothing, like the weights a projection streams), then (2) waits for the kernel
+ * before it, reads a word of `after` (device; may be NULL -- the attention output it would consume)
+ * and copies produce_bytes bytes from produce_src to produce (device; the next call's q, k or v), so
+ * that those are written at the very end of the kernel.  overlap != 0: launched with programmatic
+ * stream serialization (it may start beside the kernel before it and lets the next one start early);
+ * 0: an ordinary launch.  Sizes are multiples of 16, pointers 16-byte aligned. */
+int rlkv_debug_standin(void* dst, const void* src, size_t bytes, const void* after, void* produce,
+                       const void* produce_src, size_t produce_bytes, int overlap, void* stream);
 
 /* How rlkv_step and rlkv_paged_step order the decode launches of one step, host arithmetic only (no
  * GPU).  For launch l of n_launches in a row (follows_append != 0: the first one directly follows the

@@ -30,6 +30,10 @@ SIGNATURES = {
     "rlkv_prefill": (_ci, [_vp, _ci, _vp, _vp, _ci, _vp]),
     "rlkv_decode_attention": (_ci, [_vp, _ci, _vp, _vp, _vp]),
     "rlkv_decode_attention_static_scratch": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_append_overlapped": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_decode_attention_overlapped": (_ci, [_vp, _ci, _vp, _vp, _vp]),
+    "rlkv_layer_step_overlapped": (_ci, [_vp, _ci, _vp, _vp, _vp, _vp, _vp]),
+    "rlkv_debug_standin": (_ci, [_vp, _vp, _sz, _vp, _vp, _vp, _sz, _ci, _vp]),
     "rlkv_static_scratch_bytes": (_sz, []),
     "rlkv_set_output_bf16": (_ci, [_vp, _ci]),
     "rlkv_paged_set_output_bf16": (_ci, [_vp, _ci]),
@@ -162,6 +166,23 @@ def rlkv_prefill(cache, layer, k, v, n_tokens, stream=None) -> None:
 
 def rlkv_decode_attention(cache, layer, q, out, stream=None) -> None:
     _check(lib.rlkv_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_append_overlapped(cache, layer, k, v, stream=None) -> None:
+    _check(lib.rlkv_append_overlapped(cache, layer, _ptr(k), _ptr(v), _stream(stream)))
+
+
+def rlkv_decode_attention_overlapped(cache, layer, q, out, stream=None) -> None:
+    _check(lib.rlkv_decode_attention_overlapped(cache, layer, _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_layer_step_overlapped(cache, layer, k, v, q, out, stream=None) -> None:
+    _check(lib.rlkv_layer_step_overlapped(cache, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), _stream(stream)))
+
+
+def rlkv_debug_standin(dst, src, nbytes, after, produce, produce_src, produce_bytes, overlap, stream=None) -> None:
+    _check(lib.rlkv_debug_standin(_ptr(dst), _ptr(src), int(nbytes), _ptr(after), _ptr(produce), _ptr(produce_src),
+                                  int(produce_bytes), int(overlap), _stream(stream)))
 
 
 def rlkv_decode_attention_static_scratch(cache, layer, q, out, stream=None) -> None:

@@ -15,6 +15,10 @@ namespace {
 
 __global__ void __launch_bounds__(256) append_kernel(const AppendArgs a)
 {
+    if (a.overlap) {  // launched so that it may start before the kernel that writes k and v has completed
+        grid_dep_launch();  // the next kernel may start as well: it waits for this one before it reads the new rows
+        grid_dep_wait();
+    }
     const int chunks = a.head_dim / 8;  // 16-byte pieces per row
     const long long per_token = (long long)a.batch * a.kv_heads * chunks;
     const long long total = per_token * a.n_tokens * 2;
@@ -186,8 +190,16 @@ cudaError_t launch_append(const AppendArgs& a, cudaStream_t stream)
     long long blocks = (total + 255) / 256;
     if (blocks > 148 * 16) blocks = 148 * 16;
     if (blocks < 1) blocks = 1;
-    append_kernel<<<(unsigned)blocks, 256, 0, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, append_kernel, a);
 }
 
 cudaError_t launch_append_all(const AppendAllArgs& a, cudaStream_t stream)

@@ -493,7 +493,12 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     //     anything else, and only then lets the next layer start.
     //   dep_wait == 2: any later launch of the step, which may run beside its predecessor: an otherwise
     //     idle thread of every CTA waits for the predecessor and only then lets the next launch start.
-    if (tid == 0 && !args.dep_wait) grid_dep_launch();
+    //   dep_wait == 3: a per-layer call that may start before the kernel that produces its q (and before
+    //     the append of this step's token) has completed: the producer fetches K/V tiles of older tokens
+    //     -- as many as the tile ring holds -- and waits before it fetches the query rows, the newest
+    //     tile or a ring; claims, tickets, partials and results come after a wait as well.  The next
+    //     kernel of the stream may start at once (it waits for this one itself before it reads `out`).
+    if (tid == 0 && (!args.dep_wait || args.dep_wait == 3)) grid_dep_launch();
 
     if ((smem_u32(smem) & 1023u) != 0) {  // uniform over the CTA: nobody has touched a barrier yet
         if (tid == 0) atomicCAS(args.status, kStatusOk, kStatusSmemMisaligned);
@@ -945,6 +950,17 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             bool synced = false;  // has waited for the kernels before this one
             uint32_t ppar = 0;    // PAGED: phase of the page look-up barrier
+            const bool early = a.dep_wait == 1 || a.dep_wait == 3;  // the launch may run before its inputs are complete
+            // dep_wait 3: query rows whose copy is put off until the kernel that writes them has completed
+            uint32_t late_dst[8], late_bar[8];
+            const __nv_bfloat16* late_src[8];
+            int n_late = 0;
+            auto sync_now = [&]() {
+                grid_dep_wait();
+                synced = true;
+                for (int j = 0; j < n_late; ++j) bulk_load(late_dst[j], late_src[j], G * D * 2, late_bar[j]);
+                n_late = 0;
+            };
             while (ok && k < sc.n_items) {
                 const long long ti0 = trace ? clock64() : 0;
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
@@ -979,6 +995,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 // full head's pages (-1: a compressed unit); page-table index of s_pages[0]; next tile
                 int seg_skip = 0, paged_row0 = -1, page_base = 0, paged_tile = 0, ring_next = 0;
                 int cur_tile = 0, newest_tile = -1;  // lock-step cache: the tile about to be issued, the full unit's last tile
+                // a launch that also appends the step's token (DecodeArgs::new_k): the tile and the row, inside
+                // the unit, that the token goes to; where its K row comes from
+                int new_tile = -1, new_row = 0, new_unit_row0 = 0, new_vrows = 0;
+                const __nv_bfloat16* new_src = nullptr;
                 bool asked = false;
                 const __nv_bfloat16* qsrc = nullptr;
                 for (int x = x0; ok && x < x1; ++x) {
@@ -1055,12 +1075,17 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit (waited for when that tile's turn comes, below).
                         // Everything else is older and may be fetched early.
-                        if (a.dep_wait == 1 && !synced && (k != (int)blockIdx.x || u.pos.uid >= sc.U)) {
-                            grid_dep_wait();
-                            synced = true;
-                        }
+                        if (early && !synced && (k != (int)blockIdx.x || u.pos.uid >= sc.U)) sync_now();
                         cur_tile = u.pos.tile;
                         newest_tile = u.pos.uid < sc.U ? u.tiles - 1 : -1;
+                        if (!MIXED && !STEP && a.new_k) {
+                            const int t = a.len_full - 1;  // the token of this step
+                            new_row = u.pos.uid < sc.U ? t : (t < a.new_sink ? t : a.new_sink + (t - a.new_sink) % a.new_window);
+                            new_tile = new_row / kTile;
+                            new_unit_row0 = u.row0;
+                            new_vrows = u.vrows;
+                            new_src = a.new_k + ((size_t)u.b * (a.q_heads / G) + u.head) * D;
+                        }
                         if (MIXED && u.pos.uid >= sc.U) {
                             local_row0 = u.row0;
                             local_next = u.pos.tile;
@@ -1095,9 +1120,35 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         vrow = krow + a.rows_full;
                     }
                     if (!PAGED) {
-                        if (a.dep_wait == 1 && !synced && cur_tile == newest_tile) {  // the tile that holds this step's token
-                            grid_dep_wait();
-                            synced = true;
+                        // the tile that holds this step's token; a stage whose release depends on query rows
+                        // that have not been fetched yet (the ring is full of tiles nobody can consume)
+                        if (early && !synced && (cur_tile == newest_tile || (a.dep_wait == 3 && issued >= stages))) sync_now();
+                        if (!MIXED && !STEP && cur_tile == new_tile) {
+                            // This CTA is the one that reads the tile the step's token belongs to: it writes the
+                            // token's K and V rows there itself (a bit-exact copy of the caller's rows), then makes
+                            // them visible to the tile copy it issues next.
+                            if (early && !synced) sync_now();
+                            const uint4* src_k = reinterpret_cast<const uint4*>(new_src);
+                            const uint4* src_v = reinterpret_cast<const uint4*>(a.new_v + (new_src - a.new_k));
+                            uint4* dst_k = reinterpret_cast<uint4*>(const_cast<__nv_bfloat16*>(a.pool) + (size_t)(new_unit_row0 + new_row) * D);
+                            uint4* dst_v = dst_k + (size_t)new_vrows * D / 8;
+                            constexpr int N16 = D / 8;  // 16-byte pieces per row
+#pragma unroll
+                            for (int c0 = 0; c0 < N16; c0 += 8) {
+                                uint4 rk[8], rv[8];
+#pragma unroll
+                                for (int c = 0; c < 8; ++c) {
+                                    rk[c] = __ldcg(src_k + c0 + c);
+                                    rv[c] = __ldcg(src_v + c0 + c);
+                                }
+#pragma unroll
+                                for (int c = 0; c < 8; ++c) {
+                                    dst_k[c0 + c] = rk[c];
+                                    dst_v[c0 + c] = rv[c];
+                                }
+                            }
+                            __threadfence();
+                            asm volatile("fence.proxy.async;" ::: "memory");
                         }
                         ++cur_tile;
                     }
@@ -1125,7 +1176,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         tma_load_2d(dst + S::kTileBytes, &tmap, 0, vrow, fb, stream_policy);
                     }
                     const long long tc2 = trace ? clock64() : 0;
-                    if (with_q) bulk_load(dst + kPairBytes, qsrc, G * D * 2, fb);
+                    if (with_q) {
+                        if (a.dep_wait == 3 && !synced) {  // the query rows are not there yet: fetched at sync_now()
+                            late_dst[n_late] = dst + kPairBytes;
+                            late_src[n_late] = qsrc;
+                            late_bar[n_late++] = fb;
+                        } else {
+                            bulk_load(dst + kPairBytes, qsrc, G * D * 2, fb);
+                        }
+                    }
                     if (trace) {
                         const long long tc3 = clock64();
                         cy_expect += tc1 - tc0;
@@ -1145,6 +1204,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     if (PAGED && seg_left == 0) x += seg_skip;  // the unit's tiles that do not exist
                 }
                 if (!ok) break;
+                if (early && !synced) sync_now();  // a first item shorter than the ring
                 if (PAGED && !asked) mbar_arrive(smem_u32(claim_empty));
                 ok = wait_traced(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout, trace, &ns_claim);
                 cpar ^= 1u;
@@ -1169,9 +1229,14 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         // ------------------------------------------------------------------ claim warp
         if (lane == 0) {
             uint32_t par = 0;
+            bool waited = a.dep_wait != 3;  // dep_wait 3: an earlier launch may still be using the claim counter
             for (;;) {
                 if (!wait_bounded(smem_u32(claim_empty), par, s_abort, a.status, kStatusClaimWaitTimeout)) break;
                 par ^= 1u;
+                if (!waited) {
+                    grid_dep_wait();
+                    waited = true;
+                }
                 // the counter only ever grows; this launch's claims start at claim_base
                 const int k = sc.P + (int)(atomicAdd(a.claim_counter, 1u) - a.claim_base);
                 *claim_slot = k;
@@ -1206,9 +1271,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                   1, et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
             epilogue_sync();
         }
-        if (a.dep_wait == 1) {  // from here on these warps write results, partials and tickets
+        if (a.dep_wait == 1 || a.dep_wait == 3) {  // from here on these warps write results, partials and tickets
             grid_dep_wait();
-            if (et == 0) grid_dep_launch();
+            if (et == 0 && a.dep_wait == 1) grid_dep_launch();
         }
         unsigned long long ns_idle = 0;
         int pend_n = 0;  // partial segments written but without a ticket yet (same value in every epilogue thread)

@@ -91,10 +91,52 @@ __global__ void __launch_bounds__(32, 1) read_stream_kernel(const unsigned char*
     }
 }
 
+// A stand-in for what a model runs between two attention calls (projections, MLP): it streams `n16`
+// 16-byte pieces from src to dst -- work that depends on nothing, like the weights a GEMM reads --,
+// then waits for the kernel before it (when launched to overlap), reads a word of `after` (the
+// attention output it would consume) and copies `produce_n16` pieces to `produce` (the next call's q,
+// k or v), so that those arrive at the very end of the kernel.
+__global__ void __launch_bounds__(256) standin_kernel(uint4* dst, const uint4* src, size_t n16, const float* after,
+                                                       uint4* produce, const uint4* produce_src, size_t produce_n16,
+                                                       int overlap, float* sink)
+{
+    if (overlap) grid_dep_launch();
+    const size_t stride = (size_t)gridDim.x * blockDim.x, first = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (size_t i = first; i < n16; i += stride) dst[i] = __ldcs(src + i);
+    if (overlap) grid_dep_wait();
+    if (after && first == 0) *sink = *reinterpret_cast<const volatile float*>(after);
+    for (size_t i = first; i < produce_n16; i += stride) produce[i] = produce_src[i];
+}
+
+__device__ float g_standin_sink;
+
 }  // namespace
 }  // namespace rlkv
 
 using namespace rlkv;
+
+extern "C" int rlkv_debug_standin(void* dst, const void* src, size_t bytes, const void* after, void* produce,
+                                  const void* produce_src, size_t produce_bytes, int overlap, void* stream)
+{
+    if ((bytes && (!dst || !src)) || (produce_bytes && (!produce || !produce_src)) || bytes % 16 || produce_bytes % 16 ||
+        !aligned16(dst) || !aligned16(src) || !aligned16(produce) || !aligned16(produce_src))
+        return RLKV_EINVAL;
+    float* sink = nullptr;
+    RLKV_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&sink), g_standin_sink));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(148 * 8);
+    cfg.blockDim = dim3(256);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    RLKV_CUDA(cudaLaunchKernelEx(&cfg, standin_kernel, static_cast<uint4*>(dst), static_cast<const uint4*>(src), bytes / 16,
+                                 static_cast<const float*>(after), static_cast<uint4*>(produce),
+                                 static_cast<const uint4*>(produce_src), produce_bytes / 16, overlap ? 1 : 0, sink));
+    return RLKV_OK;
+}
 
 extern "C" int rlkv_debug_read_bandwidth(const void* device_buf, size_t bytes, int launches, float* ms_out)
 {

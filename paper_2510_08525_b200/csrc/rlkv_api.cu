@@ -211,9 +211,10 @@ int make_tensor_map(rlkv_cache* c)
 
 bool valid_layer(const rlkv_cache* c, int layer) { return c && layer >= 0 && layer < c->layers; }
 
-int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s)
+int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, cudaStream_t s, bool overlap = false)
 {
     AppendArgs a;
+    a.overlap = overlap ? 1 : 0;
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
     a.full_row0 = c->lay.full_row0[layer];
     a.comp_row0 = c->lay.comp_row0[layer];
@@ -264,6 +265,9 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     a.group = c->q_heads / c->kv_heads;
     a.q_heads = c->q_heads;
     a.alpha = alpha;
+    a.new_k = a.new_v = nullptr;
+    a.new_sink = c->sink;
+    a.new_window = c->window;
     a.local_sink = n < c->sink ? n : c->sink;
     a.local_sink_tiles = (a.local_sink + kTile - 1) / kTile;
     a.local_win0 = n - c->window > c->sink ? n - c->window : c->sink;  // first token of the window
@@ -304,12 +308,15 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
 // `half`: which half of the scratch memory (partials, claim counter) the launch uses; `overlap` and
 // `dep_wait` as in launch_decode.
 int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s, int half = 0, bool overlap = false,
-              int dep_wait = 0, int* grid_out = nullptr, const float* alpha = nullptr, bool in_step = false)
+              int dep_wait = 0, int* grid_out = nullptr, const float* alpha = nullptr, bool in_step = false,
+              const void* new_k = nullptr, const void* new_v = nullptr)
 {
     DecodeArgs a;
     int grid = 0;
     int rc = build_decode_args(c, layer, q, out, a, &grid, in_step, alpha);
     if (rc) return rc;
+    a.new_k = static_cast<const __nv_bfloat16*>(new_k);  // the launch appends the token itself (len already counts it)
+    a.new_v = static_cast<const __nv_bfloat16*>(new_v);
     if (a.sched.n_slots > c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
     // mixed attention: both units of a head add into `out`
     if (alpha) RLKV_CUDA(cudaMemsetAsync(out, 0, (size_t)c->batch * c->q_heads * c->head_dim * sizeof(float), s));
@@ -347,41 +354,69 @@ Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_most)
     return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0);
 }
 
-// One decode launch for every layer of a step (all layers hold the same number of tokens).  q, out:
+// One decode launch for layers [l0, l1) of a step (all of them hold the same number of tokens).  q, out:
 // the step's [layers][batch][q_heads][head_dim] arrays.  `after_append`: the launch directly follows the
-// step's append launch and may start beside it.
-int do_decode_step(rlkv_cache* c, const void* q, void* out, cudaStream_t s, bool after_append)
+// step's append launch and may start beside it; otherwise it is an ordinary launch.  Launches of this
+// kind never overlap one another, so each uses the whole split-KV scratch.
+int do_decode_step(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStream_t s, bool after_append)
 {
-    const int n = c->len[0];
+    const int n = c->len[l0];
     const int cap = c->sink + c->window;
     DecodeArgs a;
     memset(&a, 0, sizeof a);
     a.pool = dev_at<__nv_bfloat16>(c, c->lay.off_pool);
-    a.q = static_cast<const __nv_bfloat16*>(q);
-    a.out = static_cast<float*>(out);
+    const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
+    a.q = static_cast<const __nv_bfloat16*>(q) + l0 * q_layer;
+    a.out = reinterpret_cast<float*>(static_cast<uint8_t*>(out) + l0 * q_layer * (c->out_bf16 ? 2 : 4));
     a.status = dev_at<int>(c, c->lay.off_status);
     a.trace = dev_at<unsigned long long>(c, c->lay.off_trace);
     a.rows_full = c->lay.rows_full;
     a.rows_comp = c->lay.rows_comp;
     a.len_full = n;
     a.len_comp = n < cap ? n : cap;
-    a.batch = c->batch * c->layers;
+    a.batch = c->batch * (l1 - l0);
     a.group = c->q_heads / c->kv_heads;
     a.q_heads = c->q_heads;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)c->head_dim);
     a.trace_on = c->trace_on;
     a.out_bf16 = c->out_bf16;
-    const StepArgs& st = c->step_args;
-    const int U = st.full_base[c->layers], Uc = st.comp_base[c->layers];
+    StepArgs part;                      // the tables of layers l0 .. l1-1, units counted from the first of them
+    const StepArgs* stp = &c->step_args;
+    if (l0 != 0 || l1 != c->layers) {
+        const StepArgs& all = c->step_args;
+        memset(&part, 0, sizeof part);
+        part.head_of_slot = all.head_of_slot + (size_t)l0 * c->kv_heads;
+        part.n_layers = l1 - l0;
+        part.kv_heads = all.kv_heads;
+        part.batch = all.batch;
+        for (int l = l0; l <= l1; ++l) {
+            part.full_base[l - l0] = all.full_base[l] - all.full_base[l0];
+            part.comp_base[l - l0] = all.comp_base[l] - all.comp_base[l0];
+            if (l < l1) {
+                part.full_row0[l - l0] = all.full_row0[l];
+                part.comp_row0[l - l0] = all.comp_row0[l];
+            }
+        }
+        stp = &part;
+    }
+    const StepArgs& st = *stp;
+    const int U = st.full_base[l1 - l0], Uc = st.comp_base[l1 - l0];
     const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
     if ((long long)U * tiles_full + (long long)Uc * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
     int grid = c->sm_count * c->ctas_per_sm;
     if (grid > c->lay.max_grid) grid = c->lay.max_grid;
-    a.sched = step_schedule(U, tiles_full, Uc, tiles_comp, grid, c->item_tiles);
+    // the scratch is sized for items of kDefaultItemTiles tiles once the step is large: a smaller setting
+    // (rlkv_set_decode_config) is raised until the partial records fit
+    int item_most = c->item_tiles;
+    a.sched = step_schedule(U, tiles_full, Uc, tiles_comp, grid, item_most);
+    while (a.sched.n_slots > 2 * c->lay.max_items && item_most < kDefaultItemTiles) {
+        item_most = item_most * 2 < kDefaultItemTiles ? item_most * 2 : kDefaultItemTiles;
+        a.sched = step_schedule(U, tiles_full, Uc, tiles_comp, grid, item_most);
+    }
     if (grid > a.sched.n_items) grid = a.sched.n_items;
     if (a.sched.n_slots > 2 * c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
     a.partials = dev_at<float>(c, c->lay.off_partials);                // both halves as one
-    a.tickets = dev_at<int>(c, c->lay.off_tickets);                    // one per unit of the step
+    a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)l0 * 2 * c->batch * c->kv_heads;  // one per unit of the launch
     a.claim_counter = dev_at<unsigned int>(c, c->lay.off_status) + 4;
     a.claim_base = c->claims[0];
     a.dep_wait = after_append ? 1 : 0;
@@ -732,6 +767,37 @@ int rlkv_decode_attention(rlkv_cache* c, int layer, const void* q, void* out, vo
     return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream));
 }
 
+int rlkv_append_overlapped(rlkv_cache* c, int layer, const void* k, const void* v, void* stream)
+{
+    if (!valid_layer(c, layer) || !k || !v || !aligned16(k) || !aligned16(v)) return RLKV_EINVAL;
+    if (c->len[layer] + 1 > c->max_len) return RLKV_EFULL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_append(c, layer, k, v, 1, static_cast<cudaStream_t>(stream), true);
+}
+
+int rlkv_decode_attention_overlapped(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (c->len[layer] < 1) return RLKV_EEMPTY;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream), 0, true, 3);
+}
+
+int rlkv_layer_step_overlapped(rlkv_cache* c, int layer, const void* k, const void* v, const void* q, void* out, void* stream)
+{
+    if (!valid_layer(c, layer) || !k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out))
+        return RLKV_EINVAL;
+    if (c->len[layer] + 1 > c->max_len) return RLKV_EFULL;
+    DeviceGuard g(c->device);
+    if (!g.ok) return RLKV_ECUDA;
+    c->len[layer] += 1;  // the launch writes the token's rows itself, each by the CTA that reads them
+    const int rc = do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream), 0, true, 3, nullptr, nullptr, false, k, v);
+    if (rc) c->len[layer] -= 1;
+    return rc;
+}
+
 int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
 {
     if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
@@ -785,7 +851,7 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
         const bool one_launch = step_uses_one_launch(c);  // asked before the append moves the lengths
         int rc = step_append(c, k, v, s);
         if (rc) return rc;
-        if (one_launch) return do_decode_step(c, q, out, s, true);
+        if (one_launch) return do_decode_step(c, 0, c->layers, q, out, s, true);
         return step_decode(c, 0, c->layers, q, out, s, false);
     }
     for (int l = 0; l < c->layers; ++l) {
@@ -849,13 +915,16 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
                                   c->in_stream));
         RLKV_CUDA(cudaEventRecord(c->ev_in[i], c->in_stream));
     }
-    // kernels
+    // kernels: per chunk of layers one attention launch over all its layers where the step allows it,
+    // else one launch per layer
     RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_in[0], 0));
+    const bool one_launch = step_uses_one_launch(c);
     int rc = step_append(c, dk, dv, s);
     if (rc) return rc;
     for (int i = 0; i < chunks; ++i) {
         if (i > 0) RLKV_CUDA(cudaStreamWaitEvent(s, c->ev_in[i], 0));
-        rc = step_decode(c, bounds[i], bounds[i + 1], dq, dout, s, i > 0);
+        rc = one_launch ? do_decode_step(c, bounds[i], bounds[i + 1], dq, dout, s, i == 0)
+                        : step_decode(c, bounds[i], bounds[i + 1], dq, dout, s, i > 0);
         if (rc) return rc;
         RLKV_CUDA(cudaEventRecord(c->ev_out[i], s));
         // results of the chunk

@@ -282,6 +282,12 @@ struct DecodeArgs {
     // the same rows restricted to the sink and the window: tiles 0 .. local_sink_tiles-1 cover rows
     // [0, local_sink), the tiles after them rows [local_win0, local_win0 + local_win_len).  Both
     // units add their weighted result into `out`, which the host clears before the launch.
+    // A launch that also appends the step's token (lock-step cache, one layer): the caller's new rows,
+    // [batch][kv_heads][head_dim]; token len_full - 1 of every head is written by the CTA that reads the
+    // tile it belongs to (row len_full - 1 of a full head, the ring slot of a compressed head).  Null otherwise.
+    const __nv_bfloat16* new_k;
+    const __nv_bfloat16* new_v;
+    int new_sink, new_window;
     const float* alpha;         // gates of the layer's KV heads (device, [kv_heads]); null otherwise
     int local_sink, local_sink_tiles, local_win0, local_win_len;
     Schedule sched;
@@ -341,6 +347,7 @@ struct AppendArgs {
     int batch, kv_heads, head_dim;
     int t0, n_tokens;           // tokens t0 .. t0+n_tokens-1 are appended
     int sink, window;
+    int overlap;                // the launch may start before the kernel before it has completed: wait for it first
 };
 
 // What producer and consumers need to know about the unit behind a flat tile.

@@ -543,6 +543,57 @@ def test_one_launch_step_against_launch_per_layer_and_oracle(rl, hz, cuda_device
         b.close()
 
 
+@pytest.mark.parametrize("one_launch", [0, 1], ids=["append_then_attend", "layer_step"])
+@pytest.mark.parametrize("overlap", [1, 0], ids=["neighbours_overlap", "ordinary_neighbours"])
+@pytest.mark.parametrize("shape", [(4, 4, 16, 128, 8, 16, 48, 3000), (3, 2, 8, 64, 2, 4, 60, 100), (2, 8, 32, 128, 16, 16, 112, 1500),
+                                   (2, 2, 4, 128, 3, 130, 62, 190)],
+                         ids=["many_items", "shorter_than_the_ring", "wide", "ring_just_filling"])
+def test_overlapped_per_layer_calls_wait_for_their_inputs(rl, hz, cuda_device, shape, overlap, one_launch):
+    """The chain of a model forward: before every layer's attention a stand-in kernel copies that layer's
+    k, v and q into the buffers the calls read -- at the very end of the kernel -- and
+    rlkv_append_overlapped / rlkv_decode_attention_overlapped are launched right behind it so that they
+    may start while it still runs.  Until the stand-in has finished, the buffers hold the previous
+    layer's values: a call that read its inputs too early would append wrong rows (the state check is
+    bit for bit) or attend with the wrong query.  Six steps over all layers, outputs against the
+    oracle at every step, the state at the end; the same with ordinary launches around the calls, and
+    with rlkv_layer_step_overlapped, whose one launch writes the token's rows itself."""
+    layers, Hkv, Hq, D, B, S, W, n = shape
+    mask = synth.head_mask(77, layers, Hkv, 0.4)
+    cache, oracle = build_pair(hz, layers, Hkv, Hq, D, B, n + 8, mask, S, W, cuda_device)
+    for l in range(layers):
+        feed(cache, oracle, l, rand_bf16((n, B, Hkv, D), 900 + l), rand_bf16((n, B, Hkv, D), 910 + l), True)
+    kv_elems, q_elems = B * Hkv * D, B * Hq * D
+    buf = torch.zeros(2 * kv_elems + q_elems, dtype=torch.bfloat16, device=cuda_device)   # k | v | q of the current layer
+    kb, vb, qb = buf[:kv_elems], buf[kv_elems:2 * kv_elems], buf[2 * kv_elems:]
+    work_src = torch.ones(32 << 20, dtype=torch.uint8, device=cuda_device)                # the stand-in's own traffic
+    work_dst = torch.empty_like(work_src)
+    out = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
+    for t in range(6):
+        K, V, Q = rand_bf16((layers, B, Hkv, D), 920 + t), rand_bf16((layers, B, Hkv, D), 930 + t), rand_bf16((layers, B, Hq, D), 940 + t)
+        src = [torch.cat([K[l].reshape(-1), V[l].reshape(-1), Q[l].reshape(-1)]).to(cuda_device) for l in range(layers)]
+        torch.cuda.synchronize()
+        for l in range(layers):
+            rl.rlkv_debug_standin(work_dst, work_src, work_src.numel(), out[l - 1] if l else None, buf, src[l],
+                                  buf.numel() * 2, overlap)
+            if one_launch:
+                rl.rlkv_layer_step_overlapped(cache.handle, l, kb, vb, qb, out[l])
+            else:
+                rl.rlkv_append_overlapped(cache.handle, l, kb, vb)
+                rl.rlkv_decode_attention_overlapped(cache.handle, l, qb, out[l])
+        torch.cuda.synchronize()
+        got = out.cpu().numpy()
+        for l in range(layers):
+            assert oracle.append(l, K[l], V[l]) == 0
+            check_out(got[l], oracle.decode(l, Q[l]))
+    check_state(cache, oracle)
+    # the overlapped call and the ordinary one cut the work alike: the same bits
+    ref = cache.decode(0, qb)
+    again = torch.empty_like(ref)
+    rl.rlkv_decode_attention_overlapped(cache.handle, 0, qb, again)
+    assert torch.equal(ref, again)
+    assert cache.status() == 0
+
+
 def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):
     """Nine layers, so that rlkv_step_host brings inputs in and takes results out in chunks on its side
     streams, and consecutive calls alternate between its two input staging areas: five steps in a row
@@ -566,7 +617,7 @@ def test_step_host_in_chunks_over_several_steps(rl, hz, cuda_device):
         k, v, q = (x.to(cuda_device) for x in ins[t])
         ref = torch.empty((layers, B, Hq, D), dtype=torch.float32, device=cuda_device)
         rl.rlkv_step(b.handle, k, v, q, ref)
-        assert torch.allclose(ref.cpu(), outs[t], atol=1e-4, rtol=0)
+        assert torch.allclose(ref.cpu(), outs[t], atol=5e-4, rtol=0)   # cut differently: rounding noise only
         for l in range(layers):
             oracle.append(l, ins[t][0][l], ins[t][1][l])
             check_out(outs[t][l].numpy(), oracle.decode(l, ins[t][2][l]))
