@@ -828,11 +828,12 @@ def run_ours(args, w, mask):
     # a quarter to seven quarters of it (same total), launches cycling through the layers
     paged = None
     if not args.no_paged and world == 1:
-        pl, reps = min(4, w.layers), max(K, 8)
+        pl, reps = w.layers, max(K, 8)
         n = w.context + 1
         pmask = mask[:pl * w.kv_heads]
         spread = [max(1, int(round(n * (0.25 + 1.5 * i / max(1, w.batch - 1))))) for i in range(w.batch)]
-        paged = {"workload": f"first {pl} layers of the {w.name} mask, {w.batch} sequences, launches back to back"}
+        paged = {"workload": f"the {pl} layers of the {w.name} mask, {w.batch} sequences; launch_us: rlkv_paged_decode_attention "
+                             f"launches back to back; in_step: rlkv_paged_step (one append launch, one attention launch over all layers)"}
         variants = [("uniform", [n] * w.batch, False), ("ragged", spread, False)]
         if w.head_dim == 128:
             variants.append(("uniform_fp8", [n] * w.batch, True))   # every K/V row as an E4M3 code
@@ -852,18 +853,19 @@ def run_ours(args, w, mask):
                                    vv.reshape(t1 - t0, w.kv_heads, w.head_dim))
             q = q0
             pout = torch.empty((pl, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
-            for i in range(2 * pl):
+            lreps = max(2, (reps * 4) // pl)
+            for i in range(pl):
                 rl.rlkv_paged_decode_attention(pc.handle, i % pl, slots, q[i % pl], pout[i % pl], stream)
             torch.cuda.synchronize()
             e0.record(stream)
-            for i in range(reps * pl):
+            for i in range(lreps * pl):
                 rl.rlkv_paged_decode_attention(pc.handle, i % pl, slots, q[i % pl], pout[i % pl], stream)
             e1.record(stream)
             torch.cuda.synchronize()
-            us = 1e3 * e0.elapsed_time(e1) / (reps * pl)
+            us = 1e3 * e0.elapsed_time(e1) / (lreps * pl)
             nbytes = sum(pc.step_bytes(l, slots) for l in range(pl)) / pl
             paged[name] = {"launch_us": us, "algorithmic_bytes_per_launch": nbytes, "achieved_gbs": nbytes / (us * 1e-6) / 1e9,
-                           "lengths": [min(lens), max(lens)], "launches_timed": reps * pl}
+                           "lengths": [min(lens), max(lens)], "launches_timed": lreps * pl}
             # the same layers through rlkv_paged_step (one token appended per step, launches overlapped)
             kk, vv = kv0[0][:pl].contiguous(), kv0[1][:pl].contiguous()
             qq = q[:pl].contiguous()

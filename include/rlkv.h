@@ -279,11 +279,17 @@ int rlkv_paged_decode_attention(rlkv_paged* cache, int layer, const int* slots, 
  * second dimension belongs to slots[i] (HOST int[n]).  Results are those of rlkv_paged_append and
  * rlkv_paged_decode_attention layer by layer (up to floating-point summation order).  As in rlkv_step
  * all inputs are there before the first launch, so the step is one append launch for all layers and
- * the layers' attention launches, overlapped on the device; the buffers must be complete at the call
+ * one attention launch over the K/V rows of every layer (or the layers' attention launches, overlapped
+ * on the device: see rlkv_paged_set_step_mode); the buffers must be complete at the call
  * and stay untouched until the work on `stream` has finished.  Every listed sequence must have the
  * same length in all layers (RLKV_EINVAL otherwise); RLKV_EFULL as for rlkv_paged_append. */
 int rlkv_paged_step(rlkv_paged* cache, const int* slots, int n, const void* k, const void* v,
                     const void* q, void* out, void* stream);
+/* As rlkv_set_step_mode, for rlkv_paged_step: 0 (the default) one attention launch over the K/V rows
+ * of every layer where the step's split-KV records fit the scratch (else one launch per layer), 1
+ * always one launch per layer, 2 as 0 (RLKV_EINVAL if the shape has more than 128 layers or 4096
+ * (layer, KV head) pairs). */
+int rlkv_paged_set_step_mode(rlkv_paged* cache, int mode);
 /* As rlkv_set_output_bf16, for rlkv_paged_decode_attention and rlkv_paged_step. */
 int rlkv_paged_set_output_bf16(rlkv_paged* cache, int on);
 int rlkv_paged_length(const rlkv_paged* cache, int layer, int slot, int* len_out);

@@ -37,6 +37,7 @@ SIGNATURES = {
     "rlkv_static_scratch_bytes": (_sz, []),
     "rlkv_set_output_bf16": (_ci, [_vp, _ci]),
     "rlkv_paged_set_output_bf16": (_ci, [_vp, _ci]),
+    "rlkv_paged_set_step_mode": (_ci, [_vp, _ci]),
     "rlkv_decode_mixed_attention": (_ci, [_vp, _ci, _vp, _vp, _vp, _vp]),
     "rlkv_step": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "rlkv_step_host": (_ci, [_vp, _vp, _vp, _vp, _vp, _vp]),
@@ -203,6 +204,10 @@ def rlkv_decode_mixed_attention(cache, layer, q, alpha, out, stream=None) -> Non
 
 def rlkv_set_output_bf16(cache, on) -> None:
     _check(lib.rlkv_set_output_bf16(cache, int(bool(on))))
+
+
+def rlkv_paged_set_step_mode(cache, mode) -> None:
+    _check(lib.rlkv_paged_set_step_mode(cache, int(mode)))
 
 
 def rlkv_paged_set_output_bf16(cache, on) -> None:

@@ -28,6 +28,7 @@
 // rows looked up in a page table; also with 8-bit pages), and the whole decode step in one launch
 // (the units of every layer in one flat tile space); see the notes above decode_kernel.
 #include <cuda_fp16.h>
+#include <stddef.h>
 
 #include "rlkv_internal.cuh"
 
@@ -272,7 +273,7 @@ struct Smem {
         return merge_floats(group) * 4 + kStatFloats * 4 + 32;
     }
     // paged cache only: the page-table entries of the segment being streamed, the PagedArgs
-    static constexpr int kPagedBytes = (kMaxSeqPages + 4) * 4 + (int)((sizeof(PagedArgs) + 15) / 16 * 16);
+    static constexpr int kPagedBytes = (kMaxSeqPages + 4) * 4 + (int)((sizeof(PagedArgs) + 15) / 16 * 16) + kMaxStepHeads;
     // whole-step launches only: the StepArgs and the KV head of every slot of every layer
     static constexpr int kStepBytes = (int)((sizeof(StepArgs) + 15) / 16 * 16) + kMaxStepHeads;
     __host__ __device__ static constexpr size_t bytes(int stages, int group, int mode = kModePlain)
@@ -476,7 +477,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     const PagedArgs* pg = PAGED ? s_paged : nullptr;
     // whole-step launch: the layer tables and the KV head of every slot, at the same place
     const StepArgs* stp = STEP ? reinterpret_cast<const StepArgs*>(s_paged) : nullptr;
-    unsigned char* s_heads = reinterpret_cast<unsigned char*>(s_paged) + (sizeof(StepArgs) + 15) / 16 * 16;
+    unsigned char* s_heads = PAGED ? reinterpret_cast<unsigned char*>(s_pages + kMaxSeqPages + 4)
+                                   : reinterpret_cast<unsigned char*>(s_paged) + (sizeof(StepArgs) + 15) / 16 * 16;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const Schedule& sc = a.sched;
@@ -506,12 +508,45 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     }
     for (int i = tid; i < (int)(sizeof(DecodeArgs) / sizeof(int)); i += blockDim.x)
         reinterpret_cast<int*>(s_args)[i] = reinterpret_cast<const int*>(&args)[i];
-    if (PAGED)
-        for (int i = tid; i < (int)(sizeof(PagedArgs) / sizeof(int)); i += blockDim.x)
-            reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+    if constexpr (PAGED) {
+        // only what the launch uses: reading kernel parameters with a per-thread index is slow, and the
+        // per-sequence and per-layer arrays are sized for 512 sequences and 128 layers
+        const PagedArgs& ex = *reinterpret_cast<const PagedArgs*>(&extra);
+        const bool whole = ex.step.n_layers > 1;
+        const int n_seq = whole ? ex.step.batch : args.batch;
+        auto copy_ints = [&](size_t first_byte, size_t end_byte) {
+            for (int i = (int)(first_byte / 4) + tid; i < (int)((end_byte + 3) / 4); i += blockDim.x)
+                reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+        };
+        copy_ints(0, offsetof(PagedArgs, seq_len) + (size_t)n_seq * sizeof(int));
+        copy_ints(offsetof(PagedArgs, seq_slot), offsetof(PagedArgs, seq_slot) + (size_t)n_seq * sizeof(unsigned short));
+        copy_ints(offsetof(PagedArgs, step), offsetof(PagedArgs, step) + offsetof(StepArgs, full_base));
+        if (whole) {
+            const size_t L = (size_t)ex.step.n_layers;
+            const size_t st = offsetof(PagedArgs, step);
+            copy_ints(st + offsetof(StepArgs, full_base), st + offsetof(StepArgs, full_base) + (L + 1) * 4);
+            copy_ints(st + offsetof(StepArgs, comp_base), st + offsetof(StepArgs, comp_base) + (L + 1) * 4);
+            copy_ints(st + offsetof(StepArgs, full_row0), st + offsetof(StepArgs, full_row0) + L * 4);
+            copy_ints(st + offsetof(StepArgs, comp_row0), st + offsetof(StepArgs, comp_row0) + L * 4);
+            copy_ints(offsetof(PagedArgs, scales), offsetof(PagedArgs, scales) + sizeof(const float*));
+            copy_ints(offsetof(PagedArgs, page0_8_of), offsetof(PagedArgs, page0_8_of) + L * 4);
+            copy_ints(offsetof(PagedArgs, ring0_8_of), offsetof(PagedArgs, ring0_8_of) + L * 4);
+            // the KV head of every slot of every layer (written at cache creation)
+            for (int i = tid; i < ex.step.n_layers * ex.step.kv_heads; i += blockDim.x)
+                s_heads[i] = (unsigned char)__ldg(ex.step.head_of_slot + i);
+        }
+    }
     if constexpr (STEP) {
-        for (int i = tid; i < (int)(sizeof(StepArgs) / sizeof(int)); i += blockDim.x)
-            reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+        // (the per-layer arrays are sized for 128 layers: only the layers of the launch are copied)
+        const int L = extra.n_layers;
+        auto copy_ints = [&](size_t first_byte, size_t end_byte) {
+            for (int i = (int)(first_byte / 4) + tid; i < (int)((end_byte + 3) / 4); i += blockDim.x)
+                reinterpret_cast<int*>(s_paged)[i] = reinterpret_cast<const int*>(&extra)[i];
+        };
+        copy_ints(0, offsetof(StepArgs, full_base) + (size_t)(L + 1) * 4);
+        copy_ints(offsetof(StepArgs, comp_base), offsetof(StepArgs, comp_base) + (size_t)(L + 1) * 4);
+        copy_ints(offsetof(StepArgs, full_row0), offsetof(StepArgs, full_row0) + (size_t)L * 4);
+        copy_ints(offsetof(StepArgs, comp_row0), offsetof(StepArgs, comp_row0) + (size_t)L * 4);
         for (int i = tid; i < extra.n_layers * extra.kv_heads; i += blockDim.x)  // written at cache creation
             s_heads[i] = (unsigned char)__ldg(extra.head_of_slot + i);
     }
@@ -670,7 +705,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             // this lane ends up with four consecutive tokens
                             const int ktok = wig * 16 + 4 * (li >> 1) + 2 * (lj & 1) + (li & 1);
                             const uint32_t stage0 = smem_u32(stage_base + (size_t)st * stage_bytes);
-                            const float sl2 = a.scale_log2 * pg->k_scale[u.head];  // K's scale joins the softmax scale
+                            // K's scale joins the softmax scale
+                            const float sl2 = a.scale_log2 * (pg->step.n_layers > 1 ? __ldg(pg->scales + u.layer * pg->step.kv_heads + u.head)
+                                                                                    : pg->k_scale[u.head]);
                             // scores of this lane per tile: [0], [1] token row `quad` of set A, heads 2tq and 2tq+1;
                             // [2], [3] token row `quad` of set B, the same heads
                             float sc8[2][4];
@@ -852,7 +889,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 float* stat_m = merge + S::merge_floats(G);
                 float* stat_l = stat_m + S::kWarps * kMaxGroup;
                 if (FP8 && item >= 0) {  // the rows were value(code): V's scale goes in here
-                    const float vs = pg->v_scale[u.head];
+                    const float vs = pg->step.n_layers > 1
+                                         ? __ldg(pg->scales + (pg->step.n_layers + u.layer) * pg->step.kv_heads + u.head)
+                                         : pg->v_scale[u.head];
 #pragma unroll
                     for (int mt = 0; mt < KS; ++mt) {
                         acc[mt][0] *= vs;
@@ -902,7 +941,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     // the whole unit (paged cache: all of its tiles that exist) in one segment
                     const bool complete = u.pos.tile == 0 && (PAGED ? seg_tiles >= (u.len + kTile - 1) / kTile
                                                                     : seg_tiles == u.tiles);
-                    sd->out_row = u.b * a.q_heads + u.head * G;
+                    sd->out_row = u.qrow * a.q_heads + u.head * G;
                     sd->uid = u.pos.uid;
                     sd->complete = complete ? 1 : 0;
                     sd->pslot = item < 0 ? 0 : partial_slot(sc, u.pos.band, item, u.pos.uid);
@@ -1057,20 +1096,24 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 ppar ^= 1u;
                                 page_base = first;
                                 // 16-bit pages: the first pool row of the head's pages; 8-bit pages: its first page
-                                paged_row0 = FP8 ? pg->page0_8 + (u.pos.uid - u.b * a.n_full) * pg->n_pages
-                                                 : (int)(a.full_row0 + (long long)(u.pos.uid - u.b * a.n_full) * pg->n_pages * 2 * kTile);
+                                const bool whole = pg->step.n_layers > 1;  // per-layer values come per layer
+                                paged_row0 = FP8 ? (whole ? pg->page0_8_of[u.layer] : pg->page0_8) + u.slot * pg->n_pages
+                                                 : (whole ? pg->step.full_row0[u.layer] : (int)a.full_row0) +
+                                                       u.slot * pg->n_pages * 2 * kTile;
                             } else {
                                 paged_row0 = -1;
-                                const int c = u.pos.uid - sc.U - u.b * a.n_comp;
+                                const bool whole = pg->step.n_layers > 1;
+                                const int c = u.slot;
                                 if (FP8) {  // the ring's pages follow one another
-                                    ring_next = pg->ring0_8 + (pg->seq_slot[u.b] * a.n_comp + c) * pg->ring_tiles + u.pos.tile;
+                                    ring_next = (whole ? pg->ring0_8_of[u.layer] : pg->ring0_8) +
+                                                (pg->seq_slot[u.b] * u.nclass + c) * pg->ring_tiles + u.pos.tile;
                                 } else {
-                                    krow = (int)(a.comp_row0 + ((long long)pg->seq_slot[u.b] * a.n_comp + c) * 2 * a.rows_comp) +
-                                           u.pos.tile * kTile;
+                                    krow = (whole ? pg->step.comp_row0[u.layer] : (int)a.comp_row0) +
+                                           (pg->seq_slot[u.b] * u.nclass + c) * 2 * a.rows_comp + u.pos.tile * kTile;
                                     vrow = krow + a.rows_comp;
                                 }
                             }
-                            qsrc = a.q + ((size_t)u.b * a.q_heads + (size_t)u.head * G) * D;
+                            qsrc = a.q + ((size_t)u.qrow * a.q_heads + (size_t)u.head * G) * D;
                         } else {
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit (waited for when that tile's turn comes, below).

@@ -46,7 +46,6 @@ struct Layout {
     bool step_in_one_launch = false;  // the shape allows rlkv_step to serve all layers with one decode launch
 };
 
-constexpr int kDefaultItemTiles = 32;        // launches of rlkv_step, which overlap: coarse items, few partials
 constexpr int kDefaultItemTilesAlone = 8;    // a launch on its own: finer items for an even finish
 constexpr int kMaxFanIn = 32;                // most pieces a full unit is cut into when the schedule has no bands
 
@@ -331,27 +330,6 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     if (grid_out) *grid_out = grid;
     c->launches++;
     return RLKV_OK;
-}
-
-// The schedule of a whole step in one launch: U full units of tf tiles and Uc compressed units of tc
-// tiles over all layers, for `grid` CTAs.  Two thirds of the full units go to the whole-unit prefix
-// (one static item per CTA, units streamed in one piece), as long as what remains still gives every
-// CTA a few items to claim, so that CTAs on a slower path to memory end together with the others.
-Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_most)
-{
-    const long long all_tiles = (long long)U * tf + (long long)Uc * tc;
-    int item_tiles = (int)(all_tiles / grid);
-    if (item_tiles > item_most) item_tiles = item_most;
-    if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
-    int U0 = 0;
-    if (U > 0) {
-        const long long rest_wanted = 4ll * grid * item_tiles;  // tiles left to the claimed items
-        long long most = U - (rest_wanted - (long long)Uc * tc + tf - 1) / tf;
-        if (most > U) most = U;
-        U0 = (int)(2ll * U / 3);
-        if (U0 > most) U0 = most > 0 ? (int)most : 0;
-    }
-    return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0);
 }
 
 // One decode launch for layers [l0, l1) of a step (all of them hold the same number of tokens).  q, out:

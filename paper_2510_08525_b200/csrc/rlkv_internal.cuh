@@ -294,6 +294,19 @@ struct DecodeArgs {
     unsigned char head_of_slot[kMaxKvHeads];  // KV head of full slot 0..n_full-1, then of the compressed slots
 };
 
+// A whole decode step in one launch (kModeStep kernels): what DecodeArgs cannot say.  Every layer holds
+// the same number of tokens.  The full units of all layers form one list, layer after layer (inside a
+// layer: batch row, then full-head slot), and so do the compressed units; q and out are the step's
+// [layers][batch][q_heads][head_dim] arrays, so "batch row" l * batch + b addresses them directly.
+struct StepArgs {
+    const int* head_of_slot;            // device, int [n_layers][kv_heads]: KV head of each slot (full slots first)
+    int n_layers, kv_heads, batch;
+    int full_base[kMaxStepLayers + 1];  // first full unit of layer l = batch * (full heads of the layers before it)
+    int comp_base[kMaxStepLayers + 1];  // first compressed unit of layer l, counted from the first compressed unit
+    int full_row0[kMaxStepLayers];      // first pool row of the layer's full-head / compressed-head region
+    int comp_row0[kMaxStepLayers];
+};
+
 // Paged cache (kModePaged kernels): what DecodeArgs cannot say.  The launch serves `batch` sequences;
 // entry b of q and out belongs to request slot seq_slot[b], which holds seq_len[b] tokens in this
 // layer.  Units are laid out as for the lock-step cache with every full unit given the tiles of the
@@ -316,25 +329,21 @@ struct PagedArgs {
     float k_scale[kMaxKvHeads], v_scale[kMaxKvHeads];
     int seq_len[kMaxPagedBatch];
     unsigned short seq_slot[kMaxPagedBatch];
+    // A whole step in one launch (step.n_layers > 1; every listed sequence holds the same number of tokens
+    // in all layers): the units of all layers form one list as for the lock-step cache (StepArgs, with
+    // `batch` = sequences of the call), q and out are [layers][batch][q_heads][head_dim], and what the
+    // fields above and DecodeArgs say per layer comes per layer: the regions' first pool rows from
+    // `step`, the first 8-bit pages from these arrays, the scales from device memory (k_scale
+    // [layers][kv_heads], then v_scale).  step.n_layers <= 1: a launch for one layer, these are unused.
+    StepArgs step;
+    const float* scales;
+    int page0_8_of[kMaxStepLayers], ring0_8_of[kMaxStepLayers];
 };
 // The tensor map over the 8-bit pool: rows of 128 bytes, boxes of 128 rows = one page (64 rows of K
 // codes, then the transposed V codes, two d per row).
 struct alignas(64) PagedFp8Args {
     PagedArgs pa;
     alignas(64) CUtensorMap map_k;
-};
-
-// A whole decode step in one launch (kModeStep kernels): what DecodeArgs cannot say.  Every layer holds
-// the same number of tokens.  The full units of all layers form one list, layer after layer (inside a
-// layer: batch row, then full-head slot), and so do the compressed units; q and out are the step's
-// [layers][batch][q_heads][head_dim] arrays, so "batch row" l * batch + b addresses them directly.
-struct StepArgs {
-    const int* head_of_slot;            // device, int [n_layers][kv_heads]: KV head of each slot (full slots first)
-    int n_layers, kv_heads, batch;
-    int full_base[kMaxStepLayers + 1];  // first full unit of layer l = batch * (full heads of the layers before it)
-    int comp_base[kMaxStepLayers + 1];  // first compressed unit of layer l, counted from the first compressed unit
-    int full_row0[kMaxStepLayers];      // first pool row of the layer's full-head / compressed-head region
-    int comp_row0[kMaxStepLayers];
 };
 
 struct AppendArgs {
@@ -355,9 +364,13 @@ struct UnitInfo {
     TilePos pos;
     int tiles;       // tiles of the unit
     int len;         // valid rows of the unit
-    int b, head;     // batch row (whole-step launch: layer * batch + batch row), KV head
+    int b, head;     // batch row (whole-step launch of the lock-step cache: layer * batch + batch row), KV head
+    int qrow;        // the unit's G query (and output) rows start at row qrow * q_heads + head * G
     int row0;        // lock-step cache: first pool row of the unit's K rows; its V rows start `vrows` further on
     int vrows;
+    int layer;       // paged cache: the layer (0 in a launch for one layer), the unit's slot among the heads of
+    int slot;        // its class in that layer, and how many heads of that class the layer has
+    int nclass;
 };
 
 // The layer a unit of a whole-step launch belongs to: the last l with base[l] <= unit.
@@ -383,6 +396,28 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
     u.pos = tile_pos(a.sched, x);
     u.row0 = 0;
     u.vrows = 0;
+    u.layer = 0;
+    u.slot = 0;
+    u.nclass = 0;
+    if ((MODE == kModePaged || MODE == kModePagedFp8) && pg->step.n_layers > 1) {  // the paged cache, a whole step
+        const StepArgs* ps = &pg->step;
+        const bool full = u.pos.uid < a.sched.U;
+        const int unit = full ? u.pos.uid : u.pos.uid - a.sched.U;
+        const int* base = full ? ps->full_base : ps->comp_base;
+        const int l = step_layer(base, ps->n_layers, unit);
+        const int local = unit - base[l];
+        const int nf = (ps->full_base[l + 1] - ps->full_base[l]) / ps->batch;
+        u.nclass = full ? nf : ps->kv_heads - nf;
+        u.b = local / u.nclass;
+        u.slot = local - u.b * u.nclass;
+        u.layer = l;
+        u.qrow = l * ps->batch + u.b;
+        u.tiles = full ? a.sched.tf : a.sched.tc;
+        u.head = heads[l * ps->kv_heads + (full ? u.slot : nf + u.slot)];
+        const int n = pg->seq_len[u.b];
+        u.len = full ? n : (n < pg->cap ? n : pg->cap);
+        return u;
+    }
     if (MODE == kModeStep) {
         const bool full = u.pos.uid < a.sched.U;
         const int unit = full ? u.pos.uid : u.pos.uid - a.sched.U;
@@ -395,6 +430,7 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.tiles = full ? a.sched.tf : a.sched.tc;
         u.len = full ? a.len_full : a.len_comp;
         u.b = l * st->batch + b;
+        u.qrow = u.b;
         u.head = heads[l * st->kv_heads + (full ? slot : nf + slot)];
         u.vrows = full ? a.rows_full : a.rows_comp;
         u.row0 = (full ? st->full_row0[l] : st->comp_row0[l]) + local * 2 * u.vrows;
@@ -424,9 +460,13 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.vrows = a.rows_comp;
         u.row0 = (int)(a.comp_row0 + (long long)unit * 2 * a.rows_comp);
     }
+    u.qrow = u.b;
     if (MODE == kModePaged || MODE == kModePagedFp8) {  // this sequence's own length
         const int n = pg->seq_len[u.b];
-        u.len = u.pos.uid < a.sched.U ? n : (n < pg->cap ? n : pg->cap);
+        const bool full = u.pos.uid < a.sched.U;
+        u.len = full ? n : (n < pg->cap ? n : pg->cap);
+        u.nclass = full ? a.n_full : a.n_comp;
+        u.slot = full ? u.pos.uid - u.b * a.n_full : u.pos.uid - a.sched.U - u.b * a.n_comp;
     }
     return u;
 }
@@ -434,13 +474,20 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
 // Paged cache: how many tiles of unit `uid` exist.
 __device__ inline int paged_unit_tiles(const DecodeArgs& a, const PagedArgs* pg, int uid)
 {
-    int n;
-    if (uid < a.sched.U) {
-        n = pg->seq_len[uid / a.n_full];
+    const bool full = uid < a.sched.U;
+    int b;
+    if (pg->step.n_layers > 1) {
+        const StepArgs* ps = &pg->step;
+        const int unit = full ? uid : uid - a.sched.U;
+        const int* base = full ? ps->full_base : ps->comp_base;
+        const int l = step_layer(base, ps->n_layers, unit);
+        const int nf = (ps->full_base[l + 1] - ps->full_base[l]) / ps->batch;
+        b = (unit - base[l]) / (full ? nf : ps->kv_heads - nf);
     } else {
-        n = pg->seq_len[(uid - a.sched.U) / a.n_comp];
-        if (n > pg->cap) n = pg->cap;
+        b = full ? uid / a.n_full : (uid - a.sched.U) / a.n_comp;
     }
+    int n = pg->seq_len[b];
+    if (!full && n > pg->cap) n = pg->cap;
     return (n + kTile - 1) / kTile;
 }
 

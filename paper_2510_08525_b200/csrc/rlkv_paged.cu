@@ -12,7 +12,7 @@
 //               16 KB (K codes [64 rows][128], then V codes transposed [128][64 rows]); per layer the
 //               full heads' pages [n_full(layer)][n_pages], then the rings
 //               [max_seqs][n_comp(layer)][rows_comp / 64]
-//   scales      float 1/k_scale, 1/v_scale [layers][kv_heads] (8-bit pages only)
+//   scales      float 1/k_scale, 1/v_scale, k_scale, v_scale, each [layers][kv_heads] (8-bit pages only)
 //   tables      int32 slot_of_head[layers][kv_heads]
 //   page table  int32 [max_seqs][table_stride]   (written by the append kernels)
 //   layer desc  LayerDesc[layers]  (where each layer's regions start; for the step's append launch)
@@ -38,6 +38,9 @@ struct rlkv_paged {
     int device, sm_count, stages, groups, item_tiles;
     int rows_comp, max_batch, max_items, max_grid;
     int out_bf16;
+    int step_mode;                // rlkv_paged_step: 0 chooses, 1 one decode launch per layer, 2 one for the whole step
+    bool step_in_one_launch;      // the shape allows one decode launch for a whole step
+    long long step_slots;         // partial records the scratch holds when both copies are used as one
     int fp8;                      // K/V rows (pages and rings) are held as E4M3 codes
     std::vector<float> k_scale, v_scale;  // [layers*kv_heads]
     std::vector<long long> page0_8, ring0_8;  // first full-head page / first ring page of each layer in the 8-bit pool
@@ -53,7 +56,7 @@ struct rlkv_paged {
     std::vector<int> table;       // [max_seqs][table_stride], -1 = no page
     std::vector<int> free_pages;  // stack of physical pages
     std::vector<uint8_t> open;    // [max_seqs]
-    size_t off_pool, off_tables, off_layer_desc, off_page_table, off_tickets, off_status, off_partials, total;
+    size_t off_pool, off_tables, off_head_table, off_layer_desc, off_page_table, off_tickets, off_status, off_partials, total;
     unsigned int claims[2];
     uint8_t* dev_base;
     bool owns_buffer;
@@ -129,22 +132,46 @@ int make_paged_layout(rlkv_paged& p, const uint8_t* mask, int max_seq_len)
     if (row >= (1ll << 31) || most >= (1ll << 31)) return RLKV_EINVAL;  // TMA row coordinates are 32-bit
     if (p.pages8 * 128 >= (1ll << 31)) return RLKV_EINVAL;              // a page is 128 rows of the 8-bit map
     p.pool_rows = row;
+    // A whole step in one launch uses both copies of the scratch as one.  Sized for max_batch sequences
+    // of max_seq_len tokens where that is modest (at most 64 MB more per copy); a step that needs more
+    // records than there are runs as one launch per layer.
+    p.step_in_one_launch = p.layers <= kMaxStepLayers && p.layers * p.kv_heads <= kMaxStepHeads;
+    if (p.step_in_one_launch) {
+        long long U = 0, Uc = 0;
+        for (int l = 0; l < p.layers; ++l) {
+            U += (long long)p.max_batch * p.n_full[l];
+            Uc += (long long)p.max_batch * p.n_comp[l];
+        }
+        const long long T = U * p.table_stride + Uc * (p.rows_comp / kTile);
+        const long long small = (long long)p.max_grid * kDefaultItemTiles / kMinItemTiles + 1;
+        const long long large = T / kDefaultItemTiles + 1;
+        long long fused = 2ll * p.max_grid + 2 * U + Uc + (small > large ? small : large) + 8;
+        const long long cap = most + (64ll << 20) / ((long long)partial_floats(p.head_dim, p.q_heads / p.kv_heads) * 4);
+        if ((fused + 1) / 2 > cap) fused = 2 * cap;
+        if ((fused + 1) / 2 > most) most = (fused + 1) / 2;
+    }
     p.max_items = (int)most;
+    p.step_slots = 2ll * most;
     size_t off = 0;
     p.off_pool = off;
     off = align_up(off + (size_t)row * p.head_dim * 2, 1024);
     p.off_pool8 = off;
     off = align_up(off + (size_t)p.pages8 * 2 * kTile * 128, 1024);
     p.off_scales = off;
-    off = align_up(off + (p.fp8 ? (size_t)2 * p.layers * p.kv_heads * sizeof(float) : 0), 1024);
+    off = align_up(off + (p.fp8 ? (size_t)4 * p.layers * p.kv_heads * sizeof(float) : 0), 1024);
     p.off_tables = off;
+    off = align_up(off + (size_t)p.layers * p.kv_heads * sizeof(int), 1024);
+    p.off_head_table = off;  // head_of_slot, for a whole-step launch
     off = align_up(off + (size_t)p.layers * p.kv_heads * sizeof(int), 1024);
     p.off_layer_desc = off;
     off = align_up(off + (size_t)p.layers * sizeof(LayerDesc), 1024);
     p.off_page_table = off;
     off = align_up(off + (size_t)p.max_seqs * p.table_stride * sizeof(int), 1024);
     p.off_tickets = off;
-    off = align_up(off + (size_t)2 * kMaxPagedBatch * p.kv_heads * sizeof(int), 1024);
+    {   // two copies of one ticket per unit of a layer; a whole step needs one per unit of every layer
+        const size_t per_layer = (size_t)2 * kMaxPagedBatch * p.kv_heads, whole = (size_t)p.layers * p.max_batch * p.kv_heads;
+        off = align_up(off + (per_layer > whole ? per_layer : whole) * sizeof(int), 1024);
+    }
     p.off_status = off;
     off = align_up(off + 64, 1024);
     p.off_partials = off;
@@ -255,6 +282,7 @@ static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads,
     p->layers = layers; p->kv_heads = kv_heads; p->q_heads = q_heads; p->head_dim = head_dim;
     p->max_seqs = max_seqs; p->n_pages = n_pages; p->sink = sink; p->window = window; p->max_seq_len = max_seq_len;
     p->claims[0] = p->claims[1] = 0; p->launches = 0; p->dev_base = nullptr; p->owns_buffer = false; p->out_bf16 = 0;
+    p->step_mode = 0;
     p->fp8 = fp8;
     if (fp8) {
         p->k_scale.assign(k_scale, k_scale + (size_t)layers * kv_heads);
@@ -294,16 +322,21 @@ static int paged_create(rlkv_paged** out, int layers, int kv_heads, int q_heads,
     if (e == cudaSuccess && fp8) e = cudaMemset(p->dev_base + p->off_pool8, 0, (size_t)p->pages8 * 2 * kTile * 128);
     if (e == cudaSuccess && fp8) {
         // the kernels multiply by 1 / scale: one IEEE division per head, here
-        std::vector<float> inv((size_t)2 * layers * kv_heads);
+        std::vector<float> inv((size_t)4 * layers * kv_heads);  // then the scales themselves, for a whole-step launch
         for (int i = 0; i < layers * kv_heads; ++i) {
             inv[i] = 1.0f / k_scale[i];
             inv[(size_t)layers * kv_heads + i] = 1.0f / v_scale[i];
+            inv[(size_t)2 * layers * kv_heads + i] = k_scale[i];
+            inv[(size_t)3 * layers * kv_heads + i] = v_scale[i];
         }
         e = cudaMemcpy(p->dev_base + p->off_scales, inv.data(), inv.size() * sizeof(float), cudaMemcpyHostToDevice);
     }
     if (e == cudaSuccess) e = cudaMemset(p->dev_base + p->off_page_table, 0, p->off_partials - p->off_page_table);
     if (e == cudaSuccess)
         e = cudaMemcpy(p->dev_base + p->off_tables, p->slot_of_head.data(), p->slot_of_head.size() * sizeof(int),
+                       cudaMemcpyHostToDevice);
+    if (e == cudaSuccess)
+        e = cudaMemcpy(p->dev_base + p->off_head_table, p->head_of_slot.data(), p->head_of_slot.size() * sizeof(int),
                        cudaMemcpyHostToDevice);
     if (e == cudaSuccess) {
         std::vector<LayerDesc> desc(layers);
@@ -465,8 +498,12 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
 // One decode launch (arguments checked by the caller).  `half`: which copy of tickets, claim counter
 // and partials; `overlap`, `dep_wait`: as for the lock-step cache (launch_decode, decode_kernel);
 // `in_step`: the launch belongs to rlkv_paged_step (coarser items: its neighbours hide its tail).
+// `whole_step`: one launch for every layer (`layer` is 0; q, out are the step's [layers][n][q_heads][head_dim]
+// arrays; every listed sequence holds the same number of tokens in all layers; both scratch copies are
+// used as one).  Returns RLKV_ESCRATCH, with nothing launched, if such a launch needs more partial records
+// than the scratch holds: the caller then issues one launch per layer.
 static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const void* q, void* out, cudaStream_t stream,
-                        int half, bool overlap, int dep_wait, bool in_step, int* grid_out)
+                        int half, bool overlap, int dep_wait, bool in_step, int* grid_out, bool whole_step = false)
 {
     const int* len = len_of(p, layer);
     int longest = 0;
@@ -498,13 +535,57 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
     a.out_bf16 = p->out_bf16;
     const int tiles_full = (a.len_full + kTile - 1) / kTile, tiles_comp = (a.len_comp + kTile - 1) / kTile;
     // the tiles that exist (the schedule also spans the ones that do not) decide the item size
+    int heads_full = a.n_full, heads_comp = a.n_comp;  // per sequence, over the layers the launch serves
+    if (whole_step) {
+        heads_full = heads_comp = 0;
+        for (int l = 0; l < p->layers; ++l) {
+            heads_full += p->n_full[l];
+            heads_comp += p->n_comp[l];
+        }
+    }
     long long real_tiles = 0;
+    bool equal_lengths = true;
     for (int i = 0; i < n; ++i) {
         const int t = len[slots[i]];
-        real_tiles += (long long)a.n_full * ((t + kTile - 1) / kTile) + (long long)a.n_comp * (((t < cap ? t : cap) + kTile - 1) / kTile);
+        real_tiles += (long long)heads_full * ((t + kTile - 1) / kTile) + (long long)heads_comp * (((t < cap ? t : cap) + kTile - 1) / kTile);
+        if (t != len[slots[0]]) equal_lengths = false;
     }
     int grid = p->sm_count;
     if (grid > p->max_grid) grid = p->max_grid;
+    PagedArgs pa;
+    memset(&pa, 0, sizeof pa);
+    pa.step.n_layers = 1;
+    if (whole_step) {
+        if ((long long)n * heads_full * tiles_full + (long long)n * heads_comp * tiles_comp >= (1ll << 31)) return RLKV_ESCRATCH;
+        const int most = kDefaultItemTiles * (p->fp8 ? 2 : 1);
+        // equal lengths: most full units whole in one static item per CTA; else every item is claimed
+        a.sched = step_schedule(n * heads_full, tiles_full, n * heads_comp, tiles_comp, grid, most, equal_lengths, real_tiles);
+        if (a.sched.n_slots > p->step_slots) return RLKV_ESCRATCH;
+        if (grid > a.sched.n_items) grid = a.sched.n_items;
+        a.n_full = a.n_comp = 0;
+        a.batch = n * p->layers;
+        a.partials = dev_at<float>(p, p->off_partials);
+        a.tickets = dev_at<int>(p, p->off_tickets);
+        a.claim_counter = dev_at<unsigned int>(p, p->off_status) + 4;
+        a.claim_base = p->claims[0];
+        a.dep_wait = dep_wait;
+        StepArgs& st = pa.step;
+        st.head_of_slot = dev_at<int>(p, p->off_head_table);
+        st.n_layers = p->layers;
+        st.kv_heads = p->kv_heads;
+        st.batch = n;
+        st.full_base[0] = st.comp_base[0] = 0;
+        for (int l = 0; l < p->layers; ++l) {
+            st.full_base[l + 1] = st.full_base[l] + n * p->n_full[l];
+            st.comp_base[l + 1] = st.comp_base[l] + n * p->n_comp[l];
+            st.full_row0[l] = (int)p->full_row0[l];
+            st.comp_row0[l] = (int)p->comp_row0[l];
+            pa.page0_8_of[l] = (int)p->page0_8[l];
+            pa.ring0_8_of[l] = (int)p->ring0_8[l];
+        }
+        pa.scales = dev_at<float>(p, p->off_scales) + (size_t)2 * p->layers * p->kv_heads;
+        half = 0;
+    } else {
     int item_tiles = (int)(real_tiles / grid);
     // (a tile of 8-bit pages is half the bytes, so the same grain in time is twice the tiles)
     const int most = (in_step ? kPagedItemTilesStep : p->item_tiles) * (p->fp8 ? 2 : 1);
@@ -524,7 +605,7 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
     a.claim_counter = dev_at<unsigned int>(p, p->off_status) + 4 + half;
     a.claim_base = p->claims[half];
     a.dep_wait = dep_wait;
-    PagedArgs pa;
+    }
     pa.page_table = dev_at<int>(p, p->off_page_table);
     pa.table_stride = p->table_stride;
     pa.n_pages = p->n_pages;
@@ -611,7 +692,13 @@ int rlkv_paged_step(rlkv_paged* p, const int* slots, int n, const void* k, const
     p->launches++;
     for (int l = 0; l < p->layers; ++l)
         for (int i = 0; i < n; ++i) len_of(p, l)[slots[i]] += 1;
-    // the layers' decode launches, overlapped as in rlkv_step (step_launch_mode in rlkv_host.cuh)
+    // one decode launch over all layers (it may start beside the append launch and waits for it on the
+    // device); where the step's partial records would not fit the scratch, or the caller asked for it,
+    // one launch per layer, overlapped as in rlkv_step (step_launch_mode in rlkv_host.cuh)
+    if (p->step_mode != 1 && p->step_in_one_launch && p->layers > 1) {  // (one layer: the per-layer launch is the whole step)
+        rc = paged_decode(p, 0, slots, n, q, out, s, 0, true, 1, true, nullptr, true);
+        if (rc != RLKV_ESCRATCH) return rc;
+    }
     const size_t q_layer = (size_t)n * p->q_heads * p->head_dim;
     for (int l = 0; l < p->layers; ++l) {
         const StepLaunchMode m = step_launch_mode(l == 0, true);
@@ -624,6 +711,14 @@ int rlkv_paged_step(rlkv_paged* p, const int* slots, int n, const void* k, const
 }
 
 
+
+int rlkv_paged_set_step_mode(rlkv_paged* p, int mode)
+{
+    if (!p || mode < 0 || mode > 2) return RLKV_EINVAL;
+    if (mode == 2 && !p->step_in_one_launch) return RLKV_EINVAL;
+    p->step_mode = mode;
+    return RLKV_OK;
+}
 
 int rlkv_paged_set_output_bf16(rlkv_paged* p, int on)
 {

@@ -313,21 +313,27 @@ def test_four_hundred_sequences_in_one_call(rl, hz, cuda_device):
     cache.close()
 
 
-@pytest.mark.parametrize("shape", ["small", "filling"])
-def test_paged_step_equals_the_per_layer_calls(rl, hz, cuda_device, shape):
-    """rlkv_paged_step (one append launch for all layers, the layers' attention launches overlapped)
-    over consecutive steps that cross page boundaries: every sequence against its oracle, and the page
-    accounting as the per-layer calls would leave it.  'small': launches of a few work items, each
-    started beside the one before; 'filling': launches with more than one item per SM."""
+@pytest.mark.parametrize("step_mode", [1, 2], ids=["launch_per_layer", "one_launch"])
+@pytest.mark.parametrize("shape", ["small", "filling", "uniform"])
+def test_paged_step_equals_the_per_layer_calls(rl, hz, cuda_device, shape, step_mode):
+    """rlkv_paged_step (one append launch for all layers, then one attention launch over every layer, or
+    the layers' attention launches overlapped) over consecutive steps that cross page boundaries: every
+    sequence against its oracle, and the page accounting as the per-layer calls would leave it.
+    'small': a few work items; 'filling': more than one item per SM, lengths all different (every item
+    of the whole-step launch is claimed); 'uniform': equal lengths (most units whole in one item per CTA)."""
     if shape == "small":
         layers, Hkv, Hq, D, S, W, lens = 5, 2, 8, 64, 4, 28, [60, 1, 126, 200]
         mask = [1, 0, 0, 0, 1, 1, 0, 1, 1, 0]
+    elif shape == "uniform":
+        layers, Hkv, Hq, D, S, W, lens = 4, 4, 16, 128, 16, 48, [1530] * 12
+        mask = [1, 1, 0, 1] + [0, 0, 0, 0] + [1, 1, 1, 1] + [0, 1, 1, 0]
     else:
         layers, Hkv, Hq, D, S, W, lens = 3, 8, 32, 128, 16, 112, [3000, 1500, 2900, 700, 2047, 3100, 2500, 1000]
         mask = [1] * 8 + [1, 1, 0, 1, 1, 0, 1, 1] + [0] * 8
     steps = 6
     pages = sum((n + steps + 63) // 64 for n in lens) + 1
     cache = hz.PagedCache(layers, Hkv, Hq, D, len(lens), pages, max(lens) + 64, mask, S, W, device=cuda_device)
+    rl.rlkv_paged_set_step_mode(cache.handle, step_mode)
     seqs = []
     for i, n in enumerate(lens):
         s = Seq(cache, 300 + i, max(lens) + 64)
@@ -369,6 +375,7 @@ FP8_SHAPES = [
     (1, 1, 8, 0, 5, "1", [777, 3]),
     (1, 4, 16, 16, 64, "0000", [400, 90]),
     (1, 2, 8, 16, 112, "11", [9000, 4100]),              # long rows: split over many work items
+    (3, 4, 16, 16, 112, "1011" "0110" "1111", [700] * 6),    # equal lengths: the whole step's schedule has its prefix
 ]
 
 
