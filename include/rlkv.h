@@ -167,19 +167,19 @@ size_t rlkv_static_scratch_bytes(void);
  * Every head of the layer must be a full head (the full branch needs every token): RLKV_EINVAL
  * otherwise.  q: device bf16 [batch][q_heads][head_dim]; alpha: DEVICE fp32 [kv_heads], the gates of
  * this layer, read when the kernel runs and used as they are (the paper keeps them in [0, 1]; the
- * library does not check); out: device fp32 [batch][q_heads][head_dim].  One launch: the K/V rows are
- * streamed once for the full branch, the sink and window rows a second time for the local branch
- * (sink + window rows per head, normally out of the L2), and each branch adds its weighted result
- * into `out`, which the call clears on `stream` first.  K and V rows are assumed finite.
+ * library does not check); out: device fp32 [batch][q_heads][head_dim] (bf16 after
+ * rlkv_set_output_bf16).  One launch: the K/V rows are streamed once for the full branch, the sink and
+ * window rows a second time for the local branch (sink + window rows per head, normally out of the
+ * L2); whichever CTA delivers the last piece of a head's two branches merges both and writes
+ * alpha * full + (1 - alpha) * local once.  K and V rows are assumed finite.
  * RLKV_EEMPTY if length(layer) == 0. */
 int rlkv_decode_mixed_attention(rlkv_cache* cache, int layer, const void* q, const float* alpha,
                                 void* out, void* stream);
 
-/* Output element type of rlkv_decode_attention, rlkv_decode_attention_static_scratch, rlkv_step and
- * rlkv_step_host from now on: on != 0 stores results as bf16 (the fp32 result rounded to nearest
- * even when it is stored; `out` buffers then hold bf16 elements of the same shape, half the bytes),
- * on == 0 (the default) as fp32.  The arithmetic does not change.  rlkv_decode_mixed_attention adds
- * its two branches up in the fp32 output buffer and returns RLKV_EINVAL while bf16 output is on. */
+/* Output element type of rlkv_decode_attention and its variants, rlkv_decode_mixed_attention,
+ * rlkv_step and rlkv_step_host from now on: on != 0 stores results as bf16 (the fp32 result rounded
+ * to nearest even when it is stored; `out` buffers then hold bf16 elements of the same shape, half
+ * the bytes), on == 0 (the default) as fp32.  The arithmetic does not change. */
 int rlkv_set_output_bf16(rlkv_cache* cache, int on);
 
 /* One whole decode step: for every layer, append then attend.  Device buffers:

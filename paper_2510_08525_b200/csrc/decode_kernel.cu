@@ -280,7 +280,7 @@ struct Smem {
     {
         return (size_t)stages * stage_bytes(group, mode) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
                kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
-               kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 1) * 8 /*their partial lists*/ +
+               kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 2) * 8 /*their partial lists*/ +
                (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0) +
                (mode == kModeStep ? kStepBytes : 0);
     }
@@ -297,16 +297,17 @@ struct Smem {
 // writes to `units` and `lists`.
 // (Everything comes by value or from shared memory: a reference to kernel parameters would turn
 // every use into a slow generic load inside this non-inlined function.)
-// MIXED (Eq. 1 of the paper): a unit's rows are shared by its full and its local unit; each adds
-// its result times its weight (the head's gate alpha for the full unit u < U, 1 - alpha for the
-// local one) to rows the host cleared.  Two addends on zero commute, so the sum does not depend
-// on their order.
+// MIXED (Eq. 1 of the paper): `units` lists (batch row, head) pairs; entries 0 .. R of a pair's list
+// are the records of its full unit, entry kMaxRounds + 1 those of its local unit.  Both are merged
+// and the rows get gate * full + (1 - gate) * local, written once: no clearing, no atomics, and the
+// result does not depend on which unit finished first.
+constexpr int kListStride = kMaxRounds + 2;  // (first record, count) per band, then the local unit's (MIXED)
 template <int D, bool MIXED>
 __device__ __noinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
                                          const int2* lists, int n, int t, int nt, bool dry,
                                          unsigned long long* stamp, const float* alpha, int U, int q_heads, int out_bf16)
 {
-    constexpr int D4 = D / 4, CH = 16, NB = kMaxRounds + 1;
+    constexpr int D4 = D / 4, CH = 16, NB = kListStride;
     const int E = G * D4;
     const int PF = partial_floats(D, G), PH = partial_head_floats(G);
     __threadfence();
@@ -317,13 +318,17 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
     if (ul < unit_lanes) {
         for (int j = ul; j < n; j += unit_lanes) {
             const int2* li = lists + j * NB;
-            int F = 0;
-            for (int r = 0; r <= R; ++r) F += li[r].y;
             for (int e = wide ? t - ul * E : t; e < E; e += wide ? E : nt) {
                 const int g = e / D4;
+                float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 1
+                for (int part = 0; part < (MIXED ? 2 : 1); ++part) {  // the full unit's records, then the local unit's
+                const int b0 = part ? NB - 1 : 0, b1 = part ? NB : R + 1;
+                int F = 0;
+                for (int r = b0; r < b1; ++r) F += li[r].y;
                 float M = kNegBig, L = 0.f;
                 float4 O = make_float4(0.f, 0.f, 0.f, 0.f);
-                int band = 0, off = 0;  // the record with merge index c0 is record `off` of band `band`
+                int band = b0, off = 0;  // the record with merge index c0 is record `off` of band `band`
                 for (int c0 = 0; c0 < F; c0 += CH) {
                     float mm[CH], ll[CH];
                     float4 oo[CH];
@@ -366,21 +371,19 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
                 float inv = 1.f / L;
                 if (MIXED) {
                     const float gate = __ldg(alpha + (units[j].y % q_heads) / G);
-                    inv *= units[j].x < U ? gate : 1.f - gate;
-                    if (!dry) {
-                        float* o = out + (size_t)units[j].y * D + e * 4;
-                        atomicAdd(o, O.x * inv);
-                        atomicAdd(o + 1, O.y * inv);
-                        atomicAdd(o + 2, O.z * inv);
-                        atomicAdd(o + 3, O.w * inv);
-                    }
-                } else if (!dry) {
+                    inv *= part ? 1.f - gate : gate;
+                }
+                res.x += O.x * inv;
+                res.y += O.y * inv;
+                res.z += O.z * inv;
+                res.w += O.w * inv;
+                }
+                if (!dry) {
                     if (out_bf16)
                         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)units[j].y * D + e * 4) =
-                            make_uint2(pack_bf16(O.x * inv, O.y * inv), pack_bf16(O.z * inv, O.w * inv));
+                            make_uint2(pack_bf16(res.x, res.y), pack_bf16(res.z, res.w));
                     else
-                        *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) =
-                            make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                        *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) = res;
                 }
             }
         }
@@ -403,7 +406,9 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
 //
 // MIXED: the mixed attention of Eq. 1.  The schedule's second class holds, for every full unit, a
 // LOCAL unit over the same head's sink and window rows; its tiles start at whatever row the window
-// starts (a TMA box may start at any row) and are masked past their valid rows.
+// starts (a TMA box may start at any row) and are masked past their valid rows.  Every segment of
+// either unit leaves a partial record; the pair's ticket counts the records of both, and whoever
+// delivers the last one merges both units and writes gate * full + (1 - gate) * local once.
 //
 // kModeStep: a whole decode step.  The full units of all layers are one list and so are the compressed
 // units (every layer holds the same number of tokens); a unit's layer, rows, query and output rows are
@@ -469,7 +474,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     int* todo_count = const_cast<int*>(claim_slot) + 3;
     // The arguments, copied to shared memory: the schedule and the head order are looked up with
     // run-time indices, which is slow on kernel parameters and cheap here.
-    DecodeArgs* s_args = reinterpret_cast<DecodeArgs*>(lists + kMaxTodo * (kMaxRounds + 1));
+    DecodeArgs* s_args = reinterpret_cast<DecodeArgs*>(lists + kMaxTodo * kListStride);
     const DecodeArgs& a = *s_args;
     // paged cache: lengths and request slots of the batch, then the page ids of one segment
     PagedArgs* s_paged = reinterpret_cast<PagedArgs*>(reinterpret_cast<uint8_t*>(s_args) + (sizeof(DecodeArgs) + 15) / 16 * 16);
@@ -939,8 +944,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 if (warp == 0 && lane == 0) {
                     SegDesc* sd = reinterpret_cast<SegDesc*>(stat_l + S::kWarps * kMaxGroup);
                     // the whole unit (paged cache: all of its tiles that exist) in one segment
-                    const bool complete = u.pos.tile == 0 && (PAGED ? seg_tiles >= (u.len + kTile - 1) / kTile
-                                                                    : seg_tiles == u.tiles);
+                    // (mixed attention: a pair's rows are written once both of its units are in, so every
+                    // segment goes the way of the partial records)
+                    const bool complete = !MIXED && u.pos.tile == 0 &&
+                                          (PAGED ? seg_tiles >= (u.len + kTile - 1) / kTile : seg_tiles == u.tiles);
                     sd->out_row = u.qrow * a.q_heads + u.head * G;
                     sd->uid = u.pos.uid;
                     sd->complete = complete ? 1 : 0;
@@ -1303,14 +1310,14 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         if (sc.n_items > 2 * sc.P) {
             if (et == 0) todo[kMaxTodo - 1] = make_int2(0, 0);
             epilogue_sync();
-            if (et <= kMaxRounds) {
+            if (et < kListStride) {
                 int slot = 0, count = 0;
                 if (et <= sc.R) unit_partials(sc, 0, et, slot, count);
                 // two records per band at most: one batch of loads warms the same instructions as many
-                lists[(kMaxTodo - 1) * (kMaxRounds + 1) + et] = make_int2(slot, count < 2 ? count : 2);
+                lists[(kMaxTodo - 1) * kListStride + et] = make_int2(slot, count < 2 ? count : 2);
             }
             epilogue_sync();
-            merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * (kMaxRounds + 1),
+            merge_units<D, MIXED>(a.partials, a.out, G, sc.R, todo + kMaxTodo - 1, lists + (kMaxTodo - 1) * kListStride,
                                   1, et, NE, true, nullptr, a.alpha, sc.U, a.q_heads, a.out_bf16);
             epilogue_sync();
         }
@@ -1334,8 +1341,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 if (et == 0) *todo_count = 0;
                 epilogue_sync();
             }
-            // 16 lanes per pending segment: lane r looks up the unit's partial records in band r
-            constexpr int NB = kMaxRounds + 1;
+            // 16 lanes per pending segment: lane r looks up the unit's partial records in band r (mixed
+            // attention: pend holds the pair, i.e. its full unit; lane 15 looks up the local unit's records,
+            // which all lie in the last band, and the ticket counts the records of both)
+            constexpr int NB = kListStride;
             for (int base = 0; base < pend_n * 16; base += NE) {  // whole warps take part in the shuffles
                 const int p = base + et, i = p >> 4, r = p & 15;
                 const bool on = p < pend_n * 16;
@@ -1344,6 +1353,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     if (PAGED) unit_partials(sc, pend[i].x, r, slot, count, paged_unit_tiles(a, pg, pend[i].x));
                     else unit_partials(sc, pend[i].x, r, slot, count);
                 }
+                if (MIXED && on && r == 15) unit_partials(sc, sc.U + pend[i].x, sc.R, slot, count);
                 int total = count;
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
@@ -1354,7 +1364,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     todo[idx] = pend[i];
                 }
                 idx = __shfl_sync(0xffffffffu, idx, lane & 16);  // from lane r == 0 of this 16-lane group
-                if (idx >= 0 && r < NB) lists[idx * NB + r] = make_int2(slot, count);
+                if (idx >= 0 && (r < NB - 1 || r == 15)) lists[idx * NB + (r == 15 ? NB - 1 : r)] = make_int2(slot, count);
             }
             epilogue_sync();
             pend_n = 0;
@@ -1384,11 +1394,6 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             }
             float* out_rows = a.out + (size_t)sd.out_row * D;
             float* my_part = a.partials + (size_t)sd.pslot * PF;
-            float weight = 1.f;  // MIXED: the gate's share of this unit in its output rows
-            if (MIXED) {
-                const float gate = __ldg(a.alpha + (sd.out_row % a.q_heads) / G);
-                weight = sd.uid < sc.U ? gate : 1.f - gate;
-            }
             // merge the consumer warps' states; this thread owns a few 4-float pieces of the G x D rows
             for (int e = et; e < G * D4; e += NE) {
                 const int g = e / D4, d4 = e - g * D4;
@@ -1407,13 +1412,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     O.z += o.z * wt;
                     O.w += o.w * wt;
                 }
-                if (sd.complete && MIXED) {
-                    const float inv = weight / L;
-                    atomicAdd(out_rows + e * 4, O.x * inv);
-                    atomicAdd(out_rows + e * 4 + 1, O.y * inv);
-                    atomicAdd(out_rows + e * 4 + 2, O.z * inv);
-                    atomicAdd(out_rows + e * 4 + 3, O.w * inv);
-                } else if (sd.complete) {
+                if (sd.complete) {
                     const float inv = 1.f / L;
                     if (a.out_bf16)
                         *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(a.out) + (size_t)sd.out_row * D + e * 4) =
@@ -1431,7 +1430,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(ep_empty + bi));  // the buffer may be refilled
             if (!sd.complete) {
-                if (et == 0) pend[pend_n] = make_int2(sd.uid, sd.out_row);
+                // (mixed attention: the pair, named by its full unit)
+                if (et == 0) pend[pend_n] = make_int2(MIXED && sd.uid >= sc.U ? sd.uid - sc.U : sd.uid, sd.out_row);
                 ++pend_n;
             }
         }

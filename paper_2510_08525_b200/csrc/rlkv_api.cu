@@ -8,8 +8,8 @@
 //             into a neighbouring head and a compressed head owns a constant number of rows
 //             (the constant-size pool of Section 4.3 of the paper).
 //   tables    int32 slot_of_head[layers][kv_heads], head_of_slot[layers][kv_heads]
-//   tickets   int32 [layers][2*batch*kv_heads] (split bookkeeping, zero between launches; the second
-//             half of a layer's tickets serves the local units of a mixed-attention launch)
+//   tickets   int32 [layers][2*batch*kv_heads] (split bookkeeping, zero between launches; one per unit of a
+//             launch -- a whole-step launch numbers the units of all its layers in one list)
 //   tables    then LayerDesc[layers] (where each layer's regions start; for the step's append launch)
 //   status    int32 kernel status word, then two work-claim counters (they only grow; consecutive
 //             launches of a step alternate between them)
@@ -317,8 +317,6 @@ int do_decode(rlkv_cache* c, int layer, const void* q, void* out, cudaStream_t s
     a.new_k = static_cast<const __nv_bfloat16*>(new_k);  // the launch appends the token itself (len already counts it)
     a.new_v = static_cast<const __nv_bfloat16*>(new_v);
     if (a.sched.n_slots > c->lay.max_items) return RLKV_ESCRATCH;  // cannot happen: the scratch is sized for it
-    // mixed attention: both units of a head add into `out`
-    if (alpha) RLKV_CUDA(cudaMemsetAsync(out, 0, (size_t)c->batch * c->q_heads * c->head_dim * sizeof(float), s));
     a.partials = dev_at<float>(c, c->lay.off_partials) +
                  (size_t)half * c->lay.max_items * partial_floats(c->head_dim, a.group);
     a.tickets = dev_at<int>(c, c->lay.off_tickets) + (size_t)layer * 2 * c->batch * c->kv_heads;
@@ -807,7 +805,6 @@ int rlkv_decode_mixed_attention(rlkv_cache* c, int layer, const void* q, const f
     if (!valid_layer(c, layer) || !q || !alpha || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
     if ((reinterpret_cast<uintptr_t>(alpha) & 3u) != 0) return RLKV_EINVAL;
     if (c->lay.n_comp[layer] != 0) return RLKV_EINVAL;  // the full branch needs every token of every head
-    if (c->out_bf16) return RLKV_EINVAL;                // the two branches are added up in fp32
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;

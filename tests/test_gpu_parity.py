@@ -686,13 +686,15 @@ def test_bf16_output_is_the_rounded_fp32_output(rl, hz, cuda_device):
     rl.rlkv_step_host(b16.handle, kh, vh, qh, got_h)
     torch.cuda.synchronize()
     assert torch.equal(got_h, want_h.to(torch.bfloat16))
-    # mixed attention adds up in fp32: refused while bf16 output is on; back to fp32, the cache works as before
-    allf = hz.Cache(1, Hkv, Hq, D, B, 16, np.ones(Hkv, np.uint8), S, W, device=cuda_device)
-    allf.append(0, k[0], v[0])
+    # mixed attention writes its rows once, so it can round them as well; back to fp32, the cache works as before
+    allf = hz.Cache(1, Hkv, Hq, D, B, 400, np.ones(Hkv, np.uint8), S, W, device=cuda_device)
+    allf.prefill(0, rand_bf16((300, B, Hkv, D), 93, cuda_device), rand_bf16((300, B, Hkv, D), 94, cuda_device))
+    gates = torch.rand(Hkv, device=cuda_device)
+    mixed32 = allf.decode_mixed(0, q[0], gates)
     rl.rlkv_set_output_bf16(allf.handle, 1)
-    with pytest.raises(rl.RlkvError) as e:
-        rl.rlkv_decode_mixed_attention(allf.handle, 0, q[0], torch.ones(Hkv, device=cuda_device), want[0])
-    assert e.value.code == rl.RLKV_EINVAL
+    mixed16 = torch.empty((B, Hq, D), dtype=torch.bfloat16, device=cuda_device)
+    rl.rlkv_decode_mixed_attention(allf.handle, 0, q[0], gates, mixed16)
+    assert torch.equal(mixed16, mixed32.to(torch.bfloat16))
     rl.rlkv_set_output_bf16(b16.handle, 0)
     assert torch.equal(b16.decode(1, q[1]), f32.decode(1, q[1]))
     assert f32.status() == 0 and b16.status() == 0
