@@ -530,7 +530,10 @@ def run_sweep(args, rl, harness, dev, stream):
                         "gbs": by / (us * 1e-6) / 1e9, "frac_of_nominal_8000": by / (us * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
                         "expected_ratio": (1 - s_real) + s_real * min(n, base.sink + base.window) / n,
                         "measured_ratio": None if zero_us is None else us / zero_us,
-                        "l2_resident": by < 100e6, "launch_bound": us < 10.0,
+                        "step_us": us * lp, "kv_bytes_per_step": by * lp,
+                        # the whole step's K/V rows could partly stay in the 126 MB L2 from one step to the
+                        # next / the step (one append launch, one attention launch) is set by latency
+                        "l2_resident": by * lp < 252e6, "latency_bound": us * lp < 100.0,
                         "steps": K, "warmup": W, "clocks": res["clocks"]}
                 print(json.dumps(line), flush=True)
                 del res
@@ -538,7 +541,8 @@ def run_sweep(args, rl, harness, dev, stream):
 
 
 def sweep_table(path):
-    """Markdown table of a file of --sweep lines: cells 'us per layer / TB/s (measured ratio | expected)'."""
+    """Markdown table of a file of --sweep lines: cells 'us per layer, TB/s (measured ratio / cost model)';
+    † = the whole step reads less than twice the L2's size, ‡ = the whole step takes under 100 us."""
     cells = {}
     for line in open(path):
         line = line.strip()
@@ -559,7 +563,8 @@ def sweep_table(path):
                 row.append("")
                 continue
             lp = d["layers_held"]
-            flag = ("†" if d["l2_resident"] else "") + ("‡" if d["launch_bound"] else "")
+            step_us, step_bytes = d["us_per_layer"] * lp, d["kv_bytes_per_layer"] * lp
+            flag = ("†" if step_bytes < 252e6 else "") + ("‡" if step_us < 100.0 else "")
             ratio = "" if d["measured_ratio"] is None or f == 0 else f" ({d['measured_ratio']:.2f} / {d['expected_ratio']:.2f})"
             row.append(f"{d['us_per_layer']:.0f} µs, {d['gbs'] / 1e3:.2f} TB/s{flag}{ratio}")
         print(f"| {ctx} | {batch} | {lp} | " + " | ".join(row) + " |")

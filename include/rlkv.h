@@ -353,7 +353,9 @@ int rlkv_set_decode_config(rlkv_cache* cache, int ctas_per_sm, int stages, int c
  * free descriptor (low half) and a free stage (high half); [16..26] for its first 11 work items,
  * (%globaltimer << 16) | (item & 0xffff) when the consumers started it; [27] cycles the producer
  * ran; [28..31] %globaltimer stamps inside the final merge; [32..36] producer cycles spent arming
- * barriers, issuing tile copies, issuing query copies, publishing items and locating segments.
+ * barriers, issuing tile copies, issuing query copies, publishing items and locating segments;
+ * [37..39] %globaltimer when the producer issued its first tile copy, when the CTA's set-up was done
+ * and when the producer entered its loop.
  * words_host != NULL: first synchronises the device and copies the words of the most recent launch
  * to words_host (host, 40 * 320 words) and the CTA capacity (320) to *ctas_out; then the switch is
  * applied. */
@@ -404,6 +406,13 @@ int rlkv_debug_standin(void* dst, const void* src, size_t bytes, const void* aft
  * [n_launches] each) */
 int rlkv_debug_step_plan(int n_launches, int follows_append, int* overlap_out, int* dep_wait_out,
                          int* scratch_copy_out);
+
+/* The order in which the work items of rlkv_debug_schedule's schedule are handed out, host arithmetic
+ * only: order_out[k] (host int[n_items]; `cap` = ints available) = the item CTA k starts with (k <
+ * ctas) resp. the item the (k - ctas)-th run-time claim receives.  Items made of compressed units come
+ * first among the claimed ones (many short segments: they must not be the launch's last items). */
+int rlkv_debug_claim_order(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas,
+                           int item_tiles, int whole_step, int* order_out, int cap);
 
 const char* rlkv_strerror(int code);
 

@@ -51,6 +51,7 @@ SIGNATURES = {
     "rlkv_debug_schedule": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, ctypes.POINTER(_ci), ctypes.POINTER(_ci), _vp, _vp, _ci]),
     "rlkv_set_step_mode": (_ci, [_vp, _ci]),
     "rlkv_debug_step_plan": (_ci, [_ci, _ci, _vp, _vp, _vp]),
+    "rlkv_debug_claim_order": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci]),
     "rlkv_debug_read_bandwidth": (_ci, [_vp, _sz, _ci, ctypes.POINTER(ctypes.c_float)]),
     "rlkv_strerror": (ctypes.c_char_p, [_ci]),
     "rlkv_paged_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
@@ -298,6 +299,14 @@ def rlkv_debug_read_bandwidth(buf, nbytes, launches=4) -> float:
     ms = ctypes.c_float(0)
     _check(lib.rlkv_debug_read_bandwidth(_ptr(buf), int(nbytes), int(launches), ctypes.byref(ms)))
     return float(ms.value)
+
+
+def rlkv_debug_claim_order(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, n_items, whole_step=False):
+    """int32[n_items]: the item handed to CTA k (k < ctas) / to the (k - ctas)-th claim."""
+    order = np.zeros(n_items, dtype=np.int32)
+    _check(lib.rlkv_debug_claim_order(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, int(whole_step),
+                                      order.ctypes.data, n_items))
+    return order
 
 
 def rlkv_debug_step_plan(n_launches, follows_append=True):

@@ -577,6 +577,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    if (trace && tid == 0) my_trace[38] = global_timer_ns();
 
     int issued = 0;  // producer: slots issued so far (data or empty)
     int page_lost_par = -1;  // producer, paged cache: phase of a page look-up it gave up waiting for
@@ -993,6 +994,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             unsigned long long ns_claim = 0, ns_ring = 0, ns_stage = 0;
             long long cy_expect = 0, cy_tma = 0, cy_q = 0, cy_item = 0, cy_seg = 0;
             const long long t_prod = clock64();
+            if (trace) my_trace[39] = global_timer_ns();
             int k = blockIdx.x;  // the host launches no more CTAs than there are items
             bool synced = false;  // has waited for the kernels before this one
             uint32_t ppar = 0;    // PAGED: phase of the page look-up barrier
@@ -1007,8 +1009,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 for (int j = 0; j < n_late; ++j) bulk_load(late_dst[j], late_src[j], G * D * 2, late_bar[j]);
                 n_late = 0;
             };
-            while (ok && k < sc.n_items) {
+            int k_claim = k;  // CTA c starts with item c; the claims after that are handed items in claim_to_item's order
+            while (ok && k_claim < sc.n_items) {
                 const long long ti0 = trace ? clock64() : 0;
+                k = claim_to_item(sc, k_claim);
                 const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
                 // ask the claim warp for the next item only shortly before this one is issued in
                 // full: early enough to hide the round trip, late enough that a CTA is never
@@ -1211,6 +1215,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     const long long tc0 = trace ? clock64() : 0;
                     mbar_expect_tx(fb, (FP8 ? n_sub * (kPairBytes / 2) : kPairBytes) + (with_q ? G * D * 2 : 0));
                     const uint32_t dst = smem_u32(stage_base + (size_t)s * stage_bytes);
+                    if (trace && issued == 0) my_trace[37] = global_timer_ns();
                     const long long tc1 = trace ? clock64() : 0;
                     if constexpr (FP8) {
                         // a page in one box of 128 rows of 128 bytes: 64 rows of K codes, then the transposed V
@@ -1258,7 +1263,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 if (PAGED && !asked) mbar_arrive(smem_u32(claim_empty));
                 ok = wait_traced(smem_u32(claim_full), cpar, s_abort, a.status, kStatusClaimWaitTimeout, trace, &ns_claim);
                 cpar ^= 1u;
-                if (ok) k = *claim_slot;
+                if (ok) k_claim = *claim_slot;
             }
             if (ok && wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout)) {
                 item_desc[di] = make_int4(-1, 0, 0, 0);  // no more work

@@ -1040,6 +1040,20 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
     return RLKV_OK;
 }
 
+int rlkv_debug_claim_order(int full_units, int tiles_full, int comp_units, int tiles_comp, int ctas, int item_tiles,
+                           int whole_step, int* order_out, int cap)
+{
+    if (full_units < 0 || comp_units < 0 || full_units + comp_units < 1 || tiles_full < 1 || tiles_comp < 1 ||
+        ctas < 1 || item_tiles < 1 || !order_out)
+        return RLKV_EINVAL;
+    if ((long long)full_units * tiles_full + (long long)comp_units * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
+    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+                                   : make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
+    if (cap < sc.n_items) return RLKV_ENOMEM;
+    for (int k = 0; k < sc.n_items; ++k) order_out[k] = claim_to_item(sc, k);
+    return RLKV_OK;
+}
+
 int rlkv_debug_step_plan(int n_launches, int follows_append, int* overlap_out, int* dep_wait_out, int* scratch_copy_out)
 {
     if (n_launches < 1 || !overlap_out || !dep_wait_out || !scratch_copy_out) return RLKV_EINVAL;

@@ -87,6 +87,7 @@ struct Schedule {
     int U0;                     // full units in the whole-unit prefix (0: no prefix)
     int x0, k0, s0;             // first flat tile, first item and first partial record after the prefix
     int pq, prem;               // the prefix's P items have pq tiles, the first prem one more
+    int kc;                     // first item that holds compressed tiles only (n_items if there is none)
     int base[kMaxRounds + 2];   // first flat tile of band r <= R; base[R+1]: first compressed tile
     int tb[kMaxRounds + 2];     // first tile, inside a full unit, of its slice in band r; tb[R+1] = tf
     int slot0[kMaxRounds + 1];  // first partial record of band r
@@ -133,7 +134,23 @@ inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz, 
     const int n_final = (s.T - s.base[r] + min_sz - 1) / min_sz;
     s.n_items = s.k0 + r * P + n_final;
     s.n_slots = s.slot0[r] + n_final + Ub + Uc;
+    // the last band's items are min_sz tiles from base[r] on: the first one that starts among the compressed tiles
+    s.kc = s.Uc > 0 ? s.k0 + r * P + (s.base[r + 1] - s.base[r] + min_sz - 1) / min_sz : s.n_items;
+    if (s.kc > s.n_items) s.kc = s.n_items;
     return s;
+}
+
+// The order in which items are handed out.  CTA c starts with item c (c < P); the i-th claim after that
+// (k = P + i) gets the items that hold compressed units first and the others, in order, after them: an
+// item of compressed units is many short segments, each with its own query fetch and hand-off, and
+// takes longer than its tiles say -- such items must not be the last ones of the launch.  Which CTA
+// processes which item never changes a result.
+__host__ __device__ inline int claim_to_item(const Schedule& s, int k)
+{
+    if (k < s.P || k >= s.n_items) return k;
+    const int first = s.kc > s.P ? s.kc : s.P;  // first claimable item of compressed units
+    const int nc = s.n_items - first, j = k - s.P;
+    return j < nc ? first + j : s.P + (j - nc);
 }
 
 // Upper bound of n_slots over every tf' <= tf with everything else the same (no prefix).

@@ -135,6 +135,24 @@ def test_whole_step_schedule(rl, U, tf, Uc, tc, ctas, item):
         assert (per_unit[:n_prefix] == 1).sum() >= n_prefix - 2 * ctas
 
 
+@pytest.mark.parametrize("whole_step", [False, True])
+@pytest.mark.parametrize("U,tf,Uc,tc,ctas,item", SHAPES[:8] + STEP_SHAPES[:6])
+def test_items_of_compressed_units_are_claimed_first(rl, U, tf, Uc, tc, ctas, item, whole_step):
+    """The hand-out order is a permutation of the items that keeps CTA c's first item (item c); among
+    the claimed items those that hold only compressed units come first, both groups in their own order."""
+    starts, _, tmap = rl.rlkv_debug_schedule(U, tf, Uc, tc, ctas, item, tile_map=True, whole_step=whole_step)
+    n_items = starts.size - 1
+    order = rl.rlkv_debug_claim_order(U, tf, Uc, tc, ctas, item, n_items, whole_step=whole_step)
+    assert sorted(order.tolist()) == list(range(n_items))
+    static = min(ctas, n_items)
+    assert order[:static].tolist() == list(range(static))
+    claimed = order[static:]
+    only_comp = np.array([bool((tmap[starts[k]:starts[k + 1], 0] >= U).all()) for k in claimed], dtype=bool)
+    n_c = int(only_comp.sum())
+    assert only_comp[:n_c].all() and not only_comp[n_c:].any()
+    assert (np.diff(claimed[:n_c]) > 0).all() and (np.diff(claimed[n_c:]) > 0).all()
+
+
 def test_schedule_rejects_bad_arguments(rl):
     for bad in ((0, 1, 0, 1, 148, 4), (1, 0, 0, 1, 148, 4), (1, 1, 1, 0, 148, 4), (1, 1, 0, 1, 0, 4),
                 (1, 1, 0, 1, 148, 0), (-1, 1, 2, 1, 148, 4)):
