@@ -124,7 +124,7 @@ def profiled_traffic_ratio():
     the kernel source has changed since the counters were taken."""
     import hashlib
     import re
-    prof = os.path.join(ROOT, "profiles", "decode_kernel_llama8b_4layers.md")
+    prof = os.path.join(ROOT, "profiles", "decode_kernel_step_llama8b_4layers.md")
     csrc = os.path.join(ROOT, "paper_2510_08525_b200", "csrc")
     try:
         text = open(prof).read()
