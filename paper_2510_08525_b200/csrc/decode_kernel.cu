@@ -247,6 +247,20 @@ struct SegDesc {
     int pad[3];
 };
 
+// What the producer tells the consumer warps about the next segment: they never look anything up in
+// the schedule themselves (a look-up costs about a microsecond, and while the consumers sit in one at
+// the start of a segment no stage is released: for a unit of two tiles that was as long as its tiles).
+struct SegInfo {
+    int item;              // the work item (it names the partial record); -1: no more work
+    int x;                 // flat tile of the segment's first tile
+    int seg_tiles;         // tiles of the segment in the schedule
+    int uid, tile, band;   // the unit, the segment's first tile inside it, the band
+    int tiles, len;        // tiles and valid rows of the unit
+    int qrow, head, layer; // where its query and output rows are; its KV head; its layer (paged whole step)
+    int pad;
+};
+constexpr int kSegRing = 8;  // segment descriptors in flight between producer and consumers
+
 // Shared-memory carve-up (dynamic shared memory, base aligned to 1024 bytes for the swizzle).
 template <int D, int NG>
 struct Smem {
@@ -265,7 +279,7 @@ struct Smem {
     }
     static constexpr int kMergeStride = D + kMergePad;      // floats per head row
     static constexpr int kStatFloats = 2 * kWarps * kMaxGroup;
-    static constexpr int kBarriers = 2 * 8 + 2 * kItemRing + 2 + 2 * kMergeBuffers + 2;  // the last two: page look-ups
+    static constexpr int kBarriers = 2 * 8 + 2 * kSegRing + 2 + 2 * kMergeBuffers + 2;  // the last two: page look-ups
     __host__ __device__ static constexpr int merge_floats(int group) { return kWarps * group * kMergeStride; }
     // one hand-off buffer: merge rows, per-warp max and sum, segment descriptor
     __host__ __device__ static constexpr int buffer_bytes(int group)
@@ -279,7 +293,8 @@ struct Smem {
     __host__ __device__ static constexpr size_t bytes(int stages, int group, int mode = kModePlain)
     {
         return (size_t)stages * stage_bytes(group, mode) + (size_t)kMergeBuffers * buffer_bytes(group) + kBarriers * 8 +
-               kItemRing * 16 /*items*/ + 16 /*claim slot, flags*/ + kMaxPend * 8 /*partial segments without a ticket*/ +
+               kSegRing * sizeof(SegInfo) /*segment descriptors*/ + 16 /*claim slot, flags*/ +
+               kMaxPend * 8 /*partial segments without a ticket*/ +
                kMaxTodo * 8 /*units to merge*/ + kMaxTodo * (kMaxRounds + 2) * 8 /*their partial lists*/ +
                (sizeof(DecodeArgs) + 15) / 16 * 16 + (mode == kModePaged || mode == kModePagedFp8 ? kPagedBytes : 0) +
                (mode == kModeStep ? kStepBytes : 0);
@@ -457,15 +472,15 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
     const int buffer_bytes = S::buffer_bytes(G);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(buffers + (size_t)kMergeBuffers * buffer_bytes);
     uint64_t* empty_bar = full_bar + 8;
-    uint64_t* item_full = empty_bar + 8;
-    uint64_t* item_empty = item_full + kItemRing;
-    uint64_t* claim_full = item_empty + kItemRing;
+    uint64_t* seg_full = empty_bar + 8;
+    uint64_t* seg_empty = seg_full + kSegRing;
+    uint64_t* claim_full = seg_empty + kSegRing;
     uint64_t* claim_empty = claim_full + 1;
     uint64_t* ep_full = claim_empty + 1;
     uint64_t* ep_empty = ep_full + kMergeBuffers;
     uint64_t* page_bar = ep_empty + kMergeBuffers;  // [2], the second one unused
-    int4* item_desc = reinterpret_cast<int4*>(page_bar + 2);
-    volatile int* claim_slot = reinterpret_cast<volatile int*>(item_desc + kItemRing);
+    SegInfo* seg_desc = reinterpret_cast<SegInfo*>(page_bar + 2);
+    volatile int* claim_slot = reinterpret_cast<volatile int*>(seg_desc + kSegRing);
     volatile int* ep_flag = claim_slot + 1;
     volatile int* s_abort = claim_slot + 2;
     int2* pend = reinterpret_cast<int2*>(const_cast<int*>(claim_slot) + 4);  // [kMaxPend] (unit, first output row)
@@ -560,9 +575,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
             mbar_init(smem_u32(full_bar + s), 1);
             mbar_init(smem_u32(empty_bar + s), kGroupWarps);
         }
-        for (int i = 0; i < kItemRing; ++i) {
-            mbar_init(smem_u32(item_full + i), 1);
-            mbar_init(smem_u32(item_empty + i), S::kWarps);
+        for (int i = 0; i < kSegRing; ++i) {
+            mbar_init(smem_u32(seg_full + i), 1);
+            mbar_init(smem_u32(seg_empty + i), S::kWarps);
         }
         mbar_init(smem_u32(claim_full), 1);
         mbar_init(smem_u32(claim_empty), 1);
@@ -606,23 +621,34 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
         unsigned long long ns_item = 0, ns_tile = 0, ns_merge = 0;
         const bool tr0 = trace && tid == 0;
         bool landed = false, alive = true;
+        int last_item = -1;
         while (alive) {
-            if (!wait_traced(smem_u32(item_full + di), dpar, s_abort, a.status, kStatusItemWaitTimeout, tr0, &ns_item)) break;
-            const int4 desc = item_desc[di];
-            const int item = desc.x, x0 = desc.y, x1 = desc.z;
-            if (item >= 0) {
+            // ---- the next segment, as the producer describes it: tiles [x, x + seg_tiles) of one unit
+            // (none for the stop message).  The descriptor is copied and its slot given back at once.
+            if (!wait_traced(smem_u32(seg_full + di), dpar, s_abort, a.status, kStatusItemWaitTimeout, tr0, &ns_item)) break;
+            const SegInfo sg = seg_desc[di];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(seg_empty + di));
+            if (++di == kSegRing) {
+                di = 0;
+                dpar ^= 1u;
+            }
+            const int item = sg.item, x = sg.x;
+            if (item >= 0 && item != last_item) {
                 if (tr0 && n_items < 11) my_trace[16 + n_items] = (global_timer_ns() << 16) | (unsigned long long)(item & 0xffff);
                 ++n_items;
-                // skip the empty slots the producer issued to line the slot counter up with x0
-                for (int pad = PAGED ? 0 : ((x0 - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
-                    if (turn != grp) continue;
-                    alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
-                    if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
-                }
+                last_item = item;
             }
-            for (int x = x0; alive && (item < 0 || x < x1);) {
-                // ---- the segment: tiles [x, x + seg_tiles) of one unit (none for the stop message)
+            {
                 UnitInfo u{};
+                u.pos.uid = sg.uid;
+                u.pos.tile = sg.tile;
+                u.pos.band = sg.band;
+                u.tiles = sg.tiles;
+                u.len = sg.len;
+                u.qrow = sg.qrow;
+                u.head = sg.head;
+                u.layer = sg.layer;
                 int seg_tiles = 0;
                 float m_run = kNegBig, l_run = 0.f;
                 // 8-bit pages: the first product has the tokens as rows and the heads as columns, so a lane
@@ -632,23 +658,17 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
 #pragma unroll
                 for (int mt = 0; mt < KS; ++mt) acc[mt][0] = acc[mt][1] = acc[mt][2] = acc[mt][3] = 0.f;
                 if (item >= 0) {
-                    u = locate<MODE>(a, x, pg, stp, s_heads);
-                    seg_tiles = min(x1 - x, u.pos.run);
+                    seg_tiles = sg.seg_tiles;
                     const bool local_unit = MIXED && u.pos.uid >= sc.U;
                     const bool fp8_unit = FP8;  // every unit of an 8-bit cache is pages of E4M3 codes
-                    int seg_eff = seg_tiles;  // tiles of the segment that exist
-                    if (PAGED) {
-                        seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
-                        if (seg_eff == 0) {  // nothing of this unit here: no tiles, no record
-                            x += seg_tiles;
-                            continue;
-                        }
-                        // tiles left out shift the slot counter against x: skip the producer's empty slots
-                        for (int pad = seg_eff > 0 ? ((x - cnt) % NG + NG) % NG : 0; alive && pad > 0; --pad, next_slot()) {
-                            if (turn != grp) continue;
-                            alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
-                            if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
-                        }
+                    int seg_eff = seg_tiles;  // tiles of the segment that exist (the producer announces no segment without any)
+                    if (PAGED) seg_eff = max(0, min(seg_tiles, (u.len + kTile - 1) / kTile - u.pos.tile));
+                    // skip the empty slots the producer issued to line the slot counter up with x (a new item
+                    // may start anywhere; tiles a paged unit does not have shift the counter against x)
+                    for (int pad = ((x - cnt) % NG + NG) % NG; alive && pad > 0; --pad, next_slot()) {
+                        if (turn != grp) continue;
+                        alive = wait_bounded(smem_u32(full_bar + st), ph, s_abort, a.status, kStatusFullWaitTimeout);
+                        if (alive && lane == 0) mbar_arrive(smem_u32(empty_bar + st));
                     }
                     // Q as the A operand (rows = query heads of the group, rows >= G are zero): read from
                     // the stage of this warp's first tile of the segment, where the producer put the
@@ -965,14 +985,6 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     alive = false;  // the stop message was the last thing to do
                     break;
                 }
-                x += seg_tiles;
-            }
-            if (!alive) break;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(item_empty + di));
-            if (++di == kItemRing) {
-                di = 0;
-                dpar ^= 1u;
             }
         }
         if (trace && tid == 0) {
@@ -1009,27 +1021,10 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 for (int j = 0; j < n_late; ++j) bulk_load(late_dst[j], late_src[j], G * D * 2, late_bar[j]);
                 n_late = 0;
             };
-            int k_claim = k;  // CTA c starts with item c; the claims after that are handed items in claim_to_item's order
-            while (ok && k_claim < sc.n_items) {
-                const long long ti0 = trace ? clock64() : 0;
-                k = claim_to_item(sc, k_claim);
-                const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
-                // ask the claim warp for the next item only shortly before this one is issued in
-                // full: early enough to hide the round trip, late enough that a CTA is never
-                // committed to more than the tiles in its ring plus a few
-                const int x_ask = max(x0, x1 - kClaimAhead);
-                ok = wait_traced(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout, trace,
-                                 &ns_ring);
-                if (!ok) break;
-                item_desc[di] = make_int4(k, x0, x1, 0);
-                mbar_arrive(smem_u32(item_full + di));  // release: the descriptor is visible to the waiters
-                if (++di == kItemRing) {
-                    di = 0;
-                    dpar ^= 1u;
-                }
-                if (trace) cy_item += clock64() - ti0;
-                // empty slots until the slot counter has the residue of x0
-                for (int pad = PAGED ? 0 : ((x0 - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
+            // empty slots until the slot counter has the residue of flat tile x (tile x always goes to
+            // consumer group x mod NG, whatever the CTA did before)
+            auto pad_to = [&](int x) {
+                for (int pad = ((x - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
                     ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
                     if (!ok) break;
                     mbar_arrive(smem_u32(full_bar + s));
@@ -1039,7 +1034,46 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         par ^= 1u;
                     }
                 }
+            };
+            // tells the consumer warps about the segment whose tiles come next (item < 0: no more work)
+            auto announce = [&](int item, int x, int seg_tiles, const UnitInfo& u) {
+                ok = wait_traced(smem_u32(seg_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout, trace, &ns_ring);
+                if (!ok) return;
+                SegInfo& sg = seg_desc[di];
+                sg.item = item;
+                sg.x = x;
+                sg.seg_tiles = seg_tiles;
+                sg.uid = u.pos.uid;
+                sg.tile = u.pos.tile;
+                sg.band = u.pos.band;
+                sg.tiles = u.tiles;
+                sg.len = u.len;
+                sg.qrow = u.qrow;
+                sg.head = u.head;
+                sg.layer = u.layer;
+                mbar_arrive(smem_u32(seg_full + di));  // release: the descriptor is visible to the waiters
+                if (++di == kSegRing) {
+                    di = 0;
+                    dpar ^= 1u;
+                }
+            };
+            // the unit of the segment being issued; whether that segment ends where the unit's slice ends; the
+            // region (prefix, band, compressed units) it lies in: its end, and first tile and width of a slice
+            UnitInfo cur{};
+            bool cur_slice_done = false;
+            int region_end = 0, region_tile0 = 0, region_width = 0;
+            int k_claim = k;  // CTA c starts with item c; the claims after that are handed items in claim_to_item's order
+            while (ok && k_claim < sc.n_items) {
+                const long long ti0 = trace ? clock64() : 0;
+                k = claim_to_item(sc, k_claim);
+                const int x0 = item_start(sc, k), x1 = item_start(sc, k + 1);
+                // ask the claim warp for the next item only shortly before this one is issued in
+                // full: early enough to hide the round trip, late enough that a CTA is never
+                // committed to more than the tiles in its ring plus a few
+                const int x_ask = max(x0, x1 - kClaimAhead);
+                if (trace) cy_item += clock64() - ti0;
                 int seg_left = 0, seg_idx = 0, krow = 0, vrow = 0;
+                cur_slice_done = false;  // a new item starts wherever the schedule says
                 int local_row0 = -1, local_next = 0;  // MIXED, inside a local unit: first row of its head, next tile
                 // PAGED: tiles of the segment past the unit's own length (not issued); first pool row of the
                 // full head's pages (-1: a compressed unit); page-table index of s_pages[0]; next tile
@@ -1062,8 +1096,33 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                     }
                     const long long ts0 = trace ? clock64() : 0;
                     if (seg_left == 0) {  // a new segment: where its rows are, whose query rows it needs
-                        const UnitInfo u = locate<MODE>(a, x, pg, stp, s_heads);
+                        // the unit: the successor of the one before where that one's slice was issued to its
+                        // end and the region goes on; looked up otherwise
+                        bool stepped = false;
+                        if (cur_slice_done && x < region_end) {
+                            stepped = next_unit<MODE>(a, cur, stp, s_heads);
+                            cur.pos.tile = region_tile0;
+                            cur.pos.run = region_width;
+                        }
+                        if (!stepped) {
+                            cur = locate<MODE>(a, x, pg, stp, s_heads);
+                            if (cur.pos.band < 0) {                 // the whole-unit prefix
+                                region_end = sc.x0;
+                                region_tile0 = 0;
+                                region_width = sc.tf;
+                            } else if (cur.pos.uid < sc.U) {        // a band of the full units
+                                region_end = sc.base[cur.pos.band + 1];
+                                region_tile0 = sc.tb[cur.pos.band];
+                                region_width = sc.tb[cur.pos.band + 1] - region_tile0;
+                            } else {                                // the compressed units
+                                region_end = sc.T;
+                                region_tile0 = 0;
+                                region_width = sc.tc;
+                            }
+                        }
+                        const UnitInfo& u = cur;
                         seg_left = min(x1 - x, u.pos.run);
+                        cur_slice_done = seg_left == u.pos.run;
                         seg_idx = 0;
                         local_row0 = -1;
                         if (PAGED) {
@@ -1080,17 +1139,8 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                                 grid_dep_wait();
                                 synced = true;
                             }
-                            // empty slots until the slot counter has the residue of x
-                            for (int pad = ((x - issued) % NG + NG) % NG; ok && pad > 0; --pad) {
-                                ok = wait_bounded(smem_u32(empty_bar + s), par ^ 1u, s_abort, a.status, kStatusEmptyWaitTimeout);
-                                if (!ok) break;
-                                mbar_arrive(smem_u32(full_bar + s));
-                                ++issued;
-                                if (++s == stages) {
-                                    s = 0;
-                                    par ^= 1u;
-                                }
-                            }
+                            announce(k, x, seg_eff + seg_skip, u);
+                            if (ok) pad_to(x);
                             if (!ok) break;
                             paged_tile = u.pos.tile;
                             if (u.pos.uid < sc.U) {
@@ -1126,6 +1176,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                             }
                             qsrc = a.q + ((size_t)u.qrow * a.q_heads + (size_t)u.head * G) * D;
                         } else {
+                        announce(k, x, seg_left, u);
+                        if (ok) pad_to(x);
+                        if (!ok) break;
                         // rows the append launch of this step writes: a compressed unit's ring, the
                         // last tile of a full unit (waited for when that tile's turn comes, below).
                         // Everything else is older and may be fetched early.
@@ -1265,9 +1318,9 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                 cpar ^= 1u;
                 if (ok) k_claim = *claim_slot;
             }
-            if (ok && wait_bounded(smem_u32(item_empty + di), dpar ^ 1u, s_abort, a.status, kStatusItemWaitTimeout)) {
-                item_desc[di] = make_int4(-1, 0, 0, 0);  // no more work
-                mbar_arrive(smem_u32(item_full + di));
+            if (ok) {
+                UnitInfo none{};
+                announce(-1, 0, 0, none);  // no more work
             }
             if (trace) {
                 my_trace[14] = ns_claim;

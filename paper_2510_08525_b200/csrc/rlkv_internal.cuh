@@ -385,8 +385,8 @@ struct UnitInfo {
     int qrow;        // the unit's G query (and output) rows start at row qrow * q_heads + head * G
     int row0;        // lock-step cache: first pool row of the unit's K rows; its V rows start `vrows` further on
     int vrows;
-    int layer;       // paged cache: the layer (0 in a launch for one layer), the unit's slot among the heads of
-    int slot;        // its class in that layer, and how many heads of that class the layer has
+    int layer;       // the layer (0 in a launch for one layer), the unit's slot among the heads of its class in
+    int slot;        // that layer, and how many heads of that class the layer has
     int nclass;
 };
 
@@ -444,6 +444,9 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         const int nf = (st->full_base[l + 1] - st->full_base[l]) / st->batch;
         const int per_row = full ? nf : st->kv_heads - nf;  // units of this class per batch row of the layer
         const int b = local / per_row, slot = local - b * per_row;
+        u.layer = l;
+        u.slot = slot;
+        u.nclass = per_row;
         u.tiles = full ? a.sched.tf : a.sched.tc;
         u.len = full ? a.len_full : a.len_comp;
         u.b = l * st->batch + b;
@@ -457,7 +460,9 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.tiles = a.sched.tf;
         u.len = a.len_full;
         u.b = u.pos.uid / a.n_full;
-        u.head = a.head_of_slot[u.pos.uid - u.b * a.n_full];
+        u.slot = u.pos.uid - u.b * a.n_full;
+        u.nclass = a.n_full;
+        u.head = a.head_of_slot[u.slot];
         u.vrows = a.rows_full;
         u.row0 = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full);
     } else if (MIXED) {  // the local unit of full unit uid - U
@@ -473,7 +478,9 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.tiles = a.sched.tc;
         u.len = a.len_comp;
         u.b = unit / a.n_comp;
-        u.head = a.head_of_slot[a.n_full + (unit - u.b * a.n_comp)];
+        u.slot = unit - u.b * a.n_comp;
+        u.nclass = a.n_comp;
+        u.head = a.head_of_slot[a.n_full + u.slot];
         u.vrows = a.rows_comp;
         u.row0 = (int)(a.comp_row0 + (long long)unit * 2 * a.rows_comp);
     }
@@ -486,6 +493,31 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.slot = full ? u.pos.uid - u.b * a.n_full : u.pos.uid - a.sched.U - u.b * a.n_comp;
     }
     return u;
+}
+
+// The unit after `u` in the flat tile space, for the producer's walk along an item: inside one region
+// (the whole-unit prefix, a band, the compressed units) the slices of consecutive units of a class
+// follow one another, so the next segment's unit is u's successor and nothing has to be looked up
+// from scratch (locate costs four divisions and a binary search; a compressed unit is two tiles
+// long).  `u` must come from locate or from this function; tile, run and band of the new position are
+// the caller's (they are the region's).  Returns false where the successor lies in the next layer of a
+// whole-step launch or the mode is not covered: the caller then calls locate.
+template <int MODE>
+__device__ inline bool next_unit(const DecodeArgs& a, UnitInfo& u, const StepArgs* st, const unsigned char* heads)
+{
+    if (MODE != kModePlain && MODE != kModeStep) return false;
+    const bool full = u.pos.uid < a.sched.U;
+    ++u.pos.uid;
+    u.row0 += 2 * u.vrows;  // the units of a class lie one after the other in a layer's region of the pool
+    if (++u.slot == u.nclass) {
+        u.slot = 0;
+        ++u.b;
+        if (MODE == kModeStep && u.b == (u.layer + 1) * st->batch) return false;  // the layer's last batch row is done
+    }
+    u.qrow = u.b;
+    if (MODE == kModeStep) u.head = heads[u.layer * st->kv_heads + (full ? u.slot : st->kv_heads - u.nclass + u.slot)];
+    else u.head = a.head_of_slot[(full ? 0 : a.n_full) + u.slot];
+    return true;
 }
 
 // Paged cache: how many tiles of unit `uid` exist.
