@@ -1100,7 +1100,7 @@ decode_kernel(const __grid_constant__ DecodeArgs args, const __grid_constant__ C
                         // end and the region goes on; looked up otherwise
                         bool stepped = false;
                         if (cur_slice_done && x < region_end) {
-                            stepped = next_unit<MODE>(a, cur, stp, s_heads);
+                            stepped = next_unit<MODE>(a, cur, pg, stp, s_heads);
                             cur.pos.tile = region_tile0;
                             cur.pos.run = region_width;
                         }

@@ -501,12 +501,28 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
 // from scratch (locate costs four divisions and a binary search; a compressed unit is two tiles
 // long).  `u` must come from locate or from this function; tile, run and band of the new position are
 // the caller's (they are the region's).  Returns false where the successor lies in the next layer of a
-// whole-step launch or the mode is not covered: the caller then calls locate.
+// whole-step launch, or for the local units of mixed attention: the caller then calls locate.
 template <int MODE>
-__device__ inline bool next_unit(const DecodeArgs& a, UnitInfo& u, const StepArgs* st, const unsigned char* heads)
+__device__ inline bool next_unit(const DecodeArgs& a, UnitInfo& u, const PagedArgs* pg, const StepArgs* st,
+                                 const unsigned char* heads)
 {
-    if (MODE != kModePlain && MODE != kModeStep) return false;
+    if (MODE == kModeMixed) return false;
     const bool full = u.pos.uid < a.sched.U;
+    if (MODE == kModePaged || MODE == kModePagedFp8) {  // u.b: the sequence of the call; rows come from pages
+        const bool whole = pg->step.n_layers > 1;
+        ++u.pos.uid;
+        if (++u.slot == u.nclass) {
+            u.slot = 0;
+            ++u.b;
+            if (whole && u.b == pg->step.batch) return false;  // the layer's last sequence is done
+            const int n = pg->seq_len[u.b];
+            u.len = full ? n : (n < pg->cap ? n : pg->cap);
+        }
+        u.qrow = whole ? u.layer * pg->step.batch + u.b : u.b;
+        if (whole) u.head = heads[u.layer * pg->step.kv_heads + (full ? u.slot : pg->step.kv_heads - u.nclass + u.slot)];
+        else u.head = a.head_of_slot[(full ? 0 : a.n_full) + u.slot];
+        return true;
+    }
     ++u.pos.uid;
     u.row0 += 2 * u.vrows;  // the units of a class lie one after the other in a layer's region of the pool
     if (++u.slot == u.nclass) {
