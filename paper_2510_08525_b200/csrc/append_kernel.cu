@@ -139,7 +139,7 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
             }
             unsigned char* pg = a.pool8 + page_index * (2 * kTile * 128);
             const float inv = (kv ? a.v_inv : a.k_inv)[l * a.kv_heads + h];
-            const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.n + e) * a.kv_heads + h) * a.head_dim + c * 8;
+            const __nv_bfloat16* src = (kv ? a.v : a.k) + ((long long)l * a.n + e) * a.entry_stride + (long long)h * a.head_dim + c * 8;
             const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src));
             const __nv_bfloat16* x = reinterpret_cast<const __nv_bfloat16*>(&bits);
             alignas(8) unsigned char code[8];
@@ -166,7 +166,7 @@ __global__ void __launch_bounds__(256) paged_append_kernel(const __grid_constant
             const int phys = t < a.sink ? t : a.sink + (t - a.sink) % a.window;
             row = comp_row0 + (((long long)seq * n_comp + (-slot - 1)) * 2 + kv) * a.rows_comp + phys;
         }
-        const __nv_bfloat16* src = (kv ? a.v : a.k) + (((long long)l * a.n + e) * a.kv_heads + h) * a.head_dim;
+        const __nv_bfloat16* src = (kv ? a.v : a.k) + ((long long)l * a.n + e) * a.entry_stride + (long long)h * a.head_dim;
         const uint4 bits = __ldg(reinterpret_cast<const uint4*>(src) + c);
         reinterpret_cast<uint4*>(a.pool + row * a.head_dim)[c] = bits;
     }

@@ -112,6 +112,14 @@ inline Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_
     return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0);
 }
 
+}  // namespace rlkv
+struct rlkv_paged;
+namespace rlkv {
+// Internal entry points of the paged cache for the lock-step cache kept in 8 bits (rlkv_api.cu).
+int paged_prefill_strided(rlkv_paged* p, int layer, int slot, const void* k, const void* v, int n_tokens,
+                          long long entry_stride, void* stream);
+uint64_t paged_launch_count(const rlkv_paged* p);
+
 struct DeviceGuard {
     int prev = -1;
     bool ok = true;

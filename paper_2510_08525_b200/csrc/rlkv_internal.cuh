@@ -470,7 +470,9 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.tiles = a.sched.tc;
         u.len = 0;       // its tiles' rows come from local_tile
         u.b = unit / a.n_full;
-        u.head = a.head_of_slot[unit - u.b * a.n_full];
+        u.slot = unit - u.b * a.n_full;
+        u.nclass = a.n_full;
+        u.head = a.head_of_slot[u.slot];
         u.vrows = a.rows_full;
         u.row0 = (int)(a.full_row0 + (long long)unit * 2 * a.rows_full);
     } else {
@@ -501,13 +503,13 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
 // from scratch (locate costs four divisions and a binary search; a compressed unit is two tiles
 // long).  `u` must come from locate or from this function; tile, run and band of the new position are
 // the caller's (they are the region's).  Returns false where the successor lies in the next layer of a
-// whole-step launch, or for the local units of mixed attention: the caller then calls locate.
+// whole-step launch: the caller then calls locate.
 template <int MODE>
 __device__ inline bool next_unit(const DecodeArgs& a, UnitInfo& u, const PagedArgs* pg, const StepArgs* st,
                                  const unsigned char* heads)
 {
-    if (MODE == kModeMixed) return false;
-    const bool full = u.pos.uid < a.sched.U;
+    // (mixed attention: a local unit is addressed like the full unit of the same head)
+    const bool full = u.pos.uid < a.sched.U || MODE == kModeMixed;
     if (MODE == kModePaged || MODE == kModePagedFp8) {  // u.b: the sequence of the call; rows come from pages
         const bool whole = pg->step.n_layers > 1;
         ++u.pos.uid;
@@ -632,6 +634,7 @@ struct PagedAppendArgs {
     int n, t0, first_page;
     int n_layers;               // 1 unless the launch serves every layer
     const LayerDesc* layers;    // device, [n_layers]; unused when n_layers == 1
+    long long entry_stride;     // elements from one entry of k, v to the next (kv_heads * head_dim when contiguous)
     // 8-bit storage (null: 16-bit rows): the pool of pages and rings, 1 / scale per head of the first layer
     // served ([n_layers][kv_heads]), the layer's first page when n_layers == 1
     unsigned char* pool8;

@@ -221,6 +221,7 @@ void fill_append_args(rlkv_paged* p, int layer, const void* k, const void* v, Pa
     a.window = p->window;
     a.n_layers = 1;
     a.layers = nullptr;
+    a.entry_stride = (long long)p->kv_heads * p->head_dim;
     a.pool8 = p->fp8 ? p->dev_base + p->off_pool8 : nullptr;
     a.k_inv = dev_at<float>(p, p->off_scales) + (size_t)layer * p->kv_heads;
     a.v_inv = a.k_inv + (size_t)p->layers * p->kv_heads;
@@ -451,7 +452,18 @@ int rlkv_paged_append(rlkv_paged* p, int layer, const int* slots, int n, const v
 
 int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const void* v, int n_tokens, void* stream)
 {
-    if (!valid_layer(p, layer) || !valid_slot(p, slot) || !k || !v || !aligned16(k) || !aligned16(v) || n_tokens < 1)
+    return rlkv::paged_prefill_strided(p, layer, slot, k, v, n_tokens, p ? (long long)p->kv_heads * p->head_dim : 0, stream);
+}
+
+}  // extern "C"
+
+// rlkv_paged_prefill with the tokens of k and v `entry_stride` elements apart (a multiple of 8): the rows of
+// one batch row inside a [tokens][batch][kv_heads][head_dim] array, for the lock-step cache kept in 8 bits.
+int rlkv::paged_prefill_strided(rlkv_paged* p, int layer, int slot, const void* k, const void* v, int n_tokens,
+                                long long entry_stride, void* stream)
+{
+    if (!valid_layer(p, layer) || !valid_slot(p, slot) || !k || !v || !aligned16(k) || !aligned16(v) || n_tokens < 1 ||
+        entry_stride < (long long)p->kv_heads * p->head_dim || entry_stride % 8 != 0)
         return RLKV_EINVAL;
     int* len = len_of(p, layer);
     const int t0 = len[slot];
@@ -471,7 +483,7 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
         }
     // launches of at most kMaxAppendPages pages each: every launch equals that many single appends,
     // bit for bit, and the launches run in order, so the whole equals n_tokens single appends
-    const size_t row_elems = (size_t)p->kv_heads * p->head_dim;
+    const size_t row_elems = (size_t)entry_stride;
     for (int done = 0; done < n_tokens;) {
         const int t = t0 + done;
         const int page0 = t / kTile;
@@ -482,6 +494,7 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
         fill_append_args(p, layer, static_cast<const __nv_bfloat16*>(k) + (size_t)done * row_elems,
                          static_cast<const __nv_bfloat16*>(v) + (size_t)done * row_elems, a);
         a.prefill = 1;
+        a.entry_stride = entry_stride;
         a.n = count;
         a.t0 = t;
         a.first_page = page0;
@@ -494,6 +507,10 @@ int rlkv_paged_prefill(rlkv_paged* p, int layer, int slot, const void* k, const 
     len[slot] = t0 + n_tokens;
     return RLKV_OK;
 }
+
+uint64_t rlkv::paged_launch_count(const rlkv_paged* p) { return p ? p->launches : 0; }
+
+extern "C" {
 
 // One decode launch (arguments checked by the caller).  `half`: which copy of tickets, claim counter
 // and partials; `overlap`, `dep_wait`: as for the lock-step cache (launch_decode, decode_kernel);
