@@ -69,6 +69,26 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
                       void* device_buf, size_t device_buf_bytes);
 int rlkv_cache_destroy(rlkv_cache* cache);
 
+/* The lock-step cache held in 8 bits: every K and V element of both head classes is stored as an
+ * E4M3 code with one scale per (layer, KV head) for K and one for V (format, rounding and scales as
+ * documented at rlkv_paged_create_fp8 below; k_scale, v_scale: HOST float [layers][kv_heads]).
+ * head_dim must be 128.  The handle is a thin layer over the paged 8-bit cache with one request slot
+ * per batch row and enough pages for every row to reach max_len, so no call finds the free list
+ * empty.  On such a handle rlkv_append, rlkv_prefill, rlkv_decode_attention, rlkv_step,
+ * rlkv_step_host (copies and kernels all on the caller's stream), rlkv_cache_reset (host bookkeeping
+ * only: later work must go to the stream of the earlier), rlkv_set_step_mode, rlkv_set_output_bf16,
+ * rlkv_length, rlkv_step_bytes (a K row and a V row of codes: 2 * head_dim bytes per token),
+ * rlkv_kernel_status, rlkv_launch_count and rlkv_debug_export_head (the codes, one per 16-bit element;
+ * rows that hold no token read as zero) work as documented; rlkv_set_decode_config, the overlapped
+ * per-layer calls, rlkv_decode_attention_static_scratch, rlkv_decode_mixed_attention and
+ * rlkv_debug_trace return RLKV_EINVAL. */
+int rlkv_cache_size_fp8(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                        const uint8_t* head_is_full, int sink, int window, size_t* bytes_out);
+int rlkv_cache_create_fp8(rlkv_cache** out, int layers, int kv_heads, int q_heads, int head_dim,
+                          int batch, int max_len, const uint8_t* head_is_full, int sink, int window,
+                          const float* k_scale, const float* v_scale, void* device_buf,
+                          size_t device_buf_bytes);
+
 /* All lengths back to 0 and the pools re-zeroed (asynchronous on `stream`). */
 int rlkv_cache_reset(rlkv_cache* cache, void* stream);
 

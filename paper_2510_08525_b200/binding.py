@@ -57,6 +57,8 @@ SIGNATURES = {
     "rlkv_paged_size": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
     "rlkv_paged_create": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _sz]),
     "rlkv_paged_size_fp8": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
+    "rlkv_cache_size_fp8": (_ci, [_ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, ctypes.POINTER(_sz)]),
+    "rlkv_cache_create_fp8": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _vp, _vp, _sz]),
     "rlkv_paged_create_fp8": (_ci, [ctypes.POINTER(_vp), _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp, _ci, _ci, _vp, _vp, _vp, _sz]),
     "rlkv_paged_destroy": (_ci, [_vp]),
     "rlkv_paged_seq_open": (_ci, [_vp, ctypes.POINTER(_ci)]),
@@ -147,6 +149,30 @@ def rlkv_cache_create(layers, kv_heads, q_heads, head_dim, batch, max_len, head_
     handle = _vp(0)
     _check(lib.rlkv_cache_create(ctypes.byref(handle), layers, kv_heads, q_heads, head_dim, batch, max_len,
                                  m.ctypes.data, sink, window, _ptr(device_buf), device_buf_bytes))
+    return int(handle.value)
+
+
+def rlkv_cache_size_fp8(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window) -> int:
+    m = _mask(head_is_full)
+    if m.size != layers * kv_heads:
+        raise ValueError("head_is_full must have layers*kv_heads entries")
+    out = _sz(0)
+    _check(lib.rlkv_cache_size_fp8(layers, kv_heads, q_heads, head_dim, batch, max_len, m.ctypes.data, sink, window,
+                                   ctypes.byref(out)))
+    return int(out.value)
+
+
+def rlkv_cache_create_fp8(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window,
+                          k_scale, v_scale, device_buf=None, device_buf_bytes=0) -> int:
+    m = _mask(head_is_full)
+    ks = np.ascontiguousarray(np.asarray(k_scale, dtype=np.float32).reshape(-1))
+    vs = np.ascontiguousarray(np.asarray(v_scale, dtype=np.float32).reshape(-1))
+    if m.size != layers * kv_heads or ks.size != m.size or vs.size != m.size:
+        raise ValueError("head_is_full, k_scale and v_scale must have layers*kv_heads entries")
+    handle = _vp(0)
+    _check(lib.rlkv_cache_create_fp8(ctypes.byref(handle), layers, kv_heads, q_heads, head_dim, batch, max_len,
+                                     m.ctypes.data, sink, window, ks.ctypes.data, vs.ctypes.data,
+                                     _ptr(device_buf), device_buf_bytes))
     return int(handle.value)
 
 

@@ -173,6 +173,12 @@ struct rlkv_cache {
     bool owns_buffer;
     CUtensorMap tmap;
     uint64_t launches;
+    // A cache created by rlkv_cache_create_fp8 keeps its K/V rows as 8-bit codes in a paged cache of
+    // `batch` request slots whose pages are handed out in order (fp8_* below): every call is passed on to
+    // it, and none of the device members above is used.
+    rlkv_paged* fp8;
+    std::vector<int> fp8_slots;   // the request slot of every batch row
+    uint8_t* fp8_staging;         // k, v, q, out of one step, for rlkv_step_host
 };
 
 namespace {
@@ -517,6 +523,54 @@ int step_decode(rlkv_cache* c, int l0, int l1, const void* q, void* out, cudaStr
     return RLKV_OK;
 }
 
+// ---- the lock-step cache kept in 8 bits: a thin layer over the paged cache ------------------------
+int fp8_prefill(rlkv_cache* c, int layer, const void* k, const void* v, int n_tokens, void* stream)
+{
+    if ((long long)c->len[layer] + n_tokens > c->max_len) return RLKV_EFULL;
+    const long long row = (long long)c->kv_heads * c->head_dim;
+    if (n_tokens == 1) {
+        const int rc = rlkv_paged_append(c->fp8, layer, c->fp8_slots.data(), c->batch, k, v, stream);
+        if (rc == RLKV_OK) c->len[layer] += 1;
+        return rc;
+    }
+    for (int b = 0; b < c->batch; ++b) {  // batch row b's tokens lie batch * kv_heads * head_dim elements apart
+        const int rc = paged_prefill_strided(c->fp8, layer, c->fp8_slots[b], static_cast<const __nv_bfloat16*>(k) + b * row,
+                                             static_cast<const __nv_bfloat16*>(v) + b * row, n_tokens, c->batch * row, stream);
+        if (rc) return rc;
+    }
+    c->len[layer] += n_tokens;
+    return RLKV_OK;
+}
+
+int fp8_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* out, void* stream)
+{
+    const int rc = rlkv_paged_step(c->fp8, c->fp8_slots.data(), c->batch, k, v, q, out, stream);
+    if (rc == RLKV_OK)
+        for (int l = 0; l < c->layers; ++l) c->len[l] += 1;
+    return rc;
+}
+
+int fp8_export(rlkv_cache* c, int layer, int b, int h, void* k_host, void* v_host, int* rows_out, int32_t* token_of_slot)
+{
+    // the paged export gives a full head's rows in token order, which is this cache's physical order;
+    // rows that hold no token are reported as zeros
+    const bool full = c->is_full[(size_t)layer * c->kv_heads + h] != 0;
+    const int rows = full ? c->max_len : c->sink + c->window;
+    memset(k_host, 0, (size_t)rows * c->head_dim * 2);
+    memset(v_host, 0, (size_t)rows * c->head_dim * 2);
+    for (int s = 0; s < rows; ++s) token_of_slot[s] = -1;
+    int got = 0;
+    const int rc = rlkv_paged_debug_export_head(c->fp8, layer, c->fp8_slots[b], h, k_host, v_host, &got, token_of_slot);
+    if (rc) return rc;
+    for (int s = 0; s < rows; ++s)  // a ring slot no token has reached since the reset may hold older codes
+        if (token_of_slot[s] < 0) {
+            memset(static_cast<uint8_t*>(k_host) + (size_t)s * c->head_dim * 2, 0, (size_t)c->head_dim * 2);
+            memset(static_cast<uint8_t*>(v_host) + (size_t)s * c->head_dim * 2, 0, (size_t)c->head_dim * 2);
+        }
+    *rows_out = rows;
+    return RLKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -569,6 +623,8 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     c->trace_on = 0;
     c->out_bf16 = 0;
     c->step_mode = 0;
+    c->fp8 = nullptr;
+    c->fp8_staging = nullptr;
     c->claims[0] = c->claims[1] = 0;
     c->in_stream = c->out_stream = nullptr;
     c->ev_step[0] = c->ev_step[1] = c->ev_done = nullptr;
@@ -672,10 +728,101 @@ int rlkv_cache_create(rlkv_cache** out, int layers, int kv_heads, int q_heads, i
     return RLKV_OK;
 }
 
+namespace {
+struct Fp8Sizes {
+    size_t paged, kv, q, out, total;
+};
+int fp8_sizes(Fp8Sizes& z, int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+              const uint8_t* head_is_full, int sink, int window)
+{
+    int rc = check_shape(layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    const int pages = batch * ((max_len + kTile - 1) / kTile);  // every row can reach max_len: no call ever finds the free list empty
+    rc = rlkv_paged_size_fp8(layers, kv_heads, q_heads, head_dim, batch, pages, max_len, head_is_full, sink, window, &z.paged);
+    if (rc) return rc;
+    z.paged = align_up(z.paged, 1024);
+    z.kv = align_up((size_t)layers * batch * kv_heads * head_dim * 2, 256);
+    z.q = align_up((size_t)layers * batch * q_heads * head_dim * 2, 256);
+    z.out = 2 * z.q;
+    z.total = z.paged + 2 * z.kv + z.q + z.out;
+    return RLKV_OK;
+}
+}  // namespace
+
+int rlkv_cache_size_fp8(int layers, int kv_heads, int q_heads, int head_dim, int batch, int max_len,
+                        const uint8_t* head_is_full, int sink, int window, size_t* bytes_out)
+{
+    if (!bytes_out) return RLKV_EINVAL;
+    Fp8Sizes z;
+    const int rc = fp8_sizes(z, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    *bytes_out = z.total;
+    return RLKV_OK;
+}
+
+int rlkv_cache_create_fp8(rlkv_cache** out, int layers, int kv_heads, int q_heads, int head_dim, int batch,
+                          int max_len, const uint8_t* head_is_full, int sink, int window, const float* k_scale,
+                          const float* v_scale, void* device_buf, size_t device_buf_bytes)
+{
+    if (!out) return RLKV_EINVAL;
+    *out = nullptr;
+    if (!k_scale || !v_scale) return RLKV_EINVAL;
+    Fp8Sizes z;
+    int rc = fp8_sizes(z, layers, kv_heads, q_heads, head_dim, batch, max_len, head_is_full, sink, window);
+    if (rc) return rc;
+    rlkv_cache* c = new (std::nothrow) rlkv_cache();
+    if (!c) return RLKV_ENOMEM;
+    c->layers = layers; c->kv_heads = kv_heads; c->q_heads = q_heads; c->head_dim = head_dim;
+    c->batch = batch; c->max_len = max_len; c->sink = sink; c->window = window;
+    c->dev_base = nullptr; c->owns_buffer = false; c->launches = 0;
+    c->trace_on = 0; c->out_bf16 = 0; c->step_mode = 0;
+    c->fp8 = nullptr; c->fp8_staging = nullptr;
+    c->in_stream = c->out_stream = nullptr;
+    c->ev_step[0] = c->ev_step[1] = c->ev_done = nullptr;
+    for (int i = 0; i < 4; ++i) c->ev_in[i] = c->ev_out[i] = nullptr;
+    c->is_full.assign(head_is_full, head_is_full + (size_t)layers * kv_heads);
+    c->len.assign(layers, 0);
+    auto fail = [&](int code) {
+        if (c->fp8) rlkv_paged_destroy(c->fp8);
+        if (c->owns_buffer && c->dev_base) cudaFree(c->dev_base);
+        delete c;
+        return code;
+    };
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
+    if (device_buf) {
+        if ((reinterpret_cast<uintptr_t>(device_buf) & 1023u) != 0) return fail(RLKV_EINVAL);
+        if (device_buf_bytes < z.total) return fail(RLKV_ENOMEM);
+        c->dev_base = static_cast<uint8_t*>(device_buf);
+    } else {
+        void* p = nullptr;
+        e = cudaMalloc(&p, z.total);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return fail(RLKV_ENOMEM);
+        }
+        c->dev_base = static_cast<uint8_t*>(p);
+        c->owns_buffer = true;
+    }
+    c->fp8_staging = c->dev_base + z.paged;
+    const int pages = batch * ((max_len + kTile - 1) / kTile);
+    rc = rlkv_paged_create_fp8(&c->fp8, layers, kv_heads, q_heads, head_dim, batch, pages, max_len, head_is_full, sink,
+                               window, k_scale, v_scale, c->dev_base, z.paged);
+    if (rc) return fail(rc);
+    c->fp8_slots.assign(batch, -1);
+    for (int b = 0; b < batch; ++b) {
+        rc = rlkv_paged_seq_open(c->fp8, &c->fp8_slots[b]);
+        if (rc) return fail(rc);
+    }
+    *out = c;
+    return RLKV_OK;
+}
+
 int rlkv_cache_destroy(rlkv_cache* c)
 {
     if (!c) return RLKV_EINVAL;
     int rc = RLKV_OK;
+    if (c->fp8) rc = rlkv_paged_destroy(c->fp8);  // synchronises the device; the buffer is this handle's
     {
         DeviceGuard g(c->device);
         destroy_copy_objects(c);
@@ -694,6 +841,20 @@ int rlkv_cache_reset(rlkv_cache* c, void* stream)
     if (!c) return RLKV_EINVAL;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    if (c->fp8) {
+        // Host bookkeeping only: every row's slot is closed (its pages go back to the free list) and
+        // opened again.  Work enqueued later on the stream of the earlier calls runs after them.
+        for (int b = 0; b < c->batch; ++b) {
+            int rc = rlkv_paged_seq_close(c->fp8, c->fp8_slots[b]);
+            if (rc) return rc;
+        }
+        for (int b = 0; b < c->batch; ++b) {
+            int rc = rlkv_paged_seq_open(c->fp8, &c->fp8_slots[b]);
+            if (rc) return rc;
+        }
+        std::fill(c->len.begin(), c->len.end(), 0);
+        return RLKV_OK;
+    }
     int rc = zero_state(c, static_cast<cudaStream_t>(stream));
     if (rc) return rc;
     std::fill(c->len.begin(), c->len.end(), 0);
@@ -703,6 +864,7 @@ int rlkv_cache_reset(rlkv_cache* c, void* stream)
 
 int rlkv_set_decode_config(rlkv_cache* c, int ctas_per_sm, int stages, int consumer_groups, int item_tiles)
 {
+    if (c && c->fp8) return RLKV_EINVAL;  // the paged launches behind an 8-bit cache have one configuration
     if (!c || ctas_per_sm < 0 || ctas_per_sm > 2 || stages < 0 || stages == 1 || stages > 8 ||
         consumer_groups < 0 || consumer_groups > kMaxConsumerGroups ||
         (item_tiles != 0 && (item_tiles < kMinItemTiles || item_tiles > 1024)))
@@ -731,6 +893,7 @@ int rlkv_prefill(rlkv_cache* c, int layer, const void* k, const void* v, int n_t
     if ((long long)c->len[layer] + n_tokens > c->max_len) return RLKV_EFULL;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    if (c->fp8) return fp8_prefill(c, layer, k, v, n_tokens, stream);
     return do_append(c, layer, k, v, n_tokens, static_cast<cudaStream_t>(stream));
 }
 
@@ -740,12 +903,13 @@ int rlkv_decode_attention(rlkv_cache* c, int layer, const void* q, void* out, vo
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    if (c->fp8) return rlkv_paged_decode_attention(c->fp8, layer, c->fp8_slots.data(), c->batch, q, out, stream);
     return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream));
 }
 
 int rlkv_append_overlapped(rlkv_cache* c, int layer, const void* k, const void* v, void* stream)
 {
-    if (!valid_layer(c, layer) || !k || !v || !aligned16(k) || !aligned16(v)) return RLKV_EINVAL;
+    if (!valid_layer(c, layer) || c->fp8 || !k || !v || !aligned16(k) || !aligned16(v)) return RLKV_EINVAL;
     if (c->len[layer] + 1 > c->max_len) return RLKV_EFULL;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
@@ -754,7 +918,7 @@ int rlkv_append_overlapped(rlkv_cache* c, int layer, const void* k, const void* 
 
 int rlkv_decode_attention_overlapped(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
 {
-    if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (!valid_layer(c, layer) || c->fp8 || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
@@ -763,7 +927,8 @@ int rlkv_decode_attention_overlapped(rlkv_cache* c, int layer, const void* q, vo
 
 int rlkv_layer_step_overlapped(rlkv_cache* c, int layer, const void* k, const void* v, const void* q, void* out, void* stream)
 {
-    if (!valid_layer(c, layer) || !k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) || !aligned16(out))
+    if (!valid_layer(c, layer) || c->fp8 || !k || !v || !q || !out || !aligned16(k) || !aligned16(v) || !aligned16(q) ||
+        !aligned16(out))
         return RLKV_EINVAL;
     if (c->len[layer] + 1 > c->max_len) return RLKV_EFULL;
     DeviceGuard g(c->device);
@@ -776,7 +941,7 @@ int rlkv_layer_step_overlapped(rlkv_cache* c, int layer, const void* k, const vo
 
 int rlkv_decode_attention_static_scratch(rlkv_cache* c, int layer, const void* q, void* out, void* stream)
 {
-    if (!valid_layer(c, layer) || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (!valid_layer(c, layer) || c->fp8 || !q || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
@@ -788,6 +953,7 @@ size_t rlkv_static_scratch_bytes(void) { return kStaticScratchBytes; }
 int rlkv_set_step_mode(rlkv_cache* c, int mode)
 {
     if (!c || mode < 0 || mode > 2) return RLKV_EINVAL;
+    if (c->fp8) return rlkv_paged_set_step_mode(c->fp8, mode);
     if (mode == 2 && !c->lay.step_in_one_launch) return RLKV_EINVAL;
     c->step_mode = mode;
     return RLKV_OK;
@@ -796,13 +962,17 @@ int rlkv_set_step_mode(rlkv_cache* c, int mode)
 int rlkv_set_output_bf16(rlkv_cache* c, int on)
 {
     if (!c) return RLKV_EINVAL;
+    if (c->fp8) {
+        const int rc = rlkv_paged_set_output_bf16(c->fp8, on);
+        if (rc) return rc;
+    }
     c->out_bf16 = on ? 1 : 0;
     return RLKV_OK;
 }
 
 int rlkv_decode_mixed_attention(rlkv_cache* c, int layer, const void* q, const float* alpha, void* out, void* stream)
 {
-    if (!valid_layer(c, layer) || !q || !alpha || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
+    if (!valid_layer(c, layer) || c->fp8 || !q || !alpha || !out || !aligned16(q) || !aligned16(out)) return RLKV_EINVAL;
     if ((reinterpret_cast<uintptr_t>(alpha) & 3u) != 0) return RLKV_EINVAL;
     if (c->lay.n_comp[layer] != 0) return RLKV_EINVAL;  // the full branch needs every token of every head
     if (c->len[layer] < 1) return RLKV_EEMPTY;
@@ -819,6 +989,7 @@ int rlkv_step(rlkv_cache* c, const void* k, const void* v, const void* q, void* 
         if (c->len[l] >= c->max_len) return RLKV_EFULL;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    if (c->fp8) return fp8_step(c, k, v, q, out, stream);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t kv_layer = (size_t)c->batch * c->kv_heads * c->head_dim;
     const size_t q_layer = (size_t)c->batch * c->q_heads * c->head_dim;
@@ -851,6 +1022,19 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t kv_bytes = (size_t)c->layers * c->batch * c->kv_heads * c->head_dim * 2;
     const size_t q_bytes = (size_t)c->layers * c->batch * c->q_heads * c->head_dim * 2;
+    if (c->fp8) {  // in, step, out, all on the caller's stream
+        uint8_t* dk = c->fp8_staging;
+        uint8_t* dv = dk + align_up(kv_bytes, 256);
+        uint8_t* dq = dv + align_up(kv_bytes, 256);
+        uint8_t* dout = dq + align_up(q_bytes, 256);
+        RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, s));
+        RLKV_CUDA(cudaMemcpyAsync(dv, v_host, kv_bytes, cudaMemcpyHostToDevice, s));
+        RLKV_CUDA(cudaMemcpyAsync(dq, q_host, q_bytes, cudaMemcpyHostToDevice, s));
+        const int rc = fp8_step(c, dk, dv, dq, dout, stream);
+        if (rc) return rc;
+        RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * (c->out_bf16 ? 1 : 2), cudaMemcpyDeviceToHost, s));
+        return RLKV_OK;
+    }
     const int chunks = c->layers >= 8 ? 4 : 1;
     if (chunks == 1 || c->layers > kMaxStepLayers) {
         uint8_t* dk = c->dev_base + c->lay.off_k;
@@ -925,6 +1109,7 @@ int rlkv_length(const rlkv_cache* c, int layer, int* len_out)
 int rlkv_step_bytes(const rlkv_cache* c, int layer, uint64_t* kv_bytes_out)
 {
     if (!valid_layer(c, layer) || !kv_bytes_out) return RLKV_EINVAL;
+    if (c->fp8) return rlkv_paged_step_bytes(c->fp8, layer, c->fp8_slots.data(), c->batch, kv_bytes_out);
     const uint64_t n = (uint64_t)c->len[layer], cap = (uint64_t)c->sink + c->window;
     const uint64_t row_pair = (uint64_t)c->head_dim * 2 * 2;  // one K row + one V row
     const uint64_t rows = (uint64_t)c->lay.n_full[layer] * n + (uint64_t)c->lay.n_comp[layer] * (n < cap ? n : cap);
@@ -940,6 +1125,7 @@ int rlkv_debug_export_head(rlkv_cache* c, int layer, int b, int h, void* k_host,
         return RLKV_EINVAL;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    if (c->fp8) return fp8_export(c, layer, b, h, k_host, v_host, rows_out, token_of_slot);
     RLKV_CUDA(cudaDeviceSynchronize());
     const int slot = c->slot_of_head[layer * c->kv_heads + h];
     const int n = c->len[layer];
@@ -978,6 +1164,7 @@ int rlkv_debug_export_head(rlkv_cache* c, int layer, int b, int h, void* k_host,
 int rlkv_kernel_status(rlkv_cache* c, int* status_out)
 {
     if (!c || !status_out) return RLKV_EINVAL;
+    if (c->fp8) return rlkv_paged_kernel_status(c->fp8, status_out);
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
     RLKV_CUDA(cudaDeviceSynchronize());
@@ -987,7 +1174,7 @@ int rlkv_kernel_status(rlkv_cache* c, int* status_out)
 
 int rlkv_debug_trace(rlkv_cache* c, int enable, unsigned long long* words_host, int* ctas_out)
 {
-    if (!c) return RLKV_EINVAL;
+    if (!c || c->fp8) return RLKV_EINVAL;
     if (words_host) {
         if (!ctas_out) return RLKV_EINVAL;
         DeviceGuard g(c->device);
@@ -1069,7 +1256,7 @@ int rlkv_debug_step_plan(int n_launches, int follows_append, int* overlap_out, i
 int rlkv_launch_count(const rlkv_cache* c, uint64_t* launches_out)
 {
     if (!c || !launches_out) return RLKV_EINVAL;
-    *launches_out = c->launches;
+    *launches_out = c->fp8 ? paged_launch_count(c->fp8) : c->launches;
     return RLKV_OK;
 }
 
