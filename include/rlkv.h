@@ -188,9 +188,9 @@ size_t rlkv_static_scratch_bytes(void);
  * otherwise.  q: device bf16 [batch][q_heads][head_dim]; alpha: DEVICE fp32 [kv_heads], the gates of
  * this layer, read when the kernel runs and used as they are (the paper keeps them in [0, 1]; the
  * library does not check); out: device fp32 [batch][q_heads][head_dim] (bf16 after
- * rlkv_set_output_bf16).  One launch: the K/V rows are streamed once for the full branch, the sink and
- * window rows a second time for the local branch (sink + window rows per head, normally out of the
- * L2); whichever CTA delivers the last piece of a head's two branches merges both and writes
+ * rlkv_set_output_bf16).  One launch and one pass: every K/V row is read once -- the softmax state
+ * over the sink and window rows is the local branch and, merged with the state over the rows between
+ * them, the full branch; whichever CTA delivers the last piece of a head merges them and writes
  * alpha * full + (1 - alpha) * local once.  K and V rows are assumed finite.
  * RLKV_EEMPTY if length(layer) == 0. */
 int rlkv_decode_mixed_attention(rlkv_cache* cache, int layer, const void* q, const float* alpha,

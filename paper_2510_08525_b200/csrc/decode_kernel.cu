@@ -313,12 +313,14 @@ struct Smem {
 // (Everything comes by value or from shared memory: a reference to kernel parameters would turn
 // every use into a slow generic load inside this non-inlined function.)
 // MIXED (Eq. 1 of the paper): `units` lists (batch row, head) pairs; entries 0 .. R of a pair's list
-// are the records of its full unit, entry kMaxRounds + 1 those of its local unit.  Both are merged
-// and the rows get gate * full + (1 - gate) * local, written once: no clearing, no atomics, and the
+// are the records of its first unit -- the tokens between the sink and the window --, entry
+// kMaxRounds + 1 those of its local unit (sink and window).  No token is read twice: the full branch
+// of Eq. 1 is the merge of ALL the pair's records, the local branch the merge of the local unit's, and
+// the rows get gate * full + (1 - gate) * local, written once: no clearing, no atomics, and the
 // result does not depend on which unit finished first.
 constexpr int kListStride = kMaxRounds + 2;  // (first record, count) per band, then the local unit's (MIXED)
-template <int D, bool MIXED>
-__device__ __noinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
+template <int D>
+__device__ __noinline__ void merge_units_plain(const float* partials, float* out, int G, int R, const int2* units,
                                          const int2* lists, int n, int t, int nt, bool dry,
                                          unsigned long long* stamp, const float* alpha, int U, int q_heads, int out_bf16)
 {
@@ -337,7 +339,7 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
                 const int g = e / D4;
                 float4 res = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll 1
-                for (int part = 0; part < (MIXED ? 2 : 1); ++part) {  // the full unit's records, then the local unit's
+                for (int part = 0; part < (1); ++part) {  // the full unit's records, then the local unit's
                 const int b0 = part ? NB - 1 : 0, b1 = part ? NB : R + 1;
                 int F = 0;
                 for (int r = b0; r < b1; ++r) F += li[r].y;
@@ -384,7 +386,7 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
                 }
                 if (stamp && t == 0 && j == ul) stamp[3] = global_timer_ns();
                 float inv = 1.f / L;
-                if (MIXED) {
+                if (false) {
                     const float gate = __ldg(alpha + (units[j].y % q_heads) / G);
                     inv *= part ? 1.f - gate : gate;
                 }
@@ -405,6 +407,129 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
     }
 }
 
+// Mixed attention (see above): one pass over all records of a pair, the local unit's also into a second state.
+template <int D>
+__device__ __noinline__ void merge_units_mixed(const float* partials, float* out, int G, int R, const int2* units,
+                                         const int2* lists, int n, int t, int nt, bool dry,
+                                         unsigned long long* stamp, const float* alpha, int U, int q_heads, int out_bf16)
+{
+    constexpr int D4 = D / 4, CH = 16, NB = kListStride;
+    constexpr bool MIXED = true;
+    const int E = G * D4;
+    const int PF = partial_floats(D, G), PH = partial_head_floats(G);
+    __threadfence();
+    if (stamp && t == 0) stamp[0] = global_timer_ns();
+    const bool wide = nt >= E;                  // enough threads for one piece each, of nt / E units at a time
+    const int unit_lanes = wide ? nt / E : 1;
+    const int ul = wide ? t / E : 0;
+    if (ul < unit_lanes) {
+        for (int j = ul; j < n; j += unit_lanes) {
+            const int2* li = lists + j * NB;
+            for (int e = wide ? t - ul * E : t; e < E; e += wide ? E : nt) {
+                const int g = e / D4;
+                // MIXED: all records of the pair make the full branch (list entries R + 1 .. NB - 2 are empty);
+                // the local unit's, which come last, also go into a second state: one pass, one trip
+                const int b1 = MIXED ? NB : R + 1;
+                int F = 0;
+                for (int r = 0; r < b1; ++r) F += li[r].y;
+                const int first_local = MIXED ? F - li[NB - 1].y : F;
+                float M = kNegBig, L = 0.f, M2 = kNegBig, L2 = 0.f;
+                float4 O = make_float4(0.f, 0.f, 0.f, 0.f), O2 = make_float4(0.f, 0.f, 0.f, 0.f);
+                int band = 0, off = 0;  // the record with merge index c0 is record `off` of band `band`
+                for (int c0 = 0; c0 < F; c0 += CH) {
+                    float mm[CH], ll[CH];
+                    float4 oo[CH];
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const bool on = c0 + c < F;
+                        if (on)
+                            while (off >= li[band].y) {
+                                off -= li[band].y;
+                                ++band;
+                            }
+                        const float* pc = partials + (size_t)(on ? li[band].x + off : 0) * PF;
+                        mm[c] = on ? __ldcg(pc + g) : kNegBig;
+                        ll[c] = on ? __ldcg(pc + G + g) : 0.f;
+                        oo[c] = on ? __ldcg(reinterpret_cast<const float4*>(pc + PH) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                        ++off;
+                    }
+                    float Mc = M;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) Mc = fmaxf(Mc, mm[c]);
+                    if (stamp && t == 0 && j == ul && c0 == 0) stamp[2] = global_timer_ns();
+                    const float keep = exp2f(M - Mc);
+                    L *= keep;
+                    O.x *= keep;
+                    O.y *= keep;
+                    O.z *= keep;
+                    O.w *= keep;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const float w = exp2f(mm[c] - Mc);
+                        L += ll[c] * w;
+                        O.x += oo[c].x * w;
+                        O.y += oo[c].y * w;
+                        O.z += oo[c].z * w;
+                        O.w += oo[c].w * w;
+                    }
+                    M = Mc;
+                    if (MIXED && c0 + CH > first_local) {  // the batch holds records of the local unit
+                        float Mc2 = M2;
+#pragma unroll
+                        for (int c = 0; c < CH; ++c)
+                            if (c0 + c >= first_local) Mc2 = fmaxf(Mc2, mm[c]);
+                        const float keep2 = exp2f(M2 - Mc2);
+                        L2 *= keep2;
+                        O2.x *= keep2;
+                        O2.y *= keep2;
+                        O2.z *= keep2;
+                        O2.w *= keep2;
+#pragma unroll
+                        for (int c = 0; c < CH; ++c)
+                            if (c0 + c >= first_local) {
+                                const float w = exp2f(mm[c] - Mc2);
+                                L2 += ll[c] * w;
+                                O2.x += oo[c].x * w;
+                                O2.y += oo[c].y * w;
+                                O2.z += oo[c].z * w;
+                                O2.w += oo[c].w * w;
+                            }
+                        M2 = Mc2;
+                    }
+                }
+                if (stamp && t == 0 && j == ul) stamp[3] = global_timer_ns();
+                float inv = 1.f / L;
+                float4 res;
+                if (MIXED) {
+                    const float gate = __ldg(alpha + (units[j].y % q_heads) / G);
+                    inv *= gate;
+                    const float inv2 = (1.f - gate) / L2;
+                    res = make_float4(O.x * inv + O2.x * inv2, O.y * inv + O2.y * inv2, O.z * inv + O2.z * inv2,
+                                      O.w * inv + O2.w * inv2);
+                } else {
+                    res = make_float4(O.x * inv, O.y * inv, O.z * inv, O.w * inv);
+                }
+                if (!dry) {
+                    if (out_bf16)
+                        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(out) + (size_t)units[j].y * D + e * 4) =
+                            make_uint2(pack_bf16(res.x, res.y), pack_bf16(res.z, res.w));
+                    else
+                        *reinterpret_cast<float4*>(out + (size_t)units[j].y * D + e * 4) = res;
+                }
+            }
+        }
+    }
+}
+
+template <int D, bool MIXED>
+__device__ __forceinline__ void merge_units(const float* partials, float* out, int G, int R, const int2* units,
+                                            const int2* lists, int n, int t, int nt, bool dry,
+                                            unsigned long long* stamp, const float* alpha, int U, int q_heads, int out_bf16)
+{
+    if constexpr (MIXED) merge_units_mixed<D>(partials, out, G, R, units, lists, n, t, nt, dry, stamp, alpha, U, q_heads, out_bf16);
+    else merge_units_plain<D>(partials, out, G, R, units, lists, n, t, nt, dry, stamp, alpha, U, q_heads, out_bf16);
+}
+
 // ---------------------------------------------------------------------------------------------
 // The kernel.  Warp roles: 0 .. 4*NG-1 consumers (group = warp / 4); then one producer warp (TMA);
 // one claim warp (fetches the next work item from the global counter while the producer streams the
@@ -419,11 +544,13 @@ __device__ __noinline__ void merge_units(const float* partials, float* out, int 
 // same group (stages is a multiple of NG).  Where an item starts on the wrong residue the producer
 // issues an empty slot first.
 //
-// MIXED: the mixed attention of Eq. 1.  The schedule's second class holds, for every full unit, a
-// LOCAL unit over the same head's sink and window rows; its tiles start at whatever row the window
-// starts (a TMA box may start at any row) and are masked past their valid rows.  Every segment of
-// either unit leaves a partial record; the pair's ticket counts the records of both, and whoever
-// delivers the last one merges both units and writes gate * full + (1 - gate) * local once.
+// MIXED: the mixed attention of Eq. 1, every row read once.  The first class of units covers the rows
+// between sink and window of every (batch row, head), the second class holds its LOCAL unit over the
+// sink and window rows; tiles start at whatever row the range starts (a TMA box may start at any row)
+// and are masked past their valid rows.  Every segment of either unit leaves a partial record; the
+// pair's ticket counts the records of both, and whoever delivers the last one merges them -- all
+// records for the full branch, the local unit's for the local branch -- and writes
+// gate * full + (1 - gate) * local once.
 //
 // kModeStep: a whole decode step.  The full units of all layers are one list and so are the compressed
 // units (every layer holds the same number of tokens); a unit's layer, rows, query and output rows are

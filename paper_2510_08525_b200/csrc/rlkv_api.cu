@@ -245,8 +245,10 @@ int do_append(rlkv_cache* c, int layer, const void* k, const void* v, int n_toke
 
 // Everything of a decode launch except where its split-KV work area lives.  Returns the grid size
 // in *grid_out.
-// `alpha` != null: a mixed-attention launch (every head of the layer is full): the second class of
-// units are the local units, one per (batch row, head), over the head's sink and window rows.
+// `alpha` != null: a mixed-attention launch (every head of the layer is full, and the layer holds more
+// than sink + window tokens): the first class of units covers the tokens between the sink and the
+// window, the second class are the local units, one per (batch row, head), over the head's sink and
+// window rows.  No row is read twice: the full branch of Eq. 1 merges both units' records.
 int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, DecodeArgs& a, int* grid_out,
                       bool in_step = false, const float* alpha = nullptr)
 {
@@ -277,6 +279,7 @@ int build_decode_args(rlkv_cache* c, int layer, const void* q, void* out, Decode
     a.local_sink_tiles = (a.local_sink + kTile - 1) / kTile;
     a.local_win0 = n - c->window > c->sink ? n - c->window : c->sink;  // first token of the window
     a.local_win_len = n > a.local_win0 ? n - a.local_win0 : 0;
+    if (alpha) a.len_full = n - c->window - c->sink;  // > 0: the caller sends shorter layers to the plain kernel
     const int tiles_full = (a.len_full + kTile - 1) / kTile;
     const int tiles_comp = alpha ? a.local_sink_tiles + (a.local_win_len + kTile - 1) / kTile : (a.len_comp + kTile - 1) / kTile;
     const int second_class = alpha ? a.n_full : a.n_comp;  // units per batch row beside the full ones
@@ -978,6 +981,8 @@ int rlkv_decode_mixed_attention(rlkv_cache* c, int layer, const void* q, const f
     if (c->len[layer] < 1) return RLKV_EEMPTY;
     DeviceGuard g(c->device);
     if (!g.ok) return RLKV_ECUDA;
+    // up to sink + window tokens every token is local: both branches of Eq. 1 are the plain attention
+    if (c->len[layer] <= c->sink + c->window) return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream));
     return do_decode(c, layer, q, out, static_cast<cudaStream_t>(stream), 0, false, false, nullptr, alpha);
 }
 

@@ -294,11 +294,13 @@ struct DecodeArgs {
     float scale_log2;           // log2(e) / sqrt(head_dim)
     int trace_on;
     int out_bf16;               // results are rounded to bf16 (nearest even) when they are stored
-    // Mixed attention (paper, Eq. 1; MIXED kernels only).  Every head of the layer is full; beside
-    // the FULL unit of each (batch row, head) the schedule's second class holds a LOCAL unit over
-    // the same rows restricted to the sink and the window: tiles 0 .. local_sink_tiles-1 cover rows
-    // [0, local_sink), the tiles after them rows [local_win0, local_win0 + local_win_len).  Both
-    // units add their weighted result into `out`, which the host clears before the launch.
+    // Mixed attention (paper, Eq. 1; MIXED kernels only).  Every head of the layer is full and holds
+    // more than sink + window tokens.  The first class of units covers, per (batch row, head), the
+    // len_full rows between the sink and the window (from row local_sink on); the second class holds a
+    // LOCAL unit over the sink and the window: tiles 0 .. local_sink_tiles-1 cover rows
+    // [0, local_sink), the tiles after them rows [local_win0, local_win0 + local_win_len).  No row
+    // belongs to both; the local branch of Eq. 1 is the merge of the local unit's partial records, the
+    // full branch the merge of both units' (merge_units).
     // A launch that also appends the step's token (lock-step cache, one layer): the caller's new rows,
     // [batch][kv_heads][head_dim]; token len_full - 1 of every head is written by the CTA that reads the
     // tile it belongs to (row len_full - 1 of a full head, the ring slot of a compressed head).  Null otherwise.
@@ -465,6 +467,9 @@ __device__ inline UnitInfo locate(const DecodeArgs& a, int x, const PagedArgs* p
         u.head = a.head_of_slot[u.slot];
         u.vrows = a.rows_full;
         u.row0 = (int)(a.full_row0 + (long long)u.pos.uid * 2 * a.rows_full);
+        // mixed attention: the first class covers the tokens between the sink and the window only (len_full
+        // of them, from row local_sink on); sink and window are read once, by the local unit
+        if (MIXED) u.row0 += a.local_sink;
     } else if (MIXED) {  // the local unit of full unit uid - U
         const int unit = u.pos.uid - a.sched.U;
         u.tiles = a.sched.tc;
