@@ -835,7 +835,7 @@ def run_ours(args, w, mask):
         pl, reps = w.layers, max(K, 8)
         n = w.context + 1
         pmask = mask[:pl * w.kv_heads]
-        spread = [max(1, int(round(n * (0.25 + 1.5 * i / max(1, w.batch - 1))))) for i in range(w.batch)]
+        spread = harness.paged_spread_lengths(n, w.batch)
         paged = {"workload": f"the {pl} layers of the {w.name} mask, {w.batch} sequences; launch_us: rlkv_paged_decode_attention "
                              f"launches back to back; in_step: rlkv_paged_step (one append launch, one attention launch over all layers)"}
         variants = [("uniform", [n] * w.batch, False), ("ragged", spread, False)]
@@ -847,14 +847,7 @@ def run_ours(args, w, mask):
             pc = harness.PagedCache(pl, w.kv_heads, w.q_heads, w.head_dim, w.batch, pages, max(lens) + 128, pmask,
                                     w.sink, w.window, device=dev, k_scale=scales, v_scale=scales)
             slots = [pc.open_seq() for _ in lens]
-            for i, x in enumerate(lens):
-                for l in range(pl):
-                    for t0 in range(0, x, 4096):
-                        t1 = min(x, t0 + 4096)
-                        kk = synth.rows(w.seed + 1 + i, synth.STREAM_K, l, t0, t1, 1, w.kv_heads, w.head_dim, dev)
-                        vv = synth.rows(w.seed + 1 + i, synth.STREAM_V, l, t0, t1, 1, w.kv_heads, w.head_dim, dev)
-                        pc.prefill(l, slots[i], kk.reshape(t1 - t0, w.kv_heads, w.head_dim),
-                                   vv.reshape(t1 - t0, w.kv_heads, w.head_dim))
+            harness.fill_paged(pc, w, slots, lens)
             q = q0
             pout = torch.empty((pl, w.batch, w.q_heads, w.head_dim), dtype=torch.float32, device=dev)
             lreps = max(2, (reps * 4) // pl)

@@ -170,3 +170,34 @@ class PagedCache:
 
     def status(self) -> int:
         return rl.rlkv_paged_kernel_status(self.handle)
+
+
+def paged_seq_seed(w: synth.Workload, i: int) -> int:
+    """Sequence i of a paged batch draws its rows from a generator of its own (batch 1)."""
+    return w.seed + 1 + i
+
+
+def fill_paged(pc: PagedCache, w: synth.Workload, slots, lens, chunk: int = 4096) -> None:
+    """Prefill tokens 0 .. lens[i]-1 of every layer of sequence slots[i] from the seeded generator."""
+    for i, x in enumerate(lens):
+        for layer in range(pc.layers):
+            for t0 in range(0, x, chunk):
+                t1 = min(x, t0 + chunk)
+                kk = synth.rows(paged_seq_seed(w, i), synth.STREAM_K, layer, t0, t1, 1, w.kv_heads, w.head_dim, pc.device)
+                vv = synth.rows(paged_seq_seed(w, i), synth.STREAM_V, layer, t0, t1, 1, w.kv_heads, w.head_dim, pc.device)
+                pc.prefill(layer, slots[i], kk.reshape(t1 - t0, w.kv_heads, w.head_dim),
+                           vv.reshape(t1 - t0, w.kv_heads, w.head_dim))
+    torch.cuda.synchronize(pc.device)
+
+
+def paged_step_inputs(pc: PagedCache, w: synth.Workload, lens):
+    """k, v [layers][n][Hkv][D], q [layers][n][Hq][D] (bf16) of the step that appends token lens[i] to sequence i."""
+    def stack(stream, heads):
+        return torch.stack([torch.cat([synth.rows(paged_seq_seed(w, i), stream, layer, x, x + 1, 1, heads, w.head_dim, pc.device)[0]
+                                       for i, x in enumerate(lens)]) for layer in range(pc.layers)]).contiguous()
+    return stack(synth.STREAM_K, w.kv_heads), stack(synth.STREAM_V, w.kv_heads), stack(synth.STREAM_Q, w.q_heads)
+
+
+def paged_spread_lengths(n: int, batch: int):
+    """Lengths from a quarter to seven quarters of n, about the same total as batch sequences of n."""
+    return [max(1, int(round(n * (0.25 + 1.5 * i / max(1, batch - 1))))) for i in range(batch)]
