@@ -1040,7 +1040,7 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
         RLKV_CUDA(cudaMemcpyAsync(out_host, dout, q_bytes * (c->out_bf16 ? 1 : 2), cudaMemcpyDeviceToHost, s));
         return RLKV_OK;
     }
-    const int chunks = c->layers >= 8 ? 4 : 1;
+    const int chunks = c->layers >= 8 ? 2 : 1;
     if (chunks == 1 || c->layers > kMaxStepLayers) {
         uint8_t* dk = c->dev_base + c->lay.off_k;
         uint8_t* dv = c->dev_base + c->lay.off_v;
@@ -1057,8 +1057,11 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
     // Inputs come in on one side stream, results go out on another, both beside the kernels on the
     // caller's stream.  The input staging area exists twice and calls alternate between the copies,
     // so this call's inputs can be copied in while the kernels of the call before still read theirs.
-    // The layers go in four chunks: a short first one (little to wait for before the first kernel),
-    // a short last one (little to copy out after the last kernel).
+    // The layers go in two chunks, the last eighth apart: little is left to copy out after the last
+    // kernel, and the results of the first chunk leave while the second is computed.  (Every further
+    // chunk costs a launch, about 25 us measured; four chunks -- a short first one for the inputs as
+    // well -- measured 50 us slower per step once consecutive calls overlap, since the inputs of a call
+    // then arrive during the call before anyway.)
     const int p = (int)(c->host_steps++ & 1);
     const size_t in_bytes = c->lay.off_out - c->lay.off_k;          // k, v, q of one copy
     uint8_t* dk = c->dev_base + c->lay.off_k + (p ? c->lay.off_in2 - c->lay.off_k : 0);
@@ -1067,8 +1070,8 @@ int rlkv_step_host(rlkv_cache* c, const void* k_host, const void* v_host, const 
     uint8_t* dout = c->dev_base + c->lay.off_out;
     (void)in_bytes;
     const size_t q_layer = q_bytes / c->layers;
-    const int L = c->layers, head = L / 16 > 0 ? L / 16 : 1, tail = L / 8 > 0 ? L / 8 : 1;
-    const int bounds[5] = {0, head, head + (L - head - tail) / 2, L - tail, L};
+    const int L = c->layers, tail = L / 8 > 0 ? L / 8 : 1;
+    const int bounds[3] = {0, L - tail, L};
     // inputs: this copy of the staging area was last read by the kernels of the call before last
     RLKV_CUDA(cudaStreamWaitEvent(c->in_stream, c->ev_step[p], 0));
     RLKV_CUDA(cudaMemcpyAsync(dk, k_host, kv_bytes, cudaMemcpyHostToDevice, c->in_stream));
