@@ -27,7 +27,7 @@ head classes come from a seeded global selection (see synth/).
 
 --loop runs only the long decode loop (on --workload cot); --sweep prints one JSON line per cell of
 the compression x context x batch grid instead of the bench line, and --sweep-table FILE turns such
-lines into the markdown table of the benchmark spec.
+lines into a markdown table.
 
 With N > 1 (torchrun) every rank runs the same workload on its own GPU: the path shards by batch
 rows / replicas with no exchange step, so there is no collective on the data path (weak scaling).
