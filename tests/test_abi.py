@@ -141,3 +141,23 @@ def test_paged_fp8_size_is_half_the_pool(binding):
     with pytest.raises(binding.RlkvError) as e:
         binding.rlkv_paged_size_fp8(**{**ok, "head_dim": 64})
     assert e.value.code == binding.RLKV_EINVAL
+
+
+def test_fp8_cache_size_needs_no_device(binding):
+    """rlkv_cache_size_fp8: host arithmetic only.  The cache is the paged 8-bit cache with one slot per
+    batch row and batch * ceil(max_len / 64) pages plus a staging area for one step's k, v, q and
+    results; a longer cache grows by 16 KB per full head, batch row and 64 tokens."""
+    ok = dict(layers=2, kv_heads=2, q_heads=8, head_dim=128, batch=3, max_len=1000, head_is_full=[1, 0, 1, 1], sink=4, window=60)
+    base = binding.rlkv_cache_size_fp8(**ok)
+    pages = 3 * ((1000 + 63) // 64)
+    paged = binding.rlkv_paged_size_fp8(2, 2, 8, 128, 3, pages, 1000, [1, 0, 1, 1], 4, 60)
+    staging = 2 * 2 * 3 * 2 * 128 * 2 + 2 * 3 * 8 * 128 * 2 + 2 * 3 * 8 * 128 * 4    # k, v; q; results in fp32
+    assert paged <= base - staging < paged + 1024 + 4 * 256                          # alignment only
+    longer = binding.rlkv_cache_size_fp8(**{**ok, "max_len": 1000 + 64 * 10})
+    grown = longer - base
+    codes = 3 * 10 * 3 * 2 * 64 * 128                     # 3 full heads, 10 more pages per batch row, 16 KB a page
+    assert codes <= grown < codes + (1 << 16)             # the rest: page tables and partial records
+    for bad in (dict(head_dim=64), dict(batch=0), dict(max_len=0), dict(q_heads=7), dict(window=0)):
+        with pytest.raises(binding.RlkvError) as e:
+            binding.rlkv_cache_size_fp8(**{**ok, **bad})
+        assert e.value.code == binding.RLKV_EINVAL
