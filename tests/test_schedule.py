@@ -112,8 +112,9 @@ def test_whole_step_schedule(rl, U, tf, Uc, tc, ctas, item):
         part = sizes[:ctas]
         assert part.max() - part.min() <= 1
         x0 = int(starts[ctas])
-        assert x0 % tf == 0 and x0 // tf <= (2 * U) // 3 + 1       # whole units, at most two thirds of them
-        assert T - x0 >= 4 * ctas * small - tf                     # enough left for every CTA to claim a few items
+        assert x0 % tf == 0 and x0 // tf <= U                      # whole units
+        assert T - x0 >= 6 * ctas * small - tf                     # enough left for every CTA to claim a few items
+        assert T - x0 < 6 * ctas * small + tf + Uc * tc            # and no more than that
         rest = sizes[ctas:]
         assert (rest[:-1] == small).all() and 1 <= rest[-1] <= small
     else:
