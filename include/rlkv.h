@@ -387,7 +387,9 @@ int rlkv_debug_trace(rlkv_cache* cache, int enable, unsigned long long* words_ho
  * shrink geometrically down to item_tiles; *n_slots_out is the number of partial-result records a
  * launch of this shape may write.  whole_step != 0: the schedule rlkv_step uses for one launch over
  * all layers instead (most full units whole, unit after unit, in one equal item per CTA; the rest and
- * the compressed units unit after unit in items of item_tiles tiles, fewer where the step is small).  Optional outputs (host; `cap` = ints available in starts_out
+ * the compressed units unit after unit in items of item_tiles tiles, fewer where the step is small;
+ * whole_step == 2: the form rlkv_paged_step uses for sequences of unequal lengths, whose whole units
+ * are handed out one by one instead of in one equal item per CTA).  Optional outputs (host; `cap` = ints available in starts_out
  * and 4-int records available in tile_map_out): starts_out[k] = first flat tile of item k, then
  * the total; tile_map_out[4x..4x+3] = unit, tile inside the unit, consecutive tiles of the unit
  * from x on, partial record of the segment holding flat tile x.  RLKV_EKERNEL if the schedule's

@@ -1204,7 +1204,7 @@ int rlkv_debug_schedule(int full_units, int tiles_full, int comp_units, int tile
         ctas < 1 || item_tiles < 1 || !n_items_out || !n_slots_out)
         return RLKV_EINVAL;
     if ((long long)full_units * tiles_full + (long long)comp_units * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
-    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, true, -1, whole_step == 2)
                                    : make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
     *n_items_out = sc.n_items;
     *n_slots_out = sc.n_slots;
@@ -1242,7 +1242,7 @@ int rlkv_debug_claim_order(int full_units, int tiles_full, int comp_units, int t
         ctas < 1 || item_tiles < 1 || !order_out)
         return RLKV_EINVAL;
     if ((long long)full_units * tiles_full + (long long)comp_units * tiles_comp >= (1ll << 31)) return RLKV_EINVAL;
-    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles)
+    const Schedule sc = whole_step ? step_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles, true, -1, whole_step == 2)
                                    : make_schedule(full_units, tiles_full, comp_units, tiles_comp, ctas, item_tiles);
     if (cap < sc.n_items) return RLKV_ENOMEM;
     for (int k = 0; k < sc.n_items; ++k) order_out[k] = claim_to_item(sc, k);

@@ -93,10 +93,11 @@ constexpr int kDefaultItemTiles = 32;  // largest "smallest work item" of launch
 // every CTA about six items to claim, so that CTAs on a slower path to memory end together with the
 // others (measured: CTAs differ by about 1 % in the tiles they get through; with a third of the units
 // left to claim, as at first, the step was 1 % slower -- every claimed unit is cut into 4-5 pieces).
-// `prefix` false: no whole-unit prefix, every item is claimed (a paged batch of unequal lengths: equal
-// tile ranges would hold unequal numbers of tiles that exist).
+// `prefix` false: no whole-unit prefix, every item is claimed.  `unit_items`: the prefix is claimed unit
+// by unit (a paged batch of unequal lengths: equal tile ranges would hold unequal numbers of tiles that
+// exist, whole units can still be streamed in one piece).
 inline Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_most, bool prefix = true,
-                              long long real_tiles = -1)
+                              long long real_tiles = -1, bool unit_items = false)
 {
     // (paged cache: `real_tiles` of the tiles exist, and they decide the item size)
     const long long all_tiles = real_tiles >= 0 ? real_tiles : (long long)U * tf + (long long)Uc * tc;
@@ -105,12 +106,14 @@ inline Schedule step_schedule(int U, int tf, int Uc, int tc, int grid, int item_
     if (item_tiles < kMinItemTiles) item_tiles = kMinItemTiles;
     int U0 = 0;
     if (U > 0 && prefix) {
-        const long long rest_wanted = 6ll * grid * item_tiles;  // tiles left to the claimed items
+        long long rest_wanted = 6ll * grid * item_tiles;  // tiles left to the claimed items
+        const long long flat_tiles = (long long)U * tf + (long long)Uc * tc;
+        if (real_tiles > 0 && real_tiles < flat_tiles) rest_wanted = rest_wanted * flat_tiles / real_tiles;  // ... that exist
         long long most = U - (rest_wanted - (long long)Uc * tc + tf - 1) / tf;
         if (most > U) most = U;
         U0 = most > 0 ? (int)most : 0;
     }
-    return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0);
+    return make_schedule(U, tf, Uc, tc, grid, item_tiles, U0, 0, unit_items);
 }
 
 }  // namespace rlkv

@@ -76,6 +76,9 @@ __host__ __device__ constexpr int partial_floats(int head_dim, int group) {
 // items (items 0 .. P-1, one per CTA), so most units are streamed in one piece by one CTA and only
 // the units an item boundary falls into are split.  The remaining U - U0 units follow in bands as
 // above (`rounds` = 0: in one band, i.e. unit after unit, cut into items of min_sz tiles).
+// `unit_items`: the prefix is handed out unit by unit instead (one item per unit, CTA c starts with
+// unit c and the others are claimed): for units of unequal real length (a paged batch of sequences of
+// different lengths), where P equal tile ranges would not be P equal amounts of work.
 struct Schedule {
     int P;                      // CTAs
     int R;                      // bands handed out in P equal items (the factoring rounds)
@@ -95,7 +98,8 @@ struct Schedule {
     int irem[kMaxRounds];
 };
 
-inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz, int U0 = 0, int rounds = kMaxRounds)
+inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz, int U0 = 0, int rounds = kMaxRounds,
+                              bool unit_items = false)
 {
     Schedule s{};
     s.P = P;
@@ -108,10 +112,11 @@ inline Schedule make_schedule(int U, int tf, int Uc, int tc, int P, int min_sz, 
     if (U0 < 0 || (long long)U0 * s.tf < P) U0 = 0;  // every prefix item holds at least one tile
     s.U0 = U0;
     s.x0 = U0 * s.tf;
-    s.k0 = U0 > 0 ? P : 0;
-    s.s0 = U0 > 0 ? P + U0 : 0;
-    s.pq = U0 > 0 ? s.x0 / P : 0;
-    s.prem = U0 > 0 ? s.x0 % P : 0;
+    if (unit_items && U0 < P) U0 = s.U0 = s.x0 = 0;          // every CTA starts with a unit of its own
+    s.k0 = U0 > 0 ? (unit_items ? U0 : P) : 0;
+    s.s0 = U0 > 0 ? s.k0 + U0 : 0;
+    s.pq = U0 > 0 ? (unit_items ? s.tf : s.x0 / P) : 0;
+    s.prem = U0 > 0 && !unit_items ? s.x0 % P : 0;
     const int Ub = U - U0;  // full units laid out in bands
     int r = 0;
     s.base[0] = s.x0;

@@ -575,8 +575,8 @@ static int paged_decode(rlkv_paged* p, int layer, const int* slots, int n, const
     if (whole_step) {
         if ((long long)n * heads_full * tiles_full + (long long)n * heads_comp * tiles_comp >= (1ll << 31)) return RLKV_ESCRATCH;
         const int most = kDefaultItemTiles * (p->fp8 ? 2 : 1);
-        // equal lengths: most full units whole in one static item per CTA; else every item is claimed
-        a.sched = step_schedule(n * heads_full, tiles_full, n * heads_comp, tiles_comp, grid, most, equal_lengths, real_tiles);
+        // equal lengths: most full units whole in one static item per CTA; else the same units, claimed one by one
+        a.sched = step_schedule(n * heads_full, tiles_full, n * heads_comp, tiles_comp, grid, most, true, real_tiles, !equal_lengths);
         if (a.sched.n_slots > p->step_slots) return RLKV_ESCRATCH;
         if (grid > a.sched.n_items) grid = a.sched.n_items;
         a.n_full = a.n_comp = 0;

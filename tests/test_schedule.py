@@ -136,6 +136,47 @@ def test_whole_step_schedule(rl, U, tf, Uc, tc, ctas, item):
         assert (per_unit[:n_prefix] == 1).sum() >= n_prefix - 2 * ctas
 
 
+@pytest.mark.parametrize("U,tf,Uc,tc,ctas,item", STEP_SHAPES)
+def test_whole_step_schedule_with_units_as_items(rl, U, tf, Uc, tc, ctas, item):
+    """The whole-step schedule of a paged batch of unequal lengths: the prefix is handed out unit by unit
+    (item u = unit u, whole), the rest as in the other form.  Every tile exactly once, one partial record
+    per segment, none shared; the hand-out order still starts CTA c with item c."""
+    starts, n_slots, tmap = rl.rlkv_debug_schedule(U, tf, Uc, tc, ctas, item, tile_map=True, whole_step=2)
+    T = U * tf + Uc * tc
+    assert starts[0] == 0 and starts[-1] == T
+    sizes = np.diff(starts)
+    assert (sizes >= 1).all()
+    n_items = sizes.size
+    uid, tile, run, slot = tmap[:, 0], tmap[:, 1], tmap[:, 2], tmap[:, 3]
+    want = [(u, t) for u in range(U) for t in range(tf)] + [(U + u, t) for u in range(Uc) for t in range(tc)]
+    assert list(zip(uid.tolist(), tile.tolist())) == want
+    small = min(item, max(2, T // ctas))
+    n_prefix = 0
+    while n_prefix < n_items and n_prefix < U and sizes[n_prefix] == tf and starts[n_prefix] == n_prefix * tf and tf > small:
+        n_prefix += 1
+    if n_prefix:
+        assert n_prefix >= ctas                                    # every CTA starts with a unit of its own
+        assert T - n_prefix * tf >= 6 * ctas * small - tf          # enough left for every CTA to claim a few items
+        rest = sizes[n_prefix:]
+        assert (rest[:-1] == small).all() and 1 <= rest[-1] <= small
+    item_of = np.repeat(np.arange(n_items), sizes)
+    new_seg = np.ones(T, bool)
+    new_seg[1:] = (item_of[1:] != item_of[:-1]) | (uid[1:] != uid[:-1])
+    seg_id = np.cumsum(new_seg) - 1
+    seg_slot = {}
+    for x in range(T):
+        seg_slot.setdefault(int(seg_id[x]), set()).add(int(slot[x]))
+    assert all(len(v) == 1 for v in seg_slot.values())
+    slots = [next(iter(v)) for v in seg_slot.values()]
+    assert len(set(slots)) == len(slots) and max(slots) < n_slots
+    per_unit = np.bincount(uid[new_seg], minlength=U + Uc)
+    assert (per_unit[:n_prefix] == 1).all()                        # a unit of the prefix is never cut
+    order = rl.rlkv_debug_claim_order(U, tf, Uc, tc, ctas, item, n_items, whole_step=2)
+    assert sorted(order.tolist()) == list(range(n_items))
+    static = min(ctas, n_items)
+    assert order[:static].tolist() == list(range(static))
+
+
 @pytest.mark.parametrize("whole_step", [False, True])
 @pytest.mark.parametrize("U,tf,Uc,tc,ctas,item", SHAPES[:8] + STEP_SHAPES[:6])
 def test_items_of_compressed_units_are_claimed_first(rl, U, tf, Uc, tc, ctas, item, whole_step):
